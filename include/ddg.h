@@ -1,0 +1,177 @@
+/*
+ * ddg.h — C ABI of the B200 (sm_100a) DDG training-step library.
+ *
+ * The library runs one iteration of decoupled parallel backpropagation with delayed gradients (DDG):
+ * a feed-forward network is cut into K modules of consecutive layers; in iteration t every module k
+ * runs its forward pass on the current minibatch (Section 2, Eq. 3), its backward pass on the sample of
+ * iteration s = t-K+k with the activations and weights it stored then and the error gradient it received
+ * from module k+1 one iteration ago (Section 3.1, Eq. 6-7), and then updates its own weights with that
+ * delayed gradient (Section 3.3, Eq. 8-9, Algorithm 1; Algorithm 2 for Adam).  All K modules run
+ * concurrently as K CUDA streams on one GPU; activation, weight-version and error-gradient history lives
+ * in per-module device ring buffers owned by the context.
+ *
+ * Conventions for every call
+ *   - Pointers are marked "device" or "host".  The caller owns every buffer it passes; the library owns
+ *     everything else and frees it in ddg_destroy.  No torch / C++ types cross this boundary.
+ *   - Every call returns a ddg_status.  Nothing throws.  After DDG_ERR_CUDA or DDG_ERR_TIMEOUT the context
+ *     answers DDG_ERR_STATE until it is destroyed.  ddg_last_error gives a library-owned message.
+ *   - The library needs a CUDA device of compute capability 10.0; there is no CPU fallback.
+ *   - A context is used from one host thread at a time.
+ *
+ * Flat parameter order ("canonical order") used by get/set weights and gradients: layers in network order;
+ * per layer the conv / FC weight ([Cout][Cin][3][3] or [out][in], row-major), then bias, then BN gamma, then
+ * BN beta; a basic block contributes conv1.w, bn1.gamma, bn1.beta, conv2.w, bn2.gamma, bn2.beta.  Always
+ * fp32, whatever the internal storage.
+ */
+#ifndef DDG_H_
+#define DDG_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ddg_ctx ddg_ctx; /* opaque */
+
+typedef enum {
+    DDG_OK = 0,
+    DDG_ERR_INVALID_ARG = 1, /* NULL pointer, wrong size, index out of range */
+    DDG_ERR_BAD_SPEC = 2,    /* layer list / split points do not describe a valid network */
+    DDG_ERR_UNSUPPORTED = 3, /* valid, but not implemented (e.g. conv bias) */
+    DDG_ERR_OOM = 4,         /* device or host allocation failed */
+    DDG_ERR_CUDA = 5,        /* a CUDA call or kernel failed; message in ddg_last_error */
+    DDG_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out (reported at the next sync point) */
+    DDG_ERR_STATE = 7        /* call not allowed in the context's current state */
+} ddg_status;
+
+/* Layer kinds.  The paper only names "ResNet" (Section 5, Table 2); the formulas are the usual ones:
+ *  DDG_FC             y = x W^T + b                     (c_in -> c_out, optional bias, optional ReLU)
+ *  DDG_CONV3X3        3x3 cross-correlation, pad 1, stride 1|2, no bias (optional ReLU)
+ *  DDG_BN             train-mode batch normalisation over (N,H,W), biased variance, eps 1e-5 (optional ReLU)
+ *  DDG_RELU           max(x, 0), derivative 0 at 0
+ *  DDG_BASIC_BLOCK    out = relu(bn2(conv2(relu(bn1(conv1(x))))) + sc(x)); conv1 has the stride;
+ *                     sc = identity, or for stride 2 / wider output x[:, ::2, ::2] zero-padded in channels
+ *  DDG_GLOBAL_AVGPOOL mean over H x W  */
+typedef enum {
+    DDG_FC = 0, DDG_CONV3X3 = 1, DDG_BN = 2, DDG_RELU = 3, DDG_BASIC_BLOCK = 4, DDG_GLOBAL_AVGPOOL = 5
+} ddg_layer_kind;
+
+typedef struct {
+    int kind;       /* ddg_layer_kind */
+    int c_in;       /* input channels / features */
+    int c_out;      /* output channels / features (= c_in for BN, RELU, GLOBAL_AVGPOOL) */
+    int stride;     /* 1 or 2 (conv, block); ignored otherwise */
+    int has_bias;   /* FC only */
+    int relu_after; /* FC, CONV3X3, BN: apply ReLU to the output */
+} ddg_layer;
+
+typedef enum { DDG_OPT_SGD = 0, DDG_OPT_ADAM = 1 } ddg_opt_kind;
+
+/* Optimiser.  SGD: d = g + weight_decay*w; v = momentum*v + d; w -= lr*v (Eq. 9 when momentum = decay = 0).
+ * Adam: Algorithm 2, bias correction with the global iteration count.  A module whose delayed gradient does
+ * not exist yet (t-K+k < 0, Eq. 8) is left untouched in that iteration. */
+typedef struct {
+    int kind; /* ddg_opt_kind */
+    float lr, momentum, weight_decay, beta1, beta2, eps;
+} ddg_opt;
+
+typedef enum { DDG_FP32 = 0, DDG_BF16 = 1 } ddg_precision;
+
+typedef struct {
+    int precision;  /* DDG_FP32: everything fp32.  DDG_BF16: activations, error gradients and the weight
+                       versions the sweeps read are bf16; accumulation, statistics, loss, parameter
+                       gradients, master weights and optimiser state are fp32. */
+    int batch;      /* B */
+    int in_c, in_h, in_w;   /* input is [B][in_c][in_h][in_w] fp32 (use in_h = in_w = 1 for an MLP) */
+    int num_classes;
+    unsigned long long seed; /* seed of the library's own He-normal initialisation */
+    int use_graph;  /* 1: replay the steady-state iteration as CUDA graphs (one per ring phase) */
+    int debug_checks; /* 1: stamp ring slots with the iteration that wrote them and verify on use */
+    void *const *streams; /* host array of K cudaStream_t to run the modules on, or NULL (library creates K) */
+} ddg_cfg;
+
+/* Build a context: validates the network (Section 2: L layers; Section 3: K groups of consecutive layers,
+ * `split_after` = the K-1 strictly increasing 0-based layer indices after which a new module starts; NULL when
+ * K = 1), allocates all device state, initialises the weights from cfg->seed.  host pointers only. */
+ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_after, int K,
+                      const ddg_opt *opt, const ddg_cfg *cfg, ddg_ctx **out);
+
+/* One DDG iteration (Algorithm 1 / 2 with the sweeps of Eq. 3 and Eq. 6-7).
+ *   x_dev: device, fp32, [B][in_c][in_h][in_w]; y_dev: device, int32 labels [B].
+ *   loss_host: host, nullable.  Non-NULL: the call waits for the iteration and writes the mean cross-entropy
+ *   of this iteration's forward pass.  NULL: the call only enqueues work; x_dev / y_dev must stay valid until
+ *   ddg_sync (or a later call with loss_host != NULL) returns. */
+ddg_status ddg_step(ddg_ctx *ctx, const float *x_dev, const int *y_dev, float *loss_host);
+
+/* The same iteration with host inputs: copies x_host / y_host (host, same shapes) to the device on the
+ * context's first stream, runs ddg_step and, when loss_host is non-NULL, waits and returns the loss. */
+ddg_status ddg_step_host(ddg_ctx *ctx, const float *x_host, const int *y_host, float *loss_host);
+
+/* The stepsize sequence {gamma_t} of Algorithm 1 is driven by the caller. */
+ddg_status ddg_set_lr(ddg_ctx *ctx, float lr);
+
+/* n: total parameter count; per_module: host array of K counts (nullable). */
+ddg_status ddg_param_count(const ddg_ctx *ctx, size_t *n, size_t *per_module);
+
+/* Copy the fp32 master weights out / in, canonical order, n = total parameter count.  dst/src is a device
+ * pointer when *_on_device != 0, else host.  Both calls wait for all enqueued work first.  ddg_set_weights is
+ * only allowed before the first step (afterwards: DDG_ERR_STATE). */
+ddg_status ddg_get_weights(ddg_ctx *ctx, float *dst, size_t n, int dst_on_device);
+ddg_status ddg_set_weights(ddg_ctx *ctx, const float *src, size_t n, int src_on_device);
+
+/* The delayed gradient g_k^t (Eq. 8) that module k (0-based) applied in the last iteration, canonical order
+ * of that module's slice, n = per_module[k].  *sample (nullable) receives s = t-K+k (1-based k), or -1 with a
+ * zero-filled dst while the module is in warm-up. */
+ddg_status ddg_get_grads(ddg_ctx *ctx, int k, float *dst, size_t n, int dst_on_device, long *sample);
+
+/* Device address of the last iteration's loss (fp32 scalar), for consumers that stay on the device. */
+ddg_status ddg_get_loss_dev(ddg_ctx *ctx, const float **loss_dev);
+
+/* Number of the library's kernel launches the last ddg_step issued (graph replays count their kernel nodes). */
+ddg_status ddg_last_step_launches(const ddg_ctx *ctx, long *launches);
+
+/* Wait for all K streams; surfaces deferred device-side errors. */
+ddg_status ddg_sync(ddg_ctx *ctx);
+
+const char *ddg_last_error(const ddg_ctx *ctx); /* ctx may be NULL: error of the last failed ddg_create */
+void ddg_destroy(ddg_ctx *ctx);
+
+/* ---------------------------------------------------------------------------------------------------------
+ * Single-kernel entry points, for per-kernel parity tests and roofline measurements.  All pointers are device
+ * pointers; tensors are NHWC ([B][H][W][C]) in the precision given (fp32 or bf16 elements); weights are in
+ * canonical [Cout][Cin][3][3] order in the same element type; parameter gradients and statistics are fp32.
+ * `stream` is a cudaStream_t (NULL = default stream).  The calls only enqueue.
+ * --------------------------------------------------------------------------------------------------------- */
+
+/* y = conv3x3(x, w), pad 1 (layer forward, Eq. 3).  x [B][H][W][Cin], y [B][Ho][Wo][Cout], Ho = (H-1)/stride+1. */
+ddg_status ddg_conv3x3_fwd(int precision, const void *x, const void *w, void *y, int B, int H, int W, int Cin,
+                           int Cout, int stride, void *stream);
+/* dx = conv3x3 input gradient (Eq. 5 / Eq. 7).  dy [B][Ho][Wo][Cout], dx [B][H][W][Cin]. */
+ddg_status ddg_conv3x3_dgrad(int precision, const void *dy, const void *w, void *dx, int B, int H, int W, int Cin,
+                             int Cout, int stride, void *stream);
+/* dw = conv3x3 weight gradient (Eq. 4 / Eq. 6), fp32 [Cout][Cin][3][3].  scratch: device, fp32,
+ * ddg_conv3x3_wgrad_scratch_elems(...) elements, contents undefined on entry and exit. */
+size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride);
+ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float *dw, float *scratch, int B, int H,
+                             int W, int Cin, int Cout, int stride, void *stream);
+/* Batch-norm forward, fused: statistics over (B,H,W), then y = [relu](gamma*xhat + beta [+ res]).  res nullable
+ * (same shape as y).  gamma/beta in the activation element type; mean/invstd fp32 [C] outputs; scratch fp32,
+ * ddg_bn_scratch_elems(C) elements. */
+size_t ddg_bn_scratch_elems(int C);
+ddg_status ddg_bn_fwd(int precision, const void *x, const void *gamma, const void *beta, const void *res, void *y,
+                      float *mean, float *invstd, float *scratch, int B, int HW, int C, int relu, void *stream);
+/* Batch-norm backward: dz = dout * [out > 0] when relu != 0 (out = forward output), else dout;
+ * dgamma = sum dz*xhat, dbeta = sum dz, dx = gamma*invstd*(dz - dbeta/n - xhat*dgamma/n). */
+ddg_status ddg_bn_bwd(int precision, const void *dout, const void *out, const void *x, const void *gamma,
+                      const float *mean, const float *invstd, void *dx, float *dgamma, float *dbeta, float *scratch,
+                      int B, int HW, int C, int relu, void *stream);
+/* Fused SGD update over n parameters (Eq. 9 with momentum and weight decay): d = g + wd*w; v = mu*v + d;
+ * w -= lr*v; w_version = cast(w).  w, v, g fp32; w_version in the precision's element type. */
+ddg_status ddg_sgd_update(int precision, float *w, float *v, const float *g, void *w_version, size_t n, float lr,
+                          float momentum, float weight_decay, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DDG_H_ */

@@ -27,9 +27,12 @@
  *     switches to the literal "gradient = 0" update, which still decays and moves momentum).
  *   - the backward sweep of module k differentiates at the stored weights w^s (flag
  *     ORC_USE_CURRENT_WEIGHTS switches to the current weights, the other possible reading).
- *   - flag ORC_ROUND_BF16 rounds stored activations, error gradients and the weights that the sweeps
- *     read to bfloat16 (round to nearest even), to separate format error from mistakes when the CUDA
- *     path runs with bfloat16 storage.
+ *   - flags ORC_ROUND_BF16 / ORC_ROUND_FP32 imitate a storage format: every tensor a sweep stores
+ *     (activations, error gradients) and the weights the sweeps read are rounded to bfloat16 or to
+ *     float (round to nearest even); batch statistics, logits, loss, parameter gradients, master
+ *     weights and optimiser state are rounded to float in both.  All arithmetic between two stores
+ *     stays fp64.  This separates format error from mistakes, and it makes the ReLU decisions of a
+ *     path that stores the same formats agree with the oracle's.
  *
  * Parity pins (tests/test_oracle_*.py): finite differences, closed forms for softmax-CE and batch
  * norm, brute-force convolution, K=1 == plain backprop, delayed gradient == true gradient at the
@@ -49,7 +52,7 @@
 
 enum { ORC_FC = 0, ORC_CONV3X3 = 1, ORC_BN = 2, ORC_RELU = 3, ORC_BASIC_BLOCK = 4, ORC_GLOBAL_AVGPOOL = 5 };
 enum { ORC_SGD = 0, ORC_ADAM = 1 };
-enum { ORC_USE_CURRENT_WEIGHTS = 1, ORC_WARMUP_DECAY = 2, ORC_ROUND_BF16 = 4 };
+enum { ORC_USE_CURRENT_WEIGHTS = 1, ORC_WARMUP_DECAY = 2, ORC_ROUND_BF16 = 4, ORC_ROUND_FP32 = 8 };
 
 typedef struct { int kind, c_in, c_out, stride, has_bias, relu_after; } orc_layer;
 
@@ -238,6 +241,34 @@ void orc_bn_backward(int B, int C, int HW, const double *x, const double *mean, 
     }
 }
 
+/* the normalisation alone, from given statistics (used when the statistics were rounded for storage) */
+void orc_bn_apply(int B, int C, int HW, const double *x, const double *gamma, const double *beta, const double *mean,
+                  const double *invstd, double *y) {
+    for (int c = 0; c < C; ++c)
+        for (int n = 0; n < B; ++n) {
+            const double *xp = x + ((size_t)n * C + c) * HW;
+            double *yp = y + ((size_t)n * C + c) * HW;
+            for (int i = 0; i < HW; ++i) yp[i] = gamma[c] * (xp[i] - mean[c]) * invstd[c] + beta[c];
+        }
+}
+
+/* the input gradient alone, from given (possibly storage-rounded) dgamma / dbeta */
+void orc_bn_backward_apply(int B, int C, int HW, const double *x, const double *mean, const double *invstd,
+                           const double *gamma, const double *dy, const double *dgamma, const double *dbeta,
+                           double *dx) {
+    const double cnt = (double)B * HW;
+    for (int c = 0; c < C; ++c)
+        for (int n = 0; n < B; ++n) {
+            const double *xp = x + ((size_t)n * C + c) * HW;
+            const double *dp = dy + ((size_t)n * C + c) * HW;
+            double *dxp = dx + ((size_t)n * C + c) * HW;
+            for (int i = 0; i < HW; ++i) {
+                const double xh = (xp[i] - mean[c]) * invstd[c];
+                dxp[i] = gamma[c] * invstd[c] * (dp[i] - dbeta[c] / cnt - xh * dgamma[c] / cnt);
+            }
+        }
+}
+
 void orc_relu_forward(size_t n, const double *x, double *y) {
     for (size_t i = 0; i < n; ++i) y[i] = x[i] > 0.0 ? x[i] : 0.0;
 }
@@ -359,13 +390,43 @@ typedef struct {
     hist_t **hist;          /* hist[k][slot] */
     int **labels_hist;      /* labels of the in-flight iterations */
     long *labels_s;
+    /* ReLU decisions that floating point cannot settle: see orc_set_tie_policy */
+    double tie_tau;
+    long tie_up, tie_count;
 } orc_ctx;
 
 static size_t tsize(const orc_ctx *c, int C, int H, int W) { return (size_t)c->B * C * H * W; }
 
+/* storage rounding of activations, error gradients and sweep weights */
 static void maybe_round(const orc_ctx *c, double *p, size_t n) {
-    if (!(c->flags & ORC_ROUND_BF16)) return;
-    for (size_t i = 0; i < n; ++i) p[i] = bf16_round(p[i]);
+    if (c->flags & ORC_ROUND_BF16) for (size_t i = 0; i < n; ++i) p[i] = bf16_round(p[i]);
+    else if (c->flags & ORC_ROUND_FP32) for (size_t i = 0; i < n; ++i) p[i] = (double)(float)p[i];
+}
+
+/* storage rounding of what is kept in float in both formats */
+static void maybe_round32(const orc_ctx *c, double *p, size_t n) {
+    if (c->flags & (ORC_ROUND_BF16 | ORC_ROUND_FP32)) for (size_t i = 0; i < n; ++i) p[i] = (double)(float)p[i];
+}
+
+/* batch norm forward with the statistics passing through storage */
+static void bn_forward_stored(const orc_ctx *c, int B, int C, int HW, const double *x, const double *gamma,
+                              const double *beta, double *y, double *mean, double *invstd) {
+    orc_bn_forward(B, C, HW, x, gamma, beta, y, mean, invstd);
+    if (c->flags & (ORC_ROUND_BF16 | ORC_ROUND_FP32)) {
+        maybe_round32(c, mean, C); maybe_round32(c, invstd, C);
+        orc_bn_apply(B, C, HW, x, gamma, beta, mean, invstd, y);
+    }
+}
+
+/* batch norm backward with dgamma / dbeta passing through storage */
+static void bn_backward_stored(const orc_ctx *c, int B, int C, int HW, const double *x, const double *mean,
+                               const double *invstd, const double *gamma, const double *dy, double *dx,
+                               double *dgamma, double *dbeta) {
+    orc_bn_backward(B, C, HW, x, mean, invstd, gamma, dy, dx, dgamma, dbeta);
+    if (c->flags & (ORC_ROUND_BF16 | ORC_ROUND_FP32)) {
+        maybe_round32(c, dgamma, C); maybe_round32(c, dbeta, C);
+        orc_bn_backward_apply(B, C, HW, x, mean, invstd, gamma, dy, dgamma, dbeta, dx);
+    }
 }
 
 static void free_cache(cache_t *q) {
@@ -380,9 +441,26 @@ static double *dup(const double *src, size_t n) {
     return p;
 }
 
+/* y = relu(pre) at one ReLU site of the network.  A pre-activation closer to zero than tie_tau is a decision
+ * that two correct floating-point evaluations may take differently (relu'(0) jumps).  With tie_tau > 0 such
+ * elements are numbered in traversal order and forced: "off" (output 0, derivative 0) by default, "on" (output a
+ * positive value far below any rounding, derivative 1) for element number tie_up, or for all when tie_up == -2.
+ * The forward values move by less than tie_tau either way. */
+static void relu_site(orc_ctx *c, size_t n, const double *pre, double *y) {
+    for (size_t i = 0; i < n; ++i) {
+        const double p = pre[i];
+        if (c->tie_tau > 0.0 && fabs(p) < c->tie_tau) {
+            const long idx = c->tie_count++;
+            y[i] = (c->tie_up == -2 || idx == c->tie_up) ? 1e-30 : 0.0;
+        } else {
+            y[i] = p > 0.0 ? p : 0.0;
+        }
+    }
+}
+
 /* forward sweep of one layer (Eq. 3).  `w` points at the layer's own parameter slice.  Returns the
  * freshly allocated output; fills `q` with what the backward sweep needs. */
-static double *layer_forward(const orc_ctx *c, const layer_t *L, const double *w, const double *x, cache_t *q) {
+static double *layer_forward(orc_ctx *c, const layer_t *L, const double *w, const double *x, cache_t *q) {
     const int B = c->B;
     const size_t n_in = tsize(c, L->C_in, L->H_in, L->W_in), n_out = tsize(c, L->C_out, L->H_out, L->W_out);
     const int is_last = (L == &c->layers[c->n_layers - 1]);
@@ -391,22 +469,23 @@ static double *layer_forward(const orc_ctx *c, const layer_t *L, const double *w
     switch (L->spec.kind) {
     case ORC_FC:
         orc_fc_forward(B, L->C_in, L->C_out, x, w, L->spec.has_bias ? w + (size_t)L->C_in * L->C_out : NULL, y);
-        if (L->spec.relu_after) orc_relu_forward(n_out, y, y);
-        if (!is_last) maybe_round(c, y, n_out); /* the network output (logits) stays unrounded */
+        if (L->spec.relu_after) relu_site(c, n_out, y, y);
+        if (!is_last) maybe_round(c, y, n_out);
+        else maybe_round32(c, y, n_out); /* the network output (logits) is kept in float */
         break;
     case ORC_CONV3X3:
         orc_conv3x3_forward(B, L->C_in, L->H_in, L->W_in, L->C_out, L->spec.stride, x, w, y);
-        if (L->spec.relu_after) orc_relu_forward(n_out, y, y);
+        if (L->spec.relu_after) relu_site(c, n_out, y, y);
         maybe_round(c, y, n_out);
         break;
     case ORC_BN:
         q->m1 = dalloc(L->C_in); q->is1 = dalloc(L->C_in);
-        orc_bn_forward(B, L->C_in, L->H_in * L->W_in, x, w, w + L->C_in, y, q->m1, q->is1);
-        if (L->spec.relu_after) orc_relu_forward(n_out, y, y);
+        bn_forward_stored(c, B, L->C_in, L->H_in * L->W_in, x, w, w + L->C_in, y, q->m1, q->is1);
+        if (L->spec.relu_after) relu_site(c, n_out, y, y);
         maybe_round(c, y, n_out);
         break;
     case ORC_RELU:
-        orc_relu_forward(n_out, x, y);
+        relu_site(c, n_out, x, y);
         break;
     case ORC_GLOBAL_AVGPOOL:
         orc_avgpool_forward(B, L->C_in, L->H_in * L->W_in, x, y);
@@ -421,16 +500,16 @@ static double *layer_forward(const orc_ctx *c, const layer_t *L, const double *w
         q->m1 = dalloc(Co); q->is1 = dalloc(Co); q->m2 = dalloc(Co); q->is2 = dalloc(Co);
         orc_conv3x3_forward(B, Ci, L->H_in, L->W_in, Co, st, x, w1, q->y1);
         maybe_round(c, q->y1, n_out);
-        orc_bn_forward(B, Co, HWo, q->y1, g1, b1, q->a1, q->m1, q->is1);
-        orc_relu_forward(n_out, q->a1, q->a1);
+        bn_forward_stored(c, B, Co, HWo, q->y1, g1, b1, q->a1, q->m1, q->is1);
+        relu_site(c, n_out, q->a1, q->a1);
         maybe_round(c, q->a1, n_out);
         orc_conv3x3_forward(B, Co, L->H_out, L->W_out, Co, 1, q->a1, w2, q->y2);
         maybe_round(c, q->y2, n_out);
         double *z = dalloc(n_out), *sc = dalloc(n_out);
-        orc_bn_forward(B, Co, HWo, q->y2, g2, b2, z, q->m2, q->is2);
+        bn_forward_stored(c, B, Co, HWo, q->y2, g2, b2, z, q->m2, q->is2);
         orc_shortcut_forward(B, Ci, L->H_in, L->W_in, Co, st, x, sc);
         for (size_t i = 0; i < n_out; ++i) z[i] += sc[i];
-        orc_relu_forward(n_out, z, y);
+        relu_site(c, n_out, z, y);
         maybe_round(c, y, n_out);
         free(z); free(sc);
         break;
@@ -462,7 +541,7 @@ static double *layer_backward(const orc_ctx *c, const layer_t *L, const double *
         break;
     case ORC_BN:
         if (L->spec.relu_after) orc_relu_backward(n_out, q->y, dy, dy);
-        orc_bn_backward(B, L->C_in, L->H_in * L->W_in, q->x, q->m1, q->is1, w, dy, dx, gw, gw + L->C_in);
+        bn_backward_stored(c, B, L->C_in, L->H_in * L->W_in, q->x, q->m1, q->is1, w, dy, dx, gw, gw + L->C_in);
         break;
     case ORC_RELU:
         orc_relu_backward(n_out, q->y, dy, dx);
@@ -479,12 +558,12 @@ static double *layer_backward(const orc_ctx *c, const layer_t *L, const double *
         double *dz = dalloc(n_out), *dy2 = dalloc(n_out), *da1 = dalloc(n_out), *dy1 = dalloc(n_out);
         double *dsc = dalloc(n_in);
         orc_relu_backward(n_out, q->y, dy, dz);               /* through the final relu */
-        orc_bn_backward(B, Co, HWo, q->y2, q->m2, q->is2, g2, dz, dy2, gg2, gb2);
+        bn_backward_stored(c, B, Co, HWo, q->y2, q->m2, q->is2, g2, dz, dy2, gg2, gb2);
         maybe_round(c, dy2, n_out);
         orc_conv3x3_backward(B, Co, L->H_out, L->W_out, Co, 1, q->a1, w2, dy2, da1, gw2);
         maybe_round(c, da1, n_out);
         orc_relu_backward(n_out, q->a1, da1, da1);
-        orc_bn_backward(B, Co, HWo, q->y1, q->m1, q->is1, g1, da1, dy1, gg1, gb1);
+        bn_backward_stored(c, B, Co, HWo, q->y1, q->m1, q->is1, g1, da1, dy1, gg1, gb1);
         maybe_round(c, dy1, n_out);
         orc_conv3x3_backward(B, Ci, L->H_in, L->W_in, Co, st, q->x, w1, dy1, dx, gw1);
         orc_shortcut_backward(B, Ci, L->H_in, L->W_in, Co, st, dz, dsc);
@@ -495,6 +574,7 @@ static double *layer_backward(const orc_ctx *c, const layer_t *L, const double *
     default: abort();
     }
     if (!is_first) maybe_round(c, dx, n_in);
+    maybe_round32(c, gw, L->p_cnt); /* parameter gradients are kept in float */
     free(dy);
     return dx;
 }
@@ -606,6 +686,11 @@ void orc_get_weights(const orc_ctx *c, double *w) { memcpy(w, c->w, c->P * sizeo
 void orc_set_lr(orc_ctx *c, double lr) { c->lr = lr; }
 long orc_iteration(const orc_ctx *c) { return c->t; }
 
+/* Near-zero ReLU decisions (see relu_site): tau = 0 switches the mechanism off (default).  up_index = -1 forces
+ * all of them off, -2 all on, i >= 0 only the i-th on.  orc_tie_count = how many the last forward sweep met. */
+void orc_set_tie_policy(orc_ctx *c, double tau, long up_index) { c->tie_tau = tau; c->tie_up = up_index; }
+long orc_tie_count(const orc_ctx *c) { return c->tie_count; }
+
 /* last applied delayed gradient of module k (0-based).  Returns the sample index s it belongs to, or -1
  * when the module was still in warm-up at the last step (Eq. 8: gradient is zero, dst is zero-filled). */
 int orc_get_grads(const orc_ctx *c, int k, double *dst) {
@@ -623,6 +708,7 @@ static double *sweep_weights(const orc_ctx *c, const double *w, size_t n) {
 
 /* loss of the whole net at the current weights, no state change (for finite-difference pins) */
 double orc_loss_only(orc_ctx *c, const double *x, const int *y) {
+    c->tie_count = 0;
     double *h = dup(x, tsize(c, c->in_c, c->in_h, c->in_w));
     maybe_round(c, h, tsize(c, c->in_c, c->in_h, c->in_w));
     for (int l = 0; l < c->n_layers; ++l) {
@@ -634,6 +720,7 @@ double orc_loss_only(orc_ctx *c, const double *x, const int *y) {
     }
     double loss;
     orc_softmax_ce(c->B, c->num_classes, h, y, &loss, NULL);
+    maybe_round32(c, &loss, 1);
     free(h);
     return loss;
 }
@@ -647,6 +734,7 @@ double orc_step(orc_ctx *c, const double *x, const int *y) {
     c->labels_s[slot_t] = t;
 
     /* 1. forward sweep through modules 1..K with the current weights w^t (Eq. 3); keep h^t and w^t */
+    c->tie_count = 0;
     double *h = dup(x, tsize(c, c->in_c, c->in_h, c->in_w));
     maybe_round(c, h, tsize(c, c->in_c, c->in_h, c->in_w));
     for (int k = 0; k < K; ++k) {
@@ -668,6 +756,8 @@ double orc_step(orc_ctx *c, const double *x, const int *y) {
         hist_t *rec = &c->hist[K - 1][slot_t];
         rec->delta = dalloc((size_t)c->B * c->num_classes);
         orc_softmax_ce(c->B, c->num_classes, h, y, &loss, rec->delta);
+        maybe_round32(c, rec->delta, (size_t)c->B * c->num_classes);
+        maybe_round32(c, &loss, 1);
         rec->has_delta = 1;
     }
     free(h);
@@ -719,6 +809,7 @@ double orc_step(orc_ctx *c, const double *x, const int *y) {
                 c->v[i] = c->mu * c->v[i] + d;
                 c->w[i] -= c->lr * c->v[i];
             }
+            maybe_round32(c, c->v + o, n); maybe_round32(c, c->w + o, n);
         } else { /* Algorithm 2: bias correction with the global count t+1 */
             const double c1 = 1.0 - pow(c->b1, (double)(t + 1)), c2 = 1.0 - pow(c->b2, (double)(t + 1));
             for (size_t i = o; i < o + n; ++i) {
@@ -727,6 +818,7 @@ double orc_step(orc_ctx *c, const double *x, const int *y) {
                 c->m2nd[i] = c->b2 * c->m2nd[i] + (1.0 - c->b2) * gi * gi;
                 c->w[i] -= c->lr * (c->v[i] / c1) / (sqrt(c->m2nd[i] / c2) + c->eps);
             }
+            maybe_round32(c, c->v + o, n); maybe_round32(c, c->m2nd + o, n); maybe_round32(c, c->w + o, n);
         }
     }
     c->t = t + 1;

@@ -1,0 +1,108 @@
+// Single-kernel C-ABI entry points (per-kernel parity tests and roofline measurements).
+#include "../../include/ddg.h"
+#include "common.cuh"
+#include "conv_tc.h"
+#include "kernels.h"
+
+using namespace ddg;
+
+namespace {
+bool bad_prec(int p) { return p != DDG_FP32 && p != DDG_BF16; }
+ddg_status init_once() {
+    static int rc = -1;
+    if (rc < 0) { rc = conv_direct_init(); if (rc == 0) rc = conv_tc_init(); }
+    return rc == 0 ? DDG_OK : DDG_ERR_CUDA;
+}
+ddg_status done() { return cudaGetLastError() == cudaSuccess ? DDG_OK : DDG_ERR_CUDA; }
+bool conv_shape_ok(int B, int H, int W, int Cin, int Cout, int stride) {
+    return B >= 1 && H >= 1 && W >= 1 && Cin >= 1 && Cout >= 1 && (stride == 1 || stride == 2) && Cin <= 256 &&
+           Cout <= 256 && (size_t)Cin * Cout <= 4096;
+}
+}  // namespace
+
+extern "C" {
+
+ddg_status ddg_conv3x3_fwd(int precision, const void *x, const void *w, void *y, int B, int H, int W, int Cin,
+                           int Cout, int stride, void *stream) {
+    if (bad_prec(precision) || !x || !w || !y) return DDG_ERR_INVALID_ARG;
+    if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (precision == DDG_BF16 && conv_tc_supported(B, H, W, Cin, Cout, stride))
+        launch_conv_tc(0, x, w, y, B, H, W, Cin, Shortcut{}, s);
+    else
+        launch_conv_fwd_direct(precision, x, w, y, B, H, W, Cin, Cout, stride, 0, s);
+    return done();
+}
+
+ddg_status ddg_conv3x3_dgrad(int precision, const void *dy, const void *w, void *dx, int B, int H, int W, int Cin,
+                             int Cout, int stride, void *stream) {
+    if (bad_prec(precision) || !dy || !w || !dx) return DDG_ERR_INVALID_ARG;
+    if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (precision == DDG_BF16 && conv_tc_supported(B, H, W, Cin, Cout, stride))
+        launch_conv_tc(1, dy, w, dx, B, H, W, Cin, Shortcut{}, s);
+    else
+        launch_conv_dgrad_direct(precision, dy, w, dx, B, H, W, Cin, Cout, stride, Shortcut{}, s);
+    return done();
+}
+
+size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride) {
+    if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return 0;
+    size_t a = conv_wgrad_scratch_elems(B, H, W, Cin, Cout, stride), b = wgrad_tc_scratch_elems();
+    return a > b ? a : b;
+}
+
+ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float *dw, float *scratch, int B, int H,
+                             int W, int Cin, int Cout, int stride, void *stream) {
+    if (bad_prec(precision) || !x || !dy || !dw || !scratch) return DDG_ERR_INVALID_ARG;
+    if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (precision == DDG_BF16 && wgrad_tc_supported(B, H, W, Cin, Cout, stride))
+        launch_wgrad_tc(x, dy, dw, scratch, B, H, W, Cin, s);
+    else
+        launch_conv_wgrad_direct(precision, x, dy, dw, scratch, B, H, W, Cin, Cout, stride, s);
+    return done();
+}
+
+size_t ddg_bn_scratch_elems(int C) { return C >= 1 && C <= 256 ? bn_scratch_elems(C) : 0; }
+
+ddg_status ddg_bn_fwd(int precision, const void *x, const void *gamma, const void *beta, const void *res, void *y,
+                      float *mean, float *invstd, float *scratch, int B, int HW, int C, int relu, void *stream) {
+    if (bad_prec(precision) || !x || !gamma || !beta || !y || !mean || !invstd || !scratch) return DDG_ERR_INVALID_ARG;
+    if (B < 1 || HW < 1 || C < 1 || C > 256) return DDG_ERR_UNSUPPORTED;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;  // the CTA ticket counter
+    launch_bn_stats(precision, x, mean, invstd, scratch, (long)B * HW, C, s);
+    Shortcut sc{};
+    if (res) { sc.mode = 1; sc.a = res; }
+    launch_bn_apply(precision, x, gamma, beta, mean, invstd, sc, y, B, HW, 1, C, relu, s);
+    return done();
+}
+
+ddg_status ddg_bn_bwd(int precision, const void *dout, const void *out, const void *x, const void *gamma,
+                      const float *mean, const float *invstd, void *dx, float *dgamma, float *dbeta, float *scratch,
+                      int B, int HW, int C, int relu, void *stream) {
+    if (bad_prec(precision) || !dout || !x || !gamma || !mean || !invstd || !dx || !dgamma || !dbeta || !scratch ||
+        (relu && !out))
+        return DDG_ERR_INVALID_ARG;
+    if (B < 1 || HW < 1 || C < 1 || C > 256) return DDG_ERR_UNSUPPORTED;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;
+    launch_bn_bwd_reduce(precision, dout, out, x, mean, invstd, dgamma, dbeta, scratch, (long)B * HW, C, relu, s);
+    launch_bn_bwd_apply(precision, dout, out, x, gamma, mean, invstd, dgamma, dbeta, dx, (long)B * HW, C, relu, s);
+    return done();
+}
+
+ddg_status ddg_sgd_update(int precision, float *w, float *v, const float *g, void *w_version, size_t n, float lr,
+                          float momentum, float weight_decay, void *stream) {
+    if (bad_prec(precision) || !w || !v || !g || !w_version) return DDG_ERR_INVALID_ARG;
+    UpdateArgs a{};
+    a.mode = 0; a.lr = lr; a.mu = momentum; a.wd = weight_decay;
+    launch_update(precision, w, v, nullptr, g, w_version, n, a, (cudaStream_t)stream);
+    return done();
+}
+
+}  // extern "C"

@@ -1,0 +1,27 @@
+// Tensor-core (tcgen05 / TMEM / TMA) 3x3 convolution path for bf16 NHWC tensors on sm_100a.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "kernels.h"
+
+namespace ddg {
+
+// Shapes the tensor-core kernels take: stride 1, Cin == Cout in {16, 32, 64}, 128-pixel tiles that cover whole
+// image rows (W in {8, 16, 32}, and B*H*W a multiple of 128).
+bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
+// dir 0: dst = conv3x3(src, w) (forward).  dir 1: dst = input gradient of conv3x3 given src = dy; with
+// sc.mode == 1 the identity-shortcut gradient sc.a * [sc.b > 0] is added before the store.
+int launch_conv_tc(int dir, const void *src, const void *w, void *dst, int B, int H, int W, int C, Shortcut sc,
+                   cudaStream_t s);
+
+bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
+size_t wgrad_tc_scratch_elems();
+int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C,
+                    cudaStream_t s);
+
+// One-time per-process set-up (function attributes, driver entry points).  Returns a cudaError_t value.
+int conv_tc_init();
+int conv_direct_init();
+
+}  // namespace ddg

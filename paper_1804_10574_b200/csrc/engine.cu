@@ -1,0 +1,759 @@
+// Host side of the DDG library: network planning, per-module ring buffers, the K-stream schedule of one DDG
+// iteration (Algorithm 1 with the sweeps of Eq. 3 and Eq. 6-7), CUDA-graph replay, and the C ABI.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <memory>
+#include <string>
+#include <vector>
+
+#include "../../include/ddg.h"
+#include "common.cuh"
+#include "conv_tc.h"
+#include "kernels.h"
+
+using namespace ddg;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+struct TensorRef {
+    int module;   // arena that holds the tensor (-1: none)
+    size_t off;   // byte offset inside one arena slot
+};
+
+struct LayerPlan {
+    ddg_layer spec;
+    int Cin, Hin, Win, Cout, Hout, Wout;
+    int module;
+    size_t p_off;  // element offset of the layer's parameters inside its module's parameter slice
+    size_t p_cnt;
+    TensorRef in, out;            // layer input (may live in the previous module's arena) and output
+    TensorRef y1, a1, y2, stats;  // basic block intermediates; stats = fp32 [4][C] (mean1,invstd1,mean2,invstd2)
+    bool is_first, is_last;
+};
+
+struct Module {
+    int first, last;            // layer range
+    int R;                      // ring length K-k+1 (k 1-based): activation slots and weight versions
+    size_t P;                   // parameter count
+    size_t p_off_global;        // offset of the slice in the canonical flat vector
+    size_t arena_bytes;         // one activation slot
+    char *arena = nullptr;      // R slots
+    float *w = nullptr, *v = nullptr, *m2 = nullptr, *g = nullptr;
+    char *wver = nullptr;       // R weight versions in the compute precision
+    char *tmp[3] = {nullptr, nullptr, nullptr};  // error-gradient temporaries of the backward sweep
+    size_t tmp_bytes = 0;
+    float *bn_scratch = nullptr, *wg_scratch = nullptr;
+    char *delta_out[2] = {nullptr, nullptr};  // error gradient w.r.t. this module's input, double buffered
+    size_t delta_bytes = 0;
+    long last_sample = -1;
+    cudaStream_t stream = nullptr;
+    bool own_stream = false;
+    cudaEvent_t ev_fwd = nullptr, ev_bwd = nullptr, ev_join = nullptr;
+};
+
+}  // namespace
+
+struct ddg_ctx {
+    int K = 0, n_layers = 0, prec = 0, B = 0, in_c = 0, in_h = 0, in_w = 0, classes = 0;
+    ddg_opt opt{};
+    ddg_cfg cfg{};
+    std::vector<LayerPlan> layers;
+    std::vector<Module> mods;
+    size_t P = 0;
+    long t = 0;
+    int period = 1;
+    float *x_stage = nullptr;  // K staged copies of the input batch (fp32 NCHW) and labels
+    int *y_stage = nullptr;
+    size_t x_elems = 0;
+    float *dlogits = nullptr, *loss_dev = nullptr;
+    float *pinned_loss = nullptr;
+    cudaEvent_t ev_fork = nullptr;
+    std::vector<cudaGraphExec_t> graphs;
+    std::vector<long> graph_launches;
+    long launches = 0;
+    bool broken = false;
+    std::string err;
+};
+
+namespace {
+
+void set_err(ddg_ctx *c, const char *fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    if (c) c->err = buf;
+    g_create_error = buf;
+}
+
+#define CU(call)                                                                                     \
+    do {                                                                                             \
+        cudaError_t e_ = (call);                                                                     \
+        if (e_ != cudaSuccess) {                                                                     \
+            set_err(ctx, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), __FILE__, __LINE__); \
+            if (ctx) ctx->broken = true;                                                             \
+            return e_ == cudaErrorMemoryAllocation ? DDG_ERR_OOM : DDG_ERR_CUDA;                     \
+        }                                                                                            \
+    } while (0)
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t layer_params(const ddg_layer &s) {
+    switch (s.kind) {
+    case DDG_FC: return (size_t)s.c_in * s.c_out + (s.has_bias ? s.c_out : 0);
+    case DDG_CONV3X3: return (size_t)s.c_in * s.c_out * 9;
+    case DDG_BN: return 2 * (size_t)s.c_in;
+    case DDG_BASIC_BLOCK: return (size_t)s.c_in * s.c_out * 9 + (size_t)s.c_out * s.c_out * 9 + 4 * (size_t)s.c_out;
+    default: return 0;
+    }
+}
+
+int gcd_i(int a, int b) { return b ? gcd_i(b, a % b) : a; }
+
+char *slot_ptr(ddg_ctx *c, TensorRef r, long iter) {
+    Module &m = c->mods[r.module];
+    return m.arena + (size_t)(iter % m.R) * m.arena_bytes + r.off;
+}
+
+// ---- convolution dispatch: tensor-core path where it applies, CUDA cores otherwise --------------------
+int conv_fwd(ddg_ctx *c, const void *x, const void *w, void *y, int H, int W, int Cin, int Cout, int stride, int relu,
+             cudaStream_t s) {
+    if (c->prec == P_BF16 && !relu && conv_tc_supported(c->B, H, W, Cin, Cout, stride))
+        return launch_conv_tc(0, x, w, y, c->B, H, W, Cin, Shortcut{}, s);
+    return launch_conv_fwd_direct(c->prec, x, w, y, c->B, H, W, Cin, Cout, stride, relu, s);
+}
+int conv_dgrad(ddg_ctx *c, const void *dy, const void *w, void *dx, int H, int W, int Cin, int Cout, int stride,
+               Shortcut sc, cudaStream_t s) {
+    if (c->prec == P_BF16 && sc.mode != 2 && conv_tc_supported(c->B, H, W, Cin, Cout, stride))
+        return launch_conv_tc(1, dy, w, dx, c->B, H, W, Cin, sc, s);
+    return launch_conv_dgrad_direct(c->prec, dy, w, dx, c->B, H, W, Cin, Cout, stride, sc, s);
+}
+int conv_wgrad(ddg_ctx *c, Module &m, const void *x, const void *dy, float *dw, int H, int W, int Cin, int Cout,
+               int stride, cudaStream_t s) {
+    if (c->prec == P_BF16 && wgrad_tc_supported(c->B, H, W, Cin, Cout, stride))
+        return launch_wgrad_tc(x, dy, dw, m.wg_scratch, c->B, H, W, Cin, s);
+    return launch_conv_wgrad_direct(c->prec, x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cout, stride, s);
+}
+
+// ---- forward sweep of module k on the minibatch of iteration t (Eq. 3) --------------------------------
+long forward_module(ddg_ctx *c, int k, long t) {
+    Module &m = c->mods[k];
+    cudaStream_t s = m.stream;
+    const size_t es = elem_size(c->prec);
+    const char *wv = m.wver + (size_t)(t % m.R) * m.P * es;
+    long n = 0;
+    for (int l = m.first; l <= m.last; ++l) {
+        LayerPlan &L = c->layers[l];
+        const char *w = wv + L.p_off * es;
+        const void *in;
+        if (L.is_first) {  // layout shim: staged NCHW fp32 -> NHWC in the compute precision, kept in the arena
+            char *xin = slot_ptr(c, L.in, t);
+            n += launch_shim(c->prec, c->x_stage + (size_t)(t % c->K) * c->x_elems, xin, c->B, c->in_c, c->in_h,
+                             c->in_w, s);
+            in = xin;
+        } else {
+            in = slot_ptr(c, L.in, t);
+        }
+        char *out = slot_ptr(c, L.out, t);
+        const int B = c->B;
+        switch (L.spec.kind) {
+        case DDG_FC:
+            n += launch_fc_fwd(c->prec, in, w, L.spec.has_bias ? w + (size_t)L.Cin * L.Cout * es : nullptr, out, B,
+                               L.Cin, L.Cout, L.spec.relu_after, L.is_last, s);
+            break;
+        case DDG_CONV3X3:
+            n += conv_fwd(c, in, w, out, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, L.spec.relu_after, s);
+            break;
+        case DDG_BN: {
+            float *st = (float *)slot_ptr(c, L.stats, t);
+            n += launch_bn_stats(c->prec, in, st, st + L.Cin, m.bn_scratch, (long)B * L.Hin * L.Win, L.Cin, s);
+            n += launch_bn_apply(c->prec, in, w, w + (size_t)L.Cin * es, st, st + L.Cin, Shortcut{}, out, B, L.Hin,
+                                 L.Win, L.Cin, L.spec.relu_after, s);
+            break;
+        }
+        case DDG_RELU:
+            n += launch_relu_fwd(c->prec, in, out, (size_t)B * L.Cin * L.Hin * L.Win, s);
+            break;
+        case DDG_GLOBAL_AVGPOOL:
+            n += launch_avgpool_fwd(c->prec, in, out, B, L.Hin * L.Win, L.Cin, s);
+            break;
+        case DDG_BASIC_BLOCK: {
+            const int Ci = L.Cin, Co = L.Cout, st = L.spec.stride;
+            const char *w1 = w, *g1 = w1 + (size_t)Co * Ci * 9 * es, *b1 = g1 + (size_t)Co * es;
+            const char *w2 = b1 + (size_t)Co * es, *g2 = w2 + (size_t)Co * Co * 9 * es, *b2 = g2 + (size_t)Co * es;
+            char *y1 = slot_ptr(c, L.y1, t), *a1 = slot_ptr(c, L.a1, t), *y2 = slot_ptr(c, L.y2, t);
+            float *stt = (float *)slot_ptr(c, L.stats, t);
+            const long npix = (long)B * L.Hout * L.Wout;
+            n += conv_fwd(c, in, w1, y1, L.Hin, L.Win, Ci, Co, st, 0, s);
+            n += launch_bn_stats(c->prec, y1, stt, stt + Co, m.bn_scratch, npix, Co, s);
+            n += launch_bn_apply(c->prec, y1, g1, b1, stt, stt + Co, Shortcut{}, a1, B, L.Hout, L.Wout, Co, 1, s);
+            n += conv_fwd(c, a1, w2, y2, L.Hout, L.Wout, Co, Co, 1, 0, s);
+            n += launch_bn_stats(c->prec, y2, stt + 2 * Co, stt + 3 * Co, m.bn_scratch, npix, Co, s);
+            Shortcut sc{};
+            sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
+            sc.a = in; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win;
+            n += launch_bn_apply(c->prec, y2, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out, B, L.Hout, L.Wout, Co, 1, s);
+            break;
+        }
+        }
+    }
+    if (k == c->K - 1) {  // loss f and the up-to-date error gradient of the last module
+        LayerPlan &L = c->layers[m.last];
+        n += launch_softmax_ce(c->prec, (const float *)slot_ptr(c, L.out, t), c->y_stage + (size_t)(t % c->K) * c->B,
+                               c->loss_dev, c->dlogits, c->B, c->classes, s);
+    }
+    return n;
+}
+
+// ---- backward sweep of module k at iteration t on the stored sample sidx = t-K+k (Eq. 6-7) ------------
+long backward_module(ddg_ctx *c, int k, long t, long sidx) {
+    Module &m = c->mods[k];
+    cudaStream_t s = m.stream;
+    const size_t es = elem_size(c->prec);
+    const char *wv = m.wver + (size_t)(sidx % m.R) * m.P * es;  // the weights w^s of the stored iteration
+    long n = 0;
+    const int B = c->B;
+    const char *cur = (k == c->K - 1) ? (const char *)c->dlogits : c->mods[k + 1].delta_out[(t + 1) % 2];
+    int cur_tmp = -1;
+    auto pick = [&](int e1, int e2) { for (int i = 0; i < 3; ++i) if (i != e1 && i != e2) return i; return 0; };
+    for (int l = m.last; l >= m.first; --l) {
+        LayerPlan &L = c->layers[l];
+        const char *w = wv + L.p_off * es;
+        float *gw = m.g + L.p_off;
+        const char *in = slot_ptr(c, L.in, sidx);
+        const char *out = slot_ptr(c, L.out, sidx);
+        const bool mod_first = (l == m.first);
+        const bool need_dx = !L.is_first;
+        // destination of the error gradient w.r.t. the layer input
+        int dst_tmp = -1;
+        char *dst = nullptr;
+        if (need_dx) {
+            if (mod_first) dst = m.delta_out[t % 2];
+            else { dst_tmp = pick(cur_tmp, -1); dst = m.tmp[dst_tmp]; }
+        }
+        switch (L.spec.kind) {
+        case DDG_FC:
+            n += launch_fc_bwd(c->prec, in, w, out, cur, dst, gw, L.spec.has_bias ? gw + (size_t)L.Cin * L.Cout : nullptr,
+                               B, L.Cin, L.Cout, L.spec.relu_after, L.is_last, s);
+            break;
+        case DDG_CONV3X3: {
+            const char *dy = cur;
+            if (L.spec.relu_after) {
+                int tm = pick(cur_tmp, dst_tmp);
+                n += launch_relu_bwd(c->prec, out, cur, m.tmp[tm], (size_t)B * L.Cout * L.Hout * L.Wout, s);
+                dy = m.tmp[tm];
+            }
+            if (need_dx)
+                n += conv_dgrad(c, dy, w, dst, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, Shortcut{}, s);
+            n += conv_wgrad(c, m, in, dy, gw, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, s);
+            break;
+        }
+        case DDG_BN: {
+            const float *st = (const float *)slot_ptr(c, L.stats, sidx);
+            const long npix = (long)B * L.Hin * L.Win;
+            n += launch_bn_bwd_reduce(c->prec, cur, out, in, st, st + L.Cin, gw, gw + L.Cin, m.bn_scratch, npix, L.Cin,
+                                      L.spec.relu_after, s);
+            char *d = dst ? dst : m.tmp[pick(cur_tmp, -1)];
+            n += launch_bn_bwd_apply(c->prec, cur, out, in, w, st, st + L.Cin, gw, gw + L.Cin, d, npix, L.Cin,
+                                     L.spec.relu_after, s);
+            break;
+        }
+        case DDG_RELU:
+            if (need_dx) n += launch_relu_bwd(c->prec, out, cur, dst, (size_t)B * L.Cin * L.Hin * L.Win, s);
+            break;
+        case DDG_GLOBAL_AVGPOOL:
+            if (need_dx) n += launch_avgpool_bwd(c->prec, cur, dst, B, L.Hin * L.Win, L.Cin, s);
+            break;
+        case DDG_BASIC_BLOCK: {
+            const int Ci = L.Cin, Co = L.Cout, st = L.spec.stride;
+            const size_t nw1 = (size_t)Co * Ci * 9, nw2 = (size_t)Co * Co * 9;
+            const char *w1 = w, *g1 = w1 + nw1 * es, *w2 = g1 + 2 * (size_t)Co * es, *g2 = w2 + nw2 * es;
+            float *gw1 = gw, *gg1 = gw1 + nw1, *gb1 = gg1 + Co, *gw2 = gb1 + Co, *gg2 = gw2 + nw2, *gb2 = gg2 + Co;
+            const char *y1 = slot_ptr(c, L.y1, sidx), *a1 = slot_ptr(c, L.a1, sidx), *y2 = slot_ptr(c, L.y2, sidx);
+            const float *stt = (const float *)slot_ptr(c, L.stats, sidx);
+            const long npix = (long)B * L.Hout * L.Wout;
+            // the two scratch temporaries are the ones not holding the incoming error gradient
+            const int tA = pick(cur_tmp, -1), tB = pick(cur_tmp, tA);
+            char *dy2 = m.tmp[tA], *da1 = m.tmp[tB], *dy1 = m.tmp[tA];
+            n += launch_bn_bwd_reduce(c->prec, cur, out, y2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, m.bn_scratch, npix, Co,
+                                      1, s);
+            n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s);
+            n += conv_dgrad(c, dy2, w2, da1, L.Hout, L.Wout, Co, Co, 1, Shortcut{}, s);
+            n += conv_wgrad(c, m, a1, dy2, gw2, L.Hout, L.Wout, Co, Co, 1, s);
+            n += launch_bn_bwd_reduce(c->prec, da1, a1, y1, stt, stt + Co, gg1, gb1, m.bn_scratch, npix, Co, 1, s);
+            n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
+            if (need_dx) {
+                Shortcut sc{};
+                sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
+                sc.a = cur; sc.b = out; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win;
+                char *dx = mod_first ? dst : da1;  // da1 is dead once bn1's backward has run
+                n += conv_dgrad(c, dy1, w1, dx, L.Hin, L.Win, Ci, Co, st, sc, s);
+                if (!mod_first) { dst = dx; dst_tmp = tB; }
+            }
+            n += conv_wgrad(c, m, in, dy1, gw1, L.Hin, L.Win, Ci, Co, st, s);
+            break;
+        }
+        }
+        cur = dst;
+        cur_tmp = dst_tmp;
+    }
+    return n;
+}
+
+// ---- update of module k with its delayed gradient (Eq. 8-9; Algorithm 1 / 2) --------------------------
+long update_module(ddg_ctx *c, int k, long t, bool have_grad) {
+    Module &m = c->mods[k];
+    UpdateArgs a{};
+    a.lr = c->opt.lr; a.mu = c->opt.momentum; a.wd = c->opt.weight_decay;
+    a.b1 = c->opt.beta1; a.b2 = c->opt.beta2; a.eps = c->opt.eps;
+    if (!have_grad) a.mode = 2;  // Eq. 8: the delayed gradient does not exist yet; leave the module untouched
+    else if (c->opt.kind == DDG_OPT_ADAM) {
+        a.mode = 1;
+        a.c1c = 1.0 - pow((double)a.b1, (double)(t + 1));
+        a.c2c = 1.0 - pow((double)a.b2, (double)(t + 1));
+    } else a.mode = 0;
+    if (a.mode == 2 && m.R == 1) return 0;
+    char *wv = m.wver + (size_t)((t + 1) % m.R) * m.P * elem_size(c->prec);
+    return launch_update(c->prec, m.w, m.v, m.m2, m.g, wv, m.P, a, m.stream);
+}
+
+// Enqueue one whole iteration on the K streams.  `in_capture`: the cross-iteration waits are dropped because
+// successive graph launches are already ordered.
+ddg_status enqueue_iteration(ddg_ctx *ctx, long t, bool in_capture, long *launches) {
+    const int K = ctx->K;
+    long n = 0;
+    // forward sweep, module 1..K in order; module k+1 waits for module k's output
+    for (int k = 0; k < K; ++k) {
+        Module &m = ctx->mods[k];
+        if (k > 0) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k - 1].ev_fwd, 0));
+        n += forward_module(ctx, k, t);
+        if (k < K - 1) CU(cudaEventRecord(m.ev_fwd, m.stream));
+    }
+    // backward sweeps and updates: independent across modules within the iteration ("for k in parallel")
+    for (int k = 0; k < K; ++k) {
+        Module &m = ctx->mods[k];
+        const long sidx = t - K + (k + 1);
+        if (sidx >= 0) {
+            if (k < K - 1 && !in_capture) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k + 1].ev_bwd, 0));
+            n += backward_module(ctx, k, t, sidx);
+            if (k > 0 && !in_capture) CU(cudaEventRecord(m.ev_bwd, m.stream));
+        }
+        n += update_module(ctx, k, t, sidx >= 0);
+        m.last_sample = sidx >= 0 ? sidx : -1;
+    }
+    CU(cudaGetLastError());
+    *launches = n;
+    return DDG_OK;
+}
+
+ddg_status capture_phase(ddg_ctx *ctx, long t, int phase) {
+    const int K = ctx->K;
+    cudaStream_t s0 = ctx->mods[0].stream;
+    CU(cudaStreamBeginCapture(s0, cudaStreamCaptureModeThreadLocal));
+    ddg_status st = DDG_OK;
+    long n = 0;
+    cudaError_t e = cudaEventRecord(ctx->ev_fork, s0);
+    for (int k = 1; k < K && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(ctx->mods[k].stream, ctx->ev_fork, 0);
+    if (e == cudaSuccess) st = enqueue_iteration(ctx, t, true, &n);
+    for (int k = 1; k < K && e == cudaSuccess && st == DDG_OK; ++k) {
+        e = cudaEventRecord(ctx->mods[k].ev_join, ctx->mods[k].stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s0, ctx->mods[k].ev_join, 0);
+    }
+    cudaGraph_t graph = nullptr;
+    cudaError_t e2 = cudaStreamEndCapture(s0, &graph);
+    if (st != DDG_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+    CU(e);
+    CU(e2);
+    cudaGraphExec_t exec = nullptr;
+    cudaError_t e3 = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    CU(e3);
+    ctx->graphs[phase] = exec;
+    ctx->graph_launches[phase] = n;
+    return DDG_OK;
+}
+
+ddg_status init_weights(ddg_ctx *ctx) {
+    for (int l = 0; l < ctx->n_layers; ++l) {
+        LayerPlan &L = ctx->layers[l];
+        Module &m = ctx->mods[L.module];
+        float *w = m.w + L.p_off;
+        cudaStream_t s = m.stream;
+        const unsigned long long seed = ctx->cfg.seed;
+        switch (L.spec.kind) {
+        case DDG_FC:
+            launch_fill_normal(w, (size_t)L.Cin * L.Cout, sqrtf(2.f / L.Cin), seed, 2 * l, s);
+            if (L.spec.has_bias) launch_fill_const(w + (size_t)L.Cin * L.Cout, L.Cout, 0.f, s);
+            break;
+        case DDG_CONV3X3:
+            launch_fill_normal(w, (size_t)L.Cin * L.Cout * 9, sqrtf(2.f / (9 * L.Cin)), seed, 2 * l, s);
+            break;
+        case DDG_BN:
+            launch_fill_const(w, L.Cin, 1.f, s);
+            launch_fill_const(w + L.Cin, L.Cin, 0.f, s);
+            break;
+        case DDG_BASIC_BLOCK: {
+            const size_t nw1 = (size_t)L.Cout * L.Cin * 9, nw2 = (size_t)L.Cout * L.Cout * 9;
+            launch_fill_normal(w, nw1, sqrtf(2.f / (9 * L.Cin)), seed, 2 * l, s);
+            launch_fill_const(w + nw1, L.Cout, 1.f, s);
+            launch_fill_const(w + nw1 + L.Cout, L.Cout, 0.f, s);
+            launch_fill_normal(w + nw1 + 2 * L.Cout, nw2, sqrtf(2.f / (9 * L.Cout)), seed, 2 * l + 1, s);
+            launch_fill_const(w + nw1 + 2 * L.Cout + nw2, L.Cout, 1.f, s);
+            launch_fill_const(w + nw1 + 3 * L.Cout + nw2, L.Cout, 0.f, s);
+            break;
+        }
+        default: break;
+        }
+    }
+    for (auto &m : ctx->mods) launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream);
+    CU(cudaGetLastError());
+    for (auto &m : ctx->mods) CU(cudaStreamSynchronize(m.stream));
+    return DDG_OK;
+}
+
+ddg_status sync_all(ddg_ctx *ctx) {
+    for (auto &m : ctx->mods) CU(cudaStreamSynchronize(m.stream));
+    return DDG_OK;
+}
+
+}  // namespace
+
+// ========================================================================================================
+// C ABI
+// ========================================================================================================
+extern "C" {
+
+const char *ddg_last_error(const ddg_ctx *ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+void ddg_destroy(ddg_ctx *ctx) {
+    if (!ctx) return;
+    for (auto &m : ctx->mods)
+        if (m.stream) cudaStreamSynchronize(m.stream);
+    for (auto g : ctx->graphs)
+        if (g) cudaGraphExecDestroy(g);
+    for (auto &m : ctx->mods) {
+        cudaFree(m.arena); cudaFree(m.w); cudaFree(m.v); cudaFree(m.m2); cudaFree(m.g); cudaFree(m.wver);
+        for (char *p : m.tmp) cudaFree(p);
+        cudaFree(m.bn_scratch); cudaFree(m.wg_scratch);
+        cudaFree(m.delta_out[0]); cudaFree(m.delta_out[1]);
+        if (m.ev_fwd) cudaEventDestroy(m.ev_fwd);
+        if (m.ev_bwd) cudaEventDestroy(m.ev_bwd);
+        if (m.ev_join) cudaEventDestroy(m.ev_join);
+        if (m.own_stream && m.stream) cudaStreamDestroy(m.stream);
+    }
+    cudaFree(ctx->x_stage); cudaFree(ctx->y_stage); cudaFree(ctx->dlogits); cudaFree(ctx->loss_dev);
+    if (ctx->pinned_loss) cudaFreeHost(ctx->pinned_loss);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    delete ctx;
+}
+
+ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_after, int K, const ddg_opt *opt,
+                      const ddg_cfg *cfg, ddg_ctx **out) {
+    ddg_ctx *ctx = nullptr;  // CU() reports into the thread-local create error while this is null
+    if (!layers || !opt || !cfg || !out || n_layers < 1 || K < 1 || (K > 1 && !split_after)) {
+        set_err(nullptr, "ddg_create: NULL argument or non-positive count");
+        return DDG_ERR_INVALID_ARG;
+    }
+    *out = nullptr;
+    if (K > n_layers || K > 8) { set_err(nullptr, "ddg_create: K=%d out of range (1..min(8, layers))", K); return DDG_ERR_BAD_SPEC; }
+    if (cfg->batch < 1 || cfg->in_c < 1 || cfg->in_h < 1 || cfg->in_w < 1 || cfg->num_classes < 1 ||
+        (cfg->precision != DDG_FP32 && cfg->precision != DDG_BF16)) {
+        set_err(nullptr, "ddg_create: bad configuration");
+        return DDG_ERR_INVALID_ARG;
+    }
+    if (opt->kind != DDG_OPT_SGD && opt->kind != DDG_OPT_ADAM) { set_err(nullptr, "ddg_create: unknown optimiser"); return DDG_ERR_INVALID_ARG; }
+    for (int k = 0; k + 1 < K; ++k)
+        if (split_after[k] < 0 || split_after[k] >= n_layers - 1 || (k > 0 && split_after[k] <= split_after[k - 1])) {
+            set_err(nullptr, "ddg_create: split points must be strictly increasing layer indices in [0, n_layers-2]");
+            return DDG_ERR_BAD_SPEC;
+        }
+    int dev_count = 0;
+    if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count == 0) {
+        set_err(nullptr, "ddg_create: no CUDA device; this library has no CPU path");
+        return DDG_ERR_CUDA;
+    }
+    int dev = 0, major = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (major != 10) { set_err(nullptr, "ddg_create: needs a compute-capability 10.x device (found %d.x)", major); return DDG_ERR_UNSUPPORTED; }
+
+    {
+        cudaError_t ie = (cudaError_t)conv_direct_init();
+        if (ie == cudaSuccess) ie = (cudaError_t)conv_tc_init();
+        if (ie != cudaSuccess) { set_err(nullptr, "kernel set-up failed: %s", cudaGetErrorString(ie)); return DDG_ERR_CUDA; }
+    }
+    std::unique_ptr<ddg_ctx, void (*)(ddg_ctx *)> holder(new ddg_ctx, ddg_destroy);
+    ddg_ctx *c = holder.get();
+    c->K = K; c->n_layers = n_layers; c->prec = cfg->precision == DDG_BF16 ? P_BF16 : P_F32;
+    c->B = cfg->batch; c->in_c = cfg->in_c; c->in_h = cfg->in_h; c->in_w = cfg->in_w; c->classes = cfg->num_classes;
+    c->opt = *opt; c->cfg = *cfg;
+    const size_t es = elem_size(c->prec);
+
+    // ---- shapes and validation (Section 2: a chain of L layers) ----
+    c->layers.resize(n_layers);
+    int C = c->in_c, H = c->in_h, W = c->in_w;
+    for (int l = 0; l < n_layers; ++l) {
+        LayerPlan &L = c->layers[l];
+        L.spec = layers[l];
+        L.Cin = C; L.Hin = H; L.Win = W;
+        L.is_first = (l == 0); L.is_last = (l == n_layers - 1);
+        const ddg_layer &s = layers[l];
+        bool ok = true;
+        switch (s.kind) {
+        case DDG_FC: ok = (H == 1 && W == 1 && s.c_in == C && s.c_out >= 1); C = s.c_out; break;
+        case DDG_CONV3X3:
+            ok = (s.c_in == C && s.c_out >= 1 && (s.stride == 1 || s.stride == 2));
+            if (ok && s.has_bias) { set_err(nullptr, "layer %d: convolution bias is not supported", l); return DDG_ERR_UNSUPPORTED; }
+            C = s.c_out; H = (H - 1) / s.stride + 1; W = (W - 1) / s.stride + 1; break;
+        case DDG_BASIC_BLOCK:
+            ok = (s.c_in == C && s.c_out >= s.c_in && (s.stride == 1 || s.stride == 2) &&
+                  (s.stride == 2 || s.c_out == s.c_in));
+            C = s.c_out; H = (H - 1) / s.stride + 1; W = (W - 1) / s.stride + 1; break;
+        case DDG_BN: ok = (s.c_in == C); break;
+        case DDG_RELU: break;
+        case DDG_GLOBAL_AVGPOOL: H = 1; W = 1; break;
+        default: ok = false;
+        }
+        if (!ok) { set_err(nullptr, "layer %d: specification does not fit its input [%d,%d,%d]", l, L.Cin, L.Hin, L.Win); return DDG_ERR_BAD_SPEC; }
+        if ((s.kind == DDG_CONV3X3 || s.kind == DDG_BASIC_BLOCK || s.kind == DDG_BN || s.kind == DDG_GLOBAL_AVGPOOL) &&
+            (C > 256 || L.Cin > 256 || (size_t)L.Cin * C > 4096)) {
+            set_err(nullptr, "layer %d: channel counts above 64x64 (or 256 for BN / pooling) are not supported", l);
+            return DDG_ERR_UNSUPPORTED;
+        }
+        L.Cout = C; L.Hout = H; L.Wout = W;
+        L.p_cnt = layer_params(s);
+    }
+    if (layers[n_layers - 1].kind != DDG_FC || C != c->classes) {
+        set_err(nullptr, "the last layer must be an FC layer with num_classes outputs");
+        return DDG_ERR_BAD_SPEC;
+    }
+
+    // ---- modules (Section 3: K groups of consecutive layers) and arena layout ----
+    c->mods.resize(K);
+    size_t p_global = 0;
+    for (int k = 0; k < K; ++k) {
+        Module &m = c->mods[k];
+        m.first = k == 0 ? 0 : split_after[k - 1] + 1;
+        m.last = k == K - 1 ? n_layers - 1 : split_after[k];
+        m.R = K - k;  // K-k+1 with 1-based k
+        m.p_off_global = p_global;
+        size_t off = 0, p = 0;
+        auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+        for (int l = m.first; l <= m.last; ++l) {
+            LayerPlan &L = c->layers[l];
+            L.module = k;
+            L.p_off = p;
+            p += L.p_cnt;
+            const size_t n_in = (size_t)c->B * L.Cin * L.Hin * L.Win, n_out = (size_t)c->B * L.Cout * L.Hout * L.Wout;
+            if (l == 0) L.in = {0, take(n_in * es)};                      // the shimmed input lives in module 1's arena
+            else L.in = c->layers[l - 1].out;                             // may point into the previous module's arena
+            L.out = {k, take(L.is_last ? n_out * sizeof(float) : n_out * es)};
+            if (L.spec.kind == DDG_BASIC_BLOCK) {
+                L.y1 = {k, take(n_out * es)}; L.a1 = {k, take(n_out * es)}; L.y2 = {k, take(n_out * es)};
+                L.stats = {k, take(4 * (size_t)L.Cout * sizeof(float))};
+            } else if (L.spec.kind == DDG_BN) {
+                L.stats = {k, take(2 * (size_t)L.Cin * sizeof(float))};
+            }
+            m.tmp_bytes = std::max(m.tmp_bytes, std::max(n_in, n_out) * es);
+        }
+        m.P = p;
+        m.arena_bytes = off;
+        p_global += p;
+    }
+    c->P = p_global;
+    c->period = 2;
+    for (int k = 0; k < K; ++k) c->period = c->period / gcd_i(c->period, c->mods[k].R) * c->mods[k].R;
+    c->graphs.assign(c->period, nullptr);
+    c->graph_launches.assign(c->period, 0);
+
+    // ---- device state ----
+    ctx = c;  // from here on CU() records into the context
+    for (int k = 0; k < K; ++k) {
+        Module &m = c->mods[k];
+        if (cfg->streams) m.stream = (cudaStream_t)cfg->streams[k];
+        else { CU(cudaStreamCreateWithFlags(&m.stream, cudaStreamNonBlocking)); m.own_stream = true; }
+        CU(cudaEventCreateWithFlags(&m.ev_fwd, cudaEventDisableTiming));
+        CU(cudaEventCreateWithFlags(&m.ev_bwd, cudaEventDisableTiming));
+        CU(cudaEventCreateWithFlags(&m.ev_join, cudaEventDisableTiming));
+        const size_t pn = std::max<size_t>(m.P, 1);
+        CU(cudaMalloc(&m.arena, m.arena_bytes * m.R));
+        CU(cudaMemset(m.arena, 0, m.arena_bytes * m.R));
+        CU(cudaMalloc(&m.w, pn * 4)); CU(cudaMalloc(&m.v, pn * 4)); CU(cudaMalloc(&m.g, pn * 4));
+        CU(cudaMemset(m.v, 0, pn * 4)); CU(cudaMemset(m.g, 0, pn * 4)); CU(cudaMemset(m.w, 0, pn * 4));
+        if (opt->kind == DDG_OPT_ADAM) { CU(cudaMalloc(&m.m2, pn * 4)); CU(cudaMemset(m.m2, 0, pn * 4)); }
+        CU(cudaMalloc(&m.wver, pn * es * m.R));
+        CU(cudaMemset(m.wver, 0, pn * es * m.R));
+        for (auto &p : m.tmp) CU(cudaMalloc(&p, m.tmp_bytes));
+        size_t bn_max = 0, wg_max = 0;
+        for (int l = m.first; l <= m.last; ++l) {
+            LayerPlan &L = c->layers[l];
+            if (L.spec.kind == DDG_BN || L.spec.kind == DDG_BASIC_BLOCK) bn_max = std::max(bn_max, bn_scratch_elems(L.Cout));
+            if (L.spec.kind == DDG_CONV3X3)
+                wg_max = std::max(wg_max, conv_wgrad_scratch_elems(c->B, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride));
+            if (L.spec.kind == DDG_BASIC_BLOCK) {
+                wg_max = std::max(wg_max, conv_wgrad_scratch_elems(c->B, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride));
+                wg_max = std::max(wg_max, conv_wgrad_scratch_elems(c->B, L.Hout, L.Wout, L.Cout, L.Cout, 1));
+            }
+        }
+        wg_max = std::max(wg_max, wgrad_tc_scratch_elems());
+        CU(cudaMalloc(&m.bn_scratch, std::max<size_t>(bn_max, 64) * 4));
+        CU(cudaMemset(m.bn_scratch, 0, std::max<size_t>(bn_max, 64) * 4));
+        CU(cudaMalloc(&m.wg_scratch, std::max<size_t>(wg_max, 64) * 4));
+        CU(cudaMemset(m.wg_scratch, 0, std::max<size_t>(wg_max, 64) * 4));
+        if (k > 0) {
+            LayerPlan &L = c->layers[m.first];
+            m.delta_bytes = (size_t)c->B * L.Cin * L.Hin * L.Win * es;
+            for (auto &p : m.delta_out) { CU(cudaMalloc(&p, m.delta_bytes)); CU(cudaMemset(p, 0, m.delta_bytes)); }
+        }
+    }
+    c->x_elems = (size_t)c->B * c->in_c * c->in_h * c->in_w;
+    CU(cudaMalloc(&c->x_stage, c->x_elems * 4 * K));
+    CU(cudaMalloc(&c->y_stage, (size_t)c->B * 4 * K));
+    CU(cudaMalloc(&c->dlogits, (size_t)c->B * c->classes * 4));
+    CU(cudaMalloc(&c->loss_dev, 4));
+    CU(cudaMemset(c->loss_dev, 0, 4));
+    CU(cudaMallocHost(&c->pinned_loss, 4));
+    CU(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+    ddg_status st = init_weights(c);
+    if (st != DDG_OK) { g_create_error = c->err; return st; }
+    *out = holder.release();
+    return DDG_OK;
+}
+
+static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float *loss_host, cudaMemcpyKind kind) {
+    if (!ctx || !x || !y) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    const long t = ctx->t;
+    const int K = ctx->K;
+    cudaStream_t s0 = ctx->mods[0].stream;
+    // stage the batch: the sweeps (and graph replays) read library-owned buffers
+    CU(cudaMemcpyAsync(ctx->x_stage + (size_t)(t % K) * ctx->x_elems, x, ctx->x_elems * 4, kind, s0));
+    CU(cudaMemcpyAsync(ctx->y_stage + (size_t)(t % K) * ctx->B, y, (size_t)ctx->B * 4, kind, s0));
+    const bool steady = t >= K - 1;
+    if (ctx->cfg.use_graph && steady) {
+        const int phase = (int)(t % ctx->period);
+        if (!ctx->graphs[phase]) {
+            // first visit of this ring phase: record the iteration as a graph, then replay it like any other
+            ddg_status st = sync_all(ctx);
+            if (st != DDG_OK) return st;
+            st = capture_phase(ctx, t, phase);
+            if (st != DDG_OK) { ctx->broken = true; return st; }
+        }
+        CU(cudaGraphLaunch(ctx->graphs[phase], s0));
+        ctx->launches = ctx->graph_launches[phase];
+        for (int k = 0; k < K; ++k) ctx->mods[k].last_sample = t - K + (k + 1);
+    } else {
+        ddg_status st = enqueue_iteration(ctx, t, false, &ctx->launches);
+        if (st != DDG_OK) return st;
+    }
+    ctx->t = t + 1;
+    if (loss_host) {
+        if (ctx->cfg.use_graph && steady) {
+            CU(cudaMemcpyAsync(ctx->pinned_loss, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, s0));
+        } else {
+            CU(cudaMemcpyAsync(ctx->pinned_loss, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, ctx->mods[K - 1].stream));
+        }
+        ddg_status st = sync_all(ctx);
+        if (st != DDG_OK) return st;
+        *loss_host = *ctx->pinned_loss;
+    }
+    return DDG_OK;
+}
+
+ddg_status ddg_step(ddg_ctx *ctx, const float *x_dev, const int *y_dev, float *loss_host) {
+    return step_common(ctx, x_dev, y_dev, loss_host, cudaMemcpyDeviceToDevice);
+}
+
+ddg_status ddg_step_host(ddg_ctx *ctx, const float *x_host, const int *y_host, float *loss_host) {
+    return step_common(ctx, x_host, y_host, loss_host, cudaMemcpyHostToDevice);
+}
+
+ddg_status ddg_set_lr(ddg_ctx *ctx, float lr) {
+    if (!ctx) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    if (lr != ctx->opt.lr) {
+        // captured graphs have the step size baked into their update nodes: drop them, they are re-recorded
+        ddg_status st = sync_all(ctx);
+        if (st != DDG_OK) return st;
+        for (auto &g : ctx->graphs) if (g) { cudaGraphExecDestroy(g); g = nullptr; }
+    }
+    ctx->opt.lr = lr;
+    return DDG_OK;
+}
+
+ddg_status ddg_param_count(const ddg_ctx *ctx, size_t *n, size_t *per_module) {
+    if (!ctx || !n) return DDG_ERR_INVALID_ARG;
+    *n = ctx->P;
+    if (per_module) for (int k = 0; k < ctx->K; ++k) per_module[k] = ctx->mods[k].P;
+    return DDG_OK;
+}
+
+ddg_status ddg_get_weights(ddg_ctx *ctx, float *dst, size_t n, int on_device) {
+    if (!ctx || !dst || n != ctx->P) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    ddg_status st = sync_all(ctx);
+    if (st != DDG_OK) return st;
+    for (auto &m : ctx->mods)
+        CU(cudaMemcpy(dst + m.p_off_global, m.w, m.P * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost));
+    return DDG_OK;
+}
+
+ddg_status ddg_set_weights(ddg_ctx *ctx, const float *src, size_t n, int on_device) {
+    if (!ctx || !src || n != ctx->P) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken || ctx->t != 0) { if (ctx) set_err(ctx, "ddg_set_weights is only allowed before the first step"); return DDG_ERR_STATE; }
+    ddg_status st = sync_all(ctx);
+    if (st != DDG_OK) return st;
+    for (auto &m : ctx->mods) {
+        CU(cudaMemcpy(m.w, src + m.p_off_global, m.P * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice));
+        CU(cudaMemset(m.v, 0, m.P * 4));
+        if (m.m2) CU(cudaMemset(m.m2, 0, m.P * 4));
+        launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream);
+    }
+    CU(cudaGetLastError());
+    return sync_all(ctx);
+}
+
+ddg_status ddg_get_grads(ddg_ctx *ctx, int k, float *dst, size_t n, int on_device, long *sample) {
+    if (!ctx || !dst || k < 0 || k >= ctx->K || n != ctx->mods[k].P) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    ddg_status st = sync_all(ctx);
+    if (st != DDG_OK) return st;
+    Module &m = ctx->mods[k];
+    if (sample) *sample = m.last_sample;
+    if (m.last_sample < 0) {
+        if (on_device) CU(cudaMemset(dst, 0, n * 4)); else memset(dst, 0, n * 4);
+        return DDG_OK;
+    }
+    CU(cudaMemcpy(dst, m.g, n * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost));
+    return DDG_OK;
+}
+
+ddg_status ddg_get_loss_dev(ddg_ctx *ctx, const float **loss_dev) {
+    if (!ctx || !loss_dev) return DDG_ERR_INVALID_ARG;
+    *loss_dev = ctx->loss_dev;
+    return DDG_OK;
+}
+
+ddg_status ddg_last_step_launches(const ddg_ctx *ctx, long *launches) {
+    if (!ctx || !launches) return DDG_ERR_INVALID_ARG;
+    *launches = ctx->launches;
+    return DDG_OK;
+}
+
+ddg_status ddg_sync(ddg_ctx *ctx) {
+    if (!ctx) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    ddg_status st = sync_all(ctx);
+    if (st != DDG_OK) return st;
+    CU(cudaGetLastError());
+    return DDG_OK;
+}
+
+}  // extern "C"

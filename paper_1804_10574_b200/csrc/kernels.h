@@ -1,0 +1,81 @@
+// Internal launcher interface between the host engine and the kernels.  Every launcher only enqueues on the
+// given stream and returns the number of kernel launches it issued.  `prec` is 0 (fp32 tensors) or 1 (bf16).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+namespace ddg {
+
+enum { P_F32 = 0, P_BF16 = 1 };
+
+static inline size_t elem_size(int prec) { return prec == P_BF16 ? 2 : 4; }
+
+// Shortcut input of a residual add (forward) or its gradient (backward).
+//   mode 0: none.  mode 1: identity (same shape as the tensor it is added to).
+//   mode 2: parameter-free down-sampling shortcut: spatial stride 2, channels >= c_small are zero.
+struct Shortcut {
+    int mode;
+    const void *a;   // forward: block input x.          backward: error gradient of the block output
+    const void *b;   // forward: unused.                 backward: block output (for the ReLU mask)
+    int c_small;     // channels of the narrower tensor (block input)
+    int h_big, w_big;  // spatial size of the block input (the larger map)
+};
+
+// ---- layout / small layers --------------------------------------------------------------------------
+int launch_shim(int prec, const float *x_nchw, void *out_nhwc, int B, int C, int H, int W, cudaStream_t s);
+int launch_relu_fwd(int prec, const void *x, void *y, size_t n, cudaStream_t s);
+int launch_relu_bwd(int prec, const void *y, const void *dy, void *dx, size_t n, cudaStream_t s);
+int launch_avgpool_fwd(int prec, const void *x, void *y, int B, int HW, int C, cudaStream_t s);
+int launch_avgpool_bwd(int prec, const void *dy, void *dx, int B, int HW, int C, cudaStream_t s);
+
+// FC: x [B][in] (prec), W [out][in] (prec), bias [out] (prec, nullable).  out_f32: y (and dy) are fp32.
+int launch_fc_fwd(int prec, const void *x, const void *W, const void *bias, void *y, int B, int in, int out,
+                  int relu, int out_f32, cudaStream_t s);
+// dx nullable.  y is the forward output (needed when relu).  dW/db fp32.
+int launch_fc_bwd(int prec, const void *x, const void *W, const void *y, const void *dy, void *dx, float *dW,
+                  float *db, int B, int in, int out, int relu, int out_f32, cudaStream_t s);
+
+// loss = mean CE, dlogits = (softmax - onehot)/B; logits/dlogits fp32 [B][C].
+int launch_softmax_ce(int prec, const float *logits, const int *labels, float *loss, float *dlogits, int B, int C,
+                      cudaStream_t s);
+
+// ---- batch norm -------------------------------------------------------------------------------------
+size_t bn_scratch_elems(int C);
+int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *scratch, long npix, int C,
+                    cudaStream_t s);
+// y = [relu](gamma*(x-mean)*invstd + beta + shortcut).  y is [B][H][W][C].
+int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta, const float *mean,
+                    const float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu, cudaStream_t s);
+// sums[0..C) = sum dz, sums[C..2C) = sum dz*xhat with dz = dout*[out>0] (relu) ; also written to dbeta/dgamma.
+int launch_bn_bwd_reduce(int prec, const void *dout, const void *out, const void *x, const float *mean,
+                         const float *invstd, float *dgamma, float *dbeta, float *scratch, long npix, int C, int relu,
+                         cudaStream_t s);
+int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void *x, const void *gamma,
+                        const float *mean, const float *invstd, const float *dgamma, const float *dbeta, void *dx,
+                        long npix, int C, int relu, cudaStream_t s);
+
+// ---- 3x3 convolution, CUDA-core kernels (any shape; used for fp32 and for shapes the tensor-core path skips) --
+int launch_conv_fwd_direct(int prec, const void *x, const void *w, void *y, int B, int H, int W, int Cin, int Cout,
+                           int stride, int relu, cudaStream_t s);
+int launch_conv_dgrad_direct(int prec, const void *dy, const void *w, void *dx, int B, int H, int W, int Cin,
+                             int Cout, int stride, Shortcut sc, cudaStream_t s);
+size_t conv_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride);
+int launch_conv_wgrad_direct(int prec, const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W,
+                             int Cin, int Cout, int stride, cudaStream_t s);
+
+// ---- optimiser --------------------------------------------------------------------------------------
+// mode 0: SGD momentum/decay step.  mode 1: Adam step (c1, c2 = bias corrections).  mode 2: no step, only
+// refresh the weight version.  w/v/m2 fp32 master state, g fp32, wv = version slot in `prec`.
+struct UpdateArgs {
+    int mode;
+    float lr, mu, wd, b1, b2, eps;
+    double c1c, c2c;  // Adam bias corrections 1-beta1^(t+1), 1-beta2^(t+1)
+};
+int launch_update(int prec, float *w, float *v, float *m2, const float *g, void *wv, size_t n, UpdateArgs a,
+                  cudaStream_t s);
+int launch_cast(int prec, const float *src, void *dst, size_t n, cudaStream_t s);
+int launch_fill_normal(float *dst, size_t n, float stddev, unsigned long long seed, unsigned long long stream_id,
+                       cudaStream_t s);
+int launch_fill_const(float *dst, size_t n, float v, cudaStream_t s);
+
+}  // namespace ddg

@@ -1,0 +1,571 @@
+// Memory-bound kernels of the DDG step: layout shim, batch-norm statistics / apply / backward, ReLU, global
+// mean pool, small FC layers, softmax cross-entropy, and the fused delayed-gradient optimiser update.
+// All are coalesced 16-byte-vector kernels with fp32 arithmetic; reductions are two-stage with a fixed
+// summation order (per-CTA partials, last CTA folds them), so results are reproducible run to run.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace ddg {
+
+static constexpr int kThreads = 256;
+static constexpr int kMaxPartials = 592;  // 4 CTAs per SM on 148 SMs
+static constexpr float kBnEps = 1e-5f;
+
+#define DISPATCH_PREC(prec, ...)                       \
+    do {                                               \
+        if ((prec) == P_BF16) { typedef bf16 T; __VA_ARGS__; } \
+        else { typedef float T; __VA_ARGS__; }         \
+    } while (0)
+
+// ------------------------------------------------------------------------------------------------------
+// input shim: NCHW fp32 -> NHWC T
+// ------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void shim_kernel(const float *__restrict__ x, T *__restrict__ out, int B, int C, int HW) {
+    long i = (long)blockIdx.x * blockDim.x + threadIdx.x;  // (n, p)
+    if (i >= (long)B * HW) return;
+    long n = i / HW, p = i % HW;
+    for (int c = 0; c < C; ++c) out[i * C + c] = from_f<T>(x[(n * C + c) * HW + p]);
+}
+
+int launch_shim(int prec, const float *x, void *out, int B, int C, int H, int W, cudaStream_t s) {
+    long n = (long)B * H * W;
+    DISPATCH_PREC(prec, shim_kernel<T><<<ceil_div(n, kThreads), kThreads, 0, s>>>(x, (T *)out, B, C, H * W));
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// ReLU
+// ------------------------------------------------------------------------------------------------------
+template <typename T> __global__ void relu_fwd_kernel(const T *x, T *y, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) { float v = to_f(x[i]); y[i] = from_f<T>(v > 0.f ? v : 0.f); }
+}
+template <typename T> __global__ void relu_bwd_kernel(const T *y, const T *dy, T *dx, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dx[i] = to_f(y[i]) > 0.f ? dy[i] : from_f<T>(0.f);
+}
+int launch_relu_fwd(int prec, const void *x, void *y, size_t n, cudaStream_t s) {
+    DISPATCH_PREC(prec, relu_fwd_kernel<T><<<ceil_div(n, kThreads), kThreads, 0, s>>>((const T *)x, (T *)y, n));
+    return 1;
+}
+int launch_relu_bwd(int prec, const void *y, const void *dy, void *dx, size_t n, cudaStream_t s) {
+    DISPATCH_PREC(prec, relu_bwd_kernel<T><<<ceil_div(n, kThreads), kThreads, 0, s>>>((const T *)y, (const T *)dy,
+                                                                                      (T *)dx, n));
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// global mean pool: x [B][HW][C] -> y [B][C]
+// ------------------------------------------------------------------------------------------------------
+template <typename T> __global__ void avgpool_fwd_kernel(const T *x, T *y, int HW, int C) {
+    typedef typename AccOf<T>::type A;
+    __shared__ A sm[kThreads];
+    const int n = blockIdx.x, lanes = blockDim.x / C;  // host guarantees C <= blockDim
+    const int c = threadIdx.x % C, lane = threadIdx.x / C;
+    A acc = 0;
+    if (lane < lanes)
+        for (int p = lane; p < HW; p += lanes) acc += (A)to_f(x[((size_t)n * HW + p) * C + c]);
+    sm[threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.x < C) {
+        A t = 0;
+        for (int l = 0; l < lanes; ++l) t += sm[l * C + c];
+        y[(size_t)n * C + c] = from_a<T>(t / (A)HW);
+    }
+}
+template <typename T> __global__ void avgpool_bwd_kernel(const T *dy, T *dx, int HW, int C, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    size_t b = i / ((size_t)HW * C);
+    int c = (int)(i % C);
+    typedef typename AccOf<T>::type A;
+    dx[i] = from_a<T>((A)to_f(dy[b * C + c]) / (A)HW);
+}
+int launch_avgpool_fwd(int prec, const void *x, void *y, int B, int HW, int C, cudaStream_t s) {
+    DISPATCH_PREC(prec, avgpool_fwd_kernel<T><<<B, kThreads, 0, s>>>((const T *)x, (T *)y, HW, C));
+    return 1;
+}
+int launch_avgpool_bwd(int prec, const void *dy, void *dx, int B, int HW, int C, cudaStream_t s) {
+    size_t n = (size_t)B * HW * C;
+    DISPATCH_PREC(prec, avgpool_bwd_kernel<T><<<ceil_div(n, kThreads), kThreads, 0, s>>>((const T *)dy, (T *)dx, HW,
+                                                                                        C, n));
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// small FC layers (CUDA cores; the FC layers of these networks are a few MFLOP)
+// ------------------------------------------------------------------------------------------------------
+// one warp per output element y[b][o]
+template <typename T, typename TO>
+__global__ void fc_fwd_kernel(const T *x, const T *W, const T *bias, TO *y, int B, int in, int out, int relu) {
+    long warp = ((long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (warp >= (long)B * out) return;
+    typedef typename AccOf<T>::type A;
+    int b = (int)(warp / out), o = (int)(warp % out);
+    A acc = 0;
+    for (int i = lane; i < in; i += 32) acc += (A)to_f(x[(size_t)b * in + i]) * (A)to_f(W[(size_t)o * in + i]);
+    acc = warp_sum(acc);
+    if (lane == 0) {
+        if (bias) acc += (A)to_f(bias[o]);
+        if (relu && acc < 0) acc = 0;
+        y[(size_t)b * out + o] = from_a<TO>(acc);
+    }
+}
+template <typename TO> __device__ __forceinline__ float masked_dy(const TO *y, const TO *dy, size_t i, int relu) {
+    float d = to_f(dy[i]);
+    if (relu && !(to_f(y[i]) > 0.f)) d = 0.f;
+    return d;
+}
+// dx[b][i] = sum_o dz[b][o] W[o][i]
+template <typename T, typename TO>
+__global__ void fc_dx_kernel(const T *W, const TO *y, const TO *dy, T *dx, int B, int in, int out, int relu) {
+    long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long)B * in) return;
+    typedef typename AccOf<T>::type A;
+    int b = (int)(idx / in), i = (int)(idx % in);
+    A acc = 0;
+    for (int o = 0; o < out; ++o)
+        acc += (A)masked_dy(y, dy, (size_t)b * out + o, relu) * (A)to_f(W[(size_t)o * in + i]);
+    dx[idx] = from_a<T>(acc);
+}
+// dW[o][i] = sum_b dz[b][o] x[b][i]; db[o] = sum_b dz[b][o]   (thread per (o, i); i == in handles the bias)
+template <typename T, typename TO>
+__global__ void fc_dw_kernel(const T *x, const TO *y, const TO *dy, float *dW, float *db, int B, int in, int out,
+                             int relu) {
+    long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    int cols = in + 1;
+    if (idx >= (long)out * cols) return;
+    typedef typename AccOf<T>::type A;
+    int o = (int)(idx / cols), i = (int)(idx % cols);
+    A acc = 0;
+    if (i < in) {
+        for (int b = 0; b < B; ++b)
+            acc += (A)masked_dy(y, dy, (size_t)b * out + o, relu) * (A)to_f(x[(size_t)b * in + i]);
+        dW[(size_t)o * in + i] = (float)acc;
+    } else if (db) {
+        for (int b = 0; b < B; ++b) acc += (A)masked_dy(y, dy, (size_t)b * out + o, relu);
+        db[o] = (float)acc;
+    }
+}
+int launch_fc_fwd(int prec, const void *x, const void *W, const void *bias, void *y, int B, int in, int out, int relu,
+                  int out_f32, cudaStream_t s) {
+    long threads = (long)B * out * 32;
+    DISPATCH_PREC(prec, {
+        if (out_f32)
+            fc_fwd_kernel<T, float><<<ceil_div(threads, kThreads), kThreads, 0, s>>>((const T *)x, (const T *)W,
+                                                                                    (const T *)bias, (float *)y, B, in,
+                                                                                    out, relu);
+        else
+            fc_fwd_kernel<T, T><<<ceil_div(threads, kThreads), kThreads, 0, s>>>((const T *)x, (const T *)W,
+                                                                                (const T *)bias, (T *)y, B, in, out,
+                                                                                relu);
+    });
+    return 1;
+}
+int launch_fc_bwd(int prec, const void *x, const void *W, const void *y, const void *dy, void *dx, float *dW, float *db,
+                  int B, int in, int out, int relu, int out_f32, cudaStream_t s) {
+    int n = 0;
+    DISPATCH_PREC(prec, {
+        if (out_f32) {
+            if (dx) { fc_dx_kernel<T, float><<<ceil_div((long)B * in, kThreads), kThreads, 0, s>>>(
+                          (const T *)W, (const float *)y, (const float *)dy, (T *)dx, B, in, out, relu); ++n; }
+            fc_dw_kernel<T, float><<<ceil_div((long)out * (in + 1), kThreads), kThreads, 0, s>>>(
+                (const T *)x, (const float *)y, (const float *)dy, dW, db, B, in, out, relu);
+        } else {
+            if (dx) { fc_dx_kernel<T, T><<<ceil_div((long)B * in, kThreads), kThreads, 0, s>>>(
+                          (const T *)W, (const T *)y, (const T *)dy, (T *)dx, B, in, out, relu); ++n; }
+            fc_dw_kernel<T, T><<<ceil_div((long)out * (in + 1), kThreads), kThreads, 0, s>>>(
+                (const T *)x, (const T *)y, (const T *)dy, dW, db, B, in, out, relu);
+        }
+    });
+    return n + 1;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// softmax cross-entropy: one CTA, one warp per row, fixed-order final sum
+// ------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float exp_a(float v) { return expf(v); }
+__device__ __forceinline__ double exp_a(double v) { return exp(v); }
+__device__ __forceinline__ float log_a(float v) { return logf(v); }
+__device__ __forceinline__ double log_a(double v) { return log(v); }
+
+template <typename A>
+__global__ void softmax_ce_kernel(const float *logits, const int *labels, float *loss, float *dlogits, int B, int C) {
+    __shared__ A wsum[32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    A acc = 0;
+    for (int b = warp; b < B; b += nw) {
+        const float *z = logits + (size_t)b * C;
+        float mx = -INFINITY;
+        for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
+        mx = warp_max(mx);
+        A se = 0;
+        for (int c = lane; c < C; c += 32) se += exp_a((A)z[c] - (A)mx);
+        se = warp_sum(se);
+        const int y = labels[b];
+        for (int c = lane; c < C; c += 32)
+            dlogits[(size_t)b * C + c] = (float)((exp_a((A)z[c] - (A)mx) / se - (c == y ? (A)1 : (A)0)) / (A)B);
+        acc += log_a(se) + (A)mx - (A)z[y];
+    }
+    if (lane == 0) wsum[warp] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        A t = 0;
+        for (int w = 0; w < nw; ++w) t += wsum[w];
+        *loss = (float)(t / (A)B);
+    }
+}
+int launch_softmax_ce(int prec, const float *logits, const int *labels, float *loss, float *dlogits, int B, int C,
+                      cudaStream_t s) {
+    if (prec == P_BF16) softmax_ce_kernel<float><<<1, 1024, 0, s>>>(logits, labels, loss, dlogits, B, C);
+    else softmax_ce_kernel<double><<<1, 1024, 0, s>>>(logits, labels, loss, dlogits, B, C);
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// batch norm
+// ------------------------------------------------------------------------------------------------------
+// ticket counter (32 floats) + per-CTA partial sums, sized for the fp64 partials of the fp32 mode
+size_t bn_scratch_elems(int C) { return 32 + (size_t)kMaxPartials * 2 * C * 2; }
+
+static int bn_grid(long npix, int lanes) {
+    long g = (npix + (long)lanes * 8 - 1) / ((long)lanes * 8);
+    if (g < 1) g = 1;
+    if (g > kMaxPartials) g = kMaxPartials;
+    return (int)g;
+}
+
+// Two per-channel sums over all pixels.  MODE 0: (sum x, sum x^2) -> mean, invstd.
+// MODE 1: (sum dz, sum dz*xhat) -> dbeta, dgamma, with dz = dout * [out > 0] when relu.
+template <typename T, int VEC, int MODE>
+__global__ void __launch_bounds__(kThreads)
+bn_reduce_kernel(const T *__restrict__ x, const T *__restrict__ dout, const T *__restrict__ out,
+                 const float *__restrict__ mean_in, const float *__restrict__ invstd_in, float *o0, float *o1,
+                 float *scratch, long npix, int C, int relu) {
+    typedef typename AccOf<T>::type A;
+    __shared__ A sm[kThreads * VEC];
+    __shared__ bool is_last;
+    unsigned *counter = reinterpret_cast<unsigned *>(scratch);
+    A *part = reinterpret_cast<A *>(scratch + 32);
+    const int groups = C / VEC, lanes = kThreads / groups;
+    const int g = threadIdx.x % groups, lane = threadIdx.x / groups;
+    A s0[VEC], s1[VEC], mu[VEC], is[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) { s0[j] = 0; s1[j] = 0; mu[j] = 0; is[j] = 0; }
+    if (MODE == 1 && lane < lanes) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) { mu[j] = mean_in[g * VEC + j]; is[j] = invstd_in[g * VEC + j]; }
+    }
+    if (lane < lanes) {
+        for (long p = (long)blockIdx.x * lanes + lane; p < npix; p += (long)gridDim.x * lanes) {
+            A xv[VEC];
+            load_a<T, A, VEC>(x + p * C + g * VEC, xv);
+            if (MODE == 0) {
+#pragma unroll
+                for (int j = 0; j < VEC; ++j) { s0[j] += xv[j]; s1[j] += xv[j] * xv[j]; }
+            } else {
+                A dv[VEC];
+                load_a<T, A, VEC>(dout + p * C + g * VEC, dv);
+                if (relu) {
+                    float ov[VEC];
+                    load_f<T, VEC>(out + p * C + g * VEC, ov);
+#pragma unroll
+                    for (int j = 0; j < VEC; ++j) if (!(ov[j] > 0.f)) dv[j] = 0;
+                }
+#pragma unroll
+                for (int j = 0; j < VEC; ++j) { s0[j] += dv[j]; s1[j] += dv[j] * (xv[j] - mu[j]) * is[j]; }
+            }
+        }
+    }
+    // fold the pixel lanes of this CTA in a fixed order
+    for (int pass = 0; pass < 2; ++pass) {
+        __syncthreads();
+        if (lane < lanes) {
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) sm[lane * C + g * VEC + j] = pass == 0 ? s0[j] : s1[j];
+        }
+        __syncthreads();
+        if (threadIdx.x < C) {
+            A t = 0;
+            for (int l = 0; l < lanes; ++l) t += sm[l * C + threadIdx.x];
+            part[(size_t)blockIdx.x * 2 * C + pass * C + threadIdx.x] = t;
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int c = threadIdx.x; c < C; c += kThreads) {
+        double a = 0.0, b = 0.0;
+        for (unsigned i = 0; i < gridDim.x; ++i) {
+            a += (double)__ldcg(part + (size_t)i * 2 * C + c);
+            b += (double)__ldcg(part + (size_t)i * 2 * C + C + c);
+        }
+        if (MODE == 0) {
+            double m = a / (double)npix, var = b / (double)npix - m * m;
+            if (var < 0.0) var = 0.0;
+            o0[c] = (float)m;
+            o1[c] = (float)(1.0 / sqrt(var + (double)kBnEps));
+        } else {
+            o0[c] = (float)a;  // dbeta
+            o1[c] = (float)b;  // dgamma
+        }
+    }
+    if (threadIdx.x == 0) *counter = 0u;
+}
+
+template <typename T> static int vec_for(int C) { return (C % Vec16<T>::N == 0) ? Vec16<T>::N : 1; }
+
+int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *scratch, long npix, int C,
+                    cudaStream_t s) {
+    DISPATCH_PREC(prec, {
+        if (vec_for<T>(C) > 1) {
+            constexpr int V = Vec16<T>::N;
+            bn_reduce_kernel<T, V, 0><<<bn_grid(npix, kThreads / (C / V)), kThreads, 0, s>>>(
+                (const T *)x, nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
+        } else {
+            bn_reduce_kernel<T, 1, 0><<<bn_grid(npix, kThreads / C), kThreads, 0, s>>>(
+                (const T *)x, nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
+        }
+    });
+    return 1;
+}
+
+int launch_bn_bwd_reduce(int prec, const void *dout, const void *out, const void *x, const float *mean,
+                         const float *invstd, float *dgamma, float *dbeta, float *scratch, long npix, int C, int relu,
+                         cudaStream_t s) {
+    DISPATCH_PREC(prec, {
+        if (vec_for<T>(C) > 1) {
+            constexpr int V = Vec16<T>::N;
+            bn_reduce_kernel<T, V, 1><<<bn_grid(npix, kThreads / (C / V)), kThreads, 0, s>>>(
+                (const T *)x, (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
+        } else {
+            bn_reduce_kernel<T, 1, 1><<<bn_grid(npix, kThreads / C), kThreads, 0, s>>>(
+                (const T *)x, (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
+        }
+    });
+    return 1;
+}
+
+// y = [relu](gamma*(x-mean)*invstd + beta + shortcut)
+template <typename T, int VEC>
+__global__ void __launch_bounds__(kThreads)
+bn_apply_kernel(const T *__restrict__ x, const T *__restrict__ gamma, const T *__restrict__ beta,
+                const float *__restrict__ mean, const float *__restrict__ invstd, Shortcut sc, T *__restrict__ y,
+                long nvec, int H, int W, int C, int relu) {
+    long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nvec) return;
+    const int groups = C / VEC;
+    const int c0 = (int)(i % groups) * VEC;
+    const long p = i / groups;
+    typedef typename AccOf<T>::type A;
+    A v[VEC];
+    load_a<T, A, VEC>(x + p * C + c0, v);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j)
+        v[j] = (A)to_f(gamma[c0 + j]) * (v[j] - (A)mean[c0 + j]) * (A)invstd[c0 + j] + (A)to_f(beta[c0 + j]);
+    if (sc.mode == 1) {
+        A r[VEC];
+        load_a<T, A, VEC>((const T *)sc.a + p * C + c0, r);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) v[j] += r[j];
+    } else if (sc.mode == 2) {
+        if (c0 < sc.c_small) {  // host guarantees c_small % VEC == 0 on the vector path
+            const int wo = (int)(p % W), ho = (int)((p / W) % H);
+            const long n = p / ((long)W * H);
+            const long q = (n * sc.h_big + 2 * ho) * sc.w_big + 2 * wo;
+            A r[VEC];
+            load_a<T, A, VEC>((const T *)sc.a + q * sc.c_small + c0, r);
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) if (c0 + j < sc.c_small) v[j] += r[j];
+        }
+    }
+    if (relu) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) v[j] = v[j] > 0 ? v[j] : (A)0;
+    }
+    store_a<T, A, VEC>(y + p * C + c0, v);
+}
+
+int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta, const float *mean,
+                    const float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu, cudaStream_t s) {
+    const long npix = (long)B * H * W;
+    DISPATCH_PREC(prec, {
+        constexpr int V = Vec16<T>::N;
+        if (C % V == 0 && (sc.mode != 2 || sc.c_small % V == 0)) {
+            long nvec = npix * (C / V);
+            bn_apply_kernel<T, V><<<ceil_div(nvec, kThreads), kThreads, 0, s>>>(
+                (const T *)x, (const T *)gamma, (const T *)beta, mean, invstd, sc, (T *)y, nvec, H, W, C, relu);
+        } else {
+            long nvec = npix * C;
+            bn_apply_kernel<T, 1><<<ceil_div(nvec, kThreads), kThreads, 0, s>>>(
+                (const T *)x, (const T *)gamma, (const T *)beta, mean, invstd, sc, (T *)y, nvec, H, W, C, relu);
+        }
+    });
+    return 1;
+}
+
+// dx = gamma*invstd*(dz - dbeta/n - xhat*dgamma/n)
+template <typename T, int VEC>
+__global__ void __launch_bounds__(kThreads)
+bn_bwd_apply_kernel(const T *__restrict__ dout, const T *__restrict__ out, const T *__restrict__ x,
+                    const T *__restrict__ gamma, const float *__restrict__ mean, const float *__restrict__ invstd,
+                    const float *__restrict__ dgamma, const float *__restrict__ dbeta, T *__restrict__ dx, long nvec,
+                    long npix, int C, int relu) {
+    long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nvec) return;
+    const int groups = C / VEC;
+    const int c0 = (int)(i % groups) * VEC;
+    const long p = i / groups;
+    typedef typename AccOf<T>::type A;
+    A xv[VEC], dv[VEC];
+    load_a<T, A, VEC>(x + p * C + c0, xv);
+    load_a<T, A, VEC>(dout + p * C + c0, dv);
+    if (relu) {
+        float ov[VEC];
+        load_f<T, VEC>(out + p * C + c0, ov);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) if (!(ov[j] > 0.f)) dv[j] = 0;
+    }
+    const A cnt = (A)npix;
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        const int c = c0 + j;
+        const A xh = (xv[j] - (A)mean[c]) * (A)invstd[c];
+        dv[j] = (A)to_f(gamma[c]) * (A)invstd[c] * (dv[j] - (A)dbeta[c] / cnt - xh * (A)dgamma[c] / cnt);
+    }
+    store_a<T, A, VEC>(dx + p * C + c0, dv);
+}
+
+int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void *x, const void *gamma,
+                        const float *mean, const float *invstd, const float *dgamma, const float *dbeta, void *dx,
+                        long npix, int C, int relu, cudaStream_t s) {
+    DISPATCH_PREC(prec, {
+        constexpr int V = Vec16<T>::N;
+        if (C % V == 0) {
+            long nvec = npix * (C / V);
+            bn_bwd_apply_kernel<T, V><<<ceil_div(nvec, kThreads), kThreads, 0, s>>>(
+                (const T *)dout, (const T *)out, (const T *)x, (const T *)gamma, mean, invstd, dgamma, dbeta, (T *)dx,
+                nvec, npix, C, relu);
+        } else {
+            long nvec = npix * C;
+            bn_bwd_apply_kernel<T, 1><<<ceil_div(nvec, kThreads), kThreads, 0, s>>>(
+                (const T *)dout, (const T *)out, (const T *)x, (const T *)gamma, mean, invstd, dgamma, dbeta, (T *)dx,
+                nvec, npix, C, relu);
+        }
+    });
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// optimiser update with the delayed gradient (Eq. 9 / Algorithm 1, Algorithm 2) + weight-version refresh
+// ------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+update_kernel(float *__restrict__ w, float *__restrict__ v, float *__restrict__ m2, const float *__restrict__ g,
+              T *__restrict__ wv, size_t n, UpdateArgs a) {
+    size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= n) return;
+    const bool full = (i + 4 <= n) && ((reinterpret_cast<uintptr_t>(w + i) & 15) == 0) &&
+                      ((reinterpret_cast<uintptr_t>(v + i) & 15) == 0) &&
+                      ((reinterpret_cast<uintptr_t>(g + i) & 15) == 0) &&
+                      (a.mode != 1 || (reinterpret_cast<uintptr_t>(m2 + i) & 15) == 0);
+    const int cnt = (int)((n - i) < 4 ? (n - i) : 4);
+    float wv4[4], vv[4], gv[4], mv[4];
+    if (full) {
+        *reinterpret_cast<float4 *>(wv4) = *reinterpret_cast<const float4 *>(w + i);
+        if (a.mode != 2) {
+            *reinterpret_cast<float4 *>(vv) = *reinterpret_cast<const float4 *>(v + i);
+            *reinterpret_cast<float4 *>(gv) = *reinterpret_cast<const float4 *>(g + i);
+            if (a.mode == 1) *reinterpret_cast<float4 *>(mv) = *reinterpret_cast<const float4 *>(m2 + i);
+        }
+    } else {
+        for (int j = 0; j < cnt; ++j) {
+            wv4[j] = w[i + j];
+            if (a.mode != 2) { vv[j] = v[i + j]; gv[j] = g[i + j]; if (a.mode == 1) mv[j] = m2[i + j]; }
+        }
+    }
+    typedef typename AccOf<T>::type A;  // the master state is fp32 either way; A is the arithmetic in between
+    if (a.mode == 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const A d = (A)gv[j] + (A)a.wd * (A)wv4[j];
+            const A vn = (A)a.mu * (A)vv[j] + d;
+            vv[j] = (float)vn;
+            wv4[j] = (float)((A)wv4[j] - (A)a.lr * vn);
+        }
+    } else if (a.mode == 1) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const A m1 = (A)a.b1 * (A)vv[j] + ((A)1 - (A)a.b1) * (A)gv[j];
+            const A m2n = (A)a.b2 * (A)mv[j] + ((A)1 - (A)a.b2) * (A)gv[j] * (A)gv[j];
+            vv[j] = (float)m1;
+            mv[j] = (float)m2n;
+            wv4[j] = (float)((A)wv4[j] - (A)a.lr * (m1 / (A)a.c1c) / (sqrt(m2n / (A)a.c2c) + (A)a.eps));
+        }
+    }
+    if (full) {
+        if (a.mode != 2) {
+            *reinterpret_cast<float4 *>(w + i) = *reinterpret_cast<const float4 *>(wv4);
+            *reinterpret_cast<float4 *>(v + i) = *reinterpret_cast<const float4 *>(vv);
+            if (a.mode == 1) *reinterpret_cast<float4 *>(m2 + i) = *reinterpret_cast<const float4 *>(mv);
+        }
+    } else if (a.mode != 2) {
+        for (int j = 0; j < cnt; ++j) { w[i + j] = wv4[j]; v[i + j] = vv[j]; if (a.mode == 1) m2[i + j] = mv[j]; }
+    }
+    for (int j = 0; j < cnt; ++j) wv[i + j] = from_f<T>(wv4[j]);
+}
+
+int launch_update(int prec, float *w, float *v, float *m2, const float *g, void *wv, size_t n, UpdateArgs a,
+                  cudaStream_t s) {
+    if (n == 0) return 0;
+    DISPATCH_PREC(prec, update_kernel<T><<<ceil_div((n + 3) / 4, kThreads), kThreads, 0, s>>>(w, v, m2, g, (T *)wv, n, a));
+    return 1;
+}
+
+int launch_cast(int prec, const float *src, void *dst, size_t n, cudaStream_t s) {
+    UpdateArgs a = {};
+    a.mode = 2;
+    return launch_update(prec, const_cast<float *>(src), nullptr, nullptr, nullptr, dst, n, a, s);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// weight initialisation: counter-based normal draws (splitmix64 hash of (seed, stream, index) + Box-Muller)
+// ------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+    z += 0x9e3779b97f4a7c15ull;
+    z = (z ^ (z >> 30)) * 0xbf58476d1ce4e5b9ull;
+    z = (z ^ (z >> 27)) * 0x94d049bb133111ebull;
+    return z ^ (z >> 31);
+}
+__global__ void fill_normal_kernel(float *dst, size_t n, float stddev, unsigned long long seed,
+                                   unsigned long long stream_id) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    unsigned long long h = mix64(mix64(seed ^ (stream_id * 0xd1342543de82ef95ull)) + i);
+    unsigned long long h2 = mix64(h);
+    float u1 = ((h >> 40) + 1.0f) * (1.0f / 16777217.0f);  // (0, 1)
+    float u2 = (h2 >> 40) * (1.0f / 16777216.0f);
+    dst[i] = stddev * sqrtf(-2.f * logf(u1)) * cospif(2.f * u2);
+}
+__global__ void fill_const_kernel(float *dst, size_t n, float v) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = v;
+}
+int launch_fill_normal(float *dst, size_t n, float stddev, unsigned long long seed, unsigned long long stream_id,
+                       cudaStream_t s) {
+    if (n == 0) return 0;
+    fill_normal_kernel<<<ceil_div(n, kThreads), kThreads, 0, s>>>(dst, n, stddev, seed, stream_id);
+    return 1;
+}
+int launch_fill_const(float *dst, size_t n, float v, cudaStream_t s) {
+    if (n == 0) return 0;
+    fill_const_kernel<<<ceil_div(n, kThreads), kThreads, 0, s>>>(dst, n, v);
+    return 1;
+}
+
+}  // namespace ddg

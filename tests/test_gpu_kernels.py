@@ -1,0 +1,122 @@
+"""Per-kernel GPU parity through the single-kernel C-ABI entry points, against the oracle's primitives on the same
+seeded inputs.  Shapes span several tiles, ragged tails, both strides and both precisions."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ddg_oracle as orc
+from tests.parity import rel
+
+pytestmark = pytest.mark.gpu
+
+TOL = {0: 1e-5, 1: 6e-3}   # fp32: accumulation order only; bf16: inputs are exact bf16, output rounding 2^-9
+
+
+def tdtype(prec):
+    return torch.bfloat16 if prec else torch.float32
+
+
+def to_dev(a_nchw, prec):
+    """fp64 NCHW numpy -> device NHWC tensor in the precision; returns (tensor, the values it holds as fp64 NCHW)."""
+    t = torch.from_numpy(np.ascontiguousarray(a_nchw)).to(tdtype(prec))
+    held = t.to(torch.float64).numpy()
+    if t.dim() == 4:
+        t = t.permute(0, 2, 3, 1).contiguous()
+    return t.cuda(), held
+
+
+def from_dev(t_nhwc):
+    return t_nhwc.to(torch.float64).cpu().permute(0, 3, 1, 2).contiguous().numpy()
+
+
+SHAPES = [  # B, H, W, Cin, Cout, stride
+    (2, 8, 8, 16, 16, 1), (3, 32, 32, 16, 16, 1), (5, 16, 16, 32, 32, 1), (9, 8, 8, 64, 64, 1),
+    (3, 32, 32, 16, 32, 2), (3, 16, 16, 32, 64, 2), (4, 32, 32, 3, 16, 1), (2, 7, 5, 5, 12, 1), (2, 9, 7, 6, 10, 2),
+    (128, 8, 8, 64, 64, 1),
+]
+
+
+@pytest.mark.parametrize("prec", [0, 1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_conv3x3_fwd_dgrad_wgrad(shape, prec):
+    from paper_1804_10574_b200 import binding
+    B, H, W, Ci, Co, st = shape
+    rng = np.random.default_rng(11)
+    Ho, Wo = (H - 1) // st + 1, (W - 1) // st + 1
+    x, xh = to_dev(rng.standard_normal((B, Ci, H, W)), prec)
+    w = torch.from_numpy(rng.standard_normal((Co, Ci, 3, 3)) * np.sqrt(2.0 / (9 * Ci))).to(tdtype(prec))
+    wh = w.to(torch.float64).numpy()
+    w = w.cuda()
+    dy, dyh = to_dev(rng.standard_normal((B, Co, Ho, Wo)), prec)
+    y = torch.empty(B, Ho, Wo, Co, dtype=tdtype(prec), device="cuda")
+    dx = torch.empty(B, H, W, Ci, dtype=tdtype(prec), device="cuda")
+    dw = torch.empty(Co, Ci, 3, 3, dtype=torch.float32, device="cuda")
+    scratch = torch.empty(max(1, binding.conv3x3_wgrad_scratch_elems(B, H, W, Ci, Co, st)), dtype=torch.float32,
+                          device="cuda")
+    binding.conv3x3_fwd(prec, x, w, y, B, H, W, Ci, Co, st)
+    binding.conv3x3_dgrad(prec, dy, w, dx, B, H, W, Ci, Co, st)
+    binding.conv3x3_wgrad(prec, x, dy, dw, scratch, B, H, W, Ci, Co, st)
+    torch.cuda.synchronize()
+    y_ref = orc.conv3x3_forward(xh, wh, st)
+    dx_ref, dw_ref = orc.conv3x3_backward(xh, wh, dyh, st)
+    assert rel(from_dev(y), y_ref) < TOL[prec]
+    assert rel(from_dev(dx), dx_ref) < TOL[prec]
+    assert rel(dw.cpu().numpy(), dw_ref) < 1e-5   # fp32 output from exact inputs in both precisions
+    # a second call on the same scratch gives the same bits (fixed summation order)
+    dw2 = torch.empty_like(dw)
+    binding.conv3x3_wgrad(prec, x, dy, dw2, scratch, B, H, W, Ci, Co, st)
+    torch.cuda.synchronize()
+    assert torch.equal(dw, dw2)
+
+
+@pytest.mark.parametrize("prec", [0, 1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("shape", [(4, 64, 16), (7, 1024, 16), (33, 256, 32), (128, 64, 64), (3, 35, 12), (2, 3, 8)],
+                         ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("relu,res", [(0, 0), (1, 0), (1, 1)])
+def test_bn_fwd_bwd(shape, prec, relu, res):
+    from paper_1804_10574_b200 import binding
+    B, HW, C = shape
+    rng = np.random.default_rng(5)
+    x, xh = to_dev((rng.standard_normal((B, C, HW, 1)) * 1.5 + 0.3), prec)
+    gamma = torch.from_numpy(1 + 0.2 * rng.standard_normal(C)).to(tdtype(prec))
+    beta = torch.from_numpy(0.2 * rng.standard_normal(C)).to(tdtype(prec))
+    gh, bh = gamma.to(torch.float64).numpy(), beta.to(torch.float64).numpy()
+    r, rh = to_dev(rng.standard_normal((B, C, HW, 1)), prec)
+    dout, douth = to_dev(rng.standard_normal((B, C, HW, 1)), prec)
+    y = torch.empty_like(x)
+    dx = torch.empty_like(x)
+    mean, invstd, dg, db = (torch.empty(C, dtype=torch.float32, device="cuda") for _ in range(4))
+    scratch = torch.full((binding.bn_scratch_elems(C),), 7.0, dtype=torch.float32, device="cuda")  # junk on entry
+    binding.bn_fwd(prec, x, gamma.cuda(), beta.cuda(), r if res else None, y, mean, invstd, scratch, B, HW, C, relu)
+    binding.bn_bwd(prec, dout, y, x, gamma.cuda(), mean, invstd, dx, dg, db, scratch, B, HW, C, relu)
+    torch.cuda.synchronize()
+    y_ref, m_ref, is_ref = orc.bn_forward(xh, gh, bh)
+    if res:
+        y_ref = y_ref + rh
+    if relu:
+        y_ref = np.maximum(y_ref, 0)
+    assert rel(mean.cpu().numpy(), m_ref) < 1e-5 and rel(invstd.cpu().numpy(), is_ref) < 1e-5
+    assert rel(from_dev(y), y_ref) < TOL[prec]
+    # backward reference uses the mask of the output the GPU actually stored
+    dz = douth * (from_dev(y) > 0) if relu else douth
+    dx_ref, dg_ref, db_ref = orc.bn_backward(xh, m_ref, is_ref, gh, dz)
+    tol_s = 2e-5 if HW * B > 4 else 1e-3
+    assert rel(db.cpu().numpy(), db_ref) < tol_s and rel(dg.cpu().numpy(), dg_ref) < tol_s
+    assert rel(from_dev(dx), dx_ref) < max(TOL[prec], tol_s)
+
+
+@pytest.mark.parametrize("prec", [0, 1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("n", [1, 5, 1024, 1733812])
+def test_sgd_update(n, prec):
+    from paper_1804_10574_b200 import binding
+    rng = np.random.default_rng(3)
+    w, v, g = (rng.standard_normal(n).astype(np.float32) for _ in range(3))
+    wd, vd, gd = (torch.from_numpy(a).cuda() for a in (w, v, g))
+    wv = torch.empty(n, dtype=tdtype(prec), device="cuda")
+    binding.sgd_update(prec, wd, vd, gd, wv, n, 0.1, 0.9, 5e-4)
+    torch.cuda.synchronize()
+    d = g.astype(np.float64) + 5e-4 * w
+    v_ref = 0.9 * v + d
+    w_ref = w - 0.1 * v_ref
+    assert rel(vd.cpu().numpy(), v_ref) < 1e-6 and rel(wd.cpu().numpy(), w_ref) < 1e-6
+    assert torch.equal(wv, wd.to(tdtype(prec)))      # the version slot is the cast of the new master weights

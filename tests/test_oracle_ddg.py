@@ -221,3 +221,18 @@ def test_bf16_rounding_switch_perturbs_but_does_not_change_the_method():
             assert sa == sb
             if sa >= 0:
                 assert 1e-5 < rel(gb, ga) < 0.3
+
+
+def test_fp32_storage_rounding_is_a_tiny_perturbation_of_the_exact_run():
+    """ORC_ROUND_FP32 only rounds what is stored: the run must stay within float rounding of the exact one."""
+    net = dict(layers=nets.resnet(1, 10), in_shape=(3, 16, 16), num_classes=10, batch=4)
+    a, _ = make(net, [2], lr=0.05, momentum=0.9, weight_decay=5e-4)
+    b, _ = make(net, [2], lr=0.05, momentum=0.9, weight_decay=5e-4, flags=orc.ROUND_FP32)
+    for t in range(3):
+        la, lb = a.step(*data(net, t)), b.step(*data(net, t))
+        assert abs(la - lb) < 1e-5
+    assert rel(b.get_weights(), a.get_weights()) < 1e-5
+    w = b.get_weights()
+    np.testing.assert_array_equal(w, w.astype(np.float32).astype(np.float64))   # master weights are float values
+    sb, gb = b.get_grads(1)
+    np.testing.assert_array_equal(gb, gb.astype(np.float32).astype(np.float64))
