@@ -1,0 +1,266 @@
+#!/usr/bin/env python3
+"""Benchmark of the DDG training step: images/sec of one DDG iteration (ResNet-110, K=4, batch 128, bf16 storage)
+on synthetic CIFAR-shaped data, one B200 per process.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--net resnet110] [--modules 4]
+
+N > 1 (under torchrun) runs N independent replicas (the method does not shard across GPUs here): `value` is the sum
+over replicas, timed as the max over ranks.  `--impl reference` times the CPU oracle on a bounded sample of the same
+workload on the host cores.  One JSON line is printed by rank 0.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "DDG train images/sec (ResNet-110, K=4, 1 B200)"
+
+
+def parse():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=200)
+    p.add_argument("--warmup", type=int, default=20)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--net", default="resnet110", choices=["resnet110", "resnet56", "resnet8", "mlp"])
+    p.add_argument("--modules", type=int, default=0, help="K; 0 = the configuration's own split")
+    p.add_argument("--batch", type=int, default=0)
+    p.add_argument("--no-graph", action="store_true")
+    p.add_argument("--cpu-batch", type=int, default=8, help="batch of the bounded CPU-oracle sample")
+    p.add_argument("--cpu-steps", type=int, default=0, help="timed oracle steps (0 = K+1)")
+    p.add_argument("--skip-cpu", action="store_true")
+    return p.parse_args()
+
+
+def workload(args):
+    from paper_1804_10574_b200 import nets
+    cfg = dict(nets.config(args.net))
+    if args.modules:
+        cfg["split_after"] = nets.split_even_blocks(cfg["layers"], args.modules) if args.net.startswith("resnet") \
+            else cfg["split_after"]
+    if args.batch:
+        cfg["batch"] = args.batch
+    return cfg
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 7 and r[3 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def time_oracle(cfg, batch, n_steps):
+    """The CPU oracle as it stands, on a bounded sample of the workload: same net and split, smaller batch."""
+    from oracle import ddg_oracle as orc
+    from paper_1804_10574_b200 import synth
+    K = len(cfg["split_after"]) + 1
+    o = cfg["opt"]
+    ref = orc.Oracle(cfg["layers"], cfg["split_after"], batch, cfg["in_shape"], cfg["num_classes"], lr=o["lr"],
+                     momentum=o["momentum"], weight_decay=o["weight_decay"],
+                     flags=orc.ROUND_BF16 if cfg["precision"] == "bf16" else orc.ROUND_FP32)
+    ref.set_weights(synth.init_weights(cfg["layers"]).astype(np.float64))
+    data = [synth.batch(t, batch, cfg["in_shape"], cfg["num_classes"]) for t in range(K - 1 + n_steps)]
+    for t in range(K - 1):                      # fill the pipeline: untimed
+        ref.step(*data[t])
+    t0 = time.perf_counter()
+    for t in range(K - 1, K - 1 + n_steps):
+        ref.step(*data[t])
+    dt = time.perf_counter() - t0
+    ref.close()
+    cores = len(os.sched_getaffinity(0))
+    threads = int(os.environ.get("OMP_NUM_THREADS", cores))
+    return {"value": batch * n_steps / dt, "unit": "images/s", "cores": min(cores, threads), "kind": "oracle",
+            "sample": "%d full DDG iterations of the same network and split at batch %d (of %d), fp64, after K-1 "
+                      "untimed pipeline-fill iterations" % (n_steps, batch, cfg["batch"]), "seconds": dt}
+
+
+def dominant_kernel_roofline(torch, binding, cfg, peaks):
+    """Times the kernel with the largest share of the step (3x3 convolution forward on the widest feature map) alone,
+    at the workload's shape and launch configuration, with CUDA events on its stream."""
+    B, H, W, C = cfg["batch"], 32, 32, 16
+    x = torch.randn(B, H, W, C, device="cuda").to(torch.bfloat16)
+    w = (torch.randn(C, C, 3, 3, device="cuda") * (2.0 / (9 * C)) ** 0.5).to(torch.bfloat16)
+    y = torch.empty_like(x)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    s = torch.cuda.current_stream()
+    for _ in range(3):
+        binding.conv3x3_fwd(1, x, w, y, B, H, W, C, C, 1, s.cuda_stream)
+    times = []
+    for _ in range(20):
+        flush.zero_()                                  # evict the tensors from L2 between timed launches
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s)
+        binding.conv3x3_fwd(1, x, w, y, B, H, W, C, C, 1, s.cuda_stream)
+        e1.record(s)
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e-3)
+    dt = float(np.mean(times))
+    alg_bytes = 2 * x.numel() * 2 + w.numel() * 2     # read x, write y (bf16) + weights
+    achieved = alg_bytes / dt / 1e9
+    peak = peaks.get("hbm_gbs", 6650.0)
+    return {"kernel": "conv3x3_fwd 16->16 32x32 B=%d bf16" % B, "bound": "hbm", "achieved": achieved, "peak": peak,
+            "unit": "GB/s", "frac": achieved / peak, "traffic": None, "launch_us": dt * 1e6,
+            "peak_source": "measured" if "hbm_gbs" in peaks else "fallback"}
+
+
+def main():
+    args = parse()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = workload(args)
+    K = len(cfg["split_after"]) + 1
+    wl = "%s K=%d batch %d %s, synthetic CIFAR-shaped N(0,1) images, %d classes" % (
+        args.net, K, cfg["batch"], cfg["precision"], cfg["num_classes"])
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        n = args.cpu_steps or min(max(args.steps, 1), 2)
+        times = [time_oracle(cfg, args.cpu_batch, 1) for _ in range(min(args.warmup, 1))]   # one warm-up sample
+        r = time_oracle(cfg, args.cpu_batch, n)
+        out = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": "images/s", "n_gpus": 0,
+               "steps": n, "warmup": len(times), "ms_per_step": 1e3 * r["seconds"] / n, "higher_is_better": True,
+               "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+               "config": {"workload": wl, "sample": r["sample"]},
+               "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+               "e2e": {"value": r["value"], "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(out))
+        return 0
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the DDG step has no CPU path")
+    torch.cuda.set_device(local)
+    from paper_1804_10574_b200 import binding, synth
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    streams = [torch.cuda.Stream() for _ in range(K)]
+    o = cfg["opt"]
+    net = binding.Ddg(cfg["layers"], cfg["split_after"], cfg["batch"], cfg["in_shape"], cfg["num_classes"],
+                      precision=cfg["precision"], lr=o["lr"], momentum=o["momentum"], weight_decay=o["weight_decay"],
+                      use_graph=not args.no_graph, streams=[s.cuda_stream for s in streams])
+    net.set_weights(synth.init_weights(cfg["layers"]))
+    n_batches = K + 2
+    host = [synth.batch(t, cfg["batch"], cfg["in_shape"], cfg["num_classes"]) for t in range(n_batches)]
+    dev = [(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()) for x, y in host]
+    pinned = [(torch.from_numpy(x).pin_memory(), torch.from_numpy(y).pin_memory()) for x, y in host]
+    warm = max(args.warmup, K - 1 + 3)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident throughput: inputs already in HBM, no host round trip inside the timed region ----
+    for t in range(warm):
+        net.step(*dev[t % n_batches], want_loss=False)
+    net.sync()
+    launches_per_step = net.last_step_launches()
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(streams[0])
+    for t in range(args.steps):
+        net.step(*dev[(warm + t) % n_batches], want_loss=False)
+    net.sync()                       # all K streams drained; the end event then lands after every kernel of the region
+    e1.record(streams[0])
+    barrier()
+    dt = e0.elapsed_time(e1) * 1e-3
+    clocks = sampler.stop()
+
+    # ---- end to end through the public call with host buffers: H2D of x, y and D2H of the loss every step ----
+    for t in range(3):
+        net.step_host(*pinned[t % n_batches])
+    barrier()
+    n_e2e = max(10, args.steps // 4)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(streams[0])
+    for t in range(n_e2e):
+        loss = net.step_host(*pinned[t % n_batches])
+    f1.record(streams[0])
+    barrier()
+    dt_e2e = f0.elapsed_time(f1) * 1e-3
+
+    tt = torch.tensor([dt, dt_e2e], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    dt, dt_e2e = float(tt[0]), float(tt[1])
+
+    if rank == 0:
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except Exception:
+            pass
+        roof = dominant_kernel_roofline(torch, binding, cfg, peaks)
+        cpu = None
+        if world == 1 and not args.skip_cpu:
+            r = time_oracle(cfg, args.cpu_batch, args.cpu_steps or 2)
+            cpu = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        imgs = cfg["batch"] * args.steps * world
+        x_bytes = int(np.prod((cfg["batch"],) + tuple(cfg["in_shape"]))) * 4
+        out = {"metric": METRIC, "value": imgs / dt, "unit": "images/s", "n_gpus": world, "steps": args.steps,
+               "warmup": warm, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "bf16" if cfg["precision"] == "bf16" else "f32", "data": "synthetic",
+               "config": {"workload": wl, "parallelism": "%d CUDA streams on one GPU%s" % (
+                   K, "" if world == 1 else ", %d independent replicas" % world),
+                   "cuda_graph": not args.no_graph,
+                   "l2": "no flush: one iteration touches > 1 GB of activations, far above the 126 MB L2",
+                   "final_loss": loss},
+               "clocks": clocks, "gpu_launches": int(launches_per_step * args.steps),
+               "e2e": {"value": cfg["batch"] * n_e2e * world / dt_e2e, "unit": "images/s",
+                       "h2d_bytes_per_step": x_bytes + cfg["batch"] * 4, "d2h_bytes_per_step": 4, "steps": n_e2e},
+               "roofline": roof, "cpu_baseline": cpu}
+        print(json.dumps(out))
+    net.destroy()
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -129,11 +129,15 @@ class Ddg:
             raise DdgError(rc, (_lib.ddg_last_error(self._h) or b"").decode())
 
     def destroy(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:
             _lib.ddg_destroy(self._h)
             self._h = None
 
-    __del__ = destroy
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
     def step(self, x_dev, y_dev, want_loss=True):
         loss = ctypes.c_float()

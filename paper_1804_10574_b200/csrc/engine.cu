@@ -621,6 +621,8 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
     CU(cudaMemset(c->loss_dev, 0, 4));
     CU(cudaMallocHost(&c->pinned_loss, 4));
     CU(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+    // the memsets above ran on the legacy default stream, which the non-blocking module streams do not wait for
+    CU(cudaDeviceSynchronize());
     ddg_status st = init_weights(c);
     if (st != DDG_OK) { g_create_error = c->err; return st; }
     *out = holder.release();
@@ -702,6 +704,7 @@ ddg_status ddg_get_weights(ddg_ctx *ctx, float *dst, size_t n, int on_device) {
     if (st != DDG_OK) return st;
     for (auto &m : ctx->mods)
         CU(cudaMemcpy(dst + m.p_off_global, m.w, m.P * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost));
+    if (on_device) CU(cudaDeviceSynchronize());
     return DDG_OK;
 }
 
@@ -714,8 +717,9 @@ ddg_status ddg_set_weights(ddg_ctx *ctx, const float *src, size_t n, int on_devi
         CU(cudaMemcpy(m.w, src + m.p_off_global, m.P * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice));
         CU(cudaMemset(m.v, 0, m.P * 4));
         if (m.m2) CU(cudaMemset(m.m2, 0, m.P * 4));
-        launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream);
     }
+    CU(cudaDeviceSynchronize());  // default-stream copies and memsets are not ordered against the module streams
+    for (auto &m : ctx->mods) launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream);
     CU(cudaGetLastError());
     return sync_all(ctx);
 }
@@ -728,10 +732,11 @@ ddg_status ddg_get_grads(ddg_ctx *ctx, int k, float *dst, size_t n, int on_devic
     Module &m = ctx->mods[k];
     if (sample) *sample = m.last_sample;
     if (m.last_sample < 0) {
-        if (on_device) CU(cudaMemset(dst, 0, n * 4)); else memset(dst, 0, n * 4);
+        if (on_device) { CU(cudaMemset(dst, 0, n * 4)); CU(cudaDeviceSynchronize()); } else memset(dst, 0, n * 4);
         return DDG_OK;
     }
     CU(cudaMemcpy(dst, m.g, n * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost));
+    if (on_device) CU(cudaDeviceSynchronize());
     return DDG_OK;
 }
 

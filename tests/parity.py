@@ -77,9 +77,17 @@ class TieExplainer:
 
 
 def run_pair(cfg, steps, tol, loss_tol, precision=None, split_after=None, use_graph=False, opt="sgd",
-             perturb_affine=0.1, batch=None, check_every=1, lr_schedule=None):
+             perturb_affine=0.1, batch=None, check_every=1, lr_schedule=None, noise_mult=None):
     """Step both implementations `steps` times; assert parity at every `check_every`-th step.  Returns the worst
-    relative errors seen, for reporting."""
+    relative errors seen, for reporting.
+
+    noise_mult (bf16 production kernels): rounding every stored tensor to bf16 makes two evaluations that differ in
+    the last bit before a store decorrelate within a few layers (a one-ulp difference of one activation flips the
+    rounding of a share of the next layer's outputs), so a path that accumulates in fp32 cannot reproduce the
+    oracle's bf16 decisions and its gradients carry an independent draw of the same format noise.  The oracle
+    measures that noise itself: e_orc = rel(oracle with bf16 storage, exact oracle) per tensor.  A gradient tensor
+    passes if it is within `tol` of the bf16-storage oracle, or if its distance to the exact oracle is at most
+    noise_mult * e_orc + tol."""
     from paper_1804_10574_b200 import binding
     layers = cfg["layers"]
     split_after = cfg["split_after"] if split_after is None else split_after
@@ -100,9 +108,15 @@ def run_pair(cfg, steps, tol, loss_tol, precision=None, split_after=None, use_gr
     w0 = synth.init_weights(layers, perturb_affine=perturb_affine)
     ref.set_weights(w0.astype(np.float64))
     gpu.set_weights(w0)
+    exact = None
+    if noise_mult is not None:
+        exact = orc.Oracle(layers, split_after, B, cfg["in_shape"], cfg["num_classes"], opt=opt, lr=o["lr"],
+                           momentum=o["momentum"], weight_decay=o["weight_decay"], beta1=f32(0.9), beta2=f32(0.999),
+                           eps=f32(1e-8), flags=0)
+        exact.set_weights(w0.astype(np.float64))
     assert gpu.n_params == ref.n_params and gpu.per_module == ref.per_module
     segs = segments_by_module(layers, split_after)
-    worst = dict(loss=0.0, grad=0.0, weight=0.0, tie_steps=0)
+    worst = dict(loss=0.0, grad=0.0, weight=0.0, tie_steps=0, grad_vs_exact=0.0, oracle_bf16_vs_exact=0.0)
     wbuf = np.empty(gpu.n_params, dtype=np.float32)
     ties = TieExplainer(cfg, B, flags)
     snapshots, batches = {}, {}
@@ -116,6 +130,10 @@ def run_pair(cfg, steps, tol, loss_tol, precision=None, split_after=None, use_gr
         snapshots.pop(t - K - 1, None); batches.pop(t - K - 1, None)
         loss_gpu = gpu.step(xd, yd)
         loss_ref = ref.step(x, y)
+        if exact is not None:
+            if lr_schedule is not None:
+                exact.set_lr(f32(lr_schedule(t)))
+            exact.step(x, y)
         if t % check_every and t != steps - 1:
             continue
         dl = abs(loss_gpu - loss_ref) / max(1.0, abs(loss_ref))
@@ -130,6 +148,20 @@ def run_pair(cfg, steps, tol, loss_tol, precision=None, split_after=None, use_gr
             s_ref, g_ref = ref.get_grads(k)
             assert s_gpu == s_ref == (t - K + k + 1 if t - K + k + 1 >= 0 else -1), (t, k, s_gpu, s_ref)
             resid = None
+            if exact is not None and s_ref >= 0:
+                g_ex = exact.get_grads(k)[1]
+                for name, a, b in segs[k]:
+                    e_gpu, e_orc = rel(gbuf[a:b], g_ex[a:b]), rel(g_ref[a:b], g_ex[a:b])
+                    worst["grad"] = max(worst["grad"], rel(gbuf[a:b], g_ref[a:b]))
+                    worst["grad_vs_exact"] = max(worst["grad_vs_exact"], e_gpu)
+                    worst["oracle_bf16_vs_exact"] = max(worst["oracle_bf16_vs_exact"], e_orc)
+                    assert rel(gbuf[a:b], g_ref[a:b]) <= tol or e_gpu <= noise_mult * e_orc + tol, \
+                        "step %d module %d grad %s: %.3e from the exact oracle, format noise %.3e" % (t, k, name, e_gpu, e_orc)
+                    e = rel(wbuf[off + a:off + b], wref[off + a:off + b])
+                    worst["weight"] = max(worst["weight"], e)
+                    assert e <= tol, "step %d module %d weight %s: rel %.3e > %.1e" % (t, k, name, e, tol)
+                off += gpu.per_module[k]
+                continue
             if s_ref >= 0 and any(rel(gbuf[a:b], g_ref[a:b]) > tol for _, a, b in segs[k]):
                 # not within tolerance of the oracle's own ReLU decisions: is it another valid set of decisions?
                 resid, coef, n_ties = ties.residual(s_ref, snapshots[s_ref], *batches[s_ref], mod_off[k],
@@ -154,4 +186,6 @@ def run_pair(cfg, steps, tol, loss_tol, precision=None, split_after=None, use_gr
             off += gpu.per_module[k]
     gpu.destroy()
     ref.close()
+    if exact is not None:
+        exact.close()
     return worst

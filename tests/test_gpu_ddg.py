@@ -64,7 +64,7 @@ def test_generic_layers_fp32():
 
 def test_resnet8_k2_bf16():
     cfg = dict(nets.config("resnet8"), opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
-    w = run_pair(cfg, 6, BF16_TOL, 5e-3, precision="bf16")
+    w = run_pair(cfg, 6, BF16_TOL, 5e-3, precision="bf16", noise_mult=2.0)
     print("resnet8 bf16 worst", w)
 
 
@@ -72,7 +72,7 @@ def test_resnet20_k3_bf16_graph():
     L = nets.resnet(3, 10)
     cfg = dict(layers=L, split_after=nets.split_even_blocks(L, 3), batch=32, in_shape=(3, 32, 32), num_classes=10,
                precision="bf16", opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
-    w = run_pair(cfg, 8, BF16_TOL, 5e-3, use_graph=True)
+    w = run_pair(cfg, 8, BF16_TOL, 5e-3, use_graph=True, noise_mult=2.0)
     print("resnet20 bf16 worst", w)
 
 
