@@ -144,6 +144,10 @@ void ddg_destroy(ddg_ctx *ctx);
  * `stream` is a cudaStream_t (NULL = default stream).  The calls only enqueue.
  * --------------------------------------------------------------------------------------------------------- */
 
+/* 1 when the bf16 forward / input-gradient convolution of this shape runs on the tensor-core (tcgen05) kernels,
+ * 2 when the weight gradient does too (3 = both), 0 when the CUDA-core kernels take it.  Needs a CUDA device. */
+int ddg_tensor_core_path(int B, int H, int W, int Cin, int Cout, int stride);
+
 /* y = conv3x3(x, w), pad 1 (layer forward, Eq. 3).  x [B][H][W][Cin], y [B][Ho][Wo][Cout], Ho = (H-1)/stride+1. */
 ddg_status ddg_conv3x3_fwd(int precision, const void *x, const void *w, void *y, int B, int H, int W, int Cin,
                            int Cout, int stride, void *stream);

@@ -26,7 +26,7 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_set_weights", "ddg_get_grads", "ddg_get_loss_dev", "ddg_last_step_launches", "ddg_sync",
            "ddg_last_error", "ddg_destroy", "ddg_conv3x3_fwd", "ddg_conv3x3_dgrad",
            "ddg_conv3x3_wgrad_scratch_elems", "ddg_conv3x3_wgrad", "ddg_bn_scratch_elems", "ddg_bn_fwd", "ddg_bn_bwd",
-           "ddg_sgd_update"]
+           "ddg_sgd_update", "ddg_tensor_core_path"]
 
 
 class Layer(ctypes.Structure):
@@ -71,6 +71,7 @@ _lib.ddg_bn_scratch_elems.argtypes = [_i]
 _lib.ddg_bn_scratch_elems.restype = _sz
 _lib.ddg_bn_fwd.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_bn_bwd.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
+_lib.ddg_tensor_core_path.argtypes = [_i] * 6
 _lib.ddg_sgd_update.argtypes = [_i, _vp, _vp, _vp, _vp, _sz, _f, _f, _f, _vp]
 
 
@@ -181,6 +182,10 @@ class Ddg:
 def _ok(rc):
     if rc != 0:
         raise DdgError(rc, "kernel entry point failed")
+
+
+def tensor_core_path(B, H, W, Cin, Cout, stride):
+    return _lib.ddg_tensor_core_path(B, H, W, Cin, Cout, stride)
 
 
 def conv3x3_fwd(prec, x, w, y, B, H, W, Cin, Cout, stride, stream=None):

@@ -22,6 +22,11 @@ bool conv_shape_ok(int B, int H, int W, int Cin, int Cout, int stride) {
 
 extern "C" {
 
+int ddg_tensor_core_path(int B, int H, int W, int Cin, int Cout, int stride) {
+    if (init_once() != DDG_OK) return 0;
+    return (conv_tc_supported(B, H, W, Cin, Cout, stride) ? 1 : 0) | (wgrad_tc_supported(B, H, W, Cin, Cout, stride) ? 2 : 0);
+}
+
 ddg_status ddg_conv3x3_fwd(int precision, const void *x, const void *w, void *y, int B, int H, int W, int Cin,
                            int Cout, int stride, void *stream) {
     if (bad_prec(precision) || !x || !w || !y) return DDG_ERR_INVALID_ARG;

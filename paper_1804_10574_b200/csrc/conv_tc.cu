@@ -1,11 +1,576 @@
-// Tensor-core convolution path (placeholder until the tcgen05 kernels land: nothing is routed here yet).
+// Tensor-core 3x3 convolution for bf16 NHWC tensors on sm_100a: implicit GEMM on tcgen05 with TMEM accumulators,
+// the im2col operand streamed by TMA (one shifted, zero-filled box per filter tap), the filter resident in shared
+// memory for the life of a persistent CTA.
+//
+//   forward  y[p][co]  = sum_{tap,ci} x[p + tap][ci]  * w[co][ci][tap]
+//   dgrad    dx[p][ci] = sum_{tap,co} dy[p + tap][co] * w[co][ci][8 - tap]     (stride 1: the same kernel, filter flipped)
+//
+// One CTA tile is 128 consecutive output pixels (whole image rows) x C channels: per tap one 128 x C x C MMA group
+// (UMMA M=128, N=C, K=16 per instruction), accumulated over the 9 taps in TMEM.  Warp roles: warp 0 issues TMA, warp 1
+// issues MMAs, warps 2-5 drain TMEM, add the shortcut gradient where asked, convert to bf16 and store.  Two TMEM
+// accumulator stages let the epilogue of tile i overlap the MMAs of tile i+1.  Every mbarrier wait is bounded: when
+// one runs out, the CTA raises an error word that the host reads at its next sync point, and leaves.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include "common.cuh"
 #include "conv_tc.h"
 
 namespace ddg {
-bool conv_tc_supported(int, int, int, int, int, int) { return false; }
-int launch_conv_tc(int, const void *, const void *, void *, int, int, int, int, Shortcut, cudaStream_t) { return 0; }
-bool wgrad_tc_supported(int, int, int, int, int, int) { return false; }
-size_t wgrad_tc_scratch_elems() { return 0; }
-int launch_wgrad_tc(const void *, const void *, float *, float *, int, int, int, int, cudaStream_t) { return 0; }
-int conv_tc_init() { return 0; }
+
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kStages = 8;
+constexpr int kTcThreads = 192;
+constexpr unsigned kSpinLimit = 1u << 24;  // bounded waits: ~ a second at worst, then the CTA gives up
+
+__device__ int g_tc_error = 0;  // 0 = fine; otherwise the code of the wait that ran out
+
+// ---- thin PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the error word and the CTA's abort flag) when the limit is hit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code) {
+    for (unsigned i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (i > 4096) __nanosleep(64);
+    }
+    *abort_flag = 1;
+    atomicCAS(&g_tc_error, 0, code);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], "
+        "[%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
+        "[%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major (or MN-major) bf16 tile whose rows are one swizzle span wide
+// (32, 64 or 128 bytes): 8-row groups are `sbo` bytes apart; the leading-dimension field is not used by these
+// layouts and carries its canonical value 1.
+__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout_type,
+                                              uint32_t lbo_bytes = 16) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fff);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+    d |= (uint64_t)layout_type << 61;
+    return d;
+}
+
+template <int C> struct TcCfg {
+    static constexpr int row_bytes = C * 2;                           // one pixel's channels = one swizzle span
+    static constexpr uint32_t layout = C == 64 ? 2u : (C == 32 ? 4u : 6u);  // 128B / 64B / 32B swizzle
+    static constexpr uint32_t swz_mask = C == 64 ? 7u : (C == 32 ? 3u : 1u);
+    static constexpr int w_tap_bytes = C * C * 2;
+    static constexpr int a_stage_bytes = kTileM * C * 2;
+    static constexpr int tmem_cols = (2 * C < 32) ? 32 : 2 * C;       // two accumulator stages, power of two >= 32
+    static constexpr size_t smem_bytes = 2048 + 9 * (size_t)w_tap_bytes + (size_t)kStages * a_stage_bytes + 256;
+};
+
+// byte offset of element (row, k) inside a swizzled tile whose rows are row_bytes wide
+template <int C> __device__ __forceinline__ uint32_t swz_off(int row, int k) {
+    uint32_t off = (uint32_t)row * TcCfg<C>::row_bytes + (uint32_t)k * 2;
+    return off ^ (((off >> 7) & TcCfg<C>::swz_mask) << 4);
+}
+
+template <int C>
+__global__ void __launch_bounds__(kTcThreads, 1)
+conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, bf16 *__restrict__ dst,
+                  int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
+                  const bf16 *__restrict__ res_dout,
+                  const bf16 *__restrict__ res_out) {
+    typedef TcCfg<C> Cfg;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw);
+    const uint32_t w_base = base;
+    const uint32_t a_base = base + 9 * Cfg::w_tap_bytes;  // multiple of 1024 for every C (9*512, 9*2048, 9*8192 -> pad)
+    const uint32_t a_base_al = (a_base + 1023u) & ~1023u;
+    uint8_t *tail = smem + (a_base_al - base) + kStages * Cfg::a_stage_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[kStages], empty[kStages], tfull[2], tempty[2]
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kStages + 4) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kStages + 4) * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {  // TMEM allocation is a whole-warp operation; the same warp frees it at the end
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                     "r"((uint32_t)Cfg::tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // filter -> shared memory, as 9 K-major [C rows = output channel of this pass][C = contraction channel] tiles
+    for (int i = threadIdx.x; i < 9 * C * C; i += kTcThreads) {
+        const int tap = i / (C * C), r = (i / C) % C, k = i % C;
+        const size_t g = dgrad ? ((size_t)(k * C + r) * 9 + (8 - tap)) : ((size_t)(r * C + k) * 9 + tap);
+        *reinterpret_cast<bf16 *>(smem + tap * Cfg::w_tap_bytes + swz_off<C>(r, k)) = w[g];
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    const int tiles_per_img = H / rows_per_tile;  // tiles per image when a tile lies inside one image
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                int n0, h0;
+                if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }  // a tile spans whole images
+                else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
+                for (int tap = 0; tap < 9 && ok; ++tap) {
+                    ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 1);
+                    if (!ok) break;
+                    mbar_expect_tx(full_bar(s), Cfg::a_stage_bytes);
+                    tma_load_4d(a_base_al + s * Cfg::a_stage_bytes, &tmap, full_bar(s), 0, tap % 3 - 1, h0 + tap / 3 - 1, n0);
+                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) {  // let copies already in flight land before the CTA can exit
+                for (int i = 0; i < 2000; ++i) __nanosleep(100);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(C >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            int s = 0;
+            uint32_t ph = 0;
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+                const int a = it & 1;
+                const uint32_t aph = (it >> 1) & 1u;
+                ok = mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * C);
+                for (int tap = 0; tap < 9 && ok; ++tap) {
+                    ok = mbar_wait(full_bar(s), ph, abort_flag, 3);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t adesc = make_desc(a_base_al + s * Cfg::a_stage_bytes, 8 * Cfg::row_bytes, Cfg::layout);
+                    const uint64_t bdesc = make_desc(w_base + tap * Cfg::w_tap_bytes, 8 * Cfg::row_bytes, Cfg::layout);
+#pragma unroll
+                    for (int k = 0; k < C / 16; ++k)  // 16 channels = 32 bytes further along the contraction axis
+                        tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (tap | k) != 0);
+                    tc_commit(empty_bar(s));  // the stage is free once these MMAs have read it
+                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                }
+                if (ok) tc_commit(tfull_bar(a));
+            }
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> registers -> bf16 -> global ----------------
+        const int q = warp & 3;  // a warp may only touch TMEM lanes [32*(warp%4), +32)
+        int it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+            const int a = it & 1;
+            const uint32_t aph = (it >> 1) & 1u;
+            ok = mbar_wait(tfull_bar(a), aph, abort_flag, 4);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            float acc[C];
+#pragma unroll
+            for (int c0 = 0; c0 < C; c0 += 16) {
+                float v[16];
+                tc_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * C + c0), v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) acc[c0 + j] = v[j];
+            }
+            tc_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(a));  // accumulator stage may be overwritten by the next tile but one
+            const size_t pix = (size_t)tile * kTileM + 32 * q + lane;
+            if (res_dout != nullptr) {  // identity-shortcut gradient: + dout * [out > 0]
+#pragma unroll
+                for (int c0 = 0; c0 < C; c0 += 8) {
+                    float d[8], o[8];
+                    load_f<bf16, 8>(res_dout + pix * C + c0, d);
+                    load_f<bf16, 8>(res_out + pix * C + c0, o);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) if (o[j] > 0.f) acc[c0 + j] += d[j];
+                }
+            }
+#pragma unroll
+            for (int c0 = 0; c0 < C; c0 += 8) {
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = acc[c0 + j];
+                store_f<bf16, 8>(dst + pix * C + c0, v);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::tmem_cols)
+                     : "memory");
+    }
+}
+
+
+// ---------------------------------------------------------------------------------------------------------
+// Weight gradient on the tensor cores:  dw[co][ci][ky][kx] = sum_p dy[p][co] * x[p + (ky-1, kx-1)][ci].
+// The contraction runs over pixels, so both operands are used "MN-major": a TMA tile [128 pixels][C channels] is
+// read by the MMA with the channel axis as its M (or N) axis and the pixel axis as K, 16 pixels per instruction.
+// grid = (pixel chunks, 3 filter rows).  A CTA keeps D[co][(kx, ci)] for its filter row in TMEM over all of its
+// pixel tiles, then writes one fp32 partial [3][C][C]; the fold kernel sums the chunks in a fixed order.
+// The MMA shape is M=128 whatever C is: rows >= C of the accumulator are never read (their operand rows alias
+// other rows of the same dy tile).
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kWgStages = 3;
+constexpr int kWgMaxChunks = 49;
+
+template <int C> struct WgCfg {
+    static constexpr int tile_bytes = kTileM * C * 2;
+    static constexpr int stage_bytes = 4 * tile_bytes;               // dy tile + 3 shifted x tiles
+    static constexpr int ncols = 3 * C;
+    static constexpr int tmem_cols = ncols <= 64 ? 64 : (ncols <= 128 ? 128 : 256);
+    static constexpr size_t smem_bytes = 1024 + (size_t)kWgStages * stage_bytes + 256;
+};
+
+template <int C>
+__global__ void __launch_bounds__(kTcThreads, 1)
+wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
+                float *__restrict__ part, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles) {
+    typedef TcCfg<C> Cfg;
+    typedef WgCfg<C> Wg;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *tail = smem_raw + (base - raw) + kWgStages * Wg::stage_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[kWgStages], empty[kWgStages], done
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kWgStages + 1) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kWgStages + 1) * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kWgStages + s); };
+    const uint32_t done_bar = bar0 + 8u * (2 * kWgStages);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ky = blockIdx.y;
+    const int t0 = (int)((long)n_tiles * blockIdx.x / gridDim.x), t1 = (int)((long)n_tiles * (blockIdx.x + 1) / gridDim.x);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kWgStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(done_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                     "r"((uint32_t)Wg::tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    const int tiles_per_img = H / rows_per_tile;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = t0; tile < t1 && ok; ++tile) {
+                int n0, h0;
+                if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }
+                else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
+                ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 11);
+                if (!ok) break;
+                const uint32_t st = base + s * Wg::stage_bytes;
+                mbar_expect_tx(full_bar(s), Wg::stage_bytes);
+                tma_load_4d(st, &tmap_dy, full_bar(s), 0, 0, h0, n0);
+                for (int kx = 0; kx < 3; ++kx)
+                    tma_load_4d(st + (1 + kx) * Wg::tile_bytes, &tmap_x, full_bar(s), 0, kx - 1, h0 + ky - 1, n0);
+                if (++s == kWgStages) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) for (int i = 0; i < 2000; ++i) __nanosleep(100);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // both operands MN-major (bits 15, 16); fp32 accumulate; bf16 inputs; M = 128, N = 3C
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+                                   ((uint32_t)(Wg::ncols >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = t0; tile < t1 && ok; ++tile) {
+                ok = mbar_wait(full_bar(s), ph, abort_flag, 12);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t st = base + s * Wg::stage_bytes;
+#pragma unroll
+                for (int k = 0; k < kTileM / 16; ++k) {
+                    // 16 pixels further along the contraction axis = 16 rows of the tile
+                    const uint32_t koff = (uint32_t)k * 16 * Cfg::row_bytes;
+                    // dy: the M axis walks the C channels of a row, then (rows >= C, ignored) other rows of the same tile
+                    const uint64_t adesc = make_desc(st + koff, 8 * Cfg::row_bytes, Cfg::layout, 2 * C * C);
+                    // x: the N axis walks the C channels, then the next filter column's tile
+                    const uint64_t bdesc = make_desc(st + Wg::tile_bytes + koff, 8 * Cfg::row_bytes, Cfg::layout, Wg::tile_bytes);
+                    tc_mma_bf16(tmem_base, adesc, bdesc, idesc, (tile != t0) || (k != 0));
+                }
+                tc_commit(empty_bar(s));
+                if (++s == kWgStages) { s = 0; ph ^= 1u; }
+            }
+            if (ok) tc_commit(done_bar);
+        }
+    } else {
+        const int q = warp & 3;
+        bool ok = mbar_wait(done_bar, 0, abort_flag, 13);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok && 32 * q < C) {  // only accumulator rows < C carry the result
+            tc_fence_after();
+            const int co = 32 * q + lane;
+            float *out = part + ((size_t)blockIdx.x * 9 + (size_t)ky * 3) * C * C;
+#pragma unroll 1
+            for (int c0 = 0; c0 < Wg::ncols; c0 += 16) {
+                float v[16];
+                tc_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, v);
+                tc_wait_ld();
+                if (co < C) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) out[(size_t)(c0 + j) * C + co] = v[j];  // [(kx, ci)][co]
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Wg::tmem_cols)
+                     : "memory");
+    }
+}
+
+// dw[co][ci][tap] = sum over chunks of part[chunk][tap][ci][co]   (fixed order)
+__global__ void wgrad_tc_fold_kernel(const float *__restrict__ part, float *__restrict__ dw, int chunks, int C) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int total = 9 * C * C;
+    if (i >= total) return;
+    float t = 0.f;
+    for (int c = 0; c < chunks; ++c) t += part[(size_t)c * total + i];
+    const int co = i % C, ci = (i / C) % C, tap = i / (C * C);
+    dw[((size_t)co * C + ci) * 9 + tap] = t;
+}
+
+// ---- host side: tensor maps ------------------------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+
+struct MapKey {
+    const void *ptr; int B, H, W, C;
+    bool operator<(const MapKey &o) const { return std::tie(ptr, B, H, W, C) < std::tie(o.ptr, o.B, o.H, o.W, o.C); }
+};
+std::map<MapKey, CUtensorMap> g_maps;
+std::mutex g_maps_mu;
+
+void tile_geometry(int H, int W, int *rows_per_tile, int *imgs_per_tile) {
+    int r = kTileM / W;
+    if (r > H) r = H;
+    *rows_per_tile = r;
+    *imgs_per_tile = kTileM / (W * r);
+}
+
+// Tensor map of an NHWC bf16 tensor with a box of one 128-pixel tile: (C, W, rows, images), zero fill outside.
+bool get_map(const void *ptr, int B, int H, int W, int C, CUtensorMap *out) {
+    std::lock_guard<std::mutex> lock(g_maps_mu);
+    MapKey key{ptr, B, H, W, C};
+    auto it = g_maps.find(key);
+    if (it != g_maps.end()) { *out = it->second; return true; }
+    int rows, imgs;
+    tile_geometry(H, W, &rows, &imgs);
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)W, (cuuint32_t)rows, (cuuint32_t)imgs};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUtensorMapSwizzle swz = C == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (C == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    CUtensorMap m;
+    CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return false;
+    if (g_maps.size() > 4096) g_maps.clear();
+    g_maps[key] = m;
+    *out = m;
+    return true;
+}
+
+int g_num_sms = 148;
+
+template <int C>
+int launch_tc(int dir, const void *src, const void *w, void *dst, int B, int H, int W, Shortcut sc, cudaStream_t s) {
+    CUtensorMap map;
+    if (!get_map(src, B, H, W, C, &map)) return -1;
+    int rows, imgs;
+    tile_geometry(H, W, &rows, &imgs);
+    const int n_tiles = (int)((long)B * H * W / kTileM);
+    const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
+    conv3x3_tc_kernel<C><<<grid, kTcThreads, TcCfg<C>::smem_bytes, s>>>(
+        map, (const bf16 *)w, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, sc.mode == 1 ? (const bf16 *)sc.a : nullptr,
+        sc.mode == 1 ? (const bf16 *)sc.b : nullptr);
+    return 1;
+}
+
+}  // namespace
+
+bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
+    if (!g_encode) return false;
+    if (stride != 1 || Cin != Cout || (Cin != 16 && Cin != 32 && Cin != 64)) return false;
+    if (W > kTileM || kTileM % W != 0) return false;
+    const int r = kTileM / W;
+    if (r <= H) { if (H % r != 0) return false; }
+    else { if (kTileM % (H * W) != 0 || B % (kTileM / (H * W)) != 0) return false; }
+    return ((long)B * H * W) % kTileM == 0;
+}
+
+int launch_conv_tc(int dir, const void *src, const void *w, void *dst, int B, int H, int W, int C, Shortcut sc,
+                   cudaStream_t s) {
+    switch (C) {
+    case 16: return launch_tc<16>(dir, src, w, dst, B, H, W, sc, s);
+    case 32: return launch_tc<32>(dir, src, w, dst, B, H, W, sc, s);
+    case 64: return launch_tc<64>(dir, src, w, dst, B, H, W, sc, s);
+    }
+    return -1;
+}
+
+bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
+    return conv_tc_supported(B, H, W, Cin, Cout, stride);
+}
+size_t wgrad_tc_scratch_elems() { return (size_t)kWgMaxChunks * 9 * 64 * 64; }
+
+namespace {
+template <int C>
+int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, cudaStream_t s) {
+    CUtensorMap mx, md;
+    if (!get_map(x, B, H, W, C, &mx) || !get_map(dy, B, H, W, C, &md)) return -1;
+    int rows, imgs;
+    tile_geometry(H, W, &rows, &imgs);
+    const int n_tiles = (int)((long)B * H * W / kTileM);
+    const int chunks = n_tiles < kWgMaxChunks ? n_tiles : kWgMaxChunks;
+    wgrad_tc_kernel<C><<<dim3(chunks, 3), kTcThreads, WgCfg<C>::smem_bytes, s>>>(mx, md, scratch, H, W, rows, imgs, n_tiles);
+    wgrad_tc_fold_kernel<<<ceil_div(9 * C * C, 256), 256, 0, s>>>(scratch, dw, chunks, C);
+    return 2;
+}
+}  // namespace
+
+int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C,
+                    cudaStream_t s) {
+    switch (C) {
+    case 16: return launch_wg<16>(x, dy, dw, scratch, B, H, W, s);
+    case 32: return launch_wg<32>(x, dy, dw, scratch, B, H, W, s);
+    case 64: return launch_wg<64>(x, dy, dw, scratch, B, H, W, s);
+    }
+    return -1;
+}
+
+int conv_tc_error() {
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int)) != cudaSuccess) return -1;
+    return v;
+}
+
+int conv_tc_init() {
+    static int rc = -1;
+    if (rc >= 0) return rc;
+    cudaDriverEntryPointQueryResult q;
+    void *fn = nullptr;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) { cudaGetLastError(); rc = 0; return rc; }  // path stays off
+    g_encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+    e = cudaFuncSetAttribute(conv3x3_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<16>::smem_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<32>::smem_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<64>::smem_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wgrad_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WgCfg<16>::smem_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wgrad_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WgCfg<32>::smem_bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(wgrad_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WgCfg<64>::smem_bytes);
+    rc = (int)e;
+    return rc;
+}
+
 }  // namespace ddg

@@ -22,6 +22,8 @@ int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, in
 
 // One-time per-process set-up (function attributes, driver entry points).  Returns a cudaError_t value.
 int conv_tc_init();
+// Error word raised by a tensor-core kernel whose bounded wait ran out (0 = none, -1 = cannot be read).
+int conv_tc_error();
 int conv_direct_init();
 
 }  // namespace ddg

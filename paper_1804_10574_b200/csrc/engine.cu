@@ -420,6 +420,14 @@ ddg_status init_weights(ddg_ctx *ctx) {
 
 ddg_status sync_all(ddg_ctx *ctx) {
     for (auto &m : ctx->mods) CU(cudaStreamSynchronize(m.stream));
+    if (ctx->prec == P_BF16) {
+        const int code = conv_tc_error();
+        if (code != 0) {
+            set_err(ctx, "a tensor-core kernel gave up on a bounded wait (code %d)", code);
+            ctx->broken = true;
+            return code > 0 ? DDG_ERR_TIMEOUT : DDG_ERR_CUDA;
+        }
+    }
     return DDG_OK;
 }
 

@@ -61,7 +61,8 @@ def test_conv3x3_fwd_dgrad_wgrad(shape, prec):
     dx_ref, dw_ref = orc.conv3x3_backward(xh, wh, dyh, st)
     assert rel(from_dev(y), y_ref) < TOL[prec]
     assert rel(from_dev(dx), dx_ref) < TOL[prec]
-    assert rel(dw.cpu().numpy(), dw_ref) < 1e-5   # fp32 output from exact inputs in both precisions
+    # fp32 output from exact inputs in both precisions; the tensor-core path accumulates in fp32 over all pixels
+    assert rel(dw.cpu().numpy(), dw_ref) < (2e-4 if prec and binding.tensor_core_path(B, H, W, Ci, Co, st) & 2 else 1e-5)
     # a second call on the same scratch gives the same bits (fixed summation order)
     dw2 = torch.empty_like(dw)
     binding.conv3x3_wgrad(prec, x, dy, dw2, scratch, B, H, W, Ci, Co, st)
@@ -120,3 +121,11 @@ def test_sgd_update(n, prec):
     w_ref = w - 0.1 * v_ref
     assert rel(vd.cpu().numpy(), v_ref) < 1e-6 and rel(wd.cpu().numpy(), w_ref) < 1e-6
     assert torch.equal(wv, wd.to(tdtype(prec)))      # the version slot is the cast of the new master weights
+
+
+def test_tensor_core_path_takes_the_resnet_shapes():
+    from paper_1804_10574_b200 import binding
+    for B, H, W, C in [(128, 32, 32, 16), (128, 16, 16, 32), (128, 8, 8, 64), (2, 8, 8, 16), (3, 32, 32, 16)]:
+        assert binding.tensor_core_path(B, H, W, C, C, 1) & 1, (B, H, W, C)
+    assert binding.tensor_core_path(128, 32, 32, 16, 32, 2) & 1 == 0      # stride 2 stays on CUDA cores
+    assert binding.tensor_core_path(9, 8, 8, 64, 64, 1) & 1 == 0          # 576 pixels: not whole 128-pixel tiles
