@@ -165,6 +165,19 @@ ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float
 size_t ddg_bn_scratch_elems(int C);
 ddg_status ddg_bn_fwd(int precision, const void *x, const void *gamma, const void *beta, const void *res, void *y,
                       float *mean, float *invstd, float *scratch, int B, int HW, int C, int relu, void *stream);
+/* The same operation as ddg_bn_fwd without the scratch argument, for callers that cannot allocate device memory
+ * (code running inside someone else's memory pool, latency-critical loops that must avoid cudaMalloc's implicit
+ * synchronisation, processes whose device memory is budgeted up front).  The paper has no counterpart: this is a
+ * deployment convenience.  The scratch lives in a fixed array inside the library image (about 592 KiB per GPU that
+ * loads the library, held until the process exits), which limits the call to C <= 64; larger C returns
+ * DDG_ERR_UNSUPPORTED with a message in ddg_last_error(NULL).  The call itself allocates nothing (no cudaMalloc,
+ * cudaFree or allocating library routine).  The first call on each device looks up the array's device address
+ * (with that device current): make that first call before any stream capture.  All calls share the one array and
+ * it keeps the previous call's contents (the call clears the part that must start at zero), so two calls that
+ * overlap on the GPU - different streams, or the same call from two threads - race; serialise them. */
+ddg_status ddg_bn_fwd_noalloc(int precision, const void *x, const void *gamma, const void *beta, const void *res,
+                              void *y, float *mean, float *invstd, int B, int HW, int C, int relu, void *stream);
+
 /* Batch-norm backward: dz = dout * [out > 0] when relu != 0 (out = forward output), else dout;
  * dgamma = sum dz*xhat, dbeta = sum dz, dx = gamma*invstd*(dz - dbeta/n - xhat*dgamma/n). */
 ddg_status ddg_bn_bwd(int precision, const void *dout, const void *out, const void *x, const void *gamma,

@@ -26,7 +26,7 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_set_weights", "ddg_get_grads", "ddg_get_loss_dev", "ddg_last_step_launches", "ddg_sync",
            "ddg_last_error", "ddg_destroy", "ddg_conv3x3_fwd", "ddg_conv3x3_dgrad",
            "ddg_conv3x3_wgrad_scratch_elems", "ddg_conv3x3_wgrad", "ddg_bn_scratch_elems", "ddg_bn_fwd", "ddg_bn_bwd",
-           "ddg_sgd_update", "ddg_tensor_core_path"]
+           "ddg_sgd_update", "ddg_tensor_core_path", "ddg_bn_fwd_noalloc"]
 
 
 class Layer(ctypes.Structure):
@@ -72,6 +72,7 @@ _lib.ddg_bn_scratch_elems.restype = _sz
 _lib.ddg_bn_fwd.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_bn_bwd.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_tensor_core_path.argtypes = [_i] * 6
+_lib.ddg_bn_fwd_noalloc.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_sgd_update.argtypes = [_i, _vp, _vp, _vp, _vp, _sz, _f, _f, _f, _vp]
 
 
@@ -211,6 +212,12 @@ def bn_scratch_elems(C):
 def bn_fwd(prec, x, gamma, beta, res, y, mean, invstd, scratch, B, HW, C, relu, stream=None):
     _ok(_lib.ddg_bn_fwd(prec, _ptr(x), _ptr(gamma), _ptr(beta), _ptr(res), _ptr(y), _ptr(mean), _ptr(invstd),
                         _ptr(scratch), B, HW, C, int(relu), stream))
+
+
+def bn_fwd_noalloc(prec, x, gamma, beta, res, y, mean, invstd, B, HW, C, relu, stream=None):
+    """ddg_bn_fwd with the scratch inside the library (C <= 64): allocates nothing.  Returns the status code."""
+    return _lib.ddg_bn_fwd_noalloc(prec, _ptr(x), _ptr(gamma), _ptr(beta), _ptr(res), _ptr(y), _ptr(mean),
+                                   _ptr(invstd), B, HW, C, int(relu), stream)
 
 
 def bn_bwd(prec, dout, out, x, gamma, mean, invstd, dx, dgamma, dbeta, scratch, B, HW, C, relu, stream=None):

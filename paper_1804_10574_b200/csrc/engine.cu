@@ -433,6 +433,11 @@ ddg_status sync_all(ddg_ctx *ctx) {
 
 }  // namespace
 
+namespace ddg {
+// lets the other translation units leave a message for ddg_last_error(NULL)
+void set_global_error(const char *msg) { g_create_error = msg; }
+}  // namespace ddg
+
 // ========================================================================================================
 // C ABI
 // ========================================================================================================
