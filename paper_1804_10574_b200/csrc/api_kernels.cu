@@ -34,7 +34,7 @@ ddg_status ddg_conv3x3_fwd(int precision, const void *x, const void *w, void *y,
     if (init_once() != DDG_OK) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     if (precision == DDG_BF16 && conv_tc_supported(B, H, W, Cin, Cout, stride))
-        launch_conv_tc(0, x, w, y, B, H, W, Cin, Shortcut{}, s);
+        launch_conv_tc(0, x, w, nullptr, y, B, H, W, Cin, Shortcut{}, s);
     else
         launch_conv_fwd_direct(precision, x, w, y, B, H, W, Cin, Cout, stride, 0, s);
     return done();
@@ -47,7 +47,7 @@ ddg_status ddg_conv3x3_dgrad(int precision, const void *dy, const void *w, void 
     if (init_once() != DDG_OK) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     if (precision == DDG_BF16 && conv_tc_supported(B, H, W, Cin, Cout, stride))
-        launch_conv_tc(1, dy, w, dx, B, H, W, Cin, Shortcut{}, s);
+        launch_conv_tc(1, dy, w, nullptr, dx, B, H, W, Cin, Shortcut{}, s);
     else
         launch_conv_dgrad_direct(precision, dy, w, dx, B, H, W, Cin, Cout, stride, Shortcut{}, s);
     return done();

@@ -5,11 +5,17 @@
 //   forward  y[p][co]  = sum_{tap,ci} x[p + tap][ci]  * w[co][ci][tap]
 //   dgrad    dx[p][ci] = sum_{tap,co} dy[p + tap][co] * w[co][ci][8 - tap]     (stride 1: the same kernel, filter flipped)
 //
-// One CTA tile is 128 consecutive output pixels (whole image rows) x C channels: per tap one 128 x C x C MMA group
-// (UMMA M=128, N=C, K=16 per instruction), accumulated over the 9 taps in TMEM.  Warp roles: warp 0 issues TMA, warp 1
-// issues MMAs, warps 2-5 drain TMEM, add the shortcut gradient where asked, convert to bf16 and store.  Two TMEM
-// accumulator stages let the epilogue of tile i overlap the MMAs of tile i+1.  Every mbarrier wait is bounded: when
-// one runs out, the CTA raises an error word that the host reads at its next sync point, and leaves.
+// One CTA tile is 128 consecutive output pixels (whole image rows) x C channels.  The input rows are loaded ONCE per
+// tile, unshifted in the column direction: the MMAs produce, per filter column kx, the partial result
+// P_kx[p][co] = sum_{ky,ci} x[p + (ky-1) rows][ci] * w[co][ci][ky][kx] at the INPUT column (UMMA M=128, N=3C, K=16 per
+// instruction, the three filter columns stacked along N), and the epilogue adds the three partials across
+// neighbouring pixels, y[h][w] = P_0[h][w-1] + P_1[h][w] + P_2[h][w+1], with warp shuffles (a warp holds whole image
+// rows; the image border contributes zero).  The filter-row shift costs nothing: the three rows read the same TMA box
+// at offsets of 0, W and 2W pixels, which are whole swizzle periods, so only the descriptor start address moves.
+// Warp roles: warp 0 issues TMA, warp 1 issues MMAs, warps 2-5 drain TMEM, combine, add the shortcut gradient where
+// asked, convert to bf16 and store.  Two TMEM accumulator stages let the epilogue of tile i overlap the MMAs of tile
+// i+1.  Every mbarrier wait is bounded: when one runs out, the CTA raises an error word that the host reads at its
+// next sync point, and leaves.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
@@ -25,7 +31,6 @@ namespace ddg {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kStages = 8;
 constexpr int kTcThreads = 192;
 constexpr unsigned kSpinLimit = 1u << 24;  // bounded waits: ~ a second at worst, then the CTA gives up
 
@@ -117,51 +122,115 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t sbo_bytes,
     return d;
 }
 
+constexpr int kMaxStages = 16;
+
 template <int C> struct TcCfg {
     static constexpr int row_bytes = C * 2;                           // one pixel's channels = one swizzle span
     static constexpr uint32_t layout = C == 64 ? 2u : (C == 32 ? 4u : 6u);  // 128B / 64B / 32B swizzle
     static constexpr uint32_t swz_mask = C == 64 ? 7u : (C == 32 ? 3u : 1u);
-    static constexpr int w_tap_bytes = C * C * 2;
-    static constexpr int a_stage_bytes = kTileM * C * 2;
-    static constexpr int tmem_cols = (2 * C < 32) ? 32 : 2 * C;       // two accumulator stages, power of two >= 32
-    static constexpr size_t smem_bytes = 2048 + 9 * (size_t)w_tap_bytes + (size_t)kStages * a_stage_bytes + 256;
+    static constexpr int w_row_tile_bytes = 3 * C * C * 2;            // one filter row: [3C rows = (kx, out ch)][C]
+    static constexpr int w_bytes = 3 * w_row_tile_bytes;
+    static constexpr int tile_bytes = kTileM * C * 2;
+    static constexpr int tmem_cols = C == 16 ? 128 : (C == 32 ? 256 : 512);  // two stages of 3C columns, power of two
 };
 
 // byte offset of element (row, k) inside a swizzled tile whose rows are row_bytes wide
-template <int C> __device__ __forceinline__ uint32_t swz_off(int row, int k) {
+template <int C> __host__ __device__ __forceinline__ uint32_t swz_off(int row, int k) {
     uint32_t off = (uint32_t)row * TcCfg<C>::row_bytes + (uint32_t)k * 2;
     return off ^ (((off >> 7) & TcCfg<C>::swz_mask) << 4);
 }
 
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// Shared-memory plan of the convolution kernel (all offsets from a 1024-byte aligned base).
+struct ConvSmem {
+    uint32_t w_off, a_off, tail_off;
+};
+template <int C> __host__ __device__ inline ConvSmem conv_smem_plan(int n_stages, int stage_bytes) {
+    ConvSmem p;
+    p.w_off = 0;
+    p.a_off = (TcCfg<C>::w_bytes + 1023u) & ~1023u;
+    p.tail_off = p.a_off + (uint32_t)n_stages * (uint32_t)stage_bytes;
+    return p;
+}
+template <int C> inline size_t conv_smem_bytes(int n_stages, int stage_bytes) {
+    return 1024 + conv_smem_plan<C>(n_stages, stage_bytes).tail_off + 512;
+}
+
+// Filter images for the tensor-core kernels: per convolution two blocks of 3 swizzled K-major [3C][C] bf16 tiles (one
+// per filter row; rows = filter column x channel of this pass, k = contraction channel): the forward one (row =
+// output channel, k = input channel) and the input-gradient one (row = input channel, k = output channel, taps
+// flipped).  One thread per (tap, row, k).
+struct PackJob { long src_off; long dst_off; int C; int first_elem; };
+
+// image element (tap = ky*3+kx, row r, k): filter row tile ky, row kx*C + r of that tile
+template <int C> __device__ __forceinline__ uint32_t w_img_off(int tap, int r, int k) {
+    return (uint32_t)(tap / 3) * TcCfg<C>::w_row_tile_bytes + swz_off<C>((tap % 3) * C + r, k);
+}
+template <int C> __device__ __forceinline__ void pack_one(const bf16 *w, uint8_t *dst, int i) {
+    const int tap = i / (C * C), r = (i / C) % C, k = i % C;
+    const uint32_t o = w_img_off<C>(tap, r, k);
+    *reinterpret_cast<bf16 *>(dst + o) = w[(size_t)(r * C + k) * 9 + tap];
+    *reinterpret_cast<bf16 *>(dst + TcCfg<C>::w_bytes + o) = w[(size_t)(k * C + r) * 9 + (8 - tap)];
+}
+
+__global__ void pack_filters_kernel(const bf16 *__restrict__ wver, uint8_t *__restrict__ packed,
+                                    const PackJob *__restrict__ jobs, int n_jobs, int total) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    int lo = 0, hi = n_jobs - 1;  // last job whose first element is <= e
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (jobs[mid].first_elem <= e) lo = mid; else hi = mid - 1;
+    }
+    const PackJob j = jobs[lo];
+    const int i = e - j.first_elem;
+    if (j.C == 16) pack_one<16>(wver + j.src_off, packed + j.dst_off, i);
+    else if (j.C == 32) pack_one<32>(wver + j.src_off, packed + j.dst_off, i);
+    else pack_one<64>(wver + j.src_off, packed + j.dst_off, i);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// forward / input gradient.
+//   slab == 1 (tile inside one image): one TMA box of (rows+2) image rows per tile; filter row ky reads it at an offset
+//              of ky*W pixels.
+//   slab == 0 (tile = several whole small images): one TMA box of the tile shifted by ky-1 rows per filter row (3 per
+//              tile), zero-filled at the image border.
+// ---------------------------------------------------------------------------------------------------------
 template <int C>
 __global__ void __launch_bounds__(kTcThreads, 1)
-conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, bf16 *__restrict__ dst,
-                  int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
-                  const bf16 *__restrict__ res_dout,
+conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
+                  bf16 *__restrict__ dst, int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
+                  int slab, int n_stages, int stage_bytes, const bf16 *__restrict__ res_dout,
                   const bf16 *__restrict__ res_out) {
     typedef TcCfg<C> Cfg;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *smem = smem_raw + (base - raw);
-    const uint32_t w_base = base;
-    const uint32_t a_base = base + 9 * Cfg::w_tap_bytes;  // multiple of 1024 for every C (9*512, 9*2048, 9*8192 -> pad)
-    const uint32_t a_base_al = (a_base + 1023u) & ~1023u;
-    uint8_t *tail = smem + (a_base_al - base) + kStages * Cfg::a_stage_bytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[kStages], empty[kStages], tfull[2], tempty[2]
-    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kStages + 4) * 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kStages + 4) * 8 + 8);
+    const ConvSmem plan = conv_smem_plan<C>(n_stages, stage_bytes);
+    const uint32_t w_base = base + plan.w_off, a_base = base + plan.a_off;
+    uint8_t *tail = smem + plan.tail_off;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[2], tempty[2], wbar
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 5) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 5) * 8 + 8);
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
-    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
-    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
+    const uint32_t w_bar = bar0 + 8u * (2 * kMaxStages + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        mbar_init(w_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -171,22 +240,29 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // filter -> shared memory, as 9 K-major [C rows = output channel of this pass][C = contraction channel] tiles
-    for (int i = threadIdx.x; i < 9 * C * C; i += kTcThreads) {
-        const int tap = i / (C * C), r = (i / C) % C, k = i % C;
-        const size_t g = dgrad ? ((size_t)(k * C + r) * 9 + (8 - tap)) : ((size_t)(r * C + k) * 9 + tap);
-        *reinterpret_cast<bf16 *>(smem + tap * Cfg::w_tap_bytes + swz_off<C>(r, k)) = w[g];
+    if (w_packed == nullptr) {
+        // filter in canonical order: stage it here as 9 K-major [C rows = output channel of this pass][C] tiles
+        for (int i = threadIdx.x; i < 9 * C * C; i += kTcThreads) {
+            const int tap = i / (C * C), r = (i / C) % C, k = i % C;
+            const size_t g = dgrad ? ((size_t)(k * C + r) * 9 + (8 - tap)) : ((size_t)(r * C + k) * 9 + tap);
+            *reinterpret_cast<bf16 *>(smem + plan.w_off + w_img_off<C>(tap, r, k)) = w[g];
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-
     const int tiles_per_img = H / rows_per_tile;  // tiles per image when a tile lies inside one image
+    const int loads_per_tile = slab ? 1 : 3;
+
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
+            if (w_packed != nullptr) {  // pre-arranged filter image: one bulk copy
+                mbar_expect_tx(w_bar, Cfg::w_bytes);
+                bulk_copy_g2s(w_base, w_packed + (dgrad ? Cfg::w_bytes : 0), Cfg::w_bytes, w_bar);
+            }
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -194,12 +270,12 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                 int n0, h0;
                 if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }  // a tile spans whole images
                 else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
-                for (int tap = 0; tap < 9 && ok; ++tap) {
+                for (int j = 0; j < loads_per_tile && ok; ++j) {
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 1);
                     if (!ok) break;
-                    mbar_expect_tx(full_bar(s), Cfg::a_stage_bytes);
-                    tma_load_4d(a_base_al + s * Cfg::a_stage_bytes, &tmap, full_bar(s), 0, tap % 3 - 1, h0 + tap / 3 - 1, n0);
-                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                    mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
+                    tma_load_4d(a_base + s * stage_bytes, &tmap, full_bar(s), 0, 0, slab ? h0 - 1 : h0 + j - 1, n0);
+                    if (++s == n_stages) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {  // let copies already in flight land before the CTA can exit
@@ -209,29 +285,35 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(C >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((3 * C) >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
             int s = 0;
             uint32_t ph = 0;
             int it = 0;
             bool ok = true;
+            if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, abort_flag, 5);
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
                 const int a = it & 1;
                 const uint32_t aph = (it >> 1) & 1u;
                 ok = mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, 2);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(a * C);
-                for (int tap = 0; tap < 9 && ok; ++tap) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * 3 * C);
+                for (int j = 0; j < loads_per_tile && ok; ++j) {
                     ok = mbar_wait(full_bar(s), ph, abort_flag, 3);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t adesc = make_desc(a_base_al + s * Cfg::a_stage_bytes, 8 * Cfg::row_bytes, Cfg::layout);
-                    const uint64_t bdesc = make_desc(w_base + tap * Cfg::w_tap_bytes, 8 * Cfg::row_bytes, Cfg::layout);
+                    const uint32_t a_addr = a_base + s * stage_bytes;
+                    const int n_sub = slab ? 3 : 1;
+                    for (int i = 0; i < n_sub; ++i) {
+                        const int ky = slab ? i : j;
+                        const uint64_t adesc = make_desc(a_addr + (uint32_t)(i * W) * Cfg::row_bytes, 8 * Cfg::row_bytes, Cfg::layout);
+                        const uint64_t bdesc = make_desc(w_base + ky * Cfg::w_row_tile_bytes, 8 * Cfg::row_bytes, Cfg::layout);
 #pragma unroll
-                    for (int k = 0; k < C / 16; ++k)  // 16 channels = 32 bytes further along the contraction axis
-                        tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (tap | k) != 0);
+                        for (int k = 0; k < C / 16; ++k)  // 16 channels = 32 bytes further along the contraction axis
+                            tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (ky | k) != 0);
+                    }
                     tc_commit(empty_bar(s));  // the stage is free once these MMAs have read it
-                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                    if (++s == n_stages) { s = 0; ph ^= 1u; }
                 }
                 if (ok) tc_commit(tfull_bar(a));
             }
@@ -248,35 +330,45 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            float acc[C];
-#pragma unroll
-            for (int c0 = 0; c0 < C; c0 += 16) {
-                float v[16];
-                tc_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * C + c0), v);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) acc[c0 + j] = v[j];
-            }
-            tc_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(a));  // accumulator stage may be overwritten by the next tile but one
             const size_t pix = (size_t)tile * kTileM + 32 * q + lane;
-            if (res_dout != nullptr) {  // identity-shortcut gradient: + dout * [out > 0]
-#pragma unroll
-                for (int c0 = 0; c0 < C; c0 += 8) {
-                    float d[8], o[8];
-                    load_f<bf16, 8>(res_dout + pix * C + c0, d);
-                    load_f<bf16, 8>(res_out + pix * C + c0, o);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) if (o[j] > 0.f) acc[c0 + j] += d[j];
+            const int wcol = lane % W;  // W divides 32: a warp holds whole image rows
+            const uint32_t t_row = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * 3 * C);
+#pragma unroll 1
+            for (int c0 = 0; c0 < C; c0 += 16) {
+                float p0[16], p1[16], p2[16];
+                tc_ld16(t_row + (uint32_t)c0, p0);            // filter column 0: belongs to the pixel on the right
+                tc_ld16(t_row + (uint32_t)(C + c0), p1);
+                tc_ld16(t_row + (uint32_t)(2 * C + c0), p2);  // filter column 2: belongs to the pixel on the left
+                tc_wait_ld();
+                if (c0 + 16 >= C) {  // last read of this accumulator stage: hand it back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(a));
                 }
-            }
+                float acc[16];
 #pragma unroll
-            for (int c0 = 0; c0 < C; c0 += 8) {
-                float v[8];
+                for (int j = 0; j < 16; ++j) {
+                    const float left = __shfl_up_sync(0xffffffffu, p0[j], 1);
+                    const float right = __shfl_down_sync(0xffffffffu, p2[j], 1);
+                    acc[j] = p1[j] + (wcol > 0 ? left : 0.f) + (wcol < W - 1 ? right : 0.f);
+                }
+                if (res_dout != nullptr) {  // identity-shortcut gradient: + dout * [out > 0]
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = acc[c0 + j];
-                store_f<bf16, 8>(dst + pix * C + c0, v);
+                    for (int h = 0; h < 16; h += 8) {
+                        float d[8], o[8];
+                        load_f<bf16, 8>(res_dout + pix * C + c0 + h, d);
+                        load_f<bf16, 8>(res_out + pix * C + c0 + h, o);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) if (o[j] > 0.f) acc[h + j] += d[j];
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < 16; h += 8) {
+                    float v[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[j] = acc[h + j];
+                    store_f<bf16, 8>(dst + pix * C + c0 + h, v);
+                }
             }
         }
     }
@@ -289,57 +381,55 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     }
 }
 
-
 // ---------------------------------------------------------------------------------------------------------
 // Weight gradient on the tensor cores:  dw[co][ci][ky][kx] = sum_p dy[p][co] * x[p + (ky-1, kx-1)][ci].
-// The contraction runs over pixels, so both operands are used "MN-major": a TMA tile [128 pixels][C channels] is
-// read by the MMA with the channel axis as its M (or N) axis and the pixel axis as K, 16 pixels per instruction.
-// grid = (pixel chunks, 3 filter rows).  A CTA keeps D[co][(kx, ci)] for its filter row in TMEM over all of its
-// pixel tiles, then writes one fp32 partial [3][C][C]; the fold kernel sums the chunks in a fixed order.
-// The MMA shape is M=128 whatever C is: rows >= C of the accumulator are never read (their operand rows alias
-// other rows of the same dy tile).
+// The contraction runs over pixels, so both operands are used "MN-major": a TMA tile [pixels][C channels] is read by
+// the MMA with the channel axis as its M (or N) axis and the pixel axis as K, 16 pixels per instruction.  The MMA
+// shape is M=128 whatever C is: rows >= C of the accumulator are never read (their operand rows alias other rows of
+// the same dy tile).  N = 3C: three filter taps stacked through the descriptor's leading-dimension offset.
+//   slab == 0: grid (pixel chunks, 3 filter rows); per tile the dy box and three shifted x boxes (one per filter
+//              column); the three stacked taps are the filter columns.  TMEM holds D[co][(kx, ci)].
+//   slab == 1: grid (pixel chunks, 1); per tile the dy box and three x boxes of (rows+2) image rows (one per filter
+//              column); the three stacked taps are the filter rows (row offsets 0, W, 2W pixels inside the box).  TMEM
+//              holds all nine taps D[co][(kx, ky, ci)].
+// A CTA accumulates over all of its pixel tiles in TMEM, then writes one fp32 partial; the fold kernel sums the chunks
+// in a fixed order.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int kWgStages = 3;
-constexpr int kWgMaxChunks = 49;
+constexpr int kWgMaxChunks = 148;
 
-template <int C> struct WgCfg {
-    static constexpr int tile_bytes = kTileM * C * 2;
-    static constexpr int stage_bytes = 4 * tile_bytes;               // dy tile + 3 shifted x tiles
-    static constexpr int ncols = 3 * C;
-    static constexpr int tmem_cols = ncols <= 64 ? 64 : (ncols <= 128 ? 128 : 256);
-    static constexpr size_t smem_bytes = 1024 + (size_t)kWgStages * stage_bytes + 256;
-};
+struct WgSmem { uint32_t tail_off; };
 
 template <int C>
 __global__ void __launch_bounds__(kTcThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
-                float *__restrict__ part, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles) {
+                float *__restrict__ part, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles, int slab,
+                int n_stages, int x_box_bytes, int tmem_cols) {
     typedef TcCfg<C> Cfg;
-    typedef WgCfg<C> Wg;
+    const int stage_bytes = Cfg::tile_bytes + 3 * x_box_bytes;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t *tail = smem_raw + (base - raw) + kWgStages * Wg::stage_bytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[kWgStages], empty[kWgStages], done
-    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kWgStages + 1) * 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kWgStages + 1) * 8 + 8);
+    uint8_t *tail = smem_raw + (base - raw) + (size_t)n_stages * stage_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], done
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 1) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 1) * 8 + 8);
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (kWgStages + s); };
-    const uint32_t done_bar = bar0 + 8u * (2 * kWgStages);
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+    const uint32_t done_bar = bar0 + 8u * (2 * kMaxStages);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ky = blockIdx.y;
+    const int ky_cta = blockIdx.y;
     const int t0 = (int)((long)n_tiles * blockIdx.x / gridDim.x), t1 = (int)((long)n_tiles * (blockIdx.x + 1) / gridDim.x);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kWgStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(done_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
-                     "r"((uint32_t)Wg::tmem_cols)
+                     "r"((uint32_t)tmem_cols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -360,12 +450,13 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
                 ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 11);
                 if (!ok) break;
-                const uint32_t st = base + s * Wg::stage_bytes;
-                mbar_expect_tx(full_bar(s), Wg::stage_bytes);
+                const uint32_t st = base + s * stage_bytes;
+                mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
                 tma_load_4d(st, &tmap_dy, full_bar(s), 0, 0, h0, n0);
                 for (int kx = 0; kx < 3; ++kx)
-                    tma_load_4d(st + (1 + kx) * Wg::tile_bytes, &tmap_x, full_bar(s), 0, kx - 1, h0 + ky - 1, n0);
-                if (++s == kWgStages) { s = 0; ph ^= 1u; }
+                    tma_load_4d(st + Cfg::tile_bytes + kx * x_box_bytes, &tmap_x, full_bar(s), 0, kx - 1,
+                                slab ? h0 - 1 : h0 + ky_cta - 1, n0);
+                if (++s == n_stages) { s = 0; ph ^= 1u; }
             }
             if (!ok) for (int i = 0; i < 2000; ++i) __nanosleep(100);
         }
@@ -373,7 +464,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         if (lane == 0) {
             // both operands MN-major (bits 15, 16); fp32 accumulate; bf16 inputs; M = 128, N = 3C
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
-                                   ((uint32_t)(Wg::ncols >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+                                   ((uint32_t)((3 * C) >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -381,19 +472,33 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 ok = mbar_wait(full_bar(s), ph, abort_flag, 12);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t st = base + s * Wg::stage_bytes;
+                const uint32_t st = base + s * stage_bytes;
+                if (slab) {
+                    for (int kx = 0; kx < 3; ++kx) {
 #pragma unroll
-                for (int k = 0; k < kTileM / 16; ++k) {
-                    // 16 pixels further along the contraction axis = 16 rows of the tile
-                    const uint32_t koff = (uint32_t)k * 16 * Cfg::row_bytes;
-                    // dy: the M axis walks the C channels of a row, then (rows >= C, ignored) other rows of the same tile
-                    const uint64_t adesc = make_desc(st + koff, 8 * Cfg::row_bytes, Cfg::layout, 2 * C * C);
-                    // x: the N axis walks the C channels, then the next filter column's tile
-                    const uint64_t bdesc = make_desc(st + Wg::tile_bytes + koff, 8 * Cfg::row_bytes, Cfg::layout, Wg::tile_bytes);
-                    tc_mma_bf16(tmem_base, adesc, bdesc, idesc, (tile != t0) || (k != 0));
+                        for (int k = 0; k < kTileM / 16; ++k) {
+                            const uint32_t koff = (uint32_t)k * 16 * Cfg::row_bytes;  // 16 pixels along the contraction axis
+                            const uint64_t adesc = make_desc(st + koff, 8 * Cfg::row_bytes, Cfg::layout, 2 * C * C);
+                            // N walks the C channels, then the next filter row: W pixels further down the same box
+                            const uint64_t bdesc = make_desc(st + Cfg::tile_bytes + kx * x_box_bytes + koff, 8 * Cfg::row_bytes,
+                                                             Cfg::layout, (uint32_t)W * Cfg::row_bytes);
+                            tc_mma_bf16(tmem_base + (uint32_t)(kx * 3 * C), adesc, bdesc, idesc, (tile != t0) || (k != 0));
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < kTileM / 16; ++k) {
+                        const uint32_t koff = (uint32_t)k * 16 * Cfg::row_bytes;
+                        // dy: M walks the C channels of a row, then (rows >= C, ignored) other rows of the same tile
+                        const uint64_t adesc = make_desc(st + koff, 8 * Cfg::row_bytes, Cfg::layout, 2 * C * C);
+                        // x: N walks the C channels, then the next filter column's box
+                        const uint64_t bdesc = make_desc(st + Cfg::tile_bytes + koff, 8 * Cfg::row_bytes, Cfg::layout,
+                                                         (uint32_t)x_box_bytes);
+                        tc_mma_bf16(tmem_base, adesc, bdesc, idesc, (tile != t0) || (k != 0));
+                    }
                 }
                 tc_commit(empty_bar(s));
-                if (++s == kWgStages) { s = 0; ph ^= 1u; }
+                if (++s == n_stages) { s = 0; ph ^= 1u; }
             }
             if (ok) tc_commit(done_bar);
         }
@@ -404,15 +509,19 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         if (ok && 32 * q < C) {  // only accumulator rows < C carry the result
             tc_fence_after();
             const int co = 32 * q + lane;
-            float *out = part + ((size_t)blockIdx.x * 9 + (size_t)ky * 3) * C * C;
+            float *out = part + (size_t)blockIdx.x * 9 * C * C;
+            const int ncols = slab ? 9 * C : 3 * C;
 #pragma unroll 1
-            for (int c0 = 0; c0 < Wg::ncols; c0 += 16) {
+            for (int c0 = 0; c0 < ncols; c0 += 16) {
                 float v[16];
                 tc_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, v);
                 tc_wait_ld();
                 if (co < C) {
+                    // column c0..c0+15 = 16 input channels of one tap
+                    const int g = c0 / C, ci0 = c0 % C;
+                    const int tap = slab ? (g % 3) * 3 + g / 3 : ky_cta * 3 + g;   // slab: g = kx*3 + ky
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) out[(size_t)(c0 + j) * C + co] = v[j];  // [(kx, ci)][co]
+                    for (int j = 0; j < 16; ++j) out[((size_t)tap * C + ci0 + j) * C + co] = v[j];  // [tap][ci][co]
                 }
             }
         }
@@ -421,7 +530,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Wg::tmem_cols)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
                      : "memory");
     }
 }
@@ -441,8 +550,10 @@ __global__ void wgrad_tc_fold_kernel(const float *__restrict__ part, float *__re
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 
 struct MapKey {
-    const void *ptr; int B, H, W, C;
-    bool operator<(const MapKey &o) const { return std::tie(ptr, B, H, W, C) < std::tie(o.ptr, o.B, o.H, o.W, o.C); }
+    const void *ptr; int B, H, W, C, rows, imgs;
+    bool operator<(const MapKey &o) const {
+        return std::tie(ptr, B, H, W, C, rows, imgs) < std::tie(o.ptr, o.B, o.H, o.W, o.C, o.rows, o.imgs);
+    }
 };
 std::map<MapKey, CUtensorMap> g_maps;
 std::mutex g_maps_mu;
@@ -454,14 +565,12 @@ void tile_geometry(int H, int W, int *rows_per_tile, int *imgs_per_tile) {
     *imgs_per_tile = kTileM / (W * r);
 }
 
-// Tensor map of an NHWC bf16 tensor with a box of one 128-pixel tile: (C, W, rows, images), zero fill outside.
-bool get_map(const void *ptr, int B, int H, int W, int C, CUtensorMap *out) {
+// Tensor map of an NHWC bf16 tensor with a box of (C, W, rows, imgs), zero fill outside the tensor.
+bool get_map(const void *ptr, int B, int H, int W, int C, int rows, int imgs, CUtensorMap *out) {
     std::lock_guard<std::mutex> lock(g_maps_mu);
-    MapKey key{ptr, B, H, W, C};
+    MapKey key{ptr, B, H, W, C, rows, imgs};
     auto it = g_maps.find(key);
     if (it != g_maps.end()) { *out = it->second; return true; }
-    int rows, imgs;
-    tile_geometry(H, W, &rows, &imgs);
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
     cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
     cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)W, (cuuint32_t)rows, (cuuint32_t)imgs};
@@ -472,26 +581,56 @@ bool get_map(const void *ptr, int B, int H, int W, int C, CUtensorMap *out) {
                           CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return false;
-    if (g_maps.size() > 4096) g_maps.clear();
+    if (g_maps.size() > 8192) g_maps.clear();
     g_maps[key] = m;
     *out = m;
     return true;
 }
 
 int g_num_sms = 148;
+constexpr int kSmemBudget = 200 * 1024;
+constexpr int kSmemMax = 227 * 1024;
 
 template <int C>
-int launch_tc(int dir, const void *src, const void *w, void *dst, int B, int H, int W, Shortcut sc, cudaStream_t s) {
-    CUtensorMap map;
-    if (!get_map(src, B, H, W, C, &map)) return -1;
+int launch_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W,
+              Shortcut sc, cudaStream_t s) {
     int rows, imgs;
     tile_geometry(H, W, &rows, &imgs);
+    const int slab = (imgs == 1) ? 1 : 0;
+    const int box_rows = slab ? rows + 2 : rows;
+    CUtensorMap map;
+    if (32 % W != 0 || !get_map(src, B, H, W, C, box_rows, imgs, &map)) return -1;
+    const int stage_bytes = box_rows * imgs * W * C * 2;
+    int n_stages = (kSmemBudget - (int)conv_smem_plan<C>(0, 0).a_off) / stage_bytes;
+    if (n_stages > kMaxStages) n_stages = kMaxStages;
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
-    conv3x3_tc_kernel<C><<<grid, kTcThreads, TcCfg<C>::smem_bytes, s>>>(
-        map, (const bf16 *)w, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, sc.mode == 1 ? (const bf16 *)sc.a : nullptr,
-        sc.mode == 1 ? (const bf16 *)sc.b : nullptr);
+    conv3x3_tc_kernel<C><<<grid, kTcThreads, conv_smem_bytes<C>(n_stages, stage_bytes), s>>>(
+        map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
+        stage_bytes, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr);
     return 1;
+}
+
+template <int C>
+int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, cudaStream_t s) {
+    int rows, imgs;
+    tile_geometry(H, W, &rows, &imgs);
+    const int slab = (imgs == 1 && 9 * C <= 512) ? 1 : 0;
+    CUtensorMap mx, md;
+    if (!get_map(x, B, H, W, C, slab ? rows + 2 : rows, imgs, &mx) || !get_map(dy, B, H, W, C, rows, imgs, &md)) return -1;
+    const int x_box_bytes = (slab ? rows + 2 : rows) * imgs * W * C * 2;
+    const int stage_bytes = TcCfg<C>::tile_bytes + 3 * x_box_bytes;
+    int n_stages = kSmemBudget / stage_bytes;
+    if (n_stages > kMaxStages) n_stages = kMaxStages;
+    const int ncols = slab ? 9 * C : 3 * C;
+    const int tmem_cols = ncols <= 64 ? 64 : (ncols <= 128 ? 128 : (ncols <= 256 ? 256 : 512));
+    const int n_tiles = (int)((long)B * H * W / kTileM);
+    const int max_chunks = slab ? (C == 16 ? 148 : 74) : 49;
+    const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
+    wgrad_tc_kernel<C><<<dim3(chunks, slab ? 1 : 3), kTcThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s>>>(
+        mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
+    wgrad_tc_fold_kernel<<<ceil_div(9 * C * C, 256), 256, 0, s>>>(scratch, dw, chunks, C);
+    return 2;
 }
 
 }  // namespace
@@ -499,42 +638,37 @@ int launch_tc(int dir, const void *src, const void *w, void *dst, int B, int H, 
 bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
     if (!g_encode) return false;
     if (stride != 1 || Cin != Cout || (Cin != 16 && Cin != 32 && Cin != 64)) return false;
-    if (W > kTileM || kTileM % W != 0) return false;
+    if (W > 32 || 32 % W != 0) return false;  // a warp of the epilogue must hold whole image rows
     const int r = kTileM / W;
     if (r <= H) { if (H % r != 0) return false; }
     else { if (kTileM % (H * W) != 0 || B % (kTileM / (H * W)) != 0) return false; }
     return ((long)B * H * W) % kTileM == 0;
 }
 
-int launch_conv_tc(int dir, const void *src, const void *w, void *dst, int B, int H, int W, int C, Shortcut sc,
-                   cudaStream_t s) {
+size_t tc_packed_bytes(int C) { return 2 * (size_t)9 * C * C * 2; }
+
+int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
+                   Shortcut sc, cudaStream_t s) {
     switch (C) {
-    case 16: return launch_tc<16>(dir, src, w, dst, B, H, W, sc, s);
-    case 32: return launch_tc<32>(dir, src, w, dst, B, H, W, sc, s);
-    case 64: return launch_tc<64>(dir, src, w, dst, B, H, W, sc, s);
+    case 16: return launch_tc<16>(dir, src, w, w_packed, dst, B, H, W, sc, s);
+    case 32: return launch_tc<32>(dir, src, w, w_packed, dst, B, H, W, sc, s);
+    case 64: return launch_tc<64>(dir, src, w, w_packed, dst, B, H, W, sc, s);
     }
     return -1;
+}
+
+int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,
+                        cudaStream_t s) {
+    if (n_jobs == 0) return 0;
+    pack_filters_kernel<<<ceil_div(total_elems, 256), 256, 0, s>>>((const bf16 *)wver, (uint8_t *)packed,
+                                                                  (const PackJob *)jobs_dev, n_jobs, total_elems);
+    return 1;
 }
 
 bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
     return conv_tc_supported(B, H, W, Cin, Cout, stride);
 }
-size_t wgrad_tc_scratch_elems() { return (size_t)kWgMaxChunks * 9 * 64 * 64; }
-
-namespace {
-template <int C>
-int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, cudaStream_t s) {
-    CUtensorMap mx, md;
-    if (!get_map(x, B, H, W, C, &mx) || !get_map(dy, B, H, W, C, &md)) return -1;
-    int rows, imgs;
-    tile_geometry(H, W, &rows, &imgs);
-    const int n_tiles = (int)((long)B * H * W / kTileM);
-    const int chunks = n_tiles < kWgMaxChunks ? n_tiles : kWgMaxChunks;
-    wgrad_tc_kernel<C><<<dim3(chunks, 3), kTcThreads, WgCfg<C>::smem_bytes, s>>>(mx, md, scratch, H, W, rows, imgs, n_tiles);
-    wgrad_tc_fold_kernel<<<ceil_div(9 * C * C, 256), 256, 0, s>>>(scratch, dw, chunks, C);
-    return 2;
-}
-}  // namespace
+size_t wgrad_tc_scratch_elems() { return (size_t)kWgMaxChunks * 9 * 32 * 32 > (size_t)49 * 9 * 64 * 64 ? (size_t)kWgMaxChunks * 9 * 32 * 32 : (size_t)49 * 9 * 64 * 64; }
 
 int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C,
                     cudaStream_t s) {
@@ -563,12 +697,13 @@ int conv_tc_init() {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-    e = cudaFuncSetAttribute(conv3x3_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<16>::smem_bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<32>::smem_bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcCfg<64>::smem_bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wgrad_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WgCfg<16>::smem_bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wgrad_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WgCfg<32>::smem_bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(wgrad_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WgCfg<64>::smem_bytes);
+    const void *fns[6] = {(const void *)conv3x3_tc_kernel<16>, (const void *)conv3x3_tc_kernel<32>,
+                          (const void *)conv3x3_tc_kernel<64>, (const void *)wgrad_tc_kernel<16>,
+                          (const void *)wgrad_tc_kernel<32>, (const void *)wgrad_tc_kernel<64>};
+    for (const void *f : fns) {
+        e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+        if (e != cudaSuccess) break;
+    }
     rc = (int)e;
     return rc;
 }

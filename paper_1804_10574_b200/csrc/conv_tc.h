@@ -12,8 +12,16 @@ namespace ddg {
 bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
 // dir 0: dst = conv3x3(src, w) (forward).  dir 1: dst = input gradient of conv3x3 given src = dy; with
 // sc.mode == 1 the identity-shortcut gradient sc.a * [sc.b > 0] is added before the store.
-int launch_conv_tc(int dir, const void *src, const void *w, void *dst, int B, int H, int W, int C, Shortcut sc,
-                   cudaStream_t s);
+// w: filter in canonical [Cout][Cin][3][3] order.  w_packed (nullable): the pre-arranged filter images written by
+// launch_pack_filters for this convolution (tc_packed_bytes(C) bytes: forward image, then input-gradient image); when
+// given, the kernel fetches its filter with one bulk copy instead of re-arranging the canonical one itself.
+int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
+                   Shortcut sc, cudaStream_t s);
+size_t tc_packed_bytes(int C);
+// One launch that re-arranges the filters of many convolutions of one weight version.
+struct PackJobHost { long src_off; long dst_off; int C; int first_elem; };  // element offset in wver, byte offset in packed
+int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,
+                        cudaStream_t s);
 
 bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
 size_t wgrad_tc_scratch_elems();

@@ -34,6 +34,7 @@ struct LayerPlan {
     size_t p_cnt;
     TensorRef in, out;            // layer input (may live in the previous module's arena) and output
     TensorRef y1, a1, y2, stats;  // basic block intermediates; stats = fp32 [4][C] (mean1,invstd1,mean2,invstd2)
+    long pk1 = -1, pk2 = -1;      // byte offsets of the pre-arranged filter images (conv / conv1, conv2), -1 = none
     bool is_first, is_last;
 };
 
@@ -46,6 +47,10 @@ struct Module {
     char *arena = nullptr;      // R slots
     float *w = nullptr, *v = nullptr, *m2 = nullptr, *g = nullptr;
     char *wver = nullptr;       // R weight versions in the compute precision
+    char *packed = nullptr;     // R sets of pre-arranged filter images for the tensor-core kernels
+    size_t packed_bytes = 0;
+    void *pack_jobs = nullptr;  // device table of PackJobHost
+    int n_pack_jobs = 0, pack_elems = 0;
     char *tmp[3] = {nullptr, nullptr, nullptr};  // error-gradient temporaries of the backward sweep
     size_t tmp_bytes = 0;
     float *bn_scratch = nullptr, *wg_scratch = nullptr;
@@ -123,16 +128,16 @@ char *slot_ptr(ddg_ctx *c, TensorRef r, long iter) {
 }
 
 // ---- convolution dispatch: tensor-core path where it applies, CUDA cores otherwise --------------------
-int conv_fwd(ddg_ctx *c, const void *x, const void *w, void *y, int H, int W, int Cin, int Cout, int stride, int relu,
-             cudaStream_t s) {
+int conv_fwd(ddg_ctx *c, const void *x, const void *w, const void *wp, void *y, int H, int W, int Cin, int Cout,
+             int stride, int relu, cudaStream_t s) {
     if (c->prec == P_BF16 && !relu && conv_tc_supported(c->B, H, W, Cin, Cout, stride))
-        return launch_conv_tc(0, x, w, y, c->B, H, W, Cin, Shortcut{}, s);
+        return launch_conv_tc(0, x, w, wp, y, c->B, H, W, Cin, Shortcut{}, s);
     return launch_conv_fwd_direct(c->prec, x, w, y, c->B, H, W, Cin, Cout, stride, relu, s);
 }
-int conv_dgrad(ddg_ctx *c, const void *dy, const void *w, void *dx, int H, int W, int Cin, int Cout, int stride,
-               Shortcut sc, cudaStream_t s) {
+int conv_dgrad(ddg_ctx *c, const void *dy, const void *w, const void *wp, void *dx, int H, int W, int Cin, int Cout,
+               int stride, Shortcut sc, cudaStream_t s) {
     if (c->prec == P_BF16 && sc.mode != 2 && conv_tc_supported(c->B, H, W, Cin, Cout, stride))
-        return launch_conv_tc(1, dy, w, dx, c->B, H, W, Cin, sc, s);
+        return launch_conv_tc(1, dy, w, wp, dx, c->B, H, W, Cin, sc, s);
     return launch_conv_dgrad_direct(c->prec, dy, w, dx, c->B, H, W, Cin, Cout, stride, sc, s);
 }
 int conv_wgrad(ddg_ctx *c, Module &m, const void *x, const void *dy, float *dw, int H, int W, int Cin, int Cout,
@@ -148,6 +153,8 @@ long forward_module(ddg_ctx *c, int k, long t) {
     cudaStream_t s = m.stream;
     const size_t es = elem_size(c->prec);
     const char *wv = m.wver + (size_t)(t % m.R) * m.P * es;
+    const char *pk = m.packed ? m.packed + (size_t)(t % m.R) * m.packed_bytes : nullptr;
+    auto pkp = [&](long off) -> const void * { return (pk && off >= 0) ? pk + off : nullptr; };
     long n = 0;
     for (int l = m.first; l <= m.last; ++l) {
         LayerPlan &L = c->layers[l];
@@ -169,7 +176,7 @@ long forward_module(ddg_ctx *c, int k, long t) {
                                L.Cin, L.Cout, L.spec.relu_after, L.is_last, s);
             break;
         case DDG_CONV3X3:
-            n += conv_fwd(c, in, w, out, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, L.spec.relu_after, s);
+            n += conv_fwd(c, in, w, pkp(L.pk1), out, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, L.spec.relu_after, s);
             break;
         case DDG_BN: {
             float *st = (float *)slot_ptr(c, L.stats, t);
@@ -191,10 +198,10 @@ long forward_module(ddg_ctx *c, int k, long t) {
             char *y1 = slot_ptr(c, L.y1, t), *a1 = slot_ptr(c, L.a1, t), *y2 = slot_ptr(c, L.y2, t);
             float *stt = (float *)slot_ptr(c, L.stats, t);
             const long npix = (long)B * L.Hout * L.Wout;
-            n += conv_fwd(c, in, w1, y1, L.Hin, L.Win, Ci, Co, st, 0, s);
+            n += conv_fwd(c, in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, Co, st, 0, s);
             n += launch_bn_stats(c->prec, y1, stt, stt + Co, m.bn_scratch, npix, Co, s);
             n += launch_bn_apply(c->prec, y1, g1, b1, stt, stt + Co, Shortcut{}, a1, B, L.Hout, L.Wout, Co, 1, s);
-            n += conv_fwd(c, a1, w2, y2, L.Hout, L.Wout, Co, Co, 1, 0, s);
+            n += conv_fwd(c, a1, w2, pkp(L.pk2), y2, L.Hout, L.Wout, Co, Co, 1, 0, s);
             n += launch_bn_stats(c->prec, y2, stt + 2 * Co, stt + 3 * Co, m.bn_scratch, npix, Co, s);
             Shortcut sc{};
             sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
@@ -218,6 +225,8 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
     cudaStream_t s = m.stream;
     const size_t es = elem_size(c->prec);
     const char *wv = m.wver + (size_t)(sidx % m.R) * m.P * es;  // the weights w^s of the stored iteration
+    const char *pk = m.packed ? m.packed + (size_t)(sidx % m.R) * m.packed_bytes : nullptr;
+    auto pkp = [&](long off) -> const void * { return (pk && off >= 0) ? pk + off : nullptr; };
     long n = 0;
     const int B = c->B;
     const char *cur = (k == c->K - 1) ? (const char *)c->dlogits : c->mods[k + 1].delta_out[(t + 1) % 2];
@@ -251,7 +260,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
                 dy = m.tmp[tm];
             }
             if (need_dx)
-                n += conv_dgrad(c, dy, w, dst, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, Shortcut{}, s);
+                n += conv_dgrad(c, dy, w, pkp(L.pk1), dst, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, Shortcut{}, s);
             n += conv_wgrad(c, m, in, dy, gw, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, s);
             break;
         }
@@ -285,7 +294,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
             n += launch_bn_bwd_reduce(c->prec, cur, out, y2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, m.bn_scratch, npix, Co,
                                       1, s);
             n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s);
-            n += conv_dgrad(c, dy2, w2, da1, L.Hout, L.Wout, Co, Co, 1, Shortcut{}, s);
+            n += conv_dgrad(c, dy2, w2, pkp(L.pk2), da1, L.Hout, L.Wout, Co, Co, 1, Shortcut{}, s);
             n += conv_wgrad(c, m, a1, dy2, gw2, L.Hout, L.Wout, Co, Co, 1, s);
             n += launch_bn_bwd_reduce(c->prec, da1, a1, y1, stt, stt + Co, gg1, gb1, m.bn_scratch, npix, Co, 1, s);
             n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
@@ -294,7 +303,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
                 sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
                 sc.a = cur; sc.b = out; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win;
                 char *dx = mod_first ? dst : da1;  // da1 is dead once bn1's backward has run
-                n += conv_dgrad(c, dy1, w1, dx, L.Hin, L.Win, Ci, Co, st, sc, s);
+                n += conv_dgrad(c, dy1, w1, pkp(L.pk1), dx, L.Hin, L.Win, Ci, Co, st, sc, s);
                 if (!mod_first) { dst = dx; dst_tmp = tB; }
             }
             n += conv_wgrad(c, m, in, dy1, gw1, L.Hin, L.Win, Ci, Co, st, s);
@@ -305,6 +314,13 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
         cur_tmp = dst_tmp;
     }
     return n;
+}
+
+// Re-arrange the filters of weight version `slot` into the images the tensor-core kernels copy in one piece.
+long pack_module(Module &m, int slot, size_t es) {
+    if (!m.packed || m.n_pack_jobs == 0) return 0;
+    return launch_pack_filters(m.wver + (size_t)slot * m.P * es, m.packed + (size_t)slot * m.packed_bytes, m.pack_jobs,
+                               m.n_pack_jobs, m.pack_elems, m.stream);
 }
 
 // ---- update of module k with its delayed gradient (Eq. 8-9; Algorithm 1 / 2) --------------------------
@@ -321,7 +337,9 @@ long update_module(ddg_ctx *c, int k, long t, bool have_grad) {
     } else a.mode = 0;
     if (a.mode == 2 && m.R == 1) return 0;
     char *wv = m.wver + (size_t)((t + 1) % m.R) * m.P * elem_size(c->prec);
-    return launch_update(c->prec, m.w, m.v, m.m2, m.g, wv, m.P, a, m.stream);
+    long n = launch_update(c->prec, m.w, m.v, m.m2, m.g, wv, m.P, a, m.stream);
+    n += pack_module(m, (int)((t + 1) % m.R), elem_size(c->prec));
+    return n;
 }
 
 // Enqueue one whole iteration on the K streams.  `in_capture`: the cross-iteration waits are dropped because
@@ -412,7 +430,7 @@ ddg_status init_weights(ddg_ctx *ctx) {
         default: break;
         }
     }
-    for (auto &m : ctx->mods) launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream);
+    for (auto &m : ctx->mods) { launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream); pack_module(m, 0, elem_size(ctx->prec)); }
     CU(cudaGetLastError());
     for (auto &m : ctx->mods) CU(cudaStreamSynchronize(m.stream));
     return DDG_OK;
@@ -452,6 +470,7 @@ void ddg_destroy(ddg_ctx *ctx) {
     for (auto g : ctx->graphs)
         if (g) cudaGraphExecDestroy(g);
     for (auto &m : ctx->mods) {
+        cudaFree(m.packed); cudaFree(m.pack_jobs);
         cudaFree(m.arena); cudaFree(m.w); cudaFree(m.v); cudaFree(m.m2); cudaFree(m.g); cudaFree(m.wver);
         for (char *p : m.tmp) cudaFree(p);
         cudaFree(m.bn_scratch); cudaFree(m.wg_scratch);
@@ -616,6 +635,35 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
             }
         }
         wg_max = std::max(wg_max, wgrad_tc_scratch_elems());
+        if (c->prec == P_BF16) {  // pre-arranged filter images for the convolutions the tensor-core kernels take
+            std::vector<PackJobHost> jobs;
+            size_t pk_off = 0;
+            int elems = 0;
+            auto plan = [&](long *slot, size_t w_off, int H, int W, int Ci, int Co, int stride) {
+                if (!conv_tc_supported(c->B, H, W, Ci, Co, stride)) return;
+                *slot = (long)pk_off;
+                jobs.push_back(PackJobHost{(long)w_off, (long)pk_off, Ci, elems});
+                pk_off += tc_packed_bytes(Ci);
+                elems += 9 * Ci * Ci;
+            };
+            for (int l = m.first; l <= m.last; ++l) {
+                LayerPlan &L = c->layers[l];
+                if (L.spec.kind == DDG_CONV3X3 && !L.spec.relu_after)
+                    plan(&L.pk1, L.p_off, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride);
+                if (L.spec.kind == DDG_BASIC_BLOCK) {
+                    plan(&L.pk1, L.p_off, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride);
+                    plan(&L.pk2, L.p_off + (size_t)L.Cout * L.Cin * 9 + 2 * (size_t)L.Cout, L.Hout, L.Wout, L.Cout, L.Cout, 1);
+                }
+            }
+            if (!jobs.empty()) {
+                m.packed_bytes = pk_off;
+                m.n_pack_jobs = (int)jobs.size();
+                m.pack_elems = elems;
+                CU(cudaMalloc(&m.packed, pk_off * m.R));
+                CU(cudaMalloc(&m.pack_jobs, jobs.size() * sizeof(PackJobHost)));
+                CU(cudaMemcpy(m.pack_jobs, jobs.data(), jobs.size() * sizeof(PackJobHost), cudaMemcpyHostToDevice));
+            }
+        }
         CU(cudaMalloc(&m.bn_scratch, std::max<size_t>(bn_max, 64) * 4));
         CU(cudaMemset(m.bn_scratch, 0, std::max<size_t>(bn_max, 64) * 4));
         CU(cudaMalloc(&m.wg_scratch, std::max<size_t>(wg_max, 64) * 4));
@@ -732,7 +780,7 @@ ddg_status ddg_set_weights(ddg_ctx *ctx, const float *src, size_t n, int on_devi
         if (m.m2) CU(cudaMemset(m.m2, 0, m.P * 4));
     }
     CU(cudaDeviceSynchronize());  // default-stream copies and memsets are not ordered against the module streams
-    for (auto &m : ctx->mods) launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream);
+    for (auto &m : ctx->mods) { launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream); pack_module(m, 0, elem_size(ctx->prec)); }
     CU(cudaGetLastError());
     return sync_all(ctx);
 }
