@@ -86,7 +86,7 @@ typedef struct {
     int in_c, in_h, in_w;   /* input is [B][in_c][in_h][in_w] fp32 (use in_h = in_w = 1 for an MLP) */
     int num_classes;
     unsigned long long seed; /* seed of the library's own He-normal initialisation */
-    int use_graph;  /* 1: replay the steady-state iteration as CUDA graphs (one per ring phase) */
+    int use_graph;  /* 1: replay the steady-state iteration from CUDA graphs (one per ring phase, module and sweep) */
     int debug_checks; /* 1: stamp ring slots with the iteration that wrote them and verify on use */
     void *const *streams; /* host array of K cudaStream_t to run the modules on, or NULL (library creates K) */
 } ddg_cfg;

@@ -72,12 +72,12 @@ ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float
     return done();
 }
 
-size_t ddg_bn_scratch_elems(int C) { return C >= 1 && C <= 256 ? bn_scratch_elems(C) : 0; }
+size_t ddg_bn_scratch_elems(int C) { return C >= 1 && C <= 128 ? bn_scratch_elems(C) : 0; }
 
 ddg_status ddg_bn_fwd(int precision, const void *x, const void *gamma, const void *beta, const void *res, void *y,
                       float *mean, float *invstd, float *scratch, int B, int HW, int C, int relu, void *stream) {
     if (bad_prec(precision) || !x || !gamma || !beta || !y || !mean || !invstd || !scratch) return DDG_ERR_INVALID_ARG;
-    if (B < 1 || HW < 1 || C < 1 || C > 256) return DDG_ERR_UNSUPPORTED;
+    if (B < 1 || HW < 1 || C < 1 || C > 128) return DDG_ERR_UNSUPPORTED;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;  // the CTA ticket counter
     launch_bn_stats(precision, x, mean, invstd, scratch, (long)B * HW, C, s);
@@ -93,7 +93,7 @@ ddg_status ddg_bn_bwd(int precision, const void *dout, const void *out, const vo
     if (bad_prec(precision) || !dout || !x || !gamma || !mean || !invstd || !dx || !dgamma || !dbeta || !scratch ||
         (relu && !out))
         return DDG_ERR_INVALID_ARG;
-    if (B < 1 || HW < 1 || C < 1 || C > 256) return DDG_ERR_UNSUPPORTED;
+    if (B < 1 || HW < 1 || C < 1 || C > 128) return DDG_ERR_UNSUPPORTED;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;
     launch_bn_bwd_reduce(precision, dout, out, x, mean, invstd, dgamma, dbeta, scratch, (long)B * HW, C, relu, s);

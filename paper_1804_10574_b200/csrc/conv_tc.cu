@@ -535,15 +535,29 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     }
 }
 
-// dw[co][ci][tap] = sum over chunks of part[chunk][tap][ci][co]   (fixed order)
-__global__ void wgrad_tc_fold_kernel(const float *__restrict__ part, float *__restrict__ dw, int chunks, int C) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+// dw[co][ci][tap] = sum over chunks of part[chunk][tap][ci][co].  64 outputs per CTA, four threads per output: thread g
+// adds chunks g, g+4, ... (four independent loads in flight per thread), the four sums are combined in a fixed order.
+__global__ void __launch_bounds__(256) wgrad_tc_fold_kernel(const float *__restrict__ part, float *__restrict__ dw, int chunks, int C) {
+    __shared__ float sm[4][64];
     const int total = 9 * C * C;
-    if (i >= total) return;
-    float t = 0.f;
-    for (int c = 0; c < chunks; ++c) t += part[(size_t)c * total + i];
-    const int co = i % C, ci = (i / C) % C, tap = i / (C * C);
-    dw[((size_t)co * C + ci) * 9 + tap] = t;
+    const int o = threadIdx.x & 63, g = threadIdx.x >> 6;
+    const int i = blockIdx.x * 64 + o;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    if (i < total) {
+        int c = g;
+        for (; c + 12 < chunks; c += 16) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc[u] += __ldcg(part + (size_t)(c + 4 * u) * total + i);
+        }
+        for (; c < chunks; c += 4) acc[0] += __ldcg(part + (size_t)c * total + i);
+    }
+    sm[g][o] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    __syncthreads();
+    if (g == 0 && i < total) {
+        const float t = (sm[0][o] + sm[1][o]) + (sm[2][o] + sm[3][o]);
+        const int co = i % C, ci = (i / C) % C, tap = i / (C * C);
+        dw[((size_t)co * C + ci) * 9 + tap] = t;
+    }
 }
 
 // ---- host side: tensor maps ------------------------------------------------------------------------------
@@ -629,7 +643,7 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
     wgrad_tc_kernel<C><<<dim3(chunks, slab ? 1 : 3), kTcThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s>>>(
         mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
-    wgrad_tc_fold_kernel<<<ceil_div(9 * C * C, 256), 256, 0, s>>>(scratch, dw, chunks, C);
+    wgrad_tc_fold_kernel<<<ceil_div(9 * C * C, 64), 256, 0, s>>>(scratch, dw, chunks, C);
     return 2;
 }
 

@@ -78,7 +78,6 @@ struct ddg_ctx {
     size_t x_elems = 0;
     float *dlogits = nullptr, *loss_dev = nullptr;
     float *pinned_loss = nullptr;
-    cudaEvent_t ev_fork = nullptr;
     std::vector<cudaGraphExec_t> graphs;
     std::vector<long> graph_launches;
     long launches = 0;
@@ -342,59 +341,78 @@ long update_module(ddg_ctx *c, int k, long t, bool have_grad) {
     return n;
 }
 
-// Enqueue one whole iteration on the K streams.  `in_capture`: the cross-iteration waits are dropped because
-// successive graph launches are already ordered.
-ddg_status enqueue_iteration(ddg_ctx *ctx, long t, bool in_capture, long *launches) {
-    const int K = ctx->K;
+// One schedulable piece of an iteration: the forward sweep of module k (seg 0) or its backward sweep + update
+// (seg 1).  Inside a piece the kernels form a chain on the module's stream.
+ddg_status enqueue_segment(ddg_ctx *ctx, int k, int seg, long t, long *launches) {
+    const long sidx = t - ctx->K + (k + 1);
     long n = 0;
-    // forward sweep, module 1..K in order; module k+1 waits for module k's output
-    for (int k = 0; k < K; ++k) {
-        Module &m = ctx->mods[k];
-        if (k > 0) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k - 1].ev_fwd, 0));
-        n += forward_module(ctx, k, t);
-        if (k < K - 1) CU(cudaEventRecord(m.ev_fwd, m.stream));
-    }
-    // backward sweeps and updates: independent across modules within the iteration ("for k in parallel")
-    for (int k = 0; k < K; ++k) {
-        Module &m = ctx->mods[k];
-        const long sidx = t - K + (k + 1);
-        if (sidx >= 0) {
-            if (k < K - 1 && !in_capture) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k + 1].ev_bwd, 0));
-            n += backward_module(ctx, k, t, sidx);
-            if (k > 0 && !in_capture) CU(cudaEventRecord(m.ev_bwd, m.stream));
-        }
+    if (seg == 0) n += forward_module(ctx, k, t);
+    else {
+        if (sidx >= 0) n += backward_module(ctx, k, t, sidx);
         n += update_module(ctx, k, t, sidx >= 0);
-        m.last_sample = sidx >= 0 ? sidx : -1;
     }
     CU(cudaGetLastError());
     *launches = n;
     return DDG_OK;
 }
 
-ddg_status capture_phase(ddg_ctx *ctx, long t, int phase) {
-    const int K = ctx->K;
-    cudaStream_t s0 = ctx->mods[0].stream;
-    CU(cudaStreamBeginCapture(s0, cudaStreamCaptureModeThreadLocal));
-    ddg_status st = DDG_OK;
-    long n = 0;
-    cudaError_t e = cudaEventRecord(ctx->ev_fork, s0);
-    for (int k = 1; k < K && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(ctx->mods[k].stream, ctx->ev_fork, 0);
-    if (e == cudaSuccess) st = enqueue_iteration(ctx, t, true, &n);
-    for (int k = 1; k < K && e == cudaSuccess && st == DDG_OK; ++k) {
-        e = cudaEventRecord(ctx->mods[k].ev_join, ctx->mods[k].stream);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(s0, ctx->mods[k].ev_join, 0);
+// Run a piece: directly, or as a replay of the CUDA graph recorded for (ring phase, module, piece).  The graph holds
+// only the module's own chain; what orders the pieces against each other (module k+1's forward after module k's,
+// module k's backward after the error gradient module k+1 produced one iteration earlier) stays outside as stream
+// events, so consecutive iterations overlap exactly as they do without graphs.
+ddg_status run_segment(ddg_ctx *ctx, int k, int seg, long t, bool use_graph, long *launches) {
+    Module &m = ctx->mods[k];
+    // Adam's bias corrections change every iteration, so an update with them cannot be replayed from a recording
+    if (use_graph && seg == 1 && ctx->opt.kind == DDG_OPT_ADAM) use_graph = false;
+    if (!use_graph) return enqueue_segment(ctx, k, seg, t, launches);
+    const int phase = (int)(t % ctx->period);
+    const size_t idx = ((size_t)phase * ctx->K + k) * 2 + seg;
+    if (!ctx->graphs[idx]) {
+        CU(cudaStreamBeginCapture(m.stream, cudaStreamCaptureModeThreadLocal));
+        long n = 0;
+        ddg_status st = enqueue_segment(ctx, k, seg, t, &n);
+        cudaGraph_t graph = nullptr;
+        cudaError_t e2 = cudaStreamEndCapture(m.stream, &graph);
+        if (st != DDG_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+        CU(e2);
+        cudaGraphExec_t exec = nullptr;
+        cudaError_t e3 = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        CU(e3);
+        ctx->graphs[idx] = exec;
+        ctx->graph_launches[idx] = n;
     }
-    cudaGraph_t graph = nullptr;
-    cudaError_t e2 = cudaStreamEndCapture(s0, &graph);
-    if (st != DDG_OK) { if (graph) cudaGraphDestroy(graph); return st; }
-    CU(e);
-    CU(e2);
-    cudaGraphExec_t exec = nullptr;
-    cudaError_t e3 = cudaGraphInstantiate(&exec, graph, 0);
-    cudaGraphDestroy(graph);
-    CU(e3);
-    ctx->graphs[phase] = exec;
-    ctx->graph_launches[phase] = n;
+    CU(cudaGraphLaunch(ctx->graphs[idx], m.stream));
+    *launches = ctx->graph_launches[idx];
+    return DDG_OK;
+}
+
+// Enqueue one whole iteration on the K streams.
+ddg_status enqueue_iteration(ddg_ctx *ctx, long t, bool use_graph, long *launches) {
+    const int K = ctx->K;
+    long total = 0, n = 0;
+    // forward sweep, module 1..K in order; module k+1 waits for module k's output
+    for (int k = 0; k < K; ++k) {
+        Module &m = ctx->mods[k];
+        if (k > 0) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k - 1].ev_fwd, 0));
+        ddg_status st = run_segment(ctx, k, 0, t, use_graph, &n);
+        if (st != DDG_OK) return st;
+        total += n;
+        if (k < K - 1) CU(cudaEventRecord(m.ev_fwd, m.stream));
+    }
+    // backward sweeps and updates: independent across modules within the iteration ("for k in parallel").  Ascending
+    // k, so that module k waits for the error gradient module k+1 recorded in the PREVIOUS iteration.
+    for (int k = 0; k < K; ++k) {
+        Module &m = ctx->mods[k];
+        const long sidx = t - K + (k + 1);
+        if (sidx >= 0 && k < K - 1) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k + 1].ev_bwd, 0));
+        ddg_status st = run_segment(ctx, k, 1, t, use_graph, &n);
+        if (st != DDG_OK) return st;
+        total += n;
+        if (sidx >= 0 && k > 0) CU(cudaEventRecord(m.ev_bwd, m.stream));
+        m.last_sample = sidx >= 0 ? sidx : -1;
+    }
+    *launches = total;
     return DDG_OK;
 }
 
@@ -482,7 +500,6 @@ void ddg_destroy(ddg_ctx *ctx) {
     }
     cudaFree(ctx->x_stage); cudaFree(ctx->y_stage); cudaFree(ctx->dlogits); cudaFree(ctx->loss_dev);
     if (ctx->pinned_loss) cudaFreeHost(ctx->pinned_loss);
-    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     delete ctx;
 }
 
@@ -555,8 +572,8 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
         }
         if (!ok) { set_err(nullptr, "layer %d: specification does not fit its input [%d,%d,%d]", l, L.Cin, L.Hin, L.Win); return DDG_ERR_BAD_SPEC; }
         if ((s.kind == DDG_CONV3X3 || s.kind == DDG_BASIC_BLOCK || s.kind == DDG_BN || s.kind == DDG_GLOBAL_AVGPOOL) &&
-            (C > 256 || L.Cin > 256 || (size_t)L.Cin * C > 4096)) {
-            set_err(nullptr, "layer %d: channel counts above 64x64 (or 256 for BN / pooling) are not supported", l);
+            (C > 128 || L.Cin > 128 || (size_t)L.Cin * C > 4096)) {
+            set_err(nullptr, "layer %d: channel counts above 64x64 (or 128 for BN / pooling) are not supported", l);
             return DDG_ERR_UNSUPPORTED;
         }
         L.Cout = C; L.Hout = H; L.Wout = W;
@@ -602,8 +619,8 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
     c->P = p_global;
     c->period = 2;
     for (int k = 0; k < K; ++k) c->period = c->period / gcd_i(c->period, c->mods[k].R) * c->mods[k].R;
-    c->graphs.assign(c->period, nullptr);
-    c->graph_launches.assign(c->period, 0);
+    c->graphs.assign((size_t)c->period * K * 2, nullptr);
+    c->graph_launches.assign((size_t)c->period * K * 2, 0);
 
     // ---- device state ----
     ctx = c;  // from here on CU() records into the context
@@ -681,7 +698,6 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
     CU(cudaMalloc(&c->loss_dev, 4));
     CU(cudaMemset(c->loss_dev, 0, 4));
     CU(cudaMallocHost(&c->pinned_loss, 4));
-    CU(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
     // the memsets above ran on the legacy default stream, which the non-blocking module streams do not wait for
     CU(cudaDeviceSynchronize());
     ddg_status st = init_weights(c);
@@ -699,31 +715,14 @@ static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float 
     // stage the batch: the sweeps (and graph replays) read library-owned buffers
     CU(cudaMemcpyAsync(ctx->x_stage + (size_t)(t % K) * ctx->x_elems, x, ctx->x_elems * 4, kind, s0));
     CU(cudaMemcpyAsync(ctx->y_stage + (size_t)(t % K) * ctx->B, y, (size_t)ctx->B * 4, kind, s0));
+    // the first K-1 iterations have modules in warm-up and a different shape: they are not recorded
     const bool steady = t >= K - 1;
-    if (ctx->cfg.use_graph && steady) {
-        const int phase = (int)(t % ctx->period);
-        if (!ctx->graphs[phase]) {
-            // first visit of this ring phase: record the iteration as a graph, then replay it like any other
-            ddg_status st = sync_all(ctx);
-            if (st != DDG_OK) return st;
-            st = capture_phase(ctx, t, phase);
-            if (st != DDG_OK) { ctx->broken = true; return st; }
-        }
-        CU(cudaGraphLaunch(ctx->graphs[phase], s0));
-        ctx->launches = ctx->graph_launches[phase];
-        for (int k = 0; k < K; ++k) ctx->mods[k].last_sample = t - K + (k + 1);
-    } else {
-        ddg_status st = enqueue_iteration(ctx, t, false, &ctx->launches);
-        if (st != DDG_OK) return st;
-    }
+    ddg_status st = enqueue_iteration(ctx, t, ctx->cfg.use_graph && steady, &ctx->launches);
+    if (st != DDG_OK) { ctx->broken = true; return st; }
     ctx->t = t + 1;
     if (loss_host) {
-        if (ctx->cfg.use_graph && steady) {
-            CU(cudaMemcpyAsync(ctx->pinned_loss, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, s0));
-        } else {
-            CU(cudaMemcpyAsync(ctx->pinned_loss, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, ctx->mods[K - 1].stream));
-        }
-        ddg_status st = sync_all(ctx);
+        CU(cudaMemcpyAsync(ctx->pinned_loss, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, ctx->mods[K - 1].stream));
+        st = sync_all(ctx);
         if (st != DDG_OK) return st;
         *loss_host = *ctx->pinned_loss;
     }

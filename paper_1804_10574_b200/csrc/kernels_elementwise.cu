@@ -299,12 +299,20 @@ bn_reduce_kernel(const T *__restrict__ x, const T *__restrict__ dout, const T *_
     __syncthreads();
     if (!is_last) return;
     __threadfence();
+    // fold the per-CTA partials with the whole CTA: value v (0..2C) is summed by kThreads/(2C) threads over interleaved
+    // partials (several loads in flight each), then combined in a fixed order
+    __shared__ double fold[kThreads];
+    const int nval = 2 * C;
+    const int ways = kThreads / nval;  // >= 1: C <= 128 on this path, checked by the host
+    const int v = threadIdx.x % nval, way = threadIdx.x / nval;
+    double acc = 0.0;
+    if (way < ways)
+        for (unsigned i = way; i < gridDim.x; i += ways) acc += (double)__ldcg(part + (size_t)i * 2 * C + v);
+    fold[threadIdx.x] = acc;
+    __syncthreads();
     for (int c = threadIdx.x; c < C; c += kThreads) {
         double a = 0.0, b = 0.0;
-        for (unsigned i = 0; i < gridDim.x; ++i) {
-            a += (double)__ldcg(part + (size_t)i * 2 * C + c);
-            b += (double)__ldcg(part + (size_t)i * 2 * C + C + c);
-        }
+        for (int w = 0; w < ways; ++w) { a += fold[w * nval + c]; b += fold[w * nval + C + c]; }
         if (MODE == 0) {
             double m = a / (double)npix, var = b / (double)npix - m * m;
             if (var < 0.0) var = 0.0;
