@@ -154,6 +154,16 @@ ddg_status ddg_conv3x3_fwd(int precision, const void *x, const void *w, void *y,
 /* dx = conv3x3 input gradient (Eq. 5 / Eq. 7).  dy [B][Ho][Wo][Cout], dx [B][H][W][Cin]. */
 ddg_status ddg_conv3x3_dgrad(int precision, const void *dy, const void *w, void *dx, int B, int H, int W, int Cin,
                              int Cout, int stride, void *stream);
+/* The tensor-core convolution reads its filter from a pre-arranged image (what the training step keeps per weight
+ * version, refreshed by the optimiser update): ddg_conv3x3_packed_bytes gives its size for a stride-1 C->C bf16
+ * convolution on [B][H][W][C] (0 when the tensor-core path does not take the shape), ddg_conv3x3_pack writes it from a
+ * canonical bf16 filter, ddg_conv3x3_packed runs the forward (dgrad = 0) or input-gradient (dgrad = 1) convolution
+ * with it (Eq. 3 / Eq. 5).  All pointers device. */
+size_t ddg_conv3x3_packed_bytes(int B, int H, int W, int C);
+ddg_status ddg_conv3x3_pack(const void *w, void *packed, int C, void *stream);
+ddg_status ddg_conv3x3_packed(int dgrad, const void *src, const void *w, const void *packed, void *dst, int B, int H,
+                              int W, int C, void *stream);
+
 /* dw = conv3x3 weight gradient (Eq. 4 / Eq. 6), fp32 [Cout][Cin][3][3].  scratch: device, fp32,
  * ddg_conv3x3_wgrad_scratch_elems(...) elements, contents undefined on entry and exit. */
 size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride);

@@ -26,7 +26,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_set_weights", "ddg_get_grads", "ddg_get_loss_dev", "ddg_last_step_launches", "ddg_sync",
            "ddg_last_error", "ddg_destroy", "ddg_conv3x3_fwd", "ddg_conv3x3_dgrad",
            "ddg_conv3x3_wgrad_scratch_elems", "ddg_conv3x3_wgrad", "ddg_bn_scratch_elems", "ddg_bn_fwd", "ddg_bn_bwd",
-           "ddg_sgd_update", "ddg_tensor_core_path", "ddg_bn_fwd_noalloc"]
+           "ddg_sgd_update", "ddg_tensor_core_path", "ddg_bn_fwd_noalloc",
+           "ddg_conv3x3_packed_bytes", "ddg_conv3x3_pack", "ddg_conv3x3_packed"]
 
 
 class Layer(ctypes.Structure):
@@ -72,6 +73,10 @@ _lib.ddg_bn_scratch_elems.restype = _sz
 _lib.ddg_bn_fwd.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_bn_bwd.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_tensor_core_path.argtypes = [_i] * 6
+_lib.ddg_conv3x3_packed_bytes.argtypes = [_i] * 4
+_lib.ddg_conv3x3_packed_bytes.restype = _sz
+_lib.ddg_conv3x3_pack.argtypes = [_vp, _vp, _i, _vp]
+_lib.ddg_conv3x3_packed.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_bn_fwd_noalloc.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_sgd_update.argtypes = [_i, _vp, _vp, _vp, _vp, _sz, _f, _f, _f, _vp]
 
@@ -187,6 +192,18 @@ def _ok(rc):
 
 def tensor_core_path(B, H, W, Cin, Cout, stride):
     return _lib.ddg_tensor_core_path(B, H, W, Cin, Cout, stride)
+
+
+def conv3x3_packed_bytes(B, H, W, C):
+    return _lib.ddg_conv3x3_packed_bytes(B, H, W, C)
+
+
+def conv3x3_pack(w, packed, C, stream=None):
+    _ok(_lib.ddg_conv3x3_pack(_ptr(w), _ptr(packed), C, stream))
+
+
+def conv3x3_packed(dgrad, src, w, packed, dst, B, H, W, C, stream=None):
+    _ok(_lib.ddg_conv3x3_packed(int(dgrad), _ptr(src), _ptr(w), _ptr(packed), _ptr(dst), B, H, W, C, stream))
 
 
 def conv3x3_fwd(prec, x, w, y, B, H, W, Cin, Cout, stride, stream=None):

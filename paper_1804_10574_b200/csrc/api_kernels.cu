@@ -53,6 +53,27 @@ ddg_status ddg_conv3x3_dgrad(int precision, const void *dy, const void *w, void 
     return done();
 }
 
+size_t ddg_conv3x3_packed_bytes(int B, int H, int W, int C) {
+    if (init_once() != DDG_OK || !conv_tc_supported(B, H, W, C, C, 1)) return 0;
+    return tc_packed_bytes(C);
+}
+
+ddg_status ddg_conv3x3_pack(const void *w, void *packed, int C, void *stream) {
+    if (!w || !packed) return DDG_ERR_INVALID_ARG;
+    if (C != 16 && C != 32 && C != 64) return DDG_ERR_UNSUPPORTED;
+    launch_pack_one(w, packed, C, (cudaStream_t)stream);
+    return done();
+}
+
+ddg_status ddg_conv3x3_packed(int dgrad, const void *src, const void *w, const void *packed, void *dst, int B, int H,
+                              int W, int C, void *stream) {
+    if (!src || !w || !packed || !dst) return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_supported(B, H, W, C, C, 1)) return DDG_ERR_UNSUPPORTED;
+    launch_conv_tc(dgrad ? 1 : 0, src, w, packed, dst, B, H, W, C, Shortcut{}, (cudaStream_t)stream);
+    return done();
+}
+
 size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride) {
     if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return 0;
     size_t a = conv_wgrad_scratch_elems(B, H, W, Cin, Cout, stride), b = wgrad_tc_scratch_elems();

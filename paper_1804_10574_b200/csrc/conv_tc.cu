@@ -12,8 +12,8 @@
 // neighbouring pixels, y[h][w] = P_0[h][w-1] + P_1[h][w] + P_2[h][w+1], with warp shuffles (a warp holds whole image
 // rows; the image border contributes zero).  The filter-row shift costs nothing: the three rows read the same TMA box
 // at offsets of 0, W and 2W pixels, which are whole swizzle periods, so only the descriptor start address moves.
-// Warp roles: warp 0 issues TMA, warp 1 issues MMAs, warps 2-5 drain TMEM, combine, add the shortcut gradient where
-// asked, convert to bf16 and store.  Two TMEM accumulator stages let the epilogue of tile i overlap the MMAs of tile
+// Warp roles: warp 0 issues TMA, warp 1 issues MMAs, warps 2-9 (two groups, one per accumulator stage) drain TMEM,
+// combine, add the shortcut gradient where asked, convert to bf16 and store.  Two TMEM accumulator stages let the epilogue of tile i overlap the MMAs of tile
 // i+1.  Every mbarrier wait is bounded: when one runs out, the CTA raises an error word that the host reads at its
 // next sync point, and leaves.
 #include <cuda.h>
@@ -31,7 +31,8 @@ namespace ddg {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;   // convolution: TMA warp, MMA warp, two groups of four epilogue warps
+constexpr int kWgThreads = 192;   // weight gradient: TMA warp, MMA warp, four epilogue warps
 constexpr unsigned kSpinLimit = 1u << 24;  // bounded waits: ~ a second at worst, then the CTA gives up
 
 __device__ int g_tc_error = 0;  // 0 = fine; otherwise the code of the wait that ran out
@@ -131,7 +132,8 @@ template <int C> struct TcCfg {
     static constexpr int w_row_tile_bytes = 3 * C * C * 2;            // one filter row: [3C rows = (kx, out ch)][C]
     static constexpr int w_bytes = 3 * w_row_tile_bytes;
     static constexpr int tile_bytes = kTileM * C * 2;
-    static constexpr int tmem_cols = C == 16 ? 128 : (C == 32 ? 256 : 512);  // two stages of 3C columns, power of two
+    static constexpr int acc_stages = C == 64 ? 2 : 4;                // TMEM accumulator stages of 3C columns each
+    static constexpr int tmem_cols = C == 16 ? 256 : 512;             // acc_stages * 3C rounded up to a power of two
 };
 
 // byte offset of element (row, k) inside a swizzled tile whose rows are row_bytes wide
@@ -194,6 +196,15 @@ __global__ void pack_filters_kernel(const bf16 *__restrict__ wver, uint8_t *__re
     else pack_one<64>(wver + j.src_off, packed + j.dst_off, i);
 }
 
+// the same for one convolution, job passed by value
+__global__ void pack_one_filter_kernel(const bf16 *__restrict__ w, uint8_t *__restrict__ packed, int C) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 9 * C * C) return;
+    if (C == 16) pack_one<16>(w, packed, i);
+    else if (C == 32) pack_one<32>(w, packed, i);
+    else pack_one<64>(w, packed, i);
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // forward / input gradient.
 //   slab == 1 (tile inside one image): one TMA box of (rows+2) image rows per tile; filter row ky reads it at an offset
@@ -215,21 +226,21 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     const ConvSmem plan = conv_smem_plan<C>(n_stages, stage_bytes);
     const uint32_t w_base = base + plan.w_off, a_base = base + plan.a_off;
     uint8_t *tail = smem + plan.tail_off;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[2], tempty[2], wbar
-    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 5) * 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 5) * 8 + 8);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[4], tempty[4], wbar
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 9) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 9) * 8 + 8);
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + a); };
-    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
-    const uint32_t w_bar = bar0 + 8u * (2 * kMaxStages + 4);
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 4 + a); };
+    const uint32_t w_bar = bar0 + 8u * (2 * kMaxStages + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        for (int a = 0; a < Cfg::acc_stages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
         mbar_init(w_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -292,8 +303,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
             bool ok = true;
             if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, abort_flag, 5);
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-                const int a = it & 1;
-                const uint32_t aph = (it >> 1) & 1u;
+                const int a = it % Cfg::acc_stages;
+                const uint32_t aph = (it / Cfg::acc_stages) & 1u;
                 ok = mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, 2);
                 if (!ok) break;
                 tc_fence_after();
@@ -320,12 +331,14 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
         }
     } else {
         // ---------------- epilogue: TMEM -> registers -> bf16 -> global ----------------
+        // Two groups of four warps; group g drains every other tile, so two epilogues overlap.
         const int q = warp & 3;  // a warp may only touch TMEM lanes [32*(warp%4), +32)
-        int it = 0;
+        const int grp = (warp - 2) >> 2;
+        int it = grp;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-            const int a = it & 1;
-            const uint32_t aph = (it >> 1) & 1u;
+        for (int tile = blockIdx.x + grp * gridDim.x; tile < n_tiles && ok; tile += 2 * gridDim.x, it += 2) {
+            const int a = it % Cfg::acc_stages;
+            const uint32_t aph = (it / Cfg::acc_stages) & 1u;
             ok = mbar_wait(tfull_bar(a), aph, abort_flag, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -400,7 +413,7 @@ constexpr int kWgMaxChunks = 148;
 struct WgSmem { uint32_t tail_off; };
 
 template <int C>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kWgThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 float *__restrict__ part, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles, int slab,
                 int n_stages, int x_box_bytes, int tmem_cols) {
@@ -641,7 +654,7 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int max_chunks = slab ? (C == 16 ? 148 : 74) : 49;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
-    wgrad_tc_kernel<C><<<dim3(chunks, slab ? 1 : 3), kTcThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s>>>(
+    wgrad_tc_kernel<C><<<dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s>>>(
         mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
     wgrad_tc_fold_kernel<<<ceil_div(9 * C * C, 64), 256, 0, s>>>(scratch, dw, chunks, C);
     return 2;
@@ -676,6 +689,11 @@ int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, in
     if (n_jobs == 0) return 0;
     pack_filters_kernel<<<ceil_div(total_elems, 256), 256, 0, s>>>((const bf16 *)wver, (uint8_t *)packed,
                                                                   (const PackJob *)jobs_dev, n_jobs, total_elems);
+    return 1;
+}
+
+int launch_pack_one(const void *w, void *packed, int C, cudaStream_t s) {
+    pack_one_filter_kernel<<<ceil_div(9 * C * C, 256), 256, 0, s>>>((const bf16 *)w, (uint8_t *)packed, C);
     return 1;
 }
 

@@ -20,6 +20,7 @@ int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed
 size_t tc_packed_bytes(int C);
 // One launch that re-arranges the filters of many convolutions of one weight version.
 struct PackJobHost { long src_off; long dst_off; int C; int first_elem; };  // element offset in wver, byte offset in packed
+int launch_pack_one(const void *w, void *packed, int C, cudaStream_t s);
 int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,
                         cudaStream_t s);
 

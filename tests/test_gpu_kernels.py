@@ -129,3 +129,25 @@ def test_tensor_core_path_takes_the_resnet_shapes():
         assert binding.tensor_core_path(B, H, W, C, C, 1) & 1, (B, H, W, C)
     assert binding.tensor_core_path(128, 32, 32, 16, 32, 2) & 1 == 0      # stride 2 stays on CUDA cores
     assert binding.tensor_core_path(9, 8, 8, 64, 64, 1) & 1 == 0          # 576 pixels: not whole 128-pixel tiles
+
+
+@pytest.mark.parametrize("shape", [(3, 32, 32, 16), (5, 16, 16, 32), (128, 8, 8, 64)], ids=lambda s: "x".join(map(str, s)))
+def test_conv3x3_with_prearranged_filter_matches_oracle(shape):
+    """The filter-image path the training step uses (pack once, bulk-copied by the kernel), forward and dgrad."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = shape
+    rng = np.random.default_rng(13)
+    x, xh = to_dev(rng.standard_normal((B, C, H, W)), 1)
+    dy, dyh = to_dev(rng.standard_normal((B, C, H, W)), 1)
+    w = torch.from_numpy(rng.standard_normal((C, C, 3, 3)) * np.sqrt(2.0 / (9 * C))).to(torch.bfloat16)
+    wh = w.to(torch.float64).numpy()
+    w = w.cuda()
+    pk = torch.empty(binding.conv3x3_packed_bytes(B, H, W, C), dtype=torch.uint8, device="cuda")
+    assert pk.numel() == 2 * 9 * C * C * 2
+    binding.conv3x3_pack(w, pk, C)
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    binding.conv3x3_packed(0, x, w, pk, y, B, H, W, C)
+    binding.conv3x3_packed(1, dy, w, pk, dx, B, H, W, C)
+    torch.cuda.synchronize()
+    assert rel(from_dev(y), orc.conv3x3_forward(xh, wh, 1)) < TOL[1]
+    assert rel(from_dev(dx), orc.conv3x3_backward(xh, wh, dyh, 1)[0]) < TOL[1]
