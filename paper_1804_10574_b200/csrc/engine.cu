@@ -60,6 +60,10 @@ struct Module {
     cudaStream_t stream = nullptr;
     bool own_stream = false;
     cudaEvent_t ev_fwd = nullptr, ev_bwd = nullptr, ev_join = nullptr;
+    // weight gradients run beside the error-gradient chain, on a second stream of the module
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_side[4] = {nullptr, nullptr, nullptr, nullptr};
+    char *dyring[4] = {nullptr, nullptr, nullptr, nullptr};  // conv-output error gradients, kept until their wgrad ran
 };
 
 }  // namespace
@@ -231,6 +235,25 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
     const char *cur = (k == c->K - 1) ? (const char *)c->dlogits : c->mods[k + 1].delta_out[(t + 1) % 2];
     int cur_tmp = -1;
     auto pick = [&](int e1, int e2) { for (int i = 0; i < 3; ++i) if (i != e1 && i != e2) return i; return 0; };
+    // The weight gradient of a convolution needs only (layer input, dy); nothing on the way down to the module input
+    // waits for it.  It runs on the module's side stream; dy lives in a ring of four buffers so that the chain can move
+    // on, and the chain only waits when it comes back to a buffer whose weight gradient has not finished.
+    int dy_i = 0, last_side = -1;
+    bool ring_used[4] = {false, false, false, false};
+    auto ring_next = [&]() -> int {
+        const int j = dy_i++ & 3;
+        if (ring_used[j]) cudaStreamWaitEvent(s, m.ev_side[j], 0);
+        return j;
+    };
+    auto side_wgrad = [&](int j, const void *x_in, const void *dy, float *gwp, int H, int W, int Ci, int Co, int st) {
+        cudaEventRecord(m.ev_fork, s);
+        cudaStreamWaitEvent(m.side, m.ev_fork, 0);
+        n += conv_wgrad(c, m, x_in, dy, gwp, H, W, Ci, Co, st, m.side);
+        cudaEventRecord(m.ev_side[j], m.side);
+        ring_used[j] = true;
+        last_side = j;
+    };
+    auto side_join = [&]() { if (last_side >= 0) cudaStreamWaitEvent(s, m.ev_side[last_side], 0); };
     for (int l = m.last; l >= m.first; --l) {
         LayerPlan &L = c->layers[l];
         const char *w = wv + L.p_off * es;
@@ -260,6 +283,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
             }
             if (need_dx)
                 n += conv_dgrad(c, dy, w, pkp(L.pk1), dst, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, Shortcut{}, s);
+            side_join();  // this one runs on the chain's own stream and shares the weight-gradient scratch
             n += conv_wgrad(c, m, in, dy, gw, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, s);
             break;
         }
@@ -289,14 +313,19 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
             const long npix = (long)B * L.Hout * L.Wout;
             // the two scratch temporaries are the ones not holding the incoming error gradient
             const int tA = pick(cur_tmp, -1), tB = pick(cur_tmp, tA);
-            char *dy2 = m.tmp[tA], *da1 = m.tmp[tB], *dy1 = m.tmp[tA];
+            (void)tA;
+            const int j2 = ring_next();
+            char *dy2 = m.dyring[j2], *da1 = m.tmp[tB];
             n += launch_bn_bwd_reduce(c->prec, cur, out, y2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, m.bn_scratch, npix, Co,
                                       1, s);
             n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s);
+            side_wgrad(j2, a1, dy2, gw2, L.Hout, L.Wout, Co, Co, 1);
             n += conv_dgrad(c, dy2, w2, pkp(L.pk2), da1, L.Hout, L.Wout, Co, Co, 1, Shortcut{}, s);
-            n += conv_wgrad(c, m, a1, dy2, gw2, L.Hout, L.Wout, Co, Co, 1, s);
+            const int j1 = ring_next();
+            char *dy1 = m.dyring[j1];
             n += launch_bn_bwd_reduce(c->prec, da1, a1, y1, stt, stt + Co, gg1, gb1, m.bn_scratch, npix, Co, 1, s);
             n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
+            side_wgrad(j1, in, dy1, gw1, L.Hin, L.Win, Ci, Co, st);
             if (need_dx) {
                 Shortcut sc{};
                 sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
@@ -305,13 +334,13 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
                 n += conv_dgrad(c, dy1, w1, pkp(L.pk1), dx, L.Hin, L.Win, Ci, Co, st, sc, s);
                 if (!mod_first) { dst = dx; dst_tmp = tB; }
             }
-            n += conv_wgrad(c, m, in, dy1, gw1, L.Hin, L.Win, Ci, Co, st, s);
             break;
         }
         }
         cur = dst;
         cur_tmp = dst_tmp;
     }
+    side_join();  // the update that follows reads every gradient of the module
     return n;
 }
 
@@ -491,6 +520,10 @@ void ddg_destroy(ddg_ctx *ctx) {
         cudaFree(m.packed); cudaFree(m.pack_jobs);
         cudaFree(m.arena); cudaFree(m.w); cudaFree(m.v); cudaFree(m.m2); cudaFree(m.g); cudaFree(m.wver);
         for (char *p : m.tmp) cudaFree(p);
+        for (char *p : m.dyring) cudaFree(p);
+        if (m.side) { cudaStreamSynchronize(m.side); cudaStreamDestroy(m.side); }
+        if (m.ev_fork) cudaEventDestroy(m.ev_fork);
+        for (auto e : m.ev_side) if (e) cudaEventDestroy(e);
         cudaFree(m.bn_scratch); cudaFree(m.wg_scratch);
         cudaFree(m.delta_out[0]); cudaFree(m.delta_out[1]);
         if (m.ev_fwd) cudaEventDestroy(m.ev_fwd);
@@ -640,6 +673,10 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
         CU(cudaMalloc(&m.wver, pn * es * m.R));
         CU(cudaMemset(m.wver, 0, pn * es * m.R));
         for (auto &p : m.tmp) CU(cudaMalloc(&p, m.tmp_bytes));
+        for (auto &p : m.dyring) CU(cudaMalloc(&p, m.tmp_bytes));
+        CU(cudaStreamCreateWithFlags(&m.side, cudaStreamNonBlocking));
+        CU(cudaEventCreateWithFlags(&m.ev_fork, cudaEventDisableTiming));
+        for (auto &e : m.ev_side) CU(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
         size_t bn_max = 0, wg_max = 0;
         for (int l = m.first; l <= m.last; ++l) {
             LayerPlan &L = c->layers[l];
