@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace ddg {
 
 typedef __nv_bfloat16 bf16;
@@ -68,5 +70,31 @@ __device__ __forceinline__ float warp_max(float v) {
 }
 
 static inline int ceil_div(long a, long b) { return (int)((a + b - 1) / b); }
+
+// Programmatic dependent launch.  Every kernel of the library is launched with programmatic stream serialisation: the
+// next kernel of the stream may be scheduled while this one is still running, so that its launch latency and its
+// prologue overlap this kernel's tail.  The contract that keeps this correct: every kernel executes pdl_wait() before
+// its first access to global memory that an earlier kernel may write or still read; the wait returns when all
+// preceding kernels of the stream have completed and their writes are visible.  pdl_launch() tells the scheduler that
+// the next kernel may start being placed.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+bool pdl_enabled();  // defined in engine.cu; DDG_PDL=0 in the environment switches the launch attribute off
+
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 }  // namespace ddg

@@ -182,6 +182,8 @@ template <int C> __device__ __forceinline__ void pack_one(const bf16 *w, uint8_t
 
 __global__ void pack_filters_kernel(const bf16 *__restrict__ wver, uint8_t *__restrict__ packed,
                                     const PackJob *__restrict__ jobs, int n_jobs, int total) {
+    pdl_launch();
+    pdl_wait();
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= total) return;
     int lo = 0, hi = n_jobs - 1;  // last job whose first element is <= e
@@ -198,6 +200,8 @@ __global__ void pack_filters_kernel(const bf16 *__restrict__ wver, uint8_t *__re
 
 // the same for one convolution, job passed by value
 __global__ void pack_one_filter_kernel(const bf16 *__restrict__ w, uint8_t *__restrict__ packed, int C) {
+    pdl_launch();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= 9 * C * C) return;
     if (C == 16) pack_one<16>(w, packed, i);
@@ -251,6 +255,10 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // launch latency, barrier set-up and the TMEM allocation above overlap the previous kernel's tail; nothing before
+    // this point touches global memory
+    pdl_launch();
+    pdl_wait();
     if (w_packed == nullptr) {
         // filter in canonical order: stage it here as 9 K-major [C rows = output channel of this pass][C] tiles
         for (int i = threadIdx.x; i < 9 * C * C; i += kTcThreads) {
@@ -446,6 +454,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    pdl_launch();
+    pdl_wait();  // everything above is on-chip set-up; global memory is first touched below
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -551,6 +561,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 // dw[co][ci][tap] = sum over chunks of part[chunk][tap][ci][co].  64 outputs per CTA, four threads per output: thread g
 // adds chunks g, g+4, ... (four independent loads in flight per thread), the four sums are combined in a fixed order.
 __global__ void __launch_bounds__(256) wgrad_tc_fold_kernel(const float *__restrict__ part, float *__restrict__ dw, int chunks, int C) {
+    pdl_launch();
+    pdl_wait();
     __shared__ float sm[4][64];
     const int total = 9 * C * C;
     const int o = threadIdx.x & 63, g = threadIdx.x >> 6;
@@ -632,8 +644,7 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     if (n_stages > kMaxStages) n_stages = kMaxStages;
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
-    conv3x3_tc_kernel<C><<<grid, kTcThreads, conv_smem_bytes<C>(n_stages, stage_bytes), s>>>(
-        map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
+    launch_k(conv3x3_tc_kernel<C>, grid, kTcThreads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
         stage_bytes, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr);
     return 1;
 }
@@ -654,9 +665,8 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int max_chunks = slab ? (C == 16 ? 148 : 74) : 49;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
-    wgrad_tc_kernel<C><<<dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s>>>(
-        mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
-    wgrad_tc_fold_kernel<<<ceil_div(9 * C * C, 64), 256, 0, s>>>(scratch, dw, chunks, C);
+    launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
+    launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C);
     return 2;
 }
 
@@ -687,13 +697,13 @@ int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed
 int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,
                         cudaStream_t s) {
     if (n_jobs == 0) return 0;
-    pack_filters_kernel<<<ceil_div(total_elems, 256), 256, 0, s>>>((const bf16 *)wver, (uint8_t *)packed,
+    launch_k(pack_filters_kernel, ceil_div(total_elems, 256), 256, 0, s, (const bf16 *)wver, (uint8_t *)packed,
                                                                   (const PackJob *)jobs_dev, n_jobs, total_elems);
     return 1;
 }
 
 int launch_pack_one(const void *w, void *packed, int C, cudaStream_t s) {
-    pack_one_filter_kernel<<<ceil_div(9 * C * C, 256), 256, 0, s>>>((const bf16 *)w, (uint8_t *)packed, C);
+    launch_k(pack_one_filter_kernel, ceil_div(9 * C * C, 256), 256, 0, s, (const bf16 *)w, (uint8_t *)packed, C);
     return 1;
 }
 

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -499,6 +500,10 @@ ddg_status sync_all(ddg_ctx *ctx) {
 }  // namespace
 
 namespace ddg {
+bool pdl_enabled() {
+    static const bool on = [] { const char *e = getenv("DDG_PDL"); return !(e && e[0] == '0'); }();
+    return on;
+}
 // lets the other translation units leave a message for ddg_last_error(NULL)
 void set_global_error(const char *msg) { g_create_error = msg; }
 }  // namespace ddg

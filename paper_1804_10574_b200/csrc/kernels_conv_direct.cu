@@ -23,6 +23,8 @@ template <typename T, int DGRAD>
 __global__ void __launch_bounds__(kConvThreads)
 conv3x3_direct_kernel(const T *__restrict__ src, const T *__restrict__ w, T *__restrict__ dst, int B, int Hs, int Ws,
                       int Cs, int Hd, int Wd, int Cd, int stride, int relu, Shortcut sc) {
+    pdl_launch();
+    pdl_wait();
     extern __shared__ float wsm[];
     const int Cin = DGRAD ? Cd : Cs, Cout = DGRAD ? Cs : Cd;
     for (int i = threadIdx.x; i < 9 * Cs * Cd; i += blockDim.x) {
@@ -128,8 +130,7 @@ static void conv_direct_launch(const void *src, const void *w, void *dst, int B,
     const int groups = (Cd + kCdt - 1) / kCdt;
     const int pix_per_cta = kConvThreads / groups;
     const long npix = (long)B * Hd * Wd;
-    conv3x3_direct_kernel<T, DGRAD><<<ceil_div(npix, pix_per_cta), kConvThreads, smem, s>>>(
-        (const T *)src, (const T *)w, (T *)dst, B, Hs, Ws, Cs, Hd, Wd, Cd, stride, relu, sc);
+    launch_k(conv3x3_direct_kernel<T, DGRAD>, ceil_div(npix, pix_per_cta), kConvThreads, smem, s, (const T *)src, (const T *)w, (T *)dst, B, Hs, Ws, Cs, Hd, Wd, Cd, stride, relu, sc);
 }
 
 int conv_direct_init() {
@@ -185,6 +186,8 @@ __global__ void __launch_bounds__(kWgThreads)
 conv3x3_wgrad_partial_kernel(const T *__restrict__ x, const T *__restrict__ dy,
                              typename AccOf<T>::type *__restrict__ part, int B, int H, int W, int Cin, int Ho, int Wo,
                              int Cout, int stride, int ci_per) {
+    pdl_launch();
+    pdl_wait();
     typedef typename AccOf<T>::type A;
     extern __shared__ float sm[];
     float *xs = sm;                         // [(W+2)][Cin] with a zero halo column on each side
@@ -238,6 +241,8 @@ conv3x3_wgrad_partial_kernel(const T *__restrict__ x, const T *__restrict__ dy,
 template <typename A>
 __global__ void conv3x3_wgrad_fold_kernel(const A *__restrict__ part, float *__restrict__ dw, int chunks, int Cin,
                                           int Cout) {
+    pdl_launch();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;  // index into [tap][ci][co]
     const int total = 9 * Cin * Cout;
     if (i >= total) return;
@@ -258,9 +263,9 @@ int launch_conv_wgrad_direct(int prec, const void *x, const void *dy, float *dw,
     dim3 grid(chunks, 3);
     DISPATCH_PREC(prec, {
         typedef typename AccOf<T>::type A;
-        conv3x3_wgrad_partial_kernel<T><<<grid, kWgThreads, smem, s>>>((const T *)x, (const T *)dy, (A *)scratch, B, H, W,
+        launch_k(conv3x3_wgrad_partial_kernel<T>, grid, kWgThreads, smem, s, (const T *)x, (const T *)dy, (A *)scratch, B, H, W,
                                                                      Cin, Ho, Wo, Cout, stride, ci_per);
-        conv3x3_wgrad_fold_kernel<A><<<ceil_div(9 * Cin * Cout, 256), 256, 0, s>>>((const A *)scratch, dw, chunks, Cin,
+        launch_k(conv3x3_wgrad_fold_kernel<A>, ceil_div(9 * Cin * Cout, 256), 256, 0, s, (const A *)scratch, dw, chunks, Cin,
                                                                                   Cout);
     });
     return 2;

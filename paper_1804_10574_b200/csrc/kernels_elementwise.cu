@@ -22,6 +22,8 @@ static constexpr float kBnEps = 1e-5f;
 // ------------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void shim_kernel(const float *__restrict__ x, T *__restrict__ out, int B, int C, int HW) {
+    pdl_launch();
+    pdl_wait();
     long i = (long)blockIdx.x * blockDim.x + threadIdx.x;  // (n, p)
     if (i >= (long)B * HW) return;
     long n = i / HW, p = i % HW;
@@ -30,7 +32,7 @@ __global__ void shim_kernel(const float *__restrict__ x, T *__restrict__ out, in
 
 int launch_shim(int prec, const float *x, void *out, int B, int C, int H, int W, cudaStream_t s) {
     long n = (long)B * H * W;
-    DISPATCH_PREC(prec, shim_kernel<T><<<ceil_div(n, kThreads), kThreads, 0, s>>>(x, (T *)out, B, C, H * W));
+    DISPATCH_PREC(prec, launch_k(shim_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, x, (T *)out, B, C, H * W));
     return 1;
 }
 
@@ -38,19 +40,23 @@ int launch_shim(int prec, const float *x, void *out, int B, int C, int H, int W,
 // ReLU
 // ------------------------------------------------------------------------------------------------------
 template <typename T> __global__ void relu_fwd_kernel(const T *x, T *y, size_t n) {
+    pdl_launch();
+    pdl_wait();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) { float v = to_f(x[i]); y[i] = from_f<T>(v > 0.f ? v : 0.f); }
 }
 template <typename T> __global__ void relu_bwd_kernel(const T *y, const T *dy, T *dx, size_t n) {
+    pdl_launch();
+    pdl_wait();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) dx[i] = to_f(y[i]) > 0.f ? dy[i] : from_f<T>(0.f);
 }
 int launch_relu_fwd(int prec, const void *x, void *y, size_t n, cudaStream_t s) {
-    DISPATCH_PREC(prec, relu_fwd_kernel<T><<<ceil_div(n, kThreads), kThreads, 0, s>>>((const T *)x, (T *)y, n));
+    DISPATCH_PREC(prec, launch_k(relu_fwd_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, (const T *)x, (T *)y, n));
     return 1;
 }
 int launch_relu_bwd(int prec, const void *y, const void *dy, void *dx, size_t n, cudaStream_t s) {
-    DISPATCH_PREC(prec, relu_bwd_kernel<T><<<ceil_div(n, kThreads), kThreads, 0, s>>>((const T *)y, (const T *)dy,
+    DISPATCH_PREC(prec, launch_k(relu_bwd_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, (const T *)y, (const T *)dy,
                                                                                       (T *)dx, n));
     return 1;
 }
@@ -59,6 +65,8 @@ int launch_relu_bwd(int prec, const void *y, const void *dy, void *dx, size_t n,
 // global mean pool: x [B][HW][C] -> y [B][C]
 // ------------------------------------------------------------------------------------------------------
 template <typename T> __global__ void avgpool_fwd_kernel(const T *x, T *y, int HW, int C) {
+    pdl_launch();
+    pdl_wait();
     typedef typename AccOf<T>::type A;
     __shared__ A sm[kThreads];
     const int n = blockIdx.x, lanes = blockDim.x / C;  // host guarantees C <= blockDim
@@ -75,6 +83,8 @@ template <typename T> __global__ void avgpool_fwd_kernel(const T *x, T *y, int H
     }
 }
 template <typename T> __global__ void avgpool_bwd_kernel(const T *dy, T *dx, int HW, int C, size_t n) {
+    pdl_launch();
+    pdl_wait();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     size_t b = i / ((size_t)HW * C);
@@ -83,12 +93,12 @@ template <typename T> __global__ void avgpool_bwd_kernel(const T *dy, T *dx, int
     dx[i] = from_a<T>((A)to_f(dy[b * C + c]) / (A)HW);
 }
 int launch_avgpool_fwd(int prec, const void *x, void *y, int B, int HW, int C, cudaStream_t s) {
-    DISPATCH_PREC(prec, avgpool_fwd_kernel<T><<<B, kThreads, 0, s>>>((const T *)x, (T *)y, HW, C));
+    DISPATCH_PREC(prec, launch_k(avgpool_fwd_kernel<T>, B, kThreads, 0, s, (const T *)x, (T *)y, HW, C));
     return 1;
 }
 int launch_avgpool_bwd(int prec, const void *dy, void *dx, int B, int HW, int C, cudaStream_t s) {
     size_t n = (size_t)B * HW * C;
-    DISPATCH_PREC(prec, avgpool_bwd_kernel<T><<<ceil_div(n, kThreads), kThreads, 0, s>>>((const T *)dy, (T *)dx, HW,
+    DISPATCH_PREC(prec, launch_k(avgpool_bwd_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, (const T *)dy, (T *)dx, HW,
                                                                                         C, n));
     return 1;
 }
@@ -99,6 +109,8 @@ int launch_avgpool_bwd(int prec, const void *dy, void *dx, int B, int HW, int C,
 // one warp per output element y[b][o]
 template <typename T, typename TO>
 __global__ void fc_fwd_kernel(const T *x, const T *W, const T *bias, TO *y, int B, int in, int out, int relu) {
+    pdl_launch();
+    pdl_wait();
     long warp = ((long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int lane = threadIdx.x & 31;
     if (warp >= (long)B * out) return;
@@ -121,6 +133,8 @@ template <typename TO> __device__ __forceinline__ float masked_dy(const TO *y, c
 // dx[b][i] = sum_o dz[b][o] W[o][i]
 template <typename T, typename TO>
 __global__ void fc_dx_kernel(const T *W, const TO *y, const TO *dy, T *dx, int B, int in, int out, int relu) {
+    pdl_launch();
+    pdl_wait();
     long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long)B * in) return;
     typedef typename AccOf<T>::type A;
@@ -134,6 +148,8 @@ __global__ void fc_dx_kernel(const T *W, const TO *y, const TO *dy, T *dx, int B
 template <typename T, typename TO>
 __global__ void fc_dw_kernel(const T *x, const TO *y, const TO *dy, float *dW, float *db, int B, int in, int out,
                              int relu) {
+    pdl_launch();
+    pdl_wait();
     long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
     int cols = in + 1;
     if (idx >= (long)out * cols) return;
@@ -154,11 +170,11 @@ int launch_fc_fwd(int prec, const void *x, const void *W, const void *bias, void
     long threads = (long)B * out * 32;
     DISPATCH_PREC(prec, {
         if (out_f32)
-            fc_fwd_kernel<T, float><<<ceil_div(threads, kThreads), kThreads, 0, s>>>((const T *)x, (const T *)W,
+            launch_k(fc_fwd_kernel<T, float>, ceil_div(threads, kThreads), kThreads, 0, s, (const T *)x, (const T *)W,
                                                                                     (const T *)bias, (float *)y, B, in,
                                                                                     out, relu);
         else
-            fc_fwd_kernel<T, T><<<ceil_div(threads, kThreads), kThreads, 0, s>>>((const T *)x, (const T *)W,
+            launch_k(fc_fwd_kernel<T, T>, ceil_div(threads, kThreads), kThreads, 0, s, (const T *)x, (const T *)W,
                                                                                 (const T *)bias, (T *)y, B, in, out,
                                                                                 relu);
     });
@@ -169,15 +185,11 @@ int launch_fc_bwd(int prec, const void *x, const void *W, const void *y, const v
     int n = 0;
     DISPATCH_PREC(prec, {
         if (out_f32) {
-            if (dx) { fc_dx_kernel<T, float><<<ceil_div((long)B * in, kThreads), kThreads, 0, s>>>(
-                          (const T *)W, (const float *)y, (const float *)dy, (T *)dx, B, in, out, relu); ++n; }
-            fc_dw_kernel<T, float><<<ceil_div((long)out * (in + 1), kThreads), kThreads, 0, s>>>(
-                (const T *)x, (const float *)y, (const float *)dy, dW, db, B, in, out, relu);
+            if (dx) { launch_k(fc_dx_kernel<T, float>, ceil_div((long)B * in, kThreads), kThreads, 0, s, (const T *)W, (const float *)y, (const float *)dy, (T *)dx, B, in, out, relu); ++n; }
+            launch_k(fc_dw_kernel<T, float>, ceil_div((long)out * (in + 1), kThreads), kThreads, 0, s, (const T *)x, (const float *)y, (const float *)dy, dW, db, B, in, out, relu);
         } else {
-            if (dx) { fc_dx_kernel<T, T><<<ceil_div((long)B * in, kThreads), kThreads, 0, s>>>(
-                          (const T *)W, (const T *)y, (const T *)dy, (T *)dx, B, in, out, relu); ++n; }
-            fc_dw_kernel<T, T><<<ceil_div((long)out * (in + 1), kThreads), kThreads, 0, s>>>(
-                (const T *)x, (const T *)y, (const T *)dy, dW, db, B, in, out, relu);
+            if (dx) { launch_k(fc_dx_kernel<T, T>, ceil_div((long)B * in, kThreads), kThreads, 0, s, (const T *)W, (const T *)y, (const T *)dy, (T *)dx, B, in, out, relu); ++n; }
+            launch_k(fc_dw_kernel<T, T>, ceil_div((long)out * (in + 1), kThreads), kThreads, 0, s, (const T *)x, (const T *)y, (const T *)dy, dW, db, B, in, out, relu);
         }
     });
     return n + 1;
@@ -193,6 +205,8 @@ __device__ __forceinline__ double log_a(double v) { return log(v); }
 
 template <typename A>
 __global__ void softmax_ce_kernel(const float *logits, const int *labels, float *loss, float *dlogits, int B, int C) {
+    pdl_launch();
+    pdl_wait();
     __shared__ A wsum[32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
     A acc = 0;
@@ -219,8 +233,8 @@ __global__ void softmax_ce_kernel(const float *logits, const int *labels, float 
 }
 int launch_softmax_ce(int prec, const float *logits, const int *labels, float *loss, float *dlogits, int B, int C,
                       cudaStream_t s) {
-    if (prec == P_BF16) softmax_ce_kernel<float><<<1, 1024, 0, s>>>(logits, labels, loss, dlogits, B, C);
-    else softmax_ce_kernel<double><<<1, 1024, 0, s>>>(logits, labels, loss, dlogits, B, C);
+    if (prec == P_BF16) launch_k(softmax_ce_kernel<float>, 1, 1024, 0, s, logits, labels, loss, dlogits, B, C);
+    else launch_k(softmax_ce_kernel<double>, 1, 1024, 0, s, logits, labels, loss, dlogits, B, C);
     return 1;
 }
 
@@ -244,6 +258,8 @@ __global__ void __launch_bounds__(kThreads)
 bn_reduce_kernel(const T *__restrict__ x, const T *__restrict__ dout, const T *__restrict__ out,
                  const float *__restrict__ mean_in, const float *__restrict__ invstd_in, float *o0, float *o1,
                  float *scratch, long npix, int C, int relu) {
+    pdl_launch();
+    pdl_wait();
     typedef typename AccOf<T>::type A;
     __shared__ A sm[kThreads * VEC];
     __shared__ bool is_last;
@@ -333,11 +349,9 @@ int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *
     DISPATCH_PREC(prec, {
         if (vec_for<T>(C) > 1) {
             constexpr int V = Vec16<T>::N;
-            bn_reduce_kernel<T, V, 0><<<bn_grid(npix, kThreads / (C / V)), kThreads, 0, s>>>(
-                (const T *)x, nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
+            launch_k(bn_reduce_kernel<T, V, 0>, bn_grid(npix, kThreads / (C / V)), kThreads, 0, s, (const T *)x, nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
         } else {
-            bn_reduce_kernel<T, 1, 0><<<bn_grid(npix, kThreads / C), kThreads, 0, s>>>(
-                (const T *)x, nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
+            launch_k(bn_reduce_kernel<T, 1, 0>, bn_grid(npix, kThreads / C), kThreads, 0, s, (const T *)x, nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
         }
     });
     return 1;
@@ -349,11 +363,9 @@ int launch_bn_bwd_reduce(int prec, const void *dout, const void *out, const void
     DISPATCH_PREC(prec, {
         if (vec_for<T>(C) > 1) {
             constexpr int V = Vec16<T>::N;
-            bn_reduce_kernel<T, V, 1><<<bn_grid(npix, kThreads / (C / V)), kThreads, 0, s>>>(
-                (const T *)x, (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
+            launch_k(bn_reduce_kernel<T, V, 1>, bn_grid(npix, kThreads / (C / V)), kThreads, 0, s, (const T *)x, (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
         } else {
-            bn_reduce_kernel<T, 1, 1><<<bn_grid(npix, kThreads / C), kThreads, 0, s>>>(
-                (const T *)x, (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
+            launch_k(bn_reduce_kernel<T, 1, 1>, bn_grid(npix, kThreads / C), kThreads, 0, s, (const T *)x, (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
         }
     });
     return 1;
@@ -365,6 +377,8 @@ __global__ void __launch_bounds__(kThreads)
 bn_apply_kernel(const T *__restrict__ x, const T *__restrict__ gamma, const T *__restrict__ beta,
                 const float *__restrict__ mean, const float *__restrict__ invstd, Shortcut sc, T *__restrict__ y,
                 long nvec, int H, int W, int C, int relu) {
+    pdl_launch();
+    pdl_wait();
     long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= nvec) return;
     const int groups = C / VEC;
@@ -406,12 +420,10 @@ int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta
         constexpr int V = Vec16<T>::N;
         if (C % V == 0 && (sc.mode != 2 || sc.c_small % V == 0)) {
             long nvec = npix * (C / V);
-            bn_apply_kernel<T, V><<<ceil_div(nvec, kThreads), kThreads, 0, s>>>(
-                (const T *)x, (const T *)gamma, (const T *)beta, mean, invstd, sc, (T *)y, nvec, H, W, C, relu);
+            launch_k(bn_apply_kernel<T, V>, ceil_div(nvec, kThreads), kThreads, 0, s, (const T *)x, (const T *)gamma, (const T *)beta, mean, invstd, sc, (T *)y, nvec, H, W, C, relu);
         } else {
             long nvec = npix * C;
-            bn_apply_kernel<T, 1><<<ceil_div(nvec, kThreads), kThreads, 0, s>>>(
-                (const T *)x, (const T *)gamma, (const T *)beta, mean, invstd, sc, (T *)y, nvec, H, W, C, relu);
+            launch_k(bn_apply_kernel<T, 1>, ceil_div(nvec, kThreads), kThreads, 0, s, (const T *)x, (const T *)gamma, (const T *)beta, mean, invstd, sc, (T *)y, nvec, H, W, C, relu);
         }
     });
     return 1;
@@ -424,6 +436,8 @@ bn_bwd_apply_kernel(const T *__restrict__ dout, const T *__restrict__ out, const
                     const T *__restrict__ gamma, const float *__restrict__ mean, const float *__restrict__ invstd,
                     const float *__restrict__ dgamma, const float *__restrict__ dbeta, T *__restrict__ dx, long nvec,
                     long npix, int C, int relu) {
+    pdl_launch();
+    pdl_wait();
     long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= nvec) return;
     const int groups = C / VEC;
@@ -456,13 +470,11 @@ int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void 
         constexpr int V = Vec16<T>::N;
         if (C % V == 0) {
             long nvec = npix * (C / V);
-            bn_bwd_apply_kernel<T, V><<<ceil_div(nvec, kThreads), kThreads, 0, s>>>(
-                (const T *)dout, (const T *)out, (const T *)x, (const T *)gamma, mean, invstd, dgamma, dbeta, (T *)dx,
+            launch_k(bn_bwd_apply_kernel<T, V>, ceil_div(nvec, kThreads), kThreads, 0, s, (const T *)dout, (const T *)out, (const T *)x, (const T *)gamma, mean, invstd, dgamma, dbeta, (T *)dx,
                 nvec, npix, C, relu);
         } else {
             long nvec = npix * C;
-            bn_bwd_apply_kernel<T, 1><<<ceil_div(nvec, kThreads), kThreads, 0, s>>>(
-                (const T *)dout, (const T *)out, (const T *)x, (const T *)gamma, mean, invstd, dgamma, dbeta, (T *)dx,
+            launch_k(bn_bwd_apply_kernel<T, 1>, ceil_div(nvec, kThreads), kThreads, 0, s, (const T *)dout, (const T *)out, (const T *)x, (const T *)gamma, mean, invstd, dgamma, dbeta, (T *)dx,
                 nvec, npix, C, relu);
         }
     });
@@ -476,6 +488,8 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 update_kernel(float *__restrict__ w, float *__restrict__ v, float *__restrict__ m2, const float *__restrict__ g,
               T *__restrict__ wv, size_t n, UpdateArgs a) {
+    pdl_launch();
+    pdl_wait();
     size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= n) return;
     const bool full = (i + 4 <= n) && ((reinterpret_cast<uintptr_t>(w + i) & 15) == 0) &&
@@ -531,7 +545,7 @@ update_kernel(float *__restrict__ w, float *__restrict__ v, float *__restrict__ 
 int launch_update(int prec, float *w, float *v, float *m2, const float *g, void *wv, size_t n, UpdateArgs a,
                   cudaStream_t s) {
     if (n == 0) return 0;
-    DISPATCH_PREC(prec, update_kernel<T><<<ceil_div((n + 3) / 4, kThreads), kThreads, 0, s>>>(w, v, m2, g, (T *)wv, n, a));
+    DISPATCH_PREC(prec, launch_k(update_kernel<T>, ceil_div((n + 3) / 4, kThreads), kThreads, 0, s, w, v, m2, g, (T *)wv, n, a));
     return 1;
 }
 
@@ -552,6 +566,8 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
 }
 __global__ void fill_normal_kernel(float *dst, size_t n, float stddev, unsigned long long seed,
                                    unsigned long long stream_id) {
+    pdl_launch();
+    pdl_wait();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     unsigned long long h = mix64(mix64(seed ^ (stream_id * 0xd1342543de82ef95ull)) + i);
@@ -561,18 +577,20 @@ __global__ void fill_normal_kernel(float *dst, size_t n, float stddev, unsigned 
     dst[i] = stddev * sqrtf(-2.f * logf(u1)) * cospif(2.f * u2);
 }
 __global__ void fill_const_kernel(float *dst, size_t n, float v) {
+    pdl_launch();
+    pdl_wait();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) dst[i] = v;
 }
 int launch_fill_normal(float *dst, size_t n, float stddev, unsigned long long seed, unsigned long long stream_id,
                        cudaStream_t s) {
     if (n == 0) return 0;
-    fill_normal_kernel<<<ceil_div(n, kThreads), kThreads, 0, s>>>(dst, n, stddev, seed, stream_id);
+    launch_k(fill_normal_kernel, ceil_div(n, kThreads), kThreads, 0, s, dst, n, stddev, seed, stream_id);
     return 1;
 }
 int launch_fill_const(float *dst, size_t n, float v, cudaStream_t s) {
     if (n == 0) return 0;
-    fill_const_kernel<<<ceil_div(n, kThreads), kThreads, 0, s>>>(dst, n, v);
+    launch_k(fill_const_kernel, ceil_div(n, kThreads), kThreads, 0, s, dst, n, v);
     return 1;
 }
 

@@ -1,6 +1,6 @@
 """Per-kernel sweep over the ResNet-110 layer shapes through the single-kernel C-ABI entry points.
 
-    python -m paper_1804_10574_b200.kernel_sweep [--batch 1024] [--only NAME] [--iters 20] [--json]
+    python -m paper_1804_10574_b200.kernel_sweep [--batch 1024] [--only NAME] [--iters 20] [--json] [--warm]
 
 Times every kernel alone with CUDA events on its stream, flushing L2 between launches, and prints the algorithmic
 bytes and flops per launch against the measured HBM / bf16 tensor peaks (MEASURED_PEAKS.json at the repository root,
@@ -32,7 +32,10 @@ def timed(fn, iters, flush):
     ts = []
     s = torch.cuda.current_stream()
     for _ in range(iters):
-        flush.zero_()
+        if flush is not None:
+            flush.zero_()
+        else:
+            torch.cuda._sleep(200000)   # keeps the GPU busy without touching L2 while the host enqueues what follows
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(s)
         fn()
@@ -103,9 +106,11 @@ def main():
     ap.add_argument("--only", default="")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--json", action="store_true")
+    ap.add_argument("--warm", action="store_true", help="do not flush L2 between launches (operands as the previous "
+                    "kernel of a training step leaves them)")
     a = ap.parse_args()
     hbm, tf, src = peaks()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush = None if a.warm else torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     rows = []
     for name, fn, nbytes, flops, tc, _keep in cases(a.batch):
         if a.only and a.only not in name:
