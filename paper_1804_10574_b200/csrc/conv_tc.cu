@@ -132,8 +132,8 @@ template <int C> struct TcCfg {
     static constexpr int w_row_tile_bytes = 3 * C * C * 2;            // one filter row: [3C rows = (kx, out ch)][C]
     static constexpr int w_bytes = 3 * w_row_tile_bytes;
     static constexpr int tile_bytes = kTileM * C * 2;
-    static constexpr int acc_stages = C == 64 ? 2 : 4;                // TMEM accumulator stages of 3C columns each
-    static constexpr int tmem_cols = C == 16 ? 256 : 512;             // acc_stages * 3C rounded up to a power of two
+    static constexpr int acc_stages = 2;                              // TMEM accumulator stages of 3C columns each
+    static constexpr int tmem_cols = C == 16 ? 128 : (C == 32 ? 256 : 512);  // 2 * 3C rounded up to a power of two
 };
 
 // byte offset of element (row, k) inside a swizzled tile whose rows are row_bytes wide
@@ -627,7 +627,9 @@ bool get_map(const void *ptr, int B, int H, int W, int C, int rows, int imgs, CU
 }
 
 int g_num_sms = 148;
-constexpr int kSmemBudget = 200 * 1024;
+// Shared memory a CTA may take for its pipeline stages: about half an SM, so that kernels of two modules (streams) can
+// share an SM instead of queueing behind each other.
+constexpr int kSmemBudget = 100 * 1024;
 constexpr int kSmemMax = 227 * 1024;
 
 template <int C>
@@ -642,6 +644,7 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     const int stage_bytes = box_rows * imgs * W * C * 2;
     int n_stages = (kSmemBudget - (int)conv_smem_plan<C>(0, 0).a_off) / stage_bytes;
     if (n_stages > kMaxStages) n_stages = kMaxStages;
+    if (n_stages < 3) n_stages = 3;
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
     launch_k(conv3x3_tc_kernel<C>, grid, kTcThreads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
@@ -660,6 +663,7 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int stage_bytes = TcCfg<C>::tile_bytes + 3 * x_box_bytes;
     int n_stages = kSmemBudget / stage_bytes;
     if (n_stages > kMaxStages) n_stages = kMaxStages;
+    if (n_stages < 2) n_stages = 2;
     const int ncols = slab ? 9 * C : 3 * C;
     const int tmem_cols = ncols <= 64 ? 64 : (ncols <= 128 ? 128 : (ncols <= 256 ? 256 : 512));
     const int n_tiles = (int)((long)B * H * W / kTileM);

@@ -342,12 +342,145 @@ bn_reduce_kernel(const T *__restrict__ x, const T *__restrict__ dout, const T *_
     if (threadIdx.x == 0) *counter = 0u;
 }
 
+// Fast path of the per-channel reductions (C/VEC a power of two <= 32): 512-thread CTAs, at most one per SM; the
+// tensor is walked as a flat array of 16-byte vectors with a stride that is a multiple of the vectors per pixel, so a
+// thread always sees the same channels; four vectors per trip with all loads issued first.  Folding order is fixed:
+// lanes of a warp by xor-shuffles, warps of a CTA in index order, CTAs in index order by the last CTA to finish.
+static constexpr int kRedThreads = 512;
+
+template <typename T, int VEC, int MODE>
+__global__ void __launch_bounds__(kRedThreads)
+bn_reduce_fast_kernel(const T *__restrict__ x, const T *__restrict__ dout, const T *__restrict__ out,
+                      const float *__restrict__ mean_in, const float *__restrict__ invstd_in, float *o0, float *o1,
+                      float *scratch, long npix, int C, int relu) {
+    pdl_launch();
+    pdl_wait();
+    typedef typename AccOf<T>::type A;
+    constexpr int kWarps = kRedThreads / 32;
+    __shared__ A sm[kWarps][2 * 128];  // per-warp sums of the 2C values (C <= 128)
+    __shared__ bool is_last;
+    unsigned *counter = reinterpret_cast<unsigned *>(scratch);
+    A *part = reinterpret_cast<A *>(scratch + 32);
+    const int groups = C / VEC;
+    const long nvec = npix * groups;
+    const long tid = (long)blockIdx.x * kRedThreads + threadIdx.x, stride = (long)gridDim.x * kRedThreads;
+    const int grp = (int)(tid & (groups - 1)), c0 = grp * VEC;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    A s0[VEC], s1[VEC], mu[VEC], is[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        s0[j] = 0; s1[j] = 0;
+        mu[j] = MODE == 1 ? (A)mean_in[c0 + j] : (A)0;
+        is[j] = MODE == 1 ? (A)invstd_in[c0 + j] : (A)0;
+    }
+    for (long i0 = tid; i0 < nvec; i0 += 4 * stride) {
+        A xv[4][VEC], dv[4][VEC];
+        float ov[4][VEC];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long i = i0 + u * stride;
+            if (i < nvec) {
+                load_a<T, A, VEC>(x + i * VEC, xv[u]);
+                if (MODE == 1) {
+                    load_a<T, A, VEC>(dout + i * VEC, dv[u]);
+                    if (relu) load_f<T, VEC>(out + i * VEC, ov[u]);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (i0 + u * stride < nvec) {
+#pragma unroll
+                for (int j = 0; j < VEC; ++j) {
+                    if (MODE == 0) { s0[j] += xv[u][j]; s1[j] += xv[u][j] * xv[u][j]; }
+                    else {
+                        A d = dv[u][j];
+                        if (relu && !(ov[u][j] > 0.f)) d = 0;
+                        s0[j] += d; s1[j] += d * (xv[u][j] - mu[j]) * is[j];
+                    }
+                }
+            }
+        }
+    }
+    // lanes of a warp that hold the same channels: lane ids equal modulo `groups`
+    for (int o = 16; o >= groups; o >>= 1) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+            s0[j] += __shfl_xor_sync(0xffffffffu, s0[j], o);
+            s1[j] += __shfl_xor_sync(0xffffffffu, s1[j], o);
+        }
+    }
+    if (lane < groups) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) { sm[warp][c0 + j] = s0[j]; sm[warp][C + c0 + j] = s1[j]; }
+    }
+    __syncthreads();
+    if (threadIdx.x < 2 * C) {
+        A t = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) t += sm[w][threadIdx.x];
+        part[(size_t)blockIdx.x * 2 * C + threadIdx.x] = t;
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    __shared__ double fold[kRedThreads];
+    const int nval = 2 * C, ways = kRedThreads / nval;
+    const int v = threadIdx.x % nval, way = threadIdx.x / nval;
+    double acc = 0.0;
+    if (way < ways) {
+        double a4[4] = {0.0, 0.0, 0.0, 0.0};
+        unsigned i = way;
+        for (; i + 3 * ways < gridDim.x; i += 4 * ways) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) a4[u] += (double)__ldcg(part + (size_t)(i + u * ways) * nval + v);
+        }
+        for (; i < gridDim.x; i += ways) a4[0] += (double)__ldcg(part + (size_t)i * nval + v);
+        acc = (a4[0] + a4[1]) + (a4[2] + a4[3]);
+    }
+    fold[threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.x < C) {
+        const int c = threadIdx.x;
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < ways; ++w) { a += fold[w * nval + c]; b += fold[w * nval + C + c]; }
+        if (MODE == 0) {
+            double m = a / (double)npix, var = b / (double)npix - m * m;
+            if (var < 0.0) var = 0.0;
+            o0[c] = (float)m;
+            o1[c] = (float)(1.0 / sqrt(var + (double)kBnEps));
+        } else {
+            o0[c] = (float)a;  // dbeta
+            o1[c] = (float)b;  // dgamma
+        }
+    }
+    if (threadIdx.x == 0) *counter = 0u;
+}
+
+static bool red_fast_ok(int C, int V) {
+    if (C % V != 0 || C > 128) return false;
+    const int groups = C / V;
+    return (groups & (groups - 1)) == 0 && groups <= 32;
+}
+static int red_fast_grid(long nvec) {
+    long g = (nvec + 4L * kRedThreads - 1) / (4L * kRedThreads);
+    if (g > 148) g = 148;
+    return (int)(g < 1 ? 1 : g);
+}
+
 template <typename T> static int vec_for(int C) { return (C % Vec16<T>::N == 0) ? Vec16<T>::N : 1; }
 
 int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *scratch, long npix, int C,
                     cudaStream_t s) {
     DISPATCH_PREC(prec, {
-        if (vec_for<T>(C) > 1) {
+        if (red_fast_ok(C, Vec16<T>::N)) {
+            constexpr int V = Vec16<T>::N;
+            launch_k(bn_reduce_fast_kernel<T, V, 0>, red_fast_grid(npix * (C / V)), kRedThreads, 0, s, (const T *)x, nullptr,
+                     nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
+        } else if (vec_for<T>(C) > 1) {
             constexpr int V = Vec16<T>::N;
             launch_k(bn_reduce_kernel<T, V, 0>, bn_grid(npix, kThreads / (C / V)), kThreads, 0, s, (const T *)x, nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
         } else {
@@ -361,7 +494,11 @@ int launch_bn_bwd_reduce(int prec, const void *dout, const void *out, const void
                          const float *invstd, float *dgamma, float *dbeta, float *scratch, long npix, int C, int relu,
                          cudaStream_t s) {
     DISPATCH_PREC(prec, {
-        if (vec_for<T>(C) > 1) {
+        if (red_fast_ok(C, Vec16<T>::N)) {
+            constexpr int V = Vec16<T>::N;
+            launch_k(bn_reduce_fast_kernel<T, V, 1>, red_fast_grid(npix * (C / V)), kRedThreads, 0, s, (const T *)x,
+                     (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
+        } else if (vec_for<T>(C) > 1) {
             constexpr int V = Vec16<T>::N;
             launch_k(bn_reduce_kernel<T, V, 1>, bn_grid(npix, kThreads / (C / V)), kThreads, 0, s, (const T *)x, (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
         } else {
