@@ -87,7 +87,7 @@ ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float
     if (init_once() != DDG_OK) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     if (precision == DDG_BF16 && wgrad_tc_supported(B, H, W, Cin, Cout, stride))
-        launch_wgrad_tc(x, dy, dw, scratch, B, H, W, Cin, s);
+        launch_wgrad_tc(x, dy, dw, scratch, B, H, W, Cin, Cin, s);
     else
         launch_conv_wgrad_direct(precision, x, dy, dw, scratch, B, H, W, Cin, Cout, stride, s);
     return done();

@@ -167,17 +167,20 @@ template <int C> inline size_t conv_smem_bytes(int n_stages, int stage_bytes) {
 // per filter row; rows = filter column x channel of this pass, k = contraction channel): the forward one (row =
 // output channel, k = input channel) and the input-gradient one (row = input channel, k = output channel, taps
 // flipped).  One thread per (tap, row, k).
-struct PackJob { long src_off; long dst_off; int C; int first_elem; };
+struct PackJob { long src_off; long dst_off; int C; int first_elem; int cin_real; int pad_; };
 
 // image element (tap = ky*3+kx, row r, k): filter row tile ky, row kx*C + r of that tile
 template <int C> __device__ __forceinline__ uint32_t w_img_off(int tap, int r, int k) {
     return (uint32_t)(tap / 3) * TcCfg<C>::w_row_tile_bytes + swz_off<C>((tap % 3) * C + r, k);
 }
-template <int C> __device__ __forceinline__ void pack_one(const bf16 *w, uint8_t *dst, int i) {
+// cin: input channels the canonical filter really has; channels cin..C-1 of the images are zero (a first layer whose
+// input was zero-padded to C channels)
+template <int C> __device__ __forceinline__ void pack_one(const bf16 *w, uint8_t *dst, int i, int cin) {
     const int tap = i / (C * C), r = (i / C) % C, k = i % C;
     const uint32_t o = w_img_off<C>(tap, r, k);
-    *reinterpret_cast<bf16 *>(dst + o) = w[(size_t)(r * C + k) * 9 + tap];
-    *reinterpret_cast<bf16 *>(dst + TcCfg<C>::w_bytes + o) = w[(size_t)(k * C + r) * 9 + (8 - tap)];
+    const bf16 zero = __float2bfloat16_rn(0.f);
+    *reinterpret_cast<bf16 *>(dst + o) = k < cin ? w[(size_t)(r * cin + k) * 9 + tap] : zero;
+    *reinterpret_cast<bf16 *>(dst + TcCfg<C>::w_bytes + o) = r < cin ? w[(size_t)(k * cin + r) * 9 + (8 - tap)] : zero;
 }
 
 __global__ void pack_filters_kernel(const bf16 *__restrict__ wver, uint8_t *__restrict__ packed,
@@ -193,9 +196,9 @@ __global__ void pack_filters_kernel(const bf16 *__restrict__ wver, uint8_t *__re
     }
     const PackJob j = jobs[lo];
     const int i = e - j.first_elem;
-    if (j.C == 16) pack_one<16>(wver + j.src_off, packed + j.dst_off, i);
-    else if (j.C == 32) pack_one<32>(wver + j.src_off, packed + j.dst_off, i);
-    else pack_one<64>(wver + j.src_off, packed + j.dst_off, i);
+    if (j.C == 16) pack_one<16>(wver + j.src_off, packed + j.dst_off, i, j.cin_real);
+    else if (j.C == 32) pack_one<32>(wver + j.src_off, packed + j.dst_off, i, j.cin_real);
+    else pack_one<64>(wver + j.src_off, packed + j.dst_off, i, j.cin_real);
 }
 
 // the same for one convolution, job passed by value
@@ -204,9 +207,9 @@ __global__ void pack_one_filter_kernel(const bf16 *__restrict__ w, uint8_t *__re
     pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= 9 * C * C) return;
-    if (C == 16) pack_one<16>(w, packed, i);
-    else if (C == 32) pack_one<32>(w, packed, i);
-    else pack_one<64>(w, packed, i);
+    if (C == 16) pack_one<16>(w, packed, i, C);
+    else if (C == 32) pack_one<32>(w, packed, i, C);
+    else pack_one<64>(w, packed, i, C);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -560,7 +563,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 
 // dw[co][ci][tap] = sum over chunks of part[chunk][tap][ci][co].  64 outputs per CTA, four threads per output: thread g
 // adds chunks g, g+4, ... (four independent loads in flight per thread), the four sums are combined in a fixed order.
-__global__ void __launch_bounds__(256) wgrad_tc_fold_kernel(const float *__restrict__ part, float *__restrict__ dw, int chunks, int C) {
+__global__ void __launch_bounds__(256) wgrad_tc_fold_kernel(const float *__restrict__ part, float *__restrict__ dw, int chunks, int C,
+                                                            int cin) {
     pdl_launch();
     pdl_wait();
     __shared__ float sm[4][64];
@@ -581,7 +585,7 @@ __global__ void __launch_bounds__(256) wgrad_tc_fold_kernel(const float *__restr
     if (g == 0 && i < total) {
         const float t = (sm[0][o] + sm[1][o]) + (sm[2][o] + sm[3][o]);
         const int co = i % C, ci = (i / C) % C, tap = i / (C * C);
-        dw[((size_t)co * C + ci) * 9 + tap] = t;
+        if (ci < cin) dw[((size_t)co * cin + ci) * 9 + tap] = t;  // cin < C: the input was zero-padded to C channels
     }
 }
 
@@ -653,7 +657,7 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
 }
 
 template <int C>
-int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, cudaStream_t s) {
+int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int cin, cudaStream_t s) {
     int rows, imgs;
     tile_geometry(H, W, &rows, &imgs);
     const int slab = (imgs == 1 && 9 * C <= 512) ? 1 : 0;
@@ -670,7 +674,7 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int max_chunks = slab ? (C == 16 ? 148 : 74) : 49;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
     launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
-    launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C);
+    launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C, cin);
     return 2;
 }
 
@@ -716,12 +720,12 @@ bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
 }
 size_t wgrad_tc_scratch_elems() { return (size_t)kWgMaxChunks * 9 * 32 * 32 > (size_t)49 * 9 * 64 * 64 ? (size_t)kWgMaxChunks * 9 * 32 * 32 : (size_t)49 * 9 * 64 * 64; }
 
-int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C,
+int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C, int cin_real,
                     cudaStream_t s) {
     switch (C) {
-    case 16: return launch_wg<16>(x, dy, dw, scratch, B, H, W, s);
-    case 32: return launch_wg<32>(x, dy, dw, scratch, B, H, W, s);
-    case 64: return launch_wg<64>(x, dy, dw, scratch, B, H, W, s);
+    case 16: return launch_wg<16>(x, dy, dw, scratch, B, H, W, cin_real, s);
+    case 32: return launch_wg<32>(x, dy, dw, scratch, B, H, W, cin_real, s);
+    case 64: return launch_wg<64>(x, dy, dw, scratch, B, H, W, cin_real, s);
     }
     return -1;
 }

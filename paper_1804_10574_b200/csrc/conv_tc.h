@@ -19,14 +19,15 @@ int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed
                    Shortcut sc, cudaStream_t s);
 size_t tc_packed_bytes(int C);
 // One launch that re-arranges the filters of many convolutions of one weight version.
-struct PackJobHost { long src_off; long dst_off; int C; int first_elem; };  // element offset in wver, byte offset in packed
+struct PackJobHost { long src_off; long dst_off; int C; int first_elem; int cin_real; int pad_; };  // element offset in wver, byte offset in packed
 int launch_pack_one(const void *w, void *packed, int C, cudaStream_t s);
 int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,
                         cudaStream_t s);
 
 bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
 size_t wgrad_tc_scratch_elems();
-int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C,
+// cin_real < C: x was zero-padded from cin_real to C channels; dw is the canonical [C][cin_real][3][3] gradient.
+int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C, int cin_real,
                     cudaStream_t s);
 
 // One-time per-process set-up (function attributes, driver entry points).  Returns a cudaError_t value.

@@ -36,6 +36,7 @@ struct LayerPlan {
     TensorRef in, out;            // layer input (may live in the previous module's arena) and output
     TensorRef y1, a1, y2, stats;  // basic block intermediates; stats = fp32 [4][C] (mean1,invstd1,mean2,invstd2)
     long pk1 = -1, pk2 = -1;      // byte offsets of the pre-arranged filter images (conv / conv1, conv2), -1 = none
+    int pad_c = 0;                // first conv only: its input is stored zero-padded to this many channels (0 = as is)
     bool is_first, is_last;
 };
 
@@ -147,7 +148,7 @@ int conv_dgrad(ddg_ctx *c, const void *dy, const void *w, const void *wp, void *
 int conv_wgrad(ddg_ctx *c, Module &m, const void *x, const void *dy, float *dw, int H, int W, int Cin, int Cout,
                int stride, cudaStream_t s) {
     if (c->prec == P_BF16 && wgrad_tc_supported(c->B, H, W, Cin, Cout, stride))
-        return launch_wgrad_tc(x, dy, dw, m.wg_scratch, c->B, H, W, Cin, s);
+        return launch_wgrad_tc(x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cin, s);
     return launch_conv_wgrad_direct(c->prec, x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cout, stride, s);
 }
 
@@ -167,7 +168,7 @@ long forward_module(ddg_ctx *c, int k, long t) {
         if (L.is_first) {  // layout shim: staged NCHW fp32 -> NHWC in the compute precision, kept in the arena
             char *xin = slot_ptr(c, L.in, t);
             n += launch_shim(c->prec, c->x_stage + (size_t)(t % c->K) * c->x_elems, xin, c->B, c->in_c, c->in_h,
-                             c->in_w, s);
+                             c->in_w, L.pad_c ? L.pad_c : c->in_c, s);
             in = xin;
         } else {
             in = slot_ptr(c, L.in, t);
@@ -180,7 +181,10 @@ long forward_module(ddg_ctx *c, int k, long t) {
                                L.Cin, L.Cout, L.spec.relu_after, L.is_last, s);
             break;
         case DDG_CONV3X3:
-            n += conv_fwd(c, in, w, pkp(L.pk1), out, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, L.spec.relu_after, s);
+            if (L.pad_c)  // stem on the tensor cores: input and filter image zero-padded to pad_c channels
+                n += launch_conv_tc(0, in, w, pkp(L.pk1), out, B, L.Hin, L.Win, L.pad_c, Shortcut{}, s);
+            else
+                n += conv_fwd(c, in, w, pkp(L.pk1), out, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, L.spec.relu_after, s);
             break;
         case DDG_BN: {
             float *st = (float *)slot_ptr(c, L.stats, t);
@@ -285,7 +289,8 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
             if (need_dx)
                 n += conv_dgrad(c, dy, w, pkp(L.pk1), dst, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, Shortcut{}, s);
             side_join();  // this one runs on the chain's own stream and shares the weight-gradient scratch
-            n += conv_wgrad(c, m, in, dy, gw, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, s);
+            if (L.pad_c) n += launch_wgrad_tc(in, dy, gw, m.wg_scratch, B, L.Hin, L.Win, L.pad_c, L.Cin, s);
+            else n += conv_wgrad(c, m, in, dy, gw, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride, s);
             break;
         }
         case DDG_BN: {
@@ -638,7 +643,15 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
             L.module = k;
             L.p_off = p;
             p += L.p_cnt;
-            const size_t n_in = (size_t)c->B * L.Cin * L.Hin * L.Win, n_out = (size_t)c->B * L.Cout * L.Hout * L.Wout;
+            size_t n_in = (size_t)c->B * L.Cin * L.Hin * L.Win;
+            const size_t n_out = (size_t)c->B * L.Cout * L.Hout * L.Wout;
+            if (l == 0 && c->prec == P_BF16 && L.spec.kind == DDG_CONV3X3 && !L.spec.relu_after && L.spec.stride == 1 &&
+                L.Cin < 16 && L.Cout == 16 && conv_tc_supported(c->B, L.Hin, L.Win, 16, 16, 1)) {
+                // a narrow first convolution (3 input channels) runs on the tensor-core kernels with its input stored
+                // zero-padded to 16 channels
+                L.pad_c = 16;
+                n_in = (size_t)c->B * 16 * L.Hin * L.Win;
+            }
             if (l == 0) L.in = {0, take(n_in * es)};                      // the shimmed input lives in module 1's arena
             else L.in = c->layers[l - 1].out;                             // may point into the previous module's arena
             L.out = {k, take(L.is_last ? n_out * sizeof(float) : n_out * es)};
@@ -698,16 +711,18 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
             std::vector<PackJobHost> jobs;
             size_t pk_off = 0;
             int elems = 0;
-            auto plan = [&](long *slot, size_t w_off, int H, int W, int Ci, int Co, int stride) {
+            auto plan = [&](long *slot, size_t w_off, int H, int W, int Ci, int Co, int stride, int cin_real = 0) {
                 if (!conv_tc_supported(c->B, H, W, Ci, Co, stride)) return;
                 *slot = (long)pk_off;
-                jobs.push_back(PackJobHost{(long)w_off, (long)pk_off, Ci, elems});
+                jobs.push_back(PackJobHost{(long)w_off, (long)pk_off, Ci, elems, cin_real ? cin_real : Ci, 0});
                 pk_off += tc_packed_bytes(Ci);
                 elems += 9 * Ci * Ci;
             };
             for (int l = m.first; l <= m.last; ++l) {
                 LayerPlan &L = c->layers[l];
-                if (L.spec.kind == DDG_CONV3X3 && !L.spec.relu_after)
+                if (L.spec.kind == DDG_CONV3X3 && L.pad_c)
+                    plan(&L.pk1, L.p_off, L.Hin, L.Win, L.pad_c, L.Cout, 1, L.Cin);
+                else if (L.spec.kind == DDG_CONV3X3 && !L.spec.relu_after)
                     plan(&L.pk1, L.p_off, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride);
                 if (L.spec.kind == DDG_BASIC_BLOCK) {
                     plan(&L.pk1, L.p_off, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride);

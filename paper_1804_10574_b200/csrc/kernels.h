@@ -22,7 +22,8 @@ struct Shortcut {
 };
 
 // ---- layout / small layers --------------------------------------------------------------------------
-int launch_shim(int prec, const float *x_nchw, void *out_nhwc, int B, int C, int H, int W, cudaStream_t s);
+// Cpad >= C: channels per pixel of the output; the extra channels are written as zero.
+int launch_shim(int prec, const float *x_nchw, void *out_nhwc, int B, int C, int H, int W, int Cpad, cudaStream_t s);
 int launch_relu_fwd(int prec, const void *x, void *y, size_t n, cudaStream_t s);
 int launch_relu_bwd(int prec, const void *y, const void *dy, void *dx, size_t n, cudaStream_t s);
 int launch_avgpool_fwd(int prec, const void *x, void *y, int B, int HW, int C, cudaStream_t s);

@@ -21,18 +21,19 @@ static constexpr float kBnEps = 1e-5f;
 // input shim: NCHW fp32 -> NHWC T
 // ------------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void shim_kernel(const float *__restrict__ x, T *__restrict__ out, int B, int C, int HW) {
+__global__ void shim_kernel(const float *__restrict__ x, T *__restrict__ out, int B, int C, int HW, int Cpad) {
     pdl_launch();
     pdl_wait();
     long i = (long)blockIdx.x * blockDim.x + threadIdx.x;  // (n, p)
     if (i >= (long)B * HW) return;
     long n = i / HW, p = i % HW;
-    for (int c = 0; c < C; ++c) out[i * C + c] = from_f<T>(x[(n * C + c) * HW + p]);
+    for (int c = 0; c < C; ++c) out[i * Cpad + c] = from_f<T>(x[(n * C + c) * HW + p]);
+    for (int c = C; c < Cpad; ++c) out[i * Cpad + c] = from_f<T>(0.f);  // zero channels up to the padded width
 }
 
-int launch_shim(int prec, const float *x, void *out, int B, int C, int H, int W, cudaStream_t s) {
+int launch_shim(int prec, const float *x, void *out, int B, int C, int H, int W, int Cpad, cudaStream_t s) {
     long n = (long)B * H * W;
-    DISPATCH_PREC(prec, launch_k(shim_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, x, (T *)out, B, C, H * W));
+    DISPATCH_PREC(prec, launch_k(shim_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, x, (T *)out, B, C, H * W, Cpad));
     return 1;
 }
 
