@@ -671,7 +671,7 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int ncols = slab ? 9 * C : 3 * C;
     const int tmem_cols = ncols <= 64 ? 64 : (ncols <= 128 ? 128 : (ncols <= 256 ? 256 : 512));
     const int n_tiles = (int)((long)B * H * W / kTileM);
-    const int max_chunks = slab ? (C == 16 ? 148 : 74) : 49;
+    const int max_chunks = slab ? (C == 16 ? 74 : 37) : 24;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
     launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
     launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C, cin);
