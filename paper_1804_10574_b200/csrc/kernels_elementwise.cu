@@ -349,8 +349,8 @@ bn_reduce_kernel(const T *__restrict__ x, const T *__restrict__ dout, const T *_
 // lanes of a warp by xor-shuffles, warps of a CTA in index order, CTAs in index order by the last CTA to finish.
 static constexpr int kRedThreads = 512;
 
-template <typename T, int VEC, int MODE>
-__global__ void __launch_bounds__(kRedThreads)
+template <typename T, int VEC, int MODE, int U>
+__global__ void __launch_bounds__(kRedThreads, U == 2 ? 2 : 1)
 bn_reduce_fast_kernel(const T *__restrict__ x, const T *__restrict__ dout, const T *__restrict__ out,
                       const float *__restrict__ mean_in, const float *__restrict__ invstd_in, float *o0, float *o1,
                       float *scratch, long npix, int C, int relu) {
@@ -374,11 +374,13 @@ bn_reduce_fast_kernel(const T *__restrict__ x, const T *__restrict__ dout, const
         mu[j] = MODE == 1 ? (A)mean_in[c0 + j] : (A)0;
         is[j] = MODE == 1 ? (A)invstd_in[c0 + j] : (A)0;
     }
-    for (long i0 = tid; i0 < nvec; i0 += 4 * stride) {
-        A xv[4][VEC], dv[4][VEC];
-        float ov[4][VEC];
+    // U vectors per trip: 4 with one CTA per SM (small tensors: one trip, lowest latency), 2 with two CTAs per SM
+    // (large tensors: more loads in flight per SM)
+    for (long i0 = tid; i0 < nvec; i0 += U * stride) {
+        A xv[U][VEC], dv[U][VEC];
+        float ov[U][VEC];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             const long i = i0 + u * stride;
             if (i < nvec) {
                 load_a<T, A, VEC>(x + i * VEC, xv[u]);
@@ -389,7 +391,7 @@ bn_reduce_fast_kernel(const T *__restrict__ x, const T *__restrict__ dout, const
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             if (i0 + u * stride < nvec) {
 #pragma unroll
                 for (int j = 0; j < VEC; ++j) {
@@ -466,9 +468,9 @@ static bool red_fast_ok(int C, int V) {
     const int groups = C / V;
     return (groups & (groups - 1)) == 0 && groups <= 32;
 }
-static int red_fast_grid(long nvec) {
+static int red_fast_grid(long nvec, int per_sm) {
     long g = (nvec + 4L * kRedThreads - 1) / (4L * kRedThreads);
-    if (g > 148) g = 148;
+    if (g > 148 * per_sm) g = 148 * per_sm;
     return (int)(g < 1 ? 1 : g);
 }
 
@@ -479,8 +481,8 @@ int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *
     DISPATCH_PREC(prec, {
         if (red_fast_ok(C, Vec16<T>::N)) {
             constexpr int V = Vec16<T>::N;
-            launch_k(bn_reduce_fast_kernel<T, V, 0>, red_fast_grid(npix * (C / V)), kRedThreads, 0, s, (const T *)x, nullptr,
-                     nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
+            launch_k(bn_reduce_fast_kernel<T, V, 0, 4>, red_fast_grid(npix * (C / V), 1), kRedThreads, 0, s, (const T *)x,
+                     nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
         } else if (vec_for<T>(C) > 1) {
             constexpr int V = Vec16<T>::N;
             launch_k(bn_reduce_kernel<T, V, 0>, bn_grid(npix, kThreads / (C / V)), kThreads, 0, s, (const T *)x, nullptr, nullptr, nullptr, nullptr, mean, invstd, scratch, npix, C, 0);
@@ -497,8 +499,13 @@ int launch_bn_bwd_reduce(int prec, const void *dout, const void *out, const void
     DISPATCH_PREC(prec, {
         if (red_fast_ok(C, Vec16<T>::N)) {
             constexpr int V = Vec16<T>::N;
-            launch_k(bn_reduce_fast_kernel<T, V, 1>, red_fast_grid(npix * (C / V)), kRedThreads, 0, s, (const T *)x,
-                     (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
+            const long nvec = npix * (C / V);
+            if (nvec > 16L * 148 * kRedThreads)  // large: two CTAs per SM keep more loads in flight
+                launch_k(bn_reduce_fast_kernel<T, V, 1, 2>, red_fast_grid(nvec, 2), kRedThreads, 0, s, (const T *)x,
+                         (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
+            else
+                launch_k(bn_reduce_fast_kernel<T, V, 1, 4>, red_fast_grid(nvec, 1), kRedThreads, 0, s, (const T *)x,
+                         (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
         } else if (vec_for<T>(C) > 1) {
             constexpr int V = Vec16<T>::N;
             launch_k(bn_reduce_kernel<T, V, 1>, bn_grid(npix, kThreads / (C / V)), kThreads, 0, s, (const T *)x, (const T *)dout, (const T *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
