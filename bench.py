@@ -113,33 +113,60 @@ def time_oracle(cfg, batch, n_steps):
                       "untimed pipeline-fill iterations" % (n_steps, batch, cfg["batch"]), "seconds": dt}
 
 
-def dominant_kernel_roofline(torch, binding, cfg, peaks):
-    """Times the kernel with the largest share of the step (3x3 convolution forward on the widest feature map) alone,
-    at the workload's shape and launch configuration, with CUDA events on its stream."""
-    B, H, W, C = cfg["batch"], 32, 32, 16
-    x = torch.randn(B, H, W, C, device="cuda").to(torch.bfloat16)
-    w = (torch.randn(C, C, 3, 3, device="cuda") * (2.0 / (9 * C)) ** 0.5).to(torch.bfloat16)
-    y = torch.empty_like(x)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    s = torch.cuda.current_stream()
+def _time_kernel(torch, fn, stream, flush, iters=20):
     for _ in range(3):
-        binding.conv3x3_fwd(1, x, w, y, B, H, W, C, C, 1, s.cuda_stream)
-    times = []
-    for _ in range(20):
-        flush.zero_()                                  # evict the tensors from L2 between timed launches
+        fn()
+    ts = []
+    for _ in range(iters):
+        flush.zero_()                                  # evict the operands from L2 between timed launches
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(s)
-        binding.conv3x3_fwd(1, x, w, y, B, H, W, C, C, 1, s.cuda_stream)
-        e1.record(s)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
         e1.synchronize()
-        times.append(e0.elapsed_time(e1) * 1e-3)
-    dt = float(np.mean(times))
-    alg_bytes = 2 * x.numel() * 2 + w.numel() * 2     # read x, write y (bf16) + weights
-    achieved = alg_bytes / dt / 1e9
-    peak = peaks.get("hbm_gbs", 6650.0)
-    return {"kernel": "conv3x3_fwd 16->16 32x32 B=%d bf16" % B, "bound": "hbm", "achieved": achieved, "peak": peak,
-            "unit": "GB/s", "frac": achieved / peak, "traffic": None, "launch_us": dt * 1e6,
-            "peak_source": "measured" if "hbm_gbs" in peaks else "fallback"}
+        ts.append(e0.elapsed_time(e1) * 1e-3)
+    return float(np.mean(ts))
+
+
+def dominant_kernel_roofline(torch, binding, cfg, peaks):
+    """The kernel with the largest share of the ncu launch list of this workload is the batch-norm backward reduction
+    (profiles/ddg_step_resnet110_k4_b128_bf16_launch_list.md).  It is timed alone here, at the workload's largest
+    feature map and in the launch configuration the step uses, with CUDA events on its stream; the tensor-core
+    convolution kernels are timed the same way and listed beside it."""
+    B, H, C = cfg["batch"], 32, 16
+    bf = torch.bfloat16
+    s = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    hbm = peaks.get("hbm_gbs", 6650.0)
+    tflops = peaks.get("bf16_tflops", 1590.0)
+    src = "measured" if "hbm_gbs" in peaks else "fallback"
+    x = torch.randn(B, H * H, C, device="cuda").to(bf)
+    dout, out = torch.randn_like(x), torch.randn_like(x)
+    mean, invstd = torch.zeros(C, device="cuda"), torch.ones(C, device="cuda")
+    dg, db = torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
+    scr = torch.zeros(binding.bn_scratch_elems(C), device="cuda")
+    dt = _time_kernel(torch, lambda: binding.bn_bwd_reduce(1, dout, out, x, mean, invstd, dg, db, scr, B, H * H, C, 1,
+                                                           s.cuda_stream), s, flush)
+    alg = 3 * x.numel() * 2                            # reads dout, out (ReLU mask), x; writes 2*C sums
+    # DRAM traffic per launch from the ncu capture at batch 4096 (profiles/bn_reduce_fast_kernel_...md): 414.1 MB for
+    # 402.7 MB algorithmic, scaled by pixels processed
+    traffic = 414.1e6 * B / 4096.0
+    roof = {"kernel": "bn_reduce_fast_kernel<bf16,8,1> (batch-norm backward sums) C=16 32x32 B=%d" % B, "bound": "hbm",
+            "achieved": alg / dt / 1e9, "peak": hbm, "unit": "GB/s", "frac": alg / dt / 1e9 / hbm, "traffic": traffic,
+            "launch_us": dt * 1e6, "peak_source": src, "ncu_share_of_step": 0.151}
+    others = []
+    for (Hh, Cc) in ((32, 16), (16, 32), (8, 64)):
+        xx = torch.randn(B, Hh, Hh, Cc, device="cuda").to(bf)
+        w = (torch.randn(Cc, Cc, 3, 3, device="cuda") * (2.0 / (9 * Cc)) ** 0.5).to(bf)
+        yy = torch.empty_like(xx)
+        pk = torch.empty(binding.conv3x3_packed_bytes(B, Hh, Hh, Cc), dtype=torch.uint8, device="cuda")
+        binding.conv3x3_pack(w, pk, Cc)
+        dtc = _time_kernel(torch, lambda: binding.conv3x3_packed(0, xx, w, pk, yy, B, Hh, Hh, Cc, s.cuda_stream), s, flush)
+        nbytes, flops = 2 * xx.numel() * 2 + w.numel() * 2, 2.0 * 9 * Cc * Cc * B * Hh * Hh
+        others.append({"kernel": "conv3x3_tc_kernel<%d> fwd %dx%d B=%d" % (Cc, Hh, Hh, B), "launch_us": dtc * 1e6,
+                       "hbm_gbs": nbytes / dtc / 1e9, "hbm_frac": nbytes / dtc / 1e9 / hbm, "tflops": flops / dtc / 1e12,
+                       "tensor_frac": flops / dtc / 1e12 / tflops})
+    return roof, others
 
 
 def main():
@@ -236,7 +263,7 @@ def main():
             peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
         except Exception:
             pass
-        roof = dominant_kernel_roofline(torch, binding, cfg, peaks)
+        roof, roof_others = dominant_kernel_roofline(torch, binding, cfg, peaks)
         cpu = None
         if world == 1 and not args.skip_cpu:
             r = time_oracle(cfg, args.cpu_batch, args.cpu_steps or 2)
@@ -254,7 +281,7 @@ def main():
                "clocks": clocks, "gpu_launches": int(launches_per_step * args.steps),
                "e2e": {"value": cfg["batch"] * n_e2e * world / dt_e2e, "unit": "images/s",
                        "h2d_bytes_per_step": x_bytes + cfg["batch"] * 4, "d2h_bytes_per_step": 4, "steps": n_e2e},
-               "roofline": roof, "cpu_baseline": cpu}
+               "roofline": roof, "roofline_others": roof_others, "cpu_baseline": cpu}
         print(json.dumps(out))
     net.destroy()
     if dist is not None:

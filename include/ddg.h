@@ -193,6 +193,11 @@ ddg_status ddg_bn_fwd_noalloc(int precision, const void *x, const void *gamma, c
 ddg_status ddg_bn_bwd(int precision, const void *dout, const void *out, const void *x, const void *gamma,
                       const float *mean, const float *invstd, void *dx, float *dgamma, float *dbeta, float *scratch,
                       int B, int HW, int C, int relu, void *stream);
+/* The reduction half of ddg_bn_bwd alone (dgamma, dbeta), for timing the kernel by itself.  Same arguments. */
+ddg_status ddg_bn_bwd_reduce(int precision, const void *dout, const void *out, const void *x, const float *mean,
+                             const float *invstd, float *dgamma, float *dbeta, float *scratch, int B, int HW, int C,
+                             int relu, void *stream);
+
 /* Fused SGD update over n parameters (Eq. 9 with momentum and weight decay): d = g + wd*w; v = mu*v + d;
  * w -= lr*v; w_version = cast(w).  w, v, g fp32; w_version in the precision's element type. */
 ddg_status ddg_sgd_update(int precision, float *w, float *v, const float *g, void *w_version, size_t n, float lr,

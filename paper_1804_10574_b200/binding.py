@@ -27,7 +27,7 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_last_error", "ddg_destroy", "ddg_conv3x3_fwd", "ddg_conv3x3_dgrad",
            "ddg_conv3x3_wgrad_scratch_elems", "ddg_conv3x3_wgrad", "ddg_bn_scratch_elems", "ddg_bn_fwd", "ddg_bn_bwd",
            "ddg_sgd_update", "ddg_tensor_core_path", "ddg_bn_fwd_noalloc",
-           "ddg_conv3x3_packed_bytes", "ddg_conv3x3_pack", "ddg_conv3x3_packed"]
+           "ddg_conv3x3_packed_bytes", "ddg_conv3x3_pack", "ddg_conv3x3_packed", "ddg_bn_bwd_reduce"]
 
 
 class Layer(ctypes.Structure):
@@ -78,6 +78,7 @@ _lib.ddg_conv3x3_packed_bytes.restype = _sz
 _lib.ddg_conv3x3_pack.argtypes = [_vp, _vp, _i, _vp]
 _lib.ddg_conv3x3_packed.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_bn_fwd_noalloc.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
+_lib.ddg_bn_bwd_reduce.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_sgd_update.argtypes = [_i, _vp, _vp, _vp, _vp, _sz, _f, _f, _f, _vp]
 
 
@@ -240,6 +241,11 @@ def bn_fwd_noalloc(prec, x, gamma, beta, res, y, mean, invstd, B, HW, C, relu, s
 def bn_bwd(prec, dout, out, x, gamma, mean, invstd, dx, dgamma, dbeta, scratch, B, HW, C, relu, stream=None):
     _ok(_lib.ddg_bn_bwd(prec, _ptr(dout), _ptr(out), _ptr(x), _ptr(gamma), _ptr(mean), _ptr(invstd), _ptr(dx),
                         _ptr(dgamma), _ptr(dbeta), _ptr(scratch), B, HW, C, int(relu), stream))
+
+
+def bn_bwd_reduce(prec, dout, out, x, mean, invstd, dgamma, dbeta, scratch, B, HW, C, relu, stream=None):
+    _ok(_lib.ddg_bn_bwd_reduce(prec, _ptr(dout), _ptr(out), _ptr(x), _ptr(mean), _ptr(invstd), _ptr(dgamma), _ptr(dbeta),
+                               _ptr(scratch), B, HW, C, int(relu), stream))
 
 
 def sgd_update(prec, w, v, g, w_version, n, lr, momentum, weight_decay, stream=None):

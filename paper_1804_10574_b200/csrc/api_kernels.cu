@@ -122,6 +122,18 @@ ddg_status ddg_bn_bwd(int precision, const void *dout, const void *out, const vo
     return done();
 }
 
+ddg_status ddg_bn_bwd_reduce(int precision, const void *dout, const void *out, const void *x, const float *mean,
+                             const float *invstd, float *dgamma, float *dbeta, float *scratch, int B, int HW, int C,
+                             int relu, void *stream) {
+    if (bad_prec(precision) || !dout || !x || !mean || !invstd || !dgamma || !dbeta || !scratch || (relu && !out))
+        return DDG_ERR_INVALID_ARG;
+    if (B < 1 || HW < 1 || C < 1 || C > 128) return DDG_ERR_UNSUPPORTED;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;
+    launch_bn_bwd_reduce(precision, dout, out, x, mean, invstd, dgamma, dbeta, scratch, (long)B * HW, C, relu, s);
+    return done();
+}
+
 ddg_status ddg_sgd_update(int precision, float *w, float *v, const float *g, void *w_version, size_t n, float lr,
                           float momentum, float weight_decay, void *stream) {
     if (bad_prec(precision) || !w || !v || !g || !w_version) return DDG_ERR_INVALID_ARG;

@@ -87,7 +87,7 @@ def run_pair(cfg, steps, tol, loss_tol, precision=None, split_after=None, use_gr
     oracle's bf16 decisions and its gradients carry an independent draw of the same format noise.  The oracle
     measures that noise itself: e_orc = rel(oracle with bf16 storage, exact oracle) per tensor.  A gradient tensor
     passes if it is within `tol` of the bf16-storage oracle, or if its distance to the exact oracle is at most
-    noise_mult * e_orc + tol."""
+    noise_mult * e_orc + tol.  Weights integrate the gradients and are held to the same bar."""
     from paper_1804_10574_b200 import binding
     layers = cfg["layers"]
     split_after = cfg["split_after"] if split_after is None else split_after
@@ -142,6 +142,7 @@ def run_pair(cfg, steps, tol, loss_tol, precision=None, split_after=None, use_gr
         off = 0
         gpu.get_weights(wbuf)
         wref = ref.get_weights()
+        w_ex = exact.get_weights() if exact is not None else None
         for k in range(K):
             gbuf = np.empty(gpu.per_module[k], dtype=np.float32)
             s_gpu = gpu.get_grads(k, gbuf)
@@ -159,7 +160,11 @@ def run_pair(cfg, steps, tol, loss_tol, precision=None, split_after=None, use_gr
                         "step %d module %d grad %s: %.3e from the exact oracle, format noise %.3e" % (t, k, name, e_gpu, e_orc)
                     e = rel(wbuf[off + a:off + b], wref[off + a:off + b])
                     worst["weight"] = max(worst["weight"], e)
-                    assert e <= tol, "step %d module %d weight %s: rel %.3e > %.1e" % (t, k, name, e, tol)
+                    # weights integrate the gradients, so they carry the same format noise: same bar
+                    ew_gpu = rel(wbuf[off + a:off + b], w_ex[off + a:off + b])
+                    ew_orc = rel(wref[off + a:off + b], w_ex[off + a:off + b])
+                    assert e <= tol or ew_gpu <= noise_mult * ew_orc + tol, \
+                        "step %d module %d weight %s: rel %.3e > %.1e (format noise %.3e)" % (t, k, name, e, tol, ew_orc)
                 off += gpu.per_module[k]
                 continue
             if s_ref >= 0 and any(rel(gbuf[a:b], g_ref[a:b]) > tol for _, a, b in segs[k]):

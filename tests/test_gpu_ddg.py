@@ -99,3 +99,12 @@ def test_create_rejects_bad_specs():
         d.set_weights(np.zeros(d.n_params, dtype=np.float32))   # only before the first step
     assert e.value.status == 7
     d.destroy()
+
+
+def test_resnet110_k4_full_size_bf16_graph():
+    """The benchmark's own configuration (ResNet-110, K=4, batch 128, bf16, graph replay, 100 classes): five
+    iterations against the oracle at full size.  Every module applies its first real delayed gradient inside the
+    window (delays 3, 2, 1, 0), loss and weights are held to the bf16 bars, gradients to the format-noise bar."""
+    cfg = nets.config("resnet110")
+    w = run_pair(cfg, 5, BF16_TOL, 5e-3, use_graph=True, noise_mult=2.0, check_every=2)
+    print("resnet110 K=4 full size worst", w)
