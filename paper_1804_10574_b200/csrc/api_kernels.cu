@@ -24,6 +24,7 @@ extern "C" {
 
 int ddg_tensor_core_path(int B, int H, int W, int Cin, int Cout, int stride) {
     if (init_once() != DDG_OK) return 0;
+    if (conv_tc_s2_supported(B, H, W, Cin, Cout, stride)) return 3;
     return (conv_tc_supported(B, H, W, Cin, Cout, stride) ? 1 : 0) | (wgrad_tc_supported(B, H, W, Cin, Cout, stride) ? 2 : 0);
 }
 
@@ -35,6 +36,8 @@ ddg_status ddg_conv3x3_fwd(int precision, const void *x, const void *w, void *y,
     cudaStream_t s = (cudaStream_t)stream;
     if (precision == DDG_BF16 && conv_tc_supported(B, H, W, Cin, Cout, stride))
         launch_conv_tc(0, x, w, nullptr, y, B, H, W, Cin, Shortcut{}, s);
+    else if (precision == DDG_BF16 && conv_tc_s2_supported(B, H, W, Cin, Cout, stride))
+        launch_conv_tc_s2(0, x, w, nullptr, y, B, H, W, Cin, Shortcut{}, s);
     else
         launch_conv_fwd_direct(precision, x, w, y, B, H, W, Cin, Cout, stride, 0, s);
     return done();
@@ -48,6 +51,8 @@ ddg_status ddg_conv3x3_dgrad(int precision, const void *dy, const void *w, void 
     cudaStream_t s = (cudaStream_t)stream;
     if (precision == DDG_BF16 && conv_tc_supported(B, H, W, Cin, Cout, stride))
         launch_conv_tc(1, dy, w, nullptr, dx, B, H, W, Cin, Shortcut{}, s);
+    else if (precision == DDG_BF16 && conv_tc_s2_supported(B, H, W, Cin, Cout, stride))
+        launch_conv_tc_s2(1, dy, w, nullptr, dx, B, H, W, Cin, Shortcut{}, s);
     else
         launch_conv_dgrad_direct(precision, dy, w, dx, B, H, W, Cin, Cout, stride, Shortcut{}, s);
     return done();
@@ -88,6 +93,8 @@ ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float
     cudaStream_t s = (cudaStream_t)stream;
     if (precision == DDG_BF16 && wgrad_tc_supported(B, H, W, Cin, Cout, stride))
         launch_wgrad_tc(x, dy, dw, scratch, B, H, W, Cin, Cin, s);
+    else if (precision == DDG_BF16 && conv_tc_s2_supported(B, H, W, Cin, Cout, stride))
+        launch_wgrad_tc_s2(x, dy, dw, scratch, B, H, W, Cin, s);
     else
         launch_conv_wgrad_direct(precision, x, dy, dw, scratch, B, H, W, Cin, Cout, stride, s);
     return done();

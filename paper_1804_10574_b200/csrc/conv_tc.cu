@@ -183,6 +183,21 @@ template <int C> __device__ __forceinline__ void pack_one(const bf16 *w, uint8_t
     *reinterpret_cast<bf16 *>(dst + TcCfg<C>::w_bytes + o) = r < cin ? w[(size_t)(k * cin + r) * 9 + (8 - tap)] : zero;
 }
 
+// filter images of a stride-2 convolution with Ci input channels (Co = 2 Ci): nine [Co][Ci] K-major tiles for the forward
+// pass, then nine [Ci][Co] K-major tiles for the input gradient; tile index = ky*3+kx in both
+template <int CI> struct S2Cfg {
+    static constexpr int CO = 2 * CI;
+    static constexpr int tap_bytes = CO * CI * 2;
+    static constexpr int img_bytes = 9 * tap_bytes;
+};
+template <int CI> __device__ __forceinline__ void pack_s2_one(const bf16 *w, uint8_t *dst, int i) {
+    constexpr int CO = 2 * CI;
+    const int tap = i / (CO * CI), co = (i / CI) % CO, ci = i % CI;
+    const bf16 v = w[(size_t)(co * CI + ci) * 9 + tap];
+    *reinterpret_cast<bf16 *>(dst + tap * S2Cfg<CI>::tap_bytes + swz_off<CI>(co, ci)) = v;
+    *reinterpret_cast<bf16 *>(dst + S2Cfg<CI>::img_bytes + tap * S2Cfg<CI>::tap_bytes + swz_off<CO>(ci, co)) = v;
+}
+
 __global__ void pack_filters_kernel(const bf16 *__restrict__ wver, uint8_t *__restrict__ packed,
                                     const PackJob *__restrict__ jobs, int n_jobs, int total) {
     pdl_launch();
@@ -196,6 +211,11 @@ __global__ void pack_filters_kernel(const bf16 *__restrict__ wver, uint8_t *__re
     }
     const PackJob j = jobs[lo];
     const int i = e - j.first_elem;
+    if (j.pad_ == 1) {  // stride-2 convolution with C input channels
+        if (j.C == 16) pack_s2_one<16>(wver + j.src_off, packed + j.dst_off, i);
+        else pack_s2_one<32>(wver + j.src_off, packed + j.dst_off, i);
+        return;
+    }
     if (j.C == 16) pack_one<16>(wver + j.src_off, packed + j.dst_off, i, j.cin_real);
     else if (j.C == 32) pack_one<32>(wver + j.src_off, packed + j.dst_off, i, j.cin_real);
     else pack_one<64>(wver + j.src_off, packed + j.dst_off, i, j.cin_real);
@@ -561,14 +581,374 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Stride-2 3x3 convolution (the first convolution of a down-sampling residual block, Cout = 2 Cin) on the tensor
+// cores.  Output pixel (oy, ox) reads input pixels (2oy+ky-1, 2ox+kx-1): for one filter tap these are every second
+// pixel of every second row, which one TMA box fetches when the input [B][H][W][Ci] is described as the 5-D tensor
+// (2 Ci, W/2, 2, H/2, B): a pixel PAIR is the innermost axis (the column parity px selects its first or second half),
+// the row parity py is an axis of extent 2, and the zero fill of the pair axis and the half-row axis gives the padding.
+//   forward : per tile of 128 output pixels, nine tap boxes [128][Ci], nine MMAs (M=128, N=Co, K=Ci) into one
+//             accumulator.
+//   dgrad   : the input pixels fall into four parity classes (py, px); a class-(py,px) pixel (2j+py, 2i+px) receives
+//             taps ky = 1 (py = 0) or ky in {0, 2} (py = 1) from output rows j+1 / j, and likewise in x.  A tile is 128
+//             input pixels of one class; its (1+py)(1+px) operand boxes are the dy tile shifted by 0/1 rows and columns
+//             (zero-filled past the last row / column), MMAs M=128, N=Ci, K=Co.
+// The pipeline (TMA warp, MMA warp, two epilogue groups, bounded waits) is that of the stride-1 kernel; one pipeline
+// stage is one operand box.
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], "
+        "[%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+
+// KC: contraction channels (channels of the operand tensor); NC: channels of the result.  MODE 0 forward (KC = Ci,
+// NC = Co), MODE 1 input gradient (KC = Co, NC = Ci).  Hs x Ws is the SMALL (output-resolution) map; rows_per_tile /
+// imgs_per_tile describe a 128-pixel tile of it.  n_sp = number of such tiles.
+template <int KC, int NC, int MODE>
+__global__ void __launch_bounds__(kTcThreads, 1)
+conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
+                     bf16 *__restrict__ dst, int Hs, int Ws, int rows_per_tile, int imgs_per_tile, int n_sp, int n_stages,
+                     const bf16 *__restrict__ res_dout, const bf16 *__restrict__ res_out) {
+    typedef TcCfg<KC> Cfg;
+    constexpr int CI = MODE == 0 ? KC : NC;
+    constexpr int tap_bytes = KC * NC * 2;
+    constexpr int w_bytes = 9 * tap_bytes;
+    constexpr int stage_bytes = Cfg::tile_bytes;
+    constexpr int tmem_cols = 2 * NC < 32 ? 32 : 2 * NC;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw);
+    const uint32_t w_base = base, a_base = base + ((w_bytes + 1023u) & ~1023u);
+    uint8_t *tail = smem + ((w_bytes + 1023u) & ~1023u) + (size_t)n_stages * stage_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[4], tempty[4], wbar
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 9) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 9) * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 4 + a); };
+    const uint32_t w_bar = bar0 + 8u * (2 * kMaxStages + 8);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = MODE == 0 ? n_sp : 4 * n_sp;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        mbar_init(w_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                     "r"((uint32_t)tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    pdl_launch();
+    pdl_wait();  // nothing above touches global memory
+    if (w_packed == nullptr) {  // canonical filter [Co][Ci][3][3]: arrange the nine tiles of this pass here
+        constexpr int CO = 2 * CI;
+        for (int i = threadIdx.x; i < 9 * CO * CI; i += kTcThreads) {
+            const int tap = i / (CO * CI), co = (i / CI) % CO, ci = i % CI;
+            const uint32_t o = (uint32_t)tap * tap_bytes + (MODE == 0 ? swz_off<KC>(co, ci) : swz_off<KC>(ci, co));
+            *reinterpret_cast<bf16 *>(smem + o) = w[(size_t)(co * CI + ci) * 9 + tap];
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    const int tiles_per_img = Hs / rows_per_tile;
+    // spatial tile -> (first image, first row of the small map)
+    auto tile_origin = [&](int sp, int *n0, int *h0) {
+        if (imgs_per_tile > 1) { *n0 = sp * imgs_per_tile; *h0 = 0; }
+        else { *n0 = sp / tiles_per_img; *h0 = (sp % tiles_per_img) * rows_per_tile; }
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            if (w_packed != nullptr) {
+                mbar_expect_tx(w_bar, w_bytes);
+                bulk_copy_g2s(w_base, w_packed, w_bytes, w_bar);
+            }
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const int cls = MODE == 0 ? 0 : tile / n_sp, sp = MODE == 0 ? tile : tile % n_sp;
+                const int py = cls >> 1, px = cls & 1;
+                int n0, h0;
+                tile_origin(sp, &n0, &h0);
+                const int n_loads = MODE == 0 ? 9 : (1 + py) * (1 + px);
+                for (int j = 0; j < n_loads && ok; ++j) {
+                    ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 21);
+                    if (!ok) break;
+                    mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
+                    const uint32_t d = a_base + s * stage_bytes;
+                    if (MODE == 0) {
+                        const int ky = j / 3, kx = j % 3;
+                        // column 2ox+kx-1: kx = 1 -> first pixel of pair ox; kx = 0 / 2 -> second pixel of pair ox-1 / ox
+                        tma_load_5d(d, &tmap, full_bar(s), kx == 1 ? 0 : KC, kx == 0 ? -1 : 0, ky == 1 ? 0 : 1,
+                                    h0 + (ky == 0 ? -1 : 0), n0);
+                    } else {
+                        const int sy = px ? j >> 1 : j, sx = px ? j & 1 : 0;
+                        tma_load_4d(d, &tmap, full_bar(s), 0, sx, h0 + sy, n0);
+                    }
+                    if (++s == n_stages) { s = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) for (int i = 0; i < 2000; ++i) __nanosleep(100);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NC >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            int s = 0;
+            uint32_t ph = 0;
+            int it = 0;
+            bool ok = true;
+            if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, abort_flag, 25);
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+                const int cls = MODE == 0 ? 0 : tile / n_sp;
+                const int py = cls >> 1, px = cls & 1;
+                const int n_loads = MODE == 0 ? 9 : (1 + py) * (1 + px);
+                const int a = it & 1;
+                const uint32_t aph = (it >> 1) & 1u;
+                ok = mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, 22);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * NC);
+                for (int j = 0; j < n_loads && ok; ++j) {
+                    ok = mbar_wait(full_bar(s), ph, abort_flag, 23);
+                    if (!ok) break;
+                    tc_fence_after();
+                    int tap = j;
+                    if (MODE == 1) {
+                        const int sy = px ? j >> 1 : j, sx = px ? j & 1 : 0;
+                        // dx row 2j'+1 takes ky = 0 from output row j'+1 (the shifted box) and ky = 2 from row j'
+                        const int ky = py ? (sy ? 0 : 2) : 1, kx = px ? (sx ? 0 : 2) : 1;
+                        tap = ky * 3 + kx;
+                    }
+                    const uint64_t adesc = make_desc(a_base + s * stage_bytes, 8 * Cfg::row_bytes, Cfg::layout);
+                    const uint64_t bdesc = make_desc(w_base + tap * tap_bytes, 8 * Cfg::row_bytes, Cfg::layout);
+#pragma unroll
+                    for (int k = 0; k < KC / 16; ++k) tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (j | k) != 0);
+                    tc_commit(empty_bar(s));
+                    if (++s == n_stages) { s = 0; ph ^= 1u; }
+                }
+                if (ok) tc_commit(tfull_bar(a));
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int grp = (warp - 2) >> 2;
+        int it = grp;
+        bool ok = true;
+        for (int tile = blockIdx.x + grp * gridDim.x; tile < n_tiles && ok; tile += 2 * gridDim.x, it += 2) {
+            const int a = it & 1;
+            const uint32_t aph = (it >> 1) & 1u;
+            ok = mbar_wait(tfull_bar(a), aph, abort_flag, 24);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int cls = MODE == 0 ? 0 : tile / n_sp, sp = MODE == 0 ? tile : tile % n_sp;
+            const int pl = 32 * q + lane;
+            const size_t pix_small = (size_t)sp * kTileM + pl;  // pixel of the small map, linear over [B][Hs][Ws]
+            size_t pix_dst = pix_small;
+            if (MODE == 1) {
+                const int py = cls >> 1, px = cls & 1;
+                int n0, h0;
+                tile_origin(sp, &n0, &h0);
+                const int i = pl % Ws, jr = (pl / Ws) % rows_per_tile, nl = pl / (Ws * rows_per_tile);
+                pix_dst = ((size_t)(n0 + nl) * (2 * Hs) + 2 * (h0 + jr) + py) * (size_t)(2 * Ws) + 2 * i + px;
+            }
+            const uint32_t t_row = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * NC);
+#pragma unroll 1
+            for (int c0 = 0; c0 < NC; c0 += 16) {
+                float acc[16];
+                tc_ld16(t_row + (uint32_t)c0, acc);
+                tc_wait_ld();
+                if (c0 + 16 >= NC) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(a));
+                }
+                if (MODE == 1 && cls == 0 && res_dout != nullptr) {
+                    // gradient of the parameter-free shortcut: the block input at (2j, 2i), channel c, was added to channel
+                    // c of the block output at (j, i); the output has KC channels
+#pragma unroll
+                    for (int h = 0; h < 16; h += 8) {
+                        float d[8], o[8];
+                        load_f<bf16, 8>(res_dout + pix_small * KC + c0 + h, d);
+                        load_f<bf16, 8>(res_out + pix_small * KC + c0 + h, o);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) if (o[j] > 0.f) acc[h + j] += d[j];
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < 16; h += 8) {
+                    float v[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[j] = acc[h + j];
+                    store_f<bf16, 8>(dst + pix_dst * NC + c0 + h, v);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
+                     : "memory");
+    }
+}
+
+// Weight gradient of the stride-2 convolution: dw[co][ci][tap] = sum_p dy[p][co] * x[tap box][p][ci].  Per tile of 128
+// output pixels one dy box and the nine tap boxes of the forward pass; both operands MN-major (pixels are the
+// contraction axis), M = 128 (rows >= Co unused), the taps stacked along N through the leading-dimension offset
+// (N = 9 Ci, split in two instructions when it exceeds 256).  A CTA accumulates its tiles in TMEM and writes one fp32
+// partial [tap][ci][co].
+template <int CI>
+__global__ void __launch_bounds__(kWgThreads, 1)
+wgrad_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
+                   float *__restrict__ part, int Hs, int Ws, int rows_per_tile, int imgs_per_tile, int n_tiles, int n_stages) {
+    constexpr int CO = 2 * CI;
+    typedef TcCfg<CI> CfgX;
+    typedef TcCfg<CO> CfgY;
+    constexpr int stage_bytes = CfgY::tile_bytes + 9 * CfgX::tile_bytes;
+    constexpr int n_total = 9 * CI;
+    constexpr int n_first = n_total <= 256 ? n_total : 5 * CI;  // taps 0-4, then taps 5-8
+    constexpr int tmem_cols = n_total <= 256 ? 256 : 512;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *tail = smem_raw + (base - raw) + (size_t)n_stages * stage_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 1) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 1) * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+    const uint32_t done_bar = bar0 + 8u * (2 * kMaxStages);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t0 = (int)((long)n_tiles * blockIdx.x / gridDim.x), t1 = (int)((long)n_tiles * (blockIdx.x + 1) / gridDim.x);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(done_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                     "r"((uint32_t)tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    pdl_launch();
+    pdl_wait();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    const int tiles_per_img = Hs / rows_per_tile;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = t0; tile < t1 && ok; ++tile) {
+                int n0, h0;
+                if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }
+                else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
+                ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 31);
+                if (!ok) break;
+                const uint32_t st = base + s * stage_bytes;
+                mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
+                tma_load_4d(st, &tmap_dy, full_bar(s), 0, 0, h0, n0);
+                for (int tap = 0; tap < 9; ++tap) {
+                    const int ky = tap / 3, kx = tap % 3;
+                    tma_load_5d(st + CfgY::tile_bytes + tap * CfgX::tile_bytes, &tmap_x, full_bar(s), kx == 1 ? 0 : CI,
+                                kx == 0 ? -1 : 0, ky == 1 ? 0 : 1, h0 + (ky == 0 ? -1 : 0), n0);
+                }
+                if (++s == n_stages) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) for (int i = 0; i < 2000; ++i) __nanosleep(100);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(kTileM >> 4) << 24);
+            const uint32_t idesc_a = idesc0 | ((uint32_t)(n_first >> 3) << 17);
+            const uint32_t idesc_b = idesc0 | ((uint32_t)((n_total - n_first) >> 3) << 17);
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = t0; tile < t1 && ok; ++tile) {
+                ok = mbar_wait(full_bar(s), ph, abort_flag, 32);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t st = base + s * stage_bytes;
+#pragma unroll
+                for (int k = 0; k < kTileM / 16; ++k) {
+                    // 16 pixels further along the contraction axis in each operand
+                    const uint64_t adesc = make_desc(st + (uint32_t)k * 16 * CfgY::row_bytes, 8 * CfgY::row_bytes, CfgY::layout, 2 * CO * CO);
+                    const uint32_t xb = st + CfgY::tile_bytes + (uint32_t)k * 16 * CfgX::row_bytes;
+                    const uint64_t bdesc = make_desc(xb, 8 * CfgX::row_bytes, CfgX::layout, CfgX::tile_bytes);
+                    tc_mma_bf16(tmem_base, adesc, bdesc, idesc_a, (tile != t0) || (k != 0));
+                    if (n_first < n_total) {
+                        const uint64_t bdesc2 = make_desc(xb + 5 * CfgX::tile_bytes, 8 * CfgX::row_bytes, CfgX::layout, CfgX::tile_bytes);
+                        tc_mma_bf16(tmem_base + (uint32_t)n_first, adesc, bdesc2, idesc_b, (tile != t0) || (k != 0));
+                    }
+                }
+                tc_commit(empty_bar(s));
+                if (++s == n_stages) { s = 0; ph ^= 1u; }
+            }
+            if (ok) tc_commit(done_bar);
+        }
+    } else {
+        const int q = warp & 3;
+        bool ok = mbar_wait(done_bar, 0, abort_flag, 33);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok && 32 * q < CO) {
+            tc_fence_after();
+            const int co = 32 * q + lane;
+            float *out = part + (size_t)blockIdx.x * 9 * CI * CO;
+#pragma unroll 1
+            for (int c0 = 0; c0 < n_total; c0 += 16) {
+                float v[16];
+                tc_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, v);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) out[(size_t)(c0 + j) * CO + co] = v[j];  // column = tap*Ci + ci
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
+                     : "memory");
+    }
+}
+
 // dw[co][ci][tap] = sum over chunks of part[chunk][tap][ci][co].  64 outputs per CTA, four threads per output: thread g
 // adds chunks g, g+4, ... (four independent loads in flight per thread), the four sums are combined in a fixed order.
+// C = input channels of the partials, Co = output channels, cin <= C = input channels of dw.
 __global__ void __launch_bounds__(256) wgrad_tc_fold_kernel(const float *__restrict__ part, float *__restrict__ dw, int chunks, int C,
-                                                            int cin) {
+                                                            int Co, int cin) {
     pdl_launch();
     pdl_wait();
     __shared__ float sm[4][64];
-    const int total = 9 * C * C;
+    const int total = 9 * C * Co;
     const int o = threadIdx.x & 63, g = threadIdx.x >> 6;
     const int i = blockIdx.x * 64 + o;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -584,7 +964,7 @@ __global__ void __launch_bounds__(256) wgrad_tc_fold_kernel(const float *__restr
     __syncthreads();
     if (g == 0 && i < total) {
         const float t = (sm[0][o] + sm[1][o]) + (sm[2][o] + sm[3][o]);
-        const int co = i % C, ci = (i / C) % C, tap = i / (C * C);
+        const int co = i % Co, ci = (i / Co) % C, tap = i / (C * Co);
         if (ci < cin) dw[((size_t)co * cin + ci) * 9 + tap] = t;  // cin < C: the input was zero-padded to C channels
     }
 }
@@ -626,6 +1006,30 @@ bool get_map(const void *ptr, int B, int H, int W, int C, int rows, int imgs, CU
     if (r != CUDA_SUCCESS) return false;
     if (g_maps.size() > 8192) g_maps.clear();
     g_maps[key] = m;
+    *out = m;
+    return true;
+}
+
+// Tensor map of the stride-2 view of an NHWC bf16 tensor [B][H][W][C]: axes (pixel pair = 2C, W/2, row parity, H/2, B),
+// box (C, W/2, 1, rows, imgs): one column parity of one row parity.
+std::map<MapKey, CUtensorMap> g_maps_s2;
+bool get_map_s2(const void *ptr, int B, int H, int W, int C, int rows, int imgs, CUtensorMap *out) {
+    std::lock_guard<std::mutex> lock(g_maps_mu);
+    MapKey key{ptr, B, H, W, C, rows, imgs};
+    auto it = g_maps_s2.find(key);
+    if (it != g_maps_s2.end()) { *out = it->second; return true; }
+    cuuint64_t dims[5] = {(cuuint64_t)2 * C, (cuuint64_t)W / 2, 2, (cuuint64_t)H / 2, (cuuint64_t)B};
+    cuuint64_t strides[4] = {(cuuint64_t)2 * C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)2 * W * C * 2, (cuuint64_t)H * W * C * 2};
+    cuuint32_t box[5] = {(cuuint32_t)C, (cuuint32_t)(W / 2), 1, (cuuint32_t)rows, (cuuint32_t)imgs};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUtensorMapSwizzle swz = C == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (C == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    CUtensorMap m;
+    CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return false;
+    if (g_maps_s2.size() > 1024) g_maps_s2.clear();
+    g_maps_s2[key] = m;
     *out = m;
     return true;
 }
@@ -674,11 +1078,94 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int max_chunks = slab ? (C == 16 ? 74 : 37) : 24;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
     launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
-    launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C, cin);
+    launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C, C, cin);
+    return 2;
+}
+
+template <int KC, int NC, int MODE>
+size_t s2_smem_bytes(int n_stages) {
+    return 1024 + ((9 * KC * NC * 2 + 1023) & ~1023) + (size_t)n_stages * TcCfg<KC>::tile_bytes + 512;
+}
+// H, W: the large (input-resolution) map.  dir 0: src = x [B][H][W][CI] -> dst = y [B][H/2][W/2][2CI];
+// dir 1: src = dy -> dst = dx, plus the parameter-free shortcut's gradient when sc.mode == 2.
+template <int CI>
+int launch_tc_s2(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, Shortcut sc,
+                 cudaStream_t s) {
+    constexpr int CO = 2 * CI;
+    const int Hs = H / 2, Ws = W / 2;
+    int rows, imgs;
+    tile_geometry(Hs, Ws, &rows, &imgs);
+    const int n_sp = (int)((long)B * Hs * Ws / kTileM);
+    const uint8_t *pk = (const uint8_t *)w_packed;
+    CUtensorMap map;
+    if (dir == 0) {
+        if (!get_map_s2(src, B, H, W, CI, rows, imgs, &map)) return -1;
+        int n_stages = kSmemBudget / TcCfg<CI>::tile_bytes;
+        if (n_stages > kMaxStages) n_stages = kMaxStages;
+        const int grid = n_sp < g_num_sms ? n_sp : g_num_sms;
+        launch_k(conv3x3_s2_tc_kernel<CI, CO, 0>, grid, kTcThreads, s2_smem_bytes<CI, CO, 0>(n_stages), s, map, (const bf16 *)w, pk,
+                 (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages, (const bf16 *)nullptr, (const bf16 *)nullptr);
+    } else {
+        if (!get_map(src, B, Hs, Ws, CO, rows, imgs, &map)) return -1;
+        int n_stages = (kSmemBudget - 9 * CI * CO * 2) / TcCfg<CO>::tile_bytes;
+        if (n_stages > kMaxStages) n_stages = kMaxStages;
+        if (n_stages < 3) n_stages = 3;
+        const int n_tiles = 4 * n_sp;
+        const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
+        launch_k(conv3x3_s2_tc_kernel<CO, CI, 1>, grid, kTcThreads, s2_smem_bytes<CO, CI, 1>(n_stages), s, map, (const bf16 *)w,
+                 pk ? pk + S2Cfg<CI>::img_bytes : pk, (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages,
+                 sc.mode == 2 ? (const bf16 *)sc.a : nullptr, sc.mode == 2 ? (const bf16 *)sc.b : nullptr);
+    }
+    return 1;
+}
+
+template <int CI>
+int launch_wg_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, cudaStream_t s) {
+    constexpr int CO = 2 * CI;
+    const int Hs = H / 2, Ws = W / 2;
+    int rows, imgs;
+    tile_geometry(Hs, Ws, &rows, &imgs);
+    CUtensorMap mx, md;
+    if (!get_map_s2(x, B, H, W, CI, rows, imgs, &mx) || !get_map(dy, B, Hs, Ws, CO, rows, imgs, &md)) return -1;
+    const int stage_bytes = TcCfg<CO>::tile_bytes + 9 * TcCfg<CI>::tile_bytes;
+    int n_stages = (200 * 1024) / stage_bytes;
+    if (n_stages > 4) n_stages = 4;
+    const int n_tiles = (int)((long)B * Hs * Ws / kTileM);
+    const int max_chunks = 64;
+    const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
+    launch_k(wgrad_s2_tc_kernel<CI>, chunks, kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, Hs, Ws,
+             rows, imgs, n_tiles, n_stages);
+    launch_k(wgrad_tc_fold_kernel, ceil_div(9 * CI * CO, 64), 256, 0, s, scratch, dw, chunks, CI, CO, CI);
     return 2;
 }
 
 }  // namespace
+
+// stride 2, Cout = 2 Cin, Cin in {16, 32}, output map 16x16 or 8x8 in whole 128-pixel tiles
+bool conv_tc_s2_supported(int B, int H, int W, int Cin, int Cout, int stride) {
+    if (!g_encode) return false;
+    if (stride != 2 || Cout != 2 * Cin || (Cin != 16 && Cin != 32)) return false;
+    if ((H & 1) || (W & 1)) return false;
+    const int Hs = H / 2, Ws = W / 2;
+    if (Ws < 4 || Ws > 32 || kTileM % Ws != 0) return false;
+    const int r = kTileM / Ws;
+    if (r <= Hs) { if (Hs % r != 0) return false; }
+    else { if (kTileM % (Hs * Ws) != 0 || B % (kTileM / (Hs * Ws)) != 0) return false; }
+    return ((long)B * Hs * Ws) % kTileM == 0;
+}
+size_t tc_s2_packed_bytes(int Cin) { return 2 * (size_t)9 * Cin * 2 * Cin * 2; }
+
+int launch_conv_tc_s2(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int Cin,
+                      Shortcut sc, cudaStream_t s) {
+    if (Cin == 16) return launch_tc_s2<16>(dir, src, w, w_packed, dst, B, H, W, sc, s);
+    if (Cin == 32) return launch_tc_s2<32>(dir, src, w, w_packed, dst, B, H, W, sc, s);
+    return -1;
+}
+int launch_wgrad_tc_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int Cin, cudaStream_t s) {
+    if (Cin == 16) return launch_wg_s2<16>(x, dy, dw, scratch, B, H, W, s);
+    if (Cin == 32) return launch_wg_s2<32>(x, dy, dw, scratch, B, H, W, s);
+    return -1;
+}
 
 bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
     if (!g_encode) return false;
@@ -747,9 +1234,12 @@ int conv_tc_init() {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-    const void *fns[6] = {(const void *)conv3x3_tc_kernel<16>, (const void *)conv3x3_tc_kernel<32>,
-                          (const void *)conv3x3_tc_kernel<64>, (const void *)wgrad_tc_kernel<16>,
-                          (const void *)wgrad_tc_kernel<32>, (const void *)wgrad_tc_kernel<64>};
+    const void *fns[12] = {(const void *)conv3x3_tc_kernel<16>, (const void *)conv3x3_tc_kernel<32>,
+                           (const void *)conv3x3_tc_kernel<64>, (const void *)wgrad_tc_kernel<16>,
+                           (const void *)wgrad_tc_kernel<32>, (const void *)wgrad_tc_kernel<64>,
+                           (const void *)conv3x3_s2_tc_kernel<16, 32, 0>, (const void *)conv3x3_s2_tc_kernel<32, 64, 0>,
+                           (const void *)conv3x3_s2_tc_kernel<32, 16, 1>, (const void *)conv3x3_s2_tc_kernel<64, 32, 1>,
+                           (const void *)wgrad_s2_tc_kernel<16>, (const void *)wgrad_s2_tc_kernel<32>};
     for (const void *f : fns) {
         e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
         if (e != cudaSuccess) break;

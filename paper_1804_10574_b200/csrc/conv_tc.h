@@ -19,10 +19,21 @@ int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed
                    Shortcut sc, cudaStream_t s);
 size_t tc_packed_bytes(int C);
 // One launch that re-arranges the filters of many convolutions of one weight version.
-struct PackJobHost { long src_off; long dst_off; int C; int first_elem; int cin_real; int pad_; };  // element offset in wver, byte offset in packed
+// element offset in wver, byte offset in packed; pad_ = job kind: 0 stride-1 C x C filter, 1 stride-2 C -> 2C filter
+struct PackJobHost { long src_off; long dst_off; int C; int first_elem; int cin_real; int pad_; };
 int launch_pack_one(const void *w, void *packed, int C, cudaStream_t s);
 int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,
                         cudaStream_t s);
+
+// Stride-2 convolutions of the down-sampling blocks: Cout = 2 Cin, Cin in {16, 32}, even H and W, output map in whole
+// 128-pixel tiles.  H, W are the input size.  dir as above; in dir 1 sc.mode == 2 adds the gradient of the
+// parameter-free shortcut (sc.a = gradient of the block output, sc.b = block output).  w_packed (nullable):
+// tc_s2_packed_bytes(Cin) bytes written by launch_pack_filters for a job of kind 1.
+bool conv_tc_s2_supported(int B, int H, int W, int Cin, int Cout, int stride);
+size_t tc_s2_packed_bytes(int Cin);
+int launch_conv_tc_s2(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int Cin,
+                      Shortcut sc, cudaStream_t s);
+int launch_wgrad_tc_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int Cin, cudaStream_t s);
 
 bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
 size_t wgrad_tc_scratch_elems();

@@ -137,18 +137,24 @@ int conv_fwd(ddg_ctx *c, const void *x, const void *w, const void *wp, void *y, 
              int stride, int relu, cudaStream_t s) {
     if (c->prec == P_BF16 && !relu && conv_tc_supported(c->B, H, W, Cin, Cout, stride))
         return launch_conv_tc(0, x, w, wp, y, c->B, H, W, Cin, Shortcut{}, s);
+    if (c->prec == P_BF16 && !relu && conv_tc_s2_supported(c->B, H, W, Cin, Cout, stride))
+        return launch_conv_tc_s2(0, x, w, wp, y, c->B, H, W, Cin, Shortcut{}, s);
     return launch_conv_fwd_direct(c->prec, x, w, y, c->B, H, W, Cin, Cout, stride, relu, s);
 }
 int conv_dgrad(ddg_ctx *c, const void *dy, const void *w, const void *wp, void *dx, int H, int W, int Cin, int Cout,
                int stride, Shortcut sc, cudaStream_t s) {
     if (c->prec == P_BF16 && sc.mode != 2 && conv_tc_supported(c->B, H, W, Cin, Cout, stride))
         return launch_conv_tc(1, dy, w, wp, dx, c->B, H, W, Cin, sc, s);
+    if (c->prec == P_BF16 && sc.mode != 1 && conv_tc_s2_supported(c->B, H, W, Cin, Cout, stride))
+        return launch_conv_tc_s2(1, dy, w, wp, dx, c->B, H, W, Cin, sc, s);
     return launch_conv_dgrad_direct(c->prec, dy, w, dx, c->B, H, W, Cin, Cout, stride, sc, s);
 }
 int conv_wgrad(ddg_ctx *c, Module &m, const void *x, const void *dy, float *dw, int H, int W, int Cin, int Cout,
                int stride, cudaStream_t s) {
     if (c->prec == P_BF16 && wgrad_tc_supported(c->B, H, W, Cin, Cout, stride))
         return launch_wgrad_tc(x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cin, s);
+    if (c->prec == P_BF16 && conv_tc_s2_supported(c->B, H, W, Cin, Cout, stride))
+        return launch_wgrad_tc_s2(x, dy, dw, m.wg_scratch, c->B, H, W, Cin, s);
     return launch_conv_wgrad_direct(c->prec, x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cout, stride, s);
 }
 
@@ -712,6 +718,13 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
             size_t pk_off = 0;
             int elems = 0;
             auto plan = [&](long *slot, size_t w_off, int H, int W, int Ci, int Co, int stride, int cin_real = 0) {
+                if (conv_tc_s2_supported(c->B, H, W, Ci, Co, stride)) {
+                    *slot = (long)pk_off;
+                    jobs.push_back(PackJobHost{(long)w_off, (long)pk_off, Ci, elems, Ci, 1});
+                    pk_off += tc_s2_packed_bytes(Ci);
+                    elems += 9 * Ci * Co;
+                    return;
+                }
                 if (!conv_tc_supported(c->B, H, W, Ci, Co, stride)) return;
                 *slot = (long)pk_off;
                 jobs.push_back(PackJobHost{(long)w_off, (long)pk_off, Ci, elems, cin_real ? cin_real : Ci, 0});

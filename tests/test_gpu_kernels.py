@@ -31,7 +31,8 @@ def from_dev(t_nhwc):
 
 SHAPES = [  # B, H, W, Cin, Cout, stride
     (2, 8, 8, 16, 16, 1), (3, 32, 32, 16, 16, 1), (5, 16, 16, 32, 32, 1), (9, 8, 8, 64, 64, 1),
-    (3, 32, 32, 16, 32, 2), (3, 16, 16, 32, 64, 2), (4, 32, 32, 3, 16, 1), (2, 7, 5, 5, 12, 1), (2, 9, 7, 6, 10, 2),
+    (3, 32, 32, 16, 32, 2), (3, 16, 16, 32, 64, 2), (6, 16, 16, 32, 64, 2), (7, 32, 32, 32, 64, 2), (10, 16, 16, 16, 32, 2),
+    (4, 32, 32, 3, 16, 1), (2, 7, 5, 5, 12, 1), (2, 9, 7, 6, 10, 2),
     (128, 8, 8, 64, 64, 1),
 ]
 
@@ -127,7 +128,9 @@ def test_tensor_core_path_takes_the_resnet_shapes():
     from paper_1804_10574_b200 import binding
     for B, H, W, C in [(128, 32, 32, 16), (128, 16, 16, 32), (128, 8, 8, 64), (2, 8, 8, 16), (3, 32, 32, 16)]:
         assert binding.tensor_core_path(B, H, W, C, C, 1) & 1, (B, H, W, C)
-    assert binding.tensor_core_path(128, 32, 32, 16, 32, 2) & 1 == 0      # stride 2 stays on CUDA cores
+    assert binding.tensor_core_path(128, 32, 32, 16, 32, 2) == 3           # the down-sampling convolutions too
+    assert binding.tensor_core_path(128, 16, 16, 32, 64, 2) == 3
+    assert binding.tensor_core_path(3, 16, 16, 32, 64, 2) == 0             # 8x8 output: tiles are image pairs
     assert binding.tensor_core_path(9, 8, 8, 64, 64, 1) & 1 == 0          # 576 pixels: not whole 128-pixel tiles
 
 
