@@ -159,8 +159,26 @@ template <int C> __host__ __device__ inline ConvSmem conv_smem_plan(int n_stages
     p.tail_off = p.a_off + (uint32_t)n_stages * (uint32_t)stage_bytes;
     return p;
 }
+// after the pipeline stages: 512 bytes of barriers and flags, 4 KB of per-warp batch-norm sums (8 warps x 4 channel
+// chunks x 32 lanes), 512 bytes of per-channel mean / invstd
+constexpr int kTailBytes = 512 + 4096 + 512;
 template <int C> inline size_t conv_smem_bytes(int n_stages, int stage_bytes) {
-    return 1024 + conv_smem_plan<C>(n_stages, stage_bytes).tail_off + 512;
+    return 1024 + conv_smem_plan<C>(n_stages, stage_bytes).tail_off + kTailBytes;
+}
+
+// Sum of v[i] over the 32 lanes of a warp for 32 values at once: after the call lane l holds the total of v[l] in
+// v[0].  Each step halves the values a lane keeps (31 shuffles in all instead of 32 x 5).
+__device__ __forceinline__ void warp_transpose_sum32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int step = 16; step >= 1; step >>= 1) {
+        const bool upper = (lane & step) != 0;
+#pragma unroll
+        for (int i = 0; i < step; ++i) {
+            const float send = upper ? v[i] : v[i + step];
+            const float keep = upper ? v[i + step] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
+        }
+    }
 }
 
 // Filter images for the tensor-core kernels: per convolution two blocks of 3 swizzled K-major [3C][C] bf16 tiles (one
@@ -244,7 +262,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
                   bf16 *__restrict__ dst, int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
                   int slab, int n_stages, int stage_bytes, const bf16 *__restrict__ res_dout,
-                  const bf16 *__restrict__ res_out) {
+                  const bf16 *__restrict__ res_out, float *__restrict__ stat_part, const bf16 *__restrict__ bn_mask,
+                  const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd) {
+    // stat_part != nullptr: the epilogue also reduces, per channel over the pixels of this CTA's tiles, the two sums the
+    // batch norm that follows needs, from the values as stored (rounded to bf16), and writes them to
+    // stat_part[blockIdx.x][2C]:   bn_x == nullptr: (sum y, sum y^2) for the forward statistics;
+    // otherwise (sum dz, sum dz * xhat) with dz = result * [bn_mask > 0], xhat = (bn_x - mean) * invstd: the sums of the
+    // batch-norm backward whose incoming gradient this kernel produces.
     typedef TcCfg<C> Cfg;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -256,6 +280,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[4], tempty[4], wbar
     uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 9) * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 9) * 8 + 8);
+    float (*sm_run)[4][32] = reinterpret_cast<float (*)[4][32]>(tail + 512);  // [epilogue warp][channel chunk][lane]
+    float *sm_stat = reinterpret_cast<float *>(tail + 512 + 4096);            // mean[C], invstd[C]
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
@@ -265,6 +291,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    if (stat_part != nullptr)
+        for (int i = threadIdx.x; i < 8 * 4 * 32; i += kTcThreads) (&sm_run[0][0][0])[i] = 0.f;
     if (threadIdx.x == 0) {
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < Cfg::acc_stages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
@@ -282,6 +310,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     // this point touches global memory
     pdl_launch();
     pdl_wait();
+    if (bn_x != nullptr && threadIdx.x < 2 * C)
+        sm_stat[threadIdx.x] = threadIdx.x < C ? bn_mean[threadIdx.x] : bn_invstd[threadIdx.x - C];
     if (w_packed == nullptr) {
         // filter in canonical order: stage it here as 9 K-major [C rows = output channel of this pass][C] tiles
         for (int i = threadIdx.x; i < 9 * C * C; i += kTcThreads) {
@@ -413,6 +443,33 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                     for (int j = 0; j < 8; ++j) v[j] = acc[h + j];
                     store_f<bf16, 8>(dst + pix * C + c0 + h, v);
                 }
+                if (stat_part != nullptr) {
+                    float v[32];
+                    if (bn_x == nullptr) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float r = __bfloat162float(__float2bfloat16_rn(acc[j]));
+                            v[j] = r;
+                            v[16 + j] = r * r;
+                        }
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < 16; h += 8) {
+                            float mk[8], xv[8];
+                            load_f<bf16, 8>(bn_mask + pix * C + c0 + h, mk);
+                            load_f<bf16, 8>(bn_x + pix * C + c0 + h, xv);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                float d = __bfloat162float(__float2bfloat16_rn(acc[h + j]));
+                                if (!(mk[j] > 0.f)) d = 0.f;
+                                v[h + j] = d;
+                                v[16 + h + j] = d * (xv[j] - sm_stat[c0 + h + j]) * sm_stat[C + c0 + h + j];
+                            }
+                        }
+                    }
+                    warp_transpose_sum32(v, lane);
+                    sm_run[warp - 2][c0 >> 4][lane] += v[0];  // lane l < 16: first sum of channel c0+l; else second sum
+                }
             }
         }
     }
@@ -422,6 +479,13 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::tmem_cols)
                      : "memory");
+    }
+    if (stat_part != nullptr && threadIdx.x < 2 * C) {  // the eight epilogue warps' sums in a fixed order
+        const int c = threadIdx.x % C, l = (c & 15) + 16 * (threadIdx.x / C);
+        float t = 0.f;
+#pragma unroll
+        for (int wq = 0; wq < 8; ++wq) t += sm_run[wq][c >> 4][l];
+        stat_part[(size_t)blockIdx.x * 2 * C + threadIdx.x] = t;
     }
 }
 
@@ -1042,7 +1106,7 @@ constexpr int kSmemMax = 227 * 1024;
 
 template <int C>
 int launch_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W,
-              Shortcut sc, cudaStream_t s) {
+              Shortcut sc, BnFuse bf, cudaStream_t s) {
     int rows, imgs;
     tile_geometry(H, W, &rows, &imgs);
     const int slab = (imgs == 1) ? 1 : 0;
@@ -1056,7 +1120,8 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
     launch_k(conv3x3_tc_kernel<C>, grid, kTcThreads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
-        stage_bytes, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr);
+        stage_bytes, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
+        (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd);
     return 1;
 }
 
@@ -1180,13 +1245,18 @@ bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
 size_t tc_packed_bytes(int C) { return 2 * (size_t)9 * C * C * 2; }
 
 int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
-                   Shortcut sc, cudaStream_t s) {
+                   Shortcut sc, cudaStream_t s, BnFuse bf) {
     switch (C) {
-    case 16: return launch_tc<16>(dir, src, w, w_packed, dst, B, H, W, sc, s);
-    case 32: return launch_tc<32>(dir, src, w, w_packed, dst, B, H, W, sc, s);
-    case 64: return launch_tc<64>(dir, src, w, w_packed, dst, B, H, W, sc, s);
+    case 16: return launch_tc<16>(dir, src, w, w_packed, dst, B, H, W, sc, bf, s);
+    case 32: return launch_tc<32>(dir, src, w, w_packed, dst, B, H, W, sc, bf, s);
+    case 64: return launch_tc<64>(dir, src, w, w_packed, dst, B, H, W, sc, bf, s);
     }
     return -1;
+}
+
+int conv_tc_grid(int B, int H, int W) {
+    const int n_tiles = (int)((long)B * H * W / kTileM);
+    return n_tiles < g_num_sms ? n_tiles : g_num_sms;
 }
 
 int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,

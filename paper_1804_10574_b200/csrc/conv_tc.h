@@ -15,8 +15,19 @@ bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
 // w: filter in canonical [Cout][Cin][3][3] order.  w_packed (nullable): the pre-arranged filter images written by
 // launch_pack_filters for this convolution (tc_packed_bytes(C) bytes: forward image, then input-gradient image); when
 // given, the kernel fetches its filter with one bulk copy instead of re-arranging the canonical one itself.
+// bf.part != nullptr: the kernel also leaves, in bf.part[conv_tc_grid(B, H, W)][2C], per-CTA partial sums over its
+// output for the batch norm that consumes it: with bf.x == nullptr (sum y, sum y^2) per channel (forward statistics);
+// otherwise (sum dz, sum dz * xhat), dz = output * [bf.mask > 0], xhat = (bf.x - bf.mean) * bf.invstd (the two
+// reductions of the batch-norm backward whose incoming gradient is this kernel's output).  The partials are summed
+// in a fixed order by the batch-norm kernel that follows.
+struct BnFuse {
+    float *part = nullptr;
+    const void *mask = nullptr, *x = nullptr;
+    const float *mean = nullptr, *invstd = nullptr;
+};
 int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
-                   Shortcut sc, cudaStream_t s);
+                   Shortcut sc, cudaStream_t s, BnFuse bf = BnFuse());
+int conv_tc_grid(int B, int H, int W);
 size_t tc_packed_bytes(int C);
 // One launch that re-arranges the filters of many convolutions of one weight version.
 // element offset in wver, byte offset in packed; pad_ = job kind: 0 stride-1 C x C filter, 1 stride-2 C -> 2C filter

@@ -158,6 +158,13 @@ int conv_wgrad(ddg_ctx *c, Module &m, const void *x, const void *dy, float *dw, 
     return launch_conv_wgrad_direct(c->prec, x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cout, stride, s);
 }
 
+// Batch-norm sums taken in the epilogue of the tensor-core convolution that produces the batch norm's input
+// (DDG_FUSE_BN=0 in the environment keeps the separate reduction kernels).
+bool bn_fuse_enabled() {
+    static const bool on = [] { const char *e = getenv("DDG_FUSE_BN"); return !(e && e[0] == '0'); }();
+    return on;
+}
+
 // ---- forward sweep of module k on the minibatch of iteration t (Eq. 3) --------------------------------
 long forward_module(ddg_ctx *c, int k, long t) {
     Module &m = c->mods[k];
@@ -212,15 +219,28 @@ long forward_module(ddg_ctx *c, int k, long t) {
             char *y1 = slot_ptr(c, L.y1, t), *a1 = slot_ptr(c, L.a1, t), *y2 = slot_ptr(c, L.y2, t);
             float *stt = (float *)slot_ptr(c, L.stats, t);
             const long npix = (long)B * L.Hout * L.Wout;
-            n += conv_fwd(c, in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, Co, st, 0, s);
-            n += launch_bn_stats(c->prec, y1, stt, stt + Co, m.bn_scratch, npix, Co, s);
-            n += launch_bn_apply(c->prec, y1, g1, b1, stt, stt + Co, Shortcut{}, a1, B, L.Hout, L.Wout, Co, 1, s);
-            n += conv_fwd(c, a1, w2, pkp(L.pk2), y2, L.Hout, L.Wout, Co, Co, 1, 0, s);
-            n += launch_bn_stats(c->prec, y2, stt + 2 * Co, stt + 3 * Co, m.bn_scratch, npix, Co, s);
+            // convolution followed by its batch norm; the statistics come from the convolution's epilogue where the
+            // tensor-core kernel runs, from a reduction kernel otherwise
+            auto conv_bn = [&](const void *xin, const void *wc, const void *wp, void *yc, int H, int W, int Cic, int strd,
+                               const char *gm, const char *bt, float *mean, float *invstd, Shortcut scb, void *dstb) {
+                float *part = m.bn_scratch + 32;
+                if (bn_fuse_enabled() && c->prec == P_BF16 && conv_tc_supported(B, H, W, Cic, Co, strd)) {
+                    BnFuse bf;
+                    bf.part = part;
+                    n += launch_conv_tc(0, xin, wc, wp, yc, B, H, W, Cic, Shortcut{}, s, bf);
+                    n += launch_bn_apply_part(c->prec, yc, gm, bt, part, conv_tc_grid(B, H, W), mean, invstd, scb, dstb, B,
+                                              L.Hout, L.Wout, Co, 1, s);
+                } else {
+                    n += conv_fwd(c, xin, wc, wp, yc, H, W, Cic, Co, strd, 0, s);
+                    n += launch_bn_stats(c->prec, yc, mean, invstd, m.bn_scratch, npix, Co, s);
+                    n += launch_bn_apply(c->prec, yc, gm, bt, mean, invstd, scb, dstb, B, L.Hout, L.Wout, Co, 1, s);
+                }
+            };
+            conv_bn(in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, g1, b1, stt, stt + Co, Shortcut{}, a1);
             Shortcut sc{};
             sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
             sc.a = in; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win;
-            n += launch_bn_apply(c->prec, y2, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out, B, L.Hout, L.Wout, Co, 1, s);
+            conv_bn(a1, w2, pkp(L.pk2), y2, L.Hout, L.Wout, Co, 1, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out);
             break;
         }
         }
@@ -249,6 +269,11 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
     // The weight gradient of a convolution needs only (layer input, dy); nothing on the way down to the module input
     // waits for it.  It runs on the module's side stream; dy lives in a ring of four buffers so that the chain can move
     // on, and the chain only waits when it comes back to a buffer whose weight gradient has not finished.
+    // number of per-CTA partial sums that the kernel which produced `cur` left for the batch norm that consumes it
+    // (0: none, that batch norm runs its own reduction)
+    int cur_np = 0;
+    float *bn_part = m.bn_scratch + 32;
+    const bool fuse = bn_fuse_enabled() && c->prec == P_BF16;
     int dy_i = 0, last_side = -1;
     bool ring_used[4] = {false, false, false, false};
     auto ring_next = [&]() -> int {
@@ -274,7 +299,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
         const bool mod_first = (l == m.first);
         const bool need_dx = !L.is_first;
         // destination of the error gradient w.r.t. the layer input
-        int dst_tmp = -1;
+        int dst_tmp = -1, next_np = 0;
         char *dst = nullptr;
         if (need_dx) {
             if (mod_first) dst = m.delta_out[t % 2];
@@ -328,22 +353,49 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
             (void)tA;
             const int j2 = ring_next();
             char *dy2 = m.dyring[j2], *da1 = m.tmp[tB];
-            n += launch_bn_bwd_reduce(c->prec, cur, out, y2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, m.bn_scratch, npix, Co,
-                                      1, s);
-            n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s);
+            if (cur_np > 0) {
+                n += launch_bn_bwd_apply_part(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, bn_part, cur_np, gg2, gb2,
+                                              dy2, npix, Co, 1, s);
+            } else {
+                n += launch_bn_bwd_reduce(c->prec, cur, out, y2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, m.bn_scratch, npix, Co,
+                                          1, s);
+                n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s);
+            }
             side_wgrad(j2, a1, dy2, gw2, L.Hout, L.Wout, Co, Co, 1);
-            n += conv_dgrad(c, dy2, w2, pkp(L.pk2), da1, L.Hout, L.Wout, Co, Co, 1, Shortcut{}, s);
             const int j1 = ring_next();
             char *dy1 = m.dyring[j1];
-            n += launch_bn_bwd_reduce(c->prec, da1, a1, y1, stt, stt + Co, gg1, gb1, m.bn_scratch, npix, Co, 1, s);
-            n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
+            if (fuse && conv_tc_supported(B, L.Hout, L.Wout, Co, Co, 1)) {
+                // the input gradient of conv2 is the incoming gradient of bn1: its two sums come out of the same kernel
+                BnFuse bf;
+                bf.part = bn_part; bf.mask = a1; bf.x = y1; bf.mean = stt; bf.invstd = stt + Co;
+                n += launch_conv_tc(1, dy2, w2, pkp(L.pk2), da1, B, L.Hout, L.Wout, Co, Shortcut{}, s, bf);
+                n += launch_bn_bwd_apply_part(c->prec, da1, a1, y1, g1, stt, stt + Co, bn_part, conv_tc_grid(B, L.Hout, L.Wout),
+                                              gg1, gb1, dy1, npix, Co, 1, s);
+            } else {
+                n += conv_dgrad(c, dy2, w2, pkp(L.pk2), da1, L.Hout, L.Wout, Co, Co, 1, Shortcut{}, s);
+                n += launch_bn_bwd_reduce(c->prec, da1, a1, y1, stt, stt + Co, gg1, gb1, m.bn_scratch, npix, Co, 1, s);
+                n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
+            }
             side_wgrad(j1, in, dy1, gw1, L.Hin, L.Win, Ci, Co, st);
             if (need_dx) {
                 Shortcut sc{};
                 sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
                 sc.a = cur; sc.b = out; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win;
                 char *dx = mod_first ? dst : da1;  // da1 is dead once bn1's backward has run
-                n += conv_dgrad(c, dy1, w1, pkp(L.pk1), dx, L.Hin, L.Win, Ci, Co, st, sc, s);
+                const LayerPlan *Pv = mod_first ? nullptr : &c->layers[l - 1];
+                if (fuse && Pv && Pv->spec.kind == DDG_BASIC_BLOCK && sc.mode == 1 &&
+                    conv_tc_supported(B, L.Hin, L.Win, Ci, Co, st)) {
+                    // dx is the incoming gradient of the block below, whose second batch norm reduces it first: take
+                    // those sums here (its output is this block's input, its bn2 input and statistics are in its slots)
+                    const float *pst = (const float *)slot_ptr(c, Pv->stats, sidx);
+                    BnFuse bf;
+                    bf.part = bn_part; bf.mask = in; bf.x = slot_ptr(c, Pv->y2, sidx);
+                    bf.mean = pst + 2 * Ci; bf.invstd = pst + 3 * Ci;
+                    n += launch_conv_tc(1, dy1, w1, pkp(L.pk1), dx, B, L.Hin, L.Win, Ci, sc, s, bf);
+                    next_np = conv_tc_grid(B, L.Hin, L.Win);
+                } else {
+                    n += conv_dgrad(c, dy1, w1, pkp(L.pk1), dx, L.Hin, L.Win, Ci, Co, st, sc, s);
+                }
                 if (!mod_first) { dst = dx; dst_tmp = tB; }
             }
             break;
@@ -351,6 +403,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
         }
         cur = dst;
         cur_tmp = dst_tmp;
+        cur_np = next_np;
     }
     side_join();  // the update that follows reads every gradient of the module
     return n;
