@@ -262,13 +262,15 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
                   bf16 *__restrict__ dst, int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
                   int slab, int n_stages, int stage_bytes, const bf16 *__restrict__ res_dout,
-                  const bf16 *__restrict__ res_out, float *__restrict__ stat_part, const bf16 *__restrict__ bn_mask,
+                  const bf16 *__restrict__ res_out, float *__restrict__ stat_part, unsigned *__restrict__ stat_counter,
+                  float *__restrict__ stat_o0, float *__restrict__ stat_o1, const bf16 *__restrict__ bn_mask,
                   const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd) {
     // stat_part != nullptr: the epilogue also reduces, per channel over the pixels of this CTA's tiles, the two sums the
-    // batch norm that follows needs, from the values as stored (rounded to bf16), and writes them to
-    // stat_part[blockIdx.x][2C]:   bn_x == nullptr: (sum y, sum y^2) for the forward statistics;
-    // otherwise (sum dz, sum dz * xhat) with dz = result * [bn_mask > 0], xhat = (bn_x - mean) * invstd: the sums of the
-    // batch-norm backward whose incoming gradient this kernel produces.
+    // batch norm that follows needs, from the values as stored (rounded to bf16), writes them to
+    // stat_part[blockIdx.x][2C], and the CTA that finishes last adds the partials in a fixed order:
+    //   bn_x == nullptr: (sum y, sum y^2) -> stat_o0 = mean, stat_o1 = 1/sqrt(var + eps) (forward statistics);
+    //   otherwise (sum dz, sum dz * xhat) with dz = result * [bn_mask > 0], xhat = (bn_x - mean) * invstd -> stat_o0 =
+    //   dbeta, stat_o1 = dgamma: the sums of the batch-norm backward whose incoming gradient this kernel produces.
     typedef TcCfg<C> Cfg;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -480,13 +482,54 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::tmem_cols)
                      : "memory");
     }
-    if (stat_part != nullptr && threadIdx.x < 2 * C) {  // the eight epilogue warps' sums in a fixed order
+    if (stat_part == nullptr) return;
+    if (threadIdx.x < 2 * C) {  // the eight epilogue warps' sums in a fixed order
         const int c = threadIdx.x % C, l = (c & 15) + 16 * (threadIdx.x / C);
         float t = 0.f;
 #pragma unroll
         for (int wq = 0; wq < 8; ++wq) t += sm_run[wq][c >> 4][l];
         stat_part[(size_t)blockIdx.x * 2 * C + threadIdx.x] = t;
     }
+    __threadfence();
+    __syncthreads();
+    int *is_last = reinterpret_cast<int *>(sm_stat);  // free again: the epilogue is over
+    if (threadIdx.x == 0) *is_last = (atomicAdd(stat_counter, 1u) == gridDim.x - 1) ? 1 : 0;
+    __syncthreads();
+    if (!*is_last) return;
+    __threadfence();
+    // last CTA: partials of all CTAs, `ways` threads per value, eight loads in flight per thread, fixed order
+    double *fold = reinterpret_cast<double *>(&sm_run[0][0][0]);  // kTcThreads doubles fit the 4 KB
+    constexpr int nval = 2 * C, ways = kTcThreads / nval;
+    const int v = threadIdx.x % nval, way = threadIdx.x / nval;
+    double acc = 0.0;
+    if (way < ways) {
+        double a8[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+        unsigned i = way;
+        for (; i + 7 * ways < gridDim.x; i += 8 * ways) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) a8[u] += (double)__ldcg(stat_part + (size_t)(i + u * ways) * nval + v);
+        }
+        for (; i < gridDim.x; i += ways) a8[0] += (double)__ldcg(stat_part + (size_t)i * nval + v);
+        acc = ((a8[0] + a8[1]) + (a8[2] + a8[3])) + ((a8[4] + a8[5]) + (a8[6] + a8[7]));
+    }
+    fold[threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.x < C) {
+        const int c = threadIdx.x;
+        double a = 0.0, b = 0.0;
+        for (int wy = 0; wy < ways; ++wy) { a += fold[wy * nval + c]; b += fold[wy * nval + C + c]; }
+        if (bn_x == nullptr) {
+            const double npix = (double)n_tiles * kTileM;
+            double m = a / npix, var = b / npix - m * m;
+            if (var < 0.0) var = 0.0;
+            stat_o0[c] = (float)m;
+            stat_o1[c] = (float)(1.0 / sqrt(var + 1e-5));
+        } else {
+            stat_o0[c] = (float)a;
+            stat_o1[c] = (float)b;
+        }
+    }
+    if (threadIdx.x == 0) *stat_counter = 0u;
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -1121,7 +1164,7 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
     launch_k(conv3x3_tc_kernel<C>, grid, kTcThreads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
         stage_bytes, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
-        (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd);
+        bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd);
     return 1;
 }
 

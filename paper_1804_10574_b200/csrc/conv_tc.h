@@ -15,13 +15,16 @@ bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
 // w: filter in canonical [Cout][Cin][3][3] order.  w_packed (nullable): the pre-arranged filter images written by
 // launch_pack_filters for this convolution (tc_packed_bytes(C) bytes: forward image, then input-gradient image); when
 // given, the kernel fetches its filter with one bulk copy instead of re-arranging the canonical one itself.
-// bf.part != nullptr: the kernel also leaves, in bf.part[conv_tc_grid(B, H, W)][2C], per-CTA partial sums over its
-// output for the batch norm that consumes it: with bf.x == nullptr (sum y, sum y^2) per channel (forward statistics);
-// otherwise (sum dz, sum dz * xhat), dz = output * [bf.mask > 0], xhat = (bf.x - bf.mean) * bf.invstd (the two
-// reductions of the batch-norm backward whose incoming gradient is this kernel's output).  The partials are summed
-// in a fixed order by the batch-norm kernel that follows.
+// bf.part != nullptr: the kernel also reduces its output for the batch norm that consumes it.  Per-CTA partial sums
+// go to bf.part[conv_tc_grid(B, H, W)][2C]; the CTA that finishes last (ticket in *bf.counter, zero before and after)
+// adds them in a fixed order and stores the result.  With bf.x == nullptr the sums are (sum y, sum y^2) per channel and
+// the result is the forward statistics bf.o0 = mean, bf.o1 = 1/sqrt(var + 1e-5).  Otherwise they are (sum dz, sum dz *
+// xhat), dz = output * [bf.mask > 0], xhat = (bf.x - bf.mean) * bf.invstd: the two reductions of the batch-norm
+// backward whose incoming gradient is this kernel's output; bf.o0 = dbeta, bf.o1 = dgamma.
 struct BnFuse {
     float *part = nullptr;
+    unsigned *counter = nullptr;
+    float *o0 = nullptr, *o1 = nullptr;
     const void *mask = nullptr, *x = nullptr;
     const float *mean = nullptr, *invstd = nullptr;
 };

@@ -223,18 +223,15 @@ long forward_module(ddg_ctx *c, int k, long t) {
             // tensor-core kernel runs, from a reduction kernel otherwise
             auto conv_bn = [&](const void *xin, const void *wc, const void *wp, void *yc, int H, int W, int Cic, int strd,
                                const char *gm, const char *bt, float *mean, float *invstd, Shortcut scb, void *dstb) {
-                float *part = m.bn_scratch + 32;
                 if (bn_fuse_enabled() && c->prec == P_BF16 && conv_tc_supported(B, H, W, Cic, Co, strd)) {
                     BnFuse bf;
-                    bf.part = part;
+                    bf.part = m.bn_scratch + 32; bf.counter = (unsigned *)m.bn_scratch; bf.o0 = mean; bf.o1 = invstd;
                     n += launch_conv_tc(0, xin, wc, wp, yc, B, H, W, Cic, Shortcut{}, s, bf);
-                    n += launch_bn_apply_part(c->prec, yc, gm, bt, part, conv_tc_grid(B, H, W), mean, invstd, scb, dstb, B,
-                                              L.Hout, L.Wout, Co, 1, s);
                 } else {
                     n += conv_fwd(c, xin, wc, wp, yc, H, W, Cic, Co, strd, 0, s);
                     n += launch_bn_stats(c->prec, yc, mean, invstd, m.bn_scratch, npix, Co, s);
-                    n += launch_bn_apply(c->prec, yc, gm, bt, mean, invstd, scb, dstb, B, L.Hout, L.Wout, Co, 1, s);
                 }
+                n += launch_bn_apply(c->prec, yc, gm, bt, mean, invstd, scb, dstb, B, L.Hout, L.Wout, Co, 1, s);
             };
             conv_bn(in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, g1, b1, stt, stt + Co, Shortcut{}, a1);
             Shortcut sc{};
@@ -269,10 +266,11 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
     // The weight gradient of a convolution needs only (layer input, dy); nothing on the way down to the module input
     // waits for it.  It runs on the module's side stream; dy lives in a ring of four buffers so that the chain can move
     // on, and the chain only waits when it comes back to a buffer whose weight gradient has not finished.
-    // number of per-CTA partial sums that the kernel which produced `cur` left for the batch norm that consumes it
-    // (0: none, that batch norm runs its own reduction)
-    int cur_np = 0;
+    // true when the kernel that produced `cur` already left the two sums (dbeta, dgamma) of the batch norm that
+    // consumes it in that batch norm's gradient slots
+    bool cur_sums = false;
     float *bn_part = m.bn_scratch + 32;
+    unsigned *bn_counter = (unsigned *)m.bn_scratch;
     const bool fuse = bn_fuse_enabled() && c->prec == P_BF16;
     int dy_i = 0, last_side = -1;
     bool ring_used[4] = {false, false, false, false};
@@ -299,7 +297,8 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
         const bool mod_first = (l == m.first);
         const bool need_dx = !L.is_first;
         // destination of the error gradient w.r.t. the layer input
-        int dst_tmp = -1, next_np = 0;
+        int dst_tmp = -1;
+        bool next_sums = false;
         char *dst = nullptr;
         if (need_dx) {
             if (mod_first) dst = m.delta_out[t % 2];
@@ -353,29 +352,24 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
             (void)tA;
             const int j2 = ring_next();
             char *dy2 = m.dyring[j2], *da1 = m.tmp[tB];
-            if (cur_np > 0) {
-                n += launch_bn_bwd_apply_part(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, bn_part, cur_np, gg2, gb2,
-                                              dy2, npix, Co, 1, s);
-            } else {
+            if (!cur_sums)
                 n += launch_bn_bwd_reduce(c->prec, cur, out, y2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, m.bn_scratch, npix, Co,
                                           1, s);
-                n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s);
-            }
+            n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s);
             side_wgrad(j2, a1, dy2, gw2, L.Hout, L.Wout, Co, Co, 1);
             const int j1 = ring_next();
             char *dy1 = m.dyring[j1];
             if (fuse && conv_tc_supported(B, L.Hout, L.Wout, Co, Co, 1)) {
                 // the input gradient of conv2 is the incoming gradient of bn1: its two sums come out of the same kernel
                 BnFuse bf;
-                bf.part = bn_part; bf.mask = a1; bf.x = y1; bf.mean = stt; bf.invstd = stt + Co;
+                bf.part = bn_part; bf.counter = bn_counter; bf.o0 = gb1; bf.o1 = gg1;
+                bf.mask = a1; bf.x = y1; bf.mean = stt; bf.invstd = stt + Co;
                 n += launch_conv_tc(1, dy2, w2, pkp(L.pk2), da1, B, L.Hout, L.Wout, Co, Shortcut{}, s, bf);
-                n += launch_bn_bwd_apply_part(c->prec, da1, a1, y1, g1, stt, stt + Co, bn_part, conv_tc_grid(B, L.Hout, L.Wout),
-                                              gg1, gb1, dy1, npix, Co, 1, s);
             } else {
                 n += conv_dgrad(c, dy2, w2, pkp(L.pk2), da1, L.Hout, L.Wout, Co, Co, 1, Shortcut{}, s);
                 n += launch_bn_bwd_reduce(c->prec, da1, a1, y1, stt, stt + Co, gg1, gb1, m.bn_scratch, npix, Co, 1, s);
-                n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
             }
+            n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
             side_wgrad(j1, in, dy1, gw1, L.Hin, L.Win, Ci, Co, st);
             if (need_dx) {
                 Shortcut sc{};
@@ -388,11 +382,14 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
                     // dx is the incoming gradient of the block below, whose second batch norm reduces it first: take
                     // those sums here (its output is this block's input, its bn2 input and statistics are in its slots)
                     const float *pst = (const float *)slot_ptr(c, Pv->stats, sidx);
+                    // gradient slots of the block below: conv1, gamma1, beta1, conv2, gamma2, beta2
+                    float *pg2 = m.g + Pv->p_off + (size_t)Ci * Pv->Cin * 9 + 2 * (size_t)Ci + (size_t)Ci * Ci * 9;
                     BnFuse bf;
-                    bf.part = bn_part; bf.mask = in; bf.x = slot_ptr(c, Pv->y2, sidx);
+                    bf.part = bn_part; bf.counter = bn_counter; bf.o1 = pg2; bf.o0 = pg2 + Ci;
+                    bf.mask = in; bf.x = slot_ptr(c, Pv->y2, sidx);
                     bf.mean = pst + 2 * Ci; bf.invstd = pst + 3 * Ci;
                     n += launch_conv_tc(1, dy1, w1, pkp(L.pk1), dx, B, L.Hin, L.Win, Ci, sc, s, bf);
-                    next_np = conv_tc_grid(B, L.Hin, L.Win);
+                    next_sums = true;
                 } else {
                     n += conv_dgrad(c, dy1, w1, pkp(L.pk1), dx, L.Hin, L.Win, Ci, Co, st, sc, s);
                 }
@@ -403,7 +400,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
         }
         cur = dst;
         cur_tmp = dst_tmp;
-        cur_np = next_np;
+        cur_sums = next_sums;
     }
     side_join();  // the update that follows reads every gradient of the module
     return n;

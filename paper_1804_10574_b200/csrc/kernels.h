@@ -55,16 +55,6 @@ int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void 
                         const float *mean, const float *invstd, const float *dgamma, const float *dbeta, void *dx,
                         long npix, int C, int relu, cudaStream_t s);
 
-// The same two element-wise passes when the per-channel sums come as per-CTA partials part[n_part][2C] from the
-// convolution that produced x (forward: sum x, sum x^2) or dout (backward: sum dz, sum dz*xhat): the kernel adds the
-// partials itself and stores mean / invstd (dbeta / dgamma).  -1: shape not taken (nothing was launched).
-int launch_bn_apply_part(int prec, const void *x, const void *gamma, const void *beta, const float *part, int n_part,
-                         float *mean, float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu,
-                         cudaStream_t s);
-int launch_bn_bwd_apply_part(int prec, const void *dout, const void *out, const void *x, const void *gamma,
-                             const float *mean, const float *invstd, const float *part, int n_part, float *dgamma,
-                             float *dbeta, void *dx, long npix, int C, int relu, cudaStream_t s);
-
 // ---- 3x3 convolution, CUDA-core kernels (any shape; used for fp32 and for shapes the tensor-core path skips) --
 int launch_conv_fwd_direct(int prec, const void *x, const void *w, void *y, int B, int H, int W, int Cin, int Cout,
                            int stride, int relu, cudaStream_t s);

@@ -627,166 +627,6 @@ int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void 
 }
 
 // ------------------------------------------------------------------------------------------------------
-// Batch-norm kernels whose per-channel sums arrive as per-CTA partials part[n_part][2C] left by the convolution that
-// produced their input: every CTA first adds the partials in a fixed order (all CTAs get the same bits), CTA 0 stores
-// the result where the two-kernel path would have (mean / invstd, or dbeta / dgamma), then the element-wise pass runs.
-// ------------------------------------------------------------------------------------------------------
-// tot[0..2C) = sum over partials, in double
-__device__ __forceinline__ void fold_part(const float *__restrict__ part, int n_part, int C, double *fold, double *tot) {
-    const int nval = 2 * C, ways = kThreads / nval;
-    const int v = threadIdx.x % nval, way = threadIdx.x / nval;
-    double acc = 0.0;
-    if (way < ways) {
-        double a4[4] = {0.0, 0.0, 0.0, 0.0};
-        int i = way;
-        for (; i + 3 * ways < n_part; i += 4 * ways) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) a4[u] += (double)__ldcg(part + (size_t)(i + u * ways) * nval + v);
-        }
-        for (; i < n_part; i += ways) a4[0] += (double)__ldcg(part + (size_t)i * nval + v);
-        acc = (a4[0] + a4[1]) + (a4[2] + a4[3]);
-    }
-    fold[threadIdx.x] = acc;
-    __syncthreads();
-    if (threadIdx.x < nval) {
-        double t = 0.0;
-        for (int w = 0; w < ways; ++w) t += fold[w * nval + threadIdx.x];
-        tot[threadIdx.x] = t;
-    }
-    __syncthreads();
-}
-
-template <typename T, int VEC>
-__global__ void __launch_bounds__(kThreads)
-bn_apply_part_kernel(const T *__restrict__ x, const T *__restrict__ gamma, const T *__restrict__ beta,
-                     const float *__restrict__ part, int n_part, float *__restrict__ mean_out,
-                     float *__restrict__ invstd_out, Shortcut sc, T *__restrict__ y, long nvec, long npix, int H, int W, int C,
-                     int relu) {
-    pdl_launch();
-    pdl_wait();
-    typedef typename AccOf<T>::type A;
-    __shared__ double fold[kThreads], tot[2 * 128];
-    __shared__ float s_mean[128], s_is[128];
-    fold_part(part, n_part, C, fold, tot);
-    if (threadIdx.x < C) {
-        const int c = threadIdx.x;
-        double m = tot[c] / (double)npix, var = tot[C + c] / (double)npix - m * m;
-        if (var < 0.0) var = 0.0;
-        s_mean[c] = (float)m;
-        s_is[c] = (float)(1.0 / sqrt(var + (double)kBnEps));
-        if (blockIdx.x == 0) { mean_out[c] = s_mean[c]; invstd_out[c] = s_is[c]; }
-    }
-    __syncthreads();
-    long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= nvec) return;
-    const int groups = C / VEC;
-    const int c0 = (int)(i % groups) * VEC;
-    const long p = i / groups;
-    A v[VEC];
-    load_a<T, A, VEC>(x + p * C + c0, v);
-#pragma unroll
-    for (int j = 0; j < VEC; ++j)
-        v[j] = (A)to_f(gamma[c0 + j]) * (v[j] - (A)s_mean[c0 + j]) * (A)s_is[c0 + j] + (A)to_f(beta[c0 + j]);
-    if (sc.mode == 1) {
-        A r[VEC];
-        load_a<T, A, VEC>((const T *)sc.a + p * C + c0, r);
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) v[j] += r[j];
-    } else if (sc.mode == 2) {
-        if (c0 < sc.c_small) {
-            const int wo = (int)(p % W), ho = (int)((p / W) % H);
-            const long n = p / ((long)W * H);
-            const long q = (n * sc.h_big + 2 * ho) * sc.w_big + 2 * wo;
-            A r[VEC];
-            load_a<T, A, VEC>((const T *)sc.a + q * sc.c_small + c0, r);
-#pragma unroll
-            for (int j = 0; j < VEC; ++j) if (c0 + j < sc.c_small) v[j] += r[j];
-        }
-    }
-    if (relu) {
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) v[j] = v[j] > 0 ? v[j] : (A)0;
-    }
-    store_a<T, A, VEC>(y + p * C + c0, v);
-}
-
-int launch_bn_apply_part(int prec, const void *x, const void *gamma, const void *beta, const float *part, int n_part,
-                         float *mean, float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu,
-                         cudaStream_t s) {
-    const long npix = (long)B * H * W;
-    int rc = -1;
-    DISPATCH_PREC(prec, {
-        constexpr int V = Vec16<T>::N;
-        if (C % V == 0 && C <= 128 && (sc.mode != 2 || sc.c_small % V == 0)) {
-            long nvec = npix * (C / V);
-            launch_k(bn_apply_part_kernel<T, V>, ceil_div(nvec, kThreads), kThreads, 0, s, (const T *)x, (const T *)gamma,
-                     (const T *)beta, part, n_part, mean, invstd, sc, (T *)y, nvec, npix, H, W, C, relu);
-            rc = 1;
-        }
-    });
-    return rc;
-}
-
-template <typename T, int VEC>
-__global__ void __launch_bounds__(kThreads)
-bn_bwd_apply_part_kernel(const T *__restrict__ dout, const T *__restrict__ out, const T *__restrict__ x,
-                         const T *__restrict__ gamma, const float *__restrict__ mean, const float *__restrict__ invstd,
-                         const float *__restrict__ part, int n_part, float *__restrict__ dgamma, float *__restrict__ dbeta,
-                         T *__restrict__ dx, long nvec, long npix, int C, int relu) {
-    pdl_launch();
-    pdl_wait();
-    typedef typename AccOf<T>::type A;
-    __shared__ double fold[kThreads], tot[2 * 128];
-    __shared__ float s_db[128], s_dg[128];
-    fold_part(part, n_part, C, fold, tot);
-    if (threadIdx.x < C) {
-        const int c = threadIdx.x;
-        s_db[c] = (float)tot[c];
-        s_dg[c] = (float)tot[C + c];
-        if (blockIdx.x == 0) { dbeta[c] = s_db[c]; dgamma[c] = s_dg[c]; }
-    }
-    __syncthreads();
-    long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= nvec) return;
-    const int groups = C / VEC;
-    const int c0 = (int)(i % groups) * VEC;
-    const long p = i / groups;
-    A xv[VEC], dv[VEC];
-    load_a<T, A, VEC>(x + p * C + c0, xv);
-    load_a<T, A, VEC>(dout + p * C + c0, dv);
-    if (relu) {
-        float ov[VEC];
-        load_f<T, VEC>(out + p * C + c0, ov);
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) if (!(ov[j] > 0.f)) dv[j] = 0;
-    }
-    const A cnt = (A)npix;
-#pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-        const int c = c0 + j;
-        const A xh = (xv[j] - (A)mean[c]) * (A)invstd[c];
-        dv[j] = (A)to_f(gamma[c]) * (A)invstd[c] * (dv[j] - (A)s_db[c] / cnt - xh * (A)s_dg[c] / cnt);
-    }
-    store_a<T, A, VEC>(dx + p * C + c0, dv);
-}
-
-int launch_bn_bwd_apply_part(int prec, const void *dout, const void *out, const void *x, const void *gamma,
-                             const float *mean, const float *invstd, const float *part, int n_part, float *dgamma,
-                             float *dbeta, void *dx, long npix, int C, int relu, cudaStream_t s) {
-    int rc = -1;
-    DISPATCH_PREC(prec, {
-        constexpr int V = Vec16<T>::N;
-        if (C % V == 0 && C <= 128) {
-            long nvec = npix * (C / V);
-            launch_k(bn_bwd_apply_part_kernel<T, V>, ceil_div(nvec, kThreads), kThreads, 0, s, (const T *)dout, (const T *)out,
-                     (const T *)x, (const T *)gamma, mean, invstd, part, n_part, dgamma, dbeta, (T *)dx, nvec, npix, C, relu);
-            rc = 1;
-        }
-    });
-    return rc;
-}
-
-// ------------------------------------------------------------------------------------------------------
 // optimiser update with the delayed gradient (Eq. 9 / Algorithm 1, Algorithm 2) + weight-version refresh
 // ------------------------------------------------------------------------------------------------------
 template <typename T>

@@ -62,14 +62,14 @@ def cases(B):
         tag = "%d->%d %dx%d s%d" % (Ci, Co, H, H, st)
         tc = binding.tensor_core_path(B, H, H, Ci, Co, st)
         keep = (x, dy, w, y, dx, dw, sc)
-        if tc & 1:   # as in the training step: filter image arranged beforehand (by the optimiser update)
+        if tc & 1 and st == 1 and Ci == Co:   # as in the training step: filter image arranged beforehand (by the optimiser update)
             pk = torch.empty(binding.conv3x3_packed_bytes(B, H, H, Ci), dtype=torch.uint8, device="cuda")
             binding.conv3x3_pack(w, pk, Ci)
             out.append(("conv_fwd " + tag, lambda: binding.conv3x3_packed(0, x, w, pk, y, B, H, H, Ci), io, flops, 1, keep + (pk,)))
             out.append(("conv_dgrad " + tag, lambda: binding.conv3x3_packed(1, dy, w, pk, dx, B, H, H, Ci), io, flops, 1, keep + (pk,)))
         else:
-            out.append(("conv_fwd " + tag, lambda: binding.conv3x3_fwd(1, x, w, y, B, H, H, Ci, Co, st), io, flops, 0, keep))
-            out.append(("conv_dgrad " + tag, lambda: binding.conv3x3_dgrad(1, dy, w, dx, B, H, H, Ci, Co, st), io, flops, 0, keep))
+            out.append(("conv_fwd " + tag, lambda: binding.conv3x3_fwd(1, x, w, y, B, H, H, Ci, Co, st), io, flops, tc & 1, keep))
+            out.append(("conv_dgrad " + tag, lambda: binding.conv3x3_dgrad(1, dy, w, dx, B, H, H, Ci, Co, st), io, flops, tc & 1, keep))
         out.append(("conv_wgrad " + tag, lambda: binding.conv3x3_wgrad(1, x, dy, dw, sc, B, H, H, Ci, Co, st), io, flops, (tc >> 1) & 1, keep))
 
     for H, Ci, Co, st in ((32, 16, 16, 1), (16, 32, 32, 1), (8, 64, 64, 1), (32, 16, 32, 2), (16, 32, 64, 2), (32, 3, 16, 1)):
