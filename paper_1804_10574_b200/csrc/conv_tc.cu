@@ -12,9 +12,13 @@
 // neighbouring pixels, y[h][w] = P_0[h][w-1] + P_1[h][w] + P_2[h][w+1], with warp shuffles (a warp holds whole image
 // rows; the image border contributes zero).  The filter-row shift costs nothing: the three rows read the same TMA box
 // at offsets of 0, W and 2W pixels, which are whole swizzle periods, so only the descriptor start address moves.
-// Warp roles: warp 0 issues TMA, warp 1 issues MMAs, warps 2-9 (two groups, one per accumulator stage) drain TMEM,
-// combine, add the shortcut gradient where asked, convert to bf16 and store.  Two TMEM accumulator stages let the epilogue of tile i overlap the MMAs of tile
-// i+1.  Every mbarrier wait is bounded: when one runs out, the CTA raises an error word that the host reads at its
+// Warp roles: warp 0 issues TMA, warp 1 issues MMAs, warps 2-5 and 6-9 (two groups, one per TMEM accumulator, each
+// taking every other tile) drain TMEM, combine, add the shortcut gradient where asked, convert to bf16 and store, so
+// that the epilogue of tile i overlaps the MMAs of tile i+1.  With `dual` (many small tiles per CTA: C = 16) the CTA
+// runs TWO independent pipelines over alternate tiles instead, warps 10 / 11 being the second TMA / MMA issuer, each
+// pipeline with half of the stage ring, one accumulator and one epilogue group: there the cost of a tile is the chain
+// of barrier hand-offs and instruction issue of the single MMA thread (about a thousand cycles), not data movement
+// or tensor-core time, and two chains side by side raise the tile rate of an SM.  Every mbarrier wait is bounded: when one runs out, the CTA raises an error word that the host reads at its
 // next sync point, and leaves.
 #include <cuda.h>
 #include <cudaTypedefs.h>
@@ -31,7 +35,8 @@ namespace ddg {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kTcThreads = 320;   // convolution: TMA warp, MMA warp, two groups of four epilogue warps
+constexpr int kTcThreads = 384;   // convolution: two pipelines, each a TMA warp, an MMA warp and four epilogue warps
+constexpr int kS2Threads = 320;   // stride-2 convolution: TMA warp, MMA warp, two groups of four epilogue warps
 constexpr int kWgThreads = 192;   // weight gradient: TMA warp, MMA warp, four epilogue warps
 constexpr unsigned kSpinLimit = 1u << 24;  // bounded waits: ~ a second at worst, then the CTA gives up
 
@@ -261,7 +266,7 @@ template <int C>
 __global__ void __launch_bounds__(kTcThreads, 1)
 conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
                   bf16 *__restrict__ dst, int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
-                  int slab, int n_stages, int stage_bytes, const bf16 *__restrict__ res_dout,
+                  int slab, int n_stages, int stage_bytes, int dual, const bf16 *__restrict__ res_dout,
                   const bf16 *__restrict__ res_out, float *__restrict__ stat_part, unsigned *__restrict__ stat_counter,
                   float *__restrict__ stat_o0, float *__restrict__ stat_o1, const bf16 *__restrict__ bn_mask,
                   const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd) {
@@ -294,7 +299,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (stat_part != nullptr)
-        for (int i = threadIdx.x; i < 8 * 4 * 32; i += kTcThreads) (&sm_run[0][0][0])[i] = 0.f;
+        for (int i = threadIdx.x; i < 8 * 4 * 32; i += blockDim.x) (&sm_run[0][0][0])[i] = 0.f;
     if (threadIdx.x == 0) {
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < Cfg::acc_stages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
@@ -316,7 +321,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
         sm_stat[threadIdx.x] = threadIdx.x < C ? bn_mean[threadIdx.x] : bn_invstd[threadIdx.x - C];
     if (w_packed == nullptr) {
         // filter in canonical order: stage it here as 9 K-major [C rows = output channel of this pass][C] tiles
-        for (int i = threadIdx.x; i < 9 * C * C; i += kTcThreads) {
+        for (int i = threadIdx.x; i < 9 * C * C; i += blockDim.x) {
             const int tap = i / (C * C), r = (i / C) % C, k = i % C;
             const size_t g = dgrad ? ((size_t)(k * C + r) * 9 + (8 - tap)) : ((size_t)(r * C + k) * 9 + tap);
             *reinterpret_cast<bf16 *>(smem + plan.w_off + w_img_off<C>(tap, r, k)) = w[g];
@@ -330,49 +335,57 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     const int tiles_per_img = H / rows_per_tile;  // tiles per image when a tile lies inside one image
     const int loads_per_tile = slab ? 1 : 3;
 
-    if (warp == 0) {
-        // ---------------- TMA producer ----------------
-        if (lane == 0) {
-            if (w_packed != nullptr) {  // pre-arranged filter image: one bulk copy
+    // pipeline g (0, or 0 and 1 with `dual`) owns stages [g*ring, (g+1)*ring) and takes every tile_step-th tile
+    const int ring = dual ? n_stages >> 1 : n_stages;
+    const int tile_step = dual ? 2 * gridDim.x : gridDim.x;
+    if (warp == 0 || warp == 10) {
+        // ---------------- TMA producers ----------------
+        const int g = warp == 0 ? 0 : 1;
+        if (lane == 0 && (g == 0 || dual)) {
+            if (g == 0 && w_packed != nullptr) {  // pre-arranged filter image: one bulk copy
                 mbar_expect_tx(w_bar, Cfg::w_bytes);
                 bulk_copy_g2s(w_base, w_packed + (dgrad ? Cfg::w_bytes : 0), Cfg::w_bytes, w_bar);
             }
-            int s = 0;
+            int ls = 0;
             uint32_t ph = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            for (int tile = blockIdx.x + g * gridDim.x; tile < n_tiles && ok; tile += tile_step) {
                 int n0, h0;
                 if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }  // a tile spans whole images
                 else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
                 for (int j = 0; j < loads_per_tile && ok; ++j) {
+                    const int s = g * ring + ls;
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 1);
                     if (!ok) break;
                     mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
                     tma_load_4d(a_base + s * stage_bytes, &tmap, full_bar(s), 0, 0, slab ? h0 - 1 : h0 + j - 1, n0);
-                    if (++s == n_stages) { s = 0; ph ^= 1u; }
+                    if (++ls == ring) { ls = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {  // let copies already in flight land before the CTA can exit
                 for (int i = 0; i < 2000; ++i) __nanosleep(100);
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+    } else if (warp == 1 || warp == 11) {
+        // ---------------- MMA issuers ----------------
+        const int g = warp == 1 ? 0 : 1;
+        if (lane == 0 && (g == 0 || dual)) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((3 * C) >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-            int s = 0;
+            int ls = 0, it = 0;
             uint32_t ph = 0;
-            int it = 0;
             bool ok = true;
             if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, abort_flag, 5);
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-                const int a = it % Cfg::acc_stages;
-                const uint32_t aph = (it / Cfg::acc_stages) & 1u;
+            for (int tile = blockIdx.x + g * gridDim.x; tile < n_tiles && ok; tile += tile_step, ++it) {
+                // accumulator: the pipeline's own one (dual), else the two in turn; the epilogue group of the same number
+                // drains it
+                const int a = dual ? g : (it & 1);
+                const uint32_t aph = dual ? (it & 1) : ((it >> 1) & 1);
                 ok = mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, 2);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * 3 * C);
                 for (int j = 0; j < loads_per_tile && ok; ++j) {
+                    const int s = g * ring + ls;
                     ok = mbar_wait(full_bar(s), ph, abort_flag, 3);
                     if (!ok) break;
                     tc_fence_after();
@@ -387,7 +400,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                             tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (ky | k) != 0);
                     }
                     tc_commit(empty_bar(s));  // the stage is free once these MMAs have read it
-                    if (++s == n_stages) { s = 0; ph ^= 1u; }
+                    if (++ls == ring) { ls = 0; ph ^= 1u; }
                 }
                 if (ok) tc_commit(tfull_bar(a));
             }
@@ -397,11 +410,10 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
         // Two groups of four warps; group g drains every other tile, so two epilogues overlap.
         const int q = warp & 3;  // a warp may only touch TMEM lanes [32*(warp%4), +32)
         const int grp = (warp - 2) >> 2;
-        int it = grp;
+        const int a = grp;
+        uint32_t aph = 0;
         bool ok = true;
-        for (int tile = blockIdx.x + grp * gridDim.x; tile < n_tiles && ok; tile += 2 * gridDim.x, it += 2) {
-            const int a = it % Cfg::acc_stages;
-            const uint32_t aph = (it / Cfg::acc_stages) & 1u;
+        for (int tile = blockIdx.x + grp * gridDim.x; tile < n_tiles && ok; tile += 2 * gridDim.x, aph ^= 1u) {
             ok = mbar_wait(tfull_bar(a), aph, abort_flag, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -499,7 +511,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     __threadfence();
     // last CTA: partials of all CTAs, `ways` threads per value, eight loads in flight per thread, fixed order
     double *fold = reinterpret_cast<double *>(&sm_run[0][0][0]);  // kTcThreads doubles fit the 4 KB
-    constexpr int nval = 2 * C, ways = kTcThreads / nval;
+    constexpr int nval = 2 * C;
+    const int ways = (int)blockDim.x / nval;
     const int v = threadIdx.x % nval, way = threadIdx.x / nval;
     double acc = 0.0;
     if (way < ways) {
@@ -716,7 +729,7 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map
 // NC = Co), MODE 1 input gradient (KC = Co, NC = Ci).  Hs x Ws is the SMALL (output-resolution) map; rows_per_tile /
 // imgs_per_tile describe a 128-pixel tile of it.  n_sp = number of such tiles.
 template <int KC, int NC, int MODE>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kS2Threads, 1)
 conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
                      bf16 *__restrict__ dst, int Hs, int Ws, int rows_per_tile, int imgs_per_tile, int n_sp, int n_stages,
                      const bf16 *__restrict__ res_dout, const bf16 *__restrict__ res_out) {
@@ -761,7 +774,7 @@ conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__res
     pdl_wait();  // nothing above touches global memory
     if (w_packed == nullptr) {  // canonical filter [Co][Ci][3][3]: arrange the nine tiles of this pass here
         constexpr int CO = 2 * CI;
-        for (int i = threadIdx.x; i < 9 * CO * CI; i += kTcThreads) {
+        for (int i = threadIdx.x; i < 9 * CO * CI; i += kS2Threads) {
             const int tap = i / (CO * CI), co = (i / CI) % CO, ci = i % CI;
             const uint32_t o = (uint32_t)tap * tap_bytes + (MODE == 0 ? swz_off<KC>(co, ci) : swz_off<KC>(ci, co));
             *reinterpret_cast<bf16 *>(smem + o) = w[(size_t)(co * CI + ci) * 9 + tap];
@@ -1162,8 +1175,11 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     if (n_stages < 3) n_stages = 3;
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
-    launch_k(conv3x3_tc_kernel<C>, grid, kTcThreads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
-        stage_bytes, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
+    // two pipelines per CTA where a CTA has many small tiles (each pipeline then owns half of an even stage ring)
+    const int dual = (C == 16 && slab && n_tiles >= 4 * grid) ? 1 : 0;
+    if (dual) n_stages &= ~1;
+    launch_k(conv3x3_tc_kernel<C>, grid, dual ? kTcThreads : kS2Threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
+        stage_bytes, dual, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
         bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd);
     return 1;
 }
@@ -1211,7 +1227,7 @@ int launch_tc_s2(int dir, const void *src, const void *w, const void *w_packed, 
         int n_stages = kSmemBudget / TcCfg<CI>::tile_bytes;
         if (n_stages > kMaxStages) n_stages = kMaxStages;
         const int grid = n_sp < g_num_sms ? n_sp : g_num_sms;
-        launch_k(conv3x3_s2_tc_kernel<CI, CO, 0>, grid, kTcThreads, s2_smem_bytes<CI, CO, 0>(n_stages), s, map, (const bf16 *)w, pk,
+        launch_k(conv3x3_s2_tc_kernel<CI, CO, 0>, grid, kS2Threads, s2_smem_bytes<CI, CO, 0>(n_stages), s, map, (const bf16 *)w, pk,
                  (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages, (const bf16 *)nullptr, (const bf16 *)nullptr);
     } else {
         if (!get_map(src, B, Hs, Ws, CO, rows, imgs, &map)) return -1;
@@ -1220,7 +1236,7 @@ int launch_tc_s2(int dir, const void *src, const void *w, const void *w_packed, 
         if (n_stages < 3) n_stages = 3;
         const int n_tiles = 4 * n_sp;
         const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
-        launch_k(conv3x3_s2_tc_kernel<CO, CI, 1>, grid, kTcThreads, s2_smem_bytes<CO, CI, 1>(n_stages), s, map, (const bf16 *)w,
+        launch_k(conv3x3_s2_tc_kernel<CO, CI, 1>, grid, kS2Threads, s2_smem_bytes<CO, CI, 1>(n_stages), s, map, (const bf16 *)w,
                  pk ? pk + S2Cfg<CI>::img_bytes : pk, (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages,
                  sc.mode == 2 ? (const bf16 *)sc.a : nullptr, sc.mode == 2 ? (const bf16 *)sc.b : nullptr);
     }
