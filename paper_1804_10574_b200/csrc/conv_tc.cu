@@ -266,7 +266,7 @@ template <int C>
 __global__ void __launch_bounds__(kTcThreads, 1)
 conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
                   bf16 *__restrict__ dst, int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
-                  int slab, int n_stages, int stage_bytes, int dual, const bf16 *__restrict__ res_dout,
+                  int slab, int n_stages, int stage_bytes, int dual, int tmem_cols, const bf16 *__restrict__ res_dout,
                   const bf16 *__restrict__ res_out, float *__restrict__ stat_part, unsigned *__restrict__ stat_counter,
                   float *__restrict__ stat_o0, float *__restrict__ stat_o1, const bf16 *__restrict__ bn_mask,
                   const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd) {
@@ -301,6 +301,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     if (stat_part != nullptr)
         for (int i = threadIdx.x; i < 8 * 4 * 32; i += blockDim.x) (&sm_run[0][0][0])[i] = 0.f;
     if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");  // the first TMA would otherwise wait for its descriptor
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < Cfg::acc_stages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
         mbar_init(w_bar, 1);
@@ -309,7 +310,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     }
     if (warp == 1) {  // TMEM allocation is a whole-warp operation; the same warp frees it at the end
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
-                     "r"((uint32_t)Cfg::tmem_cols)
+                     "r"((uint32_t)tmem_cols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -491,7 +492,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::tmem_cols)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
                      : "memory");
     }
     if (stat_part == nullptr) return;
@@ -1178,8 +1179,10 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     // two pipelines per CTA where a CTA has many small tiles (each pipeline then owns half of an even stage ring)
     const int dual = (C == 16 && slab && n_tiles >= 4 * grid) ? 1 : 0;
     if (dual) n_stages &= ~1;
+    // a CTA with a single tile uses one accumulator: half the TMEM columns, so that CTAs of other streams fit beside it
+    const int tmem_cols = n_tiles <= grid ? TcCfg<C>::tmem_cols / 2 : TcCfg<C>::tmem_cols;
     launch_k(conv3x3_tc_kernel<C>, grid, dual ? kTcThreads : kS2Threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
-        stage_bytes, dual, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
+        stage_bytes, dual, tmem_cols, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
         bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd);
     return 1;
 }
