@@ -568,9 +568,10 @@ template <int C>
 __global__ void __launch_bounds__(kWgThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 float *__restrict__ part, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles, int slab,
-                int n_stages, int x_box_bytes, int tmem_cols) {
+                int n_stages, int x_box_bytes, int tmem_cols, int wide) {
     typedef TcCfg<C> Cfg;
     const int stage_bytes = Cfg::tile_bytes + 3 * x_box_bytes;
+    const int box_rows = rows_per_tile + 2;  // image rows of a column box in slab mode
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -632,6 +633,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             // both operands MN-major (bits 15, 16); fp32 accumulate; bf16 inputs; M = 128, N = 3C
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
                                    ((uint32_t)((3 * C) >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            const uint32_t idesc_wide = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+                                        ((uint32_t)(((2 * box_rows + 3) * C) >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -640,7 +643,18 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t st = base + s * stage_bytes;
-                if (slab) {
+                if (slab && wide) {
+                    // one instruction per 16 pixels: N runs over the three column boxes in one go (they are contiguous
+                    // and each is box_rows image rows of W pixels), block b = kx*box_rows + ky; only ky < 3 is read back
+#pragma unroll
+                    for (int k = 0; k < kTileM / 16; ++k) {
+                        const uint32_t koff = (uint32_t)k * 16 * Cfg::row_bytes;
+                        const uint64_t adesc = make_desc(st + koff, 8 * Cfg::row_bytes, Cfg::layout, 2 * C * C);
+                        const uint64_t bdesc = make_desc(st + Cfg::tile_bytes + koff, 8 * Cfg::row_bytes, Cfg::layout,
+                                                         (uint32_t)W * Cfg::row_bytes);
+                        tc_mma_bf16(tmem_base, adesc, bdesc, idesc_wide, (tile != t0) || (k != 0));
+                    }
+                } else if (slab) {
                     for (int kx = 0; kx < 3; ++kx) {
 #pragma unroll
                         for (int k = 0; k < kTileM / 16; ++k) {
@@ -681,7 +695,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 #pragma unroll 1
             for (int c0 = 0; c0 < ncols; c0 += 16) {
                 float v[16];
-                tc_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, v);
+                // accumulator column of these 16 input channels: tap group g = c0 / C; in the wide layout group (kx, ky)
+                // sits at block kx*box_rows + ky
+                const int gq = c0 / C;
+                const int col = wide ? ((gq / 3) * box_rows + gq % 3) * C + c0 % C : c0;
+                tc_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col, v);
                 tc_wait_ld();
                 if (co < C) {
                     // column c0..c0+15 = 16 input channels of one tap
@@ -1199,12 +1217,15 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     int n_stages = kSmemBudget / stage_bytes;
     if (n_stages > kMaxStages) n_stages = kMaxStages;
     if (n_stages < 2) n_stages = 2;
-    const int ncols = slab ? 9 * C : 3 * C;
+    // slab mode with narrow channels: all nine taps from one instruction per 16 pixels when the three column boxes
+    // (contiguous, box_rows blocks of C columns each) fit one N <= 256
+    const int wide = (slab && (2 * (rows + 2) + 3) * C <= 256) ? 1 : 0;
+    const int ncols = wide ? (2 * (rows + 2) + 3) * C : (slab ? 9 * C : 3 * C);
     const int tmem_cols = ncols <= 64 ? 64 : (ncols <= 128 ? 128 : (ncols <= 256 ? 256 : 512));
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int max_chunks = slab ? (C == 16 ? 74 : 37) : 24;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
-    launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols);
+    launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols, wide);
     launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C, C, cin);
     return 2;
 }
