@@ -568,7 +568,7 @@ template <int C>
 __global__ void __launch_bounds__(kWgThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 float *__restrict__ part, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles, int slab,
-                int n_stages, int x_box_bytes, int tmem_cols, int wide) {
+                int n_stages, int x_box_bytes, int tmem_cols, int wide, int tall) {
     typedef TcCfg<C> Cfg;
     const int stage_bytes = Cfg::tile_bytes + 3 * x_box_bytes;
     const int box_rows = rows_per_tile + 2;  // image rows of a column box in slab mode
@@ -635,6 +635,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                                    ((uint32_t)((3 * C) >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
             const uint32_t idesc_wide = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
                                         ((uint32_t)(((2 * box_rows + 3) * C) >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            const uint32_t idesc_tall = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+                                        ((uint32_t)(C >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -653,6 +655,19 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                         const uint64_t bdesc = make_desc(st + Cfg::tile_bytes + koff, 8 * Cfg::row_bytes, Cfg::layout,
                                                          (uint32_t)W * Cfg::row_bytes);
                         tc_mma_bf16(tmem_base, adesc, bdesc, idesc_wide, (tile != t0) || (k != 0));
+                    }
+                } else if (slab && tall) {
+                    // operands swapped: M runs over (filter row, input channel) = the rows of column box kx, N over the
+                    // C output channels; 3 instructions per 16 pixels, C accumulator columns each
+                    for (int kx = 0; kx < 3; ++kx) {
+#pragma unroll
+                        for (int k = 0; k < kTileM / 16; ++k) {
+                            const uint32_t koff = (uint32_t)k * 16 * Cfg::row_bytes;
+                            const uint64_t adesc = make_desc(st + Cfg::tile_bytes + kx * x_box_bytes + koff, 8 * Cfg::row_bytes,
+                                                             Cfg::layout, (uint32_t)W * Cfg::row_bytes);
+                            const uint64_t bdesc = make_desc(st + koff, 8 * Cfg::row_bytes, Cfg::layout, 2 * C * C);
+                            tc_mma_bf16(tmem_base + (uint32_t)(kx * C), adesc, bdesc, idesc_tall, (tile != t0) || (k != 0));
+                        }
                     }
                 } else if (slab) {
                     for (int kx = 0; kx < 3; ++kx) {
@@ -687,7 +702,24 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         const int q = warp & 3;
         bool ok = mbar_wait(done_bar, 0, abort_flag, 13);
         ok = __all_sync(0xffffffffu, ok);
-        if (ok && 32 * q < C) {  // only accumulator rows < C carry the result
+        if (ok && tall) {
+            // accumulator row = ky*C + ci (rows >= 3C unused), column = kx*C + co: each thread writes runs of output channels
+            tc_fence_after();
+            const int r = 32 * q + lane, ky = r / C, ci = r % C;
+            float *out = part + (size_t)blockIdx.x * 9 * C * C;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 3 * C; c0 += 16) {
+                float v[16];
+                tc_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, v);
+                tc_wait_ld();
+                if (ky < 3) {
+                    const int kx = c0 / C, co0 = c0 % C;
+                    float4 *o4 = reinterpret_cast<float4 *>(out + ((size_t)(ky * 3 + kx) * C + ci) * C + co0);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) o4[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                }
+            }
+        } else if (ok && 32 * q < C) {  // only accumulator rows < C carry the result
             tc_fence_after();
             const int co = 32 * q + lane;
             float *out = part + (size_t)blockIdx.x * 9 * C * C;
@@ -1220,12 +1252,16 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     // slab mode with narrow channels: all nine taps from one instruction per 16 pixels when the three column boxes
     // (contiguous, box_rows blocks of C columns each) fit one N <= 256
     const int wide = (slab && (2 * (rows + 2) + 3) * C <= 256) ? 1 : 0;
-    const int ncols = wide ? (2 * (rows + 2) + 3) * C : (slab ? 9 * C : 3 * C);
+    // otherwise, where 128 accumulator rows hold three filter rows (C = 32), the operands are swapped: 3C columns
+    // instead of 9C, so that the kernel takes a quarter of the TMEM and leaves room for other streams' CTAs
+    const int tall = (slab && !wide && 3 * C <= kTileM) ? 1 : 0;
+    const int ncols = wide ? (2 * (rows + 2) + 3) * C : ((slab && !tall) ? 9 * C : 3 * C);
     const int tmem_cols = ncols <= 64 ? 64 : (ncols <= 128 ? 128 : (ncols <= 256 ? 256 : 512));
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int max_chunks = slab ? (C == 16 ? 74 : 37) : 24;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
-    launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols, wide);
+    // tall: the unused accumulator rows (filter rows >= 3) read up to 128 - 3C pixel rows past the last column box
+    launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512 + (tall ? 4096 : 0), s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols, wide, tall);
     launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C, C, cin);
     return 2;
 }
