@@ -113,59 +113,81 @@ def time_oracle(cfg, batch, n_steps):
                       "untimed pipeline-fill iterations" % (n_steps, batch, cfg["batch"]), "seconds": dt}
 
 
-def _time_kernel(torch, fn, stream, flush, iters=20):
-    for _ in range(3):
+def _time_back_to_back(torch, launches, stream, reps=5):
+    """Average duration of one launch when `launches` (callables on distinct buffers, together larger than L2) run
+    back to back on `stream`, as the kernels of a training step do: CUDA events around the whole sequence."""
+    for fn in launches[:3]:
         fn()
+    torch.cuda.synchronize()
     ts = []
-    for _ in range(iters):
-        flush.zero_()                                  # evict the operands from L2 between timed launches
+    for _ in range(reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        fn()
+        for fn in launches:
+            fn()
         e1.record(stream)
         e1.synchronize()
-        ts.append(e0.elapsed_time(e1) * 1e-3)
-    return float(np.mean(ts))
+        ts.append(e0.elapsed_time(e1) * 1e-3 / len(launches))
+    return float(np.median(ts))
 
 
 def dominant_kernel_roofline(torch, binding, cfg, peaks):
-    """The kernel with the largest share of the ncu launch list of this workload is the batch-norm backward reduction
-    (profiles/ddg_step_resnet110_k4_b128_bf16_launch_list.md).  It is timed alone here, at the workload's largest
-    feature map and in the launch configuration the step uses, with CUDA events on its stream; the tensor-core
-    convolution kernels are timed the same way and listed beside it."""
-    B, H, C = cfg["batch"], 32, 16
+    """The kernel with the largest share of the ncu launch list of this workload is the tensor-core convolution on the
+    16-channel 32x32 maps, conv3x3_tc_kernel<16> (profiles/ddg_step_resnet110_k4_b128_bf16_launch_list.md).  It is
+    timed here at the step's shape and launch configuration, with its pre-arranged filter image, as a sequence of
+    launches on distinct tensors (more than L2 in total) between two CUDA events on its stream.  The other
+    convolution widths and the batch-norm backward pass are timed the same way and listed beside it."""
+    B = cfg["batch"]
     bf = torch.bfloat16
     s = torch.cuda.current_stream()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     hbm = peaks.get("hbm_gbs", 6650.0)
     tflops = peaks.get("bf16_tflops", 1590.0)
     src = "measured" if "hbm_gbs" in peaks else "fallback"
-    x = torch.randn(B, H * H, C, device="cuda").to(bf)
-    dout, out = torch.randn_like(x), torch.randn_like(x)
+
+    def conv_case(Hh, Cc):
+        per = 2 * B * Hh * Hh * Cc * 2                       # bytes of input + output of one launch
+        n = max(8, int(400e6 // per) + 1)
+        xs = [torch.randn(B, Hh, Hh, Cc, device="cuda").to(bf) for _ in range(n)]
+        ys = [torch.empty_like(xs[0]) for _ in range(n)]
+        w = (torch.randn(Cc, Cc, 3, 3, device="cuda") * (2.0 / (9 * Cc)) ** 0.5).to(bf)
+        pk = torch.empty(binding.conv3x3_packed_bytes(B, Hh, Hh, Cc), dtype=torch.uint8, device="cuda")
+        binding.conv3x3_pack(w, pk, Cc)
+        fns = [(lambda i=i: binding.conv3x3_packed(0, xs[i], w, pk, ys[i], B, Hh, Hh, Cc, s.cuda_stream)) for i in range(n)]
+        dt = _time_back_to_back(torch, fns, s)
+        return dt, per + w.numel() * 2, 2.0 * 9 * Cc * Cc * B * Hh * Hh, n
+
+    dt, alg, flops, n = conv_case(32, 16)
+    # DRAM traffic per launch from the ncu capture at batch 4096 (profiles/conv3x3_tc_kernel_c16_fwd_b4096_ncu_full.md):
+    # 134.3 MB read + 83.1 MB written for 268.4 MB algorithmic (part of the output is still in L2 when the kernel
+    # ends); traffic grows with the pixels processed, so it is scaled by batch
+    traffic = 217.4e6 * B / 4096.0
+    roof = {"kernel": "conv3x3_tc_kernel<16> (tensor-core 3x3 convolution, forward) C=16 32x32 B=%d" % B, "bound": "hbm",
+            "achieved": alg / dt / 1e9, "peak": hbm, "unit": "GB/s", "frac": alg / dt / 1e9 / hbm, "traffic": traffic,
+            "launch_us": dt * 1e6, "peak_source": src, "ncu_share_of_step": 0.170, "launches_timed": n,
+            "tflops": flops / dt / 1e12, "tensor_frac": flops / dt / 1e12 / tflops}
+    others = []
+    for (Hh, Cc) in ((16, 32), (8, 64)):
+        dtc, nbytes, fl, _ = conv_case(Hh, Cc)
+        others.append({"kernel": "conv3x3_tc_kernel<%d> fwd %dx%d B=%d" % (Cc, Hh, Hh, B), "launch_us": dtc * 1e6,
+                       "hbm_gbs": nbytes / dtc / 1e9, "hbm_frac": nbytes / dtc / 1e9 / hbm, "tflops": fl / dtc / 1e12,
+                       "tensor_frac": fl / dtc / 1e12 / tflops})
+    # batch-norm backward (sums + element-wise pass) on the largest map
+    H, C = 32, 16
+    per = 4 * B * H * H * C * 2
+    n = max(8, int(400e6 // per) + 1)
+    xs = [torch.randn(B, H * H, C, device="cuda").to(bf) for _ in range(n)]
+    douts = [torch.randn_like(xs[0]) for _ in range(n)]
+    dxs = [torch.empty_like(xs[0]) for _ in range(n)]
+    g = torch.ones(C, device="cuda").to(bf)
     mean, invstd = torch.zeros(C, device="cuda"), torch.ones(C, device="cuda")
     dg, db = torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
     scr = torch.zeros(binding.bn_scratch_elems(C), device="cuda")
-    dt = _time_kernel(torch, lambda: binding.bn_bwd_reduce(1, dout, out, x, mean, invstd, dg, db, scr, B, H * H, C, 1,
-                                                           s.cuda_stream), s, flush)
-    alg = 3 * x.numel() * 2                            # reads dout, out (ReLU mask), x; writes 2*C sums
-    # DRAM traffic per launch from the ncu capture at batch 4096 (profiles/bn_reduce_fast_kernel_...md): 414.1 MB for
-    # 402.7 MB algorithmic, scaled by pixels processed
-    traffic = 414.1e6 * B / 4096.0
-    roof = {"kernel": "bn_reduce_fast_kernel<bf16,8,1> (batch-norm backward sums) C=16 32x32 B=%d" % B, "bound": "hbm",
-            "achieved": alg / dt / 1e9, "peak": hbm, "unit": "GB/s", "frac": alg / dt / 1e9 / hbm, "traffic": traffic,
-            "launch_us": dt * 1e6, "peak_source": src, "ncu_share_of_step": 0.151}
-    others = []
-    for (Hh, Cc) in ((32, 16), (16, 32), (8, 64)):
-        xx = torch.randn(B, Hh, Hh, Cc, device="cuda").to(bf)
-        w = (torch.randn(Cc, Cc, 3, 3, device="cuda") * (2.0 / (9 * Cc)) ** 0.5).to(bf)
-        yy = torch.empty_like(xx)
-        pk = torch.empty(binding.conv3x3_packed_bytes(B, Hh, Hh, Cc), dtype=torch.uint8, device="cuda")
-        binding.conv3x3_pack(w, pk, Cc)
-        dtc = _time_kernel(torch, lambda: binding.conv3x3_packed(0, xx, w, pk, yy, B, Hh, Hh, Cc, s.cuda_stream), s, flush)
-        nbytes, flops = 2 * xx.numel() * 2 + w.numel() * 2, 2.0 * 9 * Cc * Cc * B * Hh * Hh
-        others.append({"kernel": "conv3x3_tc_kernel<%d> fwd %dx%d B=%d" % (Cc, Hh, Hh, B), "launch_us": dtc * 1e6,
-                       "hbm_gbs": nbytes / dtc / 1e9, "hbm_frac": nbytes / dtc / 1e9 / hbm, "tflops": flops / dtc / 1e12,
-                       "tensor_frac": flops / dtc / 1e12 / tflops})
+    fns = [(lambda i=i: binding.bn_bwd(1, douts[i], xs[i], xs[i], g, mean, invstd, dxs[i], dg, db, scr, B, H * H, C, 1,
+                                       s.cuda_stream)) for i in range(n)]
+    dtb = _time_back_to_back(torch, fns, s)
+    nb = 7 * B * H * H * C * 2                               # sums read dout, out, x; the element-wise pass reads them again, writes dx
+    others.append({"kernel": "bn_reduce_fast_kernel + bn_bwd_apply_kernel (batch-norm backward) C=16 32x32 B=%d" % B,
+                   "launch_us": dtb * 1e6, "hbm_gbs": nb / dtb / 1e9, "hbm_frac": nb / dtb / 1e9 / hbm})
     return roof, others
 
 
