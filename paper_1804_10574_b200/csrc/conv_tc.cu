@@ -1258,8 +1258,12 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int ncols = wide ? (2 * (rows + 2) + 3) * C : ((slab && !tall) ? 9 * C : 3 * C);
     const int tmem_cols = ncols <= 64 ? 64 : (ncols <= 128 ? 128 : (ncols <= 256 ? 256 : 512));
     const int n_tiles = (int)((long)B * H * W / kTileM);
+    // pixel chunks (= CTAs, = partials to fold): few at the training step's sizes, where the kernel shares the GPU with
+    // the other streams and the fold should stay small; one per 16 tiles, up to a CTA per SM, for large batches
     const int max_chunks = slab ? (C == 16 ? 74 : 37) : 24;
-    const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
+    int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
+    const int big = n_tiles / 16 < (slab ? kWgMaxChunks : 48) ? n_tiles / 16 : (slab ? kWgMaxChunks : 48);
+    if (big > chunks) chunks = big;
     // tall: the unused accumulator rows (filter rows >= 3) read up to 128 - 3C pixel rows past the last column box
     launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512 + (tall ? 4096 : 0), s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols, wide, tall);
     launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C, C, cin);
