@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_1804_10574_b200 import nets
-from tests.parity import run_pair
+from tests.parity import rel, run_pair
 
 pytestmark = pytest.mark.gpu
 
@@ -46,6 +46,21 @@ def test_resnet8_k2_20_steps_fp32():
 def test_resnet8_other_splits_fp32(splits):
     cfg = dict(nets.config("resnet8"), opt=dict(lr=0.05, momentum=0.9, weight_decay=5e-4))
     run_pair(cfg, 6, FP32_TOL, LOSS_TOL, split_after=splits, batch=5)
+
+
+@pytest.mark.parametrize("split", [1, 2, 3, 4], ids=["after1", "after3", "after5", "after7"])
+def test_resnet8_split_positions_adam_fp32(split):
+    """The split-position sweep of Section 5.1: ResNet-8 cut after weighted layer 1, 3, 5, 7 (after the stem and after
+    each block), trained with Adam (Algorithm 2) as there."""
+    cfg = dict(nets.config("resnet8"), opt=dict(lr=1e-3, momentum=0.0, weight_decay=0.0))
+    run_pair(cfg, 6, FP32_TOL, LOSS_TOL, split_after=[split], batch=6, opt="adam")
+
+
+@pytest.mark.parametrize("split", [[1], [4], [1, 2, 3]], ids=["after1", "after7", "K4"])
+def test_resnet8_split_positions_bf16(split):
+    """The same cuts in the bf16 mode the sweep is timed in (tensor-core kernels, epilogue batch-norm sums)."""
+    cfg = dict(nets.config("resnet8"), opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
+    run_pair(cfg, 5, BF16_TOL, 5e-3, precision="bf16", split_after=split, noise_mult=2.0)
 
 
 def test_resnet8_graph_replay_matches_fp32():
@@ -108,3 +123,43 @@ def test_resnet110_k4_full_size_bf16_graph():
     cfg = nets.config("resnet110")
     w = run_pair(cfg, 5, BF16_TOL, 5e-3, use_graph=True, noise_mult=2.0, check_every=2)
     print("resnet110 K=4 full size worst", w)
+
+
+_CHILD = r"""
+import sys, numpy as np, torch
+from paper_1804_10574_b200 import binding, nets, synth
+L = nets.resnet(3, 10)
+B, shape, classes = 32, (3, 32, 32), 10
+d = binding.Ddg(L, nets.split_even_blocks(L, 3), B, shape, classes, precision="bf16", lr=0.01, momentum=0.9,
+                weight_decay=5e-4, use_graph=True)
+d.set_weights(synth.init_weights(L, perturb_affine=0.1))
+losses = []
+for t in range(6):
+    x, y = synth.batch(t, B, shape, classes)
+    losses.append(d.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()))
+w = np.empty(d.n_params, dtype=np.float32)
+d.get_weights(w)
+np.save(sys.argv[1], np.concatenate([w, np.asarray(losses, dtype=np.float32)]))
+"""
+
+
+def test_epilogue_batch_norm_sums_match_separate_reductions(tmp_path):
+    """The batch-norm sums taken in the convolution epilogues and the separate reduction kernels are two evaluations
+    of the same sums in different orders: six ResNet-20 K=3 bf16 iterations in each mode (the switch is read once per
+    process, so each runs in a child) must end with the same weights up to what a last-bit difference of a statistic
+    can move through bf16 rounding."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = {}
+    for mode in ("1", "0"):
+        f = str(tmp_path / ("w%s.npy" % mode))
+        env = dict(os.environ, DDG_FUSE_BN=mode, PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
+        subprocess.run([sys.executable, "-c", _CHILD, f], check=True, env=env, cwd=root, timeout=600)
+        out[mode] = np.load(f)
+    a, b = out["1"], out["0"]
+    assert np.all(np.isfinite(a)) and np.all(np.isfinite(b))
+    assert abs(a[-1] - b[-1]) < 5e-3 * max(1.0, abs(b[-1]))          # last loss
+    assert rel(a[:-6], b[:-6]) < 2e-3                                  # all weights, one tensor
+
