@@ -99,9 +99,12 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
 
 /* One DDG iteration (Algorithm 1 / 2 with the sweeps of Eq. 3 and Eq. 6-7).
  *   x_dev: device, fp32, [B][in_c][in_h][in_w]; y_dev: device, int32 labels [B].
- *   loss_host: host, nullable.  Non-NULL: the call waits for the iteration and writes the mean cross-entropy
- *   of this iteration's forward pass.  NULL: the call only enqueues work; x_dev / y_dev must stay valid until
- *   ddg_sync (or a later call with loss_host != NULL) returns. */
+ *   loss_host: host, nullable.  Non-NULL: the call waits until this iteration's forward sweep has produced the
+ *   loss and writes the mean cross-entropy of this iteration's minibatch; the backward sweeps and updates of the
+ *   iteration may still be running when it returns (they only feed later iterations; ddg_sync, ddg_get_weights
+ *   and ddg_get_grads wait for them).  NULL: the call only enqueues work; x_dev / y_dev must stay valid until
+ *   ddg_sync (or a later call with loss_host != NULL) returns.  The inputs are copied into library-owned staging
+ *   buffers before the forward sweep reads them, so a call that returned a loss is done with x_dev / y_dev. */
 ddg_status ddg_step(ddg_ctx *ctx, const float *x_dev, const int *y_dev, float *loss_host);
 
 /* The same iteration with host inputs: copies x_host / y_host (host, same shapes) to the device on the

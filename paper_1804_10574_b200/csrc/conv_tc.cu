@@ -86,6 +86,8 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+__device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -415,11 +417,27 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
         uint32_t aph = 0;
         bool ok = true;
         for (int tile = blockIdx.x + grp * gridDim.x; tile < n_tiles && ok; tile += 2 * gridDim.x, aph ^= 1u) {
+            const size_t pix = (size_t)tile * kTileM + 32 * q + lane;
+            // what the epilogue reads from global memory for this pixel (shortcut gradient, batch-norm mask and input) was
+            // written long ago: start fetching it now, under the TMA and MMA latency of the tile
+            if (res_dout != nullptr) {
+#pragma unroll
+                for (int o = 0; o < C * 2; o += 128) {
+                    prefetch_l1(reinterpret_cast<const char *>(res_dout + pix * C) + o);
+                    prefetch_l1(reinterpret_cast<const char *>(res_out + pix * C) + o);
+                }
+            }
+            if (bn_x != nullptr) {
+#pragma unroll
+                for (int o = 0; o < C * 2; o += 128) {
+                    prefetch_l1(reinterpret_cast<const char *>(bn_mask + pix * C) + o);
+                    prefetch_l1(reinterpret_cast<const char *>(bn_x + pix * C) + o);
+                }
+            }
             ok = mbar_wait(tfull_bar(a), aph, abort_flag, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const size_t pix = (size_t)tile * kTileM + 32 * q + lane;
             const int wcol = lane % W;  // W divides 32: a warp holds whole image rows
             const uint32_t t_row = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * 3 * C);
 #pragma unroll 1

@@ -84,6 +84,7 @@ struct ddg_ctx {
     size_t x_elems = 0;
     float *dlogits = nullptr, *loss_dev = nullptr;
     float *pinned_loss = nullptr;
+    cudaStream_t loss_stream = nullptr;  // carries the loss read-back, so that it waits for the forward sweep only
     std::vector<cudaGraphExec_t> graphs;
     std::vector<long> graph_launches;
     long launches = 0;
@@ -489,7 +490,7 @@ ddg_status enqueue_iteration(ddg_ctx *ctx, long t, bool use_graph, long *launche
         ddg_status st = run_segment(ctx, k, 0, t, use_graph, &n);
         if (st != DDG_OK) return st;
         total += n;
-        if (k < K - 1) CU(cudaEventRecord(m.ev_fwd, m.stream));
+        CU(cudaEventRecord(m.ev_fwd, m.stream));  // for module k+1; the last module's marks the loss
     }
     // backward sweeps and updates: independent across modules within the iteration ("for k in parallel").  Ascending
     // k, so that module k waits for the error gradient module k+1 recorded in the PREVIOUS iteration.
@@ -545,8 +546,8 @@ ddg_status init_weights(ddg_ctx *ctx) {
     return DDG_OK;
 }
 
-ddg_status sync_all(ddg_ctx *ctx) {
-    for (auto &m : ctx->mods) CU(cudaStreamSynchronize(m.stream));
+// error words raised by kernels whose bounded waits ran out (reads the flags as they are now; does not wait)
+ddg_status check_kernel_errors(ddg_ctx *ctx) {
     if (ctx->prec == P_BF16) {
         const int code = conv_tc_error();
         if (code != 0) {
@@ -556,6 +557,11 @@ ddg_status sync_all(ddg_ctx *ctx) {
         }
     }
     return DDG_OK;
+}
+
+ddg_status sync_all(ddg_ctx *ctx) {
+    for (auto &m : ctx->mods) CU(cudaStreamSynchronize(m.stream));
+    return check_kernel_errors(ctx);
 }
 
 }  // namespace
@@ -599,6 +605,7 @@ void ddg_destroy(ddg_ctx *ctx) {
     }
     cudaFree(ctx->x_stage); cudaFree(ctx->y_stage); cudaFree(ctx->dlogits); cudaFree(ctx->loss_dev);
     if (ctx->pinned_loss) cudaFreeHost(ctx->pinned_loss);
+    if (ctx->loss_stream) cudaStreamDestroy(ctx->loss_stream);
     delete ctx;
 }
 
@@ -818,6 +825,7 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
     CU(cudaMalloc(&c->loss_dev, 4));
     CU(cudaMemset(c->loss_dev, 0, 4));
     CU(cudaMallocHost(&c->pinned_loss, 4));
+    CU(cudaStreamCreateWithFlags(&c->loss_stream, cudaStreamNonBlocking));
     // the memsets above ran on the legacy default stream, which the non-blocking module streams do not wait for
     CU(cudaDeviceSynchronize());
     ddg_status st = init_weights(c);
@@ -841,10 +849,14 @@ static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float 
     if (st != DDG_OK) { ctx->broken = true; return st; }
     ctx->t = t + 1;
     if (loss_host) {
-        CU(cudaMemcpyAsync(ctx->pinned_loss, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, ctx->mods[K - 1].stream));
-        st = sync_all(ctx);
-        if (st != DDG_OK) return st;
+        // The loss exists once the last module's forward sweep is done: wait for that only.  The backward sweeps and
+        // updates of this iteration stay in flight and overlap the caller's next step (the decoupling DDG is about).
+        CU(cudaStreamWaitEvent(ctx->loss_stream, ctx->mods[K - 1].ev_fwd, 0));
+        CU(cudaMemcpyAsync(ctx->pinned_loss, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, ctx->loss_stream));
+        CU(cudaStreamSynchronize(ctx->loss_stream));
         *loss_host = *ctx->pinned_loss;
+        st = check_kernel_errors(ctx);  // flags raised so far; a later call or ddg_sync reports what is still running
+        if (st != DDG_OK) return st;
     }
     return DDG_OK;
 }
