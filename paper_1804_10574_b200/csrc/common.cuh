@@ -71,16 +71,16 @@ __device__ __forceinline__ float warp_max(float v) {
 
 static inline int ceil_div(long a, long b) { return (int)((a + b - 1) / b); }
 
-// Programmatic dependent launch.  Every kernel of the library is launched with programmatic stream serialisation: the
-// next kernel of the stream may be scheduled while this one is still running, so that its launch latency and its
-// prologue overlap this kernel's tail.  The contract that keeps this correct: every kernel executes pdl_wait() before
+// Programmatic dependent launch.  Where pdl_enabled() says so (single kernels, single-module networks) a kernel is
+// launched with programmatic stream serialisation: the next kernel of the stream may be scheduled while this one is
+// still running, so that its launch latency and its prologue overlap this kernel's tail.  The contract that keeps this correct: every kernel executes pdl_wait() before
 // its first access to global memory that an earlier kernel may write or still read; the wait returns when all
 // preceding kernels of the stream have completed and their writes are visible.  pdl_launch() tells the scheduler that
 // the next kernel may start being placed.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-bool pdl_enabled();  // defined in engine.cu; DDG_PDL=0 in the environment switches the launch attribute off
+bool pdl_enabled();  // defined in engine.cu: off while a multi-module iteration is enqueued; DDG_PDL=0/1 forces it
 
 template <typename... KArgs, typename... Args>
 inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {

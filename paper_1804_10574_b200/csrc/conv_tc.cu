@@ -12,14 +12,15 @@
 // neighbouring pixels, y[h][w] = P_0[h][w-1] + P_1[h][w] + P_2[h][w+1], with warp shuffles (a warp holds whole image
 // rows; the image border contributes zero).  The filter-row shift costs nothing: the three rows read the same TMA box
 // at offsets of 0, W and 2W pixels, which are whole swizzle periods, so only the descriptor start address moves.
-// Warp roles: warp 0 issues TMA, warp 1 issues MMAs, warps 2-5 and 6-9 (two groups, one per TMEM accumulator, each
-// taking every other tile) drain TMEM, combine, add the shortcut gradient where asked, convert to bf16 and store, so
-// that the epilogue of tile i overlaps the MMAs of tile i+1.  With `dual` (many small tiles per CTA: C = 16) the CTA
-// runs TWO independent pipelines over alternate tiles instead, warps 10 / 11 being the second TMA / MMA issuer, each
-// pipeline with half of the stage ring, one accumulator and one epilogue group: there the cost of a tile is the chain
-// of barrier hand-offs and instruction issue of the single MMA thread (about a thousand cycles), not data movement
-// or tensor-core time, and two chains side by side raise the tile rate of an SM.  Every mbarrier wait is bounded: when one runs out, the CTA raises an error word that the host reads at its
-// next sync point, and leaves.
+// Warp roles: a CTA runs P independent pipelines (1, 2 or 4) over interleaved tiles, each with its own TMA-issuing
+// warp (warps 0..P-1), MMA-issuing warp (warps P..2P-1), share of the stage ring and TMEM accumulators; the remaining
+// warps are epilogue groups of four (one warp per TMEM lane quarter) that drain TMEM, combine, add the shortcut gradient
+// where asked, convert to bf16 and store, shared out among the pipelines as EpiPlan says.  Why several pipelines: the
+// cost of a tile is the chain of barrier hand-offs and tcgen05 instruction issue of its single MMA thread (150-200
+// cycles per operation, a thousand and more per tile), not data movement, tensor-core or epilogue time (removing the
+// stores, the shuffles and two of the three TMEM loads of the epilogue changes the kernel's time by under 10 %), so
+// chains side by side raise the tile rate of an SM.  Every mbarrier wait is bounded: when one runs out, the CTA raises
+// an error word that the host reads at its next sync point, and leaves.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
@@ -35,7 +36,7 @@ namespace ddg {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kTcThreads = 384;   // convolution: two pipelines, each a TMA warp, an MMA warp and four epilogue warps
+constexpr int kTcMaxThreads = 768;  // convolution: at most four pipelines (TMA warp, MMA warp, four epilogue warps each)
 constexpr int kS2Threads = 320;   // stride-2 convolution: TMA warp, MMA warp, two groups of four epilogue warps
 constexpr int kWgThreads = 192;   // weight gradient: TMA warp, MMA warp, four epilogue warps
 constexpr unsigned kSpinLimit = 1u << 24;  // bounded waits: ~ a second at worst, then the CTA gives up
@@ -166,9 +167,9 @@ template <int C> __host__ __device__ inline ConvSmem conv_smem_plan(int n_stages
     p.tail_off = p.a_off + (uint32_t)n_stages * (uint32_t)stage_bytes;
     return p;
 }
-// after the pipeline stages: 512 bytes of barriers and flags, 4 KB of per-warp batch-norm sums (8 warps x 4 channel
-// chunks x 32 lanes), 512 bytes of per-channel mean / invstd
-constexpr int kTailBytes = 512 + 4096 + 512;
+// after the pipeline stages: 512 bytes of barriers and flags, 8 KB of per-warp batch-norm sums (up to 16 epilogue
+// warps x 4 channel chunks x 32 lanes), 512 bytes of per-channel mean / invstd
+constexpr int kTailBytes = 512 + 8192 + 512;
 template <int C> inline size_t conv_smem_bytes(int n_stages, int stage_bytes) {
     return 1024 + conv_smem_plan<C>(n_stages, stage_bytes).tail_off + kTailBytes;
 }
@@ -264,11 +265,20 @@ __global__ void pack_one_filter_kernel(const bf16 *__restrict__ w, uint8_t *__re
 //   slab == 0 (tile = several whole small images): one TMA box of the tile shifted by ky-1 rows per filter row (3 per
 //              tile), zero-filled at the image border.
 // ---------------------------------------------------------------------------------------------------------
+// How the epilogue warp groups (four warps each, one per TMEM lane quarter; the warps after the 2 * n_pipes issuing
+// warps) share the tiles of a pipeline.  A pipeline numbers its tiles it = 0, 1, ...; tile `it` accumulates in the
+// pipeline's accumulator it % n_acc and is drained by the `split` groups of slot it % n_slots, each of which takes an
+// equal share of the tile's 16-channel chunks.
+//   n_slots = 2, split = 1: two groups take alternate tiles (the epilogue of one overlaps the next one's);
+//   n_slots = 1, split = 2: two groups halve every tile (shorter epilogue where a CTA has one or two tiles).
+struct EpiPlan { int n_pipes, n_acc, n_slots, split; };
+
+// (bound of 768 threads: caps the kernel at 80 registers, so that two 384-thread CTAs of different streams share an SM)
 template <int C>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(768, 1)
 conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
                   bf16 *__restrict__ dst, int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
-                  int slab, int n_stages, int stage_bytes, int dual, int tmem_cols, const bf16 *__restrict__ res_dout,
+                  int slab, int n_stages, int stage_bytes, int tmem_cols, EpiPlan plan_e, const bf16 *__restrict__ res_dout,
                   const bf16 *__restrict__ res_out, float *__restrict__ stat_part, unsigned *__restrict__ stat_counter,
                   float *__restrict__ stat_o0, float *__restrict__ stat_o1, const bf16 *__restrict__ bn_mask,
                   const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd) {
@@ -290,7 +300,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 9) * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 9) * 8 + 8);
     float (*sm_run)[4][32] = reinterpret_cast<float (*)[4][32]>(tail + 512);  // [epilogue warp][channel chunk][lane]
-    float *sm_stat = reinterpret_cast<float *>(tail + 512 + 4096);            // mean[C], invstd[C]
+    float *sm_stat = reinterpret_cast<float *>(tail + 512 + 8192);            // mean[C], invstd[C]
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
@@ -301,11 +311,11 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (stat_part != nullptr)
-        for (int i = threadIdx.x; i < 8 * 4 * 32; i += blockDim.x) (&sm_run[0][0][0])[i] = 0.f;
+        for (int i = threadIdx.x; i < 16 * 4 * 32; i += blockDim.x) (&sm_run[0][0][0])[i] = 0.f;
     if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");  // the first TMA would otherwise wait for its descriptor
         for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < Cfg::acc_stages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        for (int a = 0; a < 4; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4 * plan_e.split); }
         mbar_init(w_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -338,13 +348,14 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     const int tiles_per_img = H / rows_per_tile;  // tiles per image when a tile lies inside one image
     const int loads_per_tile = slab ? 1 : 3;
 
-    // pipeline g (0, or 0 and 1 with `dual`) owns stages [g*ring, (g+1)*ring) and takes every tile_step-th tile
-    const int ring = dual ? n_stages >> 1 : n_stages;
-    const int tile_step = dual ? 2 * gridDim.x : gridDim.x;
-    if (warp == 0 || warp == 10) {
+    // pipeline g owns stages [g*ring, (g+1)*ring) and takes every tile_step-th tile
+    const int n_pipes = plan_e.n_pipes;
+    const int ring = n_stages / n_pipes;
+    const int tile_step = n_pipes * gridDim.x;
+    if (warp < n_pipes) {
         // ---------------- TMA producers ----------------
-        const int g = warp == 0 ? 0 : 1;
-        if (lane == 0 && (g == 0 || dual)) {
+        const int g = warp;
+        if (lane == 0) {
             if (g == 0 && w_packed != nullptr) {  // pre-arranged filter image: one bulk copy
                 mbar_expect_tx(w_bar, Cfg::w_bytes);
                 bulk_copy_g2s(w_base, w_packed + (dgrad ? Cfg::w_bytes : 0), Cfg::w_bytes, w_bar);
@@ -369,20 +380,19 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                 for (int i = 0; i < 2000; ++i) __nanosleep(100);
             }
         }
-    } else if (warp == 1 || warp == 11) {
+    } else if (warp < 2 * n_pipes) {
         // ---------------- MMA issuers ----------------
-        const int g = warp == 1 ? 0 : 1;
-        if (lane == 0 && (g == 0 || dual)) {
+        const int g = warp - n_pipes;
+        if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((3 * C) >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
             int ls = 0, it = 0;
             uint32_t ph = 0;
             bool ok = true;
             if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, abort_flag, 5);
             for (int tile = blockIdx.x + g * gridDim.x; tile < n_tiles && ok; tile += tile_step, ++it) {
-                // accumulator: the pipeline's own one (dual), else the two in turn; the epilogue group of the same number
-                // drains it
-                const int a = dual ? g : (it & 1);
-                const uint32_t aph = dual ? (it & 1) : ((it >> 1) & 1);
+                // the pipeline's accumulators in turn
+                const int a = g * plan_e.n_acc + it % plan_e.n_acc;
+                const uint32_t aph = (uint32_t)(it / plan_e.n_acc) & 1u;
                 ok = mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, 2);
                 if (!ok) break;
                 tc_fence_after();
@@ -410,13 +420,19 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
         }
     } else {
         // ---------------- epilogue: TMEM -> registers -> bf16 -> global ----------------
-        // Two groups of four warps; group g drains every other tile, so two epilogues overlap.
         const int q = warp & 3;  // a warp may only touch TMEM lanes [32*(warp%4), +32)
-        const int grp = (warp - 2) >> 2;
-        const int a = grp;
-        uint32_t aph = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x + grp * gridDim.x; tile < n_tiles && ok; tile += 2 * gridDim.x, aph ^= 1u) {
+        const int ew = warp - 2 * n_pipes;  // index among the epilogue warps
+        const int grp = ew >> 2;
+        const int per_pipe = plan_e.n_slots * plan_e.split;
+        const int pipe = grp / per_pipe, slot = (grp % per_pipe) / plan_e.split, share = grp % plan_e.split;
+        constexpr int kChunks = C / 16;
+        const int c_begin = 16 * (share * kChunks / plan_e.split), c_end = 16 * ((share + 1) * kChunks / plan_e.split);
+        bool ok = pipe < n_pipes;  // a group the plan has no work for leaves at once
+        for (int it = slot; ok; it += plan_e.n_slots) {
+            const int tile = blockIdx.x + pipe * gridDim.x + it * tile_step;
+            if (tile >= n_tiles) break;
+            const int a = pipe * plan_e.n_acc + it % plan_e.n_acc;
+            const uint32_t aph = (uint32_t)(it / plan_e.n_acc) & 1u;
             const size_t pix = (size_t)tile * kTileM + 32 * q + lane;
             // what the epilogue reads from global memory for this pixel (shortcut gradient, batch-norm mask and input) was
             // written long ago: start fetching it now, under the TMA and MMA latency of the tile
@@ -441,13 +457,13 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
             const int wcol = lane % W;  // W divides 32: a warp holds whole image rows
             const uint32_t t_row = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * 3 * C);
 #pragma unroll 1
-            for (int c0 = 0; c0 < C; c0 += 16) {
+            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 float p0[16], p1[16], p2[16];
                 tc_ld16(t_row + (uint32_t)c0, p0);            // filter column 0: belongs to the pixel on the right
                 tc_ld16(t_row + (uint32_t)(C + c0), p1);
                 tc_ld16(t_row + (uint32_t)(2 * C + c0), p2);  // filter column 2: belongs to the pixel on the left
                 tc_wait_ld();
-                if (c0 + 16 >= C) {  // last read of this accumulator stage: hand it back to the MMA warp
+                if (c0 + 16 >= c_end) {  // this group's last read of the accumulator: hand it back to the MMA warp
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(a));
@@ -501,7 +517,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                         }
                     }
                     warp_transpose_sum32(v, lane);
-                    sm_run[warp - 2][c0 >> 4][lane] += v[0];  // lane l < 16: first sum of channel c0+l; else second sum
+                    sm_run[ew][c0 >> 4][lane] += v[0];  // lane l < 16: first sum of channel c0+l; else second sum
                 }
             }
         }
@@ -514,11 +530,11 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                      : "memory");
     }
     if (stat_part == nullptr) return;
-    if (threadIdx.x < 2 * C) {  // the eight epilogue warps' sums in a fixed order
+    if (threadIdx.x < 2 * C) {  // the epilogue warps' sums in a fixed order
         const int c = threadIdx.x % C, l = (c & 15) + 16 * (threadIdx.x / C);
         float t = 0.f;
 #pragma unroll
-        for (int wq = 0; wq < 8; ++wq) t += sm_run[wq][c >> 4][l];
+        for (int wq = 0; wq < 16; ++wq) t += sm_run[wq][c >> 4][l];
         stat_part[(size_t)blockIdx.x * 2 * C + threadIdx.x] = t;
     }
     __threadfence();
@@ -529,7 +545,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     if (!*is_last) return;
     __threadfence();
     // last CTA: partials of all CTAs, `ways` threads per value, eight loads in flight per thread, fixed order
-    double *fold = reinterpret_cast<double *>(&sm_run[0][0][0]);  // kTcThreads doubles fit the 4 KB
+    double *fold = reinterpret_cast<double *>(&sm_run[0][0][0]);  // one double per thread fits the 8 KB
     constexpr int nval = 2 * C;
     const int ways = (int)blockDim.x / nval;
     const int v = threadIdx.x % nval, way = threadIdx.x / nval;
@@ -1239,18 +1255,39 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     CUtensorMap map;
     if (32 % W != 0 || !get_map(src, B, H, W, C, box_rows, imgs, &map)) return -1;
     const int stage_bytes = box_rows * imgs * W * C * 2;
-    int n_stages = (kSmemBudget - (int)conv_smem_plan<C>(0, 0).a_off) / stage_bytes;
-    if (n_stages > kMaxStages) n_stages = kMaxStages;
-    if (n_stages < 3) n_stages = 3;
     const int n_tiles = (int)((long)B * H * W / kTileM);
     const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
-    // two pipelines per CTA where a CTA has many small tiles (each pipeline then owns half of an even stage ring)
-    const int dual = (C == 16 && slab && n_tiles >= 4 * grid) ? 1 : 0;
-    if (dual) n_stages &= ~1;
-    // a CTA with a single tile uses one accumulator: half the TMEM columns, so that CTAs of other streams fit beside it
-    const int tmem_cols = n_tiles <= grid ? TcCfg<C>::tmem_cols / 2 : TcCfg<C>::tmem_cols;
-    launch_k(conv3x3_tc_kernel<C>, grid, dual ? kTcThreads : kS2Threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
-        stage_bytes, dual, tmem_cols, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
+    // Pipelines per CTA and epilogue plan.
+    //   C = 16 (one 16-channel chunk per tile): two pipelines where a CTA has at least four tiles, four where it has at
+    //   least sixteen (large batches); below that one pipeline whose two epilogue groups take alternate tiles.
+    //   C >= 32: the two groups of a pipeline halve every tile, which shortens the epilogue of CTAs with one or two tiles
+    //   (the training step's sizes); two pipelines where a CTA has at least three tiles.
+    // A CTA with a single tile uses one accumulator: half the TMEM columns, so that CTAs of other streams fit beside it.
+    EpiPlan ep;
+    if (C == 16) {
+        const int P = !slab ? 1 : (n_tiles >= 16 * grid ? 4 : (n_tiles >= 4 * grid ? 2 : 1));
+        const int n_acc = P > 1 ? 1 : (n_tiles <= grid ? 1 : 2);
+        ep = EpiPlan{P, n_acc, n_acc, 1};
+    } else {
+        const int P = n_tiles >= 3 * grid ? 2 : 1;
+        const int n_acc = n_tiles <= grid ? 1 : ((P == 2 && C == 64) ? 1 : 2);  // 2 x 2 x 192 columns would not fit
+        ep = EpiPlan{P, n_acc, 1, 2};
+    }
+    const int groups = ep.n_pipes * ep.n_slots * ep.split;
+    const int threads = 32 * (2 * ep.n_pipes + 4 * (groups < 2 ? 2 : groups));
+    // CTAs with many tiles take the whole SM's shared memory for the stage ring; the others about half of it
+    const int budget = n_tiles >= 8 * grid ? kSmemMax - 1024 - kTailBytes : kSmemBudget;
+    int n_stages = (budget - (int)conv_smem_plan<C>(0, 0).a_off) / stage_bytes;
+    if (n_stages > kMaxStages) n_stages = kMaxStages;
+    const int min_ring = 3;
+    if (n_stages < min_ring * ep.n_pipes) n_stages = min_ring * ep.n_pipes;
+    n_stages -= n_stages % ep.n_pipes;
+    const int acc_cols = ep.n_pipes * ep.n_acc * 3 * C;
+    int tmem_cols = 32;
+    while (tmem_cols < acc_cols) tmem_cols <<= 1;
+    if (tmem_cols > 512 || conv_smem_bytes<C>(n_stages, stage_bytes) > (size_t)kSmemMax) return -1;
+    launch_k(conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
+        stage_bytes, tmem_cols, ep, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
         bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd);
     return 1;
 }

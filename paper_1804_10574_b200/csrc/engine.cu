@@ -567,9 +567,16 @@ ddg_status sync_all(ddg_ctx *ctx) {
 }  // namespace
 
 namespace ddg {
+// Programmatic dependent launch pays where one stream has the GPU to itself (K = 1, single kernels): the next
+// kernel's launch latency hides under the running one.  With several module streams it loses: a kernel that was
+// placed early holds its shared memory, TMEM columns and registers while it waits for its predecessor, and keeps the
+// other modules' CTAs off the SM (measured on ResNet-110, K = 4: 2.13 ms per iteration with, 1.99 ms without).  The
+// engine therefore clears this flag while it enqueues an iteration of a multi-module network.  DDG_PDL=0 / 1 in the
+// environment forces the launch attribute off / on.
+thread_local bool t_pdl_wanted = true;
 bool pdl_enabled() {
-    static const bool on = [] { const char *e = getenv("DDG_PDL"); return !(e && e[0] == '0'); }();
-    return on;
+    static const int forced = [] { const char *e = getenv("DDG_PDL"); return e ? (e[0] == '0' ? 0 : 1) : -1; }();
+    return forced >= 0 ? forced == 1 : t_pdl_wanted;
 }
 // lets the other translation units leave a message for ddg_last_error(NULL)
 void set_global_error(const char *msg) { g_create_error = msg; }
@@ -845,7 +852,9 @@ static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float 
     CU(cudaMemcpyAsync(ctx->y_stage + (size_t)(t % K) * ctx->B, y, (size_t)ctx->B * 4, kind, s0));
     // the first K-1 iterations have modules in warm-up and a different shape: they are not recorded
     const bool steady = t >= K - 1;
+    ddg::t_pdl_wanted = ctx->K == 1;
     ddg_status st = enqueue_iteration(ctx, t, ctx->cfg.use_graph && steady, &ctx->launches);
+    ddg::t_pdl_wanted = true;
     if (st != DDG_OK) { ctx->broken = true; return st; }
     ctx->t = t + 1;
     if (loss_host) {

@@ -474,10 +474,161 @@ static int red_fast_grid(long nvec, int per_sm) {
     return (int)(g < 1 ? 1 : g);
 }
 
+__device__ __forceinline__ void unpack_bf16x8(const uint4 &q, float (&f)[8]) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        f[2 * k] = __uint_as_float(w[k] << 16);
+        f[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+}
+__device__ __forceinline__ uint4 pack_bf16x8(const float (&f)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
+        w[k] = *reinterpret_cast<const uint32_t *>(&h);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+
+// Reductions over large bf16 tensors (more vectors than one trip of the kernel above covers): one 768-thread CTA per
+// SM (few partials for the last CTA to fold), operands kept as raw 16-byte registers with the loads of U vectors of
+// each issued before the first use, so that an SM has ~70 KB of loads in flight.  The second backward sum is accumulated as sum dz*(x - mean) and scaled by
+// invstd once at the end.  Same fixed folding order as above: lanes, warps, then CTAs in index order by the last CTA.
+static constexpr int kBigThreads = 768;
+
+template <int MODE, int U>
+__global__ void __launch_bounds__(kBigThreads, 1)
+bn_reduce_big_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ dout, const bf16 *__restrict__ out,
+                     const float *__restrict__ mean_in, const float *__restrict__ invstd_in, float *o0, float *o1,
+                     float *scratch, long npix, int C, int relu) {
+    pdl_launch();
+    pdl_wait();
+    constexpr int kWarps = kBigThreads / 32;
+    __shared__ float sm[kWarps][2 * 128];
+    __shared__ bool is_last;
+    __shared__ double fold[kBigThreads];
+    unsigned *counter = reinterpret_cast<unsigned *>(scratch);
+    float *part = scratch + 32;
+    const int groups = C / 8;
+    const long nvec = npix * groups;
+    const long tid = (long)blockIdx.x * kBigThreads + threadIdx.x, stride = (long)gridDim.x * kBigThreads;
+    const int c0 = (int)(tid & (groups - 1)) * 8;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float s0[8], s1[8], mu[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { s0[j] = 0.f; s1[j] = 0.f; mu[j] = MODE == 1 ? mean_in[c0 + j] : 0.f; }
+    const uint4 *x4 = reinterpret_cast<const uint4 *>(x), *d4 = reinterpret_cast<const uint4 *>(dout),
+                *o4 = reinterpret_cast<const uint4 *>(out);
+    for (long i0 = tid; i0 < nvec; i0 += U * stride) {
+        uint4 xq[U], dq[U], oq[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long i = i0 + u * stride;
+            if (i < nvec) {
+                xq[u] = x4[i];
+                if (MODE == 1) {
+                    dq[u] = d4[i];
+                    if (relu) oq[u] = o4[i];
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (i0 + u * stride < nvec) {
+                float xv[8], dv[8], ov[8];
+                unpack_bf16x8(xq[u], xv);
+                if (MODE == 1) {
+                    unpack_bf16x8(dq[u], dv);
+                    if (relu) unpack_bf16x8(oq[u], ov);
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (MODE == 0) { s0[j] += xv[j]; s1[j] = fmaf(xv[j], xv[j], s1[j]); }
+                    else {
+                        const float d = (relu && !(ov[j] > 0.f)) ? 0.f : dv[j];
+                        s0[j] += d;
+                        s1[j] = fmaf(d, xv[j] - mu[j], s1[j]);
+                    }
+                }
+            }
+        }
+    }
+    for (int o = 16; o >= groups; o >>= 1) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            s0[j] += __shfl_xor_sync(0xffffffffu, s0[j], o);
+            s1[j] += __shfl_xor_sync(0xffffffffu, s1[j], o);
+        }
+    }
+    if (lane < groups) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { sm[warp][c0 + j] = s0[j]; sm[warp][C + c0 + j] = s1[j]; }
+    }
+    __syncthreads();
+    if (threadIdx.x < 2 * C) {
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) t += sm[w][threadIdx.x];
+        part[(size_t)blockIdx.x * 2 * C + threadIdx.x] = t;
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int nval = 2 * C, ways = kBigThreads / nval;
+    const int v = threadIdx.x % nval, way = threadIdx.x / nval;
+    double acc = 0.0;
+    if (way < ways) {
+        double a8[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+        unsigned i = way;
+        for (; i + 7 * ways < gridDim.x; i += 8 * ways) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) a8[u] += (double)__ldcg(part + (size_t)(i + u * ways) * nval + v);
+        }
+        for (; i < gridDim.x; i += ways) a8[0] += (double)__ldcg(part + (size_t)i * nval + v);
+        acc = ((a8[0] + a8[1]) + (a8[2] + a8[3])) + ((a8[4] + a8[5]) + (a8[6] + a8[7]));
+    }
+    fold[threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.x < C) {
+        const int c = threadIdx.x;
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < ways; ++w) { a += fold[w * nval + c]; b += fold[w * nval + C + c]; }
+        if (MODE == 0) {
+            double m = a / (double)npix, var = b / (double)npix - m * m;
+            if (var < 0.0) var = 0.0;
+            o0[c] = (float)m;
+            o1[c] = (float)(1.0 / sqrt(var + (double)kBnEps));
+        } else {
+            o0[c] = (float)a;                             // dbeta
+            o1[c] = (float)(b * (double)invstd_in[c]);  // dgamma
+        }
+    }
+    if (threadIdx.x == 0) *counter = 0u;
+}
+
+static bool red_big_ok(int prec, long nvec, int C) {
+    return prec == P_BF16 && C % 8 == 0 && C <= 128 && red_fast_ok(C, 8) && nvec > 16L * 148 * kRedThreads;
+}
+static int red_big_grid(long nvec, int U) {
+    long g = (nvec + (long)kBigThreads * U - 1) / ((long)kBigThreads * U);
+    return (int)(g > 148 ? 148 : g);
+}
+
 template <typename T> static int vec_for(int C) { return (C % Vec16<T>::N == 0) ? Vec16<T>::N : 1; }
 
 int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *scratch, long npix, int C,
                     cudaStream_t s) {
+    if (red_big_ok(prec, npix * (C / 8), C)) {
+        launch_k(bn_reduce_big_kernel<0, 4>, red_big_grid(npix * (C / 8), 4), kBigThreads, 0, s, (const bf16 *)x, (const bf16 *)nullptr,
+                 (const bf16 *)nullptr, (const float *)nullptr, (const float *)nullptr, mean, invstd, scratch, npix, C, 0);
+        return 1;
+    }
     DISPATCH_PREC(prec, {
         if (red_fast_ok(C, Vec16<T>::N)) {
             constexpr int V = Vec16<T>::N;
@@ -496,6 +647,11 @@ int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *
 int launch_bn_bwd_reduce(int prec, const void *dout, const void *out, const void *x, const float *mean,
                          const float *invstd, float *dgamma, float *dbeta, float *scratch, long npix, int C, int relu,
                          cudaStream_t s) {
+    if (red_big_ok(prec, npix * (C / 8), C)) {
+        launch_k(bn_reduce_big_kernel<1, 2>, red_big_grid(npix * (C / 8), 2), kBigThreads, 0, s, (const bf16 *)x, (const bf16 *)dout,
+                 (const bf16 *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
+        return 1;
+    }
     DISPATCH_PREC(prec, {
         if (red_fast_ok(C, Vec16<T>::N)) {
             constexpr int V = Vec16<T>::N;
@@ -558,9 +714,94 @@ bn_apply_kernel(const T *__restrict__ x, const T *__restrict__ gamma, const T *_
     store_a<T, A, VEC>(y + p * C + c0, v);
 }
 
+// Fast path of the element-wise pass for bf16 tensors (no shortcut or the identity shortcut; C/8 a power of two):
+// the per-channel constants are folded once per CTA into scale = gamma*invstd and shift = beta - mean*scale (shared
+// memory, then registers: the flat 16-byte-vector walk keeps a thread on the same 8 channels), a thread issues the
+// loads of U vectors of every operand, kept as raw 16-byte registers, before it uses the first, and the grid is
+// capped at three CTAs per SM.
+static constexpr int kApplyCtasPerSm = 3;
+
+template <int U>
+__global__ void __launch_bounds__(kThreads, kApplyCtasPerSm)
+bn_apply_fast_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ gamma, const bf16 *__restrict__ beta,
+                     const float *__restrict__ mean, const float *__restrict__ invstd, const bf16 *__restrict__ res,
+                     bf16 *__restrict__ y, long nvec, int C, int relu) {
+    __shared__ float sm_scale[128], sm_shift[128];
+    pdl_launch();
+    pdl_wait();
+    for (int c = threadIdx.x; c < C; c += kThreads) {
+        const float sc = to_f(gamma[c]) * invstd[c];
+        sm_scale[c] = sc;
+        sm_shift[c] = to_f(beta[c]) - mean[c] * sc;
+    }
+    __syncthreads();
+    const int groups = C / 8;
+    const long tid = (long)blockIdx.x * kThreads + threadIdx.x, stride = (long)gridDim.x * kThreads;
+    const int c0 = (int)(tid & (groups - 1)) * 8;
+    float sc[8], sh[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { sc[j] = sm_scale[c0 + j]; sh[j] = sm_shift[c0 + j]; }
+    const uint4 *x4 = reinterpret_cast<const uint4 *>(x), *r4 = reinterpret_cast<const uint4 *>(res);
+    uint4 *y4 = reinterpret_cast<uint4 *>(y);
+    for (long i0 = tid; i0 < nvec; i0 += U * stride) {
+        uint4 xq[U], rq[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long i = i0 + u * stride;
+            if (i < nvec) {
+                xq[u] = x4[i];
+                if (res != nullptr) rq[u] = r4[i];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long i = i0 + u * stride;
+            if (i < nvec) {
+                float v[8], r[8];
+                unpack_bf16x8(xq[u], v);
+                if (res != nullptr) unpack_bf16x8(rq[u], r);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float t = fmaf(v[j], sc[j], sh[j]);
+                    if (res != nullptr) t += r[j];
+                    v[j] = (relu && !(t > 0.f)) ? 0.f : t;
+                }
+                y4[i] = pack_bf16x8(v);
+            }
+        }
+    }
+}
+
+static bool apply_fast_ok(int C, int V) {
+    if (C % V != 0 || C > 128) return false;
+    const int groups = C / V;
+    return (groups & (groups - 1)) == 0 && groups <= 32;
+}
+// vectors per thread and trip: as many as still leave every SM its three CTAs
+static int apply_unroll(long nvec) {
+    const long full = 148L * kApplyCtasPerSm * kThreads;
+    return nvec >= 4 * full ? 4 : (nvec >= 2 * full ? 2 : 1);
+}
+static int apply_grid(long nvec, int U) {
+    long g = (nvec + (long)kThreads * U - 1) / ((long)kThreads * U);
+    if (g > 148L * kApplyCtasPerSm) g = 148L * kApplyCtasPerSm;
+    return (int)(g < 1 ? 1 : g);
+}
+
 int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta, const float *mean,
                     const float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu, cudaStream_t s) {
     const long npix = (long)B * H * W;
+    if (prec == P_BF16 && sc.mode != 2 && apply_fast_ok(C, Vec16<bf16>::N)) {
+        typedef bf16 T;
+        constexpr int V = Vec16<T>::N;
+        const long nvec = npix * (C / V);
+        const int U = apply_unroll(nvec);
+        const T *res = sc.mode == 1 ? (const T *)sc.a : nullptr;
+        auto k = U == 4 ? bn_apply_fast_kernel<4> : (U == 2 ? bn_apply_fast_kernel<2> : bn_apply_fast_kernel<1>);
+        launch_k(k, apply_grid(nvec, U), kThreads, 0, s, (const T *)x, (const T *)gamma, (const T *)beta, mean, invstd, res,
+                 (T *)y, nvec, C, relu);
+        return 1;
+    }
     DISPATCH_PREC(prec, {
         constexpr int V = Vec16<T>::N;
         if (C % V == 0 && (sc.mode != 2 || sc.c_small % V == 0)) {
@@ -608,9 +849,78 @@ bn_bwd_apply_kernel(const T *__restrict__ dout, const T *__restrict__ out, const
     store_a<T, A, VEC>(dx + p * C + c0, dv);
 }
 
+// Fast path for bf16 tensors, laid out like bn_apply_fast_kernel.  With gi = gamma*invstd and n pixels,
+//   dx = gi*(dz - dbeta/n - xhat*dgamma/n) = gi*dz + k1*x + k0,  k1 = -gi*invstd*dgamma/n,  k0 = -gi*dbeta/n - k1*mean.
+template <int U>
+__global__ void __launch_bounds__(kThreads, kApplyCtasPerSm)
+bn_bwd_apply_fast_kernel(const bf16 *__restrict__ dout, const bf16 *__restrict__ out, const bf16 *__restrict__ x,
+                         const bf16 *__restrict__ gamma, const float *__restrict__ mean, const float *__restrict__ invstd,
+                         const float *__restrict__ dgamma, const float *__restrict__ dbeta, bf16 *__restrict__ dx,
+                         long nvec, long npix, int C, int relu) {
+    __shared__ float sm_gi[128], sm_k1[128], sm_k0[128];
+    pdl_launch();
+    pdl_wait();
+    for (int c = threadIdx.x; c < C; c += kThreads) {
+        const float inv_n = 1.f / (float)npix;
+        const float gi = to_f(gamma[c]) * invstd[c];
+        const float k1 = -gi * invstd[c] * dgamma[c] * inv_n;
+        sm_gi[c] = gi;
+        sm_k1[c] = k1;
+        sm_k0[c] = -gi * dbeta[c] * inv_n - k1 * mean[c];
+    }
+    __syncthreads();
+    const int groups = C / 8;
+    const long tid = (long)blockIdx.x * kThreads + threadIdx.x, stride = (long)gridDim.x * kThreads;
+    const int c0 = (int)(tid & (groups - 1)) * 8;
+    float gi[8], k1[8], k0[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { gi[j] = sm_gi[c0 + j]; k1[j] = sm_k1[c0 + j]; k0[j] = sm_k0[c0 + j]; }
+    const uint4 *x4 = reinterpret_cast<const uint4 *>(x), *d4 = reinterpret_cast<const uint4 *>(dout),
+                *o4 = reinterpret_cast<const uint4 *>(out);
+    uint4 *dx4 = reinterpret_cast<uint4 *>(dx);
+    for (long i0 = tid; i0 < nvec; i0 += U * stride) {
+        uint4 xq[U], dq[U], oq[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long i = i0 + u * stride;
+            if (i < nvec) {
+                xq[u] = x4[i];
+                dq[u] = d4[i];
+                if (relu) oq[u] = o4[i];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long i = i0 + u * stride;
+            if (i < nvec) {
+                float xv[8], dv[8], ov[8];
+                unpack_bf16x8(xq[u], xv);
+                unpack_bf16x8(dq[u], dv);
+                if (relu) unpack_bf16x8(oq[u], ov);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float d = (relu && !(ov[j] > 0.f)) ? 0.f : dv[j];
+                    dv[j] = fmaf(gi[j], d, fmaf(k1[j], xv[j], k0[j]));
+                }
+                dx4[i] = pack_bf16x8(dv);
+            }
+        }
+    }
+}
+
 int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void *x, const void *gamma,
                         const float *mean, const float *invstd, const float *dgamma, const float *dbeta, void *dx,
                         long npix, int C, int relu, cudaStream_t s) {
+    if (prec == P_BF16 && apply_fast_ok(C, Vec16<bf16>::N)) {
+        typedef bf16 T;
+        constexpr int V = Vec16<T>::N;
+        const long nvec = npix * (C / V);
+        const int U = apply_unroll(nvec) >= 2 ? 2 : 1;  // three operands: two vectors of each in flight per thread
+        auto k = U == 2 ? bn_bwd_apply_fast_kernel<2> : bn_bwd_apply_fast_kernel<1>;
+        launch_k(k, apply_grid(nvec, U), kThreads, 0, s, (const T *)dout, (const T *)out, (const T *)x, (const T *)gamma, mean,
+                 invstd, dgamma, dbeta, (T *)dx, nvec, npix, C, relu);
+        return 1;
+    }
     DISPATCH_PREC(prec, {
         constexpr int V = Vec16<T>::N;
         if (C % V == 0) {
@@ -629,68 +939,82 @@ int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void 
 // ------------------------------------------------------------------------------------------------------
 // optimiser update with the delayed gradient (Eq. 9 / Algorithm 1, Algorithm 2) + weight-version refresh
 // ------------------------------------------------------------------------------------------------------
+static constexpr int kUpdVecs = 2;  // float4 groups per thread, all loads issued before the first use
+
+// one parameter: master weight, first (and second) moment, gradient
+template <typename A>
+__device__ __forceinline__ void update_one(float &w, float &v, float &m2, float g, const UpdateArgs &a) {
+    if (a.mode == 0) {
+        const A d = (A)g + (A)a.wd * (A)w;
+        const A vn = (A)a.mu * (A)v + d;
+        v = (float)vn;
+        w = (float)((A)w - (A)a.lr * vn);
+    } else if (a.mode == 1) {
+        const A m1 = (A)a.b1 * (A)v + ((A)1 - (A)a.b1) * (A)g;
+        const A m2n = (A)a.b2 * (A)m2 + ((A)1 - (A)a.b2) * (A)g * (A)g;
+        v = (float)m1;
+        m2 = (float)m2n;
+        w = (float)((A)w - (A)a.lr * (m1 / (A)a.c1c) / (sqrt(m2n / (A)a.c2c) + (A)a.eps));
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 update_kernel(float *__restrict__ w, float *__restrict__ v, float *__restrict__ m2, const float *__restrict__ g,
               T *__restrict__ wv, size_t n, UpdateArgs a) {
     pdl_launch();
     pdl_wait();
-    size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-    if (i >= n) return;
-    const bool full = (i + 4 <= n) && ((reinterpret_cast<uintptr_t>(w + i) & 15) == 0) &&
-                      ((reinterpret_cast<uintptr_t>(v + i) & 15) == 0) &&
-                      ((reinterpret_cast<uintptr_t>(g + i) & 15) == 0) &&
-                      (a.mode != 1 || (reinterpret_cast<uintptr_t>(m2 + i) & 15) == 0);
-    const int cnt = (int)((n - i) < 4 ? (n - i) : 4);
-    float wv4[4], vv[4], gv[4], mv[4];
-    if (full) {
-        *reinterpret_cast<float4 *>(wv4) = *reinterpret_cast<const float4 *>(w + i);
-        if (a.mode != 2) {
-            *reinterpret_cast<float4 *>(vv) = *reinterpret_cast<const float4 *>(v + i);
-            *reinterpret_cast<float4 *>(gv) = *reinterpret_cast<const float4 *>(g + i);
-            if (a.mode == 1) *reinterpret_cast<float4 *>(mv) = *reinterpret_cast<const float4 *>(m2 + i);
-        }
-    } else {
-        for (int j = 0; j < cnt; ++j) {
-            wv4[j] = w[i + j];
-            if (a.mode != 2) { vv[j] = v[i + j]; gv[j] = g[i + j]; if (a.mode == 1) mv[j] = m2[i + j]; }
-        }
-    }
     typedef typename AccOf<T>::type A;  // the master state is fp32 either way; A is the arithmetic in between
-    if (a.mode == 0) {
+    const size_t span = (size_t)gridDim.x * blockDim.x * 4;  // elements one pass of the grid covers
+    const size_t base = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(g) |
+                           reinterpret_cast<uintptr_t>(m2) | (reinterpret_cast<uintptr_t>(wv) * (16 / (4 * sizeof(T))));
+    if ((bits & 15) == 0 && base + (kUpdVecs - 1) * span + 4 <= n) {
+        float4 W[kUpdVecs], V[kUpdVecs], G[kUpdVecs], M[kUpdVecs];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const A d = (A)gv[j] + (A)a.wd * (A)wv4[j];
-            const A vn = (A)a.mu * (A)vv[j] + d;
-            vv[j] = (float)vn;
-            wv4[j] = (float)((A)wv4[j] - (A)a.lr * vn);
+        for (int u = 0; u < kUpdVecs; ++u) {
+            const size_t i = base + u * span;
+            W[u] = *reinterpret_cast<const float4 *>(w + i);
+            if (a.mode != 2) {
+                V[u] = *reinterpret_cast<const float4 *>(v + i);
+                G[u] = *reinterpret_cast<const float4 *>(g + i);
+                if (a.mode == 1) M[u] = *reinterpret_cast<const float4 *>(m2 + i);
+            }
         }
-    } else if (a.mode == 1) {
 #pragma unroll
+        for (int u = 0; u < kUpdVecs; ++u) {
+            const size_t i = base + u * span;
+            update_one<A>(W[u].x, V[u].x, M[u].x, G[u].x, a);
+            update_one<A>(W[u].y, V[u].y, M[u].y, G[u].y, a);
+            update_one<A>(W[u].z, V[u].z, M[u].z, G[u].z, a);
+            update_one<A>(W[u].w, V[u].w, M[u].w, G[u].w, a);
+            if (a.mode != 2) {
+                *reinterpret_cast<float4 *>(w + i) = W[u];
+                *reinterpret_cast<float4 *>(v + i) = V[u];
+                if (a.mode == 1) *reinterpret_cast<float4 *>(m2 + i) = M[u];
+            }
+            const float o[4] = {W[u].x, W[u].y, W[u].z, W[u].w};
+            store_f<T, 4>(wv + i, o);
+        }
+        return;
+    }
+    for (int u = 0; u < kUpdVecs; ++u) {  // ragged end or unaligned arrays: element by element
         for (int j = 0; j < 4; ++j) {
-            const A m1 = (A)a.b1 * (A)vv[j] + ((A)1 - (A)a.b1) * (A)gv[j];
-            const A m2n = (A)a.b2 * (A)mv[j] + ((A)1 - (A)a.b2) * (A)gv[j] * (A)gv[j];
-            vv[j] = (float)m1;
-            mv[j] = (float)m2n;
-            wv4[j] = (float)((A)wv4[j] - (A)a.lr * (m1 / (A)a.c1c) / (sqrt(m2n / (A)a.c2c) + (A)a.eps));
+            const size_t i = base + u * span + j;
+            if (i >= n) break;
+            float wi = w[i], vi = 0.f, mi = 0.f, gi = 0.f;
+            if (a.mode != 2) { vi = v[i]; gi = g[i]; if (a.mode == 1) mi = m2[i]; }
+            update_one<A>(wi, vi, mi, gi, a);
+            if (a.mode != 2) { w[i] = wi; v[i] = vi; if (a.mode == 1) m2[i] = mi; }
+            wv[i] = from_f<T>(wi);
         }
     }
-    if (full) {
-        if (a.mode != 2) {
-            *reinterpret_cast<float4 *>(w + i) = *reinterpret_cast<const float4 *>(wv4);
-            *reinterpret_cast<float4 *>(v + i) = *reinterpret_cast<const float4 *>(vv);
-            if (a.mode == 1) *reinterpret_cast<float4 *>(m2 + i) = *reinterpret_cast<const float4 *>(mv);
-        }
-    } else if (a.mode != 2) {
-        for (int j = 0; j < cnt; ++j) { w[i + j] = wv4[j]; v[i + j] = vv[j]; if (a.mode == 1) m2[i + j] = mv[j]; }
-    }
-    for (int j = 0; j < cnt; ++j) wv[i + j] = from_f<T>(wv4[j]);
 }
 
 int launch_update(int prec, float *w, float *v, float *m2, const float *g, void *wv, size_t n, UpdateArgs a,
                   cudaStream_t s) {
     if (n == 0) return 0;
-    DISPATCH_PREC(prec, launch_k(update_kernel<T>, ceil_div((n + 3) / 4, kThreads), kThreads, 0, s, w, v, m2, g, (T *)wv, n, a));
+    DISPATCH_PREC(prec, launch_k(update_kernel<T>, ceil_div((n + 3) / 4, (long)kThreads * kUpdVecs), kThreads, 0, s, w, v, m2, g, (T *)wv, n, a));
     return 1;
 }
 

@@ -71,8 +71,40 @@ def test_conv3x3_fwd_dgrad_wgrad(shape, prec):
     assert torch.equal(dw, dw2)
 
 
+# enough tiles per CTA for the launch plans that large batches get (four epilogue groups, deep stage rings, chunked
+# weight gradient), with a ragged last wave
+@pytest.mark.parametrize("shape", [(301, 32, 32, 16, 16, 1), (231, 16, 16, 32, 32, 1), (902, 8, 8, 64, 64, 1)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_conv3x3_many_tiles(shape):
+    test_conv3x3_fwd_dgrad_wgrad(shape, 1)
+
+
+# The launch plan (pipelines per CTA, epilogue groups, stage ring) depends on the number of tiles, the arithmetic of
+# an output pixel does not: a batch of the kernel-sweep size must give, image for image, the bits that the same images
+# give in small batches (whose plan the oracle comparisons above cover).
+@pytest.mark.parametrize("shape", [(1024, 32, 32, 16), (1024, 16, 16, 32), (4096, 8, 8, 64)], ids=lambda s: "x".join(map(str, s)))
+def test_conv3x3_large_batch_equals_small_batches(shape):
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = shape
+    g = torch.Generator(device="cuda").manual_seed(17)
+    x = torch.randn(B, H, W, C, device="cuda", generator=g).to(torch.bfloat16)
+    w = (torch.randn(C, C, 3, 3, device="cuda", generator=g) * (2.0 / (9 * C)) ** 0.5).to(torch.bfloat16)
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    binding.conv3x3_fwd(1, x, w, y, B, H, W, C, C, 1)
+    binding.conv3x3_dgrad(1, x, w, dx, B, H, W, C, C, 1)
+    step = 64
+    for i in (0, B // 2, B - step):   # first, middle and last slice
+        ys, dxs = torch.empty_like(x[i:i + step]), torch.empty_like(x[i:i + step])
+        binding.conv3x3_fwd(1, x[i:i + step], w, ys, step, H, W, C, C, 1)
+        binding.conv3x3_dgrad(1, x[i:i + step], w, dxs, step, H, W, C, C, 1)
+        torch.cuda.synchronize()
+        assert torch.equal(ys, y[i:i + step]) and torch.equal(dxs, dx[i:i + step]), (shape, i)
+
+
 @pytest.mark.parametrize("prec", [0, 1], ids=["fp32", "bf16"])
-@pytest.mark.parametrize("shape", [(4, 64, 16), (7, 1024, 16), (33, 256, 32), (128, 64, 64), (3, 35, 12), (2, 3, 8)],
+# the last shape is large enough for the many-vectors-per-thread variants of the reductions and element-wise passes
+@pytest.mark.parametrize("shape", [(4, 64, 16), (7, 1024, 16), (33, 256, 32), (128, 64, 64), (3, 35, 12), (2, 3, 8),
+                                   (601, 1024, 16)],
                          ids=lambda s: "x".join(map(str, s)))
 @pytest.mark.parametrize("relu,res", [(0, 0), (1, 0), (1, 1)])
 def test_bn_fwd_bwd(shape, prec, relu, res):
