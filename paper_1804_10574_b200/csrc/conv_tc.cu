@@ -24,6 +24,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
 #include <map>
 #include <mutex>
 #include <tuple>
@@ -1256,23 +1257,30 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     if (32 % W != 0 || !get_map(src, B, H, W, C, box_rows, imgs, &map)) return -1;
     const int stage_bytes = box_rows * imgs * W * C * 2;
     const int n_tiles = (int)((long)B * H * W / kTileM);
-    const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
+    const int sms = g_num_sms;
     // Pipelines per CTA and epilogue plan.
-    //   C = 16 (one 16-channel chunk per tile): two pipelines where a CTA has at least four tiles, four where it has at
+    //   C = 16 (one 16-channel chunk per tile): two pipelines where an SM has at least four tiles, four where it has at
     //   least sixteen (large batches); below that one pipeline whose two epilogue groups take alternate tiles.
-    //   C >= 32: the two groups of a pipeline halve every tile, which shortens the epilogue of CTAs with one or two tiles
-    //   (the training step's sizes); two pipelines where a CTA has at least three tiles.
-    // A CTA with a single tile uses one accumulator: half the TMEM columns, so that CTAs of other streams fit beside it.
+    //   C >= 32: one pipeline whose two groups halve every tile where an SM has a single tile (shorter epilogue); for
+    //   C = 32 two pipelines with one group each where it has two (both tiles side by side; C = 64 would need all 512
+    //   TMEM columns for that); two pipelines with two groups each where it has three or more.
+    // A pipeline with a single tile uses one accumulator: fewer TMEM columns, so that CTAs of other streams fit beside it.
     EpiPlan ep;
     if (C == 16) {
-        const int P = !slab ? 1 : (n_tiles >= 16 * grid ? 4 : (n_tiles >= 4 * grid ? 2 : 1));
-        const int n_acc = P > 1 ? 1 : (n_tiles <= grid ? 1 : 2);
+        const int P = !slab ? 1 : (n_tiles >= 16 * sms ? 4 : (n_tiles >= 4 * sms ? 2 : 1));
+        const int n_acc = P > 1 ? 1 : (n_tiles <= sms ? 1 : 2);
         ep = EpiPlan{P, n_acc, n_acc, 1};
+    } else if (n_tiles >= 3 * sms) {
+        ep = EpiPlan{2, C == 64 ? 1 : 2, 1, 2};  // 2 x 2 x 192 columns would not fit
+    } else if (C == 32 && n_tiles > sms) {
+        ep = EpiPlan{2, 1, 1, 1};
     } else {
-        const int P = n_tiles >= 3 * grid ? 2 : 1;
-        const int n_acc = n_tiles <= grid ? 1 : ((P == 2 && C == 64) ? 1 : 2);  // 2 x 2 x 192 columns would not fit
-        ep = EpiPlan{P, n_acc, 1, 2};
+        ep = EpiPlan{1, n_tiles <= sms ? 1 : 2, 1, 2};
     }
+    // as few CTAs as give every pipeline the same number of tiles as a full grid would give the busiest one: the kernel
+    // takes as long, and the SMs left over are free for the other streams
+    const int per_pipe = (n_tiles + sms * ep.n_pipes - 1) / (sms * ep.n_pipes);
+    const int grid = (n_tiles + per_pipe * ep.n_pipes - 1) / (per_pipe * ep.n_pipes);
     const int groups = ep.n_pipes * ep.n_slots * ep.split;
     const int threads = 32 * (2 * ep.n_pipes + 4 * (groups < 2 ? 2 : groups));
     // CTAs with many tiles take the whole SM's shared memory for the stage ring; the others about half of it
