@@ -88,6 +88,26 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// one 32-byte store (16 bf16 channels of a pixel): every 32-byte sector of the output is written whole, by one request
+__device__ __forceinline__ void st_global_32(void *p, const uint32_t (&v)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+
+// the matching 32-byte load, unpacked to 16 floats
+__device__ __forceinline__ void ld_global_32(const bf16 *p, float (&f)[16]) {
+    uint32_t v[8];
+    asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "l"(p));
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        f[2 * k] = __uint_as_float(v[k] << 16);
+        f[2 * k + 1] = __uint_as_float(v[k] & 0xffff0000u);
+    }
+}
+
 __device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -477,21 +497,20 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                     acc[j] = p1[j] + (wcol > 0 ? left : 0.f) + (wcol < W - 1 ? right : 0.f);
                 }
                 if (res_dout != nullptr) {  // identity-shortcut gradient: + dout * [out > 0]
+                    float d[16], o[16];
+                    ld_global_32(res_dout + pix * C + c0, d);
+                    ld_global_32(res_out + pix * C + c0, o);
 #pragma unroll
-                    for (int h = 0; h < 16; h += 8) {
-                        float d[8], o[8];
-                        load_f<bf16, 8>(res_dout + pix * C + c0 + h, d);
-                        load_f<bf16, 8>(res_out + pix * C + c0 + h, o);
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) if (o[j] > 0.f) acc[h + j] += d[j];
-                    }
+                    for (int j = 0; j < 16; ++j) if (o[j] > 0.f) acc[j] += d[j];
                 }
+                {
+                    uint32_t pk[8];
 #pragma unroll
-                for (int h = 0; h < 16; h += 8) {
-                    float v[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[j] = acc[h + j];
-                    store_f<bf16, 8>(dst + pix * C + c0 + h, v);
+                    for (int j = 0; j < 8; ++j) {
+                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[2 * j], acc[2 * j + 1]);
+                        pk[j] = *reinterpret_cast<const uint32_t *>(&b2);
+                    }
+                    st_global_32(dst + pix * C + c0, pk);
                 }
                 if (stat_part != nullptr) {
                     float v[32];
@@ -503,18 +522,15 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                             v[16 + j] = r * r;
                         }
                     } else {
+                        float mk[16], xv[16];
+                        ld_global_32(bn_mask + pix * C + c0, mk);
+                        ld_global_32(bn_x + pix * C + c0, xv);
 #pragma unroll
-                        for (int h = 0; h < 16; h += 8) {
-                            float mk[8], xv[8];
-                            load_f<bf16, 8>(bn_mask + pix * C + c0 + h, mk);
-                            load_f<bf16, 8>(bn_x + pix * C + c0 + h, xv);
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                float d = __bfloat162float(__float2bfloat16_rn(acc[h + j]));
-                                if (!(mk[j] > 0.f)) d = 0.f;
-                                v[h + j] = d;
-                                v[16 + h + j] = d * (xv[j] - sm_stat[c0 + h + j]) * sm_stat[C + c0 + h + j];
-                            }
+                        for (int j = 0; j < 16; ++j) {
+                            float d = __bfloat162float(__float2bfloat16_rn(acc[j]));
+                            if (!(mk[j] > 0.f)) d = 0.f;
+                            v[j] = d;
+                            v[16 + j] = d * (xv[j] - sm_stat[c0 + j]) * sm_stat[C + c0 + j];
                         }
                     }
                     warp_transpose_sum32(v, lane);
