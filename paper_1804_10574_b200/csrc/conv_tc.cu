@@ -1257,9 +1257,10 @@ bool get_map_s2(const void *ptr, int B, int H, int W, int C, int rows, int imgs,
 }
 
 int g_num_sms = 148;
-// Shared memory a CTA may take for its pipeline stages: about half an SM, so that kernels of two modules (streams) can
-// share an SM instead of queueing behind each other.
-constexpr int kSmemBudget = 100 * 1024;
+// Shared memory a CTA may take for its pipeline stages: less than half an SM, so that kernels of two modules (streams)
+// can share an SM instead of queueing behind each other (K = 4 step, ms per iteration at 56 / 64 / 72 / 80 / 100 / 128
+// KB: 1.870 / 1.884 / 1.844 / 1.844 - 1.857 / 1.874 / 2.068).
+constexpr int kSmemBudget = 80 * 1024;
 constexpr int kSmemMax = 227 * 1024;
 
 template <int C>
@@ -1325,7 +1326,12 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     if (!get_map(x, B, H, W, C, slab ? rows + 2 : rows, imgs, &mx) || !get_map(dy, B, H, W, C, rows, imgs, &md)) return -1;
     const int x_box_bytes = (slab ? rows + 2 : rows) * imgs * W * C * 2;
     const int stage_bytes = TcCfg<C>::tile_bytes + 3 * x_box_bytes;
-    int n_stages = kSmemBudget / stage_bytes;
+    const int n_tiles_all = (int)((long)B * H * W / kTileM);
+    // many tiles per CTA (large batches): the whole SM's shared memory for the stage ring, so that the loads of the next
+    // tiles are in flight while this one is multiplied (batch 4096: 72 -> 68 us at 32 channels, 53 -> 44 us at 64);
+    // otherwise the half-SM budget: taking more in the training step cost 4 % of the K = 4 iteration
+    const int budget = n_tiles_all >= 8 * g_num_sms ? kSmemMax - 2048 - (C == 32 ? 4096 : 0) : kSmemBudget;
+    int n_stages = budget / stage_bytes;
     if (n_stages > kMaxStages) n_stages = kMaxStages;
     if (n_stages < 2) n_stages = 2;
     // slab mode with narrow channels: all nine taps from one instruction per 16 pixels when the three column boxes

@@ -784,7 +784,10 @@ static int apply_unroll(long nvec) {
 }
 static int apply_grid(long nvec, int U) {
     long g = (nvec + (long)kThreads * U - 1) / ((long)kThreads * U);
-    if (g > 148L * kApplyCtasPerSm) g = 148L * kApplyCtasPerSm;
+    // tensors of the training step's size: two CTAs per SM, which leaves registers for a convolution CTA of another
+    // stream beside them (K = 4 step 0.8 % faster than with three); large tensors: three, for the loads in flight
+    const int cap = U == 4 ? kApplyCtasPerSm : 2;
+    if (g > 148L * cap) g = 148L * cap;
     return (int)(g < 1 ? 1 : g);
 }
 
