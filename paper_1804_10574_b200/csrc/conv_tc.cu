@@ -1294,10 +1294,13 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     } else {
         ep = EpiPlan{1, n_tiles <= sms ? 1 : 2, 1, 2};
     }
-    // as few CTAs as give every pipeline the same number of tiles as a full grid would give the busiest one: the kernel
-    // takes as long, and the SMs left over are free for the other streams
+    // Several module streams: as few CTAs as give every pipeline the same number of tiles as a full grid would give the
+    // busiest one; the kernel's critical path is as long, and the SMs left over are free for the other streams (K = 4
+    // step -2 %).  A kernel that has the GPU to itself takes every SM (a few pipelines then finish early).
     const int per_pipe = (n_tiles + sms * ep.n_pipes - 1) / (sms * ep.n_pipes);
-    const int grid = (n_tiles + per_pipe * ep.n_pipes - 1) / (per_pipe * ep.n_pipes);
+    const int balanced = (n_tiles + per_pipe * ep.n_pipes - 1) / (per_pipe * ep.n_pipes);
+    const int full = (n_tiles + ep.n_pipes - 1) / ep.n_pipes < sms ? (n_tiles + ep.n_pipes - 1) / ep.n_pipes : sms;
+    const int grid = gpu_shared_by_streams() ? balanced : full;
     const int groups = ep.n_pipes * ep.n_slots * ep.split;
     const int threads = 32 * (2 * ep.n_pipes + 4 * (groups < 2 ? 2 : groups));
     // CTAs with many tiles take the whole SM's shared memory for the stage ring; the others about half of it

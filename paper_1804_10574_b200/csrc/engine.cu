@@ -578,6 +578,9 @@ bool pdl_enabled() {
     static const int forced = [] { const char *e = getenv("DDG_PDL"); return e ? (e[0] == '0' ? 0 : 1) : -1; }();
     return forced >= 0 ? forced == 1 : t_pdl_wanted;
 }
+// True while the engine enqueues an iteration of a multi-module network: the launchers then size grids so that SMs are
+// left over for the other modules' kernels where that costs the kernel itself nothing.
+bool gpu_shared_by_streams() { return !t_pdl_wanted; }
 // lets the other translation units leave a message for ddg_last_error(NULL)
 void set_global_error(const char *msg) { g_create_error = msg; }
 }  // namespace ddg
