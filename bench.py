@@ -114,17 +114,26 @@ def time_oracle(cfg, batch, n_steps):
 
 
 def _time_back_to_back(torch, launches, stream, reps=5):
-    """Average duration of one launch when `launches` (callables on distinct buffers, together larger than L2) run
-    back to back on `stream`, as the kernels of a training step do: CUDA events around the whole sequence."""
+    """Average device time of one launch when `launches` (callables on distinct buffers, together larger than L2) run
+    back to back, as the kernels of a training step do.  The sequence is recorded once into a CUDA graph on a side
+    stream and replayed (the step replays graphs too): enqueueing one launch at a time from Python takes longer than
+    a launch runs, which would time the interpreter instead of the kernels.  CUDA events around each replay."""
+    side = torch.cuda.Stream()
     for fn in launches[:3]:
-        fn()
+        fn(stream.cuda_stream)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for fn in launches:
+            fn(side.cuda_stream)
+    for _ in range(2):
+        graph.replay()
     torch.cuda.synchronize()
     ts = []
     for _ in range(reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for fn in launches:
-            fn()
+        graph.replay()
         e1.record(stream)
         e1.synchronize()
         ts.append(e0.elapsed_time(e1) * 1e-3 / len(launches))
@@ -135,7 +144,7 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
     """The kernel with the largest share of the ncu launch list of this workload is the tensor-core convolution on the
     16-channel 32x32 maps, conv3x3_tc_kernel<16> (profiles/ddg_step_resnet110_k4_b128_bf16_launch_list.md).  It is
     timed here at the step's shape and launch configuration, with its pre-arranged filter image, as a sequence of
-    launches on distinct tensors (more than L2 in total) between two CUDA events on its stream.  The other
+    launches on distinct tensors (more than L2 in total), replayed as one CUDA graph between two CUDA events.  The other
     convolution widths and the batch-norm backward pass are timed the same way and listed beside it."""
     B = cfg["batch"]
     bf = torch.bfloat16
@@ -152,7 +161,7 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
         w = (torch.randn(Cc, Cc, 3, 3, device="cuda") * (2.0 / (9 * Cc)) ** 0.5).to(bf)
         pk = torch.empty(binding.conv3x3_packed_bytes(B, Hh, Hh, Cc), dtype=torch.uint8, device="cuda")
         binding.conv3x3_pack(w, pk, Cc)
-        fns = [(lambda i=i: binding.conv3x3_packed(0, xs[i], w, pk, ys[i], B, Hh, Hh, Cc, s.cuda_stream)) for i in range(n)]
+        fns = [(lambda st, i=i: binding.conv3x3_packed(0, xs[i], w, pk, ys[i], B, Hh, Hh, Cc, st)) for i in range(n)]
         dt = _time_back_to_back(torch, fns, s)
         return dt, per + w.numel() * 2, 2.0 * 9 * Cc * Cc * B * Hh * Hh, n
 
@@ -182,8 +191,8 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
     mean, invstd = torch.zeros(C, device="cuda"), torch.ones(C, device="cuda")
     dg, db = torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
     scr = torch.zeros(binding.bn_scratch_elems(C), device="cuda")
-    fns = [(lambda i=i: binding.bn_bwd(1, douts[i], xs[i], xs[i], g, mean, invstd, dxs[i], dg, db, scr, B, H * H, C, 1,
-                                       s.cuda_stream)) for i in range(n)]
+    fns = [(lambda st, i=i: binding.bn_bwd(1, douts[i], xs[i], xs[i], g, mean, invstd, dxs[i], dg, db, scr, B, H * H, C, 1,
+                                           st)) for i in range(n)]
     dtb = _time_back_to_back(torch, fns, s)
     nb = 7 * B * H * H * C * 2                               # sums read dout, out, x; the element-wise pass reads them again, writes dx
     others.append({"kernel": "bn_reduce_fast_kernel + bn_bwd_apply_fast_kernel (batch-norm backward) C=16 32x32 B=%d" % B,
