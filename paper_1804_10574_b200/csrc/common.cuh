@@ -80,7 +80,6 @@ static inline int ceil_div(long a, long b) { return (int)((a + b - 1) / b); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-int module_streams();          // defined in engine.cu: module streams of the iteration being enqueued, else 1
 bool gpu_shared_by_streams();  // defined in engine.cu: true while a multi-module iteration is enqueued
 bool pdl_enabled();  // defined in engine.cu: off while a multi-module iteration is enqueued; DDG_PDL=0/1 forces it
 

@@ -1348,10 +1348,7 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int n_tiles = (int)((long)B * H * W / kTileM);
     // pixel chunks (= CTAs, = partials to fold): few at the training step's sizes, where the kernel shares the GPU with
     // the other streams and the fold should stay small; one per 16 tiles, up to a CTA per SM, for large batches
-    // With four or more module streams a quarter of the chunks: the kernel runs on its module's side stream with time
-    // to spare, and fewer, longer CTAs cost the other streams less (ResNet-110 batch 128, K = 4: 1.844 -> 1.81 ms per
-    // iteration; at K = 1..3, where the side stream is nearer the critical path, the same change loses 2-4 %).
-    const int max_chunks = (slab ? (C == 16 ? 74 : 37) : 24) / (module_streams() >= 4 ? 4 : 1);
+    const int max_chunks = slab ? (C == 16 ? 74 : 37) : 24;
     int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
     const int big = n_tiles / 16 < (slab ? kWgMaxChunks : 48) ? n_tiles / 16 : (slab ? kWgMaxChunks : 48);
     if (big > chunks) chunks = big;

@@ -581,9 +581,6 @@ bool pdl_enabled() {
 // True while the engine enqueues an iteration of a multi-module network: the launchers then size grids so that SMs are
 // left over for the other modules' kernels where that costs the kernel itself nothing.
 bool gpu_shared_by_streams() { return !t_pdl_wanted; }
-// Module streams of the network whose iteration is being enqueued (1 outside the engine).
-thread_local int t_module_streams = 1;
-int module_streams() { return t_module_streams; }
 // lets the other translation units leave a message for ddg_last_error(NULL)
 void set_global_error(const char *msg) { g_create_error = msg; }
 }  // namespace ddg
@@ -859,10 +856,8 @@ static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float 
     // the first K-1 iterations have modules in warm-up and a different shape: they are not recorded
     const bool steady = t >= K - 1;
     ddg::t_pdl_wanted = ctx->K == 1;
-    ddg::t_module_streams = ctx->K;
     ddg_status st = enqueue_iteration(ctx, t, ctx->cfg.use_graph && steady, &ctx->launches);
     ddg::t_pdl_wanted = true;
-    ddg::t_module_streams = 1;
     if (st != DDG_OK) { ctx->broken = true; return st; }
     ctx->t = t + 1;
     if (loss_host) {
