@@ -167,12 +167,12 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
 
     dt, alg, flops, n = conv_case(32, 16)
     # DRAM traffic per launch from the ncu capture at batch 4096 (profiles/conv3x3_tc_kernel_c16_fwd_b4096_ncu_full.md):
-    # 134.3 MB read + 82.6 MB written for 268.4 MB algorithmic (part of the output is still in L2 when the kernel
+    # 134.3 MB read + 88.5 MB written for 268.4 MB algorithmic (part of the output is still in L2 when the kernel
     # ends); traffic grows with the pixels processed, so it is scaled by batch
-    traffic = 216.9e6 * B / 4096.0
+    traffic = 222.8e6 * B / 4096.0
     roof = {"kernel": "conv3x3_tc_kernel<16> (tensor-core 3x3 convolution, forward) C=16 32x32 B=%d" % B, "bound": "hbm",
             "achieved": alg / dt / 1e9, "peak": hbm, "unit": "GB/s", "frac": alg / dt / 1e9 / hbm, "traffic": traffic,
-            "launch_us": dt * 1e6, "peak_source": src, "ncu_share_of_step": 0.190, "launches_timed": n,
+            "launch_us": dt * 1e6, "peak_source": src, "ncu_share_of_step": 0.187, "launches_timed": n,
             "tflops": flops / dt / 1e12, "tensor_frac": flops / dt / 1e12 / tflops}
     others = []
     for (Hh, Cc) in ((16, 32), (8, 64)):
