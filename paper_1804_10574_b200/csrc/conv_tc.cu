@@ -1506,6 +1506,10 @@ int conv_tc_error() {
     return v;
 }
 
+int conv_tc_error_async(int *pinned_dst, cudaStream_t s) {
+    return cudaMemcpyFromSymbolAsync(pinned_dst, g_tc_error, sizeof(int), 0, cudaMemcpyDeviceToHost, s) == cudaSuccess ? 0 : -1;
+}
+
 int conv_tc_init() {
     static int rc = -1;
     if (rc >= 0) return rc;

@@ -59,6 +59,8 @@ int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, in
 int conv_tc_init();
 // Error word raised by a tensor-core kernel whose bounded wait ran out (0 = none, -1 = cannot be read).
 int conv_tc_error();
+// the same word copied into pinned host memory on a stream (0 on success); the caller synchronises the stream
+int conv_tc_error_async(int *pinned_dst, cudaStream_t s);
 int conv_direct_init();
 
 }  // namespace ddg

@@ -834,7 +834,7 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
     CU(cudaMalloc(&c->dlogits, (size_t)c->B * c->classes * 4));
     CU(cudaMalloc(&c->loss_dev, 4));
     CU(cudaMemset(c->loss_dev, 0, 4));
-    CU(cudaMallocHost(&c->pinned_loss, 4));
+    CU(cudaMallocHost(&c->pinned_loss, 8));  // the loss, and the tensor-core kernels' error word read with it
     CU(cudaStreamCreateWithFlags(&c->loss_stream, cudaStreamNonBlocking));
     // the memsets above ran on the legacy default stream, which the non-blocking module streams do not wait for
     CU(cudaDeviceSynchronize());
@@ -865,10 +865,17 @@ static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float 
         // updates of this iteration stay in flight and overlap the caller's next step (the decoupling DDG is about).
         CU(cudaStreamWaitEvent(ctx->loss_stream, ctx->mods[K - 1].ev_fwd, 0));
         CU(cudaMemcpyAsync(ctx->pinned_loss, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, ctx->loss_stream));
+        // error flags raised so far ride along (a later call or ddg_sync reports what is still running): one host wait
+        int *flag = reinterpret_cast<int *>(ctx->pinned_loss + 1);
+        *flag = 0;
+        if (ctx->prec == P_BF16 && conv_tc_error_async(flag, ctx->loss_stream) != 0) return DDG_ERR_CUDA;
         CU(cudaStreamSynchronize(ctx->loss_stream));
         *loss_host = *ctx->pinned_loss;
-        st = check_kernel_errors(ctx);  // flags raised so far; a later call or ddg_sync reports what is still running
-        if (st != DDG_OK) return st;
+        if (*flag != 0) {
+            set_err(ctx, "a tensor-core kernel gave up on a bounded wait (code %d)", *flag);
+            ctx->broken = true;
+            return DDG_ERR_TIMEOUT;
+        }
     }
     return DDG_OK;
 }
