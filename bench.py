@@ -153,9 +153,9 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
     tflops = peaks.get("bf16_tflops", 1590.0)
     src = "measured" if "hbm_gbs" in peaks else "fallback"
 
-    def conv_case(Hh, Cc):
+    def conv_case(Hh, Cc, B=B):
         per = 2 * B * Hh * Hh * Cc * 2                       # bytes of input + output of one launch
-        n = max(8, int(400e6 // per) + 1)
+        n = max(8, int(400e6 // per) + 1) if B <= 1024 else max(2, int(400e6 // per) + 1)
         xs = [torch.randn(B, Hh, Hh, Cc, device="cuda").to(bf) for _ in range(n)]
         ys = [torch.empty_like(xs[0]) for _ in range(n)]
         w = (torch.randn(Cc, Cc, 3, 3, device="cuda") * (2.0 / (9 * Cc)) ** 0.5).to(bf)
@@ -180,6 +180,13 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
         others.append({"kernel": "conv3x3_tc_kernel<%d> fwd %dx%d B=%d" % (Cc, Hh, Hh, B), "launch_us": dtc * 1e6,
                        "hbm_gbs": nbytes / dtc / 1e9, "hbm_frac": nbytes / dtc / 1e9 / hbm, "tflops": fl / dtc / 1e12,
                        "tensor_frac": fl / dtc / 1e12 / tflops})
+    # the same kernels at the kernel-sweep size, where a launch moves enough data for bandwidth to matter
+    for (Hh, Cc) in ((32, 16), (16, 32), (8, 64)):
+        dtc, nbytes, fl, _ = conv_case(Hh, Cc, 4096)
+        others.append({"kernel": "conv3x3_tc_kernel<%d> fwd %dx%d B=4096 (kernel-sweep size)" % (Cc, Hh, Hh),
+                       "launch_us": dtc * 1e6, "hbm_gbs": nbytes / dtc / 1e9, "hbm_frac": nbytes / dtc / 1e9 / hbm,
+                       "tflops": fl / dtc / 1e12, "tensor_frac": fl / dtc / 1e12 / tflops})
+    torch.cuda.empty_cache()
     # batch-norm backward (sums + element-wise pass) on the largest map
     H, C = 32, 16
     per = 4 * B * H * H * C * 2
