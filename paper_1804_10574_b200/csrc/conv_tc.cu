@@ -8,7 +8,7 @@
 // One CTA tile is 128 consecutive output pixels (whole image rows) x C channels.  The input rows are loaded ONCE per
 // tile, unshifted in the column direction: the MMAs produce, per filter column kx, the partial result
 // P_kx[p][co] = sum_{ky,ci} x[p + (ky-1) rows][ci] * w[co][ci][ky][kx] at the INPUT column (UMMA M=128, N=3C, K=16 per
-// instruction, the three filter columns stacked along N), and the epilogue adds the three partials across
+// instruction, the three filter columns stacked along N, chunk of 16 output channels by chunk), and the epilogue adds the three partials across
 // neighbouring pixels, y[h][w] = P_0[h][w-1] + P_1[h][w] + P_2[h][w+1], with warp shuffles (a warp holds whole image
 // rows; the image border contributes zero).  The filter-row shift costs nothing: the three rows read the same TMA box
 // at offsets of 0, W and 2W pixels, which are whole swizzle periods, so only the descriptor start address moves.
@@ -138,6 +138,20 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 32 consecutive columns into two 16-value halves (one instruction: issuing a tcgen05.ld costs its warp ~70 ns)
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&a)[16], float (&b)[16]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { a[i] = __uint_as_float(r[i]); b[i] = __uint_as_float(r[16 + i]); }
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major (or MN-major) bf16 tile whose rows are one swizzle span wide
@@ -160,7 +174,7 @@ template <int C> struct TcCfg {
     static constexpr int row_bytes = C * 2;                           // one pixel's channels = one swizzle span
     static constexpr uint32_t layout = C == 64 ? 2u : (C == 32 ? 4u : 6u);  // 128B / 64B / 32B swizzle
     static constexpr uint32_t swz_mask = C == 64 ? 7u : (C == 32 ? 3u : 1u);
-    static constexpr int w_row_tile_bytes = 3 * C * C * 2;            // one filter row: [3C rows = (kx, out ch)][C]
+    static constexpr int w_row_tile_bytes = 3 * C * C * 2;            // one filter row: [3C rows = (chunk, kx, out ch % 16)][C]
     static constexpr int w_bytes = 3 * w_row_tile_bytes;
     static constexpr int tile_bytes = kTileM * C * 2;
     static constexpr int acc_stages = 2;                              // TMEM accumulator stages of 3C columns each
@@ -218,9 +232,11 @@ __device__ __forceinline__ void warp_transpose_sum32(float (&v)[32], int lane) {
 // flipped).  One thread per (tap, row, k).
 struct PackJob { long src_off; long dst_off; int C; int first_elem; int cin_real; int pad_; };
 
-// image element (tap = ky*3+kx, row r, k): filter row tile ky, row kx*C + r of that tile
+// image element (tap = ky*3+kx, row r, k): filter row tile ky; within it the rows (= accumulator columns) are ordered
+// (16-channel chunk of r, kx, r mod 16), so that the three filter-column partials of a chunk are 48 consecutive
+// accumulator columns and the epilogue fetches them with two TMEM loads
 template <int C> __device__ __forceinline__ uint32_t w_img_off(int tap, int r, int k) {
-    return (uint32_t)(tap / 3) * TcCfg<C>::w_row_tile_bytes + swz_off<C>((tap % 3) * C + r, k);
+    return (uint32_t)(tap / 3) * TcCfg<C>::w_row_tile_bytes + swz_off<C>((r >> 4) * 48 + (tap % 3) * 16 + (r & 15), k);
 }
 // cin: input channels the canonical filter really has; channels cin..C-1 of the images are zero (a first layer whose
 // input was zero-padded to C channels)
@@ -482,9 +498,9 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
 #pragma unroll 1
             for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 float p0[16], p1[16], p2[16];
-                tc_ld16(t_row + (uint32_t)c0, p0);            // filter column 0: belongs to the pixel on the right
-                tc_ld16(t_row + (uint32_t)(C + c0), p1);
-                tc_ld16(t_row + (uint32_t)(2 * C + c0), p2);  // filter column 2: belongs to the pixel on the left
+                // p0: filter column 0, belongs to the pixel on the right; p2: filter column 2, to the pixel on the left
+                tc_ld32(t_row + (uint32_t)(3 * c0), p0, p1);  // the chunk's three pieces are 48 consecutive columns
+                tc_ld16(t_row + (uint32_t)(3 * c0) + 32u, p2);
                 tc_wait_ld();
                 if (c0 + 16 >= c_end) {  // this group's last read of the accumulator: hand it back to the MMA warp
                     tc_fence_before();
