@@ -35,7 +35,8 @@ def parse():
     p.add_argument("--batch", type=int, default=0)
     p.add_argument("--no-graph", action="store_true")
     p.add_argument("--cpu-batch", type=int, default=8, help="batch of the bounded CPU-oracle sample")
-    p.add_argument("--cpu-steps", type=int, default=0, help="timed oracle steps (0 = K+1)")
+    p.add_argument("--cpu-steps", type=int, default=0, help="timed oracle iterations (0 = 20 beside the GPU arm; "
+                   "min(--steps, 100) for --impl reference)")
     p.add_argument("--skip-cpu", action="store_true")
     return p.parse_args()
 
@@ -235,7 +236,9 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return 0
-        n = args.cpu_steps or min(max(args.steps, 1), 2)
+        # a step of this arm = one oracle iteration on the bounded sample (batch 8 of 128, ~0.55 s on 16 cores); the
+        # requested steps are honoured up to 100, so that the run ends within a minute or two
+        n = args.cpu_steps or min(max(args.steps, 1), 100)
         times = [time_oracle(cfg, args.cpu_batch, 1) for _ in range(min(args.warmup, 1))]   # one warm-up sample
         r = time_oracle(cfg, args.cpu_batch, n)
         out = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": "images/s", "n_gpus": 0,
@@ -316,7 +319,7 @@ def main():
         roof, roof_others = dominant_kernel_roofline(torch, binding, cfg, peaks)
         cpu = None
         if world == 1 and not args.skip_cpu:
-            r = time_oracle(cfg, args.cpu_batch, args.cpu_steps or 2)
+            r = time_oracle(cfg, args.cpu_batch, args.cpu_steps or 20)   # ~10 s of host work
             cpu = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
         x_bytes = int(np.prod((cfg["batch"],) + tuple(cfg["in_shape"]))) * 4
         out = {"metric": METRIC, "value": job_throughput(cfg["batch"], args.steps, world, dt), "unit": "images/s", "n_gpus": world, "steps": args.steps,
