@@ -81,10 +81,14 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 bool gpu_shared_by_streams();  // defined in engine.cu: true while a multi-module iteration is enqueued
-bool pdl_enabled();  // defined in engine.cu: off while a multi-module iteration is enqueued; DDG_PDL=0/1 forces it
+// defined in engine.cu.  While a multi-module iteration is enqueued only launches that ask with `while_shared` get the
+// attribute (the tensor-core convolution: see there); DDG_PDL=0/1 in the environment forces it off / on for all
+bool pdl_enabled(bool while_shared = false);
 
+// pdl_while_shared: the launch carries the programmatic attribute also while several module streams share the GPU
 template <typename... KArgs, typename... Args>
-inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
+inline void launch_kp(bool pdl_while_shared, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                      Args &&...args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -94,8 +98,12 @@ inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cfg.numAttrs = pdl_enabled(pdl_while_shared) ? 1 : 0;
     cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
+    launch_kp(false, kernel, grid, block, smem, stream, std::forward<Args>(args)...);
 }
 
 }  // namespace ddg

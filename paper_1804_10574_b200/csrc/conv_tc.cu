@@ -1332,7 +1332,7 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     int tmem_cols = 32;
     while (tmem_cols < acc_cols) tmem_cols <<= 1;
     if (tmem_cols > 512 || conv_smem_bytes<C>(n_stages, stage_bytes) > (size_t)kSmemMax) return -1;
-    launch_k(conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
+    launch_kp(true, conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
         stage_bytes, tmem_cols, ep, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
         bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd);
     return 1;

@@ -567,16 +567,19 @@ ddg_status sync_all(ddg_ctx *ctx) {
 }  // namespace
 
 namespace ddg {
-// Programmatic dependent launch pays where one stream has the GPU to itself (K = 1, single kernels): the next
-// kernel's launch latency hides under the running one.  With several module streams it loses: a kernel that was
-// placed early holds its shared memory, TMEM columns and registers while it waits for its predecessor, and keeps the
-// other modules' CTAs off the SM (measured on ResNet-110, K = 4: 2.13 ms per iteration with, 1.99 ms without).  The
-// engine therefore clears this flag while it enqueues an iteration of a multi-module network.  DDG_PDL=0 / 1 in the
-// environment forces the launch attribute off / on.
+// Programmatic dependent launch: the next kernel of a stream is placed while this one still runs, so that its launch
+// latency and set-up hide under this one's tail.  Where one stream has the GPU to itself (K = 1, single kernels) every
+// launch carries the attribute.  With several module streams it depends on what the early-placed kernel holds while
+// it waits: the element-wise batch-norm passes (three CTAs of 256 threads and ~70 registers per SM, all SMs) keep the
+// other modules' tensor-core CTAs off the SMs, and the attribute on them alone costs the K = 4 iteration 15 % (1.82 ->
+// 2.10 ms, ResNet-110 batch 128); on the weight-gradient kernel and its fold, which run on side streams, 1 - 5 %.  On
+// the forward / input-gradient convolution alone it gains 5 % (1.82 -> 1.73 ms; end to end 53 400 -> 57 500 images/s).
+// So the engine clears the flag below while it enqueues an iteration of a multi-module network, and only launches that
+// pass `while_shared` (that convolution) keep the attribute then.  DDG_PDL=0 / 1 in the environment forces it off / on.
 thread_local bool t_pdl_wanted = true;
-bool pdl_enabled() {
+bool pdl_enabled(bool while_shared) {
     static const int forced = [] { const char *e = getenv("DDG_PDL"); return e ? (e[0] == '0' ? 0 : 1) : -1; }();
-    return forced >= 0 ? forced == 1 : t_pdl_wanted;
+    return forced >= 0 ? forced == 1 : (t_pdl_wanted || while_shared);
 }
 // True while the engine enqueues an iteration of a multi-module network: the launchers then size grids so that SMs are
 // left over for the other modules' kernels where that costs the kernel itself nothing.
