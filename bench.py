@@ -38,6 +38,7 @@ def parse():
     p.add_argument("--cpu-steps", type=int, default=0, help="timed oracle iterations (0 = 20 beside the GPU arm; "
                    "min(--steps, 100) for --impl reference)")
     p.add_argument("--skip-cpu", action="store_true")
+    p.add_argument("--skip-k1", action="store_true", help="leave out the K = 1 arm")
     return p.parse_args()
 
 
@@ -141,6 +142,27 @@ def _time_back_to_back(torch, launches, stream, reps=5):
     return float(np.median(ts))
 
 
+def ncu_counters():
+    """Figures copied from the ncu summaries under profiles/ (DRAM bytes of the dominant kernel, its share of the
+    launch list), kept in profiles/roofline_counters.json beside the summaries they come from.  Each entry names the
+    source file of its kernel with the hash that file had when the counters were taken: a kernel that has changed
+    since has no valid counters, and its figure is reported as null."""
+    import hashlib
+    try:
+        doc = json.load(open(os.path.join(ROOT, "profiles", "roofline_counters.json")))
+    except Exception:
+        return {}
+    out = {}
+    for name, ent in doc.items():
+        try:
+            src = open(os.path.join(ROOT, ent["kernel_source"]), "rb").read()
+            ent = dict(ent, valid=hashlib.sha256(src).hexdigest() == ent["kernel_source_sha256"])
+        except Exception:
+            ent = dict(ent, valid=False)
+        out[name] = ent
+    return out
+
+
 def dominant_kernel_roofline(torch, binding, cfg, peaks):
     """The kernel with the largest share of the ncu launch list of this workload is the tensor-core convolution on the
     16-channel 32x32 maps, conv3x3_tc_kernel<16> (profiles/ddg_step_resnet110_k4_b128_bf16_launch_list.md).  It is
@@ -167,13 +189,19 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
         return dt, per + w.numel() * 2, 2.0 * 9 * Cc * Cc * B * Hh * Hh, n
 
     dt, alg, flops, n = conv_case(32, 16)
-    # DRAM traffic per launch from the ncu capture at batch 4096 (profiles/conv3x3_tc_kernel_c16_fwd_b4096_ncu_full.md):
-    # 134.3 MB read + 88.5 MB written for 268.4 MB algorithmic (part of the output is still in L2 when the kernel
-    # ends); traffic grows with the pixels processed, so it is scaled by batch
-    traffic = 222.8e6 * B / 4096.0
+    # DRAM traffic per launch from the ncu capture at batch 4096 (read + written; part of the output is still in L2
+    # when the kernel ends); traffic grows with the pixels processed, so it is scaled by batch.  null when the kernel's
+    # source has changed since the capture.
+    cnt = ncu_counters()
+    c16 = cnt.get("conv3x3_tc_kernel<16> fwd 32x32")
+    traffic = None
+    if c16 and c16["valid"]:
+        traffic = (c16["dram_bytes_read"] + c16["dram_bytes_write"]) * B / float(c16["batch"])
+    share = cnt.get("launch_list resnet110 K=4 B=128", {})
     roof = {"kernel": "conv3x3_tc_kernel<16> (tensor-core 3x3 convolution, forward) C=16 32x32 B=%d" % B, "bound": "hbm",
             "achieved": alg / dt / 1e9, "peak": hbm, "unit": "GB/s", "frac": alg / dt / 1e9 / hbm, "traffic": traffic,
-            "launch_us": dt * 1e6, "peak_source": src, "ncu_share_of_step": 0.187, "launches_timed": n,
+            "launch_us": dt * 1e6, "peak_source": src,
+            "ncu_share_of_step": share.get("conv3x3_tc_kernel<16>") if share.get("valid") else None, "launches_timed": n,
             "tflops": flops / dt / 1e12, "tensor_frac": flops / dt / 1e12 / tflops}
     others = []
     for (Hh, Cc) in ((16, 32), (8, 64)):
@@ -304,9 +332,36 @@ def main():
     f0.record(streams[0])
     for t in range(n_e2e):
         loss = net.step_host(*pinned[t % n_batches])
+    net.sync()                       # the last iteration's backward sweeps and updates belong to the timed region
     f1.record(streams[0])
     barrier()
     dt_e2e = f0.elapsed_time(f1) * 1e-3
+    net.destroy()
+
+    # ---- the same kernels with K = 1 (plain backpropagation, Section 3.2), same run, same batches ----
+    k1 = None
+    if K > 1 and not args.skip_k1:
+        net1 = binding.Ddg(cfg["layers"], [], cfg["batch"], cfg["in_shape"], cfg["num_classes"],
+                           precision=cfg["precision"], lr=o["lr"], momentum=o["momentum"], weight_decay=o["weight_decay"],
+                           use_graph=not args.no_graph, streams=[streams[0].cuda_stream])
+        net1.set_weights(synth.init_weights(cfg["layers"]))
+        for t in range(max(args.warmup, 3)):
+            net1.step(*dev[t % n_batches], want_loss=False)
+        net1.sync()
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_k1 = max(10, args.steps // 2)
+        g0.record(streams[0])
+        for t in range(n_k1):
+            net1.step(*dev[t % n_batches], want_loss=False)
+        net1.sync()
+        g1.record(streams[0])
+        barrier()
+        dt_k1 = max_over_ranks([g0.elapsed_time(g1) * 1e-3], dist, "cuda")[0]
+        k1 = {"value": job_throughput(cfg["batch"], n_k1, world, dt_k1), "unit": "images/s", "ms_per_step": 1e3 * dt_k1 / n_k1,
+              "steps": n_k1, "launches_per_step": int(net1.last_step_launches()),
+              "what": "the same network, kernels and batches with K = 1 (plain backpropagation)"}
+        net1.destroy()
 
     dt, dt_e2e = max_over_ranks([dt, dt_e2e], dist, "cuda")
 
@@ -331,11 +386,13 @@ def main():
                    "l2": "no flush: one iteration touches > 1 GB of activations, far above the 126 MB L2",
                    "final_loss": loss},
                "clocks": clocks, "gpu_launches": int(launches_per_step * args.steps),
+               "launches_per_step": int(launches_per_step),
                "e2e": {"value": job_throughput(cfg["batch"], n_e2e, world, dt_e2e), "unit": "images/s",
                        "h2d_bytes_per_step": x_bytes + cfg["batch"] * 4, "d2h_bytes_per_step": 4, "steps": n_e2e},
-               "roofline": roof, "roofline_others": roof_others, "cpu_baseline": cpu}
+               "k1_baseline": k1, "roofline": roof, "roofline_others": roof_others, "cpu_baseline": cpu}
+        if k1:
+            out["k1_baseline"]["speedup_of_ddg"] = out["value"] / k1["value"]
         print(json.dumps(out))
-    net.destroy()
     if dist is not None:
         dist.destroy_process_group()
     return 0

@@ -86,9 +86,18 @@ typedef struct {
     int in_c, in_h, in_w;   /* input is [B][in_c][in_h][in_w] fp32 (use in_h = in_w = 1 for an MLP) */
     int num_classes;
     unsigned long long seed; /* seed of the library's own He-normal initialisation */
-    int use_graph;  /* 1: replay the steady-state iteration from CUDA graphs (one per ring phase, module and sweep) */
-    int debug_checks; /* 1: stamp ring slots with the iteration that wrote them and verify on use */
+    int use_graph;  /* 1: replay the steady-state iteration from CUDA graphs (one per ring phase, module and sweep),
+                       all recorded at the first iteration in which every module has a delayed gradient (t = K-1) */
+    int debug_checks; /* 1: every activation slot, weight-version slot and error-gradient buffer carries a stamp of the
+                       iteration (sample) that wrote it, set and compared on the device by one small kernel per sweep;
+                       a slot that is not the one the delay pattern of Eq. 6-8 asks for raises an error word, and the
+                       next sync point returns DDG_ERR_STATE.  Three extra launches per module and iteration. */
     void *const *streams; /* host array of K cudaStream_t to run the modules on, or NULL (library creates K) */
+    int separate_bn_sums; /* 0 (default): the batch-norm sums are taken in the epilogue of the tensor-core convolution
+                       that produces the tensor.  1: separate reduction kernels (same sums, other summation order). */
+    int launch_overlap; /* programmatic dependent launch (the next kernel of a stream is placed while the previous one
+                       still runs).  0 (default): the library's policy: every kernel when K = 1; with several module
+                       streams only the forward / input-gradient convolutions.  1: never.  2: every kernel. */
 } ddg_cfg;
 
 /* Build a context: validates the network (Section 2: L layers; Section 3: K groups of consecutive layers,
@@ -136,6 +145,18 @@ ddg_status ddg_last_step_launches(const ddg_ctx *ctx, long *launches);
 
 /* Wait for all K streams; surfaces deferred device-side errors. */
 ddg_status ddg_sync(ddg_ctx *ctx);
+
+/* Diagnostics (no counterpart in the paper).  Every device-side wait in the library is bounded: a wait that runs out
+ * raises the context's error word instead of hanging, the kernel returns, and the next sync point (ddg_sync,
+ * ddg_get_weights, ddg_get_grads, ddg_step with a loss) answers DDG_ERR_TIMEOUT, after which the context is in
+ * DDG_ERR_STATE.  ddg_debug_wait_timeout exercises exactly that path without a stuck pipeline: it enqueues, on the
+ * first module's stream, a one-CTA kernel that waits with a limit of `polls` polls (a few hundred nanoseconds each) on
+ * a barrier nothing arrives on, gives up and returns.
+ * ddg_debug_shift_stamps (contexts created with debug_checks) adds `delta` to the iteration counter module k's forward
+ * sweep stamps its ring slots with, as an indexing error of the rings would: the next sweeps see stamps that do not
+ * match and the next sync point answers DDG_ERR_STATE. */
+ddg_status ddg_debug_wait_timeout(ddg_ctx *ctx, unsigned polls);
+ddg_status ddg_debug_shift_stamps(ddg_ctx *ctx, int k, long delta);
 
 const char *ddg_last_error(const ddg_ctx *ctx); /* ctx may be NULL: error of the last failed ddg_create */
 void ddg_destroy(ddg_ctx *ctx);

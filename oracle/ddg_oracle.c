@@ -390,9 +390,6 @@ typedef struct {
     hist_t **hist;          /* hist[k][slot] */
     int **labels_hist;      /* labels of the in-flight iterations */
     long *labels_s;
-    /* ReLU decisions that floating point cannot settle: see orc_set_tie_policy */
-    double tie_tau;
-    long tie_up, tie_count;
 } orc_ctx;
 
 static size_t tsize(const orc_ctx *c, int C, int H, int W) { return (size_t)c->B * C * H * W; }
@@ -441,23 +438,6 @@ static double *dup(const double *src, size_t n) {
     return p;
 }
 
-/* y = relu(pre) at one ReLU site of the network.  A pre-activation closer to zero than tie_tau is a decision
- * that two correct floating-point evaluations may take differently (relu'(0) jumps).  With tie_tau > 0 such
- * elements are numbered in traversal order and forced: "off" (output 0, derivative 0) by default, "on" (output a
- * positive value far below any rounding, derivative 1) for element number tie_up, or for all when tie_up == -2.
- * The forward values move by less than tie_tau either way. */
-static void relu_site(orc_ctx *c, size_t n, const double *pre, double *y) {
-    for (size_t i = 0; i < n; ++i) {
-        const double p = pre[i];
-        if (c->tie_tau > 0.0 && fabs(p) < c->tie_tau) {
-            const long idx = c->tie_count++;
-            y[i] = (c->tie_up == -2 || idx == c->tie_up) ? 1e-30 : 0.0;
-        } else {
-            y[i] = p > 0.0 ? p : 0.0;
-        }
-    }
-}
-
 /* forward sweep of one layer (Eq. 3).  `w` points at the layer's own parameter slice.  Returns the
  * freshly allocated output; fills `q` with what the backward sweep needs. */
 static double *layer_forward(orc_ctx *c, const layer_t *L, const double *w, const double *x, cache_t *q) {
@@ -469,23 +449,23 @@ static double *layer_forward(orc_ctx *c, const layer_t *L, const double *w, cons
     switch (L->spec.kind) {
     case ORC_FC:
         orc_fc_forward(B, L->C_in, L->C_out, x, w, L->spec.has_bias ? w + (size_t)L->C_in * L->C_out : NULL, y);
-        if (L->spec.relu_after) relu_site(c, n_out, y, y);
+        if (L->spec.relu_after) orc_relu_forward(n_out, y, y);
         if (!is_last) maybe_round(c, y, n_out);
         else maybe_round32(c, y, n_out); /* the network output (logits) is kept in float */
         break;
     case ORC_CONV3X3:
         orc_conv3x3_forward(B, L->C_in, L->H_in, L->W_in, L->C_out, L->spec.stride, x, w, y);
-        if (L->spec.relu_after) relu_site(c, n_out, y, y);
+        if (L->spec.relu_after) orc_relu_forward(n_out, y, y);
         maybe_round(c, y, n_out);
         break;
     case ORC_BN:
         q->m1 = dalloc(L->C_in); q->is1 = dalloc(L->C_in);
         bn_forward_stored(c, B, L->C_in, L->H_in * L->W_in, x, w, w + L->C_in, y, q->m1, q->is1);
-        if (L->spec.relu_after) relu_site(c, n_out, y, y);
+        if (L->spec.relu_after) orc_relu_forward(n_out, y, y);
         maybe_round(c, y, n_out);
         break;
     case ORC_RELU:
-        relu_site(c, n_out, x, y);
+        orc_relu_forward(n_out, x, y);
         break;
     case ORC_GLOBAL_AVGPOOL:
         orc_avgpool_forward(B, L->C_in, L->H_in * L->W_in, x, y);
@@ -501,7 +481,7 @@ static double *layer_forward(orc_ctx *c, const layer_t *L, const double *w, cons
         orc_conv3x3_forward(B, Ci, L->H_in, L->W_in, Co, st, x, w1, q->y1);
         maybe_round(c, q->y1, n_out);
         bn_forward_stored(c, B, Co, HWo, q->y1, g1, b1, q->a1, q->m1, q->is1);
-        relu_site(c, n_out, q->a1, q->a1);
+        orc_relu_forward(n_out, q->a1, q->a1);
         maybe_round(c, q->a1, n_out);
         orc_conv3x3_forward(B, Co, L->H_out, L->W_out, Co, 1, q->a1, w2, q->y2);
         maybe_round(c, q->y2, n_out);
@@ -509,7 +489,7 @@ static double *layer_forward(orc_ctx *c, const layer_t *L, const double *w, cons
         bn_forward_stored(c, B, Co, HWo, q->y2, g2, b2, z, q->m2, q->is2);
         orc_shortcut_forward(B, Ci, L->H_in, L->W_in, Co, st, x, sc);
         for (size_t i = 0; i < n_out; ++i) z[i] += sc[i];
-        relu_site(c, n_out, z, y);
+        orc_relu_forward(n_out, z, y);
         maybe_round(c, y, n_out);
         free(z); free(sc);
         break;
@@ -686,11 +666,6 @@ void orc_get_weights(const orc_ctx *c, double *w) { memcpy(w, c->w, c->P * sizeo
 void orc_set_lr(orc_ctx *c, double lr) { c->lr = lr; }
 long orc_iteration(const orc_ctx *c) { return c->t; }
 
-/* Near-zero ReLU decisions (see relu_site): tau = 0 switches the mechanism off (default).  up_index = -1 forces
- * all of them off, -2 all on, i >= 0 only the i-th on.  orc_tie_count = how many the last forward sweep met. */
-void orc_set_tie_policy(orc_ctx *c, double tau, long up_index) { c->tie_tau = tau; c->tie_up = up_index; }
-long orc_tie_count(const orc_ctx *c) { return c->tie_count; }
-
 /* last applied delayed gradient of module k (0-based).  Returns the sample index s it belongs to, or -1
  * when the module was still in warm-up at the last step (Eq. 8: gradient is zero, dst is zero-filled). */
 int orc_get_grads(const orc_ctx *c, int k, double *dst) {
@@ -708,7 +683,6 @@ static double *sweep_weights(const orc_ctx *c, const double *w, size_t n) {
 
 /* loss of the whole net at the current weights, no state change (for finite-difference pins) */
 double orc_loss_only(orc_ctx *c, const double *x, const int *y) {
-    c->tie_count = 0;
     double *h = dup(x, tsize(c, c->in_c, c->in_h, c->in_w));
     maybe_round(c, h, tsize(c, c->in_c, c->in_h, c->in_w));
     for (int l = 0; l < c->n_layers; ++l) {
@@ -734,7 +708,6 @@ double orc_step(orc_ctx *c, const double *x, const int *y) {
     c->labels_s[slot_t] = t;
 
     /* 1. forward sweep through modules 1..K with the current weights w^t (Eq. 3); keep h^t and w^t */
-    c->tie_count = 0;
     double *h = dup(x, tsize(c, c->in_c, c->in_h, c->in_w));
     maybe_round(c, h, tsize(c, c->in_c, c->in_h, c->in_w));
     for (int k = 0; k < K; ++k) {

@@ -61,9 +61,6 @@ def lib():
         L.orc_loss_only.argtypes = [ctypes.c_void_p, dp, ip]
         L.orc_step.restype = ctypes.c_double
         L.orc_step.argtypes = [ctypes.c_void_p, dp, ip]
-        L.orc_set_tie_policy.argtypes = [ctypes.c_void_p, ctypes.c_double, ctypes.c_long]
-        L.orc_tie_count.restype = ctypes.c_long
-        L.orc_tie_count.argtypes = [ctypes.c_void_p]
         L.orc_bf16_round.restype = ctypes.c_double
         L.orc_bf16_round.argtypes = [ctypes.c_double]
         _lib = L
@@ -135,14 +132,6 @@ class Oracle:
         x, xp = _d(x)
         y, yp = _i(y)
         return lib().orc_loss_only(self._h, xp, yp)
-
-    def set_tie_policy(self, tau, up_index=-1):
-        """ReLU pre-activations closer to zero than tau are forced off (up_index=-1), on (-2), or only the
-        up_index-th one on; tau=0 restores plain relu."""
-        lib().orc_set_tie_policy(self._h, float(tau), int(up_index))
-
-    def tie_count(self):
-        return lib().orc_tie_count(self._h)
 
     def get_grads(self, k):
         """(sample index s or -1 during warm-up, gradient of module k, 0-based) of the last step."""

@@ -27,7 +27,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_last_error", "ddg_destroy", "ddg_conv3x3_fwd", "ddg_conv3x3_dgrad",
            "ddg_conv3x3_wgrad_scratch_elems", "ddg_conv3x3_wgrad", "ddg_bn_scratch_elems", "ddg_bn_fwd", "ddg_bn_bwd",
            "ddg_sgd_update", "ddg_tensor_core_path", "ddg_bn_fwd_noalloc",
-           "ddg_conv3x3_packed_bytes", "ddg_conv3x3_pack", "ddg_conv3x3_packed", "ddg_bn_bwd_reduce"]
+           "ddg_conv3x3_packed_bytes", "ddg_conv3x3_pack", "ddg_conv3x3_packed", "ddg_bn_bwd_reduce",
+           "ddg_debug_wait_timeout", "ddg_debug_shift_stamps"]
 
 
 class Layer(ctypes.Structure):
@@ -43,7 +44,8 @@ class Cfg(ctypes.Structure):
     _fields_ = [("precision", ctypes.c_int), ("batch", ctypes.c_int), ("in_c", ctypes.c_int), ("in_h", ctypes.c_int),
                 ("in_w", ctypes.c_int), ("num_classes", ctypes.c_int), ("seed", ctypes.c_ulonglong),
                 ("use_graph", ctypes.c_int), ("debug_checks", ctypes.c_int),
-                ("streams", ctypes.POINTER(ctypes.c_void_p))]
+                ("streams", ctypes.POINTER(ctypes.c_void_p)), ("separate_bn_sums", ctypes.c_int),
+                ("launch_overlap", ctypes.c_int)]
 
 
 _vp, _i, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -59,6 +61,8 @@ _lib.ddg_get_grads.argtypes = [_vp, _i, _vp, _sz, _i, ctypes.POINTER(ctypes.c_lo
 _lib.ddg_get_loss_dev.argtypes = [_vp, ctypes.POINTER(_vp)]
 _lib.ddg_last_step_launches.argtypes = [_vp, ctypes.POINTER(ctypes.c_long)]
 _lib.ddg_sync.argtypes = [_vp]
+_lib.ddg_debug_wait_timeout.argtypes = [_vp, ctypes.c_uint]
+_lib.ddg_debug_shift_stamps.argtypes = [_vp, _i, ctypes.c_long]
 _lib.ddg_last_error.argtypes = [_vp]
 _lib.ddg_last_error.restype = ctypes.c_char_p
 _lib.ddg_destroy.argtypes = [_vp]
@@ -109,7 +113,7 @@ class Ddg:
 
     def __init__(self, layers, split_after, batch, in_shape, num_classes, precision="fp32", opt="sgd", lr=0.01,
                  momentum=0.0, weight_decay=0.0, beta1=0.9, beta2=0.999, eps=1e-8, seed=0, use_graph=False,
-                 debug_checks=False, streams=None):
+                 debug_checks=False, streams=None, separate_bn_sums=False, launch_overlap=0):
         arr = (Layer * len(layers))(*[Layer(*map(int, l)) for l in layers])
         K = len(split_after) + 1
         sp = (ctypes.c_int * max(1, K - 1))(*split_after)
@@ -119,7 +123,7 @@ class Ddg:
             assert len(streams) == K
             st = (ctypes.c_void_p * K)(*[int(s) for s in streams])
         cfg = Cfg(BF16 if precision == "bf16" else FP32, batch, in_shape[0], in_shape[1], in_shape[2], num_classes,
-                  seed, int(use_graph), int(debug_checks), st)
+                  seed, int(use_graph), int(debug_checks), st, int(separate_bn_sums), int(launch_overlap))
         h = ctypes.c_void_p()
         rc = _lib.ddg_create(arr, len(layers), sp, K, ctypes.byref(o), ctypes.byref(cfg), ctypes.byref(h))
         if rc != 0:
@@ -184,6 +188,12 @@ class Ddg:
 
     def sync(self):
         self._check(_lib.ddg_sync(self._h))
+
+    def debug_wait_timeout(self, polls):
+        self._check(_lib.ddg_debug_wait_timeout(self._h, polls))
+
+    def debug_shift_stamps(self, k, delta):
+        self._check(_lib.ddg_debug_shift_stamps(self._h, k, delta))
 
 
 def _ok(rc):

@@ -2,9 +2,13 @@
 #include "../../include/ddg.h"
 #include "common.cuh"
 #include "conv_tc.h"
+#include <stdio.h>
+
 #include "kernels.h"
 
 using namespace ddg;
+
+namespace ddg { void set_global_error(const char *msg); }
 
 namespace {
 bool bad_prec(int p) { return p != DDG_FP32 && p != DDG_BF16; }
@@ -13,7 +17,27 @@ ddg_status init_once() {
     if (rc < 0) { rc = conv_direct_init(); if (rc == 0) rc = conv_tc_init(); }
     return rc == 0 ? DDG_OK : DDG_ERR_CUDA;
 }
-ddg_status done() { return cudaGetLastError() == cudaSuccess ? DDG_OK : DDG_ERR_CUDA; }
+// An error left pending by an earlier, unrelated CUDA call would otherwise be blamed on (and cleared by) this entry
+// point: refuse to launch on top of it and name it.
+bool pending_error() {
+    const cudaError_t e = cudaPeekAtLastError();
+    if (e == cudaSuccess) return false;
+    static thread_local char msg[256];
+    snprintf(msg, sizeof(msg), "an earlier CUDA error is still pending: %s", cudaGetErrorString(e));
+    set_global_error(msg);
+    return true;
+}
+// r: what the launcher returned (negative: it refused the launch)
+ddg_status done(int r = 0) {
+    if (r < 0) {
+        set_global_error("the kernel launcher refused the launch (tensor map or shared-memory plan)");
+        return DDG_ERR_CUDA;
+    }
+    const cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) return DDG_OK;
+    set_global_error(cudaGetErrorString(e));
+    return DDG_ERR_CUDA;
+}
 bool conv_shape_ok(int B, int H, int W, int Cin, int Cout, int stride) {
     return B >= 1 && H >= 1 && W >= 1 && Cin >= 1 && Cout >= 1 && (stride == 1 || stride == 2) && Cin <= 256 &&
            Cout <= 256 && (size_t)Cin * Cout <= 4096;
@@ -33,14 +57,16 @@ ddg_status ddg_conv3x3_fwd(int precision, const void *x, const void *w, void *y,
     if (bad_prec(precision) || !x || !w || !y) return DDG_ERR_INVALID_ARG;
     if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
     if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (pending_error()) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
+    int r;
     if (precision == DDG_BF16 && conv_tc_supported(B, H, W, Cin, Cout, stride))
-        launch_conv_tc(0, x, w, nullptr, y, B, H, W, Cin, Shortcut{}, s);
+        r = launch_conv_tc(0, x, w, nullptr, y, B, H, W, Cin, Shortcut{}, s);
     else if (precision == DDG_BF16 && conv_tc_s2_supported(B, H, W, Cin, Cout, stride))
-        launch_conv_tc_s2(0, x, w, nullptr, y, B, H, W, Cin, Shortcut{}, s);
+        r = launch_conv_tc_s2(0, x, w, nullptr, y, B, H, W, Cin, Shortcut{}, s);
     else
-        launch_conv_fwd_direct(precision, x, w, y, B, H, W, Cin, Cout, stride, 0, s);
-    return done();
+        r = launch_conv_fwd_direct(precision, x, w, y, B, H, W, Cin, Cout, stride, 0, s);
+    return done(r);
 }
 
 ddg_status ddg_conv3x3_dgrad(int precision, const void *dy, const void *w, void *dx, int B, int H, int W, int Cin,
@@ -48,14 +74,16 @@ ddg_status ddg_conv3x3_dgrad(int precision, const void *dy, const void *w, void 
     if (bad_prec(precision) || !dy || !w || !dx) return DDG_ERR_INVALID_ARG;
     if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
     if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (pending_error()) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
+    int r;
     if (precision == DDG_BF16 && conv_tc_supported(B, H, W, Cin, Cout, stride))
-        launch_conv_tc(1, dy, w, nullptr, dx, B, H, W, Cin, Shortcut{}, s);
+        r = launch_conv_tc(1, dy, w, nullptr, dx, B, H, W, Cin, Shortcut{}, s);
     else if (precision == DDG_BF16 && conv_tc_s2_supported(B, H, W, Cin, Cout, stride))
-        launch_conv_tc_s2(1, dy, w, nullptr, dx, B, H, W, Cin, Shortcut{}, s);
+        r = launch_conv_tc_s2(1, dy, w, nullptr, dx, B, H, W, Cin, Shortcut{}, s);
     else
-        launch_conv_dgrad_direct(precision, dy, w, dx, B, H, W, Cin, Cout, stride, Shortcut{}, s);
-    return done();
+        r = launch_conv_dgrad_direct(precision, dy, w, dx, B, H, W, Cin, Cout, stride, Shortcut{}, s);
+    return done(r);
 }
 
 size_t ddg_conv3x3_packed_bytes(int B, int H, int W, int C) {
@@ -66,8 +94,8 @@ size_t ddg_conv3x3_packed_bytes(int B, int H, int W, int C) {
 ddg_status ddg_conv3x3_pack(const void *w, void *packed, int C, void *stream) {
     if (!w || !packed) return DDG_ERR_INVALID_ARG;
     if (C != 16 && C != 32 && C != 64) return DDG_ERR_UNSUPPORTED;
-    launch_pack_one(w, packed, C, (cudaStream_t)stream);
-    return done();
+    if (pending_error()) return DDG_ERR_CUDA;
+    return done(launch_pack_one(w, packed, C, (cudaStream_t)stream));
 }
 
 ddg_status ddg_conv3x3_packed(int dgrad, const void *src, const void *w, const void *packed, void *dst, int B, int H,
@@ -75,8 +103,8 @@ ddg_status ddg_conv3x3_packed(int dgrad, const void *src, const void *w, const v
     if (!src || !w || !packed || !dst) return DDG_ERR_INVALID_ARG;
     if (init_once() != DDG_OK) return DDG_ERR_CUDA;
     if (!conv_tc_supported(B, H, W, C, C, 1)) return DDG_ERR_UNSUPPORTED;
-    launch_conv_tc(dgrad ? 1 : 0, src, w, packed, dst, B, H, W, C, Shortcut{}, (cudaStream_t)stream);
-    return done();
+    if (pending_error()) return DDG_ERR_CUDA;
+    return done(launch_conv_tc(dgrad ? 1 : 0, src, w, packed, dst, B, H, W, C, Shortcut{}, (cudaStream_t)stream));
 }
 
 size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride) {
@@ -90,14 +118,16 @@ ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float
     if (bad_prec(precision) || !x || !dy || !dw || !scratch) return DDG_ERR_INVALID_ARG;
     if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
     if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (pending_error()) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
+    int r;
     if (precision == DDG_BF16 && wgrad_tc_supported(B, H, W, Cin, Cout, stride))
-        launch_wgrad_tc(x, dy, dw, scratch, B, H, W, Cin, Cin, s);
+        r = launch_wgrad_tc(x, dy, dw, scratch, B, H, W, Cin, Cin, s);
     else if (precision == DDG_BF16 && conv_tc_s2_supported(B, H, W, Cin, Cout, stride))
-        launch_wgrad_tc_s2(x, dy, dw, scratch, B, H, W, Cin, s);
+        r = launch_wgrad_tc_s2(x, dy, dw, scratch, B, H, W, Cin, s);
     else
-        launch_conv_wgrad_direct(precision, x, dy, dw, scratch, B, H, W, Cin, Cout, stride, s);
-    return done();
+        r = launch_conv_wgrad_direct(precision, x, dy, dw, scratch, B, H, W, Cin, Cout, stride, s);
+    return done(r);
 }
 
 size_t ddg_bn_scratch_elems(int C) { return C >= 1 && C <= 128 ? bn_scratch_elems(C) : 0; }
@@ -106,6 +136,7 @@ ddg_status ddg_bn_fwd(int precision, const void *x, const void *gamma, const voi
                       float *mean, float *invstd, float *scratch, int B, int HW, int C, int relu, void *stream) {
     if (bad_prec(precision) || !x || !gamma || !beta || !y || !mean || !invstd || !scratch) return DDG_ERR_INVALID_ARG;
     if (B < 1 || HW < 1 || C < 1 || C > 128) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;  // the CTA ticket counter
     launch_bn_stats(precision, x, mean, invstd, scratch, (long)B * HW, C, s);
@@ -122,6 +153,7 @@ ddg_status ddg_bn_bwd(int precision, const void *dout, const void *out, const vo
         (relu && !out))
         return DDG_ERR_INVALID_ARG;
     if (B < 1 || HW < 1 || C < 1 || C > 128) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;
     launch_bn_bwd_reduce(precision, dout, out, x, mean, invstd, dgamma, dbeta, scratch, (long)B * HW, C, relu, s);
@@ -135,6 +167,7 @@ ddg_status ddg_bn_bwd_reduce(int precision, const void *dout, const void *out, c
     if (bad_prec(precision) || !dout || !x || !mean || !invstd || !dgamma || !dbeta || !scratch || (relu && !out))
         return DDG_ERR_INVALID_ARG;
     if (B < 1 || HW < 1 || C < 1 || C > 128) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;
     launch_bn_bwd_reduce(precision, dout, out, x, mean, invstd, dgamma, dbeta, scratch, (long)B * HW, C, relu, s);
@@ -144,6 +177,7 @@ ddg_status ddg_bn_bwd_reduce(int precision, const void *dout, const void *out, c
 ddg_status ddg_sgd_update(int precision, float *w, float *v, const float *g, void *w_version, size_t n, float lr,
                           float momentum, float weight_decay, void *stream) {
     if (bad_prec(precision) || !w || !v || !g || !w_version) return DDG_ERR_INVALID_ARG;
+    if (pending_error()) return DDG_ERR_CUDA;
     UpdateArgs a{};
     a.mode = 0; a.lr = lr; a.mu = momentum; a.wd = weight_decay;
     launch_update(precision, w, v, nullptr, g, w_version, n, a, (cudaStream_t)stream);

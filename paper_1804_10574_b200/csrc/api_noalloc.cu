@@ -63,6 +63,13 @@ extern "C" ddg_status ddg_bn_fwd_noalloc(int precision, const void *x, const voi
                          "with caller-provided scratch");
         return DDG_ERR_UNSUPPORTED;
     }
+    {   // an error left pending by an earlier call must not be blamed on (or cleared by) this one
+        const cudaError_t before = cudaPeekAtLastError();
+        if (before != cudaSuccess) {
+            set_global_error("ddg_bn_fwd_noalloc: an earlier CUDA error is still pending");
+            return DDG_ERR_CUDA;
+        }
+    }
     float *scratch = nullptr;
     ddg_status st = scratch_for_current_device(&scratch);
     if (st != DDG_OK) return st;

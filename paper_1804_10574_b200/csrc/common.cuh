@@ -6,6 +6,8 @@
 
 #include <utility>
 
+#include "kernels.h"
+
 namespace ddg {
 
 typedef __nv_bfloat16 bf16;
@@ -71,39 +73,34 @@ __device__ __forceinline__ float warp_max(float v) {
 
 static inline int ceil_div(long a, long b) { return (int)((a + b - 1) / b); }
 
-// Programmatic dependent launch.  Where pdl_enabled() says so (single kernels, single-module networks) a kernel is
-// launched with programmatic stream serialisation: the next kernel of the stream may be scheduled while this one is
-// still running, so that its launch latency and its prologue overlap this kernel's tail.  The contract that keeps this correct: every kernel executes pdl_wait() before
-// its first access to global memory that an earlier kernel may write or still read; the wait returns when all
-// preceding kernels of the stream have completed and their writes are visible.  pdl_launch() tells the scheduler that
-// the next kernel may start being placed.
+// Programmatic dependent launch.  A kernel launched with programmatic stream serialisation may be scheduled while the
+// previous kernel of its stream is still running, so that its launch latency and its prologue overlap that kernel's
+// tail.  The contract that keeps this correct: every kernel executes pdl_wait() before its first access to global
+// memory that an earlier kernel may write or still read; the wait returns when all preceding kernels of the stream have
+// completed and their writes are visible.  pdl_launch() tells the scheduler that the next kernel may start being placed.
+// Which launches carry the attribute is the caller's policy (Launch::pdl in kernels.h).
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-bool gpu_shared_by_streams();  // defined in engine.cu: true while a multi-module iteration is enqueued
-// defined in engine.cu.  While a multi-module iteration is enqueued only launches that ask with `while_shared` get the
-// attribute (the tensor-core convolution: see there); DDG_PDL=0/1 in the environment forces it off / on for all
-bool pdl_enabled(bool while_shared = false);
-
-// pdl_while_shared: the launch carries the programmatic attribute also while several module streams share the GPU
+// asks_pdl: the kernel is one of those that keep the attribute under Launch::pdl == 2
 template <typename... KArgs, typename... Args>
-inline void launch_kp(bool pdl_while_shared, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+inline void launch_kp(bool asks_pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, const Launch &L,
                       Args &&...args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
+    cfg.stream = L.s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl_enabled(pdl_while_shared) ? 1 : 0;
+    cfg.numAttrs = (L.pdl == 1 || (L.pdl == 2 && asks_pdl)) ? 1 : 0;
     cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 template <typename... KArgs, typename... Args>
-inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
-    launch_kp(false, kernel, grid, block, smem, stream, std::forward<Args>(args)...);
+inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, const Launch &L, Args &&...args) {
+    launch_kp(false, kernel, grid, block, smem, L, std::forward<Args>(args)...);
 }
 
 }  // namespace ddg

@@ -70,14 +70,19 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity, uint32_t
     return ok != 0;
 }
 // Bounded wait.  Returns false (and raises the error word and the CTA's abort flag) when the limit is hit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code) {
-    for (unsigned i = 0; i < kSpinLimit; ++i) {
+struct Waiter {
+    volatile int *abort_flag;  // shared memory: set by the first wait of the CTA that gives up, seen by the others
+    int *err;                  // global memory: the error word the host reads at its next sync point
+    unsigned limit;            // polls before a wait gives up
+};
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Waiter &wt, int code) {
+    for (unsigned i = 0; i < wt.limit; ++i) {
         if (mbar_try(bar, parity)) return true;
-        if ((i & 15u) == 15u && *abort_flag) return false;
+        if ((i & 15u) == 15u && *wt.abort_flag) return false;
         if (i > 4096) __nanosleep(64);
     }
-    *abort_flag = 1;
-    atomicCAS(&g_tc_error, 0, code);
+    *wt.abort_flag = 1;
+    atomicCAS(wt.err, 0, code);
     return false;
 }
 
@@ -320,7 +325,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                   int slab, int n_stages, int stage_bytes, int tmem_cols, EpiPlan plan_e, const bf16 *__restrict__ res_dout,
                   const bf16 *__restrict__ res_out, float *__restrict__ stat_part, unsigned *__restrict__ stat_counter,
                   float *__restrict__ stat_o0, float *__restrict__ stat_o1, const bf16 *__restrict__ bn_mask,
-                  const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd) {
+                  const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd,
+                  int *__restrict__ err_word) {
     // stat_part != nullptr: the epilogue also reduces, per channel over the pixels of this CTA's tiles, the two sums the
     // batch norm that follows needs, from the values as stored (rounded to bf16), writes them to
     // stat_part[blockIdx.x][2C], and the CTA that finishes last adds the partials in a fixed order:
@@ -338,6 +344,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[4], tempty[4], wbar
     uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 9) * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 9) * 8 + 8);
+    const Waiter wt{abort_flag, err_word, kSpinLimit};
     float (*sm_run)[4][32] = reinterpret_cast<float (*)[4][32]>(tail + 512);  // [epilogue warp][channel chunk][lane]
     float *sm_stat = reinterpret_cast<float *>(tail + 512 + 8192);            // mean[C], invstd[C]
     const uint32_t bar0 = smem_u32(bars);
@@ -408,7 +415,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                 else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
                 for (int j = 0; j < loads_per_tile && ok; ++j) {
                     const int s = g * ring + ls;
-                    ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 1);
+                    ok = mbar_wait(empty_bar(s), ph ^ 1u, wt, 1);
                     if (!ok) break;
                     mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
                     tma_load_4d(a_base + s * stage_bytes, &tmap, full_bar(s), 0, 0, slab ? h0 - 1 : h0 + j - 1, n0);
@@ -427,18 +434,18 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
             int ls = 0, it = 0;
             uint32_t ph = 0;
             bool ok = true;
-            if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, abort_flag, 5);
+            if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, wt, 5);
             for (int tile = blockIdx.x + g * gridDim.x; tile < n_tiles && ok; tile += tile_step, ++it) {
                 // the pipeline's accumulators in turn
                 const int a = g * plan_e.n_acc + it % plan_e.n_acc;
                 const uint32_t aph = (uint32_t)(it / plan_e.n_acc) & 1u;
-                ok = mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, 2);
+                ok = mbar_wait(tempty_bar(a), aph ^ 1u, wt, 2);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * 3 * C);
                 for (int j = 0; j < loads_per_tile && ok; ++j) {
                     const int s = g * ring + ls;
-                    ok = mbar_wait(full_bar(s), ph, abort_flag, 3);
+                    ok = mbar_wait(full_bar(s), ph, wt, 3);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = a_base + s * stage_bytes;
@@ -489,7 +496,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                     prefetch_l1(reinterpret_cast<const char *>(bn_x + pix * C) + o);
                 }
             }
-            ok = mbar_wait(tfull_bar(a), aph, abort_flag, 4);
+            ok = mbar_wait(tfull_bar(a), aph, wt, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -637,7 +644,7 @@ template <int C>
 __global__ void __launch_bounds__(kWgThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 float *__restrict__ part, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles, int slab,
-                int n_stages, int x_box_bytes, int tmem_cols, int wide, int tall) {
+                int n_stages, int x_box_bytes, int tmem_cols, int wide, int tall, int *__restrict__ err_word) {
     typedef TcCfg<C> Cfg;
     const int stage_bytes = Cfg::tile_bytes + 3 * x_box_bytes;
     const int box_rows = rows_per_tile + 2;  // image rows of a column box in slab mode
@@ -648,6 +655,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], done
     uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 1) * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 1) * 8 + 8);
+    const Waiter wt{abort_flag, err_word, kSpinLimit};
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
@@ -685,7 +693,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 int n0, h0;
                 if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }
                 else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
-                ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 11);
+                ok = mbar_wait(empty_bar(s), ph ^ 1u, wt, 11);
                 if (!ok) break;
                 const uint32_t st = base + s * stage_bytes;
                 mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
@@ -710,7 +718,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             uint32_t ph = 0;
             bool ok = true;
             for (int tile = t0; tile < t1 && ok; ++tile) {
-                ok = mbar_wait(full_bar(s), ph, abort_flag, 12);
+                ok = mbar_wait(full_bar(s), ph, wt, 12);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t st = base + s * stage_bytes;
@@ -769,7 +777,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         }
     } else {
         const int q = warp & 3;
-        bool ok = mbar_wait(done_bar, 0, abort_flag, 13);
+        bool ok = mbar_wait(done_bar, 0, wt, 13);
         ok = __all_sync(0xffffffffu, ok);
         if (ok && tall) {
             // accumulator row = ky*C + ci (rows >= 3C unused), column = kx*C + co: each thread writes runs of output channels
@@ -852,7 +860,7 @@ template <int KC, int NC, int MODE>
 __global__ void __launch_bounds__(kS2Threads, 1)
 conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
                      bf16 *__restrict__ dst, int Hs, int Ws, int rows_per_tile, int imgs_per_tile, int n_sp, int n_stages,
-                     const bf16 *__restrict__ res_dout, const bf16 *__restrict__ res_out) {
+                     const bf16 *__restrict__ res_dout, const bf16 *__restrict__ res_out, int *__restrict__ err_word) {
     typedef TcCfg<KC> Cfg;
     constexpr int CI = MODE == 0 ? KC : NC;
     constexpr int tap_bytes = KC * NC * 2;
@@ -868,6 +876,7 @@ conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__res
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[4], tempty[4], wbar
     uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 9) * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 9) * 8 + 8);
+    const Waiter wt{abort_flag, err_word, kSpinLimit};
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
@@ -928,7 +937,7 @@ conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__res
                 tile_origin(sp, &n0, &h0);
                 const int n_loads = MODE == 0 ? 9 : (1 + py) * (1 + px);
                 for (int j = 0; j < n_loads && ok; ++j) {
-                    ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 21);
+                    ok = mbar_wait(empty_bar(s), ph ^ 1u, wt, 21);
                     if (!ok) break;
                     mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
                     const uint32_t d = a_base + s * stage_bytes;
@@ -953,19 +962,19 @@ conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__res
             uint32_t ph = 0;
             int it = 0;
             bool ok = true;
-            if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, abort_flag, 25);
+            if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, wt, 25);
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
                 const int cls = MODE == 0 ? 0 : tile / n_sp;
                 const int py = cls >> 1, px = cls & 1;
                 const int n_loads = MODE == 0 ? 9 : (1 + py) * (1 + px);
                 const int a = it & 1;
                 const uint32_t aph = (it >> 1) & 1u;
-                ok = mbar_wait(tempty_bar(a), aph ^ 1u, abort_flag, 22);
+                ok = mbar_wait(tempty_bar(a), aph ^ 1u, wt, 22);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * NC);
                 for (int j = 0; j < n_loads && ok; ++j) {
-                    ok = mbar_wait(full_bar(s), ph, abort_flag, 23);
+                    ok = mbar_wait(full_bar(s), ph, wt, 23);
                     if (!ok) break;
                     tc_fence_after();
                     int tap = j;
@@ -993,7 +1002,7 @@ conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__res
         for (int tile = blockIdx.x + grp * gridDim.x; tile < n_tiles && ok; tile += 2 * gridDim.x, it += 2) {
             const int a = it & 1;
             const uint32_t aph = (it >> 1) & 1u;
-            ok = mbar_wait(tfull_bar(a), aph, abort_flag, 24);
+            ok = mbar_wait(tfull_bar(a), aph, wt, 24);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -1058,7 +1067,8 @@ conv3x3_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__res
 template <int CI>
 __global__ void __launch_bounds__(kWgThreads, 1)
 wgrad_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
-                   float *__restrict__ part, int Hs, int Ws, int rows_per_tile, int imgs_per_tile, int n_tiles, int n_stages) {
+                   float *__restrict__ part, int Hs, int Ws, int rows_per_tile, int imgs_per_tile, int n_tiles, int n_stages,
+                   int *__restrict__ err_word) {
     constexpr int CO = 2 * CI;
     typedef TcCfg<CI> CfgX;
     typedef TcCfg<CO> CfgY;
@@ -1073,6 +1083,7 @@ wgrad_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail);
     uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 1) * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 1) * 8 + 8);
+    const Waiter wt{abort_flag, err_word, kSpinLimit};
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
@@ -1109,7 +1120,7 @@ wgrad_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 int n0, h0;
                 if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }
                 else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
-                ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 31);
+                ok = mbar_wait(empty_bar(s), ph ^ 1u, wt, 31);
                 if (!ok) break;
                 const uint32_t st = base + s * stage_bytes;
                 mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
@@ -1132,7 +1143,7 @@ wgrad_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             uint32_t ph = 0;
             bool ok = true;
             for (int tile = t0; tile < t1 && ok; ++tile) {
-                ok = mbar_wait(full_bar(s), ph, abort_flag, 32);
+                ok = mbar_wait(full_bar(s), ph, wt, 32);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t st = base + s * stage_bytes;
@@ -1155,7 +1166,7 @@ wgrad_s2_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         }
     } else {
         const int q = warp & 3;
-        bool ok = mbar_wait(done_bar, 0, abort_flag, 33);
+        bool ok = mbar_wait(done_bar, 0, wt, 33);
         ok = __all_sync(0xffffffffu, ok);
         if (ok && 32 * q < CO) {
             tc_fence_after();
@@ -1275,6 +1286,9 @@ bool get_map_s2(const void *ptr, int B, int H, int W, int C, int rows, int imgs,
 }
 
 int g_num_sms = 148;
+// device address of the process-wide error word (single-kernel entry points); contexts bring their own
+int *g_tc_error_addr = nullptr;
+int *err_word_of(const Launch &L) { return L.err ? L.err : g_tc_error_addr; }
 // Shared memory a CTA may take for its pipeline stages: less than half an SM, so that kernels of two modules (streams)
 // can share an SM instead of queueing behind each other (K = 4 step, ms per iteration at 56 / 64 / 72 / 80 / 100 / 128
 // KB: 1.870 / 1.884 / 1.844 / 1.844 - 1.857 / 1.874 / 2.068).
@@ -1283,7 +1297,7 @@ constexpr int kSmemMax = 227 * 1024;
 
 template <int C>
 int launch_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W,
-              Shortcut sc, BnFuse bf, cudaStream_t s) {
+              Shortcut sc, BnFuse bf, Launch s) {
     int rows, imgs;
     tile_geometry(H, W, &rows, &imgs);
     const int slab = (imgs == 1) ? 1 : 0;
@@ -1318,7 +1332,7 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     const int per_pipe = (n_tiles + sms * ep.n_pipes - 1) / (sms * ep.n_pipes);
     const int balanced = (n_tiles + per_pipe * ep.n_pipes - 1) / (per_pipe * ep.n_pipes);
     const int full = (n_tiles + ep.n_pipes - 1) / ep.n_pipes < sms ? (n_tiles + ep.n_pipes - 1) / ep.n_pipes : sms;
-    const int grid = gpu_shared_by_streams() ? balanced : full;
+    const int grid = s.shared ? balanced : full;
     const int groups = ep.n_pipes * ep.n_slots * ep.split;
     const int threads = 32 * (2 * ep.n_pipes + 4 * (groups < 2 ? 2 : groups));
     // CTAs with many tiles take the whole SM's shared memory for the stage ring; the others about half of it
@@ -1334,12 +1348,12 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     if (tmem_cols > 512 || conv_smem_bytes<C>(n_stages, stage_bytes) > (size_t)kSmemMax) return -1;
     launch_kp(true, conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
         stage_bytes, tmem_cols, ep, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
-        bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd);
+        bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd, err_word_of(s));
     return 1;
 }
 
 template <int C>
-int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int cin, cudaStream_t s) {
+int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int cin, Launch s) {
     int rows, imgs;
     tile_geometry(H, W, &rows, &imgs);
     const int slab = (imgs == 1 && 9 * C <= 512) ? 1 : 0;
@@ -1371,7 +1385,7 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int big = n_tiles / 16 < (slab ? kWgMaxChunks : 48) ? n_tiles / 16 : (slab ? kWgMaxChunks : 48);
     if (big > chunks) chunks = big;
     // tall: the unused accumulator rows (filter rows >= 3) read up to 128 - 3C pixel rows past the last column box
-    launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512 + (tall ? 4096 : 0), s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols, wide, tall);
+    launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512 + (tall ? 4096 : 0), s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols, wide, tall, err_word_of(s));
     launch_k(wgrad_tc_fold_kernel, ceil_div(9 * C * C, 64), 256, 0, s, scratch, dw, chunks, C, C, cin);
     return 2;
 }
@@ -1384,7 +1398,7 @@ size_t s2_smem_bytes(int n_stages) {
 // dir 1: src = dy -> dst = dx, plus the parameter-free shortcut's gradient when sc.mode == 2.
 template <int CI>
 int launch_tc_s2(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, Shortcut sc,
-                 cudaStream_t s) {
+                 Launch s) {
     constexpr int CO = 2 * CI;
     const int Hs = H / 2, Ws = W / 2;
     int rows, imgs;
@@ -1398,7 +1412,7 @@ int launch_tc_s2(int dir, const void *src, const void *w, const void *w_packed, 
         if (n_stages > kMaxStages) n_stages = kMaxStages;
         const int grid = n_sp < g_num_sms ? n_sp : g_num_sms;
         launch_k(conv3x3_s2_tc_kernel<CI, CO, 0>, grid, kS2Threads, s2_smem_bytes<CI, CO, 0>(n_stages), s, map, (const bf16 *)w, pk,
-                 (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages, (const bf16 *)nullptr, (const bf16 *)nullptr);
+                 (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages, (const bf16 *)nullptr, (const bf16 *)nullptr, err_word_of(s));
     } else {
         if (!get_map(src, B, Hs, Ws, CO, rows, imgs, &map)) return -1;
         int n_stages = (kSmemBudget - 9 * CI * CO * 2) / TcCfg<CO>::tile_bytes;
@@ -1408,13 +1422,13 @@ int launch_tc_s2(int dir, const void *src, const void *w, const void *w_packed, 
         const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
         launch_k(conv3x3_s2_tc_kernel<CO, CI, 1>, grid, kS2Threads, s2_smem_bytes<CO, CI, 1>(n_stages), s, map, (const bf16 *)w,
                  pk ? pk + S2Cfg<CI>::img_bytes : pk, (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages,
-                 sc.mode == 2 ? (const bf16 *)sc.a : nullptr, sc.mode == 2 ? (const bf16 *)sc.b : nullptr);
+                 sc.mode == 2 ? (const bf16 *)sc.a : nullptr, sc.mode == 2 ? (const bf16 *)sc.b : nullptr, err_word_of(s));
     }
     return 1;
 }
 
 template <int CI>
-int launch_wg_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, cudaStream_t s) {
+int launch_wg_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, Launch s) {
     constexpr int CO = 2 * CI;
     const int Hs = H / 2, Ws = W / 2;
     int rows, imgs;
@@ -1428,7 +1442,7 @@ int launch_wg_s2(const void *x, const void *dy, float *dw, float *scratch, int B
     const int max_chunks = 64;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
     launch_k(wgrad_s2_tc_kernel<CI>, chunks, kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, Hs, Ws,
-             rows, imgs, n_tiles, n_stages);
+             rows, imgs, n_tiles, n_stages, err_word_of(s));
     launch_k(wgrad_tc_fold_kernel, ceil_div(9 * CI * CO, 64), 256, 0, s, scratch, dw, chunks, CI, CO, CI);
     return 2;
 }
@@ -1450,12 +1464,12 @@ bool conv_tc_s2_supported(int B, int H, int W, int Cin, int Cout, int stride) {
 size_t tc_s2_packed_bytes(int Cin) { return 2 * (size_t)9 * Cin * 2 * Cin * 2; }
 
 int launch_conv_tc_s2(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int Cin,
-                      Shortcut sc, cudaStream_t s) {
+                      Shortcut sc, Launch s) {
     if (Cin == 16) return launch_tc_s2<16>(dir, src, w, w_packed, dst, B, H, W, sc, s);
     if (Cin == 32) return launch_tc_s2<32>(dir, src, w, w_packed, dst, B, H, W, sc, s);
     return -1;
 }
-int launch_wgrad_tc_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int Cin, cudaStream_t s) {
+int launch_wgrad_tc_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int Cin, Launch s) {
     if (Cin == 16) return launch_wg_s2<16>(x, dy, dw, scratch, B, H, W, s);
     if (Cin == 32) return launch_wg_s2<32>(x, dy, dw, scratch, B, H, W, s);
     return -1;
@@ -1474,7 +1488,7 @@ bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
 size_t tc_packed_bytes(int C) { return 2 * (size_t)9 * C * C * 2; }
 
 int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
-                   Shortcut sc, cudaStream_t s, BnFuse bf) {
+                   Shortcut sc, Launch s, BnFuse bf) {
     switch (C) {
     case 16: return launch_tc<16>(dir, src, w, w_packed, dst, B, H, W, sc, bf, s);
     case 32: return launch_tc<32>(dir, src, w, w_packed, dst, B, H, W, sc, bf, s);
@@ -1489,14 +1503,14 @@ int conv_tc_grid(int B, int H, int W) {
 }
 
 int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,
-                        cudaStream_t s) {
+                        Launch s) {
     if (n_jobs == 0) return 0;
     launch_k(pack_filters_kernel, ceil_div(total_elems, 256), 256, 0, s, (const bf16 *)wver, (uint8_t *)packed,
                                                                   (const PackJob *)jobs_dev, n_jobs, total_elems);
     return 1;
 }
 
-int launch_pack_one(const void *w, void *packed, int C, cudaStream_t s) {
+int launch_pack_one(const void *w, void *packed, int C, Launch s) {
     launch_k(pack_one_filter_kernel, ceil_div(9 * C * C, 256), 256, 0, s, (const bf16 *)w, (uint8_t *)packed, C);
     return 1;
 }
@@ -1507,7 +1521,7 @@ bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
 size_t wgrad_tc_scratch_elems() { return (size_t)kWgMaxChunks * 9 * 32 * 32 > (size_t)49 * 9 * 64 * 64 ? (size_t)kWgMaxChunks * 9 * 32 * 32 : (size_t)49 * 9 * 64 * 64; }
 
 int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C, int cin_real,
-                    cudaStream_t s) {
+                    Launch s) {
     switch (C) {
     case 16: return launch_wg<16>(x, dy, dw, scratch, B, H, W, cin_real, s);
     case 32: return launch_wg<32>(x, dy, dw, scratch, B, H, W, cin_real, s);
@@ -1522,8 +1536,26 @@ int conv_tc_error() {
     return v;
 }
 
-int conv_tc_error_async(int *pinned_dst, cudaStream_t s) {
-    return cudaMemcpyFromSymbolAsync(pinned_dst, g_tc_error, sizeof(int), 0, cudaMemcpyDeviceToHost, s) == cudaSuccess ? 0 : -1;
+// A one-CTA kernel whose only work is a bounded wait on a barrier nothing ever arrives on: no TMA, no MMA, no TMEM.
+// The wait gives up after `polls` polls, raises the error word with code 99 and the kernel returns.  It exists so that
+// the path from a wait that ran out to the host's error status can be exercised without a stuck pipeline.
+__global__ void wait_probe_kernel(int *err_word, unsigned polls) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    pdl_launch();
+    pdl_wait();
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const Waiter wt{&abort_flag, err_word, polls};
+        mbar_wait(smem_u32(&bar), 0, wt, 99);
+    }
+}
+int launch_wait_probe(unsigned polls, Launch s) {
+    if (!g_tc_error_addr) return -1;
+    launch_k(wait_probe_kernel, 1, 32, 0, s, err_word_of(s), polls);
+    return 1;
 }
 
 int conv_tc_init() {
@@ -1537,6 +1569,12 @@ int conv_tc_init() {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+    {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_tc_error);
+        if (e != cudaSuccess) { rc = (int)e; return rc; }
+        g_tc_error_addr = static_cast<int *>(p);
+    }
     const void *fns[12] = {(const void *)conv3x3_tc_kernel<16>, (const void *)conv3x3_tc_kernel<32>,
                            (const void *)conv3x3_tc_kernel<64>, (const void *)wgrad_tc_kernel<16>,
                            (const void *)wgrad_tc_kernel<32>, (const void *)wgrad_tc_kernel<64>,

@@ -29,15 +29,15 @@ struct BnFuse {
     const float *mean = nullptr, *invstd = nullptr;
 };
 int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
-                   Shortcut sc, cudaStream_t s, BnFuse bf = BnFuse());
+                   Shortcut sc, Launch s, BnFuse bf = BnFuse());
 int conv_tc_grid(int B, int H, int W);
 size_t tc_packed_bytes(int C);
 // One launch that re-arranges the filters of many convolutions of one weight version.
 // element offset in wver, byte offset in packed; pad_ = job kind: 0 stride-1 C x C filter, 1 stride-2 C -> 2C filter
 struct PackJobHost { long src_off; long dst_off; int C; int first_elem; int cin_real; int pad_; };
-int launch_pack_one(const void *w, void *packed, int C, cudaStream_t s);
+int launch_pack_one(const void *w, void *packed, int C, Launch s);
 int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, int n_jobs, int total_elems,
-                        cudaStream_t s);
+                        Launch s);
 
 // Stride-2 convolutions of the down-sampling blocks: Cout = 2 Cin, Cin in {16, 32}, even H and W, output map in whole
 // 128-pixel tiles.  H, W are the input size.  dir as above; in dir 1 sc.mode == 2 adds the gradient of the
@@ -46,21 +46,23 @@ int launch_pack_filters(const void *wver, void *packed, const void *jobs_dev, in
 bool conv_tc_s2_supported(int B, int H, int W, int Cin, int Cout, int stride);
 size_t tc_s2_packed_bytes(int Cin);
 int launch_conv_tc_s2(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int Cin,
-                      Shortcut sc, cudaStream_t s);
-int launch_wgrad_tc_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int Cin, cudaStream_t s);
+                      Shortcut sc, Launch s);
+int launch_wgrad_tc_s2(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int Cin, Launch s);
 
 bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
 size_t wgrad_tc_scratch_elems();
 // cin_real < C: x was zero-padded from cin_real to C channels; dw is the canonical [C][cin_real][3][3] gradient.
 int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C, int cin_real,
-                    cudaStream_t s);
+                    Launch s);
 
 // One-time per-process set-up (function attributes, driver entry points).  Returns a cudaError_t value.
 int conv_tc_init();
-// Error word raised by a tensor-core kernel whose bounded wait ran out (0 = none, -1 = cannot be read).
+// The process-wide error word that kernels launched without a context's own word (Launch::err == nullptr) raise when a
+// bounded wait runs out (0 = none, -1 = cannot be read).
 int conv_tc_error();
-// the same word copied into pinned host memory on a stream (0 on success); the caller synchronises the stream
-int conv_tc_error_async(int *pinned_dst, cudaStream_t s);
+// Test aid: one CTA that waits, with a limit of `polls` polls, on a barrier nothing arrives on, then raises the error
+// word of `s` with code 99 and returns.
+int launch_wait_probe(unsigned polls, Launch s);
 int conv_direct_init();
 
 }  // namespace ddg

@@ -66,6 +66,27 @@ struct Module {
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_side[4] = {nullptr, nullptr, nullptr, nullptr};
     char *dyring[4] = {nullptr, nullptr, nullptr, nullptr};  // conv-output error gradients, kept until their wgrad ran
+    // step size and Adam bias corrections of the update that runs next, device resident (recorded updates read them)
+    double *opt_dyn = nullptr;
+    double dyn_sent[3] = {0.0, 0.0, 0.0};
+    bool dyn_valid = false;
+    // debug_checks: device counters {forward iteration, backward sample, update iteration} and one stamp per activation
+    // slot, weight-version slot and error-gradient buffer: [3 counters][R][R][2]
+    long long *stamps = nullptr;
+    long long *fcount() const { return stamps; }
+    long long *bcount() const { return stamps + 1; }
+    long long *ucount() const { return stamps + 2; }
+    long long *astamp(long i) const { return stamps + 3 + i % R; }
+    long long *wstamp(long i) const { return stamps + 3 + R + i % R; }
+    long long *dstamp(long i) const { return stamps + 3 + 2 * R + i % 2; }
+};
+
+// launch counter that remembers a launcher's refusal (negative return) instead of adding it
+struct Count {
+    long n = 0;
+    bool failed = false;
+    void operator+=(int r) { if (r < 0) failed = true; else n += r; }
+    void operator+=(const Count &o) { n += o.n; failed = failed || o.failed; }
 };
 
 }  // namespace
@@ -87,9 +108,16 @@ struct ddg_ctx {
     cudaStream_t loss_stream = nullptr;  // carries the loss read-back, so that it waits for the forward sweep only
     std::vector<cudaGraphExec_t> graphs;
     std::vector<long> graph_launches;
+    bool graphs_ready = false;
     long launches = 0;
+    int *err_word = nullptr;  // device: raised by a kernel whose bounded wait ran out or by a ring-stamp mismatch
     bool broken = false;
     std::string err;
+    // how this context's kernels are launched on stream st (Launch in kernels.h)
+    Launch lx(cudaStream_t st) const {
+        const int pdl = cfg.launch_overlap == 1 ? 0 : (cfg.launch_overlap == 2 ? 1 : (K == 1 ? 1 : 2));
+        return Launch(st, pdl, K > 1, err_word);
+    }
 };
 
 namespace {
@@ -135,7 +163,7 @@ char *slot_ptr(ddg_ctx *c, TensorRef r, long iter) {
 
 // ---- convolution dispatch: tensor-core path where it applies, CUDA cores otherwise --------------------
 int conv_fwd(ddg_ctx *c, const void *x, const void *w, const void *wp, void *y, int H, int W, int Cin, int Cout,
-             int stride, int relu, cudaStream_t s) {
+             int stride, int relu, Launch s) {
     if (c->prec == P_BF16 && !relu && conv_tc_supported(c->B, H, W, Cin, Cout, stride))
         return launch_conv_tc(0, x, w, wp, y, c->B, H, W, Cin, Shortcut{}, s);
     if (c->prec == P_BF16 && !relu && conv_tc_s2_supported(c->B, H, W, Cin, Cout, stride))
@@ -143,7 +171,7 @@ int conv_fwd(ddg_ctx *c, const void *x, const void *w, const void *wp, void *y, 
     return launch_conv_fwd_direct(c->prec, x, w, y, c->B, H, W, Cin, Cout, stride, relu, s);
 }
 int conv_dgrad(ddg_ctx *c, const void *dy, const void *w, const void *wp, void *dx, int H, int W, int Cin, int Cout,
-               int stride, Shortcut sc, cudaStream_t s) {
+               int stride, Shortcut sc, Launch s) {
     if (c->prec == P_BF16 && sc.mode != 2 && conv_tc_supported(c->B, H, W, Cin, Cout, stride))
         return launch_conv_tc(1, dy, w, wp, dx, c->B, H, W, Cin, sc, s);
     if (c->prec == P_BF16 && sc.mode != 1 && conv_tc_s2_supported(c->B, H, W, Cin, Cout, stride))
@@ -151,7 +179,7 @@ int conv_dgrad(ddg_ctx *c, const void *dy, const void *w, const void *wp, void *
     return launch_conv_dgrad_direct(c->prec, dy, w, dx, c->B, H, W, Cin, Cout, stride, sc, s);
 }
 int conv_wgrad(ddg_ctx *c, Module &m, const void *x, const void *dy, float *dw, int H, int W, int Cin, int Cout,
-               int stride, cudaStream_t s) {
+               int stride, Launch s) {
     if (c->prec == P_BF16 && wgrad_tc_supported(c->B, H, W, Cin, Cout, stride))
         return launch_wgrad_tc(x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cin, s);
     if (c->prec == P_BF16 && conv_tc_s2_supported(c->B, H, W, Cin, Cout, stride))
@@ -159,22 +187,16 @@ int conv_wgrad(ddg_ctx *c, Module &m, const void *x, const void *dy, float *dw, 
     return launch_conv_wgrad_direct(c->prec, x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cout, stride, s);
 }
 
-// Batch-norm sums taken in the epilogue of the tensor-core convolution that produces the batch norm's input
-// (DDG_FUSE_BN=0 in the environment keeps the separate reduction kernels).
-bool bn_fuse_enabled() {
-    static const bool on = [] { const char *e = getenv("DDG_FUSE_BN"); return !(e && e[0] == '0'); }();
-    return on;
-}
-
 // ---- forward sweep of module k on the minibatch of iteration t (Eq. 3) --------------------------------
-long forward_module(ddg_ctx *c, int k, long t) {
+Count forward_module(ddg_ctx *c, int k, long t) {
     Module &m = c->mods[k];
-    cudaStream_t s = m.stream;
+    const Launch s = c->lx(m.stream);
     const size_t es = elem_size(c->prec);
     const char *wv = m.wver + (size_t)(t % m.R) * m.P * es;
     const char *pk = m.packed ? m.packed + (size_t)(t % m.R) * m.packed_bytes : nullptr;
     auto pkp = [&](long off) -> const void * { return (pk && off >= 0) ? pk + off : nullptr; };
-    long n = 0;
+    Count n;
+    const bool fuse_bn = !c->cfg.separate_bn_sums;
     for (int l = m.first; l <= m.last; ++l) {
         LayerPlan &L = c->layers[l];
         const char *w = wv + L.p_off * es;
@@ -224,7 +246,7 @@ long forward_module(ddg_ctx *c, int k, long t) {
             // tensor-core kernel runs, from a reduction kernel otherwise
             auto conv_bn = [&](const void *xin, const void *wc, const void *wp, void *yc, int H, int W, int Cic, int strd,
                                const char *gm, const char *bt, float *mean, float *invstd, Shortcut scb, void *dstb) {
-                if (bn_fuse_enabled() && c->prec == P_BF16 && conv_tc_supported(B, H, W, Cic, Co, strd)) {
+                if (fuse_bn && c->prec == P_BF16 && conv_tc_supported(B, H, W, Cic, Co, strd)) {
                     BnFuse bf;
                     bf.part = m.bn_scratch + 32; bf.counter = (unsigned *)m.bn_scratch; bf.o0 = mean; bf.o1 = invstd;
                     n += launch_conv_tc(0, xin, wc, wp, yc, B, H, W, Cic, Shortcut{}, s, bf);
@@ -248,19 +270,36 @@ long forward_module(ddg_ctx *c, int k, long t) {
         n += launch_softmax_ce(c->prec, (const float *)slot_ptr(c, L.out, t), c->y_stage + (size_t)(t % c->K) * c->B,
                                c->loss_dev, c->dlogits, c->B, c->classes, s);
     }
+    if (c->cfg.debug_checks) {
+        // the weight version read must be the one written for iteration t; the activation slot now holds iteration t
+        StampOp op{};
+        op.counter = m.fcount(); op.check[0] = m.wstamp(t); op.set[0] = m.astamp(t);
+        op.advance = 1; op.code = 1000 + 100 * k; op.err = c->err_word;
+        n += launch_stamp(op, s);
+    }
     return n;
 }
 
 // ---- backward sweep of module k at iteration t on the stored sample sidx = t-K+k (Eq. 6-7) ------------
-long backward_module(ddg_ctx *c, int k, long t, long sidx) {
+Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
     Module &m = c->mods[k];
-    cudaStream_t s = m.stream;
+    const Launch s = c->lx(m.stream), side = s.on(m.side);
     const size_t es = elem_size(c->prec);
     const char *wv = m.wver + (size_t)(sidx % m.R) * m.P * es;  // the weights w^s of the stored iteration
     const char *pk = m.packed ? m.packed + (size_t)(sidx % m.R) * m.packed_bytes : nullptr;
     auto pkp = [&](long off) -> const void * { return (pk && off >= 0) ? pk + off : nullptr; };
-    long n = 0;
+    Count n;
     const int B = c->B;
+    if (c->cfg.debug_checks) {
+        // activation slot and weight version must be those of sample sidx, and the incoming error gradient the one
+        // module k+1 produced for that sample; the outgoing buffer is stamped with it
+        StampOp op{};
+        op.counter = m.bcount(); op.check[0] = m.astamp(sidx); op.check[1] = m.wstamp(sidx);
+        if (k < c->K - 1) op.check[2] = c->mods[k + 1].dstamp(t + 1);
+        if (k > 0) op.set[0] = m.dstamp(t);
+        op.advance = 1; op.code = 1000 + 100 * k + 10; op.err = c->err_word;
+        n += launch_stamp(op, s);
+    }
     const char *cur = (k == c->K - 1) ? (const char *)c->dlogits : c->mods[k + 1].delta_out[(t + 1) % 2];
     int cur_tmp = -1;
     auto pick = [&](int e1, int e2) { for (int i = 0; i < 3; ++i) if (i != e1 && i != e2) return i; return 0; };
@@ -272,7 +311,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
     bool cur_sums = false;
     float *bn_part = m.bn_scratch + 32;
     unsigned *bn_counter = (unsigned *)m.bn_scratch;
-    const bool fuse = bn_fuse_enabled() && c->prec == P_BF16;
+    const bool fuse = !c->cfg.separate_bn_sums && c->prec == P_BF16;
     int dy_i = 0, last_side = -1;
     bool ring_used[4] = {false, false, false, false};
     auto ring_next = [&]() -> int {
@@ -283,7 +322,7 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
     auto side_wgrad = [&](int j, const void *x_in, const void *dy, float *gwp, int H, int W, int Ci, int Co, int st) {
         cudaEventRecord(m.ev_fork, s);
         cudaStreamWaitEvent(m.side, m.ev_fork, 0);
-        n += conv_wgrad(c, m, x_in, dy, gwp, H, W, Ci, Co, st, m.side);
+        n += conv_wgrad(c, m, x_in, dy, gwp, H, W, Ci, Co, st, side);
         cudaEventRecord(m.ev_side[j], m.side);
         ring_used[j] = true;
         last_side = j;
@@ -408,28 +447,57 @@ long backward_module(ddg_ctx *c, int k, long t, long sidx) {
 }
 
 // Re-arrange the filters of weight version `slot` into the images the tensor-core kernels copy in one piece.
-long pack_module(Module &m, int slot, size_t es) {
+int pack_module(ddg_ctx *c, Module &m, int slot) {
     if (!m.packed || m.n_pack_jobs == 0) return 0;
+    const size_t es = elem_size(c->prec);
     return launch_pack_filters(m.wver + (size_t)slot * m.P * es, m.packed + (size_t)slot * m.packed_bytes, m.pack_jobs,
-                               m.n_pack_jobs, m.pack_elems, m.stream);
+                               m.n_pack_jobs, m.pack_elems, c->lx(m.stream));
+}
+
+// Step size and Adam bias corrections of iteration t (Algorithm 1: gamma_t; Algorithm 2: 1 - beta^(t+1) with the
+// global t), as the doubles the update kernel computes with.
+void opt_scalars(const ddg_ctx *c, long t, double out[3]) {
+    out[0] = (double)c->opt.lr;
+    out[1] = out[2] = 1.0;
+    if (c->opt.kind == DDG_OPT_ADAM) {
+        out[1] = 1.0 - pow((double)c->opt.beta1, (double)(t + 1));
+        out[2] = 1.0 - pow((double)c->opt.beta2, (double)(t + 1));
+    }
+}
+
+// Bring module k's device block of optimiser scalars up to iteration t, in stream order before its update.  Never
+// called inside a capture: the recorded update reads the block, so one recording serves every step size and iteration.
+int push_opt_scalars(ddg_ctx *c, int k, long t) {
+    Module &m = c->mods[k];
+    double v[3];
+    opt_scalars(c, t, v);
+    if (m.dyn_valid && v[0] == m.dyn_sent[0] && v[1] == m.dyn_sent[1] && v[2] == m.dyn_sent[2]) return 0;
+    m.dyn_valid = true;
+    for (int i = 0; i < 3; ++i) m.dyn_sent[i] = v[i];
+    return launch_set_opt_scalars(m.opt_dyn, v[0], v[1], v[2], c->lx(m.stream));
 }
 
 // ---- update of module k with its delayed gradient (Eq. 8-9; Algorithm 1 / 2) --------------------------
-long update_module(ddg_ctx *c, int k, long t, bool have_grad) {
+Count update_module(ddg_ctx *c, int k, long t, bool have_grad) {
     Module &m = c->mods[k];
+    const Launch s = c->lx(m.stream);
+    Count n;
     UpdateArgs a{};
-    a.lr = c->opt.lr; a.mu = c->opt.momentum; a.wd = c->opt.weight_decay;
+    a.mu = c->opt.momentum; a.wd = c->opt.weight_decay;
     a.b1 = c->opt.beta1; a.b2 = c->opt.beta2; a.eps = c->opt.eps;
+    a.dyn = m.opt_dyn;
     if (!have_grad) a.mode = 2;  // Eq. 8: the delayed gradient does not exist yet; leave the module untouched
-    else if (c->opt.kind == DDG_OPT_ADAM) {
-        a.mode = 1;
-        a.c1c = 1.0 - pow((double)a.b1, (double)(t + 1));
-        a.c2c = 1.0 - pow((double)a.b2, (double)(t + 1));
-    } else a.mode = 0;
-    if (a.mode == 2 && m.R == 1) return 0;
+    else a.mode = c->opt.kind == DDG_OPT_ADAM ? 1 : 0;
+    if (c->cfg.debug_checks) {  // the slot written below holds the weights of iteration t+1
+        StampOp op{};
+        op.counter = m.ucount(); op.set[0] = m.wstamp(t + 1); op.set_add = 1;
+        op.advance = 1; op.code = 1000 + 100 * k + 20; op.err = c->err_word;
+        n += launch_stamp(op, s);
+    }
+    if (a.mode == 2 && m.R == 1) return n;
     char *wv = m.wver + (size_t)((t + 1) % m.R) * m.P * elem_size(c->prec);
-    long n = launch_update(c->prec, m.w, m.v, m.m2, m.g, wv, m.P, a, m.stream);
-    n += pack_module(m, (int)((t + 1) % m.R), elem_size(c->prec));
+    n += launch_update(c->prec, m.w, m.v, m.m2, m.g, wv, m.P, a, s);
+    n += pack_module(c, m, (int)((t + 1) % m.R));
     return n;
 }
 
@@ -437,14 +505,53 @@ long update_module(ddg_ctx *c, int k, long t, bool have_grad) {
 // (seg 1).  Inside a piece the kernels form a chain on the module's stream.
 ddg_status enqueue_segment(ddg_ctx *ctx, int k, int seg, long t, long *launches) {
     const long sidx = t - ctx->K + (k + 1);
-    long n = 0;
+    Count n;
     if (seg == 0) n += forward_module(ctx, k, t);
     else {
         if (sidx >= 0) n += backward_module(ctx, k, t, sidx);
         n += update_module(ctx, k, t, sidx >= 0);
     }
+    if (n.failed) {
+        set_err(ctx, "a kernel launcher refused its launch (tensor map or shared-memory plan) in module %d", k);
+        return DDG_ERR_CUDA;
+    }
     CU(cudaGetLastError());
-    *launches = n;
+    *launches = n.n;
+    return DDG_OK;
+}
+
+// Record the CUDA graph of piece (k, seg) for the ring phase of iteration t (nothing runs).
+ddg_status capture_segment(ddg_ctx *ctx, int k, int seg, long t) {
+    Module &m = ctx->mods[k];
+    const size_t idx = ((size_t)(t % ctx->period) * ctx->K + k) * 2 + seg;
+    if (ctx->graphs[idx]) return DDG_OK;
+    CU(cudaStreamBeginCapture(m.stream, cudaStreamCaptureModeThreadLocal));
+    long n = 0;
+    ddg_status st = enqueue_segment(ctx, k, seg, t, &n);
+    cudaGraph_t graph = nullptr;
+    cudaError_t e2 = cudaStreamEndCapture(m.stream, &graph);
+    if (st != DDG_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+    CU(e2);
+    cudaGraphExec_t exec = nullptr;
+    cudaError_t e3 = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    CU(e3);
+    ctx->graphs[idx] = exec;
+    ctx->graph_launches[idx] = n;
+    return DDG_OK;
+}
+
+// Record every piece of every ring phase at once, at the first steady-state iteration t0: what a piece launches
+// depends on the iteration only through its ring slots (t mod R_k, t mod K, t mod 2), which repeat with the period, so
+// phase p is recorded from the first iteration >= t0 that falls into it.  Afterwards every iteration is replay only.
+ddg_status capture_all(ddg_ctx *ctx, long t0) {
+    for (long t = t0; t < t0 + ctx->period; ++t)
+        for (int k = 0; k < ctx->K; ++k)
+            for (int seg = 0; seg < 2; ++seg) {
+                ddg_status st = capture_segment(ctx, k, seg, t);
+                if (st != DDG_OK) return st;
+            }
+    ctx->graphs_ready = true;
     return DDG_OK;
 }
 
@@ -454,28 +561,16 @@ ddg_status enqueue_segment(ddg_ctx *ctx, int k, int seg, long t, long *launches)
 // events, so consecutive iterations overlap exactly as they do without graphs.
 ddg_status run_segment(ddg_ctx *ctx, int k, int seg, long t, bool use_graph, long *launches) {
     Module &m = ctx->mods[k];
-    // Adam's bias corrections change every iteration, so an update with them cannot be replayed from a recording
-    if (use_graph && seg == 1 && ctx->opt.kind == DDG_OPT_ADAM) use_graph = false;
-    if (!use_graph) return enqueue_segment(ctx, k, seg, t, launches);
-    const int phase = (int)(t % ctx->period);
-    const size_t idx = ((size_t)phase * ctx->K + k) * 2 + seg;
-    if (!ctx->graphs[idx]) {
-        CU(cudaStreamBeginCapture(m.stream, cudaStreamCaptureModeThreadLocal));
-        long n = 0;
-        ddg_status st = enqueue_segment(ctx, k, seg, t, &n);
-        cudaGraph_t graph = nullptr;
-        cudaError_t e2 = cudaStreamEndCapture(m.stream, &graph);
-        if (st != DDG_OK) { if (graph) cudaGraphDestroy(graph); return st; }
-        CU(e2);
-        cudaGraphExec_t exec = nullptr;
-        cudaError_t e3 = cudaGraphInstantiate(&exec, graph, 0);
-        cudaGraphDestroy(graph);
-        CU(e3);
-        ctx->graphs[idx] = exec;
-        ctx->graph_launches[idx] = n;
+    long extra = 0;
+    if (seg == 1 && t - ctx->K + (k + 1) >= 0) extra = push_opt_scalars(ctx, k, t);
+    if (!use_graph) {
+        ddg_status st = enqueue_segment(ctx, k, seg, t, launches);
+        *launches += extra;
+        return st;
     }
+    const size_t idx = ((size_t)(t % ctx->period) * ctx->K + k) * 2 + seg;
     CU(cudaGraphLaunch(ctx->graphs[idx], m.stream));
-    *launches = ctx->graph_launches[idx];
+    *launches = ctx->graph_launches[idx] + extra;
     return DDG_OK;
 }
 
@@ -540,23 +635,36 @@ ddg_status init_weights(ddg_ctx *ctx) {
         default: break;
         }
     }
-    for (auto &m : ctx->mods) { launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream); pack_module(m, 0, elem_size(ctx->prec)); }
+    for (auto &m : ctx->mods) { launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream); pack_module(ctx, m, 0); }
     CU(cudaGetLastError());
     for (auto &m : ctx->mods) CU(cudaStreamSynchronize(m.stream));
     return DDG_OK;
 }
 
-// error words raised by kernels whose bounded waits ran out (reads the flags as they are now; does not wait)
-ddg_status check_kernel_errors(ddg_ctx *ctx) {
-    if (ctx->prec == P_BF16) {
-        const int code = conv_tc_error();
-        if (code != 0) {
-            set_err(ctx, "a tensor-core kernel gave up on a bounded wait (code %d)", code);
-            ctx->broken = true;
-            return code > 0 ? DDG_ERR_TIMEOUT : DDG_ERR_CUDA;
-        }
+// Turn a raised error word into the context's error state.  Codes below 1000: the bounded wait with that code ran
+// out.  1000 + 100 * module + check: a ring-slot stamp did not match (debug_checks).
+ddg_status report_error_word(ddg_ctx *ctx, int code) {
+    if (code == 0) return DDG_OK;
+    ctx->broken = true;
+    if (code >= 1000) {
+        static const char *const what[] = {"weight version read by the forward sweep", "?", "?", "?", "?", "?", "?", "?", "?", "?",
+                                           "activation slot read by the backward sweep",
+                                           "weight version read by the backward sweep",
+                                           "error gradient received from the next module"};
+        const int which = (code - 1000) % 100;
+        set_err(ctx, "ring stamp mismatch in module %d: %s is not the one the iteration expects", (code - 1000) / 100,
+                which < 13 ? what[which] : "?");
+        return DDG_ERR_STATE;
     }
-    return DDG_OK;
+    set_err(ctx, "a kernel gave up on a bounded wait (code %d)", code);
+    return DDG_ERR_TIMEOUT;
+}
+
+// reads the error word as it is now (does not wait for work in flight)
+ddg_status check_kernel_errors(ddg_ctx *ctx) {
+    int code = 0;
+    CU(cudaMemcpy(&code, ctx->err_word, sizeof(int), cudaMemcpyDeviceToHost));
+    return report_error_word(ctx, code);
 }
 
 ddg_status sync_all(ddg_ctx *ctx) {
@@ -567,23 +675,6 @@ ddg_status sync_all(ddg_ctx *ctx) {
 }  // namespace
 
 namespace ddg {
-// Programmatic dependent launch: the next kernel of a stream is placed while this one still runs, so that its launch
-// latency and set-up hide under this one's tail.  Where one stream has the GPU to itself (K = 1, single kernels) every
-// launch carries the attribute.  With several module streams it depends on what the early-placed kernel holds while
-// it waits: the element-wise batch-norm passes (three CTAs of 256 threads and ~70 registers per SM, all SMs) keep the
-// other modules' tensor-core CTAs off the SMs, and the attribute on them alone costs the K = 4 iteration 15 % (1.82 ->
-// 2.10 ms, ResNet-110 batch 128); on the weight-gradient kernel and its fold, which run on side streams, 1 - 5 %.  On
-// the forward / input-gradient convolution alone it gains 5 % (1.82 -> 1.73 ms; end to end 53 400 -> 57 500 images/s).
-// So the engine clears the flag below while it enqueues an iteration of a multi-module network, and only launches that
-// pass `while_shared` (that convolution) keep the attribute then.  DDG_PDL=0 / 1 in the environment forces it off / on.
-thread_local bool t_pdl_wanted = true;
-bool pdl_enabled(bool while_shared) {
-    static const int forced = [] { const char *e = getenv("DDG_PDL"); return e ? (e[0] == '0' ? 0 : 1) : -1; }();
-    return forced >= 0 ? forced == 1 : (t_pdl_wanted || while_shared);
-}
-// True while the engine enqueues an iteration of a multi-module network: the launchers then size grids so that SMs are
-// left over for the other modules' kernels where that costs the kernel itself nothing.
-bool gpu_shared_by_streams() { return !t_pdl_wanted; }
 // lets the other translation units leave a message for ddg_last_error(NULL)
 void set_global_error(const char *msg) { g_create_error = msg; }
 }  // namespace ddg
@@ -610,6 +701,7 @@ void ddg_destroy(ddg_ctx *ctx) {
         if (m.ev_fork) cudaEventDestroy(m.ev_fork);
         for (auto e : m.ev_side) if (e) cudaEventDestroy(e);
         cudaFree(m.bn_scratch); cudaFree(m.wg_scratch);
+        cudaFree(m.opt_dyn); cudaFree(m.stamps);
         cudaFree(m.delta_out[0]); cudaFree(m.delta_out[1]);
         if (m.ev_fwd) cudaEventDestroy(m.ev_fwd);
         if (m.ev_bwd) cudaEventDestroy(m.ev_bwd);
@@ -617,6 +709,7 @@ void ddg_destroy(ddg_ctx *ctx) {
         if (m.own_stream && m.stream) cudaStreamDestroy(m.stream);
     }
     cudaFree(ctx->x_stage); cudaFree(ctx->y_stage); cudaFree(ctx->dlogits); cudaFree(ctx->loss_dev);
+    cudaFree(ctx->err_word);
     if (ctx->pinned_loss) cudaFreeHost(ctx->pinned_loss);
     if (ctx->loss_stream) cudaStreamDestroy(ctx->loss_stream);
     delete ctx;
@@ -637,6 +730,7 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
         return DDG_ERR_INVALID_ARG;
     }
     if (opt->kind != DDG_OPT_SGD && opt->kind != DDG_OPT_ADAM) { set_err(nullptr, "ddg_create: unknown optimiser"); return DDG_ERR_INVALID_ARG; }
+    if (cfg->launch_overlap < 0 || cfg->launch_overlap > 2) { set_err(nullptr, "ddg_create: launch_overlap must be 0, 1 or 2"); return DDG_ERR_INVALID_ARG; }
     for (int k = 0; k + 1 < K; ++k)
         if (split_after[k] < 0 || split_after[k] >= n_layers - 1 || (k > 0 && split_after[k] <= split_after[k - 1])) {
             set_err(nullptr, "ddg_create: split points must be strictly increasing layer indices in [0, n_layers-2]");
@@ -768,6 +862,15 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
         CU(cudaMemset(m.wver, 0, pn * es * m.R));
         for (auto &p : m.tmp) CU(cudaMalloc(&p, m.tmp_bytes));
         for (auto &p : m.dyring) CU(cudaMalloc(&p, m.tmp_bytes));
+        CU(cudaMalloc(&m.opt_dyn, 3 * sizeof(double)));
+        CU(cudaMemset(m.opt_dyn, 0, 3 * sizeof(double)));
+        {   // ring stamps: counters 0; activation stamps -1 (nothing written); weight version 0 sits in slot 0
+            std::vector<long long> init(3 + 2 * (size_t)m.R + 2, -1);
+            init[0] = init[1] = init[2] = 0;
+            init[3 + m.R] = 0;
+            CU(cudaMalloc(&m.stamps, init.size() * sizeof(long long)));
+            CU(cudaMemcpy(m.stamps, init.data(), init.size() * sizeof(long long), cudaMemcpyHostToDevice));
+        }
         CU(cudaStreamCreateWithFlags(&m.side, cudaStreamNonBlocking));
         CU(cudaEventCreateWithFlags(&m.ev_fork, cudaEventDisableTiming));
         for (auto &e : m.ev_side) CU(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
@@ -837,6 +940,8 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
     CU(cudaMalloc(&c->dlogits, (size_t)c->B * c->classes * 4));
     CU(cudaMalloc(&c->loss_dev, 4));
     CU(cudaMemset(c->loss_dev, 0, 4));
+    CU(cudaMalloc(&c->err_word, sizeof(int)));  // this context's own error word, clear at creation
+    CU(cudaMemset(c->err_word, 0, sizeof(int)));
     CU(cudaMallocHost(&c->pinned_loss, 8));  // the loss, and the tensor-core kernels' error word read with it
     CU(cudaStreamCreateWithFlags(&c->loss_stream, cudaStreamNonBlocking));
     // the memsets above ran on the legacy default stream, which the non-blocking module streams do not wait for
@@ -858,9 +963,11 @@ static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float 
     CU(cudaMemcpyAsync(ctx->y_stage + (size_t)(t % K) * ctx->B, y, (size_t)ctx->B * 4, kind, s0));
     // the first K-1 iterations have modules in warm-up and a different shape: they are not recorded
     const bool steady = t >= K - 1;
-    ddg::t_pdl_wanted = ctx->K == 1;
+    if (ctx->cfg.use_graph && steady && !ctx->graphs_ready) {
+        ddg_status cs = capture_all(ctx, t);
+        if (cs != DDG_OK) { ctx->broken = true; return cs; }
+    }
     ddg_status st = enqueue_iteration(ctx, t, ctx->cfg.use_graph && steady, &ctx->launches);
-    ddg::t_pdl_wanted = true;
     if (st != DDG_OK) { ctx->broken = true; return st; }
     ctx->t = t + 1;
     if (loss_host) {
@@ -871,14 +978,10 @@ static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float 
         // error flags raised so far ride along (a later call or ddg_sync reports what is still running): one host wait
         int *flag = reinterpret_cast<int *>(ctx->pinned_loss + 1);
         *flag = 0;
-        if (ctx->prec == P_BF16 && conv_tc_error_async(flag, ctx->loss_stream) != 0) return DDG_ERR_CUDA;
+        CU(cudaMemcpyAsync(flag, ctx->err_word, sizeof(int), cudaMemcpyDeviceToHost, ctx->loss_stream));
         CU(cudaStreamSynchronize(ctx->loss_stream));
         *loss_host = *ctx->pinned_loss;
-        if (*flag != 0) {
-            set_err(ctx, "a tensor-core kernel gave up on a bounded wait (code %d)", *flag);
-            ctx->broken = true;
-            return DDG_ERR_TIMEOUT;
-        }
+        if (*flag != 0) return report_error_word(ctx, *flag);
     }
     return DDG_OK;
 }
@@ -894,12 +997,8 @@ ddg_status ddg_step_host(ddg_ctx *ctx, const float *x_host, const int *y_host, f
 ddg_status ddg_set_lr(ddg_ctx *ctx, float lr) {
     if (!ctx) return DDG_ERR_INVALID_ARG;
     if (ctx->broken) return DDG_ERR_STATE;
-    if (lr != ctx->opt.lr) {
-        // captured graphs have the step size baked into their update nodes: drop them, they are re-recorded
-        ddg_status st = sync_all(ctx);
-        if (st != DDG_OK) return st;
-        for (auto &g : ctx->graphs) if (g) { cudaGraphExecDestroy(g); g = nullptr; }
-    }
+    // the updates (recorded or not) read the step size from a device block that each module's stream refreshes, in
+    // order, before its next update: nothing in flight is disturbed and nothing is re-recorded
     ctx->opt.lr = lr;
     return DDG_OK;
 }
@@ -933,7 +1032,7 @@ ddg_status ddg_set_weights(ddg_ctx *ctx, const float *src, size_t n, int on_devi
         if (m.m2) CU(cudaMemset(m.m2, 0, m.P * 4));
     }
     CU(cudaDeviceSynchronize());  // default-stream copies and memsets are not ordered against the module streams
-    for (auto &m : ctx->mods) { launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream); pack_module(m, 0, elem_size(ctx->prec)); }
+    for (auto &m : ctx->mods) { launch_cast(ctx->prec, m.w, m.wver, m.P, m.stream); pack_module(ctx, m, 0); }
     CU(cudaGetLastError());
     return sync_all(ctx);
 }
@@ -963,6 +1062,26 @@ ddg_status ddg_get_loss_dev(ddg_ctx *ctx, const float **loss_dev) {
 ddg_status ddg_last_step_launches(const ddg_ctx *ctx, long *launches) {
     if (!ctx || !launches) return DDG_ERR_INVALID_ARG;
     *launches = ctx->launches;
+    return DDG_OK;
+}
+
+ddg_status ddg_debug_wait_timeout(ddg_ctx *ctx, unsigned polls) {
+    if (!ctx || polls == 0) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    if (launch_wait_probe(polls, ctx->lx(ctx->mods[0].stream)) < 0) {
+        set_err(ctx, "ddg_debug_wait_timeout: the tensor-core path is not initialised");
+        return DDG_ERR_CUDA;
+    }
+    CU(cudaGetLastError());
+    return DDG_OK;
+}
+
+ddg_status ddg_debug_shift_stamps(ddg_ctx *ctx, int k, long delta) {
+    if (!ctx || k < 0 || k >= ctx->K) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    if (!ctx->cfg.debug_checks) { set_err(ctx, "ddg_debug_shift_stamps: the context was created without debug_checks"); return DDG_ERR_STATE; }
+    launch_add_to_counter(ctx->mods[k].fcount(), (long long)delta, ctx->lx(ctx->mods[k].stream));
+    CU(cudaGetLastError());
     return DDG_OK;
 }
 

@@ -125,7 +125,7 @@ conv3x3_direct_kernel(const T *__restrict__ src, const T *__restrict__ w, T *__r
 
 template <typename T, int DGRAD>
 static void conv_direct_launch(const void *src, const void *w, void *dst, int B, int Hs, int Ws, int Cs, int Hd,
-                               int Wd, int Cd, int stride, int relu, Shortcut sc, cudaStream_t s) {
+                               int Wd, int Cd, int stride, int relu, Shortcut sc, Launch s) {
     const size_t smem = (size_t)9 * Cs * Cd * sizeof(float);
     const int groups = (Cd + kCdt - 1) / kCdt;
     const int pix_per_cta = kConvThreads / groups;
@@ -147,7 +147,7 @@ int conv_direct_init() {
 }
 
 int launch_conv_fwd_direct(int prec, const void *x, const void *w, void *y, int B, int H, int W, int Cin, int Cout,
-                           int stride, int relu, cudaStream_t s) {
+                           int stride, int relu, Launch s) {
     const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
     Shortcut none = {};
     DISPATCH_PREC(prec, (conv_direct_launch<T, 0>(x, w, y, B, H, W, Cin, Ho, Wo, Cout, stride, relu, none, s)));
@@ -155,7 +155,7 @@ int launch_conv_fwd_direct(int prec, const void *x, const void *w, void *y, int 
 }
 
 int launch_conv_dgrad_direct(int prec, const void *dy, const void *w, void *dx, int B, int H, int W, int Cin, int Cout,
-                             int stride, Shortcut sc, cudaStream_t s) {
+                             int stride, Shortcut sc, Launch s) {
     const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
     DISPATCH_PREC(prec, (conv_direct_launch<T, 1>(dy, w, dx, B, Ho, Wo, Cout, H, W, Cin, stride, 0, sc, s)));
     return 1;
@@ -253,7 +253,7 @@ __global__ void conv3x3_wgrad_fold_kernel(const A *__restrict__ part, float *__r
 }
 
 int launch_conv_wgrad_direct(int prec, const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W,
-                             int Cin, int Cout, int stride, cudaStream_t s) {
+                             int Cin, int Cout, int stride, Launch s) {
     const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
     const int chunks = wgrad_chunks(B, Ho);
     const int cigs = kWgThreads / Cout;  // host guarantees Cout <= 256

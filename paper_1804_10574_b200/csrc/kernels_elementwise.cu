@@ -31,7 +31,7 @@ __global__ void shim_kernel(const float *__restrict__ x, T *__restrict__ out, in
     for (int c = C; c < Cpad; ++c) out[i * Cpad + c] = from_f<T>(0.f);  // zero channels up to the padded width
 }
 
-int launch_shim(int prec, const float *x, void *out, int B, int C, int H, int W, int Cpad, cudaStream_t s) {
+int launch_shim(int prec, const float *x, void *out, int B, int C, int H, int W, int Cpad, Launch s) {
     long n = (long)B * H * W;
     DISPATCH_PREC(prec, launch_k(shim_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, x, (T *)out, B, C, H * W, Cpad));
     return 1;
@@ -52,11 +52,11 @@ template <typename T> __global__ void relu_bwd_kernel(const T *y, const T *dy, T
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) dx[i] = to_f(y[i]) > 0.f ? dy[i] : from_f<T>(0.f);
 }
-int launch_relu_fwd(int prec, const void *x, void *y, size_t n, cudaStream_t s) {
+int launch_relu_fwd(int prec, const void *x, void *y, size_t n, Launch s) {
     DISPATCH_PREC(prec, launch_k(relu_fwd_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, (const T *)x, (T *)y, n));
     return 1;
 }
-int launch_relu_bwd(int prec, const void *y, const void *dy, void *dx, size_t n, cudaStream_t s) {
+int launch_relu_bwd(int prec, const void *y, const void *dy, void *dx, size_t n, Launch s) {
     DISPATCH_PREC(prec, launch_k(relu_bwd_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, (const T *)y, (const T *)dy,
                                                                                       (T *)dx, n));
     return 1;
@@ -93,11 +93,11 @@ template <typename T> __global__ void avgpool_bwd_kernel(const T *dy, T *dx, int
     typedef typename AccOf<T>::type A;
     dx[i] = from_a<T>((A)to_f(dy[b * C + c]) / (A)HW);
 }
-int launch_avgpool_fwd(int prec, const void *x, void *y, int B, int HW, int C, cudaStream_t s) {
+int launch_avgpool_fwd(int prec, const void *x, void *y, int B, int HW, int C, Launch s) {
     DISPATCH_PREC(prec, launch_k(avgpool_fwd_kernel<T>, B, kThreads, 0, s, (const T *)x, (T *)y, HW, C));
     return 1;
 }
-int launch_avgpool_bwd(int prec, const void *dy, void *dx, int B, int HW, int C, cudaStream_t s) {
+int launch_avgpool_bwd(int prec, const void *dy, void *dx, int B, int HW, int C, Launch s) {
     size_t n = (size_t)B * HW * C;
     DISPATCH_PREC(prec, launch_k(avgpool_bwd_kernel<T>, ceil_div(n, kThreads), kThreads, 0, s, (const T *)dy, (T *)dx, HW,
                                                                                         C, n));
@@ -167,7 +167,7 @@ __global__ void fc_dw_kernel(const T *x, const TO *y, const TO *dy, float *dW, f
     }
 }
 int launch_fc_fwd(int prec, const void *x, const void *W, const void *bias, void *y, int B, int in, int out, int relu,
-                  int out_f32, cudaStream_t s) {
+                  int out_f32, Launch s) {
     long threads = (long)B * out * 32;
     DISPATCH_PREC(prec, {
         if (out_f32)
@@ -182,7 +182,7 @@ int launch_fc_fwd(int prec, const void *x, const void *W, const void *bias, void
     return 1;
 }
 int launch_fc_bwd(int prec, const void *x, const void *W, const void *y, const void *dy, void *dx, float *dW, float *db,
-                  int B, int in, int out, int relu, int out_f32, cudaStream_t s) {
+                  int B, int in, int out, int relu, int out_f32, Launch s) {
     int n = 0;
     DISPATCH_PREC(prec, {
         if (out_f32) {
@@ -233,7 +233,7 @@ __global__ void softmax_ce_kernel(const float *logits, const int *labels, float 
     }
 }
 int launch_softmax_ce(int prec, const float *logits, const int *labels, float *loss, float *dlogits, int B, int C,
-                      cudaStream_t s) {
+                      Launch s) {
     if (prec == P_BF16) launch_k(softmax_ce_kernel<float>, 1, 1024, 0, s, logits, labels, loss, dlogits, B, C);
     else launch_k(softmax_ce_kernel<double>, 1, 1024, 0, s, logits, labels, loss, dlogits, B, C);
     return 1;
@@ -623,7 +623,7 @@ static int red_big_grid(long nvec, int U) {
 template <typename T> static int vec_for(int C) { return (C % Vec16<T>::N == 0) ? Vec16<T>::N : 1; }
 
 int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *scratch, long npix, int C,
-                    cudaStream_t s) {
+                    Launch s) {
     if (red_big_ok(prec, npix * (C / 8), C)) {
         launch_k(bn_reduce_big_kernel<0, 4>, red_big_grid(npix * (C / 8), 4), kBigThreads, 0, s, (const bf16 *)x, (const bf16 *)nullptr,
                  (const bf16 *)nullptr, (const float *)nullptr, (const float *)nullptr, mean, invstd, scratch, npix, C, 0);
@@ -646,7 +646,7 @@ int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *
 
 int launch_bn_bwd_reduce(int prec, const void *dout, const void *out, const void *x, const float *mean,
                          const float *invstd, float *dgamma, float *dbeta, float *scratch, long npix, int C, int relu,
-                         cudaStream_t s) {
+                         Launch s) {
     if (red_big_ok(prec, npix * (C / 8), C)) {
         launch_k(bn_reduce_big_kernel<1, 2>, red_big_grid(npix * (C / 8), 2), kBigThreads, 0, s, (const bf16 *)x, (const bf16 *)dout,
                  (const bf16 *)out, mean, invstd, dbeta, dgamma, scratch, npix, C, relu);
@@ -792,7 +792,7 @@ static int apply_grid(long nvec, int U) {
 }
 
 int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta, const float *mean,
-                    const float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu, cudaStream_t s) {
+                    const float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu, Launch s) {
     const long npix = (long)B * H * W;
     if (prec == P_BF16 && sc.mode != 2 && apply_fast_ok(C, Vec16<bf16>::N)) {
         typedef bf16 T;
@@ -913,7 +913,7 @@ bn_bwd_apply_fast_kernel(const bf16 *__restrict__ dout, const bf16 *__restrict__
 
 int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void *x, const void *gamma,
                         const float *mean, const float *invstd, const float *dgamma, const float *dbeta, void *dx,
-                        long npix, int C, int relu, cudaStream_t s) {
+                        long npix, int C, int relu, Launch s) {
     if (prec == P_BF16 && apply_fast_ok(C, Vec16<bf16>::N)) {
         typedef bf16 T;
         constexpr int V = Vec16<T>::N;
@@ -945,19 +945,20 @@ int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void 
 static constexpr int kUpdVecs = 2;  // float4 groups per thread, all loads issued before the first use
 
 // one parameter: master weight, first (and second) moment, gradient
+// lr, c1c, c2c: the step size and Adam's bias corrections of this iteration (by value or from the device block)
 template <typename A>
-__device__ __forceinline__ void update_one(float &w, float &v, float &m2, float g, const UpdateArgs &a) {
+__device__ __forceinline__ void update_one(float &w, float &v, float &m2, float g, const UpdateArgs &a, A lr, A c1c, A c2c) {
     if (a.mode == 0) {
         const A d = (A)g + (A)a.wd * (A)w;
         const A vn = (A)a.mu * (A)v + d;
         v = (float)vn;
-        w = (float)((A)w - (A)a.lr * vn);
+        w = (float)((A)w - lr * vn);
     } else if (a.mode == 1) {
         const A m1 = (A)a.b1 * (A)v + ((A)1 - (A)a.b1) * (A)g;
         const A m2n = (A)a.b2 * (A)m2 + ((A)1 - (A)a.b2) * (A)g * (A)g;
         v = (float)m1;
         m2 = (float)m2n;
-        w = (float)((A)w - (A)a.lr * (m1 / (A)a.c1c) / (sqrt(m2n / (A)a.c2c) + (A)a.eps));
+        w = (float)((A)w - lr * (m1 / c1c) / (sqrt(m2n / c2c) + (A)a.eps));
     }
 }
 
@@ -968,6 +969,8 @@ update_kernel(float *__restrict__ w, float *__restrict__ v, float *__restrict__ 
     pdl_launch();
     pdl_wait();
     typedef typename AccOf<T>::type A;  // the master state is fp32 either way; A is the arithmetic in between
+    const A lr = a.dyn ? (A)a.dyn[0] : (A)a.lr;
+    const A c1c = a.dyn ? (A)a.dyn[1] : (A)a.c1c, c2c = a.dyn ? (A)a.dyn[2] : (A)a.c2c;
     const size_t span = (size_t)gridDim.x * blockDim.x * 4;  // elements one pass of the grid covers
     const size_t base = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(g) |
@@ -987,10 +990,10 @@ update_kernel(float *__restrict__ w, float *__restrict__ v, float *__restrict__ 
 #pragma unroll
         for (int u = 0; u < kUpdVecs; ++u) {
             const size_t i = base + u * span;
-            update_one<A>(W[u].x, V[u].x, M[u].x, G[u].x, a);
-            update_one<A>(W[u].y, V[u].y, M[u].y, G[u].y, a);
-            update_one<A>(W[u].z, V[u].z, M[u].z, G[u].z, a);
-            update_one<A>(W[u].w, V[u].w, M[u].w, G[u].w, a);
+            update_one<A>(W[u].x, V[u].x, M[u].x, G[u].x, a, lr, c1c, c2c);
+            update_one<A>(W[u].y, V[u].y, M[u].y, G[u].y, a, lr, c1c, c2c);
+            update_one<A>(W[u].z, V[u].z, M[u].z, G[u].z, a, lr, c1c, c2c);
+            update_one<A>(W[u].w, V[u].w, M[u].w, G[u].w, a, lr, c1c, c2c);
             if (a.mode != 2) {
                 *reinterpret_cast<float4 *>(w + i) = W[u];
                 *reinterpret_cast<float4 *>(v + i) = V[u];
@@ -1007,7 +1010,7 @@ update_kernel(float *__restrict__ w, float *__restrict__ v, float *__restrict__ 
             if (i >= n) break;
             float wi = w[i], vi = 0.f, mi = 0.f, gi = 0.f;
             if (a.mode != 2) { vi = v[i]; gi = g[i]; if (a.mode == 1) mi = m2[i]; }
-            update_one<A>(wi, vi, mi, gi, a);
+            update_one<A>(wi, vi, mi, gi, a, lr, c1c, c2c);
             if (a.mode != 2) { w[i] = wi; v[i] = vi; if (a.mode == 1) m2[i] = mi; }
             wv[i] = from_f<T>(wi);
         }
@@ -1015,13 +1018,48 @@ update_kernel(float *__restrict__ w, float *__restrict__ v, float *__restrict__ 
 }
 
 int launch_update(int prec, float *w, float *v, float *m2, const float *g, void *wv, size_t n, UpdateArgs a,
-                  cudaStream_t s) {
+                  Launch s) {
     if (n == 0) return 0;
     DISPATCH_PREC(prec, launch_k(update_kernel<T>, ceil_div((n + 3) / 4, (long)kThreads * kUpdVecs), kThreads, 0, s, w, v, m2, g, (T *)wv, n, a));
     return 1;
 }
 
-int launch_cast(int prec, const float *src, void *dst, size_t n, cudaStream_t s) {
+__global__ void set_opt_scalars_kernel(double *dyn, double lr, double c1c, double c2c) {
+    pdl_launch();
+    pdl_wait();
+    if (threadIdx.x == 0) { dyn[0] = lr; dyn[1] = c1c; dyn[2] = c2c; }
+}
+int launch_set_opt_scalars(double *dyn, double lr, double c1c, double c2c, Launch s) {
+    launch_k(set_opt_scalars_kernel, 1, 32, 0, s, dyn, lr, c1c, c2c);
+    return 1;
+}
+
+__global__ void stamp_kernel(StampOp op) {
+    pdl_launch();
+    pdl_wait();
+    if (threadIdx.x != 0) return;
+    const long long now = *op.counter;
+    for (int i = 0; i < 3; ++i)
+        if (op.check[i] != nullptr && *op.check[i] != now) atomicCAS(op.err, 0, op.code + i);
+    for (int i = 0; i < 2; ++i)
+        if (op.set[i] != nullptr) *op.set[i] = now + op.set_add;
+    *op.counter = now + op.advance;
+}
+int launch_stamp(StampOp op, Launch s) {
+    launch_k(stamp_kernel, 1, 32, 0, s, op);
+    return 1;
+}
+__global__ void add_to_counter_kernel(long long *counter, long long delta) {
+    pdl_launch();
+    pdl_wait();
+    if (threadIdx.x == 0) *counter += delta;
+}
+int launch_add_to_counter(long long *counter, long long delta, Launch s) {
+    launch_k(add_to_counter_kernel, 1, 32, 0, s, counter, delta);
+    return 1;
+}
+
+int launch_cast(int prec, const float *src, void *dst, size_t n, Launch s) {
     UpdateArgs a = {};
     a.mode = 2;
     return launch_update(prec, const_cast<float *>(src), nullptr, nullptr, nullptr, dst, n, a, s);
@@ -1055,12 +1093,12 @@ __global__ void fill_const_kernel(float *dst, size_t n, float v) {
     if (i < n) dst[i] = v;
 }
 int launch_fill_normal(float *dst, size_t n, float stddev, unsigned long long seed, unsigned long long stream_id,
-                       cudaStream_t s) {
+                       Launch s) {
     if (n == 0) return 0;
     launch_k(fill_normal_kernel, ceil_div(n, kThreads), kThreads, 0, s, dst, n, stddev, seed, stream_id);
     return 1;
 }
-int launch_fill_const(float *dst, size_t n, float v, cudaStream_t s) {
+int launch_fill_const(float *dst, size_t n, float v, Launch s) {
     if (n == 0) return 0;
     launch_k(fill_const_kernel, ceil_div(n, kThreads), kThreads, 0, s, dst, n, v);
     return 1;

@@ -6,16 +6,21 @@ import pytest
 import torch
 
 from paper_1804_10574_b200 import nets
-from tests.parity import rel, run_pair
+from tests.parity import rel, run_pair  # noqa: F401
 
 pytestmark = pytest.mark.gpu
 
 FP32_TOL, BF16_TOL, LOSS_TOL = 1e-4, 2e-2, 1e-3
+RESNET8_FP32_VS_EXACT = 5e-2   # measured worst over 20 iterations: see the test
+RATIO_BAND = (0.6, 1.4)        # median of rel(gpu, exact) / rel(oracle_bf16, exact) over gradient tensors
 
 
 def test_mlp_k2_20_steps_fp32():
-    w = run_pair(nets.config("mlp"), 20, FP32_TOL, LOSS_TOL)
+    """Config 1.  Also against the exact oracle (no storage rounding anywhere): a network this small meets no ReLU
+    pre-activation within fp32 rounding of zero, so the fp32 path stays within the fp32 bar of the exact run too."""
+    w = run_pair(nets.config("mlp"), 20, FP32_TOL, LOSS_TOL, exact_too=True)
     print("mlp K=2 worst", w)
+    assert w["grad_vs_exact"] <= FP32_TOL and w["weight_vs_exact"] <= FP32_TOL
 
 
 @pytest.mark.parametrize("splits", [[], [0], [0, 1, 2]], ids=["K1", "K2_early", "K4"])
@@ -38,8 +43,44 @@ def test_mlp_diminishing_stepsize_fp32():
 
 
 def test_resnet8_k2_20_steps_fp32():
-    w = run_pair(nets.config("resnet8"), 20, FP32_TOL, LOSS_TOL)
+    """Config 2.  Bit-level agreement is with the oracle that stores fp32 where the kernels do.  Against the exact
+    oracle the loss trajectory is held to the same 1e-3; gradients and weights are reported (2.4 M ReLU decisions per
+    iteration: the few whose pre-activation lies within fp32 rounding of zero fall differently in the two runs, and
+    lr 0.1 with momentum 0.9 amplifies each such event), with a bar an order above what is seen."""
+    w = run_pair(nets.config("resnet8"), 20, FP32_TOL, LOSS_TOL, exact_too=True)
     print("resnet8 K=2 worst", w)
+    assert w["grad_vs_exact"] <= RESNET8_FP32_VS_EXACT and w["weight_vs_exact"] <= RESNET8_FP32_VS_EXACT
+
+
+def test_resnet8_first_steps_fp32_vs_exact():
+    """Before any ReLU decision has had time to be amplified (three iterations from identical weights) the fp32 path is
+    within the fp32 bar of the exact oracle as well."""
+    w = run_pair(nets.config("resnet8"), 3, FP32_TOL, LOSS_TOL, exact_too=True)
+    print("resnet8 first steps vs exact", w)
+    assert w["grad_vs_exact"] <= FP32_TOL and w["weight_vs_exact"] <= FP32_TOL
+
+
+@pytest.mark.parametrize("net,splits,batch", [("mlp", [0, 1], 16), ("mlp", [0, 1, 2], 16), ("resnet8", [1, 2, 3], 4)],
+                         ids=["mlp_K3", "mlp_K4", "resnet8_K4"])
+def test_graph_replay_over_two_ring_periods_fp32(net, splits, batch):
+    """Every recorded piece is replayed at least twice more after its recording: K-1 warm-up iterations, then two full
+    ring periods (lcm(1..K, 2): 6 at K=3, 12 at K=4) and one more.  fp32 mode, so any pointer that is wrong at
+    t + period shows as a bit-level difference; debug_checks adds the device-side ring stamps (the delay pattern of
+    Eq. 6-8 checked on the GPU itself)."""
+    K = len(splits) + 1
+    period = {3: 6, 4: 12}[K]
+    cfg = dict(nets.config(net), opt=dict(lr=0.02, momentum=0.9, weight_decay=5e-4))
+    run_pair(cfg, K - 1 + 2 * period + 1, FP32_TOL, LOSS_TOL, split_after=splits, batch=batch, use_graph=True,
+             gpu_kwargs=dict(debug_checks=True))
+
+
+def test_step_size_schedule_and_adam_keep_the_graphs_fp32():
+    """The step size sequence gamma_t (Theorem 2's diminishing sequence) and Adam's iteration-dependent bias corrections
+    live in device memory: a run that changes the step size every iteration replays the same recordings."""
+    cfg = dict(nets.config("mlp"), opt=dict(lr=0.05, momentum=0.9, weight_decay=0.0))
+    run_pair(cfg, 12, FP32_TOL, LOSS_TOL, use_graph=True, lr_schedule=lambda t: 0.05 / (1 + t))
+    cfg = dict(nets.config("resnet8"), opt=dict(lr=1e-3, momentum=0.0, weight_decay=0.0))
+    run_pair(cfg, 8, FP32_TOL, LOSS_TOL, batch=6, opt="adam", use_graph=True, lr_schedule=lambda t: 1e-3 / (1 + 0.1 * t))
 
 
 @pytest.mark.parametrize("splits", [[], [2, 3], [1, 2, 3]], ids=["K1", "K3", "K4"])
@@ -60,7 +101,7 @@ def test_resnet8_split_positions_adam_fp32(split):
 def test_resnet8_split_positions_bf16(split):
     """The same cuts in the bf16 mode the sweep is timed in (tensor-core kernels, epilogue batch-norm sums)."""
     cfg = dict(nets.config("resnet8"), opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
-    run_pair(cfg, 5, BF16_TOL, 5e-3, precision="bf16", split_after=split, noise_mult=2.0)
+    run_pair(cfg, 5, BF16_TOL, 5e-3, precision="bf16", split_after=split, noise_bar=True, ratio_band=RATIO_BAND)
 
 
 def test_resnet8_graph_replay_matches_fp32():
@@ -79,7 +120,7 @@ def test_generic_layers_fp32():
 
 def test_resnet8_k2_bf16():
     cfg = dict(nets.config("resnet8"), opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
-    w = run_pair(cfg, 6, BF16_TOL, 5e-3, precision="bf16", noise_mult=2.0)
+    w = run_pair(cfg, 6, BF16_TOL, 5e-3, precision="bf16", noise_bar=True, ratio_band=RATIO_BAND)
     print("resnet8 bf16 worst", w)
 
 
@@ -87,8 +128,30 @@ def test_resnet20_k3_bf16_graph():
     L = nets.resnet(3, 10)
     cfg = dict(layers=L, split_after=nets.split_even_blocks(L, 3), batch=32, in_shape=(3, 32, 32), num_classes=10,
                precision="bf16", opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
-    w = run_pair(cfg, 8, BF16_TOL, 5e-3, use_graph=True, noise_mult=2.0)
+    w = run_pair(cfg, 8, BF16_TOL, 5e-3, use_graph=True, noise_bar=True, ratio_band=RATIO_BAND)
     print("resnet20 bf16 worst", w)
+
+
+@pytest.mark.parametrize("c,h,stride", [(16, 32, 1), (32, 16, 1), (64, 8, 1), (16, 32, 2), (32, 16, 2)],
+                         ids=["c16", "c32", "c64", "c16_s2", "c32_s2"])
+def test_one_block_networks_bf16(c, h, stride):
+    """input -> BASIC_BLOCK -> global mean pool -> FC, K = 1, per stage width and stride: the tensor-core convolutions
+    with their fused epilogues (batch-norm sums, shortcut gradient) in the smallest network that contains them.  Only a
+    handful of bf16 stores separate the two sides here, so the plain bf16 tolerance applies without any noise rule."""
+    co = c * stride
+    L = [(nets.BASIC_BLOCK, c, co, stride, 0, 0), (nets.GLOBAL_AVGPOOL, co, co, 1, 0, 0), (nets.FC, co, 10, 1, 1, 0)]
+    cfg = dict(layers=L, split_after=[], batch=32, in_shape=(c, h, h), num_classes=10, precision="bf16",
+               opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
+    w = run_pair(cfg, 2, BF16_TOL, 5e-3)
+    print("one block c=%d stride=%d worst" % (c, stride), w)
+
+
+def test_resnet56_k2_bf16_graph():
+    """Config 3: ResNet-56 (units 9-9-9), K = 2 split at the centre (14 + 13 blocks), batch 128, bf16 storage, graph
+    replay: four iterations against the oracle at full size."""
+    cfg = nets.config("resnet56")
+    w = run_pair(cfg, 4, BF16_TOL, 5e-3, use_graph=True, noise_bar=True, ratio_band=RATIO_BAND)
+    print("resnet56 K=2 full size worst", w)
 
 
 def test_create_rejects_bad_specs():
@@ -121,45 +184,89 @@ def test_resnet110_k4_full_size_bf16_graph():
     iterations against the oracle at full size.  Every module applies its first real delayed gradient inside the
     window (delays 3, 2, 1, 0), loss and weights are held to the bf16 bars, gradients to the format-noise bar."""
     cfg = nets.config("resnet110")
-    w = run_pair(cfg, 5, BF16_TOL, 5e-3, use_graph=True, noise_mult=2.0, check_every=2)
+    w = run_pair(cfg, 5, BF16_TOL, 5e-3, use_graph=True, noise_bar=True, ratio_band=RATIO_BAND, check_every=2)
     print("resnet110 K=4 full size worst", w)
 
 
-_CHILD = r"""
-import sys, numpy as np, torch
-from paper_1804_10574_b200 import binding, nets, synth
-L = nets.resnet(3, 10)
-B, shape, classes = 32, (3, 32, 32), 10
-d = binding.Ddg(L, nets.split_even_blocks(L, 3), B, shape, classes, precision="bf16", lr=0.01, momentum=0.9,
-                weight_decay=5e-4, use_graph=True)
-d.set_weights(synth.init_weights(L, perturb_affine=0.1))
-losses = []
-for t in range(6):
-    x, y = synth.batch(t, B, shape, classes)
-    losses.append(d.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()))
-w = np.empty(d.n_params, dtype=np.float32)
-d.get_weights(w)
-np.save(sys.argv[1], np.concatenate([w, np.asarray(losses, dtype=np.float32)]))
-"""
+def _resnet20_k3_bf16_run(**kw):
+    from paper_1804_10574_b200 import binding, synth
+    L = nets.resnet(3, 10)
+    B, shape, classes = 32, (3, 32, 32), 10
+    d = binding.Ddg(L, nets.split_even_blocks(L, 3), B, shape, classes, precision="bf16", lr=0.01, momentum=0.9,
+                    weight_decay=5e-4, use_graph=True, **kw)
+    d.set_weights(synth.init_weights(L, perturb_affine=0.1))
+    losses = []
+    for t in range(6):
+        x, y = synth.batch(t, B, shape, classes)
+        losses.append(d.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()))
+    w = np.empty(d.n_params, dtype=np.float32)
+    d.get_weights(w)
+    n = d.last_step_launches()
+    d.destroy()
+    return w, losses, n
 
 
-def test_epilogue_batch_norm_sums_match_separate_reductions(tmp_path):
+def test_epilogue_batch_norm_sums_match_separate_reductions():
     """The batch-norm sums taken in the convolution epilogues and the separate reduction kernels are two evaluations
-    of the same sums in different orders: six ResNet-20 K=3 bf16 iterations in each mode (the switch is read once per
-    process, so each runs in a child) must end with the same weights up to what a last-bit difference of a statistic
-    can move through bf16 rounding."""
-    import os
-    import subprocess
-    import sys
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    out = {}
-    for mode in ("1", "0"):
-        f = str(tmp_path / ("w%s.npy" % mode))
-        env = dict(os.environ, DDG_FUSE_BN=mode, PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
-        subprocess.run([sys.executable, "-c", _CHILD, f], check=True, env=env, cwd=root, timeout=600)
-        out[mode] = np.load(f)
-    a, b = out["1"], out["0"]
-    assert np.all(np.isfinite(a)) and np.all(np.isfinite(b))
-    assert abs(a[-1] - b[-1]) < 5e-3 * max(1.0, abs(b[-1]))          # last loss
-    assert rel(a[:-6], b[:-6]) < 2e-3                                  # all weights, one tensor
+    of the same sums in different orders: six ResNet-20 K=3 bf16 iterations in each mode must end with the same
+    weights up to what a last-bit difference of a statistic can move through bf16 rounding, per parameter tensor."""
+    wa, la, na = _resnet20_k3_bf16_run()
+    wb, lb, nb = _resnet20_k3_bf16_run(separate_bn_sums=True)
+    assert nb > na                                                       # the separate reductions are extra launches
+    assert np.all(np.isfinite(wa)) and np.all(np.isfinite(wb))
+    assert abs(la[-1] - lb[-1]) < 5e-3 * max(1.0, abs(lb[-1]))
+    worst = max(rel(wa[off:off + int(np.prod(shape))], wb[off:off + int(np.prod(shape))])
+                for _, name, off, shape, _ in nets.param_segments(nets.resnet(3, 10)))
+    print("epilogue vs separate sums: worst per-tensor weight difference", worst)
+    assert worst < 5e-3
 
+
+def test_launch_overlap_settings_give_the_same_bits():
+    """The programmatic-launch policy only moves kernels in time: never / library policy / every kernel must produce
+    identical weights (fixed summation orders everywhere)."""
+    ref = _resnet20_k3_bf16_run(launch_overlap=1)[0]
+    for mode in (0, 2):
+        assert np.array_equal(ref, _resnet20_k3_bf16_run(launch_overlap=mode)[0]), mode
+
+
+def test_bounded_wait_runs_out_cleanly():
+    """A device-side wait that nothing satisfies gives up after its poll limit, the kernel returns, the next sync point
+    reports DDG_ERR_TIMEOUT, and from then on the context answers DDG_ERR_STATE; the device stays usable."""
+    from paper_1804_10574_b200 import binding
+    d = binding.Ddg(nets.mlp(), [1], 4, (64, 1, 1), 10)
+    x = torch.zeros(4, 64, device="cuda"); y = torch.zeros(4, dtype=torch.int32, device="cuda")
+    d.step(x, y)
+    d.debug_wait_timeout(2000)
+    with pytest.raises(binding.DdgError) as e:
+        d.sync()
+    assert e.value.status == 6 and "bounded wait" in str(e.value)
+    with pytest.raises(binding.DdgError) as e:
+        d.step(x, y)
+    assert e.value.status == 7
+    d.destroy()
+    # another context in the same process starts clean (every context has its own error word)
+    d2 = binding.Ddg(nets.mlp(), [1], 4, (64, 1, 1), 10)
+    d2.step(x, y)
+    d2.sync()
+    d2.destroy()
+    assert float((torch.ones(8, device="cuda") * 2).sum()) == 16.0
+
+
+def test_ring_stamps_catch_a_shifted_slot():
+    """debug_checks: with the forward counter of module 1 shifted by one, as a ring-indexing error would, the backward
+    sweep finds a stamp it does not expect and the next sync point answers DDG_ERR_STATE; unshifted runs stay clean
+    (test_graph_replay_over_two_ring_periods_fp32 runs with the stamps on)."""
+    from paper_1804_10574_b200 import binding
+    L = nets.mlp()
+    d = binding.Ddg(L, [0, 1], 4, (64, 1, 1), 10, debug_checks=True, use_graph=True)
+    x = torch.zeros(4, 64, device="cuda"); y = torch.zeros(4, dtype=torch.int32, device="cuda")
+    for _ in range(5):
+        d.step(x, y)
+    d.sync()
+    d.debug_shift_stamps(0, 1)
+    for _ in range(4):
+        d.step(x, y, want_loss=False)
+    with pytest.raises(binding.DdgError) as e:
+        d.sync()
+    assert e.value.status == 7 and "ring stamp" in str(e.value)
+    d.destroy()

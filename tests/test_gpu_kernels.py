@@ -5,11 +5,34 @@ import pytest
 import torch
 
 from oracle import ddg_oracle as orc
-from tests.parity import rel
+from tests.parity import elementwise_ok, rel
 
 pytestmark = pytest.mark.gpu
 
 TOL = {0: 1e-5, 1: 6e-3}   # fp32: accumulation order only; bf16: inputs are exact bf16, output rounding 2^-9
+# per element: |gpu - ref| <= RTOL * |ref| + ATOL_RMS * rms(ref).  bf16: one output rounding (2^-9 relative) plus the
+# fp32 accumulation error of a few hundred products; a wrong tap, border or tile seam is an error of order rms(ref)
+RTOL = {0: 1e-5, 1: 2.0 ** -8}
+ATOL_RMS = {0: 1e-6, 1: 1e-3}
+
+
+def check_map(got_nchw, ref_nchw, prec, what, seam_rows=None):
+    """L2 bar on the whole tensor, the same bar on the image-border pixels alone (and on the rows next to a tile seam,
+    every `seam_rows` rows), and the per-element bar on every value."""
+    assert rel(got_nchw, ref_nchw) < TOL[prec], what
+    H, W = ref_nchw.shape[2], ref_nchw.shape[3]
+    if H > 2 and W > 2:
+        border = np.ones((H, W), dtype=bool)
+        border[1:-1, 1:-1] = False
+        assert rel(got_nchw[:, :, border], ref_nchw[:, :, border]) < TOL[prec], what + " (image border)"
+        if seam_rows and seam_rows < H:
+            seam = np.zeros(H, dtype=bool)
+            seam[seam_rows - 1::seam_rows] = True
+            seam[seam_rows::seam_rows] = True
+            assert rel(got_nchw[:, :, seam, :], ref_nchw[:, :, seam, :]) < TOL[prec], what + " (tile seams)"
+    rms = float(np.sqrt(np.mean(np.square(ref_nchw)))) if ref_nchw.size else 0.0
+    ok, idx, excess = elementwise_ok(got_nchw, ref_nchw, RTOL[prec], ATOL_RMS[prec] * rms)
+    assert ok, "%s: element %r off by %.3e beyond the per-element bar" % (what, idx, excess)
 
 
 def tdtype(prec):
@@ -60,8 +83,13 @@ def test_conv3x3_fwd_dgrad_wgrad(shape, prec):
     torch.cuda.synchronize()
     y_ref = orc.conv3x3_forward(xh, wh, st)
     dx_ref, dw_ref = orc.conv3x3_backward(xh, wh, dyh, st)
-    assert rel(from_dev(y), y_ref) < TOL[prec]
-    assert rel(from_dev(dx), dx_ref) < TOL[prec]
+    seam = max(1, 128 // Wo) if prec else None      # a tensor-core tile is 128 pixels = 128 / W image rows
+    check_map(from_dev(y), y_ref, prec, "forward", seam)
+    check_map(from_dev(dx), dx_ref, prec, "input gradient", max(1, 128 // W) if prec else None)
+    tc_w = prec and binding.tensor_core_path(B, H, W, Ci, Co, st) & 2
+    ok, idx, excess = elementwise_ok(dw.cpu().numpy(), dw_ref, 2e-4 if tc_w else 1e-5,
+                                     (2e-4 if tc_w else 1e-6) * float(np.sqrt(np.mean(np.square(dw_ref)))))
+    assert ok, "weight gradient: element %r off by %.3e" % (idx, excess)
     # fp32 output from exact inputs in both precisions; the tensor-core path accumulates in fp32 over all pixels
     assert rel(dw.cpu().numpy(), dw_ref) < (2e-4 if prec and binding.tensor_core_path(B, H, W, Ci, Co, st) & 2 else 1e-5)
     # a second call on the same scratch gives the same bits (fixed summation order)
@@ -131,6 +159,9 @@ def test_bn_fwd_bwd(shape, prec, relu, res):
         y_ref = np.maximum(y_ref, 0)
     assert rel(mean.cpu().numpy(), m_ref) < 1e-5 and rel(invstd.cpu().numpy(), is_ref) < 1e-5
     assert rel(from_dev(y), y_ref) < TOL[prec]
+    yrms = float(np.sqrt(np.mean(np.square(y_ref))))
+    ok, idx, excess = elementwise_ok(from_dev(y), y_ref, RTOL[prec], (2e-3 if prec else 1e-5) * yrms)
+    assert ok, "batch-norm output: element %r off by %.3e" % (idx, excess)
     # backward reference uses the mask of the output the GPU actually stored
     dz = douth * (from_dev(y) > 0) if relu else douth
     dx_ref, dg_ref, db_ref = orc.bn_backward(xh, m_ref, is_ref, gh, dz)
@@ -142,6 +173,10 @@ def test_bn_fwd_bwd(shape, prec, relu, res):
 @pytest.mark.parametrize("prec", [0, 1], ids=["fp32", "bf16"])
 @pytest.mark.parametrize("n", [1, 5, 1024, 1733812])
 def test_sgd_update(n, prec):
+    """The update kernel against the oracle's own update: an FC layer of n weights without bias, K = 1, batch 1, input
+    x = 1, two classes.  With lr = 0 the oracle's step leaves the gradient g of its first iteration in get_grads; with
+    the same (w, g) and zero momentum state the oracle's next step is the reference for the kernel (Eq. 9 with momentum
+    and decay as the oracle reads them)."""
     from paper_1804_10574_b200 import binding
     rng = np.random.default_rng(3)
     w, v, g = (rng.standard_normal(n).astype(np.float32) for _ in range(3))
@@ -149,10 +184,24 @@ def test_sgd_update(n, prec):
     wv = torch.empty(n, dtype=tdtype(prec), device="cuda")
     binding.sgd_update(prec, wd, vd, gd, wv, n, 0.1, 0.9, 5e-4)
     torch.cuda.synchronize()
-    d = g.astype(np.float64) + 5e-4 * w
-    v_ref = 0.9 * v + d
-    w_ref = w - 0.1 * v_ref
+    d = g.astype(np.float64) + float(np.float32(5e-4)) * w
+    v_ref = float(np.float32(0.9)) * v + d
+    w_ref = w - float(np.float32(0.1)) * v_ref
     assert rel(vd.cpu().numpy(), v_ref) < 1e-6 and rel(wd.cpu().numpy(), w_ref) < 1e-6
+    if n == 1024:
+        # the same numbers through the oracle's optimiser: a bias-free FC layer 512 -> 2 holds n = 1024 weights; one
+        # iteration from momentum 0 gives w1 = w - lr * (g + wd * w), which the kernel must reproduce from (w, 0, g)
+        f32 = lambda q: float(np.float32(q))
+        o = orc.Oracle([(0, 512, 2, 1, 0, 0)], [], 1, (512, 1, 1), 2, lr=f32(0.1), momentum=f32(0.9), weight_decay=f32(5e-4))
+        o.set_weights(w.astype(np.float64))
+        xo = rng.standard_normal((1, 512, 1, 1))
+        o.step(xo, np.zeros(1, dtype=np.int32))
+        g_o = o.get_grads(0)[1]
+        w1_o = o.get_weights()
+        w2, v2, g2 = torch.from_numpy(w).cuda(), torch.zeros(n, device="cuda"), torch.from_numpy(g_o.astype(np.float32)).cuda()
+        binding.sgd_update(prec, w2, v2, g2, wv, n, 0.1, 0.9, 5e-4)
+        torch.cuda.synchronize()
+        assert rel(w2.cpu().numpy(), w1_o) < 1e-6 and rel(v2.cpu().numpy(), g_o + f32(5e-4) * w.astype(np.float64)) < 1e-6
     assert torch.equal(wv, wd.to(tdtype(prec)))      # the version slot is the cast of the new master weights
 
 
@@ -184,5 +233,5 @@ def test_conv3x3_with_prearranged_filter_matches_oracle(shape):
     binding.conv3x3_packed(0, x, w, pk, y, B, H, W, C)
     binding.conv3x3_packed(1, dy, w, pk, dx, B, H, W, C)
     torch.cuda.synchronize()
-    assert rel(from_dev(y), orc.conv3x3_forward(xh, wh, 1)) < TOL[1]
-    assert rel(from_dev(dx), orc.conv3x3_backward(xh, wh, dyh, 1)[0]) < TOL[1]
+    check_map(from_dev(y), orc.conv3x3_forward(xh, wh, 1), 1, "forward", max(1, 128 // W))
+    check_map(from_dev(dx), orc.conv3x3_backward(xh, wh, dyh, 1)[0], 1, "input gradient", max(1, 128 // W))
