@@ -188,6 +188,34 @@ ddg_status ddg_conv3x3_pack(const void *w, void *packed, int C, void *stream);
 ddg_status ddg_conv3x3_packed(int dgrad, const void *src, const void *w, const void *packed, void *dst, int B, int H,
                               int W, int C, void *stream);
 
+/* The fused forms the training step launches on the tensor-core path (bf16, stride 1, C -> C channels with
+ * ddg_tensor_core_path(...) & 1; other shapes: DDG_ERR_UNSUPPORTED).  packed: nullable filter image as above.
+ * scratch: device fp32, ddg_conv3x3_fused_scratch_elems(B, H, W, C) elements, contents undefined on entry and exit.
+ *
+ * ddg_conv3x3_fwd_stats: y = conv3x3(x, w) (Eq. 3) and, from the values as stored (bf16), the statistics of the batch
+ * norm that follows: mean[c] and invstd[c] = 1 / sqrt(biased variance + 1e-5) over (B, H, W), fp32 [C], taken in the
+ * convolution's epilogue (per-CTA partial sums, folded in a fixed order by the CTA that finishes last).
+ *
+ * ddg_conv3x3_dgrad_fused: dx = input gradient of conv3x3 given dy (Eq. 5 / Eq. 7), plus
+ *   - res_dout, res_out (both or neither; [B][H][W][C]): the gradient of an identity shortcut,
+ *     dx += res_dout * [res_out > 0] (the residual block's output ReLU and add, differentiated);
+ *   - bn_mask, bn_x, bn_mean, bn_invstd, dbeta, dgamma (all or none): the two reductions of the batch-norm backward
+ *     pass whose incoming gradient is dx: with dz = dx(as stored) * [bn_mask > 0] and xhat = (bn_x - mean) * invstd,
+ *     dbeta[c] = sum dz, dgamma[c] = sum dz * xhat (fp32 [C]). */
+size_t ddg_conv3x3_fused_scratch_elems(int B, int H, int W, int C);
+ddg_status ddg_conv3x3_fwd_stats(const void *x, const void *w, const void *packed, void *y, float *mean, float *invstd,
+                                 float *scratch, int B, int H, int W, int C, void *stream);
+ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
+                                   const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
+                                   const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H,
+                                   int W, int C, void *stream);
+/* Input gradient of the stride-2 convolution of a down-sampling block (Cin -> 2 Cin, bf16, tensor-core path only) with
+ * the gradient of the block's parameter-free shortcut added: dx[n][2j][2i][c] += res_dout[n][j][i][c] *
+ * [res_out[n][j][i][c] > 0] for c < Cin (the shortcut reads every second pixel of every second row and pads the
+ * channels with zeros).  dy, res_dout, res_out: [B][H/2][W/2][2 Cin]; dx: [B][H][W][Cin].  res_* nullable (both). */
+ddg_status ddg_conv3x3_s2_dgrad_shortcut(const void *dy, const void *w, void *dx, const void *res_dout,
+                                         const void *res_out, int B, int H, int W, int Cin, void *stream);
+
 /* dw = conv3x3 weight gradient (Eq. 4 / Eq. 6), fp32 [Cout][Cin][3][3].  scratch: device, fp32,
  * ddg_conv3x3_wgrad_scratch_elems(...) elements, contents undefined on entry and exit. */
 size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride);

@@ -28,7 +28,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_conv3x3_wgrad_scratch_elems", "ddg_conv3x3_wgrad", "ddg_bn_scratch_elems", "ddg_bn_fwd", "ddg_bn_bwd",
            "ddg_sgd_update", "ddg_tensor_core_path", "ddg_bn_fwd_noalloc",
            "ddg_conv3x3_packed_bytes", "ddg_conv3x3_pack", "ddg_conv3x3_packed", "ddg_bn_bwd_reduce",
-           "ddg_debug_wait_timeout", "ddg_debug_shift_stamps"]
+           "ddg_debug_wait_timeout", "ddg_debug_shift_stamps", "ddg_conv3x3_fused_scratch_elems",
+           "ddg_conv3x3_fwd_stats", "ddg_conv3x3_dgrad_fused", "ddg_conv3x3_s2_dgrad_shortcut"]
 
 
 class Layer(ctypes.Structure):
@@ -81,6 +82,11 @@ _lib.ddg_conv3x3_packed_bytes.argtypes = [_i] * 4
 _lib.ddg_conv3x3_packed_bytes.restype = _sz
 _lib.ddg_conv3x3_pack.argtypes = [_vp, _vp, _i, _vp]
 _lib.ddg_conv3x3_packed.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
+_lib.ddg_conv3x3_fused_scratch_elems.argtypes = [_i] * 4
+_lib.ddg_conv3x3_fused_scratch_elems.restype = _sz
+_lib.ddg_conv3x3_fwd_stats.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
+_lib.ddg_conv3x3_dgrad_fused.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
+_lib.ddg_conv3x3_s2_dgrad_shortcut.argtypes = [_vp] * 5 + [_i] * 4 + [_vp]
 _lib.ddg_bn_fwd_noalloc.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_bn_bwd_reduce.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_sgd_update.argtypes = [_i, _vp, _vp, _vp, _vp, _sz, _f, _f, _f, _vp]
@@ -198,7 +204,7 @@ class Ddg:
 
 def _ok(rc):
     if rc != 0:
-        raise DdgError(rc, "kernel entry point failed")
+        raise DdgError(rc, (_lib.ddg_last_error(None) or b"kernel entry point failed").decode())
 
 
 def tensor_core_path(B, H, W, Cin, Cout, stride):
@@ -215,6 +221,27 @@ def conv3x3_pack(w, packed, C, stream=None):
 
 def conv3x3_packed(dgrad, src, w, packed, dst, B, H, W, C, stream=None):
     _ok(_lib.ddg_conv3x3_packed(int(dgrad), _ptr(src), _ptr(w), _ptr(packed), _ptr(dst), B, H, W, C, stream))
+
+
+def conv3x3_fused_scratch_elems(B, H, W, C):
+    return _lib.ddg_conv3x3_fused_scratch_elems(B, H, W, C)
+
+
+def conv3x3_fwd_stats(x, w, packed, y, mean, invstd, scratch, B, H, W, C, stream=None):
+    _ok(_lib.ddg_conv3x3_fwd_stats(_ptr(x), _ptr(w), _ptr(packed), _ptr(y), _ptr(mean), _ptr(invstd), _ptr(scratch),
+                                   B, H, W, C, stream))
+
+
+def conv3x3_dgrad_fused(dy, w, packed, dx, res_dout, res_out, bn_mask, bn_x, bn_mean, bn_invstd, dbeta, dgamma, scratch,
+                        B, H, W, C, stream=None):
+    _ok(_lib.ddg_conv3x3_dgrad_fused(_ptr(dy), _ptr(w), _ptr(packed), _ptr(dx), _ptr(res_dout), _ptr(res_out),
+                                     _ptr(bn_mask), _ptr(bn_x), _ptr(bn_mean), _ptr(bn_invstd), _ptr(dbeta), _ptr(dgamma),
+                                     _ptr(scratch), B, H, W, C, stream))
+
+
+def conv3x3_s2_dgrad_shortcut(dy, w, dx, res_dout, res_out, B, H, W, Cin, stream=None):
+    _ok(_lib.ddg_conv3x3_s2_dgrad_shortcut(_ptr(dy), _ptr(w), _ptr(dx), _ptr(res_dout), _ptr(res_out), B, H, W, Cin,
+                                           stream))
 
 
 def conv3x3_fwd(prec, x, w, y, B, H, W, Cin, Cout, stride, stream=None):

@@ -107,6 +107,58 @@ ddg_status ddg_conv3x3_packed(int dgrad, const void *src, const void *w, const v
     return done(launch_conv_tc(dgrad ? 1 : 0, src, w, packed, dst, B, H, W, C, Shortcut{}, (cudaStream_t)stream));
 }
 
+size_t ddg_conv3x3_fused_scratch_elems(int B, int H, int W, int C) {
+    if (init_once() != DDG_OK || !conv_tc_supported(B, H, W, C, C, 1)) return 0;
+    return 32 + (size_t)conv_tc_grid(B, H, W) * 2 * C;  // ticket counter, then one partial [2C] per CTA
+}
+
+ddg_status ddg_conv3x3_fwd_stats(const void *x, const void *w, const void *packed, void *y, float *mean, float *invstd,
+                                 float *scratch, int B, int H, int W, int C, void *stream) {
+    if (!x || !w || !y || !mean || !invstd || !scratch) return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_supported(B, H, W, C, C, 1)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;  // the CTA ticket counter
+    BnFuse bf;
+    bf.counter = reinterpret_cast<unsigned *>(scratch); bf.part = scratch + 32; bf.o0 = mean; bf.o1 = invstd;
+    return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, s, bf));
+}
+
+ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
+                                   const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
+                                   const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H,
+                                   int W, int C, void *stream) {
+    if (!dy || !w || !dx || !scratch) return DDG_ERR_INVALID_ARG;
+    if ((res_dout == nullptr) != (res_out == nullptr)) return DDG_ERR_INVALID_ARG;
+    const bool sums = bn_mask || bn_x || bn_mean || bn_invstd || dbeta || dgamma;
+    if (sums && !(bn_mask && bn_x && bn_mean && bn_invstd && dbeta && dgamma)) return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_supported(B, H, W, C, C, 1)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;
+    Shortcut sc{};
+    if (res_dout) { sc.mode = 1; sc.a = res_dout; sc.b = res_out; }
+    BnFuse bf;
+    if (sums) {
+        bf.counter = reinterpret_cast<unsigned *>(scratch); bf.part = scratch + 32; bf.o0 = dbeta; bf.o1 = dgamma;
+        bf.mask = bn_mask; bf.x = bn_x; bf.mean = bn_mean; bf.invstd = bn_invstd;
+    }
+    return done(launch_conv_tc(1, dy, w, packed, dx, B, H, W, C, sc, s, bf));
+}
+
+ddg_status ddg_conv3x3_s2_dgrad_shortcut(const void *dy, const void *w, void *dx, const void *res_dout,
+                                         const void *res_out, int B, int H, int W, int Cin, void *stream) {
+    if (!dy || !w || !dx || (res_dout == nullptr) != (res_out == nullptr)) return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_s2_supported(B, H, W, Cin, 2 * Cin, 2)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    Shortcut sc{};
+    if (res_dout) { sc.mode = 2; sc.a = res_dout; sc.b = res_out; sc.c_small = Cin; sc.h_big = H; sc.w_big = W; }
+    return done(launch_conv_tc_s2(1, dy, w, nullptr, dx, B, H, W, Cin, sc, (cudaStream_t)stream));
+}
+
 size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride) {
     if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return 0;
     size_t a = conv_wgrad_scratch_elems(B, H, W, Cin, Cout, stride), b = wgrad_tc_scratch_elems();

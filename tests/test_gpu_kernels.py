@@ -235,3 +235,109 @@ def test_conv3x3_with_prearranged_filter_matches_oracle(shape):
     torch.cuda.synchronize()
     check_map(from_dev(y), orc.conv3x3_forward(xh, wh, 1), 1, "forward", max(1, 128 // W))
     check_map(from_dev(dx), orc.conv3x3_backward(xh, wh, dyh, 1)[0], 1, "input gradient", max(1, 128 // W))
+
+
+# ---- the fused epilogues of the training step, each against oracle primitives composed on the same bf16 inputs ----
+FUSED_SHAPES = [(3, 32, 32, 16), (5, 16, 16, 32), (128, 8, 8, 64), (2, 8, 8, 16), (8, 8, 8, 32),      # slab and image-pair tiles
+                (301, 32, 32, 16), (231, 16, 16, 32), (902, 8, 8, 64)]                                  # many tiles per CTA
+
+
+def _filter(rng, C, Co=None):
+    Co = Co or C
+    w = torch.from_numpy(rng.standard_normal((Co, C, 3, 3)) * np.sqrt(2.0 / (9 * C))).to(torch.bfloat16)
+    return w.cuda(), w.to(torch.float64).numpy()
+
+
+@pytest.mark.parametrize("shape", FUSED_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("packed", [False, True], ids=["canonical", "image"])
+def test_conv_forward_with_batch_statistics(shape, packed):
+    """Eq. 3 for conv -> batch norm: the convolution's epilogue also delivers mean and 1/sqrt(var + eps) of its (stored)
+    output.  Tensor against the oracle's convolution; statistics against the oracle's batch norm applied to the tensor
+    the GPU stored, and to the oracle's own bf16-rounded output."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = shape
+    rng = np.random.default_rng(21)
+    x, xh = to_dev(rng.standard_normal((B, C, H, W)) * 1.2 + 0.1, 1)
+    w, wh = _filter(rng, C)
+    pk = None
+    if packed:
+        pk = torch.empty(binding.conv3x3_packed_bytes(B, H, W, C), dtype=torch.uint8, device="cuda")
+        binding.conv3x3_pack(w, pk, C)
+    y = torch.empty_like(x)
+    mean, invstd = (torch.full((C,), 7.0, dtype=torch.float32, device="cuda") for _ in range(2))
+    scratch = torch.full((binding.conv3x3_fused_scratch_elems(B, H, W, C),), 3.0, dtype=torch.float32, device="cuda")
+    for _ in range(2):       # the second call finds the first one's leftovers in the scratch
+        binding.conv3x3_fwd_stats(x, w, pk, y, mean, invstd, scratch, B, H, W, C)
+    torch.cuda.synchronize()
+    y_ref = orc.conv3x3_forward(xh, wh, 1)
+    check_map(from_dev(y), y_ref, 1, "forward", max(1, 128 // W))
+    ones, zeros = np.ones(C), np.zeros(C)
+    _, m_ref, is_ref = orc.bn_forward(from_dev(y), ones, zeros)
+    assert rel(mean.cpu().numpy(), m_ref) < 2e-5 and rel(invstd.cpu().numpy(), is_ref) < 2e-5
+    y_b = torch.from_numpy(y_ref).to(torch.bfloat16).to(torch.float64).numpy()
+    _, m2, is2 = orc.bn_forward(y_b, ones, zeros)
+    assert np.max(np.abs(mean.cpu().numpy() - m2)) < 1e-3 * float(np.sqrt(np.mean(y_ref ** 2))) and rel(invstd.cpu().numpy(), is2) < 1e-3
+
+
+@pytest.mark.parametrize("shape", FUSED_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("with_shortcut,with_sums", [(True, False), (False, True), (True, True)],
+                         ids=["shortcut", "sums", "shortcut_sums"])
+def test_conv_input_gradient_with_shortcut_and_batch_norm_sums(shape, with_shortcut, with_sums):
+    """Eq. 5 / Eq. 7 as the backward sweep launches it: dx = dgrad(dy) [+ dout * [out > 0]] and the two reductions of
+    the batch-norm backward that consumes dx.  dx against the oracle's convolution backward plus the shortcut term;
+    (dbeta, dgamma) against the oracle's batch-norm backward fed the dx the GPU stored."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = shape
+    rng = np.random.default_rng(23)
+    dy, dyh = to_dev(rng.standard_normal((B, C, H, W)), 1)
+    w, wh = _filter(rng, C)
+    dout, douth = to_dev(rng.standard_normal((B, C, H, W)), 1)
+    out, outh = to_dev(np.maximum(rng.standard_normal((B, C, H, W)), 0), 1)       # a ReLU output: about half zeros
+    mask, maskh = to_dev(np.maximum(rng.standard_normal((B, C, H, W)), 0), 1)
+    bx, bxh = to_dev(rng.standard_normal((B, C, H, W)) * 1.5 + 0.3, 1)
+    _, m_ref, is_ref = orc.bn_forward(bxh, np.ones(C), np.zeros(C))
+    mean = torch.from_numpy(m_ref.astype(np.float32)).cuda()
+    invstd = torch.from_numpy(is_ref.astype(np.float32)).cuda()
+    dx = torch.empty_like(dy)
+    db, dg = (torch.full((C,), 7.0, dtype=torch.float32, device="cuda") for _ in range(2))
+    scratch = torch.full((binding.conv3x3_fused_scratch_elems(B, H, W, C),), 3.0, dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        binding.conv3x3_dgrad_fused(dy, w, None, dx, dout if with_shortcut else None, out if with_shortcut else None,
+                                    mask if with_sums else None, bx if with_sums else None,
+                                    mean if with_sums else None, invstd if with_sums else None,
+                                    db if with_sums else None, dg if with_sums else None, scratch, B, H, W, C)
+    torch.cuda.synchronize()
+    dx_ref = orc.conv3x3_backward(np.zeros_like(dyh), wh, dyh, 1)[0]
+    if with_shortcut:
+        dx_ref = dx_ref + douth * (outh > 0)
+    check_map(from_dev(dx), dx_ref, 1, "input gradient", max(1, 128 // W))
+    if with_sums:
+        dz = from_dev(dx) * (maskh > 0)
+        _, dg_ref, db_ref = orc.bn_backward(bxh, mean.double().cpu().numpy(), invstd.double().cpu().numpy(), np.ones(C), dz)
+        scale = float(np.sqrt(np.mean(dz ** 2)) * np.sqrt(B * H * W))       # size of a sum of that many such terms
+        assert np.max(np.abs(db.cpu().numpy() - db_ref)) < 2e-5 * scale, (db.cpu().numpy(), db_ref)
+        assert np.max(np.abs(dg.cpu().numpy() - dg_ref)) < 2e-5 * scale * 2, (dg.cpu().numpy(), dg_ref)
+
+
+@pytest.mark.parametrize("shape", [(3, 32, 32, 16), (6, 16, 16, 32), (7, 32, 32, 32), (10, 16, 16, 16), (128, 32, 32, 16)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_stride2_input_gradient_with_parameter_free_shortcut(shape):
+    """The down-sampling block's first convolution in the backward sweep: dx = dgrad_stride2(dy) plus the gradient of
+    the parameter-free shortcut (every second pixel of every second row, first Cin channels)."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, Ci = shape
+    Co = 2 * Ci
+    rng = np.random.default_rng(29)
+    dy, dyh = to_dev(rng.standard_normal((B, Co, H // 2, W // 2)), 1)
+    w, wh = _filter(rng, Ci, Co)
+    dout, douth = to_dev(rng.standard_normal((B, Co, H // 2, W // 2)), 1)
+    out, outh = to_dev(np.maximum(rng.standard_normal((B, Co, H // 2, W // 2)), 0), 1)
+    dx = torch.empty(B, H, W, Ci, dtype=torch.bfloat16, device="cuda")
+    binding.conv3x3_s2_dgrad_shortcut(dy, w, dx, dout, out, B, H, W, Ci)
+    torch.cuda.synchronize()
+    dx_ref = orc.conv3x3_backward(np.zeros((B, Ci, H, W)), wh, dyh, 2)[0] + orc.shortcut_backward(douth * (outh > 0), Ci, H, W, 2)
+    check_map(from_dev(dx), dx_ref, 1, "stride-2 input gradient with shortcut")
+    dx2 = torch.empty_like(dx)
+    binding.conv3x3_s2_dgrad_shortcut(dy, w, dx2, None, None, B, H, W, Ci)
+    torch.cuda.synchronize()
+    check_map(from_dev(dx2), orc.conv3x3_backward(np.zeros((B, Ci, H, W)), wh, dyh, 2)[0], 1, "stride-2 input gradient")
