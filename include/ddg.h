@@ -221,6 +221,18 @@ ddg_status ddg_conv3x3_s2_dgrad_shortcut(const void *dy, const void *w, void *dx
 size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride);
 ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float *dw, float *scratch, int B, int H,
                              int W, int Cin, int Cout, int stride, void *stream);
+/* Fully connected layer h = x W^T + b (Eq. 3) and its backward pass (Eq. 4-5 / Eq. 6-7).  x [B][in], W [out][in] and
+ * bias [out] (nullable) in the precision's element type; y and dy [B][out] are fp32 when out_f32 != 0 (the network's
+ * last layer: logits and the loss gradient), else the element type; dW [out][in] and db [out] (nullable) fp32; dx
+ * [B][in] (nullable) in the element type.  With relu != 0 the forward output is max(., 0) and the backward pass masks dy
+ * with [y > 0] (y = forward output).  In bf16 the layer runs on the tensor cores (tcgen05 MMAs fed by TMA) when
+ * ddg_fc_tensor_core_path(B, in, out) is 1 and x, W, dx, dW start on 16-byte boundaries; otherwise on CUDA cores. */
+int ddg_fc_tensor_core_path(int B, int in, int out);
+ddg_status ddg_fc_fwd(int precision, const void *x, const void *W, const void *bias, void *y, int B, int in, int out,
+                      int relu, int out_f32, void *stream);
+ddg_status ddg_fc_bwd(int precision, const void *x, const void *W, const void *y, const void *dy, void *dx, float *dW,
+                      float *db, int B, int in, int out, int relu, int out_f32, void *stream);
+
 /* Batch-norm forward, fused: statistics over (B,H,W), then y = [relu](gamma*xhat + beta [+ res]).  res nullable
  * (same shape as y).  gamma/beta in the activation element type; mean/invstd fp32 [C] outputs; scratch fp32,
  * ddg_bn_scratch_elems(C) elements. */

@@ -29,7 +29,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_sgd_update", "ddg_tensor_core_path", "ddg_bn_fwd_noalloc",
            "ddg_conv3x3_packed_bytes", "ddg_conv3x3_pack", "ddg_conv3x3_packed", "ddg_bn_bwd_reduce",
            "ddg_debug_wait_timeout", "ddg_debug_shift_stamps", "ddg_conv3x3_fused_scratch_elems",
-           "ddg_conv3x3_fwd_stats", "ddg_conv3x3_dgrad_fused", "ddg_conv3x3_s2_dgrad_shortcut"]
+           "ddg_conv3x3_fwd_stats", "ddg_conv3x3_dgrad_fused", "ddg_conv3x3_s2_dgrad_shortcut",
+           "ddg_fc_tensor_core_path", "ddg_fc_fwd", "ddg_fc_bwd"]
 
 
 class Layer(ctypes.Structure):
@@ -87,6 +88,9 @@ _lib.ddg_conv3x3_fused_scratch_elems.restype = _sz
 _lib.ddg_conv3x3_fwd_stats.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_dgrad_fused.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_s2_dgrad_shortcut.argtypes = [_vp] * 5 + [_i] * 4 + [_vp]
+_lib.ddg_fc_tensor_core_path.argtypes = [_i] * 3
+_lib.ddg_fc_fwd.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]
+_lib.ddg_fc_bwd.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]
 _lib.ddg_bn_fwd_noalloc.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_bn_bwd_reduce.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_sgd_update.argtypes = [_i, _vp, _vp, _vp, _vp, _sz, _f, _f, _f, _vp]
@@ -258,6 +262,19 @@ def conv3x3_wgrad_scratch_elems(B, H, W, Cin, Cout, stride):
 
 def conv3x3_wgrad(prec, x, dy, dw, scratch, B, H, W, Cin, Cout, stride, stream=None):
     _ok(_lib.ddg_conv3x3_wgrad(prec, _ptr(x), _ptr(dy), _ptr(dw), _ptr(scratch), B, H, W, Cin, Cout, stride, stream))
+
+
+def fc_tensor_core_path(B, n_in, n_out):
+    return _lib.ddg_fc_tensor_core_path(B, n_in, n_out)
+
+
+def fc_fwd(prec, x, W, bias, y, B, n_in, n_out, relu, out_f32, stream=None):
+    _ok(_lib.ddg_fc_fwd(prec, _ptr(x), _ptr(W), _ptr(bias), _ptr(y), B, n_in, n_out, int(relu), int(out_f32), stream))
+
+
+def fc_bwd(prec, x, W, y, dy, dx, dW, db, B, n_in, n_out, relu, out_f32, stream=None):
+    _ok(_lib.ddg_fc_bwd(prec, _ptr(x), _ptr(W), _ptr(y), _ptr(dy), _ptr(dx), _ptr(dW), _ptr(db), B, n_in, n_out,
+                        int(relu), int(out_f32), stream))
 
 
 def bn_scratch_elems(C):

@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libddg.so")
 OBJ = os.path.join(HERE, "_build")
-SOURCES = ["engine.cu", "api_kernels.cu", "kernels_elementwise.cu", "kernels_conv_direct.cu", "conv_tc.cu", "api_noalloc.cu"]
+SOURCES = ["engine.cu", "api_kernels.cu", "kernels_elementwise.cu", "kernels_conv_direct.cu", "conv_tc.cu", "fc_tc.cu", "api_noalloc.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--expt-relaxed-constexpr",
          "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

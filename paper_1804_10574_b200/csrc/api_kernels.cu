@@ -182,6 +182,37 @@ ddg_status ddg_conv3x3_wgrad(int precision, const void *x, const void *dy, float
     return done(r);
 }
 
+int ddg_fc_tensor_core_path(int B, int in, int out) {
+    if (init_once() != DDG_OK) return 0;
+    return fc_tc_shape_supported(B, in, out) ? 1 : 0;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+ddg_status ddg_fc_fwd(int precision, const void *x, const void *W, const void *bias, void *y, int B, int in, int out,
+                      int relu, int out_f32, void *stream) {
+    if (bad_prec(precision) || !x || !W || !y) return DDG_ERR_INVALID_ARG;
+    if (B < 1 || in < 1 || out < 1) return DDG_ERR_UNSUPPORTED;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (pending_error()) return DDG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (precision == DDG_BF16 && fc_tc_supported(x, W, B, in, out))
+        return done(launch_fc_fwd_tc(x, W, bias, y, B, in, out, relu, out_f32, s));
+    return done(launch_fc_fwd(precision, x, W, bias, y, B, in, out, relu, out_f32, s));
+}
+
+ddg_status ddg_fc_bwd(int precision, const void *x, const void *W, const void *y, const void *dy, void *dx, float *dW,
+                      float *db, int B, int in, int out, int relu, int out_f32, void *stream) {
+    if (bad_prec(precision) || !x || !W || !dy || !dW || (relu && !y)) return DDG_ERR_INVALID_ARG;
+    if (B < 1 || in < 1 || out < 1) return DDG_ERR_UNSUPPORTED;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (pending_error()) return DDG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (precision == DDG_BF16 && fc_tc_supported(x, W, B, in, out) && aligned16(dW) && aligned16(dx))
+        return done(launch_fc_bwd_tc(x, W, y, dy, dx, dW, db, B, in, out, relu, out_f32, s));
+    return done(launch_fc_bwd(precision, x, W, y, dy, dx, dW, db, B, in, out, relu, out_f32, s));
+}
+
 size_t ddg_bn_scratch_elems(int C) { return C >= 1 && C <= 128 ? bn_scratch_elems(C) : 0; }
 
 ddg_status ddg_bn_fwd(int precision, const void *x, const void *gamma, const void *beta, const void *res, void *y,

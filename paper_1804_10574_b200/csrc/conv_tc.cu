@@ -1430,6 +1430,7 @@ int conv_tc_init() {
         e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
         if (e != cudaSuccess) break;
     }
+    if (e == cudaSuccess) e = (cudaError_t)fc_tc_init();
     rc = (int)e;
     return rc;
 }

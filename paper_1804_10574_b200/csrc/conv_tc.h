@@ -55,6 +55,18 @@ size_t wgrad_tc_scratch_elems();
 int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C, int cin_real,
                     Launch s);
 
+// Fully connected layers on the tensor cores (fc_tc.cu): x [B][in] and W [out][in] row-major bf16, read in place by TMA.
+// Shapes taken: in a multiple of 64 up to 256, out up to 128; x and W must start on a 16-byte boundary, dx and dW too.
+// y / dy are fp32 when out_f32 (the network's last layer: logits and loss gradient), else bf16; dW / db fp32; dx (nullable)
+// bf16; y is only read when relu.  The backward launch produces dx, dW and db in one kernel.
+bool fc_tc_shape_supported(int B, int in, int out);
+bool fc_tc_supported(const void *x, const void *W, int B, int in, int out);
+int launch_fc_fwd_tc(const void *x, const void *W, const void *bias, void *y, int B, int in, int out, int relu, int out_f32,
+                     Launch s);
+int launch_fc_bwd_tc(const void *x, const void *W, const void *y, const void *dy, void *dx, float *dW, float *db, int B,
+                     int in, int out, int relu, int out_f32, Launch s);
+int fc_tc_init();
+
 // One-time per-process set-up (function attributes, driver entry points).  Returns a cudaError_t value.
 int conv_tc_init();
 // The process-wide error word that kernels launched without a context's own word (Launch::err == nullptr) raise when a

@@ -187,6 +187,21 @@ int conv_wgrad(ddg_ctx *c, Module &m, const void *x, const void *dy, float *dw, 
     return launch_conv_wgrad_direct(c->prec, x, dy, dw, m.wg_scratch, c->B, H, W, Cin, Cout, stride, s);
 }
 
+// ---- FC dispatch: tensor-core kernels in bf16 mode where shape and alignment allow, CUDA cores otherwise -----------
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+int fc_fwd(ddg_ctx *c, const void *x, const void *W, const void *bias, void *y, int in, int out, int relu, int out_f32,
+           Launch s) {
+    if (c->prec == P_BF16 && fc_tc_supported(x, W, c->B, in, out))
+        return launch_fc_fwd_tc(x, W, bias, y, c->B, in, out, relu, out_f32, s);
+    return launch_fc_fwd(c->prec, x, W, bias, y, c->B, in, out, relu, out_f32, s);
+}
+int fc_bwd(ddg_ctx *c, const void *x, const void *W, const void *y, const void *dy, void *dx, float *dW, float *db, int in,
+           int out, int relu, int out_f32, Launch s) {
+    if (c->prec == P_BF16 && fc_tc_supported(x, W, c->B, in, out) && aligned16(dW) && aligned16(dx))
+        return launch_fc_bwd_tc(x, W, y, dy, dx, dW, db, c->B, in, out, relu, out_f32, s);
+    return launch_fc_bwd(c->prec, x, W, y, dy, dx, dW, db, c->B, in, out, relu, out_f32, s);
+}
+
 // ---- forward sweep of module k on the minibatch of iteration t (Eq. 3) --------------------------------
 Count forward_module(ddg_ctx *c, int k, long t) {
     Module &m = c->mods[k];
@@ -213,8 +228,8 @@ Count forward_module(ddg_ctx *c, int k, long t) {
         const int B = c->B;
         switch (L.spec.kind) {
         case DDG_FC:
-            n += launch_fc_fwd(c->prec, in, w, L.spec.has_bias ? w + (size_t)L.Cin * L.Cout * es : nullptr, out, B,
-                               L.Cin, L.Cout, L.spec.relu_after, L.is_last, s);
+            n += fc_fwd(c, in, w, L.spec.has_bias ? w + (size_t)L.Cin * L.Cout * es : nullptr, out, L.Cin, L.Cout,
+                        L.spec.relu_after, L.is_last, s);
             break;
         case DDG_CONV3X3:
             if (L.pad_c)  // stem on the tensor cores: input and filter image zero-padded to pad_c channels
@@ -346,8 +361,8 @@ Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
         }
         switch (L.spec.kind) {
         case DDG_FC:
-            n += launch_fc_bwd(c->prec, in, w, out, cur, dst, gw, L.spec.has_bias ? gw + (size_t)L.Cin * L.Cout : nullptr,
-                               B, L.Cin, L.Cout, L.spec.relu_after, L.is_last, s);
+            n += fc_bwd(c, in, w, out, cur, dst, gw, L.spec.has_bias ? gw + (size_t)L.Cin * L.Cout : nullptr, L.Cin,
+                        L.Cout, L.spec.relu_after, L.is_last, s);
             break;
         case DDG_CONV3X3: {
             const char *dy = cur;

@@ -11,7 +11,7 @@ from tests.parity import rel, run_pair  # noqa: F401
 pytestmark = pytest.mark.gpu
 
 FP32_TOL, BF16_TOL, LOSS_TOL = 1e-4, 2e-2, 1e-3
-RATIO_BAND = (0.6, 1.4)        # median of rel(gpu, exact) / rel(oracle_bf16, exact) over gradient tensors
+RATIO_BAND = (0.85, 1.2)       # median of rel(gpu, exact) / rel(oracle_bf16, exact) over gradient tensors
 
 
 def test_mlp_k2_20_steps_fp32():
@@ -56,9 +56,11 @@ def test_resnet8_k2_20_steps_fp32():
 
 
 def test_resnet8_first_steps_fp32_vs_exact():
-    """Before any ReLU decision has had time to be amplified (three iterations from identical weights) the fp32 path is
-    within the fp32 bar of the exact oracle as well."""
-    w = run_pair(nets.config("resnet8"), 3, FP32_TOL, LOSS_TOL, exact_too=True)
+    """Where no ReLU pre-activation falls within fp32 rounding of zero (batch 4: 0.3 M decisions per iteration instead of
+    2.4 M; three iterations from identical weights) the fp32 path is within the fp32 bar of the exact oracle as well.  At
+    batch 32 the first such event already falls inside the first three iterations (seen: one gradient tensor 1.4e-2 off
+    while the weights are still within 6e-5)."""
+    w = run_pair(nets.config("resnet8"), 3, FP32_TOL, LOSS_TOL, exact_too=True, batch=4)
     print("resnet8 first steps vs exact", w)
     assert w["grad_vs_exact"] <= FP32_TOL and w["weight_vs_exact"] <= FP32_TOL
 

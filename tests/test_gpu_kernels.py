@@ -199,7 +199,7 @@ def test_sgd_update(n, prec):
         g_o = o.get_grads(0)[1]
         w1_o = o.get_weights()
         w2, v2, g2 = torch.from_numpy(w).cuda(), torch.zeros(n, device="cuda"), torch.from_numpy(g_o.astype(np.float32)).cuda()
-        binding.sgd_update(prec, w2, v2, g2, wv, n, 0.1, 0.9, 5e-4)
+        binding.sgd_update(prec, w2, v2, g2, torch.empty_like(wv), n, 0.1, 0.9, 5e-4)
         torch.cuda.synchronize()
         assert rel(w2.cpu().numpy(), w1_o) < 1e-6 and rel(v2.cpu().numpy(), g_o + f32(5e-4) * w.astype(np.float64)) < 1e-6
     assert torch.equal(wv, wd.to(tdtype(prec)))      # the version slot is the cast of the new master weights
@@ -341,3 +341,67 @@ def test_stride2_input_gradient_with_parameter_free_shortcut(shape):
     binding.conv3x3_s2_dgrad_shortcut(dy, w, dx2, None, None, B, H, W, Ci)
     torch.cuda.synchronize()
     check_map(from_dev(dx2), orc.conv3x3_backward(np.zeros((B, Ci, H, W)), wh, dyh, 2)[0], 1, "stride-2 input gradient")
+
+
+# B, in, out: the paper's heads (64 -> 10 / 100 at batch 128), the MLP's layers, a ragged batch, several batch tiles,
+# the widest shapes the tensor-core path takes, and shapes it leaves to the CUDA-core kernels (in = 96, out = 200)
+FC_SHAPES = [(128, 64, 100), (128, 64, 10), (16, 64, 128), (16, 128, 128), (16, 128, 10), (7, 64, 10), (300, 128, 100),
+             (515, 256, 128), (33, 192, 48), (5, 96, 12), (9, 64, 200)]
+
+
+@pytest.mark.parametrize("prec", [0, 1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("shape", FC_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("relu,out_f32,bias,want_dx", [(0, 1, 1, 1), (1, 0, 1, 1), (1, 0, 0, 0)],
+                         ids=["head", "hidden", "first_nobias"])
+def test_fc_fwd_bwd(shape, prec, relu, out_f32, bias, want_dx):
+    """Eq. 3-5 for a fully connected layer against the oracle's primitives: forward (bias, ReLU), input gradient,
+    weight and bias gradient, as the last layer (fp32 logits and loss gradient: the tensor-core path keeps the loss
+    gradient to ~16 bits) and as a hidden layer (bf16 in and out, ReLU mask)."""
+    from paper_1804_10574_b200 import binding
+    B, n_in, n_out = shape
+    rng = np.random.default_rng(31)
+    dt = tdtype(prec)
+    odt = torch.float32 if out_f32 else dt
+    x = torch.from_numpy(rng.standard_normal((B, n_in))).to(dt)
+    W = torch.from_numpy(rng.standard_normal((n_out, n_in)) * np.sqrt(2.0 / n_in)).to(dt)
+    b = torch.from_numpy(0.3 * rng.standard_normal(n_out)).to(dt)
+    dy = torch.from_numpy(rng.standard_normal((B, n_out)) / B).to(odt)
+    xh, Wh, bh, dyh = (t.to(torch.float64).numpy() for t in (x, W, b, dy))
+    xd, Wd, bd, dyd = x.cuda(), W.cuda(), b.cuda(), dy.cuda()
+    y = torch.empty(B, n_out, dtype=odt, device="cuda")
+    dx = torch.full((B, n_in), 7.0, dtype=dt, device="cuda")
+    dW = torch.full((n_out, n_in), 7.0, dtype=torch.float32, device="cuda")
+    db = torch.full((n_out,), 7.0, dtype=torch.float32, device="cuda")
+    binding.fc_fwd(prec, xd, Wd, bd if bias else None, y, B, n_in, n_out, relu, out_f32)
+    binding.fc_bwd(prec, xd, Wd, y, dyd, dx if want_dx else None, dW, db if bias else None, B, n_in, n_out, relu, out_f32)
+    torch.cuda.synchronize()
+    y_ref = orc.fc_forward(xh, Wh, bh if bias else np.zeros(n_out))
+    if relu:
+        y_ref = np.maximum(y_ref, 0)
+    yg = y.to(torch.float64).cpu().numpy()
+    ytol = 1e-5 if (prec == 0 or out_f32) else TOL[1]
+    assert rel(yg, y_ref) < ytol
+    rms = float(np.sqrt(np.mean(y_ref ** 2)))
+    ok, idx, excess = elementwise_ok(yg, y_ref, 1e-5 if (prec == 0 or out_f32) else RTOL[1], (1e-5 if prec == 0 else 1e-3) * rms)
+    assert ok, "fc output element %r off by %.3e" % (idx, excess)
+    dz = dyh * (yg > 0) if relu else dyh          # the mask of the output the GPU stored
+    dx_ref, dW_ref, db_ref = orc.fc_backward(xh, Wh, dz, True)
+    if want_dx:
+        assert rel(dx.to(torch.float64).cpu().numpy(), dx_ref) < TOL[prec]
+    else:
+        assert float(dx.float().min()) == 7.0                     # untouched
+    assert rel(dW.cpu().numpy(), dW_ref) < (2e-4 if prec else 1e-5)
+    ok, idx, excess = elementwise_ok(dW.cpu().numpy(), dW_ref, 2e-4 if prec else 1e-5,
+                                     (2e-4 if prec else 1e-6) * float(np.sqrt(np.mean(dW_ref ** 2))))
+    assert ok, "fc weight gradient element %r off by %.3e" % (idx, excess)
+    if bias:
+        assert rel(db.cpu().numpy(), db_ref) < 1e-5
+    else:
+        assert float(db.min()) == 7.0
+
+
+def test_fc_tensor_core_path_takes_the_paper_shapes():
+    from paper_1804_10574_b200 import binding
+    for B, i, o in [(128, 64, 100), (128, 64, 10), (16, 64, 128), (16, 128, 128), (16, 128, 10), (515, 256, 128)]:
+        assert binding.fc_tensor_core_path(B, i, o) == 1, (B, i, o)
+    assert binding.fc_tensor_core_path(5, 96, 12) == 0 and binding.fc_tensor_core_path(9, 64, 200) == 0
