@@ -32,6 +32,13 @@ def test_mlp_ragged_batch_and_momentum_fp32():
     run_pair(cfg, 8, FP32_TOL, LOSS_TOL, batch=7)
 
 
+def test_mlp_k2_bf16():
+    """Config 1 in the bf16 mode: every layer runs on the tensor-core FC kernels (forward, and dx / dW / db in one
+    launch).  A four-layer network stores few tensors, so the plain bf16 tolerance applies."""
+    w = run_pair(nets.config("mlp"), 10, BF16_TOL, 5e-3, precision="bf16")
+    print("mlp bf16 worst", w)
+
+
 def test_mlp_adam_fp32():
     cfg = dict(nets.config("mlp"), opt=dict(lr=1e-3, momentum=0.0, weight_decay=0.0))
     run_pair(cfg, 8, FP32_TOL, LOSS_TOL, opt="adam")
