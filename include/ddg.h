@@ -146,6 +146,18 @@ ddg_status ddg_last_step_launches(const ddg_ctx *ctx, long *launches);
 /* Wait for all K streams; surfaces deferred device-side errors. */
 ddg_status ddg_sync(ddg_ctx *ctx);
 
+/* Exact checkpoint / resume.  A DDG run has state in flight between iterations: module k still owes the backward sweeps
+ * of the K-k most recent samples, so besides the master weights and optimiser state a checkpoint holds every module's
+ * activation ring and weight-version ring (Section 3.1: h^s and w^s of the pending samples), the error gradients handed
+ * over but not yet consumed (Eq. 7), and the iteration count t.  ddg_state_bytes gives the size; ddg_save_state waits
+ * for all enqueued work and copies the state into a host buffer of that size; ddg_load_state restores it into a context
+ * created with the same network, split, precision, batch and optimiser kind (anything else: DDG_ERR_INVALID_ARG), after
+ * which the run continues bit for bit as the saved one would have (same kernels, fixed summation orders).  The step
+ * size is the caller's (ddg_set_lr) and is not part of the state. */
+ddg_status ddg_state_bytes(const ddg_ctx *ctx, size_t *bytes);
+ddg_status ddg_save_state(ddg_ctx *ctx, void *dst_host, size_t bytes);
+ddg_status ddg_load_state(ddg_ctx *ctx, const void *src_host, size_t bytes);
+
 /* Diagnostics (no counterpart in the paper).  Every device-side wait in the library is bounded: a wait that runs out
  * raises the context's error word instead of hanging, the kernel returns, and the next sync point (ddg_sync,
  * ddg_get_weights, ddg_get_grads, ddg_step with a loss) answers DDG_ERR_TIMEOUT, after which the context is in

@@ -30,7 +30,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_conv3x3_packed_bytes", "ddg_conv3x3_pack", "ddg_conv3x3_packed", "ddg_bn_bwd_reduce",
            "ddg_debug_wait_timeout", "ddg_debug_shift_stamps", "ddg_conv3x3_fused_scratch_elems",
            "ddg_conv3x3_fwd_stats", "ddg_conv3x3_dgrad_fused", "ddg_conv3x3_s2_dgrad_shortcut",
-           "ddg_fc_tensor_core_path", "ddg_fc_fwd", "ddg_fc_bwd"]
+           "ddg_fc_tensor_core_path", "ddg_fc_fwd", "ddg_fc_bwd", "ddg_state_bytes", "ddg_save_state",
+           "ddg_load_state"]
 
 
 class Layer(ctypes.Structure):
@@ -63,6 +64,9 @@ _lib.ddg_get_grads.argtypes = [_vp, _i, _vp, _sz, _i, ctypes.POINTER(ctypes.c_lo
 _lib.ddg_get_loss_dev.argtypes = [_vp, ctypes.POINTER(_vp)]
 _lib.ddg_last_step_launches.argtypes = [_vp, ctypes.POINTER(ctypes.c_long)]
 _lib.ddg_sync.argtypes = [_vp]
+_lib.ddg_state_bytes.argtypes = [_vp, ctypes.POINTER(_sz)]
+_lib.ddg_save_state.argtypes = [_vp, _vp, _sz]
+_lib.ddg_load_state.argtypes = [_vp, _vp, _sz]
 _lib.ddg_debug_wait_timeout.argtypes = [_vp, ctypes.c_uint]
 _lib.ddg_debug_shift_stamps.argtypes = [_vp, _i, ctypes.c_long]
 _lib.ddg_last_error.argtypes = [_vp]
@@ -198,6 +202,19 @@ class Ddg:
 
     def sync(self):
         self._check(_lib.ddg_sync(self._h))
+
+    def state_bytes(self):
+        n = ctypes.c_size_t()
+        self._check(_lib.ddg_state_bytes(self._h, ctypes.byref(n)))
+        return n.value
+
+    def save_state(self, dst_host):
+        """dst_host: a writable host buffer (numpy uint8 array) of state_bytes() bytes."""
+        self._check(_lib.ddg_save_state(self._h, _ptr(dst_host), dst_host.nbytes))
+        return dst_host
+
+    def load_state(self, src_host):
+        self._check(_lib.ddg_load_state(self._h, _ptr(src_host), src_host.nbytes))
 
     def debug_wait_timeout(self, polls):
         self._check(_lib.ddg_debug_wait_timeout(self._h, polls))

@@ -1080,6 +1080,89 @@ ddg_status ddg_last_step_launches(const ddg_ctx *ctx, long *launches) {
     return DDG_OK;
 }
 
+// ---- checkpoint / resume -------------------------------------------------------------------------------------
+namespace {
+struct StateHeader {
+    unsigned long long magic;
+    int version, K, n_layers, prec, B, opt_kind, classes, pad_;
+    unsigned long long P, body_bytes;
+    long t;
+};
+constexpr unsigned long long kStateMagic = 0x4444475f53544154ull;  // "DDG_STAT"
+
+// every device buffer that carries state from one iteration to the next, in a fixed order
+void state_regions(ddg_ctx *c, std::vector<std::pair<void *, size_t>> *out) {
+    const size_t es = elem_size(c->prec);
+    for (auto &m : c->mods) {
+        const size_t pn = m.P;
+        out->push_back({m.w, pn * 4}); out->push_back({m.v, pn * 4}); out->push_back({m.g, pn * 4});
+        if (m.m2) out->push_back({m.m2, pn * 4});
+        out->push_back({m.wver, pn * es * m.R});
+        out->push_back({m.arena, m.arena_bytes * m.R});
+        if (m.packed) out->push_back({m.packed, m.packed_bytes * m.R});
+        for (char *d : m.delta_out) if (d) out->push_back({d, m.delta_bytes});
+        out->push_back({m.stamps, (3 + 2 * (size_t)m.R + 2) * sizeof(long long)});
+    }
+    out->push_back({c->loss_dev, 4});
+}
+size_t state_body_bytes(ddg_ctx *c) {
+    std::vector<std::pair<void *, size_t>> r;
+    state_regions(c, &r);
+    size_t n = (size_t)c->K * sizeof(long);  // last_sample per module
+    for (auto &p : r) n += p.second;
+    return n;
+}
+}  // namespace
+
+ddg_status ddg_state_bytes(const ddg_ctx *ctx, size_t *bytes) {
+    if (!ctx || !bytes) return DDG_ERR_INVALID_ARG;
+    *bytes = sizeof(StateHeader) + state_body_bytes(const_cast<ddg_ctx *>(ctx));
+    return DDG_OK;
+}
+
+ddg_status ddg_save_state(ddg_ctx *ctx, void *dst_host, size_t bytes) {
+    if (!ctx || !dst_host) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    const size_t body = state_body_bytes(ctx);
+    if (bytes != sizeof(StateHeader) + body) { set_err(ctx, "ddg_save_state: buffer size does not match ddg_state_bytes"); return DDG_ERR_INVALID_ARG; }
+    ddg_status st = sync_all(ctx);
+    if (st != DDG_OK) return st;
+    StateHeader h{};
+    h.magic = kStateMagic; h.version = 1; h.K = ctx->K; h.n_layers = ctx->n_layers; h.prec = ctx->prec; h.B = ctx->B;
+    h.opt_kind = ctx->opt.kind; h.classes = ctx->classes; h.P = ctx->P; h.body_bytes = body; h.t = ctx->t;
+    char *p = static_cast<char *>(dst_host);
+    memcpy(p, &h, sizeof(h)); p += sizeof(h);
+    for (auto &m : ctx->mods) { memcpy(p, &m.last_sample, sizeof(long)); p += sizeof(long); }
+    std::vector<std::pair<void *, size_t>> r;
+    state_regions(ctx, &r);
+    for (auto &q : r) { CU(cudaMemcpy(p, q.first, q.second, cudaMemcpyDeviceToHost)); p += q.second; }
+    return DDG_OK;
+}
+
+ddg_status ddg_load_state(ddg_ctx *ctx, const void *src_host, size_t bytes) {
+    if (!ctx || !src_host || bytes < sizeof(StateHeader)) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    StateHeader h;
+    memcpy(&h, src_host, sizeof(h));
+    const size_t body = state_body_bytes(ctx);
+    if (h.magic != kStateMagic || h.version != 1 || h.K != ctx->K || h.n_layers != ctx->n_layers || h.prec != ctx->prec ||
+        h.B != ctx->B || h.opt_kind != ctx->opt.kind || h.classes != ctx->classes || h.P != ctx->P || h.body_bytes != body ||
+        bytes != sizeof(StateHeader) + body || h.t < 0) {
+        set_err(ctx, "ddg_load_state: the checkpoint was not written by a context of this shape");
+        return DDG_ERR_INVALID_ARG;
+    }
+    ddg_status st = sync_all(ctx);
+    if (st != DDG_OK) return st;
+    const char *p = static_cast<const char *>(src_host) + sizeof(h);
+    for (auto &m : ctx->mods) { memcpy(&m.last_sample, p, sizeof(long)); p += sizeof(long); m.dyn_valid = false; }
+    std::vector<std::pair<void *, size_t>> r;
+    state_regions(ctx, &r);
+    for (auto &q : r) { CU(cudaMemcpy(q.first, p, q.second, cudaMemcpyHostToDevice)); p += q.second; }
+    CU(cudaDeviceSynchronize());  // the copies ran on the default stream; the module streams do not wait for it
+    ctx->t = h.t;
+    return DDG_OK;
+}
+
 ddg_status ddg_debug_wait_timeout(ddg_ctx *ctx, unsigned polls) {
     if (!ctx || polls == 0) return DDG_ERR_INVALID_ARG;
     if (ctx->broken) return DDG_ERR_STATE;

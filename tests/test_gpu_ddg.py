@@ -282,3 +282,50 @@ def test_ring_stamps_catch_a_shifted_slot():
         d.sync()
     assert e.value.status == 7 and "ring stamp" in str(e.value)
     d.destroy()
+
+
+@pytest.mark.parametrize("net,splits,prec,opt", [("resnet8", [1, 2], "bf16", "sgd"), ("mlp", [0, 1, 2], "fp32", "adam"),
+                                                  ("resnet8", [2], "fp32", "sgd")], ids=["resnet8_K3_bf16", "mlp_K4_adam", "resnet8_K2_fp32"])
+def test_checkpoint_resume_is_exact(net, splits, prec, opt):
+    """A checkpoint taken in the middle of a run (modules owe backward sweeps for up to K-1 samples: activation rings,
+    weight versions and pending error gradients are part of the state) restored into a fresh context, and restored into
+    the context that wrote it, continues bit for bit as the uninterrupted run, graph replay on."""
+    from paper_1804_10574_b200 import binding, synth
+    cfg = nets.config(net)
+    B = 8
+    kw = dict(precision=prec, opt=opt, lr=1e-3 if opt == "adam" else 0.05, momentum=0.9, weight_decay=5e-4, use_graph=True)
+
+    def make():
+        d = binding.Ddg(cfg["layers"], splits, B, cfg["in_shape"], cfg["num_classes"], **kw)
+        d.set_weights(synth.init_weights(cfg["layers"], perturb_affine=0.1))
+        return d
+
+    def run(d, t0, t1):
+        losses = []
+        for t in range(t0, t1):
+            x, y = synth.batch(t, B, cfg["in_shape"], cfg["num_classes"])
+            losses.append(d.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()))
+        w = np.empty(d.n_params, dtype=np.float32)
+        d.get_weights(w)
+        grads = [np.empty(n, dtype=np.float32) for n in d.per_module]
+        samples = [d.get_grads(k, g) for k, g in enumerate(grads)]
+        return losses, w, grads, samples
+
+    a = make()
+    run(a, 0, 7)
+    blob = a.save_state(np.empty(a.state_bytes(), dtype=np.uint8))
+    ref = run(a, 7, 12)
+    b = make()                       # fresh context: nothing recorded, iteration count 0
+    b.load_state(blob)
+    got = run(b, 7, 12)
+    a.load_state(blob)               # roll the writer back
+    again = run(a, 7, 12)
+    for other in (got, again):
+        assert other[0] == ref[0] and np.array_equal(other[1], ref[1]) and other[3] == ref[3]
+        assert all(np.array_equal(g, h) for g, h in zip(other[2], ref[2]))
+    c = binding.Ddg(cfg["layers"], splits, B + 1, cfg["in_shape"], cfg["num_classes"], **kw)   # another batch size
+    with pytest.raises(binding.DdgError) as e:
+        c.load_state(blob)
+    assert e.value.status == 1
+    for d in (a, b, c):
+        d.destroy()
