@@ -21,6 +21,10 @@
  *     out = relu(bn2(conv2(relu(bn1(conv1(x))))) + sc(x)); parameter-free shortcut
  *     sc(x)[n,c,h,w] = x[n,c,s*h,s*w] for c < Cin and 0 for the added channels; global mean pool;
  *     fully connected head with bias; mean softmax cross-entropy; relu'(0) = 0.
+ *   - ORC_BASIC_BLOCK_PROJ is the same block with a projection shortcut in place of the parameter-free one:
+ *     sc(x) = W_s x as a 1x1 convolution with the block's stride, no bias and no batch norm (the paper only
+ *     says "ResNet"; this is the plain linear projection of the residual-learning formulation, taken as a second
+ *     workload).  Its weight W_s [Cout][Cin] follows bn2.beta in the flat parameter order.
  *   - minibatch loss and gradients are means over the batch.
  *   - momentum / weight decay: d = g + wd*w ; v = mu*v + d ; w = w - lr*v.
  *   - during a module's warm-up (s < 0) nothing at all is applied to it (flag ORC_WARMUP_DECAY
@@ -50,7 +54,8 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORC_FC = 0, ORC_CONV3X3 = 1, ORC_BN = 2, ORC_RELU = 3, ORC_BASIC_BLOCK = 4, ORC_GLOBAL_AVGPOOL = 5 };
+enum { ORC_FC = 0, ORC_CONV3X3 = 1, ORC_BN = 2, ORC_RELU = 3, ORC_BASIC_BLOCK = 4, ORC_GLOBAL_AVGPOOL = 5,
+       ORC_BASIC_BLOCK_PROJ = 6 };
 enum { ORC_SGD = 0, ORC_ADAM = 1 };
 enum { ORC_USE_CURRENT_WEIGHTS = 1, ORC_WARMUP_DECAY = 2, ORC_ROUND_BF16 = 4, ORC_ROUND_FP32 = 8 };
 
@@ -278,6 +283,52 @@ void orc_relu_backward(size_t n, const double *y, const double *dy, double *dx) 
     for (size_t i = 0; i < n; ++i) dx[i] = y[i] > 0.0 ? dy[i] : 0.0;
 }
 
+/* 1x1 convolution with a spatial stride, no padding, no bias (projection shortcut):
+ * y[n,co,ho,wo] = sum_ci w[co][ci] * x[n,ci,stride*ho,stride*wo] */
+void orc_conv1x1_forward(int B, int Cin, int H, int W, int Cout, int stride, const double *x, const double *w,
+                         double *y) {
+    const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+#pragma omp parallel for collapse(2)
+    for (int n = 0; n < B; ++n)
+        for (int co = 0; co < Cout; ++co)
+            for (int ho = 0; ho < Ho; ++ho)
+                for (int wo = 0; wo < Wo; ++wo) {
+                    double acc = 0.0;
+                    for (int ci = 0; ci < Cin; ++ci)
+                        acc += w[(size_t)co * Cin + ci] * x[(((size_t)n * Cin + ci) * H + stride * ho) * W + stride * wo];
+                    y[(((size_t)n * Cout + co) * Ho + ho) * Wo + wo] = acc;
+                }
+}
+
+/* dx[n,ci,stride*ho,stride*wo] = sum_co w[co][ci] * dy[n,co,ho,wo] (zero at the pixels the stride skips);
+ * dw[co][ci] = sum_{n,ho,wo} dy[n,co,ho,wo] * x[n,ci,stride*ho,stride*wo] */
+void orc_conv1x1_backward(int B, int Cin, int H, int W, int Cout, int stride, const double *x, const double *w,
+                          const double *dy, double *dx, double *dw) {
+    const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    memset(dx, 0, sizeof(double) * (size_t)B * Cin * H * W);
+#pragma omp parallel for collapse(2)
+    for (int n = 0; n < B; ++n)
+        for (int ci = 0; ci < Cin; ++ci)
+            for (int ho = 0; ho < Ho; ++ho)
+                for (int wo = 0; wo < Wo; ++wo) {
+                    double acc = 0.0;
+                    for (int co = 0; co < Cout; ++co)
+                        acc += w[(size_t)co * Cin + ci] * dy[(((size_t)n * Cout + co) * Ho + ho) * Wo + wo];
+                    dx[(((size_t)n * Cin + ci) * H + stride * ho) * W + stride * wo] = acc;
+                }
+#pragma omp parallel for collapse(2)
+    for (int co = 0; co < Cout; ++co)
+        for (int ci = 0; ci < Cin; ++ci) {
+            double acc = 0.0;
+            for (int n = 0; n < B; ++n)
+                for (int ho = 0; ho < Ho; ++ho)
+                    for (int wo = 0; wo < Wo; ++wo)
+                        acc += dy[(((size_t)n * Cout + co) * Ho + ho) * Wo + wo] *
+                               x[(((size_t)n * Cin + ci) * H + stride * ho) * W + stride * wo];
+            dw[(size_t)co * Cin + ci] = acc;
+        }
+}
+
 /* parameter-free shortcut: spatial subsampling by `stride`, new channels are zero */
 void orc_shortcut_forward(int B, int Cin, int H, int W, int Cout, int stride, const double *x, double *y) {
     const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
@@ -471,10 +522,11 @@ static double *layer_forward(orc_ctx *c, const layer_t *L, const double *w, cons
         orc_avgpool_forward(B, L->C_in, L->H_in * L->W_in, x, y);
         maybe_round(c, y, n_out);
         break;
-    case ORC_BASIC_BLOCK: {
+    case ORC_BASIC_BLOCK:
+    case ORC_BASIC_BLOCK_PROJ: {
         const int Ci = L->C_in, Co = L->C_out, st = L->spec.stride;
         const double *w1 = w, *g1 = w1 + (size_t)Co * Ci * 9, *b1 = g1 + Co;
-        const double *w2 = b1 + Co, *g2 = w2 + (size_t)Co * Co * 9, *b2 = g2 + Co;
+        const double *w2 = b1 + Co, *g2 = w2 + (size_t)Co * Co * 9, *b2 = g2 + Co, *ws = b2 + Co;
         const int HWo = L->H_out * L->W_out;
         q->y1 = dalloc(n_out); q->a1 = dalloc(n_out); q->y2 = dalloc(n_out);
         q->m1 = dalloc(Co); q->is1 = dalloc(Co); q->m2 = dalloc(Co); q->is2 = dalloc(Co);
@@ -487,7 +539,12 @@ static double *layer_forward(orc_ctx *c, const layer_t *L, const double *w, cons
         maybe_round(c, q->y2, n_out);
         double *z = dalloc(n_out), *sc = dalloc(n_out);
         bn_forward_stored(c, B, Co, HWo, q->y2, g2, b2, z, q->m2, q->is2);
-        orc_shortcut_forward(B, Ci, L->H_in, L->W_in, Co, st, x, sc);
+        if (L->spec.kind == ORC_BASIC_BLOCK_PROJ) {
+            orc_conv1x1_forward(B, Ci, L->H_in, L->W_in, Co, st, x, ws, sc);
+            maybe_round(c, sc, n_out); /* the projected shortcut is a stored tensor */
+        } else {
+            orc_shortcut_forward(B, Ci, L->H_in, L->W_in, Co, st, x, sc);
+        }
         for (size_t i = 0; i < n_out; ++i) z[i] += sc[i];
         orc_relu_forward(n_out, z, y);
         maybe_round(c, y, n_out);
@@ -529,10 +586,11 @@ static double *layer_backward(const orc_ctx *c, const layer_t *L, const double *
     case ORC_GLOBAL_AVGPOOL:
         orc_avgpool_backward(B, L->C_in, L->H_in * L->W_in, dy, dx);
         break;
-    case ORC_BASIC_BLOCK: {
+    case ORC_BASIC_BLOCK:
+    case ORC_BASIC_BLOCK_PROJ: {
         const int Ci = L->C_in, Co = L->C_out, st = L->spec.stride;
         const size_t nw1 = (size_t)Co * Ci * 9, nw2 = (size_t)Co * Co * 9;
-        const double *w1 = w, *g1 = w1 + nw1, *w2 = g1 + 2 * Co, *g2 = w2 + nw2;
+        const double *w1 = w, *g1 = w1 + nw1, *w2 = g1 + 2 * Co, *g2 = w2 + nw2, *ws = g2 + 2 * Co;
         double *gw1 = gw, *gg1 = gw1 + nw1, *gb1 = gg1 + Co, *gw2 = gb1 + Co, *gg2 = gw2 + nw2, *gb2 = gg2 + Co;
         const int HWo = L->H_out * L->W_out;
         double *dz = dalloc(n_out), *dy2 = dalloc(n_out), *da1 = dalloc(n_out), *dy1 = dalloc(n_out);
@@ -546,7 +604,10 @@ static double *layer_backward(const orc_ctx *c, const layer_t *L, const double *
         bn_backward_stored(c, B, Co, HWo, q->y1, q->m1, q->is1, g1, da1, dy1, gg1, gb1);
         maybe_round(c, dy1, n_out);
         orc_conv3x3_backward(B, Ci, L->H_in, L->W_in, Co, st, q->x, w1, dy1, dx, gw1);
-        orc_shortcut_backward(B, Ci, L->H_in, L->W_in, Co, st, dz, dsc);
+        if (L->spec.kind == ORC_BASIC_BLOCK_PROJ)
+            orc_conv1x1_backward(B, Ci, L->H_in, L->W_in, Co, st, q->x, ws, dz, dsc, gb2 + Co);
+        else
+            orc_shortcut_backward(B, Ci, L->H_in, L->W_in, Co, st, dz, dsc);
         for (size_t i = 0; i < n_in; ++i) dx[i] += dsc[i];
         free(dz); free(dy2); free(da1); free(dy1); free(dsc);
         break;
@@ -565,6 +626,8 @@ static size_t layer_param_count(const orc_layer *s) {
     case ORC_CONV3X3: return (size_t)s->c_in * s->c_out * 9;
     case ORC_BN: return 2 * (size_t)s->c_in;
     case ORC_BASIC_BLOCK: return (size_t)s->c_in * s->c_out * 9 + (size_t)s->c_out * s->c_out * 9 + 4 * (size_t)s->c_out;
+    case ORC_BASIC_BLOCK_PROJ:
+        return (size_t)s->c_in * s->c_out * 9 + (size_t)s->c_out * s->c_out * 9 + 4 * (size_t)s->c_out + (size_t)s->c_in * s->c_out;
     default: return 0;
     }
 }
@@ -591,8 +654,10 @@ orc_ctx *orc_create(const orc_layer *layers, int n_layers, const int *split_afte
         case ORC_FC: ok = (H == 1 && W == 1 && layers[l].c_in == C); C = layers[l].c_out; break;
         case ORC_CONV3X3:
         case ORC_BASIC_BLOCK:
+        case ORC_BASIC_BLOCK_PROJ:
             ok = (layers[l].c_in == C && (layers[l].stride == 1 || layers[l].stride == 2) &&
                   layers[l].c_out >= layers[l].c_in);
+            if (layers[l].kind == ORC_BASIC_BLOCK_PROJ) ok = (layers[l].c_in == C && (layers[l].stride == 1 || layers[l].stride == 2));
             if (layers[l].kind == ORC_CONV3X3) ok = (layers[l].c_in == C && (layers[l].stride == 1 || layers[l].stride == 2));
             C = layers[l].c_out; H = (H - 1) / layers[l].stride + 1; W = (W - 1) / layers[l].stride + 1; break;
         case ORC_BN: ok = (layers[l].c_in == C); break;

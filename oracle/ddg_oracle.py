@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ddg_oracle.c")
 _LIB = os.path.join(_HERE, "libddg_oracle.so")
 
-FC, CONV3X3, BN, RELU, BASIC_BLOCK, GLOBAL_AVGPOOL = range(6)
+FC, CONV3X3, BN, RELU, BASIC_BLOCK, GLOBAL_AVGPOOL, BASIC_BLOCK_PROJ = range(7)
 SGD, ADAM = 0, 1
 USE_CURRENT_WEIGHTS, WARMUP_DECAY, ROUND_BF16, ROUND_FP32 = 1, 2, 4, 8
 
@@ -191,6 +191,20 @@ def conv3x3_backward(x, w, dy, stride):
     B, Ci, H, Wd = x.shape
     dx, dw = np.empty_like(x), np.empty_like(w)
     _call("orc_conv3x3_backward", B, Ci, H, Wd, w.shape[0], stride, x, w, dy, dx, dw)
+    return dx, dw
+
+
+def conv1x1_forward(x, w, stride):
+    B, Ci, H, Wd = x.shape
+    y = np.empty((B, w.shape[0], (H - 1) // stride + 1, (Wd - 1) // stride + 1))
+    _call("orc_conv1x1_forward", B, Ci, H, Wd, w.shape[0], stride, x, w, y)
+    return y
+
+
+def conv1x1_backward(x, w, dy, stride):
+    B, Ci, H, Wd = x.shape
+    dx, dw = np.empty_like(x), np.empty_like(w)
+    _call("orc_conv1x1_backward", B, Ci, H, Wd, w.shape[0], stride, x, w, dy, dx, dw)
     return dx, dw
 
 

@@ -4,7 +4,7 @@ A network is a list of (kind, c_in, c_out, stride, has_bias, relu_after) tuples.
 CIFAR ResNets of Table 2 of the paper (units 1-1-1 / 9-9-9 / 18-18-18, channels 16-16-32-64, basic blocks
 without bottleneck) and a small MLP used as the first parity case.
 """
-FC, CONV3X3, BN, RELU, BASIC_BLOCK, GLOBAL_AVGPOOL = range(6)
+FC, CONV3X3, BN, RELU, BASIC_BLOCK, GLOBAL_AVGPOOL, BASIC_BLOCK_PROJ = range(7)
 
 
 def mlp(dims=(64, 128, 128, 128, 10)):
@@ -15,15 +15,18 @@ def mlp(dims=(64, 128, 128, 128, 10)):
     return layers
 
 
-def resnet(units, num_classes, channels=(16, 16, 32, 64), in_c=3):
-    """Stem conv3x3+BN+ReLU, three stages of `units` basic blocks, global mean pool, FC head (Table 2)."""
+def resnet(units, num_classes, channels=(16, 16, 32, 64), in_c=3, projection=False):
+    """Stem conv3x3+BN+ReLU, three stages of `units` basic blocks, global mean pool, FC head (Table 2).
+    projection: the blocks that change the shape (first of stages 2 and 3) take a 1x1-projection shortcut instead of
+    the parameter-free one."""
     layers = [(CONV3X3, in_c, channels[0], 1, 0, 0), (BN, channels[0], channels[0], 1, 0, 1)]
     c = channels[0]
     for stage in range(3):
         c_out = channels[stage + 1]
         for u in range(units):
             stride = 2 if (stage > 0 and u == 0) else 1
-            layers.append((BASIC_BLOCK, c, c_out, stride, 0, 0))
+            proj = projection and (stride != 1 or c != c_out)
+            layers.append((BASIC_BLOCK_PROJ if proj else BASIC_BLOCK, c, c_out, stride, 0, 0))
             c = c_out
     layers.append((GLOBAL_AVGPOOL, c, c, 1, 0, 0))
     layers.append((FC, c, num_classes, 1, 1, 0))
@@ -33,7 +36,7 @@ def resnet(units, num_classes, channels=(16, 16, 32, 64), in_c=3):
 def split_even_blocks(layers, K):
     """K-1 split indices that cut between residual blocks with (nearly) equal block counts: the first
     (n_blocks mod K) modules get one extra block; the stem stays with module 1, pool+FC with module K."""
-    blocks = [i for i, l in enumerate(layers) if l[0] == BASIC_BLOCK]
+    blocks = [i for i, l in enumerate(layers) if l[0] in (BASIC_BLOCK, BASIC_BLOCK_PROJ)]
     n = len(blocks)
     if K < 1 or K > n:
         raise ValueError("cannot cut %d blocks into %d modules" % (n, K))
@@ -54,15 +57,15 @@ def param_count(layers):
             n += ci * co * 9
         elif kind == BN:
             n += 2 * ci
-        elif kind == BASIC_BLOCK:
-            n += ci * co * 9 + co * co * 9 + 4 * co
+        elif kind in (BASIC_BLOCK, BASIC_BLOCK_PROJ):
+            n += ci * co * 9 + co * co * 9 + 4 * co + (ci * co if kind == BASIC_BLOCK_PROJ else 0)
     return n
 
 
 def param_segments(layers):
     """[(layer index, name, offset, shape, fan_in or None)] in the canonical flat order: per layer the conv/FC
     weight ([Cout][Cin][3][3] or [out][in]), bias, BN gamma, BN beta; a block gives conv1.w, bn1.gamma,
-    bn1.beta, conv2.w, bn2.gamma, bn2.beta."""
+    bn1.beta, conv2.w, bn2.gamma, bn2.beta (and proj.w [Cout][Cin] for a projection shortcut)."""
     segs, off = [], 0
 
     def add(i, name, shape, fan_in):
@@ -83,13 +86,15 @@ def param_segments(layers):
         elif kind == BN:
             add(i, "bn.gamma", (ci,), None)
             add(i, "bn.beta", (ci,), None)
-        elif kind == BASIC_BLOCK:
+        elif kind in (BASIC_BLOCK, BASIC_BLOCK_PROJ):
             add(i, "conv1.w", (co, ci, 3, 3), 9 * ci)
             add(i, "bn1.gamma", (co,), None)
             add(i, "bn1.beta", (co,), None)
             add(i, "conv2.w", (co, co, 3, 3), 9 * co)
             add(i, "bn2.gamma", (co,), None)
             add(i, "bn2.beta", (co,), None)
+            if kind == BASIC_BLOCK_PROJ:
+                add(i, "proj.w", (co, ci), ci)
     return segs
 
 

@@ -10,6 +10,7 @@ from paper_1804_10574_b200 import nets, synth
 from tests import torch_bp
 
 TINY_RESNET = dict(layers=nets.resnet(1, 5, channels=(4, 4, 8, 8)), in_shape=(3, 8, 8), num_classes=5, batch=4)
+TINY_RESNET_PROJ = dict(layers=nets.resnet(1, 5, channels=(4, 4, 8, 8), projection=True), in_shape=(3, 8, 8), num_classes=5, batch=4)
 TINY_MLP = dict(layers=nets.mlp((6, 8, 8, 7, 5)), in_shape=(6, 1, 1), num_classes=5, batch=4)
 
 
@@ -36,7 +37,7 @@ def module_slices(o):
     return out
 
 
-@pytest.mark.parametrize("net", [TINY_MLP, TINY_RESNET], ids=["mlp", "resnet"])
+@pytest.mark.parametrize("net", [TINY_MLP, TINY_RESNET, TINY_RESNET_PROJ], ids=["mlp", "resnet", "resnet_proj"])
 def test_whole_net_finite_differences(net):
     """Every layer's backward sweep, chained: the K=1 gradient equals central differences of the loss."""
     o, w0 = make(net, [], lr=0.0)
@@ -52,7 +53,7 @@ def test_whole_net_finite_differences(net):
         assert abs((fp - fm) / (2 * h) - g[i]) < 1e-6 * max(1.0, abs(g[i])), i
 
 
-@pytest.mark.parametrize("net", [TINY_MLP, TINY_RESNET], ids=["mlp", "resnet"])
+@pytest.mark.parametrize("net", [TINY_MLP, TINY_RESNET, TINY_RESNET_PROJ], ids=["mlp", "resnet", "resnet_proj"])
 def test_k1_is_plain_backprop_with_sgd(net):
     """Section 3.2: with K=1 there is no delay and DDG is backpropagation + SGD (Eq. 2), step by step."""
     lr = 0.05
@@ -69,11 +70,11 @@ def test_k1_is_plain_backprop_with_sgd(net):
         assert rel(o.get_weights(), w) < 1e-11
 
 
-@pytest.mark.parametrize("K,splits", [(2, [2]), (3, [2, 3]), (4, [1, 2, 3])])
-def test_delayed_gradient_is_true_gradient_of_stored_iteration(K, splits):
+@pytest.mark.parametrize("K,splits,net", [(2, [2], TINY_RESNET), (3, [2, 3], TINY_RESNET), (4, [1, 2, 3], TINY_RESNET),
+                                          (3, [2, 3], TINY_RESNET_PROJ)], ids=["K2", "K3", "K4", "K3_proj"])
+def test_delayed_gradient_is_true_gradient_of_stored_iteration(K, splits, net):
     """Eq. 8-9: g_k applied at iteration t is [grad f_{x_s}(w^s)]_{G(k)} with s = t-K+k; delays run from K-1
     (k=1) to 0 (k=K); zero during warm-up, when the module's weights must not move (plain SGD)."""
-    net = TINY_RESNET
     lr = 0.05
     o, w0 = make(net, splits, lr=lr)
     sl = module_slices(o)

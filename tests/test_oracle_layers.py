@@ -207,3 +207,43 @@ def test_bf16_round_is_nearest_even():
     v = torch.randn(1000, dtype=torch.float32)
     ours = np.array([orc.bf16_round(float(a)) for a in v])
     np.testing.assert_array_equal(ours, v.to(torch.bfloat16).to(torch.float64).numpy())
+
+
+# ---- 1x1 projection (shortcut of a shape-changing residual block) ---------------------------------------------
+@pytest.mark.parametrize("stride", [1, 2])
+def test_conv1x1_brute_force_center_tap_and_library(stride):
+    """Three independent statements of the same operation: explicit loops; the (already pinned) 3x3 convolution with a
+    filter that is zero except for its centre tap; the library's conv2d with a 1x1 kernel and no padding."""
+    B, Ci, H, W, Co = 2, 3, 5, 6, 4
+    x, w = RNG.standard_normal((B, Ci, H, W)), RNG.standard_normal((Co, Ci))
+    y = orc.conv1x1_forward(x, w, stride)
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+    brute = np.zeros((B, Co, Ho, Wo))
+    for n, co, ho, wo, ci in itertools.product(range(B), range(Co), range(Ho), range(Wo), range(Ci)):
+        brute[n, co, ho, wo] += w[co, ci] * x[n, ci, stride * ho, stride * wo]
+    np.testing.assert_allclose(y, brute, rtol=1e-13, atol=1e-13)
+    w3 = np.zeros((Co, Ci, 3, 3)); w3[:, :, 1, 1] = w
+    np.testing.assert_allclose(y, orc.conv3x3_forward(x, w3, stride), rtol=1e-13, atol=1e-13)
+    dy = RNG.standard_normal(y.shape)
+    xt, wt = torch.tensor(x, requires_grad=True), torch.tensor(w.reshape(Co, Ci, 1, 1), requires_grad=True)
+    yt = F.conv2d(xt, wt, None, stride, 0)
+    yt.backward(torch.tensor(dy))
+    np.testing.assert_allclose(y, yt.detach().numpy(), rtol=1e-12, atol=1e-13)
+    dx, dw = orc.conv1x1_backward(x, w, dy, stride)
+    np.testing.assert_allclose(dx, xt.grad.numpy(), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(dw, wt.grad.numpy().reshape(Co, Ci), rtol=1e-12, atol=1e-13)
+    # the pixels the stride skips receive no gradient; the centre-tap 3x3 backward agrees on both outputs
+    if stride == 2:
+        assert not dx[:, :, 1::2, :].any() and not dx[:, :, :, 1::2].any()
+    dx3, dw3 = orc.conv3x3_backward(x, w3, dy, stride)
+    np.testing.assert_allclose(dx, dx3, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(dw, dw3[:, :, 1, 1], rtol=1e-12, atol=1e-13)
+
+
+def test_conv1x1_backward_finite_differences():
+    x, w = RNG.standard_normal((2, 3, 4, 4)), RNG.standard_normal((5, 3))
+    r = RNG.standard_normal(orc.conv1x1_forward(x, w, 2).shape)
+    f = lambda: float(np.sum(orc.conv1x1_forward(x, w, 2) * r))
+    dx, dw = orc.conv1x1_backward(x, w, r, 2)
+    np.testing.assert_allclose(dx, fd_grad(f, x), rtol=1e-6, atol=1e-8)
+    np.testing.assert_allclose(dw, fd_grad(f, w), rtol=1e-6, atol=1e-8)

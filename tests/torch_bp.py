@@ -40,15 +40,18 @@ def forward(layers, w, x, y, bn_eps=1e-5):
             h = F.relu(h)
         elif kind == nets.GLOBAL_AVGPOOL:
             h = h.mean(dim=(2, 3))
-        elif kind == nets.BASIC_BLOCK:
+        elif kind in (nets.BASIC_BLOCK, nets.BASIC_BLOCK_PROJ):
             inp = h
             h = F.relu(bn(F.conv2d(inp, take(co, ci, 3, 3), None, stride, 1), co))
             h = bn(F.conv2d(h, take(co, co, 3, 3), None, 1, 1), co)
-            sc = inp[:, :, ::stride, ::stride]
-            if co > ci:
-                sc = F.pad(sc, (0, 0, 0, 0, 0, co - ci))
+            if kind == nets.BASIC_BLOCK_PROJ:
+                sc = F.conv2d(inp, take(co, ci, 1, 1), None, stride, 0)
+            else:
+                sc = inp[:, :, ::stride, ::stride]
+                if co > ci:
+                    sc = F.pad(sc, (0, 0, 0, 0, 0, co - ci))
             h = F.relu(h + sc)
-        if relu and kind != nets.BASIC_BLOCK:
+        if relu and kind not in (nets.BASIC_BLOCK, nets.BASIC_BLOCK_PROJ):
             h = F.relu(h)
     assert off == w.numel()
     return F.cross_entropy(h.reshape(h.shape[0], -1), y)
