@@ -20,8 +20,8 @@
  *
  * Flat parameter order ("canonical order") used by get/set weights and gradients: layers in network order;
  * per layer the conv / FC weight ([Cout][Cin][3][3] or [out][in], row-major), then bias, then BN gamma, then
- * BN beta; a basic block contributes conv1.w, bn1.gamma, bn1.beta, conv2.w, bn2.gamma, bn2.beta.  Always
- * fp32, whatever the internal storage.
+ * BN beta; a basic block contributes conv1.w, bn1.gamma, bn1.beta, conv2.w, bn2.gamma, bn2.beta (then the projection
+ * W_s [Cout][Cin] for DDG_BASIC_BLOCK_PROJ).  Always fp32, whatever the internal storage.
  */
 #ifndef DDG_H_
 #define DDG_H_
@@ -52,9 +52,12 @@ typedef enum {
  *  DDG_RELU           max(x, 0), derivative 0 at 0
  *  DDG_BASIC_BLOCK    out = relu(bn2(conv2(relu(bn1(conv1(x))))) + sc(x)); conv1 has the stride;
  *                     sc = identity, or for stride 2 / wider output x[:, ::2, ::2] zero-padded in channels
- *  DDG_GLOBAL_AVGPOOL mean over H x W  */
+ *  DDG_GLOBAL_AVGPOOL mean over H x W
+ *  DDG_BASIC_BLOCK_PROJ the same block with a projection shortcut: sc(x) = W_s x, a 1x1 convolution with the
+ *                     block's stride, no bias, no batch norm (any c_in -> c_out)  */
 typedef enum {
-    DDG_FC = 0, DDG_CONV3X3 = 1, DDG_BN = 2, DDG_RELU = 3, DDG_BASIC_BLOCK = 4, DDG_GLOBAL_AVGPOOL = 5
+    DDG_FC = 0, DDG_CONV3X3 = 1, DDG_BN = 2, DDG_RELU = 3, DDG_BASIC_BLOCK = 4, DDG_GLOBAL_AVGPOOL = 5,
+    DDG_BASIC_BLOCK_PROJ = 6
 } ddg_layer_kind;
 
 typedef struct {
@@ -95,6 +98,9 @@ typedef struct {
     void *const *streams; /* host array of K cudaStream_t to run the modules on, or NULL (library creates K) */
     int separate_bn_sums; /* 0 (default): the batch-norm sums are taken in the epilogue of the tensor-core convolution
                        that produces the tensor.  1: separate reduction kernels (same sums, other summation order). */
+    int separate_bn_apply; /* 0 (default): inside a residual block the first batch norm's normalise + ReLU pass runs on
+                       the operand path of the second convolution (tensor-core kernel, shared memory) instead of as a
+                       kernel of its own.  1: separate element-wise kernels everywhere (same values, bit for bit). */
     int launch_overlap; /* programmatic dependent launch (the next kernel of a stream is placed while the previous one
                        still runs).  0 (default): the library's policy: every kernel when K = 1; with several module
                        streams only the forward / input-gradient convolutions.  1: never.  2: every kernel. */
@@ -221,12 +227,37 @@ ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *pa
                                    const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
                                    const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H,
                                    int W, int C, void *stream);
+/* ddg_conv3x3_bnrelu_fwd_stats: the second convolution of a residual block as the training step launches it.  x is the
+ * RAW output of the first convolution; the kernel applies that convolution's batch norm and ReLU on its own operand
+ * path, a = relu(gamma * (x - mean_in) * invstd_in + beta) rounded to bf16 (gamma, beta bf16 [C]; mean_in, invstd_in
+ * fp32 [C]), stores a to a_out ([B][H][W][C], what the backward sweep reads) and computes y = conv3x3(a, w) with the
+ * statistics of y as ddg_conv3x3_fwd_stats does (Eq. 3 for batch norm -> ReLU -> convolution).  DDG_ERR_UNSUPPORTED
+ * where the launch plan of the shape has no room for the transform warps (very large batches). */
+ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *gamma, const void *beta, const float *mean_in,
+                                        const float *invstd_in, void *a_out, const void *w, const void *packed, void *y,
+                                        float *mean, float *invstd, float *scratch, int B, int H, int W, int C,
+                                        void *stream);
 /* Input gradient of the stride-2 convolution of a down-sampling block (Cin -> 2 Cin, bf16, tensor-core path only) with
  * the gradient of the block's parameter-free shortcut added: dx[n][2j][2i][c] += res_dout[n][j][i][c] *
  * [res_out[n][j][i][c] > 0] for c < Cin (the shortcut reads every second pixel of every second row and pads the
  * channels with zeros).  dy, res_dout, res_out: [B][H/2][W/2][2 Cin]; dx: [B][H][W][Cin].  res_* nullable (both). */
 ddg_status ddg_conv3x3_s2_dgrad_shortcut(const void *dy, const void *w, void *dx, const void *res_dout,
                                          const void *res_out, int B, int H, int W, int Cin, void *stream);
+
+/* The 1x1 convolution of a projection shortcut (Eq. 3 and Eq. 4-5 for y = W_s x with a spatial stride, no bias).
+ * x [B][H][W][Cin], w [Cout][Cin], y / dout / out [B][Ho][Wo][Cout] with Ho = (H-1)/stride+1, all in the precision's
+ * element type; Cin * Cout <= 4096.
+ *   ddg_conv1x1_fwd        y = W_s x.
+ *   ddg_conv1x1_dgrad_add  dx[n][s*h][s*w][:] += W_s^T dz[n][h][w][:], dz = dout * [out > 0] (out nullable: dz = dout);
+ *                          dx is read and written (the 3x3 convolution's input gradient is already in it).
+ *   ddg_conv1x1_wgrad      dw[co][ci] = sum dz[p][co] x[s*p][ci], fp32; scratch: ddg_conv1x1_wgrad_scratch_elems floats. */
+ddg_status ddg_conv1x1_fwd(int precision, const void *x, const void *w, void *y, int B, int H, int W, int Cin, int Cout,
+                           int stride, void *stream);
+ddg_status ddg_conv1x1_dgrad_add(int precision, const void *dout, const void *out, const void *w, void *dx, int B, int H,
+                                 int W, int Cin, int Cout, int stride, void *stream);
+size_t ddg_conv1x1_wgrad_scratch_elems(int Cin, int Cout);
+ddg_status ddg_conv1x1_wgrad(int precision, const void *x, const void *dout, const void *out, float *dw, float *scratch,
+                             int B, int H, int W, int Cin, int Cout, int stride, void *stream);
 
 /* dw = conv3x3 weight gradient (Eq. 4 / Eq. 6), fp32 [Cout][Cin][3][3].  scratch: device, fp32,
  * ddg_conv3x3_wgrad_scratch_elems(...) elements, contents undefined on entry and exit. */

@@ -31,7 +31,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_debug_wait_timeout", "ddg_debug_shift_stamps", "ddg_conv3x3_fused_scratch_elems",
            "ddg_conv3x3_fwd_stats", "ddg_conv3x3_dgrad_fused", "ddg_conv3x3_s2_dgrad_shortcut",
            "ddg_fc_tensor_core_path", "ddg_fc_fwd", "ddg_fc_bwd", "ddg_state_bytes", "ddg_save_state",
-           "ddg_load_state"]
+           "ddg_load_state", "ddg_conv1x1_fwd", "ddg_conv1x1_dgrad_add", "ddg_conv1x1_wgrad_scratch_elems",
+           "ddg_conv1x1_wgrad", "ddg_conv3x3_bnrelu_fwd_stats"]
 
 
 class Layer(ctypes.Structure):
@@ -48,7 +49,7 @@ class Cfg(ctypes.Structure):
                 ("in_w", ctypes.c_int), ("num_classes", ctypes.c_int), ("seed", ctypes.c_ulonglong),
                 ("use_graph", ctypes.c_int), ("debug_checks", ctypes.c_int),
                 ("streams", ctypes.POINTER(ctypes.c_void_p)), ("separate_bn_sums", ctypes.c_int),
-                ("launch_overlap", ctypes.c_int)]
+                ("separate_bn_apply", ctypes.c_int), ("launch_overlap", ctypes.c_int)]
 
 
 _vp, _i, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -90,8 +91,14 @@ _lib.ddg_conv3x3_packed.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_conv3x3_fused_scratch_elems.argtypes = [_i] * 4
 _lib.ddg_conv3x3_fused_scratch_elems.restype = _sz
 _lib.ddg_conv3x3_fwd_stats.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
+_lib.ddg_conv3x3_bnrelu_fwd_stats.argtypes = [_vp] * 12 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_dgrad_fused.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_s2_dgrad_shortcut.argtypes = [_vp] * 5 + [_i] * 4 + [_vp]
+_lib.ddg_conv1x1_fwd.argtypes = [_i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]
+_lib.ddg_conv1x1_dgrad_add.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]
+_lib.ddg_conv1x1_wgrad_scratch_elems.argtypes = [_i, _i]
+_lib.ddg_conv1x1_wgrad_scratch_elems.restype = _sz
+_lib.ddg_conv1x1_wgrad.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]
 _lib.ddg_fc_tensor_core_path.argtypes = [_i] * 3
 _lib.ddg_fc_fwd.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]
 _lib.ddg_fc_bwd.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]
@@ -127,7 +134,8 @@ class Ddg:
 
     def __init__(self, layers, split_after, batch, in_shape, num_classes, precision="fp32", opt="sgd", lr=0.01,
                  momentum=0.0, weight_decay=0.0, beta1=0.9, beta2=0.999, eps=1e-8, seed=0, use_graph=False,
-                 debug_checks=False, streams=None, separate_bn_sums=False, launch_overlap=0):
+                 debug_checks=False, streams=None, separate_bn_sums=False, separate_bn_apply=False,
+                 launch_overlap=0):
         arr = (Layer * len(layers))(*[Layer(*map(int, l)) for l in layers])
         K = len(split_after) + 1
         sp = (ctypes.c_int * max(1, K - 1))(*split_after)
@@ -137,7 +145,8 @@ class Ddg:
             assert len(streams) == K
             st = (ctypes.c_void_p * K)(*[int(s) for s in streams])
         cfg = Cfg(BF16 if precision == "bf16" else FP32, batch, in_shape[0], in_shape[1], in_shape[2], num_classes,
-                  seed, int(use_graph), int(debug_checks), st, int(separate_bn_sums), int(launch_overlap))
+                  seed, int(use_graph), int(debug_checks), st, int(separate_bn_sums), int(separate_bn_apply),
+                  int(launch_overlap))
         h = ctypes.c_void_p()
         rc = _lib.ddg_create(arr, len(layers), sp, K, ctypes.byref(o), ctypes.byref(cfg), ctypes.byref(h))
         if rc != 0:
@@ -253,6 +262,13 @@ def conv3x3_fwd_stats(x, w, packed, y, mean, invstd, scratch, B, H, W, C, stream
                                    B, H, W, C, stream))
 
 
+def conv3x3_bnrelu_fwd_stats(x, gamma, beta, mean_in, invstd_in, a_out, w, packed, y, mean, invstd, scratch, B, H, W, C,
+                             stream=None):
+    _ok(_lib.ddg_conv3x3_bnrelu_fwd_stats(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(mean_in), _ptr(invstd_in), _ptr(a_out),
+                                          _ptr(w), _ptr(packed), _ptr(y), _ptr(mean), _ptr(invstd), _ptr(scratch), B, H, W, C,
+                                          stream))
+
+
 def conv3x3_dgrad_fused(dy, w, packed, dx, res_dout, res_out, bn_mask, bn_x, bn_mean, bn_invstd, dbeta, dgamma, scratch,
                         B, H, W, C, stream=None):
     _ok(_lib.ddg_conv3x3_dgrad_fused(_ptr(dy), _ptr(w), _ptr(packed), _ptr(dx), _ptr(res_dout), _ptr(res_out),
@@ -279,6 +295,23 @@ def conv3x3_wgrad_scratch_elems(B, H, W, Cin, Cout, stride):
 
 def conv3x3_wgrad(prec, x, dy, dw, scratch, B, H, W, Cin, Cout, stride, stream=None):
     _ok(_lib.ddg_conv3x3_wgrad(prec, _ptr(x), _ptr(dy), _ptr(dw), _ptr(scratch), B, H, W, Cin, Cout, stride, stream))
+
+
+def conv1x1_fwd(prec, x, w, y, B, H, W, Cin, Cout, stride, stream=None):
+    _ok(_lib.ddg_conv1x1_fwd(prec, _ptr(x), _ptr(w), _ptr(y), B, H, W, Cin, Cout, stride, stream))
+
+
+def conv1x1_dgrad_add(prec, dout, out, w, dx, B, H, W, Cin, Cout, stride, stream=None):
+    _ok(_lib.ddg_conv1x1_dgrad_add(prec, _ptr(dout), _ptr(out), _ptr(w), _ptr(dx), B, H, W, Cin, Cout, stride, stream))
+
+
+def conv1x1_wgrad_scratch_elems(Cin, Cout):
+    return _lib.ddg_conv1x1_wgrad_scratch_elems(Cin, Cout)
+
+
+def conv1x1_wgrad(prec, x, dout, out, dw, scratch, B, H, W, Cin, Cout, stride, stream=None):
+    _ok(_lib.ddg_conv1x1_wgrad(prec, _ptr(x), _ptr(dout), _ptr(out), _ptr(dw), _ptr(scratch), B, H, W, Cin, Cout, stride,
+                               stream))
 
 
 def fc_tensor_core_path(B, n_in, n_out):

@@ -125,6 +125,24 @@ ddg_status ddg_conv3x3_fwd_stats(const void *x, const void *w, const void *packe
     return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, s, bf));
 }
 
+ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *gamma, const void *beta, const float *mean_in,
+                                        const float *invstd_in, void *a_out, const void *w, const void *packed, void *y,
+                                        float *mean, float *invstd, float *scratch, int B, int H, int W, int C,
+                                        void *stream) {
+    if (!x || !gamma || !beta || !mean_in || !invstd_in || !a_out || !w || !y || !mean || !invstd || !scratch)
+        return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_xform_supported(B, H, W, C, false)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(scratch, 0, 128, s) != cudaSuccess) return DDG_ERR_CUDA;
+    BnFuse bf;
+    bf.counter = reinterpret_cast<unsigned *>(scratch); bf.part = scratch + 32; bf.o0 = mean; bf.o1 = invstd;
+    InXform xf;
+    xf.gamma = gamma; xf.beta = beta; xf.mean = mean_in; xf.invstd = invstd_in; xf.a_out = a_out;
+    return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, s, bf, xf));
+}
+
 ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
                                    const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
                                    const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H,
@@ -157,6 +175,34 @@ ddg_status ddg_conv3x3_s2_dgrad_shortcut(const void *dy, const void *w, void *dx
     Shortcut sc{};
     if (res_dout) { sc.mode = 2; sc.a = res_dout; sc.b = res_out; sc.c_small = Cin; sc.h_big = H; sc.w_big = W; }
     return done(launch_conv_tc_s2(1, dy, w, nullptr, dx, B, H, W, Cin, sc, (cudaStream_t)stream));
+}
+
+ddg_status ddg_conv1x1_fwd(int precision, const void *x, const void *w, void *y, int B, int H, int W, int Cin, int Cout,
+                           int stride, void *stream) {
+    if (bad_prec(precision) || !x || !w || !y) return DDG_ERR_INVALID_ARG;
+    if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    return done(launch_conv1x1_fwd(precision, x, w, y, B, H, W, Cin, Cout, stride, (cudaStream_t)stream));
+}
+
+ddg_status ddg_conv1x1_dgrad_add(int precision, const void *dout, const void *out, const void *w, void *dx, int B, int H,
+                                 int W, int Cin, int Cout, int stride, void *stream) {
+    if (bad_prec(precision) || !dout || !w || !dx) return DDG_ERR_INVALID_ARG;
+    if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    return done(launch_conv1x1_dgrad_add(precision, dout, out, w, dx, B, H, W, Cin, Cout, stride, (cudaStream_t)stream));
+}
+
+size_t ddg_conv1x1_wgrad_scratch_elems(int Cin, int Cout) {
+    return (Cin >= 1 && Cout >= 1 && (size_t)Cin * Cout <= 4096) ? conv1x1_wgrad_scratch_elems(Cin, Cout) : 0;
+}
+
+ddg_status ddg_conv1x1_wgrad(int precision, const void *x, const void *dout, const void *out, float *dw, float *scratch,
+                             int B, int H, int W, int Cin, int Cout, int stride, void *stream) {
+    if (bad_prec(precision) || !x || !dout || !dw || !scratch) return DDG_ERR_INVALID_ARG;
+    if (!conv_shape_ok(B, H, W, Cin, Cout, stride)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    return done(launch_conv1x1_wgrad(precision, x, dout, out, dw, scratch, B, H, W, Cin, Cout, stride, (cudaStream_t)stream));
 }
 
 size_t ddg_conv3x3_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride) {

@@ -52,8 +52,9 @@ template <int C> __host__ __device__ inline ConvSmem conv_smem_plan(int n_stages
     return p;
 }
 // after the pipeline stages: 512 bytes of barriers and flags, 8 KB of per-warp batch-norm sums (up to 16 epilogue
-// warps x 4 channel chunks x 32 lanes), 512 bytes of per-channel mean / invstd
-constexpr int kTailBytes = 512 + 8192 + 512;
+// warps x 4 channel chunks x 32 lanes), 512 bytes of per-channel mean / invstd, 512 bytes of per-channel scale / shift
+// of the input transform
+constexpr int kTailBytes = 512 + 8192 + 512 + 512;
 template <int C> inline size_t conv_smem_bytes(int n_stages, int stage_bytes) {
     return 1024 + conv_smem_plan<C>(n_stages, stage_bytes).tail_off + kTailBytes;
 }
@@ -168,7 +169,13 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                   const bf16 *__restrict__ res_out, float *__restrict__ stat_part, unsigned *__restrict__ stat_counter,
                   float *__restrict__ stat_o0, float *__restrict__ stat_o1, const bf16 *__restrict__ bn_mask,
                   const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd,
-                  int *__restrict__ err_word) {
+                  const bf16 *__restrict__ xf_gamma, const bf16 *__restrict__ xf_beta, const float *__restrict__ xf_mean,
+                  const float *__restrict__ xf_invstd, bf16 *__restrict__ xf_out, int *__restrict__ err_word) {
+    // xf_gamma != nullptr (forward only): the source tensor is the raw output y of the previous convolution and this
+    // kernel applies that convolution's batch norm and ReLU on its own operand path: four transform warps per pipeline
+    // turn every TMA box, in place in shared memory, into a = relu(y * scale + shift) (scale = gamma * invstd, shift =
+    // beta - mean * scale; rows outside the image stay zero: they are the convolution's padding), store the tile's own
+    // rows of a to xf_out (the backward sweep reads them) and only then hand the stage to the MMA warp.
     // stat_part != nullptr: the epilogue also reduces, per channel over the pixels of this CTA's tiles, the two sums the
     // batch norm that follows needs, from the values as stored (rounded to bf16), writes them to
     // stat_part[blockIdx.x][2C], and the CTA that finishes last adds the partials in a fixed order:
@@ -183,18 +190,21 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     const ConvSmem plan = conv_smem_plan<C>(n_stages, stage_bytes);
     const uint32_t w_base = base + plan.w_off, a_base = base + plan.a_off;
     uint8_t *tail = smem + plan.tail_off;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[4], tempty[4], wbar
-    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (2 * kMaxStages + 9) * 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (2 * kMaxStages + 9) * 8 + 8);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);  // full[16], empty[16], tfull[4], tempty[4], wbar, raw[16]
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tail + (3 * kMaxStages + 9) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tail + (3 * kMaxStages + 9) * 8 + 8);
     const Waiter wt{abort_flag, err_word, kSpinLimit};
     float (*sm_run)[4][32] = reinterpret_cast<float (*)[4][32]>(tail + 512);  // [epilogue warp][channel chunk][lane]
     float *sm_stat = reinterpret_cast<float *>(tail + 512 + 8192);            // mean[C], invstd[C]
+    float *sm_xf = reinterpret_cast<float *>(tail + 512 + 8192 + 512);        // scale[C], shift[C] of the input transform
+    const bool xform = xf_gamma != nullptr;
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + a); };
     auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 4 + a); };
     const uint32_t w_bar = bar0 + 8u * (2 * kMaxStages + 8);
+    auto raw_bar = [&](int s) { return bar0 + 8u * (2 * kMaxStages + 9 + s); };  // box landed, not yet transformed
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -202,7 +212,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
         for (int i = threadIdx.x; i < 16 * 4 * 32; i += blockDim.x) (&sm_run[0][0][0])[i] = 0.f;
     if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");  // the first TMA would otherwise wait for its descriptor
-        for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        // with the input transform a stage is full once each of the four transform warps has arrived
+        for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), xform ? 4 : 1); mbar_init(empty_bar(s), 1); mbar_init(raw_bar(s), 1); }
         for (int a = 0; a < 4; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4 * plan_e.split); }
         mbar_init(w_bar, 1);
         *abort_flag = 0;
@@ -220,6 +231,11 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     pdl_wait();
     if (bn_x != nullptr && threadIdx.x < 2 * C)
         sm_stat[threadIdx.x] = threadIdx.x < C ? bn_mean[threadIdx.x] : bn_invstd[threadIdx.x - C];
+    if (xform && threadIdx.x < C) {  // the same two constants, computed the same way, as the element-wise batch-norm pass
+        const float sc = to_f(xf_gamma[threadIdx.x]) * xf_invstd[threadIdx.x];
+        sm_xf[threadIdx.x] = sc;
+        sm_xf[C + threadIdx.x] = to_f(xf_beta[threadIdx.x]) - xf_mean[threadIdx.x] * sc;
+    }
     if (w_packed == nullptr) {
         // filter in canonical order: stage it here as 9 K-major [C rows = output channel of this pass][C] tiles
         for (int i = threadIdx.x; i < 9 * C * C; i += blockDim.x) {
@@ -240,6 +256,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
     const int n_pipes = plan_e.n_pipes;
     const int ring = n_stages / n_pipes;
     const int tile_step = n_pipes * gridDim.x;
+    const int n_epi_groups_plan = n_pipes * plan_e.n_slots * plan_e.split;
+    const int n_epi_groups = n_epi_groups_plan < 2 ? 2 : n_epi_groups_plan;  // warps launched for the epilogue: 4 per group
     if (warp < n_pipes) {
         // ---------------- TMA producers ----------------
         const int g = warp;
@@ -259,8 +277,9 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                     const int s = g * ring + ls;
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, wt, 1);
                     if (!ok) break;
-                    mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
-                    tma_load_4d(a_base + s * stage_bytes, &tmap, full_bar(s), 0, 0, slab ? h0 - 1 : h0 + j - 1, n0);
+                    const uint32_t land = xform ? raw_bar(s) : full_bar(s);
+                    mbar_expect_tx(land, (uint32_t)stage_bytes);
+                    tma_load_4d(a_base + s * stage_bytes, &tmap, land, 0, 0, slab ? h0 - 1 : h0 + j - 1, n0);
                     if (++ls == ring) { ls = 0; ph ^= 1u; }
                 }
             }
@@ -306,7 +325,61 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                 if (ok) tc_commit(tfull_bar(a));
             }
         }
-    } else {
+    } else if (xform && warp >= 2 * n_pipes + 4 * n_epi_groups) {
+        // ---------------- input transform: raw box -> relu(batch norm) in place, the tile's own rows also to global ------
+        const int tw = warp - 2 * n_pipes - 4 * n_epi_groups;
+        const int g = tw >> 2, t128 = 32 * (tw & 3) + lane;  // pipeline, thread among its 128 transform threads
+        constexpr int kCg = C / 8;                            // 16-byte groups of channels per pixel
+        const int box_rows_img = slab ? rows_per_tile + 2 : rows_per_tile;  // image rows of a box, per image
+        const int n_vec = box_rows_img * imgs_per_tile * W * kCg;
+        int ls = 0;
+        uint32_t ph = 0;
+        bool ok = g < n_pipes;
+        for (int tile = blockIdx.x + g * gridDim.x; tile < n_tiles && ok; tile += tile_step) {
+            int n0, h0;
+            if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }
+            else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
+            for (int j = 0; j < loads_per_tile && ok; ++j) {
+                const int s = g * ring + ls;
+                ok = mbar_wait(raw_bar(s), ph, wt, 6);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                uint8_t *stage = smem + plan.a_off + (size_t)s * stage_bytes;
+                const int row_first = slab ? h0 - 1 : j - 1;   // image row of the box's first row
+                const bool owns = slab || j == 1;              // the unshifted box holds the tile's own pixels
+                for (int v = t128; v < n_vec; v += 128) {
+                    const int cg = v % kCg, p = v / kCg;       // p: pixel of the box, (image, row, column) order
+                    const int col = p % W, r = (p / W) % box_rows_img, img = p / (W * box_rows_img);
+                    const int h = row_first + r;
+                    uint4 *cell = reinterpret_cast<uint4 *>(stage + swz_off<C>(p, 8 * cg));
+                    if (h < 0 || h >= H) continue;             // padding: the zero fill stays
+                    const uint4 q = *cell;
+                    const uint32_t wq[4] = {q.x, q.y, q.z, q.w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int c0 = 8 * cg + 2 * k;
+                        float a = fmaf(__uint_as_float(wq[k] << 16), sm_xf[c0], sm_xf[C + c0]);
+                        float b = fmaf(__uint_as_float(wq[k] & 0xffff0000u), sm_xf[c0 + 1], sm_xf[C + c0 + 1]);
+                        a = a > 0.f ? a : 0.f;
+                        b = b > 0.f ? b : 0.f;
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
+                        o[k] = *reinterpret_cast<const uint32_t *>(&h2);
+                    }
+                    const uint4 res = make_uint4(o[0], o[1], o[2], o[3]);
+                    *cell = res;
+                    if (owns && (!slab || (r >= 1 && r <= rows_per_tile))) {
+                        const size_t pix = ((size_t)(n0 + img) * H + h) * W + col;
+                        *reinterpret_cast<uint4 *>(xf_out + pix * C + 8 * cg) = res;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_bar(s));
+                if (++ls == ring) { ls = 0; ph ^= 1u; }
+            }
+        }
+    } else if (warp < 2 * n_pipes + 4 * n_epi_groups) {
         // ---------------- epilogue: TMEM -> registers -> bf16 -> global ----------------
         const int q = warp & 3;  // a warp may only touch TMEM lanes [32*(warp%4), +32)
         const int ew = warp - 2 * n_pipes;  // index among the epilogue warps
@@ -1137,25 +1210,19 @@ int *err_word_of(const Launch &L) { return L.err ? L.err : g_tc_error_addr; }
 constexpr int kSmemBudget = 80 * 1024;
 constexpr int kSmemMax = 227 * 1024;
 
-template <int C>
-int launch_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W,
-              Shortcut sc, BnFuse bf, Launch s) {
-    int rows, imgs;
-    tile_geometry(H, W, &rows, &imgs);
-    const int slab = (imgs == 1) ? 1 : 0;
-    const int box_rows = slab ? rows + 2 : rows;
-    CUtensorMap map;
-    if (32 % W != 0 || !get_map(src, B, H, W, C, box_rows, imgs, &map)) return -1;
-    const int stage_bytes = box_rows * imgs * W * C * 2;
-    const int n_tiles = (int)((long)B * H * W / kTileM);
+// Launch plan of the forward / input-gradient kernel for n_tiles tiles: pipelines per CTA, epilogue groups, grid.
+//   C = 16 (one 16-channel chunk per tile): two pipelines where an SM has at least four tiles, four where it has at
+//   least sixteen (large batches); below that one pipeline whose two epilogue groups take alternate tiles.
+//   C >= 32: one pipeline whose two groups halve every tile where an SM has a single tile (shorter epilogue); for
+//   C = 32 two pipelines with one group each where it has two (both tiles side by side; C = 64 would need all 512
+//   TMEM columns for that); two pipelines with two groups each where it has three or more.
+// A pipeline with a single tile uses one accumulator: fewer TMEM columns, so that CTAs of other streams fit beside it.
+// Several module streams (shared): as few CTAs as give every pipeline the same number of tiles as a full grid would give
+// the busiest one; the kernel's critical path is as long, and the SMs left over are free for the other streams (K = 4
+// step -2 %).  A kernel that has the GPU to itself takes every SM (a few pipelines then finish early).
+struct TcPlan { EpiPlan ep; int grid, threads; };
+TcPlan tc_plan(int C, int n_tiles, int slab, bool shared, bool xform) {
     const int sms = g_num_sms;
-    // Pipelines per CTA and epilogue plan.
-    //   C = 16 (one 16-channel chunk per tile): two pipelines where an SM has at least four tiles, four where it has at
-    //   least sixteen (large batches); below that one pipeline whose two epilogue groups take alternate tiles.
-    //   C >= 32: one pipeline whose two groups halve every tile where an SM has a single tile (shorter epilogue); for
-    //   C = 32 two pipelines with one group each where it has two (both tiles side by side; C = 64 would need all 512
-    //   TMEM columns for that); two pipelines with two groups each where it has three or more.
-    // A pipeline with a single tile uses one accumulator: fewer TMEM columns, so that CTAs of other streams fit beside it.
     EpiPlan ep;
     if (C == 16) {
         const int P = !slab ? 1 : (n_tiles >= 16 * sms ? 4 : (n_tiles >= 4 * sms ? 2 : 1));
@@ -1168,15 +1235,35 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     } else {
         ep = EpiPlan{1, n_tiles <= sms ? 1 : 2, 1, 2};
     }
-    // Several module streams: as few CTAs as give every pipeline the same number of tiles as a full grid would give the
-    // busiest one; the kernel's critical path is as long, and the SMs left over are free for the other streams (K = 4
-    // step -2 %).  A kernel that has the GPU to itself takes every SM (a few pipelines then finish early).
+    TcPlan p;
+    p.ep = ep;
     const int per_pipe = (n_tiles + sms * ep.n_pipes - 1) / (sms * ep.n_pipes);
     const int balanced = (n_tiles + per_pipe * ep.n_pipes - 1) / (per_pipe * ep.n_pipes);
     const int full = (n_tiles + ep.n_pipes - 1) / ep.n_pipes < sms ? (n_tiles + ep.n_pipes - 1) / ep.n_pipes : sms;
-    const int grid = s.shared ? balanced : full;
+    p.grid = shared ? balanced : full;
     const int groups = ep.n_pipes * ep.n_slots * ep.split;
-    const int threads = 32 * (2 * ep.n_pipes + 4 * (groups < 2 ? 2 : groups));
+    // issuing warps, four warps per epilogue group, and with the input transform four more warps per pipeline
+    p.threads = 32 * (2 * ep.n_pipes + 4 * (groups < 2 ? 2 : groups) + (xform ? 4 * ep.n_pipes : 0));
+    return p;
+}
+
+template <int C>
+int launch_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W,
+              Shortcut sc, BnFuse bf, InXform xf, Launch s) {
+    int rows, imgs;
+    tile_geometry(H, W, &rows, &imgs);
+    const int slab = (imgs == 1) ? 1 : 0;
+    const int box_rows = slab ? rows + 2 : rows;
+    CUtensorMap map;
+    if (32 % W != 0 || !get_map(src, B, H, W, C, box_rows, imgs, &map)) return -1;
+    const int stage_bytes = box_rows * imgs * W * C * 2;
+    const int n_tiles = (int)((long)B * H * W / kTileM);
+    const bool xform = xf.gamma != nullptr;
+    if (xform && dir != 0) return -1;
+    const TcPlan pl = tc_plan(C, n_tiles, slab, s.shared, xform);
+    const EpiPlan ep = pl.ep;
+    const int grid = pl.grid, threads = pl.threads;
+    if (threads > 768) return -1;  // the kernel's launch bound
     // CTAs with many tiles take the whole SM's shared memory for the stage ring; the others about half of it
     const int budget = n_tiles >= 8 * grid ? kSmemMax - 1024 - kTailBytes : kSmemBudget;
     int n_stages = (budget - (int)conv_smem_plan<C>(0, 0).a_off) / stage_bytes;
@@ -1190,7 +1277,8 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     if (tmem_cols > 512 || conv_smem_bytes<C>(n_stages, stage_bytes) > (size_t)kSmemMax) return -1;
     launch_kp(true, conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
         stage_bytes, tmem_cols, ep, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
-        bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd, err_word_of(s));
+        bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd, (const bf16 *)xf.gamma,
+        (const bf16 *)xf.beta, xf.mean, xf.invstd, (bf16 *)xf.a_out, err_word_of(s));
     return 1;
 }
 
@@ -1330,13 +1418,20 @@ bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
 size_t tc_packed_bytes(int C) { return 2 * (size_t)9 * C * C * 2; }
 
 int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
-                   Shortcut sc, Launch s, BnFuse bf) {
+                   Shortcut sc, Launch s, BnFuse bf, InXform xf) {
     switch (C) {
-    case 16: return launch_tc<16>(dir, src, w, w_packed, dst, B, H, W, sc, bf, s);
-    case 32: return launch_tc<32>(dir, src, w, w_packed, dst, B, H, W, sc, bf, s);
-    case 64: return launch_tc<64>(dir, src, w, w_packed, dst, B, H, W, sc, bf, s);
+    case 16: return launch_tc<16>(dir, src, w, w_packed, dst, B, H, W, sc, bf, xf, s);
+    case 32: return launch_tc<32>(dir, src, w, w_packed, dst, B, H, W, sc, bf, xf, s);
+    case 64: return launch_tc<64>(dir, src, w, w_packed, dst, B, H, W, sc, bf, xf, s);
     }
     return -1;
+}
+
+bool conv_tc_xform_supported(int B, int H, int W, int C, bool shared) {
+    if (!conv_tc_supported(B, H, W, C, C, 1)) return false;
+    int rows, imgs;
+    tile_geometry(H, W, &rows, &imgs);
+    return tc_plan(C, (int)((long)B * H * W / kTileM), imgs == 1 ? 1 : 0, shared, true).threads <= 768;
 }
 
 int conv_tc_grid(int B, int H, int W) {

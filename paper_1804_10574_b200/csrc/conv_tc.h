@@ -28,8 +28,20 @@ struct BnFuse {
     const void *mask = nullptr, *x = nullptr;
     const float *mean = nullptr, *invstd = nullptr;
 };
+// Input transform on the operand path of the forward convolution (gamma != nullptr): src holds the raw output y of the
+// previous convolution and the kernel applies that convolution's batch norm and ReLU itself, a = relu(y * scale + shift)
+// with scale = gamma * invstd and shift = beta - mean * scale, in shared memory between the TMA box and the MMAs (rows
+// outside the image stay zero: they are this convolution's padding), and stores a to a_out (same shape as src) for the
+// backward sweep.  The arithmetic is that of the element-wise batch-norm pass, value for value.  Available where
+// conv_tc_xform_supported says so (the plan's thread count, with four transform warps per pipeline, fits the kernel).
+struct InXform {
+    const void *gamma = nullptr, *beta = nullptr;
+    const float *mean = nullptr, *invstd = nullptr;
+    void *a_out = nullptr;
+};
+bool conv_tc_xform_supported(int B, int H, int W, int C, bool shared);
 int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
-                   Shortcut sc, Launch s, BnFuse bf = BnFuse());
+                   Shortcut sc, Launch s, BnFuse bf = BnFuse(), InXform xf = InXform());
 int conv_tc_grid(int B, int H, int W);
 size_t tc_packed_bytes(int C);
 // One launch that re-arranges the filters of many convolutions of one weight version.

@@ -150,9 +150,13 @@ size_t layer_params(const ddg_layer &s) {
     case DDG_CONV3X3: return (size_t)s.c_in * s.c_out * 9;
     case DDG_BN: return 2 * (size_t)s.c_in;
     case DDG_BASIC_BLOCK: return (size_t)s.c_in * s.c_out * 9 + (size_t)s.c_out * s.c_out * 9 + 4 * (size_t)s.c_out;
+    case DDG_BASIC_BLOCK_PROJ:
+        return (size_t)s.c_in * s.c_out * 9 + (size_t)s.c_out * s.c_out * 9 + 4 * (size_t)s.c_out + (size_t)s.c_in * s.c_out;
     default: return 0;
     }
 }
+
+bool is_block(int kind) { return kind == DDG_BASIC_BLOCK || kind == DDG_BASIC_BLOCK_PROJ; }
 
 int gcd_i(int a, int b) { return b ? gcd_i(b, a % b) : a; }
 
@@ -250,32 +254,48 @@ Count forward_module(ddg_ctx *c, int k, long t) {
         case DDG_GLOBAL_AVGPOOL:
             n += launch_avgpool_fwd(c->prec, in, out, B, L.Hin * L.Win, L.Cin, s);
             break;
-        case DDG_BASIC_BLOCK: {
+        case DDG_BASIC_BLOCK:
+        case DDG_BASIC_BLOCK_PROJ: {
             const int Ci = L.Cin, Co = L.Cout, st = L.spec.stride;
             const char *w1 = w, *g1 = w1 + (size_t)Co * Ci * 9 * es, *b1 = g1 + (size_t)Co * es;
             const char *w2 = b1 + (size_t)Co * es, *g2 = w2 + (size_t)Co * Co * 9 * es, *b2 = g2 + (size_t)Co * es;
+            const char *ws = b2 + (size_t)Co * es;  // projection filter, DDG_BASIC_BLOCK_PROJ only
             char *y1 = slot_ptr(c, L.y1, t), *a1 = slot_ptr(c, L.a1, t), *y2 = slot_ptr(c, L.y2, t);
             float *stt = (float *)slot_ptr(c, L.stats, t);
             const long npix = (long)B * L.Hout * L.Wout;
             // convolution followed by its batch norm; the statistics come from the convolution's epilogue where the
             // tensor-core kernel runs, from a reduction kernel otherwise
-            auto conv_bn = [&](const void *xin, const void *wc, const void *wp, void *yc, int H, int W, int Cic, int strd,
-                               const char *gm, const char *bt, float *mean, float *invstd, Shortcut scb, void *dstb) {
+            // a convolution and the statistics of the batch norm that follows it; xf: an input transform for it to carry
+            auto conv_stats = [&](const void *xin, const void *wc, const void *wp, void *yc, int H, int W, int Cic, int strd,
+                                  float *mean, float *invstd, InXform xf) {
                 if (fuse_bn && c->prec == P_BF16 && conv_tc_supported(B, H, W, Cic, Co, strd)) {
                     BnFuse bf;
                     bf.part = m.bn_scratch + 32; bf.counter = (unsigned *)m.bn_scratch; bf.o0 = mean; bf.o1 = invstd;
-                    n += launch_conv_tc(0, xin, wc, wp, yc, B, H, W, Cic, Shortcut{}, s, bf);
+                    n += launch_conv_tc(0, xin, wc, wp, yc, B, H, W, Cic, Shortcut{}, s, bf, xf);
                 } else {
                     n += conv_fwd(c, xin, wc, wp, yc, H, W, Cic, Co, strd, 0, s);
                     n += launch_bn_stats(c->prec, yc, mean, invstd, m.bn_scratch, npix, Co, s);
                 }
-                n += launch_bn_apply(c->prec, yc, gm, bt, mean, invstd, scb, dstb, B, L.Hout, L.Wout, Co, 1, s);
             };
-            conv_bn(in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, g1, b1, stt, stt + Co, Shortcut{}, a1);
+            // bn1's normalise + ReLU pass rides on conv2's operand path where the tensor-core kernel can take it: conv2
+            // then reads the raw y1, computes a1 in shared memory and stores it for the backward sweep
+            const bool ride = !c->cfg.separate_bn_apply && fuse_bn && c->prec == P_BF16 &&
+                              conv_tc_xform_supported(B, L.Hout, L.Wout, Co, s.shared);
+            conv_stats(in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, stt, stt + Co, InXform{});
+            if (!ride) n += launch_bn_apply(c->prec, y1, g1, b1, stt, stt + Co, Shortcut{}, a1, B, L.Hout, L.Wout, Co, 1, s);
             Shortcut sc{};
             sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
             sc.a = in; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win;
-            conv_bn(a1, w2, pkp(L.pk2), y2, L.Hout, L.Wout, Co, 1, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out);
+            if (L.spec.kind == DDG_BASIC_BLOCK_PROJ) {
+                // projected shortcut W_s x into a temporary of the module (only this forward sweep reads it), then added
+                // like an identity shortcut
+                n += launch_conv1x1_fwd(c->prec, in, ws, m.tmp[0], B, L.Hin, L.Win, Ci, Co, st, s);
+                sc.mode = 1; sc.a = m.tmp[0];
+            }
+            InXform xf;
+            if (ride) { xf.gamma = g1; xf.beta = b1; xf.mean = stt; xf.invstd = stt + Co; xf.a_out = a1; }
+            conv_stats(ride ? y1 : a1, w2, pkp(L.pk2), y2, L.Hout, L.Wout, Co, 1, stt + 2 * Co, stt + 3 * Co, xf);
+            n += launch_bn_apply(c->prec, y2, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out, B, L.Hout, L.Wout, Co, 1, s);
             break;
         }
         }
@@ -394,11 +414,15 @@ Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
         case DDG_GLOBAL_AVGPOOL:
             if (need_dx) n += launch_avgpool_bwd(c->prec, cur, dst, B, L.Hin * L.Win, L.Cin, s);
             break;
-        case DDG_BASIC_BLOCK: {
+        case DDG_BASIC_BLOCK:
+        case DDG_BASIC_BLOCK_PROJ: {
             const int Ci = L.Cin, Co = L.Cout, st = L.spec.stride;
+            const bool proj = L.spec.kind == DDG_BASIC_BLOCK_PROJ;
             const size_t nw1 = (size_t)Co * Ci * 9, nw2 = (size_t)Co * Co * 9;
             const char *w1 = w, *g1 = w1 + nw1 * es, *w2 = g1 + 2 * (size_t)Co * es, *g2 = w2 + nw2 * es;
+            const char *ws = g2 + 2 * (size_t)Co * es;
             float *gw1 = gw, *gg1 = gw1 + nw1, *gb1 = gg1 + Co, *gw2 = gb1 + Co, *gg2 = gw2 + nw2, *gb2 = gg2 + Co;
+            float *gws = gb2 + Co;
             const char *y1 = slot_ptr(c, L.y1, sidx), *a1 = slot_ptr(c, L.a1, sidx), *y2 = slot_ptr(c, L.y2, sidx);
             const float *stt = (const float *)slot_ptr(c, L.stats, sidx);
             const long npix = (long)B * L.Hout * L.Wout;
@@ -426,13 +450,32 @@ Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
             }
             n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
             side_wgrad(j1, in, dy1, gw1, L.Hin, L.Win, Ci, Co, st);
-            if (need_dx) {
+            if (proj) {
+                // weight gradient of the projection, on the chain's own stream (it reads the incoming gradient in place
+                // and shares the weight-gradient scratch with the side stream: wait for what runs there first)
+                side_join();
+                n += launch_conv1x1_wgrad(c->prec, in, cur, out, gws, m.wg_scratch, B, L.Hin, L.Win, Ci, Co, st, s);
+            }
+            if (need_dx && proj) {
+                char *dx = mod_first ? dst : da1;
+                if (c->prec == P_BF16) {
+                    // tensor-core input gradient of conv1, then the projection's share added in place
+                    n += conv_dgrad(c, dy1, w1, pkp(L.pk1), dx, L.Hin, L.Win, Ci, Co, st, Shortcut{}, s);
+                    n += launch_conv1x1_dgrad_add(c->prec, cur, out, ws, dx, B, L.Hin, L.Win, Ci, Co, st, s);
+                } else {
+                    // one kernel, one rounding: the CUDA-core input gradient adds W_s^T dz before it stores
+                    Shortcut sc{};
+                    sc.mode = 3; sc.a = cur; sc.b = out; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win; sc.w = ws;
+                    n += launch_conv_dgrad_direct(c->prec, dy1, w1, dx, B, L.Hin, L.Win, Ci, Co, st, sc, s);
+                }
+                if (!mod_first) { dst = dx; dst_tmp = tB; }
+            } else if (need_dx) {
                 Shortcut sc{};
                 sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
                 sc.a = cur; sc.b = out; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win;
                 char *dx = mod_first ? dst : da1;  // da1 is dead once bn1's backward has run
                 const LayerPlan *Pv = mod_first ? nullptr : &c->layers[l - 1];
-                if (fuse && Pv && Pv->spec.kind == DDG_BASIC_BLOCK && sc.mode == 1 &&
+                if (fuse && Pv && is_block(Pv->spec.kind) && sc.mode == 1 &&
                     conv_tc_supported(B, L.Hin, L.Win, Ci, Co, st)) {
                     // dx is the incoming gradient of the block below, whose second batch norm reduces it first: take
                     // those sums here (its output is this block's input, its bn2 input and statistics are in its slots)
@@ -637,8 +680,12 @@ ddg_status init_weights(ddg_ctx *ctx) {
             launch_fill_const(w, L.Cin, 1.f, s);
             launch_fill_const(w + L.Cin, L.Cin, 0.f, s);
             break;
-        case DDG_BASIC_BLOCK: {
+        case DDG_BASIC_BLOCK:
+        case DDG_BASIC_BLOCK_PROJ: {
             const size_t nw1 = (size_t)L.Cout * L.Cin * 9, nw2 = (size_t)L.Cout * L.Cout * 9;
+            if (L.spec.kind == DDG_BASIC_BLOCK_PROJ)
+                launch_fill_normal(w + nw1 + 4 * L.Cout + nw2, (size_t)L.Cout * L.Cin, sqrtf(2.f / L.Cin), seed,
+                                   2 * l + 1000003, s);
             launch_fill_normal(w, nw1, sqrtf(2.f / (9 * L.Cin)), seed, 2 * l, s);
             launch_fill_const(w + nw1, L.Cout, 1.f, s);
             launch_fill_const(w + nw1 + L.Cout, L.Cout, 0.f, s);
@@ -793,13 +840,16 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
             ok = (s.c_in == C && s.c_out >= s.c_in && (s.stride == 1 || s.stride == 2) &&
                   (s.stride == 2 || s.c_out == s.c_in));
             C = s.c_out; H = (H - 1) / s.stride + 1; W = (W - 1) / s.stride + 1; break;
+        case DDG_BASIC_BLOCK_PROJ:
+            ok = (s.c_in == C && s.c_out >= 1 && (s.stride == 1 || s.stride == 2));
+            C = s.c_out; H = (H - 1) / s.stride + 1; W = (W - 1) / s.stride + 1; break;
         case DDG_BN: ok = (s.c_in == C); break;
         case DDG_RELU: break;
         case DDG_GLOBAL_AVGPOOL: H = 1; W = 1; break;
         default: ok = false;
         }
         if (!ok) { set_err(nullptr, "layer %d: specification does not fit its input [%d,%d,%d]", l, L.Cin, L.Hin, L.Win); return DDG_ERR_BAD_SPEC; }
-        if ((s.kind == DDG_CONV3X3 || s.kind == DDG_BASIC_BLOCK || s.kind == DDG_BN || s.kind == DDG_GLOBAL_AVGPOOL) &&
+        if ((s.kind == DDG_CONV3X3 || is_block(s.kind) || s.kind == DDG_BN || s.kind == DDG_GLOBAL_AVGPOOL) &&
             (C > 128 || L.Cin > 128 || (size_t)L.Cin * C > 4096)) {
             set_err(nullptr, "layer %d: channel counts above 64x64 (or 128 for BN / pooling) are not supported", l);
             return DDG_ERR_UNSUPPORTED;
@@ -840,7 +890,7 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
             if (l == 0) L.in = {0, take(n_in * es)};                      // the shimmed input lives in module 1's arena
             else L.in = c->layers[l - 1].out;                             // may point into the previous module's arena
             L.out = {k, take(L.is_last ? n_out * sizeof(float) : n_out * es)};
-            if (L.spec.kind == DDG_BASIC_BLOCK) {
+            if (is_block(L.spec.kind)) {
                 L.y1 = {k, take(n_out * es)}; L.a1 = {k, take(n_out * es)}; L.y2 = {k, take(n_out * es)};
                 L.stats = {k, take(4 * (size_t)L.Cout * sizeof(float))};
             } else if (L.spec.kind == DDG_BN) {
@@ -892,10 +942,11 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
         size_t bn_max = 0, wg_max = 0;
         for (int l = m.first; l <= m.last; ++l) {
             LayerPlan &L = c->layers[l];
-            if (L.spec.kind == DDG_BN || L.spec.kind == DDG_BASIC_BLOCK) bn_max = std::max(bn_max, bn_scratch_elems(L.Cout));
+            if (L.spec.kind == DDG_BN || is_block(L.spec.kind)) bn_max = std::max(bn_max, bn_scratch_elems(L.Cout));
+            if (L.spec.kind == DDG_BASIC_BLOCK_PROJ) wg_max = std::max(wg_max, conv1x1_wgrad_scratch_elems(L.Cin, L.Cout));
             if (L.spec.kind == DDG_CONV3X3)
                 wg_max = std::max(wg_max, conv_wgrad_scratch_elems(c->B, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride));
-            if (L.spec.kind == DDG_BASIC_BLOCK) {
+            if (is_block(L.spec.kind)) {
                 wg_max = std::max(wg_max, conv_wgrad_scratch_elems(c->B, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride));
                 wg_max = std::max(wg_max, conv_wgrad_scratch_elems(c->B, L.Hout, L.Wout, L.Cout, L.Cout, 1));
             }
@@ -925,7 +976,7 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
                     plan(&L.pk1, L.p_off, L.Hin, L.Win, L.pad_c, L.Cout, 1, L.Cin);
                 else if (L.spec.kind == DDG_CONV3X3 && !L.spec.relu_after)
                     plan(&L.pk1, L.p_off, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride);
-                if (L.spec.kind == DDG_BASIC_BLOCK) {
+                if (is_block(L.spec.kind)) {
                     plan(&L.pk1, L.p_off, L.Hin, L.Win, L.Cin, L.Cout, L.spec.stride);
                     plan(&L.pk2, L.p_off + (size_t)L.Cout * L.Cin * 9 + 2 * (size_t)L.Cout, L.Hout, L.Wout, L.Cout, L.Cout, 1);
                 }

@@ -32,12 +32,15 @@ struct Launch {
 // Shortcut input of a residual add (forward) or its gradient (backward).
 //   mode 0: none.  mode 1: identity (same shape as the tensor it is added to).
 //   mode 2: parameter-free down-sampling shortcut: spatial stride 2, channels >= c_small are zero.
+//   mode 3 (backward, CUDA-core input gradient only): 1x1-projection shortcut W_s [Cout][c_small] with the convolution's
+//           stride: dx[n][s*h][s*w][ci] += sum_co a[n][h][w][co] * [b > 0] * w[co][ci].
 struct Shortcut {
     int mode;
     const void *a;   // forward: block input x.          backward: error gradient of the block output
     const void *b;   // forward: unused.                 backward: block output (for the ReLU mask)
     int c_small;     // channels of the narrower tensor (block input)
     int h_big, w_big;  // spatial size of the block input (the larger map)
+    const void *w;   // mode 3: the projection filter
 };
 
 // ---- layout / small layers --------------------------------------------------------------------------
@@ -82,6 +85,19 @@ int launch_conv_dgrad_direct(int prec, const void *dy, const void *w, void *dx, 
 size_t conv_wgrad_scratch_elems(int B, int H, int W, int Cin, int Cout, int stride);
 int launch_conv_wgrad_direct(int prec, const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W,
                              int Cin, int Cout, int stride, Launch s);
+
+// ---- 1x1 convolution with a spatial stride, no bias (projection shortcut of a shape-changing block), CUDA cores ----
+// x [B][H][W][Cin], w [Cout][Cin], y [B][Ho][Wo][Cout], Ho = (H-1)/stride+1.
+int launch_conv1x1_fwd(int prec, const void *x, const void *w, void *y, int B, int H, int W, int Cin, int Cout, int stride,
+                       Launch s);
+// dx[n][s*h][s*w][ci] += sum_co dz[n][h][w][co] * w[co][ci], dz = dout * [out > 0] (out nullable: no mask); dx is read,
+// added to and stored in its element type.
+int launch_conv1x1_dgrad_add(int prec, const void *dout, const void *out, const void *w, void *dx, int B, int H, int W,
+                             int Cin, int Cout, int stride, Launch s);
+// dw[co][ci] = sum over output pixels of dz[p][co] * x[s*p][ci]; per-chunk partials in scratch, folded in a fixed order.
+size_t conv1x1_wgrad_scratch_elems(int Cin, int Cout);
+int launch_conv1x1_wgrad(int prec, const void *x, const void *dout, const void *out, float *dw, float *scratch, int B,
+                         int H, int W, int Cin, int Cout, int stride, Launch s);
 
 // ---- optimiser --------------------------------------------------------------------------------------
 // mode 0: SGD momentum/decay step.  mode 1: Adam step (c1, c2 = bias corrections).  mode 2: no step, only

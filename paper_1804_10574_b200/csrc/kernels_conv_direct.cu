@@ -104,6 +104,19 @@ conv3x3_direct_kernel(const T *__restrict__ src, const T *__restrict__ w, T *__r
                     const size_t q = (size_t)p * Cd + cd0 + j;
                     if (to_f(out[q]) > 0.f) acc[j] += (A)to_f(dout[q]);
                 }
+        } else if (sc.mode == 3) {
+            // 1x1-projection shortcut with this convolution's stride: input pixel (s*h, s*w) fed output pixel (h, w)
+            if ((hd % stride) == 0 && (wd % stride) == 0) {
+                const T *ws = (const T *)sc.w;  // [Cout][Cin]
+                const size_t q0 = ((n * Hs + hd / stride) * Ws + wd / stride) * (size_t)Cout;
+                for (int co = 0; co < Cout; ++co) {
+                    if (!(to_f(out[q0 + co]) > 0.f)) continue;
+                    const A d = (A)to_f(dout[q0 + co]);
+#pragma unroll
+                    for (int j = 0; j < kCdt; ++j)
+                        if (cd0 + j < Cd) acc[j] += d * (A)to_f(ws[(size_t)co * Cin + cd0 + j]);
+                }
+            }
         } else if ((hd % 2) == 0 && (wd % 2) == 0) {
             // block output is [B][Hs][Ws][Cout]; channel c < Cin of the input maps to the same channel
             const size_t q0 = ((n * Hs + hd / 2) * Ws + wd / 2) * (size_t)Cout;
@@ -267,6 +280,135 @@ int launch_conv_wgrad_direct(int prec, const void *x, const void *dy, float *dw,
                                                                      Cin, Ho, Wo, Cout, stride, ci_per);
         launch_k(conv3x3_wgrad_fold_kernel<A>, ceil_div(9 * Cin * Cout, 256), 256, 0, s, (const A *)scratch, dw, chunks, Cin,
                                                                                   Cout);
+    });
+    return 2;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// 1x1 convolution with a spatial stride (projection shortcut).  A few MFLOP per call: plain CUDA-core kernels.
+// ------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+conv1x1_fwd_kernel(const T *__restrict__ x, const T *__restrict__ w, T *__restrict__ y, long npix, int H, int W, int Cin,
+                   int Ho, int Wo, int Cout, int stride) {
+    pdl_launch();
+    pdl_wait();
+    const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;  // (output pixel, co)
+    if (i >= npix * Cout) return;
+    typedef typename AccOf<T>::type A;
+    const int co = (int)(i % Cout);
+    const long p = i / Cout;
+    const int wo = (int)(p % Wo), ho = (int)((p / Wo) % Ho);
+    const long n = p / ((long)Wo * Ho);
+    const T *xp = x + ((n * H + (long)stride * ho) * W + (long)stride * wo) * Cin;
+    const T *wp = w + (size_t)co * Cin;
+    A acc = 0;
+    for (int ci = 0; ci < Cin; ++ci) acc += (A)to_f(xp[ci]) * (A)to_f(wp[ci]);
+    y[i] = from_a<T>(acc);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+conv1x1_dgrad_add_kernel(const T *__restrict__ dout, const T *__restrict__ out, const T *__restrict__ w, T *__restrict__ dx,
+                         long npix, int H, int W, int Cin, int Ho, int Wo, int Cout, int stride) {
+    pdl_launch();
+    pdl_wait();
+    const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;  // (output pixel, ci)
+    if (i >= npix * Cin) return;
+    typedef typename AccOf<T>::type A;
+    const int ci = (int)(i % Cin);
+    const long p = i / Cin;
+    const int wo = (int)(p % Wo), ho = (int)((p / Wo) % Ho);
+    const long n = p / ((long)Wo * Ho);
+    T *dst = dx + ((n * H + (long)stride * ho) * W + (long)stride * wo) * Cin + ci;
+    A acc = (A)to_f(*dst);
+    for (int co = 0; co < Cout; ++co) {
+        if (out != nullptr && !(to_f(out[p * Cout + co]) > 0.f)) continue;
+        acc += (A)to_f(dout[p * Cout + co]) * (A)to_f(w[(size_t)co * Cin + ci]);
+    }
+    *dst = from_a<T>(acc);
+}
+
+static constexpr int k1x1Chunks = 64;
+size_t conv1x1_wgrad_scratch_elems(int Cin, int Cout) { return (size_t)k1x1Chunks * Cin * Cout * 2; }  // fp64 partials in fp32 mode
+
+// one CTA per chunk of output pixels; thread t owns the (co, ci) pairs t, t + 256, ...
+template <typename T>
+__global__ void __launch_bounds__(256)
+conv1x1_wgrad_partial_kernel(const T *__restrict__ x, const T *__restrict__ dout, const T *__restrict__ out,
+                             typename AccOf<T>::type *__restrict__ part, long npix, int H, int W, int Cin, int Ho, int Wo,
+                             int Cout, int stride) {
+    pdl_launch();
+    pdl_wait();
+    typedef typename AccOf<T>::type A;
+    constexpr int kMaxPairs = 16;  // Cin * Cout <= 4096
+    const int pairs = Cin * Cout;
+    A acc[kMaxPairs];
+#pragma unroll
+    for (int j = 0; j < kMaxPairs; ++j) acc[j] = 0;
+    const long p0 = npix * blockIdx.x / gridDim.x, p1 = npix * (blockIdx.x + 1) / gridDim.x;
+    for (long p = p0; p < p1; ++p) {
+        const int wo = (int)(p % Wo), ho = (int)((p / Wo) % Ho);
+        const long n = p / ((long)Wo * Ho);
+        const T *xp = x + ((n * H + (long)stride * ho) * W + (long)stride * wo) * Cin;
+#pragma unroll
+        for (int j = 0; j < kMaxPairs; ++j) {
+            const int q = threadIdx.x + j * 256;
+            if (q < pairs) {
+                const int co = q / Cin, ci = q % Cin;
+                float d = to_f(dout[p * Cout + co]);
+                if (out != nullptr && !(to_f(out[p * Cout + co]) > 0.f)) d = 0.f;
+                acc[j] += (A)d * (A)to_f(xp[ci]);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < kMaxPairs; ++j) {
+        const int q = threadIdx.x + j * 256;
+        if (q < pairs) part[(size_t)blockIdx.x * pairs + q] = acc[j];
+    }
+}
+
+template <typename A>
+__global__ void conv1x1_wgrad_fold_kernel(const A *__restrict__ part, float *__restrict__ dw, int chunks, int pairs) {
+    pdl_launch();
+    pdl_wait();
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= pairs) return;
+    A t = 0;
+    for (int c = 0; c < chunks; ++c) t += part[(size_t)c * pairs + q];
+    dw[q] = (float)t;
+}
+
+int launch_conv1x1_fwd(int prec, const void *x, const void *w, void *y, int B, int H, int W, int Cin, int Cout, int stride,
+                       Launch s) {
+    const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    const long npix = (long)B * Ho * Wo;
+    DISPATCH_PREC(prec, launch_k(conv1x1_fwd_kernel<T>, ceil_div(npix * Cout, 256), 256, 0, s, (const T *)x, (const T *)w, (T *)y,
+                                 npix, H, W, Cin, Ho, Wo, Cout, stride));
+    return 1;
+}
+
+int launch_conv1x1_dgrad_add(int prec, const void *dout, const void *out, const void *w, void *dx, int B, int H, int W,
+                             int Cin, int Cout, int stride, Launch s) {
+    const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    const long npix = (long)B * Ho * Wo;
+    DISPATCH_PREC(prec, launch_k(conv1x1_dgrad_add_kernel<T>, ceil_div(npix * Cin, 256), 256, 0, s, (const T *)dout,
+                                 (const T *)out, (const T *)w, (T *)dx, npix, H, W, Cin, Ho, Wo, Cout, stride));
+    return 1;
+}
+
+int launch_conv1x1_wgrad(int prec, const void *x, const void *dout, const void *out, float *dw, float *scratch, int B,
+                         int H, int W, int Cin, int Cout, int stride, Launch s) {
+    if ((long)Cin * Cout > 4096) return -1;
+    const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    const long npix = (long)B * Ho * Wo;
+    const int chunks = npix < k1x1Chunks ? (int)npix : k1x1Chunks;
+    DISPATCH_PREC(prec, {
+        typedef typename AccOf<T>::type A;
+        launch_k(conv1x1_wgrad_partial_kernel<T>, chunks, 256, 0, s, (const T *)x, (const T *)dout, (const T *)out, (A *)scratch,
+                 npix, H, W, Cin, Ho, Wo, Cout, stride);
+        launch_k(conv1x1_wgrad_fold_kernel<A>, ceil_div(Cin * Cout, 256), 256, 0, s, (const A *)scratch, dw, chunks, Cin * Cout);
     });
     return 2;
 }

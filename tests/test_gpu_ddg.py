@@ -116,6 +116,31 @@ def test_resnet8_split_positions_bf16(split):
     run_pair(cfg, 5, BF16_TOL, 5e-3, precision="bf16", split_after=split, noise_bar=True, ratio_band=RATIO_BAND)
 
 
+@pytest.mark.parametrize("splits", [[2], [2, 3]], ids=["K2", "K3"])
+def test_resnet8_projection_shortcuts_fp32(splits):
+    """Section 5.1's network with 1x1-projection shortcuts on the two shape-changing blocks (the second shortcut type),
+    fp32 mode: bit-level parity with the oracle over two ring periods, graph replay on."""
+    cfg = dict(nets.config("resnet8"), layers=nets.resnet(1, 10, projection=True), opt=dict(lr=0.05, momentum=0.9, weight_decay=5e-4))
+    w = run_pair(cfg, 14, FP32_TOL, LOSS_TOL, split_after=splits, batch=8, use_graph=True)
+    print("resnet8 projection fp32 worst", w)
+
+
+def test_resnet8_projection_shortcuts_bf16():
+    cfg = dict(nets.config("resnet8"), layers=nets.resnet(1, 10, projection=True), opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
+    w = run_pair(cfg, 6, BF16_TOL, 5e-3, precision="bf16", split_after=[2, 3], noise_bar=True, ratio_band=RATIO_BAND)
+    print("resnet8 projection bf16 worst", w)
+
+
+@pytest.mark.parametrize("c,h,stride", [(16, 32, 2), (32, 16, 2), (16, 16, 1)], ids=["c16_s2", "c32_s2", "c16_to_32_s1"])
+def test_one_projection_block_bf16(c, h, stride):
+    co = 2 * c
+    L = [(nets.BASIC_BLOCK_PROJ, c, co, stride, 0, 0), (nets.GLOBAL_AVGPOOL, co, co, 1, 0, 0), (nets.FC, co, 10, 1, 1, 0)]
+    cfg = dict(layers=L, split_after=[], batch=32, in_shape=(c, h, h), num_classes=10, precision="bf16",
+               opt=dict(lr=0.01, momentum=0.9, weight_decay=5e-4))
+    w = run_pair(cfg, 2, BF16_TOL, 5e-3)
+    print("one projection block c=%d stride=%d worst" % (c, stride), w)
+
+
 def test_resnet8_graph_replay_matches_fp32():
     run_pair(nets.config("resnet8"), 8, FP32_TOL, LOSS_TOL, batch=8, use_graph=True)
 
@@ -231,6 +256,16 @@ def test_epilogue_batch_norm_sums_match_separate_reductions():
                 for _, name, off, shape, _ in nets.param_segments(nets.resnet(3, 10)))
     print("epilogue vs separate sums: worst per-tensor weight difference", worst)
     assert worst < 5e-3
+
+
+def test_batch_norm_pass_on_the_operand_path_gives_the_same_bits():
+    """The first batch norm's normalise + ReLU pass inside the second convolution (shared memory, between TMA box and
+    MMA) and the separate element-wise kernel compute the same values: identical weights after six iterations, fewer
+    launches."""
+    wa, la, na = _resnet20_k3_bf16_run()
+    wb, lb, nb = _resnet20_k3_bf16_run(separate_bn_apply=True)
+    assert na < nb
+    assert la == lb and np.array_equal(wa, wb)
 
 
 def test_launch_overlap_settings_give_the_same_bits():

@@ -405,3 +405,79 @@ def test_fc_tensor_core_path_takes_the_paper_shapes():
     for B, i, o in [(128, 64, 100), (128, 64, 10), (16, 64, 128), (16, 128, 128), (16, 128, 10), (515, 256, 128)]:
         assert binding.fc_tensor_core_path(B, i, o) == 1, (B, i, o)
     assert binding.fc_tensor_core_path(5, 96, 12) == 0 and binding.fc_tensor_core_path(9, 64, 200) == 0
+
+
+@pytest.mark.parametrize("prec", [0, 1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("shape", [(128, 32, 32, 16, 32, 2), (33, 16, 16, 32, 64, 2), (3, 9, 7, 6, 10, 2), (5, 8, 8, 16, 24, 1)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_conv1x1_projection(shape, prec):
+    """The projection shortcut's 1x1 convolution (forward, input gradient added in place with the ReLU mask of the block
+    output, weight gradient) against the oracle's primitive."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, Ci, Co, st = shape
+    rng = np.random.default_rng(37)
+    Ho, Wo = (H - 1) // st + 1, (W - 1) // st + 1
+    x, xh = to_dev(rng.standard_normal((B, Ci, H, W)), prec)
+    w = torch.from_numpy(rng.standard_normal((Co, Ci)) * np.sqrt(2.0 / Ci)).to(tdtype(prec))
+    wh = w.to(torch.float64).numpy()
+    w = w.cuda()
+    dout, douth = to_dev(rng.standard_normal((B, Co, Ho, Wo)), prec)
+    out, outh = to_dev(np.maximum(rng.standard_normal((B, Co, Ho, Wo)), 0), prec)
+    base, baseh = to_dev(rng.standard_normal((B, Ci, H, W)), prec)      # what the 3x3 input gradient left in dx
+    y = torch.empty(B, Ho, Wo, Co, dtype=tdtype(prec), device="cuda")
+    dx = base.clone()
+    dw = torch.empty(Co, Ci, dtype=torch.float32, device="cuda")
+    scratch = torch.empty(binding.conv1x1_wgrad_scratch_elems(Ci, Co), dtype=torch.float32, device="cuda")
+    binding.conv1x1_fwd(prec, x, w, y, B, H, W, Ci, Co, st)
+    binding.conv1x1_dgrad_add(prec, dout, out, w, dx, B, H, W, Ci, Co, st)
+    binding.conv1x1_wgrad(prec, x, dout, out, dw, scratch, B, H, W, Ci, Co, st)
+    torch.cuda.synchronize()
+    check_map(from_dev(y), orc.conv1x1_forward(xh, wh, st), prec, "1x1 forward")
+    dz = douth * (outh > 0)
+    dx_ref, dw_ref = orc.conv1x1_backward(xh, wh, dz, st)
+    check_map(from_dev(dx), baseh + dx_ref, prec, "1x1 input gradient added in place")
+    assert rel(dw.cpu().numpy(), dw_ref) < 1e-5
+
+
+@pytest.mark.parametrize("shape", [(3, 32, 32, 16), (5, 16, 16, 32), (128, 8, 8, 64), (2, 8, 8, 16), (8, 8, 8, 32),
+                                   (128, 32, 32, 16), (128, 16, 16, 32), (301, 32, 32, 16), (231, 16, 16, 32), (902, 8, 8, 64)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_conv_forward_with_batch_norm_relu_on_its_operand_path(shape):
+    """Eq. 3 for batch norm -> ReLU -> convolution in one kernel: a = relu(bn(x)) computed in shared memory from the raw
+    x (stored to a_out), y = conv3x3(a) and the statistics of y.  a against the oracle's batch norm + ReLU (and bit for
+    bit against the element-wise kernel); y against the oracle's convolution of the a the GPU stored."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = shape
+    rng = np.random.default_rng(41)
+    x, xh = to_dev(rng.standard_normal((B, C, H, W)) * 1.3 + 0.2, 1)
+    w, wh = _filter(rng, C)
+    gamma = torch.from_numpy(1 + 0.2 * rng.standard_normal(C)).to(torch.bfloat16)
+    beta = torch.from_numpy(0.2 * rng.standard_normal(C)).to(torch.bfloat16)
+    gh, bh = gamma.to(torch.float64).numpy(), beta.to(torch.float64).numpy()
+    a_ref, m_ref, is_ref = orc.bn_forward(xh, gh, bh)
+    a_ref = np.maximum(a_ref, 0)
+    mean_in = torch.from_numpy(m_ref.astype(np.float32)).cuda()
+    invstd_in = torch.from_numpy(is_ref.astype(np.float32)).cuda()
+    a = torch.full_like(x, 7.0)
+    y = torch.empty_like(x)
+    mean, invstd = (torch.empty(C, dtype=torch.float32, device="cuda") for _ in range(2))
+    scratch = torch.zeros(binding.conv3x3_fused_scratch_elems(B, H, W, C), dtype=torch.float32, device="cuda")
+    binding.conv3x3_bnrelu_fwd_stats(x, gamma.cuda(), beta.cuda(), mean_in, invstd_in, a, w, None, y, mean, invstd, scratch,
+                                     B, H, W, C)
+    torch.cuda.synchronize()
+    arms = float(np.sqrt(np.mean(a_ref ** 2)))
+    assert rel(from_dev(a), a_ref) < TOL[1]
+    ok, idx, excess = elementwise_ok(from_dev(a), a_ref, RTOL[1], 2e-3 * arms)
+    assert ok, "transformed input: element %r off by %.3e" % (idx, excess)
+    # the same values as the element-wise batch-norm kernel gives, bit for bit
+    a2 = torch.empty_like(x)
+    m2, i2 = (torch.empty(C, dtype=torch.float32, device="cuda") for _ in range(2))
+    sc2 = torch.zeros(binding.bn_scratch_elems(C), dtype=torch.float32, device="cuda")
+    binding.bn_fwd(1, x, gamma.cuda(), beta.cuda(), None, a2, m2, i2, sc2, B, H * W, C, 1)
+    torch.cuda.synchronize()
+    if torch.equal(m2, mean_in) and torch.equal(i2, invstd_in):      # same statistics in, same bits out
+        assert torch.equal(a.view(B, H * W, C), a2.view(B, H * W, C))
+    y_ref = orc.conv3x3_forward(from_dev(a), wh, 1)
+    check_map(from_dev(y), y_ref, 1, "forward of the transformed input", max(1, 128 // W))
+    _, ms, iss = orc.bn_forward(from_dev(y), np.ones(C), np.zeros(C))
+    assert rel(mean.cpu().numpy(), ms) < 2e-5 and rel(invstd.cpu().numpy(), iss) < 2e-5
