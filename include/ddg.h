@@ -231,10 +231,12 @@ ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *pa
  * RAW output of the first convolution; the kernel applies that convolution's batch norm and ReLU on its own operand
  * path, a = relu(gamma * (x - mean_in) * invstd_in + beta) rounded to bf16 (gamma, beta bf16 [C]; mean_in, invstd_in
  * fp32 [C]), stores a to a_out ([B][H][W][C], what the backward sweep reads) and computes y = conv3x3(a, w) with the
- * statistics of y as ddg_conv3x3_fwd_stats does (Eq. 3 for batch norm -> ReLU -> convolution).  DDG_ERR_UNSUPPORTED
- * where the launch plan of the shape has no room for the transform warps (very large batches). */
-ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *gamma, const void *beta, const float *mean_in,
-                                        const float *invstd_in, void *a_out, const void *w, const void *packed, void *y,
+ * statistics of y as ddg_conv3x3_fwd_stats does (Eq. 3 for batch norm -> ReLU -> convolution).  res (nullable, same
+ * shape as x): the batch norm closes a residual block and a = relu(bn(x) + res), which is how the first convolution of
+ * the NEXT block consumes the previous block's output. */
+ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *res, const void *gamma, const void *beta,
+                                        const float *mean_in, const float *invstd_in, void *a_out, const void *w,
+                                        const void *packed, void *y,
                                         float *mean, float *invstd, float *scratch, int B, int H, int W, int C,
                                         void *stream);
 /* Input gradient of the stride-2 convolution of a down-sampling block (Cin -> 2 Cin, bf16, tensor-core path only) with

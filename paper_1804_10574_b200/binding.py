@@ -91,7 +91,7 @@ _lib.ddg_conv3x3_packed.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_conv3x3_fused_scratch_elems.argtypes = [_i] * 4
 _lib.ddg_conv3x3_fused_scratch_elems.restype = _sz
 _lib.ddg_conv3x3_fwd_stats.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
-_lib.ddg_conv3x3_bnrelu_fwd_stats.argtypes = [_vp] * 12 + [_i] * 4 + [_vp]
+_lib.ddg_conv3x3_bnrelu_fwd_stats.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_dgrad_fused.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_s2_dgrad_shortcut.argtypes = [_vp] * 5 + [_i] * 4 + [_vp]
 _lib.ddg_conv1x1_fwd.argtypes = [_i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]
@@ -262,9 +262,9 @@ def conv3x3_fwd_stats(x, w, packed, y, mean, invstd, scratch, B, H, W, C, stream
                                    B, H, W, C, stream))
 
 
-def conv3x3_bnrelu_fwd_stats(x, gamma, beta, mean_in, invstd_in, a_out, w, packed, y, mean, invstd, scratch, B, H, W, C,
-                             stream=None):
-    _ok(_lib.ddg_conv3x3_bnrelu_fwd_stats(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(mean_in), _ptr(invstd_in), _ptr(a_out),
+def conv3x3_bnrelu_fwd_stats(x, res, gamma, beta, mean_in, invstd_in, a_out, w, packed, y, mean, invstd, scratch, B, H, W,
+                             C, stream=None):
+    _ok(_lib.ddg_conv3x3_bnrelu_fwd_stats(_ptr(x), _ptr(res), _ptr(gamma), _ptr(beta), _ptr(mean_in), _ptr(invstd_in), _ptr(a_out),
                                           _ptr(w), _ptr(packed), _ptr(y), _ptr(mean), _ptr(invstd), _ptr(scratch), B, H, W, C,
                                           stream))
 

@@ -125,8 +125,9 @@ ddg_status ddg_conv3x3_fwd_stats(const void *x, const void *w, const void *packe
     return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, s, bf));
 }
 
-ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *gamma, const void *beta, const float *mean_in,
-                                        const float *invstd_in, void *a_out, const void *w, const void *packed, void *y,
+ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *res, const void *gamma, const void *beta,
+                                        const float *mean_in, const float *invstd_in, void *a_out, const void *w,
+                                        const void *packed, void *y,
                                         float *mean, float *invstd, float *scratch, int B, int H, int W, int C,
                                         void *stream) {
     if (!x || !gamma || !beta || !mean_in || !invstd_in || !a_out || !w || !y || !mean || !invstd || !scratch)
@@ -139,7 +140,7 @@ ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *gamma, const 
     BnFuse bf;
     bf.counter = reinterpret_cast<unsigned *>(scratch); bf.part = scratch + 32; bf.o0 = mean; bf.o1 = invstd;
     InXform xf;
-    xf.gamma = gamma; xf.beta = beta; xf.mean = mean_in; xf.invstd = invstd_in; xf.a_out = a_out;
+    xf.gamma = gamma; xf.beta = beta; xf.mean = mean_in; xf.invstd = invstd_in; xf.a_out = a_out; xf.res = res;
     return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, s, bf, xf));
 }
 

@@ -163,19 +163,22 @@ struct EpiPlan { int n_pipes, n_acc, n_slots, split; };
 // (bound of 768 threads: caps the kernel at 80 registers, so that two 384-thread CTAs of different streams share an SM)
 template <int C>
 __global__ void __launch_bounds__(768, 1)
-conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
+conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_res,
+                  const bf16 *__restrict__ w, const uint8_t *__restrict__ w_packed,
                   bf16 *__restrict__ dst, int dgrad, int H, int W, int rows_per_tile, int imgs_per_tile, int n_tiles,
                   int slab, int n_stages, int stage_bytes, int tmem_cols, EpiPlan plan_e, const bf16 *__restrict__ res_dout,
                   const bf16 *__restrict__ res_out, float *__restrict__ stat_part, unsigned *__restrict__ stat_counter,
                   float *__restrict__ stat_o0, float *__restrict__ stat_o1, const bf16 *__restrict__ bn_mask,
                   const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd,
                   const bf16 *__restrict__ xf_gamma, const bf16 *__restrict__ xf_beta, const float *__restrict__ xf_mean,
-                  const float *__restrict__ xf_invstd, bf16 *__restrict__ xf_out, int *__restrict__ err_word) {
+                  const float *__restrict__ xf_invstd, bf16 *__restrict__ xf_out, int xf_res, int *__restrict__ err_word) {
     // xf_gamma != nullptr (forward only): the source tensor is the raw output y of the previous convolution and this
     // kernel applies that convolution's batch norm and ReLU on its own operand path: four transform warps per pipeline
     // turn every TMA box, in place in shared memory, into a = relu(y * scale + shift) (scale = gamma * invstd, shift =
     // beta - mean * scale; rows outside the image stay zero: they are the convolution's padding), store the tile's own
-    // rows of a to xf_out (the backward sweep reads them) and only then hand the stage to the MMA warp.
+    // rows of a to xf_out (the backward sweep reads them) and only then hand the stage to the MMA warp.  xf_res != 0: the
+    // batch norm closes a residual block, a = relu(y * scale + shift + res): the stage holds a second box, fetched through
+    // tmap_res with the same coordinates, right behind the first.
     // stat_part != nullptr: the epilogue also reduces, per channel over the pixels of this CTA's tiles, the two sums the
     // batch norm that follows needs, from the values as stored (rounded to bf16), writes them to
     // stat_part[blockIdx.x][2C], and the CTA that finishes last adds the partials in a fixed order:
@@ -280,6 +283,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                     const uint32_t land = xform ? raw_bar(s) : full_bar(s);
                     mbar_expect_tx(land, (uint32_t)stage_bytes);
                     tma_load_4d(a_base + s * stage_bytes, &tmap, land, 0, 0, slab ? h0 - 1 : h0 + j - 1, n0);
+                    if (xf_res)  // the residual's box behind it (a stage is then two boxes)
+                        tma_load_4d(a_base + s * stage_bytes + stage_bytes / 2, &tmap_res, land, 0, 0, slab ? h0 - 1 : h0 + j - 1, n0);
                     if (++ls == ring) { ls = 0; ph ^= 1u; }
                 }
             }
@@ -355,12 +360,18 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const bf16 *__restri
                     if (h < 0 || h >= H) continue;             // padding: the zero fill stays
                     const uint4 q = *cell;
                     const uint32_t wq[4] = {q.x, q.y, q.z, q.w};
+                    uint32_t rq[4] = {0u, 0u, 0u, 0u};
+                    if (xf_res) {
+                        const uint4 r4 = *reinterpret_cast<const uint4 *>(stage + stage_bytes / 2 + swz_off<C>(p, 8 * cg));
+                        rq[0] = r4.x; rq[1] = r4.y; rq[2] = r4.z; rq[3] = r4.w;
+                    }
                     uint32_t o[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const int c0 = 8 * cg + 2 * k;
                         float a = fmaf(__uint_as_float(wq[k] << 16), sm_xf[c0], sm_xf[C + c0]);
                         float b = fmaf(__uint_as_float(wq[k] & 0xffff0000u), sm_xf[c0 + 1], sm_xf[C + c0 + 1]);
+                        if (xf_res) { a += __uint_as_float(rq[k] << 16); b += __uint_as_float(rq[k] & 0xffff0000u); }
                         a = a > 0.f ? a : 0.f;
                         b = b > 0.f ? b : 0.f;
                         const __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
@@ -1235,6 +1246,12 @@ TcPlan tc_plan(int C, int n_tiles, int slab, bool shared, bool xform) {
     } else {
         ep = EpiPlan{1, n_tiles <= sms ? 1 : 2, 1, 2};
     }
+    if (xform) {
+        // four transform warps per pipeline must fit the kernel's 768 threads: at most two pipelines, one epilogue group
+        // each where the plan above would launch two
+        if (ep.n_pipes > 2) ep = EpiPlan{2, 1, 1, 1};
+        if (2 * ep.n_pipes + 4 * ep.n_pipes * ep.n_slots * ep.split + 4 * ep.n_pipes > 24) ep = EpiPlan{2, ep.n_acc, 1, 1};
+    }
     TcPlan p;
     p.ep = ep;
     const int per_pipe = (n_tiles + sms * ep.n_pipes - 1) / (sms * ep.n_pipes);
@@ -1256,10 +1273,12 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     const int box_rows = slab ? rows + 2 : rows;
     CUtensorMap map;
     if (32 % W != 0 || !get_map(src, B, H, W, C, box_rows, imgs, &map)) return -1;
-    const int stage_bytes = box_rows * imgs * W * C * 2;
-    const int n_tiles = (int)((long)B * H * W / kTileM);
     const bool xform = xf.gamma != nullptr;
     if (xform && dir != 0) return -1;
+    CUtensorMap map_res = map;
+    if (xform && xf.res != nullptr && !get_map(xf.res, B, H, W, C, box_rows, imgs, &map_res)) return -1;
+    const int stage_bytes = box_rows * imgs * W * C * 2 * (xform && xf.res != nullptr ? 2 : 1);
+    const int n_tiles = (int)((long)B * H * W / kTileM);
     const TcPlan pl = tc_plan(C, n_tiles, slab, s.shared, xform);
     const EpiPlan ep = pl.ep;
     const int grid = pl.grid, threads = pl.threads;
@@ -1275,10 +1294,10 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     int tmem_cols = 32;
     while (tmem_cols < acc_cols) tmem_cols <<= 1;
     if (tmem_cols > 512 || conv_smem_bytes<C>(n_stages, stage_bytes) > (size_t)kSmemMax) return -1;
-    launch_kp(true, conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
+    launch_kp(true, conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, map_res, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
         stage_bytes, tmem_cols, ep, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
         bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd, (const bf16 *)xf.gamma,
-        (const bf16 *)xf.beta, xf.mean, xf.invstd, (bf16 *)xf.a_out, err_word_of(s));
+        (const bf16 *)xf.beta, xf.mean, xf.invstd, (bf16 *)xf.a_out, (xform && xf.res != nullptr) ? 1 : 0, err_word_of(s));
     return 1;
 }
 
@@ -1432,6 +1451,15 @@ bool conv_tc_xform_supported(int B, int H, int W, int C, bool shared) {
     int rows, imgs;
     tile_geometry(H, W, &rows, &imgs);
     return tc_plan(C, (int)((long)B * H * W / kTileM), imgs == 1 ? 1 : 0, shared, true).threads <= 768;
+}
+
+bool conv_tc_xform_keeps_plan(int B, int H, int W, int C, bool shared) {
+    if (!conv_tc_xform_supported(B, H, W, C, shared)) return false;
+    int rows, imgs;
+    tile_geometry(H, W, &rows, &imgs);
+    const int n_tiles = (int)((long)B * H * W / kTileM), slab = imgs == 1 ? 1 : 0;
+    const EpiPlan a = tc_plan(C, n_tiles, slab, shared, true).ep, b = tc_plan(C, n_tiles, slab, shared, false).ep;
+    return a.n_pipes == b.n_pipes && a.n_acc == b.n_acc && a.n_slots == b.n_slots && a.split == b.split;
 }
 
 int conv_tc_grid(int B, int H, int W) {

@@ -34,12 +34,18 @@ struct BnFuse {
 // outside the image stay zero: they are this convolution's padding), and stores a to a_out (same shape as src) for the
 // backward sweep.  The arithmetic is that of the element-wise batch-norm pass, value for value.  Available where
 // conv_tc_xform_supported says so (the plan's thread count, with four transform warps per pipeline, fits the kernel).
+// res != nullptr: the batch norm closes a residual block, a = relu(y * scale + shift + res) (res: same shape as src,
+// fetched by a second TMA box per stage).
 struct InXform {
     const void *gamma = nullptr, *beta = nullptr;
     const float *mean = nullptr, *invstd = nullptr;
     void *a_out = nullptr;
+    const void *res = nullptr;
 };
 bool conv_tc_xform_supported(int B, int H, int W, int C, bool shared);
+// true where the transform warps fit beside the launch plan the kernel would take anyway (the training step's sizes); at
+// very large batches the plan is cut down to make room for them, and the separate element-wise kernel is the better choice
+bool conv_tc_xform_keeps_plan(int B, int H, int W, int C, bool shared);
 int launch_conv_tc(int dir, const void *src, const void *w, const void *w_packed, void *dst, int B, int H, int W, int C,
                    Shortcut sc, Launch s, BnFuse bf = BnFuse(), InXform xf = InXform());
 int conv_tc_grid(int B, int H, int W);

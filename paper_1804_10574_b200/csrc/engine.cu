@@ -216,6 +216,10 @@ Count forward_module(ddg_ctx *c, int k, long t) {
     auto pkp = [&](long off) -> const void * { return (pk && off >= 0) ? pk + off : nullptr; };
     Count n;
     const bool fuse_bn = !c->cfg.separate_bn_sums;
+    // A block's closing pass out = relu(bn2(y2) + x) may be left to the first convolution of the next block, which then
+    // reads y2 and x, computes `out` on its operand path and stores it: `owed` describes such a pass.
+    InXform owed;
+    const void *owed_src = nullptr;
     for (int l = m.first; l <= m.last; ++l) {
         LayerPlan &L = c->layers[l];
         const char *w = wv + L.p_off * es;
@@ -280,8 +284,10 @@ Count forward_module(ddg_ctx *c, int k, long t) {
             // bn1's normalise + ReLU pass rides on conv2's operand path where the tensor-core kernel can take it: conv2
             // then reads the raw y1, computes a1 in shared memory and stores it for the backward sweep
             const bool ride = !c->cfg.separate_bn_apply && fuse_bn && c->prec == P_BF16 &&
-                              conv_tc_xform_supported(B, L.Hout, L.Wout, Co, s.shared);
-            conv_stats(in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, stt, stt + Co, InXform{});
+                              conv_tc_xform_keeps_plan(B, L.Hout, L.Wout, Co, s.shared);
+            conv_stats(owed_src ? owed_src : in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, stt, stt + Co, owed);
+            owed = InXform{};
+            owed_src = nullptr;
             if (!ride) n += launch_bn_apply(c->prec, y1, g1, b1, stt, stt + Co, Shortcut{}, a1, B, L.Hout, L.Wout, Co, 1, s);
             Shortcut sc{};
             sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
@@ -295,7 +301,21 @@ Count forward_module(ddg_ctx *c, int k, long t) {
             InXform xf;
             if (ride) { xf.gamma = g1; xf.beta = b1; xf.mean = stt; xf.invstd = stt + Co; xf.a_out = a1; }
             conv_stats(ride ? y1 : a1, w2, pkp(L.pk2), y2, L.Hout, L.Wout, Co, 1, stt + 2 * Co, stt + 3 * Co, xf);
-            n += launch_bn_apply(c->prec, y2, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out, B, L.Hout, L.Wout, Co, 1, s);
+            // the closing pass goes to the next block's first convolution when that is a plain stride-1 block of the same
+            // width in this module and the shortcut is the identity (the residual box then has the shape of y2)
+            bool defer = false;
+            if (ride && sc.mode == 1 && L.spec.kind == DDG_BASIC_BLOCK && l + 1 <= m.last) {
+                const LayerPlan &Nx = c->layers[l + 1];
+                defer = Nx.spec.kind == DDG_BASIC_BLOCK && Nx.spec.stride == 1 && Nx.Cin == Nx.Cout && Nx.Cin == Co &&
+                        conv_tc_xform_keeps_plan(B, Nx.Hin, Nx.Win, Nx.Cin, s.shared);
+            }
+            if (defer) {
+                owed.gamma = g2; owed.beta = b2; owed.mean = stt + 2 * Co; owed.invstd = stt + 3 * Co;
+                owed.a_out = out; owed.res = in;
+                owed_src = y2;
+            } else {
+                n += launch_bn_apply(c->prec, y2, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out, B, L.Hout, L.Wout, Co, 1, s);
+            }
             break;
         }
         }

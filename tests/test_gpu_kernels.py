@@ -442,7 +442,8 @@ def test_conv1x1_projection(shape, prec):
 @pytest.mark.parametrize("shape", [(3, 32, 32, 16), (5, 16, 16, 32), (128, 8, 8, 64), (2, 8, 8, 16), (8, 8, 8, 32),
                                    (128, 32, 32, 16), (128, 16, 16, 32), (301, 32, 32, 16), (231, 16, 16, 32), (902, 8, 8, 64)],
                          ids=lambda s: "x".join(map(str, s)))
-def test_conv_forward_with_batch_norm_relu_on_its_operand_path(shape):
+@pytest.mark.parametrize("with_res", [False, True], ids=["bn_relu", "bn_add_relu"])
+def test_conv_forward_with_batch_norm_relu_on_its_operand_path(shape, with_res):
     """Eq. 3 for batch norm -> ReLU -> convolution in one kernel: a = relu(bn(x)) computed in shared memory from the raw
     x (stored to a_out), y = conv3x3(a) and the statistics of y.  a against the oracle's batch norm + ReLU (and bit for
     bit against the element-wise kernel); y against the oracle's convolution of the a the GPU stored."""
@@ -454,16 +455,17 @@ def test_conv_forward_with_batch_norm_relu_on_its_operand_path(shape):
     gamma = torch.from_numpy(1 + 0.2 * rng.standard_normal(C)).to(torch.bfloat16)
     beta = torch.from_numpy(0.2 * rng.standard_normal(C)).to(torch.bfloat16)
     gh, bh = gamma.to(torch.float64).numpy(), beta.to(torch.float64).numpy()
+    r, rh = to_dev(rng.standard_normal((B, C, H, W)), 1)
     a_ref, m_ref, is_ref = orc.bn_forward(xh, gh, bh)
-    a_ref = np.maximum(a_ref, 0)
+    a_ref = np.maximum(a_ref + (rh if with_res else 0.0), 0)
     mean_in = torch.from_numpy(m_ref.astype(np.float32)).cuda()
     invstd_in = torch.from_numpy(is_ref.astype(np.float32)).cuda()
     a = torch.full_like(x, 7.0)
     y = torch.empty_like(x)
     mean, invstd = (torch.empty(C, dtype=torch.float32, device="cuda") for _ in range(2))
     scratch = torch.zeros(binding.conv3x3_fused_scratch_elems(B, H, W, C), dtype=torch.float32, device="cuda")
-    binding.conv3x3_bnrelu_fwd_stats(x, gamma.cuda(), beta.cuda(), mean_in, invstd_in, a, w, None, y, mean, invstd, scratch,
-                                     B, H, W, C)
+    binding.conv3x3_bnrelu_fwd_stats(x, r if with_res else None, gamma.cuda(), beta.cuda(), mean_in, invstd_in, a, w, None, y,
+                                     mean, invstd, scratch, B, H, W, C)
     torch.cuda.synchronize()
     arms = float(np.sqrt(np.mean(a_ref ** 2)))
     assert rel(from_dev(a), a_ref) < TOL[1]
@@ -473,7 +475,7 @@ def test_conv_forward_with_batch_norm_relu_on_its_operand_path(shape):
     a2 = torch.empty_like(x)
     m2, i2 = (torch.empty(C, dtype=torch.float32, device="cuda") for _ in range(2))
     sc2 = torch.zeros(binding.bn_scratch_elems(C), dtype=torch.float32, device="cuda")
-    binding.bn_fwd(1, x, gamma.cuda(), beta.cuda(), None, a2, m2, i2, sc2, B, H * W, C, 1)
+    binding.bn_fwd(1, x, gamma.cuda(), beta.cuda(), r if with_res else None, a2, m2, i2, sc2, B, H * W, C, 1)
     torch.cuda.synchronize()
     if torch.equal(m2, mean_in) and torch.equal(i2, invstd_in):      # same statistics in, same bits out
         assert torch.equal(a.view(B, H * W, C), a2.view(B, H * W, C))
