@@ -39,6 +39,7 @@ def parse():
                    "min(--steps, 100) for --impl reference)")
     p.add_argument("--skip-cpu", action="store_true")
     p.add_argument("--skip-k1", action="store_true", help="leave out the K = 1 arm")
+    p.add_argument("--fuse-bn-apply", type=int, default=0, help="ddg_cfg.fuse_bn_apply (A/B runs)")
     return p.parse_args()
 
 
@@ -292,7 +293,8 @@ def main():
     o = cfg["opt"]
     net = binding.Ddg(cfg["layers"], cfg["split_after"], cfg["batch"], cfg["in_shape"], cfg["num_classes"],
                       precision=cfg["precision"], lr=o["lr"], momentum=o["momentum"], weight_decay=o["weight_decay"],
-                      use_graph=not args.no_graph, streams=[s.cuda_stream for s in streams])
+                      use_graph=not args.no_graph, streams=[s.cuda_stream for s in streams],
+                      fuse_bn_apply=args.fuse_bn_apply)
     net.set_weights(synth.init_weights(cfg["layers"]))
     n_batches = K + 2
     host = [synth.batch(t, cfg["batch"], cfg["in_shape"], cfg["num_classes"]) for t in range(n_batches)]

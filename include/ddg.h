@@ -98,9 +98,13 @@ typedef struct {
     void *const *streams; /* host array of K cudaStream_t to run the modules on, or NULL (library creates K) */
     int separate_bn_sums; /* 0 (default): the batch-norm sums are taken in the epilogue of the tensor-core convolution
                        that produces the tensor.  1: separate reduction kernels (same sums, other summation order). */
-    int separate_bn_apply; /* 0 (default): inside a residual block the first batch norm's normalise + ReLU pass runs on
-                       the operand path of the second convolution (tensor-core kernel, shared memory) instead of as a
-                       kernel of its own.  1: separate element-wise kernels everywhere (same values, bit for bit). */
+    int fuse_bn_apply; /* Where the normalise + ReLU pass of a batch norm runs.  0 (default): element-wise kernels of
+                       their own.  1: inside a residual block, the first batch norm's pass runs on the operand path of
+                       the second convolution (transform warps between the TMA box and the MMAs).  2: also the block's
+                       closing pass relu(bn2(y2) + x), on the operand path of the NEXT block's first convolution.  Same
+                       values bit for bit, 8 % / 15 % fewer launches - and, at the sizes measured (ResNet-110, batch
+                       128), a slower iteration: the extra warps push the convolution CTA past half an SM's registers,
+                       so that kernels of two module streams no longer share an SM.  Kept as an option. */
     int launch_overlap; /* programmatic dependent launch (the next kernel of a stream is placed while the previous one
                        still runs).  0 (default): the library's policy: every kernel when K = 1; with several module
                        streams only the forward / input-gradient convolutions.  1: never.  2: every kernel. */

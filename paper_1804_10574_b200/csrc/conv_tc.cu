@@ -171,9 +171,9 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
                   float *__restrict__ stat_o0, float *__restrict__ stat_o1, const bf16 *__restrict__ bn_mask,
                   const bf16 *__restrict__ bn_x, const float *__restrict__ bn_mean, const float *__restrict__ bn_invstd,
                   const bf16 *__restrict__ xf_gamma, const bf16 *__restrict__ xf_beta, const float *__restrict__ xf_mean,
-                  const float *__restrict__ xf_invstd, bf16 *__restrict__ xf_out, int xf_res, int *__restrict__ err_word) {
+                  const float *__restrict__ xf_invstd, bf16 *__restrict__ xf_out, int xf_res, int xf_warps, int *__restrict__ err_word) {
     // xf_gamma != nullptr (forward only): the source tensor is the raw output y of the previous convolution and this
-    // kernel applies that convolution's batch norm and ReLU on its own operand path: four transform warps per pipeline
+    // kernel applies that convolution's batch norm and ReLU on its own operand path: xf_warps transform warps per pipeline
     // turn every TMA box, in place in shared memory, into a = relu(y * scale + shift) (scale = gamma * invstd, shift =
     // beta - mean * scale; rows outside the image stay zero: they are the convolution's padding), store the tile's own
     // rows of a to xf_out (the backward sweep reads them) and only then hand the stage to the MMA warp.  xf_res != 0: the
@@ -215,8 +215,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
         for (int i = threadIdx.x; i < 16 * 4 * 32; i += blockDim.x) (&sm_run[0][0][0])[i] = 0.f;
     if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");  // the first TMA would otherwise wait for its descriptor
-        // with the input transform a stage is full once each of the four transform warps has arrived
-        for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), xform ? 4 : 1); mbar_init(empty_bar(s), 1); mbar_init(raw_bar(s), 1); }
+        // with the input transform a stage is full once each of the pipeline's transform warps has arrived
+        for (int s = 0; s < n_stages; ++s) { mbar_init(full_bar(s), xform ? xf_warps : 1); mbar_init(empty_bar(s), 1); mbar_init(raw_bar(s), 1); }
         for (int a = 0; a < 4; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4 * plan_e.split); }
         mbar_init(w_bar, 1);
         *abort_flag = 0;
@@ -333,10 +333,18 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
     } else if (xform && warp >= 2 * n_pipes + 4 * n_epi_groups) {
         // ---------------- input transform: raw box -> relu(batch norm) in place, the tile's own rows also to global ------
         const int tw = warp - 2 * n_pipes - 4 * n_epi_groups;
-        const int g = tw >> 2, t128 = 32 * (tw & 3) + lane;  // pipeline, thread among its 128 transform threads
-        constexpr int kCg = C / 8;                            // 16-byte groups of channels per pixel
+        const int g = tw / xf_warps, t128 = 32 * (tw % xf_warps) + lane;  // pipeline, thread among its transform threads
+        const int xf_threads = 32 * xf_warps;
+        constexpr int kCg = C / 8;                            // 16-byte cells (8 channels) per pixel
         const int box_rows_img = slab ? rows_per_tile + 2 : rows_per_tile;  // image rows of a box, per image
-        const int n_vec = box_rows_img * imgs_per_tile * W * kCg;
+        const int n_pix = box_rows_img * imgs_per_tile * W;
+        // W and (image-pair tiles) H are powers of two; a thread keeps its cell of the pixel (the thread count is a
+        // multiple of the cells per pixel) and walks the pixels
+        const int log_w = 31 - __clz(W), log_h = 31 - __clz(H);
+        const int cg = t128 % kCg, p_first = t128 / kCg, p_step = xf_threads / kCg;
+        float sc[8], sh[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { sc[k] = sm_xf[8 * cg + k]; sh[k] = sm_xf[C + 8 * cg + k]; }
         int ls = 0;
         uint32_t ph = 0;
         bool ok = g < n_pipes;
@@ -352,36 +360,48 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
                 uint8_t *stage = smem + plan.a_off + (size_t)s * stage_bytes;
                 const int row_first = slab ? h0 - 1 : j - 1;   // image row of the box's first row
                 const bool owns = slab || j == 1;              // the unshifted box holds the tile's own pixels
-                for (int v = t128; v < n_vec; v += 128) {
-                    const int cg = v % kCg, p = v / kCg;       // p: pixel of the box, (image, row, column) order
-                    const int col = p % W, r = (p / W) % box_rows_img, img = p / (W * box_rows_img);
-                    const int h = row_first + r;
-                    uint4 *cell = reinterpret_cast<uint4 *>(stage + swz_off<C>(p, 8 * cg));
-                    if (h < 0 || h >= H) continue;             // padding: the zero fill stays
-                    const uint4 q = *cell;
-                    const uint32_t wq[4] = {q.x, q.y, q.z, q.w};
-                    uint32_t rq[4] = {0u, 0u, 0u, 0u};
-                    if (xf_res) {
-                        const uint4 r4 = *reinterpret_cast<const uint4 *>(stage + stage_bytes / 2 + swz_off<C>(p, 8 * cg));
-                        rq[0] = r4.x; rq[1] = r4.y; rq[2] = r4.z; rq[3] = r4.w;
-                    }
-                    uint32_t o[4];
+                constexpr int U = 2;                           // cells in flight per thread
+                for (int pb = p_first; pb < n_pix; pb += U * p_step) {
+                    uint4 q[U], rr[U];
+                    int hh[U];
+                    uint32_t off[U];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int c0 = 8 * cg + 2 * k;
-                        float a = fmaf(__uint_as_float(wq[k] << 16), sm_xf[c0], sm_xf[C + c0]);
-                        float b = fmaf(__uint_as_float(wq[k] & 0xffff0000u), sm_xf[c0 + 1], sm_xf[C + c0 + 1]);
-                        if (xf_res) { a += __uint_as_float(rq[k] << 16); b += __uint_as_float(rq[k] & 0xffff0000u); }
-                        a = a > 0.f ? a : 0.f;
-                        b = b > 0.f ? b : 0.f;
-                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
-                        o[k] = *reinterpret_cast<const uint32_t *>(&h2);
+                    for (int u = 0; u < U; ++u) {
+                        const int p = pb + u * p_step;
+                        const int r = slab ? (p >> log_w) : ((p >> log_w) & (H - 1));
+                        hh[u] = (p < n_pix) ? row_first + r : -1;   // -1: nothing to do (past the box, or padding)
+                        if (hh[u] >= H) hh[u] = -1;
+                        off[u] = swz_off<C>(p, 8 * cg);
+                        if (hh[u] >= 0) {
+                            q[u] = *reinterpret_cast<const uint4 *>(stage + off[u]);
+                            if (xf_res) rr[u] = *reinterpret_cast<const uint4 *>(stage + stage_bytes / 2 + off[u]);
+                        }
                     }
-                    const uint4 res = make_uint4(o[0], o[1], o[2], o[3]);
-                    *cell = res;
-                    if (owns && (!slab || (r >= 1 && r <= rows_per_tile))) {
-                        const size_t pix = ((size_t)(n0 + img) * H + h) * W + col;
-                        *reinterpret_cast<uint4 *>(xf_out + pix * C + 8 * cg) = res;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (hh[u] < 0) continue;               // padding rows: the zero fill stays
+                        const uint32_t wq[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+                        const uint32_t rq[4] = {rr[u].x, rr[u].y, rr[u].z, rr[u].w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            float a = fmaf(__uint_as_float(wq[k] << 16), sc[2 * k], sh[2 * k]);
+                            float b = fmaf(__uint_as_float(wq[k] & 0xffff0000u), sc[2 * k + 1], sh[2 * k + 1]);
+                            if (xf_res) { a += __uint_as_float(rq[k] << 16); b += __uint_as_float(rq[k] & 0xffff0000u); }
+                            a = a > 0.f ? a : 0.f;
+                            b = b > 0.f ? b : 0.f;
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(a, b);
+                            o[k] = *reinterpret_cast<const uint32_t *>(&h2);
+                        }
+                        const uint4 res = make_uint4(o[0], o[1], o[2], o[3]);
+                        *reinterpret_cast<uint4 *>(stage + off[u]) = res;
+                        const int p = pb + u * p_step;
+                        const int r = slab ? (p >> log_w) : ((p >> log_w) & (H - 1));
+                        if (owns && (!slab || (r >= 1 && r <= rows_per_tile))) {
+                            const int img = slab ? 0 : (p >> (log_w + log_h));
+                            const size_t pix = ((size_t)(n0 + img) * H + hh[u]) * W + (p & (W - 1));
+                            *reinterpret_cast<uint4 *>(xf_out + pix * C + 8 * cg) = res;
+                        }
                     }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
@@ -1231,7 +1251,7 @@ constexpr int kSmemMax = 227 * 1024;
 // Several module streams (shared): as few CTAs as give every pipeline the same number of tiles as a full grid would give
 // the busiest one; the kernel's critical path is as long, and the SMs left over are free for the other streams (K = 4
 // step -2 %).  A kernel that has the GPU to itself takes every SM (a few pipelines then finish early).
-struct TcPlan { EpiPlan ep; int grid, threads; };
+struct TcPlan { EpiPlan ep; int grid, threads, xf_warps; };
 TcPlan tc_plan(int C, int n_tiles, int slab, bool shared, bool xform) {
     const int sms = g_num_sms;
     EpiPlan ep;
@@ -1259,8 +1279,12 @@ TcPlan tc_plan(int C, int n_tiles, int slab, bool shared, bool xform) {
     const int full = (n_tiles + ep.n_pipes - 1) / ep.n_pipes < sms ? (n_tiles + ep.n_pipes - 1) / ep.n_pipes : sms;
     p.grid = shared ? balanced : full;
     const int groups = ep.n_pipes * ep.n_slots * ep.split;
-    // issuing warps, four warps per epilogue group, and with the input transform four more warps per pipeline
-    p.threads = 32 * (2 * ep.n_pipes + 4 * (groups < 2 ? 2 : groups) + (xform ? 4 * ep.n_pipes : 0));
+    // Transform warps per pipeline: every thread a CTA launches is given the kernel's 80 registers, so these warps cost
+    // register file that CTAs of the other module streams would otherwise use; one warp keeps up with a 16-channel tile
+    // (12 - 24 16-byte cells per lane), the wider tiles get two and four.
+    p.xf_warps = xform ? (C == 16 ? 1 : (C == 32 ? 2 : 4)) : 0;
+    // issuing warps, four warps per epilogue group, and the transform warps
+    p.threads = 32 * (2 * ep.n_pipes + 4 * (groups < 2 ? 2 : groups) + p.xf_warps * ep.n_pipes);
     return p;
 }
 
@@ -1287,7 +1311,8 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     const int budget = n_tiles >= 8 * grid ? kSmemMax - 1024 - kTailBytes : kSmemBudget;
     int n_stages = (budget - (int)conv_smem_plan<C>(0, 0).a_off) / stage_bytes;
     if (n_stages > kMaxStages) n_stages = kMaxStages;
-    const int min_ring = 3;
+    int min_ring = 3;
+    if (conv_smem_bytes<C>(min_ring * ep.n_pipes, stage_bytes) > (size_t)kSmemMax) min_ring = 2;  // two-box stages of wide tiles
     if (n_stages < min_ring * ep.n_pipes) n_stages = min_ring * ep.n_pipes;
     n_stages -= n_stages % ep.n_pipes;
     const int acc_cols = ep.n_pipes * ep.n_acc * 3 * C;
@@ -1297,7 +1322,7 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     launch_kp(true, conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, map_res, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
         stage_bytes, tmem_cols, ep, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
         bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd, (const bf16 *)xf.gamma,
-        (const bf16 *)xf.beta, xf.mean, xf.invstd, (bf16 *)xf.a_out, (xform && xf.res != nullptr) ? 1 : 0, err_word_of(s));
+        (const bf16 *)xf.beta, xf.mean, xf.invstd, (bf16 *)xf.a_out, (xform && xf.res != nullptr) ? 1 : 0, pl.xf_warps, err_word_of(s));
     return 1;
 }
 

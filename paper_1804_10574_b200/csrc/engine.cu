@@ -283,7 +283,7 @@ Count forward_module(ddg_ctx *c, int k, long t) {
             };
             // bn1's normalise + ReLU pass rides on conv2's operand path where the tensor-core kernel can take it: conv2
             // then reads the raw y1, computes a1 in shared memory and stores it for the backward sweep
-            const bool ride = !c->cfg.separate_bn_apply && fuse_bn && c->prec == P_BF16 &&
+            const bool ride = c->cfg.fuse_bn_apply >= 1 && fuse_bn && c->prec == P_BF16 &&
                               conv_tc_xform_keeps_plan(B, L.Hout, L.Wout, Co, s.shared);
             conv_stats(owed_src ? owed_src : in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, stt, stt + Co, owed);
             owed = InXform{};
@@ -304,7 +304,7 @@ Count forward_module(ddg_ctx *c, int k, long t) {
             // the closing pass goes to the next block's first convolution when that is a plain stride-1 block of the same
             // width in this module and the shortcut is the identity (the residual box then has the shape of y2)
             bool defer = false;
-            if (ride && sc.mode == 1 && L.spec.kind == DDG_BASIC_BLOCK && l + 1 <= m.last) {
+            if (ride && c->cfg.fuse_bn_apply >= 2 && sc.mode == 1 && L.spec.kind == DDG_BASIC_BLOCK && l + 1 <= m.last) {
                 const LayerPlan &Nx = c->layers[l + 1];
                 defer = Nx.spec.kind == DDG_BASIC_BLOCK && Nx.spec.stride == 1 && Nx.Cin == Nx.Cout && Nx.Cin == Co &&
                         conv_tc_xform_keeps_plan(B, Nx.Hin, Nx.Win, Nx.Cin, s.shared);

@@ -259,13 +259,15 @@ def test_epilogue_batch_norm_sums_match_separate_reductions():
 
 
 def test_batch_norm_pass_on_the_operand_path_gives_the_same_bits():
-    """The first batch norm's normalise + ReLU pass inside the second convolution (shared memory, between TMA box and
-    MMA) and the separate element-wise kernel compute the same values: identical weights after six iterations, fewer
+    """The normalise + ReLU passes inside the convolution that consumes them (shared memory, between TMA box and MMA;
+    fuse_bn_apply = 1: the first batch norm of a block, 2: also the block's closing pass with the shortcut) and the
+    separate element-wise kernels compute the same values: identical losses and weights after six iterations, fewer
     launches."""
     wa, la, na = _resnet20_k3_bf16_run()
-    wb, lb, nb = _resnet20_k3_bf16_run(separate_bn_apply=True)
-    assert na < nb
-    assert la == lb and np.array_equal(wa, wb)
+    wb, lb, nb = _resnet20_k3_bf16_run(fuse_bn_apply=1)
+    wc, lc, nc = _resnet20_k3_bf16_run(fuse_bn_apply=2)
+    assert nc < nb < na
+    assert la == lb == lc and np.array_equal(wa, wb) and np.array_equal(wa, wc)
 
 
 def test_launch_overlap_settings_give_the_same_bits():
