@@ -40,6 +40,7 @@ def parse():
     p.add_argument("--skip-cpu", action="store_true")
     p.add_argument("--skip-k1", action="store_true", help="leave out the K = 1 arm")
     p.add_argument("--fuse-bn-apply", type=int, default=0, help="ddg_cfg.fuse_bn_apply (A/B runs)")
+    p.add_argument("--bn-fold", type=int, default=0, help="ddg_cfg.bn_fold (A/B runs)")
     return p.parse_args()
 
 
@@ -66,7 +67,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -294,7 +295,7 @@ def main():
     net = binding.Ddg(cfg["layers"], cfg["split_after"], cfg["batch"], cfg["in_shape"], cfg["num_classes"],
                       precision=cfg["precision"], lr=o["lr"], momentum=o["momentum"], weight_decay=o["weight_decay"],
                       use_graph=not args.no_graph, streams=[s.cuda_stream for s in streams],
-                      fuse_bn_apply=args.fuse_bn_apply)
+                      fuse_bn_apply=args.fuse_bn_apply, bn_fold=args.bn_fold)
     net.set_weights(synth.init_weights(cfg["layers"]))
     n_batches = K + 2
     host = [synth.batch(t, cfg["batch"], cfg["in_shape"], cfg["num_classes"]) for t in range(n_batches)]
@@ -323,7 +324,6 @@ def main():
     e1.record(streams[0])
     barrier()
     dt = e0.elapsed_time(e1) * 1e-3
-    clocks = sampler.stop()
 
     # ---- end to end through the public call with host buffers: H2D of x, y and D2H of the loss every step ----
     for t in range(3):
@@ -338,6 +338,9 @@ def main():
     f1.record(streams[0])
     barrier()
     dt_e2e = f0.elapsed_time(f1) * 1e-3
+    # the sampler ran through both timed regions (device-resident and end-to-end): a 20-iteration region alone lasts
+    # ~40 ms, too short for nvidia-smi's sampling period to land in it reliably
+    clocks = sampler.stop()
     net.destroy()
 
     # ---- the same kernels with K = 1 (plain backpropagation, Section 3.2), same run, same batches ----

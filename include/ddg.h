@@ -105,6 +105,12 @@ typedef struct {
                        values bit for bit, 8 % / 15 % fewer launches - and, at the sizes measured (ResNet-110, batch
                        128), a slower iteration: the extra warps push the convolution CTA past half an SM's registers,
                        so that kernels of two module streams no longer share an SM.  Kept as an option. */
+    int bn_fold; /* Who adds up the per-CTA partial sums a convolution epilogue leaves for the batch norm behind it.
+                       1: the convolution's CTA that finishes last (ticket counter; costs that kernel ~4 us of serial
+                       tail, but only one CTA, which leaves the rest of the GPU to the other module streams).  2: the
+                       element-wise pass that consumes the sums, every CTA for itself (no tail; ~1.5 us more in every CTA
+                       of that pass).  0 (default): the library's policy: 2 for K = 1, 1 when several module streams
+                       share the GPU.  Both orders are fixed; the two settings differ in the last bits. */
     int launch_overlap; /* programmatic dependent launch (the next kernel of a stream is placed while the previous one
                        still runs).  0 (default): the library's policy: every kernel when K = 1; with several module
                        streams only the forward / input-gradient convolutions.  1: never.  2: every kernel. */

@@ -49,7 +49,7 @@ class Cfg(ctypes.Structure):
                 ("in_w", ctypes.c_int), ("num_classes", ctypes.c_int), ("seed", ctypes.c_ulonglong),
                 ("use_graph", ctypes.c_int), ("debug_checks", ctypes.c_int),
                 ("streams", ctypes.POINTER(ctypes.c_void_p)), ("separate_bn_sums", ctypes.c_int),
-                ("fuse_bn_apply", ctypes.c_int), ("launch_overlap", ctypes.c_int)]
+                ("fuse_bn_apply", ctypes.c_int), ("bn_fold", ctypes.c_int), ("launch_overlap", ctypes.c_int)]
 
 
 _vp, _i, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -134,7 +134,7 @@ class Ddg:
 
     def __init__(self, layers, split_after, batch, in_shape, num_classes, precision="fp32", opt="sgd", lr=0.01,
                  momentum=0.0, weight_decay=0.0, beta1=0.9, beta2=0.999, eps=1e-8, seed=0, use_graph=False,
-                 debug_checks=False, streams=None, separate_bn_sums=False, fuse_bn_apply=0,
+                 debug_checks=False, streams=None, separate_bn_sums=False, fuse_bn_apply=0, bn_fold=0,
                  launch_overlap=0):
         arr = (Layer * len(layers))(*[Layer(*map(int, l)) for l in layers])
         K = len(split_after) + 1
@@ -145,7 +145,7 @@ class Ddg:
             assert len(streams) == K
             st = (ctypes.c_void_p * K)(*[int(s) for s in streams])
         cfg = Cfg(BF16 if precision == "bf16" else FP32, batch, in_shape[0], in_shape[1], in_shape[2], num_classes,
-                  seed, int(use_graph), int(debug_checks), st, int(separate_bn_sums), int(fuse_bn_apply),
+                  seed, int(use_graph), int(debug_checks), st, int(separate_bn_sums), int(fuse_bn_apply), int(bn_fold),
                   int(launch_overlap))
         h = ctypes.c_void_p()
         rc = _lib.ddg_create(arr, len(layers), sp, K, ctypes.byref(o), ctypes.byref(cfg), ctypes.byref(h))

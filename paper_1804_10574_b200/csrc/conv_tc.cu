@@ -525,6 +525,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
         for (int wq = 0; wq < 16; ++wq) t += sm_run[wq][c >> 4][l];
         stat_part[(size_t)blockIdx.x * 2 * C + threadIdx.x] = t;
     }
+    if (stat_counter == nullptr) return;  // the kernel that consumes the sums folds the partials itself
     __threadfence();
     __syncthreads();
     int *is_last = reinterpret_cast<int *>(sm_stat);  // free again: the epilogue is over
@@ -1319,6 +1320,7 @@ int launch_tc(int dir, const void *src, const void *w, const void *w_packed, voi
     int tmem_cols = 32;
     while (tmem_cols < acc_cols) tmem_cols <<= 1;
     if (tmem_cols > 512 || conv_smem_bytes<C>(n_stages, stage_bytes) > (size_t)kSmemMax) return -1;
+    if (bf.n_part_out != nullptr) *bf.n_part_out = grid;
     launch_kp(true, conv3x3_tc_kernel<C>, grid, threads, conv_smem_bytes<C>(n_stages, stage_bytes), s, map, map_res, (const bf16 *)w, (const uint8_t *)w_packed, (bf16 *)dst, dir, H, W, rows, imgs, n_tiles, slab, n_stages,
         stage_bytes, tmem_cols, ep, sc.mode == 1 ? (const bf16 *)sc.a : nullptr, sc.mode == 1 ? (const bf16 *)sc.b : nullptr, bf.part,
         bf.counter, bf.o0, bf.o1, (const bf16 *)bf.mask, (const bf16 *)bf.x, bf.mean, bf.invstd, (const bf16 *)xf.gamma,

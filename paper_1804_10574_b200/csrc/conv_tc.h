@@ -21,9 +21,12 @@ bool conv_tc_supported(int B, int H, int W, int Cin, int Cout, int stride);
 // the result is the forward statistics bf.o0 = mean, bf.o1 = 1/sqrt(var + 1e-5).  Otherwise they are (sum dz, sum dz *
 // xhat), dz = output * [bf.mask > 0], xhat = (bf.x - bf.mean) * bf.invstd: the two reductions of the batch-norm
 // backward whose incoming gradient is this kernel's output; bf.o0 = dbeta, bf.o1 = dgamma.
+// counter == nullptr: the kernel only leaves the per-CTA partials (*n_part_out rows, one per CTA of its grid) and the
+// element-wise pass that consumes the sums folds them (BnPartials in kernels.h): no ticket, no serial tail in this kernel.
 struct BnFuse {
     float *part = nullptr;
     unsigned *counter = nullptr;
+    int *n_part_out = nullptr;
     float *o0 = nullptr, *o1 = nullptr;
     const void *mask = nullptr, *x = nullptr;
     const float *mean = nullptr, *invstd = nullptr;

@@ -113,6 +113,8 @@ struct ddg_ctx {
     int *err_word = nullptr;  // device: raised by a kernel whose bounded wait ran out or by a ring-stamp mismatch
     bool broken = false;
     std::string err;
+    // the element-wise batch-norm passes fold the convolution epilogues' partial sums themselves (ddg_cfg.bn_fold)
+    bool fold_in_consumer() const { return cfg.bn_fold == 2 || (cfg.bn_fold == 0 && K == 1); }
     // how this context's kernels are launched on stream st (Launch in kernels.h)
     Launch lx(cudaStream_t st) const {
         const int pdl = cfg.launch_overlap == 1 ? 0 : (cfg.launch_overlap == 2 ? 1 : (K == 1 ? 1 : 2));
@@ -270,25 +272,32 @@ Count forward_module(ddg_ctx *c, int k, long t) {
             // convolution followed by its batch norm; the statistics come from the convolution's epilogue where the
             // tensor-core kernel runs, from a reduction kernel otherwise
             // a convolution and the statistics of the batch norm that follows it; xf: an input transform for it to carry
+            // leave_partials: the pass that consumes the statistics is an element-wise kernel that folds the epilogue's
+            // per-CTA partial sums itself (no serial fold at the end of the convolution); returns them
             auto conv_stats = [&](const void *xin, const void *wc, const void *wp, void *yc, int H, int W, int Cic, int strd,
-                                  float *mean, float *invstd, InXform xf) {
+                                  float *mean, float *invstd, InXform xf, bool leave_partials) -> BnPartials {
+                BnPartials bp;
                 if (fuse_bn && c->prec == P_BF16 && conv_tc_supported(B, H, W, Cic, Co, strd)) {
                     BnFuse bf;
-                    bf.part = m.bn_scratch + 32; bf.counter = (unsigned *)m.bn_scratch; bf.o0 = mean; bf.o1 = invstd;
+                    bf.part = m.bn_scratch + 32; bf.o0 = mean; bf.o1 = invstd;
+                    if (leave_partials) { bf.n_part_out = &bp.n; bp.part = bf.part; }
+                    else bf.counter = (unsigned *)m.bn_scratch;
                     n += launch_conv_tc(0, xin, wc, wp, yc, B, H, W, Cic, Shortcut{}, s, bf, xf);
                 } else {
                     n += conv_fwd(c, xin, wc, wp, yc, H, W, Cic, Co, strd, 0, s);
                     n += launch_bn_stats(c->prec, yc, mean, invstd, m.bn_scratch, npix, Co, s);
                 }
+                return bp;
             };
             // bn1's normalise + ReLU pass rides on conv2's operand path where the tensor-core kernel can take it: conv2
             // then reads the raw y1, computes a1 in shared memory and stores it for the backward sweep
             const bool ride = c->cfg.fuse_bn_apply >= 1 && fuse_bn && c->prec == P_BF16 &&
                               conv_tc_xform_keeps_plan(B, L.Hout, L.Wout, Co, s.shared);
-            conv_stats(owed_src ? owed_src : in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, stt, stt + Co, owed);
+            const BnPartials bp1 = conv_stats(owed_src ? owed_src : in, w1, pkp(L.pk1), y1, L.Hin, L.Win, Ci, st, stt, stt + Co,
+                                              owed, !ride && c->fold_in_consumer() && bn_apply_takes_partials(c->prec, Co, 0));
             owed = InXform{};
             owed_src = nullptr;
-            if (!ride) n += launch_bn_apply(c->prec, y1, g1, b1, stt, stt + Co, Shortcut{}, a1, B, L.Hout, L.Wout, Co, 1, s);
+            if (!ride) n += launch_bn_apply(c->prec, y1, g1, b1, stt, stt + Co, Shortcut{}, a1, B, L.Hout, L.Wout, Co, 1, s, bp1);
             Shortcut sc{};
             sc.mode = (st == 1 && Ci == Co) ? 1 : 2;
             sc.a = in; sc.c_small = Ci; sc.h_big = L.Hin; sc.w_big = L.Win;
@@ -300,7 +309,6 @@ Count forward_module(ddg_ctx *c, int k, long t) {
             }
             InXform xf;
             if (ride) { xf.gamma = g1; xf.beta = b1; xf.mean = stt; xf.invstd = stt + Co; xf.a_out = a1; }
-            conv_stats(ride ? y1 : a1, w2, pkp(L.pk2), y2, L.Hout, L.Wout, Co, 1, stt + 2 * Co, stt + 3 * Co, xf);
             // the closing pass goes to the next block's first convolution when that is a plain stride-1 block of the same
             // width in this module and the shortcut is the identity (the residual box then has the shape of y2)
             bool defer = false;
@@ -309,12 +317,14 @@ Count forward_module(ddg_ctx *c, int k, long t) {
                 defer = Nx.spec.kind == DDG_BASIC_BLOCK && Nx.spec.stride == 1 && Nx.Cin == Nx.Cout && Nx.Cin == Co &&
                         conv_tc_xform_keeps_plan(B, Nx.Hin, Nx.Win, Nx.Cin, s.shared);
             }
+            const BnPartials bp2 = conv_stats(ride ? y1 : a1, w2, pkp(L.pk2), y2, L.Hout, L.Wout, Co, 1, stt + 2 * Co, stt + 3 * Co,
+                                              xf, !defer && c->fold_in_consumer() && bn_apply_takes_partials(c->prec, Co, sc.mode));
             if (defer) {
                 owed.gamma = g2; owed.beta = b2; owed.mean = stt + 2 * Co; owed.invstd = stt + 3 * Co;
                 owed.a_out = out; owed.res = in;
                 owed_src = y2;
             } else {
-                n += launch_bn_apply(c->prec, y2, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out, B, L.Hout, L.Wout, Co, 1, s);
+                n += launch_bn_apply(c->prec, y2, g2, b2, stt + 2 * Co, stt + 3 * Co, sc, out, B, L.Hout, L.Wout, Co, 1, s, bp2);
             }
             break;
         }
@@ -364,6 +374,7 @@ Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
     // true when the kernel that produced `cur` already left the two sums (dbeta, dgamma) of the batch norm that
     // consumes it in that batch norm's gradient slots
     bool cur_sums = false;
+    BnPartials cur_parts;  // ... as per-CTA partials that the element-wise pass folds (cur_sums is true as well)
     float *bn_part = m.bn_scratch + 32;
     unsigned *bn_counter = (unsigned *)m.bn_scratch;
     const bool fuse = !c->cfg.separate_bn_sums && c->prec == P_BF16;
@@ -394,6 +405,7 @@ Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
         // destination of the error gradient w.r.t. the layer input
         int dst_tmp = -1;
         bool next_sums = false;
+        BnPartials next_parts;
         char *dst = nullptr;
         if (need_dx) {
             if (mod_first) dst = m.delta_out[t % 2];
@@ -454,21 +466,25 @@ Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
             if (!cur_sums)
                 n += launch_bn_bwd_reduce(c->prec, cur, out, y2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, m.bn_scratch, npix, Co,
                                           1, s);
-            n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s);
+            n += launch_bn_bwd_apply(c->prec, cur, out, y2, g2, stt + 2 * Co, stt + 3 * Co, gg2, gb2, dy2, npix, Co, 1, s,
+                                     cur_sums ? cur_parts : BnPartials());
             side_wgrad(j2, a1, dy2, gw2, L.Hout, L.Wout, Co, Co, 1);
             const int j1 = ring_next();
             char *dy1 = m.dyring[j1];
+            BnPartials parts1;
             if (fuse && conv_tc_supported(B, L.Hout, L.Wout, Co, Co, 1)) {
                 // the input gradient of conv2 is the incoming gradient of bn1: its two sums come out of the same kernel
                 BnFuse bf;
-                bf.part = bn_part; bf.counter = bn_counter; bf.o0 = gb1; bf.o1 = gg1;
+                bf.part = bn_part; bf.o0 = gb1; bf.o1 = gg1;
                 bf.mask = a1; bf.x = y1; bf.mean = stt; bf.invstd = stt + Co;
+                if (c->fold_in_consumer() && bn_apply_takes_partials(c->prec, Co, 0)) { bf.n_part_out = &parts1.n; parts1.part = bn_part; }
+                else bf.counter = bn_counter;
                 n += launch_conv_tc(1, dy2, w2, pkp(L.pk2), da1, B, L.Hout, L.Wout, Co, Shortcut{}, s, bf);
             } else {
                 n += conv_dgrad(c, dy2, w2, pkp(L.pk2), da1, L.Hout, L.Wout, Co, Co, 1, Shortcut{}, s);
                 n += launch_bn_bwd_reduce(c->prec, da1, a1, y1, stt, stt + Co, gg1, gb1, m.bn_scratch, npix, Co, 1, s);
             }
-            n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s);
+            n += launch_bn_bwd_apply(c->prec, da1, a1, y1, g1, stt, stt + Co, gg1, gb1, dy1, npix, Co, 1, s, parts1);
             side_wgrad(j1, in, dy1, gw1, L.Hin, L.Win, Ci, Co, st);
             if (proj) {
                 // weight gradient of the projection, on the chain's own stream (it reads the incoming gradient in place
@@ -503,9 +519,12 @@ Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
                     // gradient slots of the block below: conv1, gamma1, beta1, conv2, gamma2, beta2
                     float *pg2 = m.g + Pv->p_off + (size_t)Ci * Pv->Cin * 9 + 2 * (size_t)Ci + (size_t)Ci * Ci * 9;
                     BnFuse bf;
-                    bf.part = bn_part; bf.counter = bn_counter; bf.o1 = pg2; bf.o0 = pg2 + Ci;
+                    bf.part = bn_part; bf.o1 = pg2; bf.o0 = pg2 + Ci;
                     bf.mask = in; bf.x = slot_ptr(c, Pv->y2, sidx);
                     bf.mean = pst + 2 * Ci; bf.invstd = pst + 3 * Ci;
+                    next_parts = BnPartials();
+                    if (c->fold_in_consumer() && bn_apply_takes_partials(c->prec, Ci, 0)) { bf.n_part_out = &next_parts.n; next_parts.part = bn_part; }
+                    else bf.counter = bn_counter;
                     n += launch_conv_tc(1, dy1, w1, pkp(L.pk1), dx, B, L.Hin, L.Win, Ci, sc, s, bf);
                     next_sums = true;
                 } else {
@@ -519,6 +538,7 @@ Count backward_module(ddg_ctx *c, int k, long t, long sidx) {
         cur = dst;
         cur_tmp = dst_tmp;
         cur_sums = next_sums;
+        cur_parts = next_parts;
     }
     side_join();  // the update that follows reads every gradient of the module
     return n;
@@ -812,6 +832,7 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
         return DDG_ERR_INVALID_ARG;
     }
     if (opt->kind != DDG_OPT_SGD && opt->kind != DDG_OPT_ADAM) { set_err(nullptr, "ddg_create: unknown optimiser"); return DDG_ERR_INVALID_ARG; }
+    if (cfg->bn_fold < 0 || cfg->bn_fold > 2 || cfg->fuse_bn_apply < 0 || cfg->fuse_bn_apply > 2) { set_err(nullptr, "ddg_create: bn_fold and fuse_bn_apply must be 0, 1 or 2"); return DDG_ERR_INVALID_ARG; }
     if (cfg->launch_overlap < 0 || cfg->launch_overlap > 2) { set_err(nullptr, "ddg_create: launch_overlap must be 0, 1 or 2"); return DDG_ERR_INVALID_ARG; }
     for (int k = 0; k + 1 < K; ++k)
         if (split_after[k] < 0 || split_after[k] >= n_layers - 1 || (k > 0 && split_after[k] <= split_after[k - 1])) {

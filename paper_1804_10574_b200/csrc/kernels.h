@@ -66,16 +66,29 @@ int launch_softmax_ce(int prec, const float *logits, const int *labels, float *l
 size_t bn_scratch_elems(int C);
 int launch_bn_stats(int prec, const void *x, float *mean, float *invstd, float *scratch, long npix, int C,
                     Launch s);
-// y = [relu](gamma*(x-mean)*invstd + beta + shortcut).  y is [B][H][W][C].
-int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta, const float *mean,
-                    const float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu, Launch s);
+// Per-CTA partial sums left by the epilogue of the convolution that produced a batch norm's input (or incoming gradient):
+// part[n][2C] fp32, rows in CTA order.  The element-wise pass that consumes the sums folds them itself, every CTA the
+// same rows in the same fixed order (so all CTAs hold identical totals and nothing has to be waited for or
+// broadcast), and its first CTA also stores the folded pair (mean, invstd) or (dbeta, dgamma) where the separate
+// reduction would have put it.  part == nullptr: the sums are already in place.
+struct BnPartials {
+    const float *part = nullptr;
+    int n = 0;
+};
+// true when launch_bn_apply / launch_bn_bwd_apply take partials for this case (the bf16 fast kernels)
+bool bn_apply_takes_partials(int prec, int C, int shortcut_mode);
+// y = [relu](gamma*(x-mean)*invstd + beta + shortcut).  y is [B][H][W][C].  With partials (sum x, sum x^2) the kernel
+// computes mean / invstd itself and WRITES them to `mean` / `invstd`.
+int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta, float *mean, float *invstd,
+                    Shortcut sc, void *y, int B, int H, int W, int C, int relu, Launch s, BnPartials bp = BnPartials());
 // sums[0..C) = sum dz, sums[C..2C) = sum dz*xhat with dz = dout*[out>0] (relu) ; also written to dbeta/dgamma.
 int launch_bn_bwd_reduce(int prec, const void *dout, const void *out, const void *x, const float *mean,
                          const float *invstd, float *dgamma, float *dbeta, float *scratch, long npix, int C, int relu,
                          Launch s);
+// With partials (sum dz, sum dz*xhat) the kernel folds them itself and WRITES dbeta / dgamma.
 int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void *x, const void *gamma,
-                        const float *mean, const float *invstd, const float *dgamma, const float *dbeta, void *dx,
-                        long npix, int C, int relu, Launch s);
+                        const float *mean, const float *invstd, float *dgamma, float *dbeta, void *dx,
+                        long npix, int C, int relu, Launch s, BnPartials bp = BnPartials());
 
 // ---- 3x3 convolution, CUDA-core kernels (any shape; used for fp32 and for shapes the tensor-core path skips) --
 int launch_conv_fwd_direct(int prec, const void *x, const void *w, void *y, int B, int H, int W, int Cin, int Cout,

@@ -721,18 +721,69 @@ bn_apply_kernel(const T *__restrict__ x, const T *__restrict__ gamma, const T *_
 // capped at three CTAs per SM.
 static constexpr int kApplyCtasPerSm = 3;
 
-template <int U>
+// Totals of n_part rows of nval = 2C per-CTA partial sums, by a whole CTA of kThreads threads, in a fixed order: the
+// rows are read as one flat array of 16-byte vectors (kThreads * 4 values per pass is a multiple of nval, so a thread
+// always meets the same four columns), up to eight independent loads in flight per thread, accumulated in double in
+// pass order; the threads that share a column are then added in index order.  Result: tot[0..nval) in shared memory.
+// fold: kThreads * 4 doubles of shared memory.
+__device__ __forceinline__ void fold_partials(const float *__restrict__ part, int n_part, int nval, double *fold, double *tot) {
+    const int t = threadIdx.x;
+    const int total4 = n_part * nval / 4;
+    double a[4] = {0.0, 0.0, 0.0, 0.0};
+    const float4 *p4 = reinterpret_cast<const float4 *>(part);
+    for (int i0 = t; i0 < total4; i0 += 8 * kThreads) {
+        float4 q[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * kThreads;
+            q[u] = i < total4 ? __ldcg(p4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { a[0] += (double)q[u].x; a[1] += (double)q[u].y; a[2] += (double)q[u].z; a[3] += (double)q[u].w; }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) fold[t * 4 + j] = a[j];
+    __syncthreads();
+    if (t < nval) {
+        // column t lives in the threads whose first vector covers it: thread (t / 4) + k * (nval / 4), element t % 4
+        double sum = 0.0;
+        for (int k = t / 4; k < kThreads; k += nval / 4) sum += fold[k * 4 + (t & 3)];
+        tot[t] = sum;
+    }
+    __syncthreads();
+}
+
+// FOLD: the statistics come as per-CTA partial sums that this kernel adds up first (an instantiation of its own: the
+// 10 KB of shared memory the fold needs would otherwise sit in every launch and keep other streams' CTAs off the SM)
+template <int U, bool FOLD>
 __global__ void __launch_bounds__(kThreads, kApplyCtasPerSm)
 bn_apply_fast_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ gamma, const bf16 *__restrict__ beta,
-                     const float *__restrict__ mean, const float *__restrict__ invstd, const bf16 *__restrict__ res,
-                     bf16 *__restrict__ y, long nvec, int C, int relu) {
+                     float *__restrict__ mean, float *__restrict__ invstd, const bf16 *__restrict__ res,
+                     bf16 *__restrict__ y, long nvec, int C, int relu, const float *__restrict__ part, int n_part) {
     __shared__ float sm_scale[128], sm_shift[128];
     pdl_launch();
     pdl_wait();
-    for (int c = threadIdx.x; c < C; c += kThreads) {
-        const float sc = to_f(gamma[c]) * invstd[c];
-        sm_scale[c] = sc;
-        sm_shift[c] = to_f(beta[c]) - mean[c] * sc;
+    if (FOLD) {
+        // statistics from the convolution epilogue's partial sums (sum x, sum x^2): every CTA folds them the same way
+        __shared__ double sm_fold[kThreads * 4], sm_tot[256];
+        fold_partials(part, n_part, 2 * C, sm_fold, sm_tot);
+        const double npix = (double)(nvec / (C / 8));
+        for (int c = threadIdx.x; c < C; c += kThreads) {
+            const double m = sm_tot[c] / npix;
+            double var = sm_tot[C + c] / npix - m * m;
+            if (var < 0.0) var = 0.0;
+            const float mf = (float)m, isf = (float)(1.0 / sqrt(var + (double)kBnEps));
+            if (blockIdx.x == 0) { mean[c] = mf; invstd[c] = isf; }  // the backward sweep reads them
+            const float sc = to_f(gamma[c]) * isf;
+            sm_scale[c] = sc;
+            sm_shift[c] = to_f(beta[c]) - mf * sc;
+        }
+    } else {
+        for (int c = threadIdx.x; c < C; c += kThreads) {
+            const float sc = to_f(gamma[c]) * invstd[c];
+            sm_scale[c] = sc;
+            sm_shift[c] = to_f(beta[c]) - mean[c] * sc;
+        }
     }
     __syncthreads();
     const int groups = C / 8;
@@ -791,18 +842,25 @@ static int apply_grid(long nvec, int U) {
     return (int)(g < 1 ? 1 : g);
 }
 
-int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta, const float *mean,
-                    const float *invstd, Shortcut sc, void *y, int B, int H, int W, int C, int relu, Launch s) {
+bool bn_apply_takes_partials(int prec, int C, int shortcut_mode) {
+    return prec == P_BF16 && shortcut_mode != 2 && apply_fast_ok(C, Vec16<bf16>::N) && (1024 % (2 * C)) == 0;
+}
+
+int launch_bn_apply(int prec, const void *x, const void *gamma, const void *beta, float *mean, float *invstd,
+                    Shortcut sc, void *y, int B, int H, int W, int C, int relu, Launch s, BnPartials bp) {
     const long npix = (long)B * H * W;
+    if (bp.part != nullptr && !bn_apply_takes_partials(prec, C, sc.mode)) return -1;
     if (prec == P_BF16 && sc.mode != 2 && apply_fast_ok(C, Vec16<bf16>::N)) {
         typedef bf16 T;
         constexpr int V = Vec16<T>::N;
         const long nvec = npix * (C / V);
         const int U = apply_unroll(nvec);
         const T *res = sc.mode == 1 ? (const T *)sc.a : nullptr;
-        auto k = U == 4 ? bn_apply_fast_kernel<4> : (U == 2 ? bn_apply_fast_kernel<2> : bn_apply_fast_kernel<1>);
+        auto k = U == 4 ? bn_apply_fast_kernel<4, false> : (U == 2 ? bn_apply_fast_kernel<2, false> : bn_apply_fast_kernel<1, false>);
+        if (bp.part != nullptr)
+            k = U == 4 ? bn_apply_fast_kernel<4, true> : (U == 2 ? bn_apply_fast_kernel<2, true> : bn_apply_fast_kernel<1, true>);
         launch_k(k, apply_grid(nvec, U), kThreads, 0, s, (const T *)x, (const T *)gamma, (const T *)beta, mean, invstd, res,
-                 (T *)y, nvec, C, relu);
+                 (T *)y, nvec, C, relu, bp.part, bp.n);
         return 1;
     }
     DISPATCH_PREC(prec, {
@@ -854,22 +912,35 @@ bn_bwd_apply_kernel(const T *__restrict__ dout, const T *__restrict__ out, const
 
 // Fast path for bf16 tensors, laid out like bn_apply_fast_kernel.  With gi = gamma*invstd and n pixels,
 //   dx = gi*(dz - dbeta/n - xhat*dgamma/n) = gi*dz + k1*x + k0,  k1 = -gi*invstd*dgamma/n,  k0 = -gi*dbeta/n - k1*mean.
-template <int U>
+template <int U, bool FOLD>
 __global__ void __launch_bounds__(kThreads, kApplyCtasPerSm)
 bn_bwd_apply_fast_kernel(const bf16 *__restrict__ dout, const bf16 *__restrict__ out, const bf16 *__restrict__ x,
                          const bf16 *__restrict__ gamma, const float *__restrict__ mean, const float *__restrict__ invstd,
-                         const float *__restrict__ dgamma, const float *__restrict__ dbeta, bf16 *__restrict__ dx,
-                         long nvec, long npix, int C, int relu) {
+                         float *__restrict__ dgamma, float *__restrict__ dbeta, bf16 *__restrict__ dx,
+                         long nvec, long npix, int C, int relu, const float *__restrict__ part, int n_part) {
     __shared__ float sm_gi[128], sm_k1[128], sm_k0[128];
     pdl_launch();
     pdl_wait();
+    __shared__ double sm_tot[FOLD ? 256 : 1];
+    if (FOLD) {
+        // (sum dz, sum dz * xhat) from the partial sums of the input-gradient convolution's epilogue
+        __shared__ double sm_fold[kThreads * 4];
+        fold_partials(part, n_part, 2 * C, sm_fold, sm_tot);
+    }
     for (int c = threadIdx.x; c < C; c += kThreads) {
+        float db, dg;
+        if (FOLD) {
+            db = (float)sm_tot[c]; dg = (float)sm_tot[C + c];
+            if (blockIdx.x == 0) { dbeta[c] = db; dgamma[c] = dg; }  // the parameter gradients of this batch norm
+        } else {
+            db = dbeta[c]; dg = dgamma[c];
+        }
         const float inv_n = 1.f / (float)npix;
         const float gi = to_f(gamma[c]) * invstd[c];
-        const float k1 = -gi * invstd[c] * dgamma[c] * inv_n;
+        const float k1 = -gi * invstd[c] * dg * inv_n;
         sm_gi[c] = gi;
         sm_k1[c] = k1;
-        sm_k0[c] = -gi * dbeta[c] * inv_n - k1 * mean[c];
+        sm_k0[c] = -gi * db * inv_n - k1 * mean[c];
     }
     __syncthreads();
     const int groups = C / 8;
@@ -912,16 +983,18 @@ bn_bwd_apply_fast_kernel(const bf16 *__restrict__ dout, const bf16 *__restrict__
 }
 
 int launch_bn_bwd_apply(int prec, const void *dout, const void *out, const void *x, const void *gamma,
-                        const float *mean, const float *invstd, const float *dgamma, const float *dbeta, void *dx,
-                        long npix, int C, int relu, Launch s) {
+                        const float *mean, const float *invstd, float *dgamma, float *dbeta, void *dx,
+                        long npix, int C, int relu, Launch s, BnPartials bp) {
+    if (bp.part != nullptr && !bn_apply_takes_partials(prec, C, 0)) return -1;
     if (prec == P_BF16 && apply_fast_ok(C, Vec16<bf16>::N)) {
         typedef bf16 T;
         constexpr int V = Vec16<T>::N;
         const long nvec = npix * (C / V);
         const int U = apply_unroll(nvec) >= 2 ? 2 : 1;  // three operands: two vectors of each in flight per thread
-        auto k = U == 2 ? bn_bwd_apply_fast_kernel<2> : bn_bwd_apply_fast_kernel<1>;
+        auto k = U == 2 ? bn_bwd_apply_fast_kernel<2, false> : bn_bwd_apply_fast_kernel<1, false>;
+        if (bp.part != nullptr) k = U == 2 ? bn_bwd_apply_fast_kernel<2, true> : bn_bwd_apply_fast_kernel<1, true>;
         launch_k(k, apply_grid(nvec, U), kThreads, 0, s, (const T *)dout, (const T *)out, (const T *)x, (const T *)gamma, mean,
-                 invstd, dgamma, dbeta, (T *)dx, nvec, npix, C, relu);
+                 invstd, dgamma, dbeta, (T *)dx, nvec, npix, C, relu, bp.part, bp.n);
         return 1;
     }
     DISPATCH_PREC(prec, {
