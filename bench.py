@@ -165,7 +165,7 @@ def ncu_counters():
     return out
 
 
-def dominant_kernel_roofline(torch, binding, cfg, peaks):
+def dominant_kernel_roofline(torch, binding, cfg, peaks, K):
     """The kernel with the largest share of the ncu launch list of this workload is the tensor-core convolution on the
     16-channel 32x32 maps, conv3x3_tc_kernel<16> (profiles/ddg_step_resnet110_k4_b128_bf16_launch_list.md).  It is
     timed here at the step's shape and launch configuration, with its pre-arranged filter image, as a sequence of
@@ -178,7 +178,10 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
     tflops = peaks.get("bf16_tflops", 1590.0)
     src = "measured" if "hbm_gbs" in peaks else "fallback"
 
-    def conv_case(Hh, Cc, B=B):
+    def conv_case(Hh, Cc, B=B, form="plain"):
+        """form: "plain" = the convolution alone; "stats" = with the batch-norm statistics epilogue, sums folded by the
+        CTA that finishes last (what the step launches while module streams share the GPU); "partials" = the epilogue
+        leaves per-CTA partial sums for the element-wise pass (what a single stream launches)."""
         per = 2 * B * Hh * Hh * Cc * 2                       # bytes of input + output of one launch
         n = max(8, int(400e6 // per) + 1) if B <= 1024 else max(2, int(400e6 // per) + 1)
         xs = [torch.randn(B, Hh, Hh, Cc, device="cuda").to(bf) for _ in range(n)]
@@ -186,11 +189,20 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
         w = (torch.randn(Cc, Cc, 3, 3, device="cuda") * (2.0 / (9 * Cc)) ** 0.5).to(bf)
         pk = torch.empty(binding.conv3x3_packed_bytes(B, Hh, Hh, Cc), dtype=torch.uint8, device="cuda")
         binding.conv3x3_pack(w, pk, Cc)
-        fns = [(lambda st, i=i: binding.conv3x3_packed(0, xs[i], w, pk, ys[i], B, Hh, Hh, Cc, st)) for i in range(n)]
+        m, iv = torch.empty(Cc, device="cuda"), torch.empty(Cc, device="cuda")
+        scr = torch.zeros(binding.conv3x3_fused_scratch_elems(B, Hh, Hh, Cc), device="cuda")
+        if form == "stats":
+            fns = [(lambda st, i=i: binding.conv3x3_fwd_stats_prepared(xs[i], w, pk, ys[i], m, iv, scr, B, Hh, Hh, Cc, st)) for i in range(n)]
+        elif form == "partials":
+            fns = [(lambda st, i=i: binding.conv3x3_fwd_partials(xs[i], w, pk, ys[i], scr, B, Hh, Hh, Cc, st)) for i in range(n)]
+        else:
+            fns = [(lambda st, i=i: binding.conv3x3_packed(0, xs[i], w, pk, ys[i], B, Hh, Hh, Cc, st)) for i in range(n)]
         dt = _time_back_to_back(torch, fns, s)
         return dt, per + w.numel() * 2, 2.0 * 9 * Cc * Cc * B * Hh * Hh, n
 
-    dt, alg, flops, n = conv_case(32, 16)
+    # the dominant kernel in the form the benchmarked step launches it: with its batch-norm statistics epilogue
+    step_form = "stats" if K > 1 else "partials"
+    dt, alg, flops, n = conv_case(32, 16, form=step_form)
     # DRAM traffic per launch from the ncu capture at batch 4096 (read + written; part of the output is still in L2
     # when the kernel ends); traffic grows with the pixels processed, so it is scaled by batch.  null when the kernel's
     # source has changed since the capture.
@@ -200,12 +212,22 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks):
     if c16 and c16["valid"]:
         traffic = (c16["dram_bytes_read"] + c16["dram_bytes_write"]) * B / float(c16["batch"])
     share = cnt.get("launch_list resnet110 K=4 B=128", {})
-    roof = {"kernel": "conv3x3_tc_kernel<16> (tensor-core 3x3 convolution, forward) C=16 32x32 B=%d" % B, "bound": "hbm",
+    roof = {"kernel": "conv3x3_tc_kernel<16> (tensor-core 3x3 convolution, forward, with the batch-norm statistics "
+                      "epilogue as the step launches it: %s) C=16 32x32 B=%d"
+                      % ("sums folded by the last CTA" if K > 1 else "per-CTA partial sums left to the element-wise pass", B),
+            "bound": "hbm",
             "achieved": alg / dt / 1e9, "peak": hbm, "unit": "GB/s", "frac": alg / dt / 1e9 / hbm, "traffic": traffic,
             "launch_us": dt * 1e6, "peak_source": src,
             "ncu_share_of_step": share.get("conv3x3_tc_kernel<16>") if share.get("valid") else None, "launches_timed": n,
             "tflops": flops / dt / 1e12, "tensor_frac": flops / dt / 1e12 / tflops}
     others = []
+    for form in ("plain", "stats", "partials"):
+        if form == step_form:
+            continue
+        dtc, nbytes, fl, _ = conv_case(32, 16, form=form)
+        others.append({"kernel": "conv3x3_tc_kernel<16> fwd 32x32 B=%d, %s" % (B, {"plain": "without the statistics epilogue",
+                       "stats": "statistics folded by the last CTA", "partials": "partial sums left to the element-wise pass"}[form]),
+                       "launch_us": dtc * 1e6, "hbm_gbs": nbytes / dtc / 1e9, "hbm_frac": nbytes / dtc / 1e9 / hbm})
     for (Hh, Cc) in ((16, 32), (8, 64)):
         dtc, nbytes, fl, _ = conv_case(Hh, Cc)
         others.append({"kernel": "conv3x3_tc_kernel<%d> fwd %dx%d B=%d" % (Cc, Hh, Hh, B), "launch_us": dtc * 1e6,
@@ -376,7 +398,7 @@ def main():
             peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
         except Exception:
             pass
-        roof, roof_others = dominant_kernel_roofline(torch, binding, cfg, peaks)
+        roof, roof_others = dominant_kernel_roofline(torch, binding, cfg, peaks, K)
         cpu = None
         if world == 1 and not args.skip_cpu:
             r = time_oracle(cfg, args.cpu_batch, args.cpu_steps or 20)   # ~10 s of host work

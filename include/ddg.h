@@ -233,10 +233,41 @@ ddg_status ddg_conv3x3_packed(int dgrad, const void *src, const void *w, const v
 size_t ddg_conv3x3_fused_scratch_elems(int B, int H, int W, int C);
 ddg_status ddg_conv3x3_fwd_stats(const void *x, const void *w, const void *packed, void *y, float *mean, float *invstd,
                                  float *scratch, int B, int H, int W, int C, void *stream);
+/* ddg_conv3x3_fwd_stats for a scratch whose first 128 bytes are already zero (every call of either form leaves them
+ * zero): no clearing memset in front of the kernel, so that consecutive launches chain exactly as they do inside the
+ * training step.  For timing the kernel in the form the step launches it. */
+ddg_status ddg_conv3x3_fwd_stats_prepared(const void *x, const void *w, const void *packed, void *y, float *mean,
+                                          float *invstd, float *scratch, int B, int H, int W, int C, void *stream);
 ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
                                    const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
                                    const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H,
                                    int W, int C, void *stream);
+/* The same two fused forms as a single stream launches them when it has the GPU to itself (K = 1): the convolution only
+ * leaves the per-CTA partial sums of its epilogue, part [*n_part_host][2C] fp32 (device, at least
+ * ddg_conv3x3_fused_scratch_elems floats; *n_part_host, host, receives the number of rows = CTAs of the launch), and
+ * the element-wise batch-norm pass that consumes the sums adds the rows up itself, every CTA the same rows in the same
+ * fixed order: no ticket counter and no serial tail in the convolution.
+ *   ddg_conv3x3_fwd_partials    y = conv3x3(x, w); partials of (sum y, sum y^2) over the values as stored.
+ *   ddg_bn_fwd_partials         out = [relu](gamma * (y - mean) * invstd + beta [+ res]) with mean / invstd computed from
+ *                               the partials and written to mean / invstd (fp32 [C]).
+ *   ddg_conv3x3_dgrad_partials  as ddg_conv3x3_dgrad_fused with the batch-norm sums left as partials of (sum dz,
+ *                               sum dz * xhat); bn_* must be given.
+ *   ddg_bn_bwd_partials         dx = gamma * invstd * (dz - dbeta / n - xhat * dgamma / n), dz = dout * [out > 0] (relu),
+ *                               with dbeta / dgamma computed from the partials and written out.
+ * bf16, C in {16, 32, 64} (DDG_ERR_UNSUPPORTED otherwise). */
+ddg_status ddg_conv3x3_fwd_partials(const void *x, const void *w, const void *packed, void *y, float *part,
+                                    int *n_part_host, int B, int H, int W, int C, void *stream);
+ddg_status ddg_bn_fwd_partials(const void *y, const void *gamma, const void *beta, const void *res, void *out,
+                               const float *part, int n_part, float *mean, float *invstd, int B, int HW, int C, int relu,
+                               void *stream);
+ddg_status ddg_conv3x3_dgrad_partials(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
+                                      const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
+                                      const float *bn_invstd, float *part, int *n_part_host, int B, int H, int W, int C,
+                                      void *stream);
+ddg_status ddg_bn_bwd_partials(const void *dout, const void *out, const void *x, const void *gamma, const float *mean,
+                               const float *invstd, void *dx, float *dgamma, float *dbeta, const float *part, int n_part,
+                               int B, int HW, int C, int relu, void *stream);
+
 /* ddg_conv3x3_bnrelu_fwd_stats: the second convolution of a residual block as the training step launches it.  x is the
  * RAW output of the first convolution; the kernel applies that convolution's batch norm and ReLU on its own operand
  * path, a = relu(gamma * (x - mean_in) * invstd_in + beta) rounded to bf16 (gamma, beta bf16 [C]; mean_in, invstd_in

@@ -32,7 +32,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_conv3x3_fwd_stats", "ddg_conv3x3_dgrad_fused", "ddg_conv3x3_s2_dgrad_shortcut",
            "ddg_fc_tensor_core_path", "ddg_fc_fwd", "ddg_fc_bwd", "ddg_state_bytes", "ddg_save_state",
            "ddg_load_state", "ddg_conv1x1_fwd", "ddg_conv1x1_dgrad_add", "ddg_conv1x1_wgrad_scratch_elems",
-           "ddg_conv1x1_wgrad", "ddg_conv3x3_bnrelu_fwd_stats"]
+           "ddg_conv1x1_wgrad", "ddg_conv3x3_bnrelu_fwd_stats", "ddg_conv3x3_fwd_partials",
+           "ddg_bn_fwd_partials", "ddg_conv3x3_dgrad_partials", "ddg_bn_bwd_partials", "ddg_conv3x3_fwd_stats_prepared"]
 
 
 class Layer(ctypes.Structure):
@@ -91,6 +92,11 @@ _lib.ddg_conv3x3_packed.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_conv3x3_fused_scratch_elems.argtypes = [_i] * 4
 _lib.ddg_conv3x3_fused_scratch_elems.restype = _sz
 _lib.ddg_conv3x3_fwd_stats.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
+_lib.ddg_conv3x3_fwd_stats_prepared.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
+_lib.ddg_conv3x3_fwd_partials.argtypes = [_vp] * 5 + [ctypes.POINTER(_i)] + [_i] * 4 + [_vp]
+_lib.ddg_bn_fwd_partials.argtypes = [_vp] * 6 + [_i, _vp, _vp, _i, _i, _i, _i, _vp]
+_lib.ddg_conv3x3_dgrad_partials.argtypes = [_vp] * 11 + [ctypes.POINTER(_i)] + [_i] * 4 + [_vp]
+_lib.ddg_bn_bwd_partials.argtypes = [_vp] * 10 + [_i] + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_bnrelu_fwd_stats.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_dgrad_fused.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_s2_dgrad_shortcut.argtypes = [_vp] * 5 + [_i] * 4 + [_vp]
@@ -260,6 +266,37 @@ def conv3x3_fused_scratch_elems(B, H, W, C):
 def conv3x3_fwd_stats(x, w, packed, y, mean, invstd, scratch, B, H, W, C, stream=None):
     _ok(_lib.ddg_conv3x3_fwd_stats(_ptr(x), _ptr(w), _ptr(packed), _ptr(y), _ptr(mean), _ptr(invstd), _ptr(scratch),
                                    B, H, W, C, stream))
+
+
+def conv3x3_fwd_stats_prepared(x, w, packed, y, mean, invstd, scratch, B, H, W, C, stream=None):
+    _ok(_lib.ddg_conv3x3_fwd_stats_prepared(_ptr(x), _ptr(w), _ptr(packed), _ptr(y), _ptr(mean), _ptr(invstd),
+                                            _ptr(scratch), B, H, W, C, stream))
+
+
+def conv3x3_fwd_partials(x, w, packed, y, part, B, H, W, C, stream=None):
+    """Returns the number of partial rows the launch left in `part`."""
+    n = ctypes.c_int()
+    _ok(_lib.ddg_conv3x3_fwd_partials(_ptr(x), _ptr(w), _ptr(packed), _ptr(y), _ptr(part), ctypes.byref(n), B, H, W, C, stream))
+    return n.value
+
+
+def bn_fwd_partials(y, gamma, beta, res, out, part, n_part, mean, invstd, B, HW, C, relu, stream=None):
+    _ok(_lib.ddg_bn_fwd_partials(_ptr(y), _ptr(gamma), _ptr(beta), _ptr(res), _ptr(out), _ptr(part), n_part, _ptr(mean),
+                                 _ptr(invstd), B, HW, C, int(relu), stream))
+
+
+def conv3x3_dgrad_partials(dy, w, packed, dx, res_dout, res_out, bn_mask, bn_x, bn_mean, bn_invstd, part, B, H, W, C,
+                           stream=None):
+    n = ctypes.c_int()
+    _ok(_lib.ddg_conv3x3_dgrad_partials(_ptr(dy), _ptr(w), _ptr(packed), _ptr(dx), _ptr(res_dout), _ptr(res_out),
+                                        _ptr(bn_mask), _ptr(bn_x), _ptr(bn_mean), _ptr(bn_invstd), _ptr(part),
+                                        ctypes.byref(n), B, H, W, C, stream))
+    return n.value
+
+
+def bn_bwd_partials(dout, out, x, gamma, mean, invstd, dx, dgamma, dbeta, part, n_part, B, HW, C, relu, stream=None):
+    _ok(_lib.ddg_bn_bwd_partials(_ptr(dout), _ptr(out), _ptr(x), _ptr(gamma), _ptr(mean), _ptr(invstd), _ptr(dx),
+                                 _ptr(dgamma), _ptr(dbeta), _ptr(part), n_part, B, HW, C, int(relu), stream))
 
 
 def conv3x3_bnrelu_fwd_stats(x, res, gamma, beta, mean_in, invstd_in, a_out, w, packed, y, mean, invstd, scratch, B, H, W,

@@ -125,6 +125,71 @@ ddg_status ddg_conv3x3_fwd_stats(const void *x, const void *w, const void *packe
     return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, s, bf));
 }
 
+ddg_status ddg_conv3x3_fwd_stats_prepared(const void *x, const void *w, const void *packed, void *y, float *mean,
+                                          float *invstd, float *scratch, int B, int H, int W, int C, void *stream) {
+    if (!x || !w || !y || !mean || !invstd || !scratch) return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_supported(B, H, W, C, C, 1)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    BnFuse bf;
+    bf.counter = reinterpret_cast<unsigned *>(scratch); bf.part = scratch + 32; bf.o0 = mean; bf.o1 = invstd;
+    return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, (cudaStream_t)stream, bf));
+}
+
+ddg_status ddg_conv3x3_fwd_partials(const void *x, const void *w, const void *packed, void *y, float *part,
+                                    int *n_part_host, int B, int H, int W, int C, void *stream) {
+    if (!x || !w || !y || !part || !n_part_host) return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_supported(B, H, W, C, C, 1)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    BnFuse bf;
+    bf.part = part; bf.n_part_out = n_part_host;
+    return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, (cudaStream_t)stream, bf));
+}
+
+ddg_status ddg_bn_fwd_partials(const void *y, const void *gamma, const void *beta, const void *res, void *out,
+                               const float *part, int n_part, float *mean, float *invstd, int B, int HW, int C, int relu,
+                               void *stream) {
+    if (!y || !gamma || !beta || !out || !part || n_part < 1 || !mean || !invstd) return DDG_ERR_INVALID_ARG;
+    if (B < 1 || HW < 1 || !bn_apply_takes_partials(DDG_BF16, C, res ? 1 : 0)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    Shortcut sc{};
+    if (res) { sc.mode = 1; sc.a = res; }
+    BnPartials bp;
+    bp.part = part; bp.n = n_part;
+    return done(launch_bn_apply(DDG_BF16, y, gamma, beta, mean, invstd, sc, out, B, HW, 1, C, relu, (cudaStream_t)stream, bp));
+}
+
+ddg_status ddg_conv3x3_dgrad_partials(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
+                                      const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
+                                      const float *bn_invstd, float *part, int *n_part_host, int B, int H, int W, int C,
+                                      void *stream) {
+    if (!dy || !w || !dx || !bn_mask || !bn_x || !bn_mean || !bn_invstd || !part || !n_part_host) return DDG_ERR_INVALID_ARG;
+    if ((res_dout == nullptr) != (res_out == nullptr)) return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_supported(B, H, W, C, C, 1)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    Shortcut sc{};
+    if (res_dout) { sc.mode = 1; sc.a = res_dout; sc.b = res_out; }
+    BnFuse bf;
+    bf.part = part; bf.n_part_out = n_part_host;
+    bf.mask = bn_mask; bf.x = bn_x; bf.mean = bn_mean; bf.invstd = bn_invstd;
+    return done(launch_conv_tc(1, dy, w, packed, dx, B, H, W, C, sc, (cudaStream_t)stream, bf));
+}
+
+ddg_status ddg_bn_bwd_partials(const void *dout, const void *out, const void *x, const void *gamma, const float *mean,
+                               const float *invstd, void *dx, float *dgamma, float *dbeta, const float *part, int n_part,
+                               int B, int HW, int C, int relu, void *stream) {
+    if (!dout || !x || !gamma || !mean || !invstd || !dx || !dgamma || !dbeta || !part || n_part < 1 || (relu && !out))
+        return DDG_ERR_INVALID_ARG;
+    if (B < 1 || HW < 1 || !bn_apply_takes_partials(DDG_BF16, C, 0)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    BnPartials bp;
+    bp.part = part; bp.n = n_part;
+    return done(launch_bn_bwd_apply(DDG_BF16, dout, out, x, gamma, mean, invstd, dgamma, dbeta, dx, (long)B * HW, C, relu,
+                                    (cudaStream_t)stream, bp));
+}
+
 ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *res, const void *gamma, const void *beta,
                                         const float *mean_in, const float *invstd_in, void *a_out, const void *w,
                                         const void *packed, void *y,

@@ -483,3 +483,59 @@ def test_conv_forward_with_batch_norm_relu_on_its_operand_path(shape, with_res):
     check_map(from_dev(y), y_ref, 1, "forward of the transformed input", max(1, 128 // W))
     _, ms, iss = orc.bn_forward(from_dev(y), np.ones(C), np.zeros(C))
     assert rel(mean.cpu().numpy(), ms) < 2e-5 and rel(invstd.cpu().numpy(), iss) < 2e-5
+
+
+@pytest.mark.parametrize("shape", [(3, 32, 32, 16), (5, 16, 16, 32), (128, 8, 8, 64), (2, 8, 8, 16), (128, 32, 32, 16),
+                                   (301, 32, 32, 16), (231, 16, 16, 32), (902, 8, 8, 64)], ids=lambda s: "x".join(map(str, s)))
+def test_partial_sums_folded_by_the_consuming_pass(shape):
+    """The form a single stream launches: the convolutions leave per-CTA partial sums and the element-wise batch-norm
+    passes add them up.  Forward: conv -> batch norm (+ residual, ReLU); backward: input-gradient convolution with the
+    two batch-norm sums -> batch-norm backward.  Against the oracle's primitives, statistics and sums teacher-forced on
+    the tensors the GPU stored; and against the other form (sums folded by the convolution's last CTA)."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = shape
+    rng = np.random.default_rng(43)
+    x, xh = to_dev(rng.standard_normal((B, C, H, W)) * 1.2 + 0.1, 1)
+    w, wh = _filter(rng, C)
+    r, rh = to_dev(rng.standard_normal((B, C, H, W)), 1)
+    gamma = torch.from_numpy(1 + 0.2 * rng.standard_normal(C)).to(torch.bfloat16)
+    beta = torch.from_numpy(0.2 * rng.standard_normal(C)).to(torch.bfloat16)
+    gh, bh = gamma.to(torch.float64).numpy(), beta.to(torch.float64).numpy()
+    y, out = torch.empty_like(x), torch.empty_like(x)
+    mean, invstd, mean2, invstd2 = (torch.full((C,), 7.0, dtype=torch.float32, device="cuda") for _ in range(4))
+    part = torch.full((binding.conv3x3_fused_scratch_elems(B, H, W, C),), 3.0, dtype=torch.float32, device="cuda")
+    n_part = binding.conv3x3_fwd_partials(x, w, None, y, part, B, H, W, C)
+    assert 1 <= n_part <= 148
+    binding.bn_fwd_partials(y, gamma.cuda(), beta.cuda(), r, out, part, n_part, mean, invstd, B, H * W, C, 1)
+    torch.cuda.synchronize()
+    check_map(from_dev(y), orc.conv3x3_forward(xh, wh, 1), 1, "forward", max(1, 128 // W))
+    o_ref, m_ref, is_ref = orc.bn_forward(from_dev(y), gh, bh)
+    assert rel(mean.cpu().numpy(), m_ref) < 2e-5 and rel(invstd.cpu().numpy(), is_ref) < 2e-5
+    o_ref = np.maximum(o_ref + rh, 0)
+    assert rel(from_dev(out), o_ref) < TOL[1]
+    ok, idx, excess = elementwise_ok(from_dev(out), o_ref, RTOL[1], 2e-3 * float(np.sqrt(np.mean(o_ref ** 2))))
+    assert ok, "batch-norm output from partials: element %r off by %.3e" % (idx, excess)
+    # the other form of the same launch pair: statistics folded by the convolution's last CTA
+    scratch = torch.zeros(binding.conv3x3_fused_scratch_elems(B, H, W, C), dtype=torch.float32, device="cuda")
+    y2 = torch.empty_like(x)
+    binding.conv3x3_fwd_stats(x, w, None, y2, mean2, invstd2, scratch, B, H, W, C)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+    assert rel(mean.cpu().numpy(), mean2.cpu().numpy()) < 1e-6 and rel(invstd.cpu().numpy(), invstd2.cpu().numpy()) < 1e-6
+    # backward
+    dy, dyh = to_dev(rng.standard_normal((B, C, H, W)), 1)
+    mask, maskh = to_dev(np.maximum(rng.standard_normal((B, C, H, W)), 0), 1)
+    bx, bxh = to_dev(rng.standard_normal((B, C, H, W)) * 1.5 + 0.3, 1)
+    _, mb, isb = orc.bn_forward(bxh, np.ones(C), np.zeros(C))
+    mbd, isbd = torch.from_numpy(mb.astype(np.float32)).cuda(), torch.from_numpy(isb.astype(np.float32)).cuda()
+    dx, dxx = torch.empty_like(x), torch.empty_like(x)
+    dg, db = (torch.full((C,), 7.0, dtype=torch.float32, device="cuda") for _ in range(2))
+    n_part = binding.conv3x3_dgrad_partials(dy, w, None, dx, None, None, mask, bx, mbd, isbd, part, B, H, W, C)
+    binding.bn_bwd_partials(dx, mask, bx, gamma.cuda(), mbd, isbd, dxx, dg, db, part, n_part, B, H * W, C, 1)
+    torch.cuda.synchronize()
+    check_map(from_dev(dx), orc.conv3x3_backward(np.zeros_like(dyh), wh, dyh, 1)[0], 1, "input gradient", max(1, 128 // W))
+    dz = from_dev(dx) * (maskh > 0)
+    dxx_ref, dg_ref, db_ref = orc.bn_backward(bxh, mbd.double().cpu().numpy(), isbd.double().cpu().numpy(), gh, dz)
+    scale = float(np.sqrt(np.mean(dz ** 2)) * np.sqrt(B * H * W))
+    assert np.max(np.abs(db.cpu().numpy() - db_ref)) < 2e-5 * scale and np.max(np.abs(dg.cpu().numpy() - dg_ref)) < 4e-5 * scale
+    assert rel(from_dev(dxx), dxx_ref) < TOL[1]
