@@ -71,6 +71,43 @@ __device__ __forceinline__ float warp_max(float v) {
     return v;
 }
 
+// Totals of n_part rows of nval = 2C per-CTA partial sums, by the first THREADS threads of a CTA (all threads of the CTA must call), in a fixed order: the
+// rows are read as one flat array of 16-byte vectors (THREADS * 4 values per pass is a multiple of nval, so a thread
+// always meets the same four columns), up to eight independent loads in flight per thread, accumulated in double in
+// pass order; the threads that share a column are then added in index order.  Result: tot[0..nval) in shared memory.
+// fold: THREADS * 4 doubles of shared memory.  The convolution's last CTA and the element-wise passes use the same routine
+// with the same THREADS, so both ways of folding give the same bits.
+template <int THREADS>
+__device__ __forceinline__ void fold_partials(const float *__restrict__ part, int n_part, int nval, double *fold, double *tot) {
+    const int t = threadIdx.x;
+    const int total4 = n_part * nval / 4;
+    if (t < THREADS) {
+        double a[4] = {0.0, 0.0, 0.0, 0.0};
+        const float4 *p4 = reinterpret_cast<const float4 *>(part);
+        for (int i0 = t; i0 < total4; i0 += 8 * THREADS) {
+            float4 q[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * THREADS;
+                q[u] = i < total4 ? __ldcg(p4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { a[0] += (double)q[u].x; a[1] += (double)q[u].y; a[2] += (double)q[u].z; a[3] += (double)q[u].w; }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) fold[t * 4 + j] = a[j];
+    }
+    __syncthreads();
+    if (t < nval) {
+        // column t lives in the threads whose first vector covers it: thread (t / 4) + k * (nval / 4), element t % 4
+        double sum = 0.0;
+        for (int k = t / 4; k < THREADS; k += nval / 4) sum += fold[k * 4 + (t & 3)];
+        tot[t] = sum;
+    }
+    __syncthreads();
+}
+
+
 static inline int ceil_div(long a, long b) { return (int)((a + b - 1) / b); }
 
 // Programmatic dependent launch.  A kernel launched with programmatic stream serialisation may be scheduled while the

@@ -526,41 +526,28 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
         stat_part[(size_t)blockIdx.x * 2 * C + threadIdx.x] = t;
     }
     if (stat_counter == nullptr) return;  // the kernel that consumes the sums folds the partials itself
-    __threadfence();
-    __syncthreads();
+    __syncthreads();  // the partial stores above are ordered before thread 0's release below by this barrier
     int *is_last = reinterpret_cast<int *>(sm_stat);  // free again: the epilogue is over
-    if (threadIdx.x == 0) *is_last = (atomicAdd(stat_counter, 1u) == gridDim.x - 1) ? 1 : 0;
+    if (threadIdx.x == 0) {
+        unsigned old;
+        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(stat_counter) : "memory");
+        *is_last = (old == gridDim.x - 1) ? 1 : 0;
+    }
     __syncthreads();
     if (!*is_last) return;
-    __threadfence();
-    // last CTA: partials of all CTAs, `ways` threads per value, eight loads in flight per thread, fixed order
-    double *fold = reinterpret_cast<double *>(&sm_run[0][0][0]);  // one double per thread fits the 8 KB
-    constexpr int nval = 2 * C;
-    const int ways = (int)blockDim.x / nval;
-    const int v = threadIdx.x % nval, way = threadIdx.x / nval;
-    double acc = 0.0;
-    if (way < ways) {
-        double a8[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
-        unsigned i = way;
-        for (; i + 7 * ways < gridDim.x; i += 8 * ways) {
-#pragma unroll
-            for (int u = 0; u < 8; ++u) a8[u] += (double)__ldcg(stat_part + (size_t)(i + u * ways) * nval + v);
-        }
-        for (; i < gridDim.x; i += ways) a8[0] += (double)__ldcg(stat_part + (size_t)i * nval + v);
-        acc = ((a8[0] + a8[1]) + (a8[2] + a8[3])) + ((a8[4] + a8[5]) + (a8[6] + a8[7]));
-    }
-    fold[threadIdx.x] = acc;
-    __syncthreads();
+    // last CTA: the partials of all CTAs, added up exactly as the element-wise passes do it (same routine, 256 threads)
+    double *fold = reinterpret_cast<double *>(&sm_run[0][0][0]);  // 256 x 4 doubles = the 8 KB of the per-warp sums
+    double *tot = reinterpret_cast<double *>(smem + plan.a_off);     // the stage ring is idle by now
+    fold_partials<256>(stat_part, (int)gridDim.x, 2 * C, fold, tot);
     if (threadIdx.x < C) {
         const int c = threadIdx.x;
-        double a = 0.0, b = 0.0;
-        for (int wy = 0; wy < ways; ++wy) { a += fold[wy * nval + c]; b += fold[wy * nval + C + c]; }
+        const double a = tot[c], b = tot[C + c];
         if (bn_x == nullptr) {
             const double npix = (double)n_tiles * kTileM;
             double m = a / npix, var = b / npix - m * m;
             if (var < 0.0) var = 0.0;
             stat_o0[c] = (float)m;
-            stat_o1[c] = (float)(1.0 / sqrt(var + 1e-5));
+            stat_o1[c] = (float)(1.0 / sqrt(var + (double)1e-5f));  // the element-wise passes' constant, bit for bit
         } else {
             stat_o0[c] = (float)a;
             stat_o1[c] = (float)b;

@@ -721,38 +721,6 @@ bn_apply_kernel(const T *__restrict__ x, const T *__restrict__ gamma, const T *_
 // capped at three CTAs per SM.
 static constexpr int kApplyCtasPerSm = 3;
 
-// Totals of n_part rows of nval = 2C per-CTA partial sums, by a whole CTA of kThreads threads, in a fixed order: the
-// rows are read as one flat array of 16-byte vectors (kThreads * 4 values per pass is a multiple of nval, so a thread
-// always meets the same four columns), up to eight independent loads in flight per thread, accumulated in double in
-// pass order; the threads that share a column are then added in index order.  Result: tot[0..nval) in shared memory.
-// fold: kThreads * 4 doubles of shared memory.
-__device__ __forceinline__ void fold_partials(const float *__restrict__ part, int n_part, int nval, double *fold, double *tot) {
-    const int t = threadIdx.x;
-    const int total4 = n_part * nval / 4;
-    double a[4] = {0.0, 0.0, 0.0, 0.0};
-    const float4 *p4 = reinterpret_cast<const float4 *>(part);
-    for (int i0 = t; i0 < total4; i0 += 8 * kThreads) {
-        float4 q[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i = i0 + u * kThreads;
-            q[u] = i < total4 ? __ldcg(p4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) { a[0] += (double)q[u].x; a[1] += (double)q[u].y; a[2] += (double)q[u].z; a[3] += (double)q[u].w; }
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) fold[t * 4 + j] = a[j];
-    __syncthreads();
-    if (t < nval) {
-        // column t lives in the threads whose first vector covers it: thread (t / 4) + k * (nval / 4), element t % 4
-        double sum = 0.0;
-        for (int k = t / 4; k < kThreads; k += nval / 4) sum += fold[k * 4 + (t & 3)];
-        tot[t] = sum;
-    }
-    __syncthreads();
-}
-
 // FOLD: the statistics come as per-CTA partial sums that this kernel adds up first (an instantiation of its own: the
 // 10 KB of shared memory the fold needs would otherwise sit in every launch and keep other streams' CTAs off the SM)
 template <int U, bool FOLD>
@@ -766,7 +734,7 @@ bn_apply_fast_kernel(const bf16 *__restrict__ x, const bf16 *__restrict__ gamma,
     if (FOLD) {
         // statistics from the convolution epilogue's partial sums (sum x, sum x^2): every CTA folds them the same way
         __shared__ double sm_fold[kThreads * 4], sm_tot[256];
-        fold_partials(part, n_part, 2 * C, sm_fold, sm_tot);
+        fold_partials<kThreads>(part, n_part, 2 * C, sm_fold, sm_tot);
         const double npix = (double)(nvec / (C / 8));
         for (int c = threadIdx.x; c < C; c += kThreads) {
             const double m = sm_tot[c] / npix;
@@ -925,7 +893,7 @@ bn_bwd_apply_fast_kernel(const bf16 *__restrict__ dout, const bf16 *__restrict__
     if (FOLD) {
         // (sum dz, sum dz * xhat) from the partial sums of the input-gradient convolution's epilogue
         __shared__ double sm_fold[kThreads * 4];
-        fold_partials(part, n_part, 2 * C, sm_fold, sm_tot);
+        fold_partials<kThreads>(part, n_part, 2 * C, sm_fold, sm_tot);
     }
     for (int c = threadIdx.x; c < C; c += kThreads) {
         float db, dg;

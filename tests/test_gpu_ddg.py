@@ -270,6 +270,14 @@ def test_batch_norm_pass_on_the_operand_path_gives_the_same_bits():
     assert la == lb == lc and np.array_equal(wa, wb) and np.array_equal(wa, wc)
 
 
+def test_both_places_of_folding_the_batch_norm_sums_give_the_same_bits():
+    """bn_fold = 1 (the convolution's last CTA) and 2 (the consuming element-wise pass) run the same folding routine on
+    the same partials: identical losses and weights."""
+    wa, la, _ = _resnet20_k3_bf16_run(bn_fold=1)
+    wb, lb, _ = _resnet20_k3_bf16_run(bn_fold=2)
+    assert la == lb and np.array_equal(wa, wb)
+
+
 def test_launch_overlap_settings_give_the_same_bits():
     """The programmatic-launch policy only moves kernels in time: never / library policy / every kernel must produce
     identical weights (fixed summation orders everywhere)."""

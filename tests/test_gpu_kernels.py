@@ -521,7 +521,7 @@ def test_partial_sums_folded_by_the_consuming_pass(shape):
     binding.conv3x3_fwd_stats(x, w, None, y2, mean2, invstd2, scratch, B, H, W, C)
     torch.cuda.synchronize()
     assert torch.equal(y, y2)
-    assert rel(mean.cpu().numpy(), mean2.cpu().numpy()) < 1e-6 and rel(invstd.cpu().numpy(), invstd2.cpu().numpy()) < 1e-6
+    assert torch.equal(mean, mean2) and torch.equal(invstd, invstd2)      # one folding routine, two places: same bits
     # backward
     dy, dyh = to_dev(rng.standard_normal((B, C, H, W)), 1)
     mask, maskh = to_dev(np.maximum(rng.standard_normal((B, C, H, W)), 0), 1)
