@@ -272,10 +272,17 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
             int ls = 0;
             uint32_t ph = 0;
             bool ok = true;
-            for (int tile = blockIdx.x + g * gridDim.x; tile < n_tiles && ok; tile += tile_step) {
+            // tile -> (first image, first row): divided once, then stepped (an integer division per tile is a hundred
+            // cycles of this thread's chain)
+            const int tile0 = blockIdx.x + g * gridDim.x;
+            const int step_n = tile_step / tiles_per_img, step_t = tile_step % tiles_per_img;
+            int n_img = tile0 / tiles_per_img, t_img = tile0 % tiles_per_img;
+            for (int tile = tile0; tile < n_tiles && ok; tile += tile_step) {
                 int n0, h0;
                 if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }  // a tile spans whole images
-                else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
+                else { n0 = n_img; h0 = t_img * rows_per_tile; }
+                n_img += step_n; t_img += step_t;
+                if (t_img >= tiles_per_img) { t_img -= tiles_per_img; ++n_img; }
                 for (int j = 0; j < loads_per_tile && ok; ++j) {
                     const int s = g * ring + ls;
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, wt, 1);
@@ -301,10 +308,11 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
             uint32_t ph = 0;
             bool ok = true;
             if (w_packed != nullptr) ok = mbar_wait(w_bar, 0, wt, 5);
+            int acc_i = 0;        // it % n_acc and the parity of it / n_acc, stepped instead of divided
+            uint32_t aph = 0;
             for (int tile = blockIdx.x + g * gridDim.x; tile < n_tiles && ok; tile += tile_step, ++it) {
                 // the pipeline's accumulators in turn
-                const int a = g * plan_e.n_acc + it % plan_e.n_acc;
-                const uint32_t aph = (uint32_t)(it / plan_e.n_acc) & 1u;
+                const int a = g * plan_e.n_acc + acc_i;
                 ok = mbar_wait(tempty_bar(a), aph ^ 1u, wt, 2);
                 if (!ok) break;
                 tc_fence_after();
@@ -328,6 +336,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
                     if (++ls == ring) { ls = 0; ph ^= 1u; }
                 }
                 if (ok) tc_commit(tfull_bar(a));
+                if (++acc_i == plan_e.n_acc) { acc_i = 0; aph ^= 1u; }
             }
         }
     } else if (xform && warp >= 2 * n_pipes + 4 * n_epi_groups) {
@@ -420,11 +429,17 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
         constexpr int kChunks = C / 16;
         const int c_begin = 16 * (share * kChunks / plan_e.split), c_end = 16 * ((share + 1) * kChunks / plan_e.split);
         bool ok = pipe < n_pipes;  // a group the plan has no work for leaves at once
-        for (int it = slot; ok; it += plan_e.n_slots) {
-            const int tile = blockIdx.x + pipe * gridDim.x + it * tile_step;
+        const int wcol = lane % W;  // W divides 32: a warp holds whole image rows
+        int acc_i = slot % plan_e.n_acc;                       // it % n_acc and the parity of it / n_acc, stepped
+        uint32_t aph = (uint32_t)(slot / plan_e.n_acc) & 1u;
+        int tile = blockIdx.x + pipe * gridDim.x + slot * tile_step;
+        const int tile_stride = plan_e.n_slots * tile_step;
+        for (; ok; tile += tile_stride) {
             if (tile >= n_tiles) break;
-            const int a = pipe * plan_e.n_acc + it % plan_e.n_acc;
-            const uint32_t aph = (uint32_t)(it / plan_e.n_acc) & 1u;
+            const int a = pipe * plan_e.n_acc + acc_i;
+            const uint32_t aph_now = aph;
+            acc_i += plan_e.n_slots;
+            while (acc_i >= plan_e.n_acc) { acc_i -= plan_e.n_acc; aph ^= 1u; }
             const size_t pix = (size_t)tile * kTileM + 32 * q + lane;
             // what the epilogue reads from global memory for this pixel (shortcut gradient, batch-norm mask and input) was
             // written long ago: start fetching it now, under the TMA and MMA latency of the tile
@@ -442,11 +457,10 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
                     prefetch_l1(reinterpret_cast<const char *>(bn_x + pix * C) + o);
                 }
             }
-            ok = mbar_wait(tfull_bar(a), aph, wt, 4);
+            ok = mbar_wait(tfull_bar(a), aph_now, wt, 4);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int wcol = lane % W;  // W divides 32: a warp holds whole image rows
             const uint32_t t_row = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * 3 * C);
 #pragma unroll 1
             for (int c0 = c_begin; c0 < c_end; c0 += 16) {
@@ -623,10 +637,12 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
+            int n_img = t0 / tiles_per_img, t_img = t0 % tiles_per_img;  // divided once, then stepped
             for (int tile = t0; tile < t1 && ok; ++tile) {
                 int n0, h0;
                 if (imgs_per_tile > 1) { n0 = tile * imgs_per_tile; h0 = 0; }
-                else { n0 = tile / tiles_per_img; h0 = (tile % tiles_per_img) * rows_per_tile; }
+                else { n0 = n_img; h0 = t_img * rows_per_tile; }
+                if (++t_img == tiles_per_img) { t_img = 0; ++n_img; }
                 ok = mbar_wait(empty_bar(s), ph ^ 1u, wt, 11);
                 if (!ok) break;
                 const uint32_t st = base + s * stage_bytes;
