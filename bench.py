@@ -390,6 +390,29 @@ def main():
               "what": "the same network, kernels and batches with K = 1 (plain backpropagation)"}
         net1.destroy()
 
+    # ---- where the iteration's time sits: device time of each module's forward piece and backward + update piece
+    # (the quantities of the method's cost model: forward sweeps in sequence, backward sweeps side by side), from a
+    # short run of its own with the piece timer on, outside every timed region ----
+    pieces = None
+    if rank == 0 and not args.skip_k1:
+        netp = binding.Ddg(cfg["layers"], cfg["split_after"], cfg["batch"], cfg["in_shape"], cfg["num_classes"],
+                           precision=cfg["precision"], lr=o["lr"], momentum=o["momentum"], weight_decay=o["weight_decay"],
+                           use_graph=not args.no_graph, streams=[s.cuda_stream for s in streams],
+                           fuse_bn_apply=args.fuse_bn_apply, bn_fold=args.bn_fold, time_pieces=True)
+        netp.set_weights(synth.init_weights(cfg["layers"]))
+        fs, bs = [], []
+        for t in range(warm + 9):
+            netp.step(*dev[t % n_batches], want_loss=False)
+            if t >= warm:
+                f, b = netp.piece_times()
+                fs.append(f)
+                bs.append(b)
+        netp.destroy()
+        pieces = {"fwd_ms": [round(float(v), 4) for v in np.median(np.array(fs), axis=0)],
+                  "bwd_upd_ms": [round(float(v), 4) for v in np.median(np.array(bs), axis=0)],
+                  "what": "median device time per module of F_k and of B_k + U_k over 9 iterations run one at a time "
+                          "(each drained before the next: no overlap between iterations, unlike the timed region)"}
+
     dt, dt_e2e = max_over_ranks([dt, dt_e2e], dist, "cuda")
 
     if rank == 0:
@@ -416,7 +439,7 @@ def main():
                "launches_per_step": int(launches_per_step),
                "e2e": {"value": job_throughput(cfg["batch"], n_e2e, world, dt_e2e), "unit": "images/s",
                        "h2d_bytes_per_step": x_bytes + cfg["batch"] * 4, "d2h_bytes_per_step": 4, "steps": n_e2e},
-               "k1_baseline": k1, "roofline": roof, "roofline_others": roof_others, "cpu_baseline": cpu}
+               "k1_baseline": k1, "pieces": pieces, "roofline": roof, "roofline_others": roof_others, "cpu_baseline": cpu}
         if k1:
             out["k1_baseline"]["speedup_of_ddg"] = out["value"] / k1["value"]
         print(json.dumps(out))

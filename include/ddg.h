@@ -114,6 +114,8 @@ typedef struct {
     int launch_overlap; /* programmatic dependent launch (the next kernel of a stream is placed while the previous one
                        still runs).  0 (default): the library's policy: every kernel when K = 1; with several module
                        streams only the forward / input-gradient convolutions.  1: never.  2: every kernel. */
+    int time_pieces; /* 1: bracket each module's forward sweep and its backward sweep + update with timing events on
+                       the module's stream (two extra event records per piece), read back by ddg_piece_times. */
 } ddg_cfg;
 
 /* Build a context: validates the network (Section 2: L layers; Section 3: K groups of consecutive layers,
@@ -158,6 +160,14 @@ ddg_status ddg_get_loss_dev(ddg_ctx *ctx, const float **loss_dev);
 
 /* Number of the library's kernel launches the last ddg_step issued (graph replays count their kernel nodes). */
 ddg_status ddg_last_step_launches(const ddg_ctx *ctx, long *launches);
+
+/* Device time of the pieces of the last iteration (contexts created with time_pieces): fwd_ms[k] = the forward sweep
+ * of module k+1 (Eq. 3 over G(k+1)), bwd_ms[k] = its backward sweep and update (Eq. 6-9), each from the moment the
+ * piece's first kernel could start on the module's stream to the end of its last, in milliseconds; the pieces of
+ * different modules overlap in time and share the GPU, which is what the method's cost model (forward in sequence,
+ * backward sweeps side by side) is about.  Host arrays of K floats; waits for the K streams.  Each piece is also an
+ * NVTX range ("F1", "B1+U1", ...) for a timeline tool. */
+ddg_status ddg_piece_times(ddg_ctx *ctx, float *fwd_ms, float *bwd_ms);
 
 /* Wait for all K streams; surfaces deferred device-side errors. */
 ddg_status ddg_sync(ddg_ctx *ctx);

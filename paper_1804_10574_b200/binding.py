@@ -33,7 +33,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_fc_tensor_core_path", "ddg_fc_fwd", "ddg_fc_bwd", "ddg_state_bytes", "ddg_save_state",
            "ddg_load_state", "ddg_conv1x1_fwd", "ddg_conv1x1_dgrad_add", "ddg_conv1x1_wgrad_scratch_elems",
            "ddg_conv1x1_wgrad", "ddg_conv3x3_bnrelu_fwd_stats", "ddg_conv3x3_fwd_partials",
-           "ddg_bn_fwd_partials", "ddg_conv3x3_dgrad_partials", "ddg_bn_bwd_partials", "ddg_conv3x3_fwd_stats_prepared"]
+           "ddg_bn_fwd_partials", "ddg_conv3x3_dgrad_partials", "ddg_bn_bwd_partials", "ddg_conv3x3_fwd_stats_prepared",
+           "ddg_piece_times"]
 
 
 class Layer(ctypes.Structure):
@@ -50,7 +51,8 @@ class Cfg(ctypes.Structure):
                 ("in_w", ctypes.c_int), ("num_classes", ctypes.c_int), ("seed", ctypes.c_ulonglong),
                 ("use_graph", ctypes.c_int), ("debug_checks", ctypes.c_int),
                 ("streams", ctypes.POINTER(ctypes.c_void_p)), ("separate_bn_sums", ctypes.c_int),
-                ("fuse_bn_apply", ctypes.c_int), ("bn_fold", ctypes.c_int), ("launch_overlap", ctypes.c_int)]
+                ("fuse_bn_apply", ctypes.c_int), ("bn_fold", ctypes.c_int), ("launch_overlap", ctypes.c_int),
+                ("time_pieces", ctypes.c_int)]
 
 
 _vp, _i, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -59,6 +61,7 @@ _lib.ddg_create.argtypes = [ctypes.POINTER(Layer), _i, ctypes.POINTER(_i), _i, c
 _lib.ddg_step.argtypes = [_vp, _vp, _vp, ctypes.POINTER(_f)]
 _lib.ddg_step_host.argtypes = [_vp, _vp, _vp, ctypes.POINTER(_f)]
 _lib.ddg_set_lr.argtypes = [_vp, _f]
+_lib.ddg_piece_times.argtypes = [_vp, ctypes.POINTER(_f), ctypes.POINTER(_f)]
 _lib.ddg_param_count.argtypes = [_vp, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
 _lib.ddg_get_weights.argtypes = [_vp, _vp, _sz, _i]
 _lib.ddg_set_weights.argtypes = [_vp, _vp, _sz, _i]
@@ -141,7 +144,7 @@ class Ddg:
     def __init__(self, layers, split_after, batch, in_shape, num_classes, precision="fp32", opt="sgd", lr=0.01,
                  momentum=0.0, weight_decay=0.0, beta1=0.9, beta2=0.999, eps=1e-8, seed=0, use_graph=False,
                  debug_checks=False, streams=None, separate_bn_sums=False, fuse_bn_apply=0, bn_fold=0,
-                 launch_overlap=0):
+                 launch_overlap=0, time_pieces=False):
         arr = (Layer * len(layers))(*[Layer(*map(int, l)) for l in layers])
         K = len(split_after) + 1
         sp = (ctypes.c_int * max(1, K - 1))(*split_after)
@@ -152,7 +155,7 @@ class Ddg:
             st = (ctypes.c_void_p * K)(*[int(s) for s in streams])
         cfg = Cfg(BF16 if precision == "bf16" else FP32, batch, in_shape[0], in_shape[1], in_shape[2], num_classes,
                   seed, int(use_graph), int(debug_checks), st, int(separate_bn_sums), int(fuse_bn_apply), int(bn_fold),
-                  int(launch_overlap))
+                  int(launch_overlap), int(time_pieces))
         h = ctypes.c_void_p()
         rc = _lib.ddg_create(arr, len(layers), sp, K, ctypes.byref(o), ctypes.byref(cfg), ctypes.byref(h))
         if rc != 0:
@@ -214,6 +217,12 @@ class Ddg:
         n = ctypes.c_long()
         self._check(_lib.ddg_last_step_launches(self._h, ctypes.byref(n)))
         return n.value
+
+    def piece_times(self):
+        """(forward ms per module, backward + update ms per module) of the last iteration; needs time_pieces."""
+        f, b = (ctypes.c_float * self.K)(), (ctypes.c_float * self.K)()
+        self._check(_lib.ddg_piece_times(self._h, f, b))
+        return list(f), list(b)
 
     def sync(self):
         self._check(_lib.ddg_sync(self._h))

@@ -11,6 +11,8 @@
 #include <string>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/ddg.h"
 #include "common.cuh"
 #include "conv_tc.h"
@@ -62,6 +64,7 @@ struct Module {
     cudaStream_t stream = nullptr;
     bool own_stream = false;
     cudaEvent_t ev_fwd = nullptr, ev_bwd = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_time[4] = {nullptr, nullptr, nullptr, nullptr};  // time_pieces: forward begin / end, backward begin / end
     // weight gradients run beside the error-gradient chain, on a second stream of the module
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_side[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -672,6 +675,27 @@ ddg_status run_segment(ddg_ctx *ctx, int k, int seg, long t, bool use_graph, lon
     return DDG_OK;
 }
 
+// A piece as a timeline tool and the piece timer see it: an NVTX range on the enqueuing thread ("F2", "B2+U2") and,
+// in contexts created with time_pieces, a timing event on the module's stream on either side.
+struct PieceRange {
+    ddg_ctx *ctx;
+    Module &m;
+    const int seg;
+    bool open = true;
+    PieceRange(ddg_ctx *c, int k, int s) : ctx(c), m(c->mods[k]), seg(s) {
+        char name[24];
+        snprintf(name, sizeof name, seg == 0 ? "F%d" : "B%d+U%d", k + 1, k + 1);
+        nvtxRangePushA(name);
+        if (m.ev_time[0]) cudaEventRecord(m.ev_time[2 * seg], m.stream);
+    }
+    cudaError_t close() {
+        open = false;
+        nvtxRangePop();
+        return m.ev_time[0] ? cudaEventRecord(m.ev_time[2 * seg + 1], m.stream) : cudaSuccess;
+    }
+    ~PieceRange() { if (open) nvtxRangePop(); }
+};
+
 // Enqueue one whole iteration on the K streams.
 ddg_status enqueue_iteration(ddg_ctx *ctx, long t, bool use_graph, long *launches) {
     const int K = ctx->K;
@@ -680,9 +704,11 @@ ddg_status enqueue_iteration(ddg_ctx *ctx, long t, bool use_graph, long *launche
     for (int k = 0; k < K; ++k) {
         Module &m = ctx->mods[k];
         if (k > 0) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k - 1].ev_fwd, 0));
+        PieceRange range(ctx, k, 0);
         ddg_status st = run_segment(ctx, k, 0, t, use_graph, &n);
         if (st != DDG_OK) return st;
         total += n;
+        if (range.close() != cudaSuccess) return DDG_ERR_CUDA;
         CU(cudaEventRecord(m.ev_fwd, m.stream));  // for module k+1; the last module's marks the loss
     }
     // backward sweeps and updates: independent across modules within the iteration ("for k in parallel").  Ascending
@@ -691,9 +717,11 @@ ddg_status enqueue_iteration(ddg_ctx *ctx, long t, bool use_graph, long *launche
         Module &m = ctx->mods[k];
         const long sidx = t - K + (k + 1);
         if (sidx >= 0 && k < K - 1) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k + 1].ev_bwd, 0));
+        PieceRange range(ctx, k, 1);
         ddg_status st = run_segment(ctx, k, 1, t, use_graph, &n);
         if (st != DDG_OK) return st;
         total += n;
+        if (range.close() != cudaSuccess) return DDG_ERR_CUDA;
         if (sidx >= 0 && k > 0) CU(cudaEventRecord(m.ev_bwd, m.stream));
         m.last_sample = sidx >= 0 ? sidx : -1;
     }
@@ -808,6 +836,7 @@ void ddg_destroy(ddg_ctx *ctx) {
         if (m.ev_fwd) cudaEventDestroy(m.ev_fwd);
         if (m.ev_bwd) cudaEventDestroy(m.ev_bwd);
         if (m.ev_join) cudaEventDestroy(m.ev_join);
+        for (auto e : m.ev_time) if (e) cudaEventDestroy(e);
         if (m.own_stream && m.stream) cudaStreamDestroy(m.stream);
     }
     cudaFree(ctx->x_stage); cudaFree(ctx->y_stage); cudaFree(ctx->dlogits); cudaFree(ctx->loss_dev);
@@ -958,6 +987,7 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
         CU(cudaEventCreateWithFlags(&m.ev_fwd, cudaEventDisableTiming));
         CU(cudaEventCreateWithFlags(&m.ev_bwd, cudaEventDisableTiming));
         CU(cudaEventCreateWithFlags(&m.ev_join, cudaEventDisableTiming));
+        if (cfg->time_pieces) for (auto &e : m.ev_time) CU(cudaEventCreate(&e));
         const size_t pn = std::max<size_t>(m.P, 1);
         CU(cudaMalloc(&m.arena, m.arena_bytes * m.R));
         CU(cudaMemset(m.arena, 0, m.arena_bytes * m.R));
@@ -1163,6 +1193,23 @@ ddg_status ddg_get_grads(ddg_ctx *ctx, int k, float *dst, size_t n, int on_devic
 ddg_status ddg_get_loss_dev(ddg_ctx *ctx, const float **loss_dev) {
     if (!ctx || !loss_dev) return DDG_ERR_INVALID_ARG;
     *loss_dev = ctx->loss_dev;
+    return DDG_OK;
+}
+
+ddg_status ddg_piece_times(ddg_ctx *ctx, float *fwd_ms, float *bwd_ms) {
+    if (!ctx || !fwd_ms || !bwd_ms) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    if (!ctx->cfg.time_pieces || ctx->t == 0) {
+        set_err(ctx, "ddg_piece_times needs a context created with time_pieces and at least one iteration");
+        return DDG_ERR_INVALID_ARG;
+    }
+    ddg_status st = sync_all(ctx);
+    if (st != DDG_OK) return st;
+    for (int k = 0; k < ctx->K; ++k) {
+        Module &m = ctx->mods[k];
+        CU(cudaEventElapsedTime(&fwd_ms[k], m.ev_time[0], m.ev_time[1]));
+        CU(cudaEventElapsedTime(&bwd_ms[k], m.ev_time[2], m.ev_time[3]));
+    }
     return DDG_OK;
 }
 

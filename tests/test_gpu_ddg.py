@@ -329,6 +329,49 @@ def test_ring_stamps_catch_a_shifted_slot():
     d.destroy()
 
 
+@pytest.mark.parametrize("graph", [False, True], ids=["eager", "graph"])
+def test_piece_times_cover_every_module(graph):
+    """time_pieces: every module's forward piece and backward + update piece of the last iteration has a positive device
+    time, a module in warm-up (no delayed gradient yet, Eq. 8) spends almost nothing in its backward piece, the pieces
+    fit inside the iteration's wall time, and the timed run produces the same weights as the untimed one."""
+    import time
+    from paper_1804_10574_b200 import binding, synth
+    L, B, shape = nets.resnet(1, 10), 32, (3, 32, 32)
+    w0 = synth.init_weights(L)
+    outs = []
+    for timed in (True, False):
+        d = binding.Ddg(L, [1, 2], B, shape, 10, precision="bf16", lr=0.01, momentum=0.9, use_graph=graph,
+                        time_pieces=timed)
+        d.set_weights(w0)
+        if not timed:
+            with pytest.raises(binding.DdgError) as e:
+                d.step(*[torch.from_numpy(a).cuda() for a in synth.batch(0, B, shape, 10)])
+                d.piece_times()
+            assert e.value.status == 1
+            d.destroy()
+            d = binding.Ddg(L, [1, 2], B, shape, 10, precision="bf16", lr=0.01, momentum=0.9, use_graph=graph)
+            d.set_weights(w0)
+        for t in range(8):
+            x, y = [torch.from_numpy(a).cuda() for a in synth.batch(t, B, shape, 10)]
+            d.sync()
+            t0 = time.perf_counter()
+            d.step(x, y, want_loss=False)
+            d.sync()
+            wall_ms = (time.perf_counter() - t0) * 1e3
+            if timed:
+                f, b = d.piece_times()
+                assert len(f) == 3 and len(b) == 3
+                assert all(v > 0 for v in f) and all(v >= 0 for v in b), (t, f, b)
+                assert max(f + b) < wall_ms + 0.5, (t, f, b, wall_ms)
+                if t == 0:      # modules 1 and 2 have no gradient yet: their backward piece is an empty update
+                    assert b[0] < 0.25 * b[2] and b[1] < 0.25 * b[2], b
+                if t >= 2:
+                    assert all(v > 0.01 for v in b), b
+        outs.append(d.get_weights(np.empty(d.n_params, dtype=np.float32)))
+        d.destroy()
+    assert np.array_equal(outs[0], outs[1])
+
+
 @pytest.mark.parametrize("net,splits,prec,opt", [("resnet8", [1, 2], "bf16", "sgd"), ("mlp", [0, 1, 2], "fp32", "adam"),
                                                   ("resnet8", [2], "fp32", "sgd")], ids=["resnet8_K3_bf16", "mlp_K4_adam", "resnet8_K2_fp32"])
 def test_checkpoint_resume_is_exact(net, splits, prec, opt):
