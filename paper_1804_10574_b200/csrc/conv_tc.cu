@@ -1278,7 +1278,13 @@ TcPlan tc_plan(int C, int n_tiles, int slab, bool shared, bool xform) {
     }
     TcPlan p;
     p.ep = ep;
-    const int per_pipe = (n_tiles + sms * ep.n_pipes - 1) / (sms * ep.n_pipes);
+    int per_pipe = (n_tiles + sms * ep.n_pipes - 1) / (sms * ep.n_pipes);
+    // ... and never a single tile per pipeline: a CTA's set-up and wind-down (barriers, TMEM, filter image, partial sums)
+    // cost as much SM time as three or four tiles, and under sharing the SM time a kernel takes is what the other
+    // streams wait for.  Half the CTAs with two tiles each: the 32- and 64-channel convolutions of the K = 4 step (256
+    // and 64 tiles) take longer alone, the iteration 6 % less (1.758 -> 1.650 ms); three tiles: 1.675; doubling the 16-
+    // channel kernels' four tiles per pipeline: 1.84.
+    if (shared && per_pipe < 2) per_pipe = 2;
     const int balanced = (n_tiles + per_pipe * ep.n_pipes - 1) / (per_pipe * ep.n_pipes);
     const int full = (n_tiles + ep.n_pipes - 1) / ep.n_pipes < sms ? (n_tiles + ep.n_pipes - 1) / ep.n_pipes : sms;
     p.grid = shared ? balanced : full;

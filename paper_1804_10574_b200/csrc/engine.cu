@@ -1007,7 +1007,11 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
             CU(cudaMalloc(&m.stamps, init.size() * sizeof(long long)));
             CU(cudaMemcpy(m.stamps, init.data(), init.size() * sizeof(long long), cudaMemcpyHostToDevice));
         }
-        CU(cudaStreamCreateWithFlags(&m.side, cudaStreamNonBlocking));
+        {   // the side stream inherits the priority of the module's stream (the caller may rank the modules)
+            int prio = 0;
+            CU(cudaStreamGetPriority(m.stream, &prio));
+            CU(cudaStreamCreateWithPriority(&m.side, cudaStreamNonBlocking, prio));
+        }
         CU(cudaEventCreateWithFlags(&m.ev_fork, cudaEventDisableTiming));
         for (auto &e : m.ev_side) CU(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
         size_t bn_max = 0, wg_max = 0;
