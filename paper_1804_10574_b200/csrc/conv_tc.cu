@@ -1250,7 +1250,10 @@ constexpr int kSmemMax = 227 * 1024;
 //   least sixteen (large batches); below that one pipeline whose two epilogue groups take alternate tiles.
 //   C >= 32: one pipeline whose two groups halve every tile where an SM has a single tile (shorter epilogue); for
 //   C = 32 two pipelines with one group each where it has two (both tiles side by side; C = 64 would need all 512
-//   TMEM columns for that); two pipelines with two groups each where it has three or more.
+//   TMEM columns for that).  Three tiles or more: C = 64 two pipelines whose two groups halve every tile; C = 32 two
+//   pipelines with two accumulators and one group each (the MMAs of the next tile run under the epilogue of this one;
+//   batch 256 / 1024 / 4096: 11.9 / 17.5 / 39.4 -> 10.8 / 16.5 / 36.5 us against two groups halving the tile), and
+//   four pipelines from sixteen tiles per SM on (batch 4096: 35.4 us).
 // A pipeline with a single tile uses one accumulator: fewer TMEM columns, so that CTAs of other streams fit beside it.
 // Several module streams (shared): as few CTAs as give every pipeline the same number of tiles as a full grid would give
 // the busiest one; the kernel's critical path is as long, and the SMs left over are free for the other streams (K = 4
@@ -1264,7 +1267,8 @@ TcPlan tc_plan(int C, int n_tiles, int slab, bool shared, bool xform) {
         const int n_acc = P > 1 ? 1 : (n_tiles <= sms ? 1 : 2);
         ep = EpiPlan{P, n_acc, n_acc, 1};
     } else if (n_tiles >= 3 * sms) {
-        ep = EpiPlan{2, C == 64 ? 1 : 2, 1, 2};  // 2 x 2 x 192 columns would not fit
+        if (C == 64) ep = EpiPlan{2, 1, 1, 2};  // 2 x 2 x 192 columns would not fit
+        else ep = n_tiles >= 16 * sms ? EpiPlan{4, 1, 1, 1} : EpiPlan{2, 2, 1, 1};
     } else if (C == 32 && n_tiles > sms) {
         ep = EpiPlan{2, 1, 1, 1};
     } else {

@@ -110,7 +110,8 @@ def test_conv3x3_many_tiles(shape):
 # The launch plan (pipelines per CTA, epilogue groups, stage ring) depends on the number of tiles, the arithmetic of
 # an output pixel does not: a batch of the kernel-sweep size must give, image for image, the bits that the same images
 # give in small batches (whose plan the oracle comparisons above cover).
-@pytest.mark.parametrize("shape", [(1024, 32, 32, 16), (1024, 16, 16, 32), (4096, 8, 8, 64)], ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("shape", [(1024, 32, 32, 16), (1024, 16, 16, 32), (1280, 16, 16, 32), (4096, 8, 8, 64)],
+                         ids=lambda s: "x".join(map(str, s)))
 def test_conv3x3_large_batch_equals_small_batches(shape):
     from paper_1804_10574_b200 import binding
     B, H, W, C = shape
