@@ -1354,7 +1354,11 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     // many tiles per CTA (large batches): the whole SM's shared memory for the stage ring, so that the loads of the next
     // tiles are in flight while this one is multiplied (batch 4096: 72 -> 68 us at 32 channels, 53 -> 44 us at 64);
     // otherwise the half-SM budget: taking more in the training step cost 4 % of the K = 4 iteration
-    const int budget = n_tiles_all >= 8 * g_num_sms ? kSmemMax - 2048 - (C == 32 ? 4096 : 0) : kSmemBudget;
+    // 32 channels, very large batches: two CTAs per SM (half the shared memory each, twice the pixel chunks): the MMA
+    // thread of this operand-swapped form is issue-bound, a second one per SM takes batch 4096 from 70.6 to 61.6 us
+    // (the 16-channel form is bound by the tensor pipe and the 64-channel one by its fold: both lose with two)
+    const bool pair = C == 32 && n_tiles_all >= 32 * g_num_sms;
+    const int budget = pair ? 110 * 1024 : (n_tiles_all >= 8 * g_num_sms ? kSmemMax - 2048 - (C == 32 ? 4096 : 0) : kSmemBudget);
     int n_stages = budget / stage_bytes;
     if (n_stages > kMaxStages) n_stages = kMaxStages;
     if (n_stages < 2) n_stages = 2;
@@ -1371,7 +1375,8 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     // the other streams and the fold should stay small; one per 16 tiles, up to a CTA per SM, for large batches
     const int max_chunks = slab ? (C == 16 ? 74 : 37) : 24;
     int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
-    const int big = n_tiles / 16 < (slab ? kWgMaxChunks : 48) ? n_tiles / 16 : (slab ? kWgMaxChunks : 48);
+    const int cap = slab ? (pair ? 2 * kWgMaxChunks : kWgMaxChunks) : 48;
+    const int big = n_tiles / 16 < cap ? n_tiles / 16 : cap;
     if (big > chunks) chunks = big;
     // tall: the unused accumulator rows (filter rows >= 3) read up to 128 - 3C pixel rows past the last column box
     launch_k(wgrad_tc_kernel<C>, dim3(chunks, slab ? 1 : 3), kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512 + (tall ? 4096 : 0), s, mx, md, scratch, H, W, rows, imgs, n_tiles, slab, n_stages, x_box_bytes, tmem_cols, wide, tall, err_word_of(s));
@@ -1523,7 +1528,8 @@ int launch_pack_one(const void *w, void *packed, int C, Launch s) {
 bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
     return conv_tc_supported(B, H, W, Cin, Cout, stride);
 }
-size_t wgrad_tc_scratch_elems() { return (size_t)kWgMaxChunks * 9 * 32 * 32 > (size_t)49 * 9 * 64 * 64 ? (size_t)kWgMaxChunks * 9 * 32 * 32 : (size_t)49 * 9 * 64 * 64; }
+// the most partials any launch leaves: 2 x 148 chunks of 9 x 32 x 32 (paired 32-channel CTAs); 64 channels: 49 chunks
+size_t wgrad_tc_scratch_elems() { return (size_t)2 * kWgMaxChunks * 9 * 32 * 32; }
 
 int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C, int cin_real,
                     Launch s) {

@@ -130,6 +130,29 @@ def test_conv3x3_large_batch_equals_small_batches(shape):
         assert torch.equal(ys, y[i:i + step]) and torch.equal(dxs, dx[i:i + step]), (shape, i)
 
 
+def test_conv3x3_wgrad_very_large_batch_equals_sum_of_parts():
+    """The weight gradient is a sum over the images of the batch: at a batch large enough for the launch plan with two
+    CTAs per SM (32 channels, 2400 images of 16x16) it must equal the sum of the weight gradients of four quarters of
+    the batch (sizes whose plan the oracle comparisons above cover) up to the order of the fp32 additions."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = 2400, 16, 16, 32
+    g = torch.Generator(device="cuda").manual_seed(23)
+    x = torch.randn(B, H, W, C, device="cuda", generator=g).to(torch.bfloat16)
+    dy = torch.randn(B, H, W, C, device="cuda", generator=g).to(torch.bfloat16)
+    scratch = torch.zeros(binding.conv3x3_wgrad_scratch_elems(B, H, W, C, C, 1), device="cuda")
+    dw = torch.empty(C, C, 3, 3, device="cuda")
+    binding.conv3x3_wgrad(1, x, dy, dw, scratch, B, H, W, C, C, 1)
+    parts = torch.zeros(C, C, 3, 3, device="cuda", dtype=torch.float64)
+    step = B // 4
+    for i in range(0, B, step):
+        dws = torch.empty(C, C, 3, 3, device="cuda")
+        binding.conv3x3_wgrad(1, x[i:i + step], dy[i:i + step], dws, scratch, step, H, W, C, C, 1)
+        parts += dws.double()
+    torch.cuda.synchronize()
+    assert rel(dw.cpu().numpy(), parts.cpu().numpy()) < 2e-6
+    assert float((dw.double() - parts).abs().max()) <= 1e-4 * float(parts.abs().max())
+
+
 @pytest.mark.parametrize("prec", [0, 1], ids=["fp32", "bf16"])
 # the last shape is large enough for the many-vectors-per-thread variants of the reductions and element-wise passes
 @pytest.mark.parametrize("shape", [(4, 64, 16), (7, 1024, 16), (33, 256, 32), (128, 64, 64), (3, 35, 12), (2, 3, 8),
