@@ -1404,7 +1404,10 @@ int launch_tc_s2(int dir, const void *src, const void *w, const void *w_packed, 
         if (!get_map_s2(src, B, H, W, CI, rows, imgs, &map)) return -1;
         int n_stages = kSmemBudget / TcCfg<CI>::tile_bytes;
         if (n_stages > kMaxStages) n_stages = kMaxStages;
-        const int grid = n_sp < g_num_sms ? n_sp : g_num_sms;
+        // two CTAs per SM where a CTA's single pipeline leaves the SM idle between hand-offs (16 -> 32 channels, batch
+        // 1024 / 4096: 39 / 126 -> 25 / 70 us); the 32 -> 64 forward is faster with one (22 / 46 against 27 / 51 us)
+        const int cap = (CI == 16 ? 2 : 1) * g_num_sms;
+        const int grid = n_sp < cap ? n_sp : cap;
         launch_k(conv3x3_s2_tc_kernel<CI, CO, 0>, grid, kS2Threads, s2_smem_bytes<CI, CO, 0>(n_stages), s, map, (const bf16 *)w, pk,
                  (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages, (const bf16 *)nullptr, (const bf16 *)nullptr, err_word_of(s));
     } else {
@@ -1413,7 +1416,9 @@ int launch_tc_s2(int dir, const void *src, const void *w, const void *w_packed, 
         if (n_stages > kMaxStages) n_stages = kMaxStages;
         if (n_stages < 3) n_stages = 3;
         const int n_tiles = 4 * n_sp;
-        const int grid = n_tiles < g_num_sms ? n_tiles : g_num_sms;
+        // two CTAs per SM (batch 1024 / 4096: 59 / 208 -> 37 / 121 us for 16 <- 32 channels, 27 / 73 -> 23 / 51 us for
+        // 32 <- 64)
+        const int grid = n_tiles < 2 * g_num_sms ? n_tiles : 2 * g_num_sms;
         launch_k(conv3x3_s2_tc_kernel<CO, CI, 1>, grid, kS2Threads, s2_smem_bytes<CO, CI, 1>(n_stages), s, map, (const bf16 *)w,
                  pk ? pk + S2Cfg<CI>::img_bytes : pk, (bf16 *)dst, Hs, Ws, rows, imgs, n_sp, n_stages,
                  sc.mode == 2 ? (const bf16 *)sc.a : nullptr, sc.mode == 2 ? (const bf16 *)sc.b : nullptr, err_word_of(s));
@@ -1433,7 +1438,9 @@ int launch_wg_s2(const void *x, const void *dy, float *dw, float *scratch, int B
     int n_stages = (200 * 1024) / stage_bytes;
     if (n_stages > 4) n_stages = 4;
     const int n_tiles = (int)((long)B * Hs * Ws / kTileM);
-    const int max_chunks = 64;
+    // pixel chunks = CTAs: 64 at the training step's sizes (a small fold), one per SM from four tiles per SM on (batch
+    // 1024 / 4096, 16 -> 32 channels: 36 / 103 -> 31 / 74 us; 32 -> 64: 23.5 / 52 -> 22 / 40 us)
+    const int max_chunks = n_tiles >= 512 ? kWgMaxChunks : 64;
     const int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
     launch_k(wgrad_s2_tc_kernel<CI>, chunks, kWgThreads, 1024 + (size_t)n_stages * stage_bytes + 512, s, mx, md, scratch, Hs, Ws,
              rows, imgs, n_tiles, n_stages, err_word_of(s));
@@ -1528,7 +1535,8 @@ int launch_pack_one(const void *w, void *packed, int C, Launch s) {
 bool wgrad_tc_supported(int B, int H, int W, int Cin, int Cout, int stride) {
     return conv_tc_supported(B, H, W, Cin, Cout, stride);
 }
-// the most partials any launch leaves: 2 x 148 chunks of 9 x 32 x 32 (paired 32-channel CTAs); 64 channels: 49 chunks
+// the most partials any launch leaves: 2 x 148 chunks of 9 x 32 x 32 (paired 32-channel CTAs) = 148 chunks of 9 x 32 x 64
+// (stride 2); 64 channels: 49 chunks
 size_t wgrad_tc_scratch_elems() { return (size_t)2 * kWgMaxChunks * 9 * 32 * 32; }
 
 int launch_wgrad_tc(const void *x, const void *dy, float *dw, float *scratch, int B, int H, int W, int C, int cin_real,
