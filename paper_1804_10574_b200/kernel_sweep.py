@@ -129,6 +129,10 @@ def main():
     for r in rows:
         print("%-34s %3s %9.1f %9.0f %6.1f%% %9.1f %6.1f%%" % (r["kernel"], "yes" if r["tensor_core"] else "no", r["us"], r["gbs"],
                                                               100 * r["hbm_frac"], r["tflops"], 100 * r["tensor_frac"]))
+    if any(r["kernel"].endswith("3->16 32x32 s1") for r in rows):
+        print("3->16: the single-kernel entry points take the 3-channel tensor as it is (CUDA-core kernels).  The bf16 training "
+              "step never launches these: its input shim stores the image zero-padded to 16 channels and the stem runs on the "
+              "16->16 tensor-core kernels above (forward and weight gradient; the input needs no gradient).")
 
 
 if __name__ == "__main__":
