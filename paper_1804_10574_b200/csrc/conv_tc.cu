@@ -1152,16 +1152,18 @@ __global__ void __launch_bounds__(256) wgrad_tc_fold_kernel(const float *__restr
     const int total = 9 * C * Co;
     const int o = threadIdx.x & 63, g = threadIdx.x >> 6;
     const int i = blockIdx.x * 64 + o;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     if (i < total) {
-        int c = g;
-        for (; c + 12 < chunks; c += 16) {
+        // batches of eight loads in flight per thread (the kernel is a chain of L2 round trips), the last one predicated
+        for (int c = g; c < chunks; c += 32) {
+            float q[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) acc[u] += __ldcg(part + (size_t)(c + 4 * u) * total + i);
+            for (int u = 0; u < 8; ++u) q[u] = (c + 4 * u < chunks) ? __ldcg(part + (size_t)(c + 4 * u) * total + i) : 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc[u] += q[u];
         }
-        for (; c < chunks; c += 4) acc[0] += __ldcg(part + (size_t)c * total + i);
     }
-    sm[g][o] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    sm[g][o] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
     __syncthreads();
     if (g == 0 && i < total) {
         const float t = (sm[0][o] + sm[1][o]) + (sm[2][o] + sm[3][o]);
