@@ -180,8 +180,10 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks, K):
 
     def conv_case(Hh, Cc, B=B, form="plain"):
         """form: "plain" = the convolution alone; "stats" = with the batch-norm statistics epilogue, sums folded by the
-        CTA that finishes last (what the step launches while module streams share the GPU); "partials" = the epilogue
-        leaves per-CTA partial sums for the element-wise pass (what a single stream launches)."""
+        CTA that finishes last (what the step launches while module streams share the GPU), timed with the launch plan
+        of a kernel that has the GPU to itself, as a kernel timed alone does; "stats_shared" = the same with the plan the
+        K > 1 step gives it (fewer CTAs, so that the other modules' kernels fit beside it: slower alone by design);
+        "partials" = the epilogue leaves per-CTA partial sums for the element-wise pass (what a single stream launches)."""
         per = 2 * B * Hh * Hh * Cc * 2                       # bytes of input + output of one launch
         n = max(8, int(400e6 // per) + 1) if B <= 1024 else max(2, int(400e6 // per) + 1)
         xs = [torch.randn(B, Hh, Hh, Cc, device="cuda").to(bf) for _ in range(n)]
@@ -193,6 +195,9 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks, K):
         scr = torch.zeros(binding.conv3x3_fused_scratch_elems(B, Hh, Hh, Cc), device="cuda")
         if form == "stats":
             fns = [(lambda st, i=i: binding.conv3x3_fwd_stats_prepared(xs[i], w, pk, ys[i], m, iv, scr, B, Hh, Hh, Cc, st)) for i in range(n)]
+        elif form == "stats_shared":
+            # the launch plan of a step with several module streams (fewer CTAs, at least two tiles per pipeline)
+            fns = [(lambda st, i=i: binding.conv3x3_fwd_stats_shared(xs[i], w, pk, ys[i], m, iv, scr, B, Hh, Hh, Cc, st)) for i in range(n)]
         elif form == "partials":
             fns = [(lambda st, i=i: binding.conv3x3_fwd_partials(xs[i], w, pk, ys[i], scr, B, Hh, Hh, Cc, st)) for i in range(n)]
         else:
@@ -213,7 +218,8 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks, K):
         traffic = (c16["dram_bytes_read"] + c16["dram_bytes_write"]) * B / float(c16["batch"])
     share = cnt.get("launch_list resnet110 K=4 B=128", {})
     roof = {"kernel": "conv3x3_tc_kernel<16> (tensor-core 3x3 convolution, forward, with the batch-norm statistics "
-                      "epilogue as the step launches it: %s) C=16 32x32 B=%d"
+                      "epilogue as the step launches it: %s; timed alone, with the grid of a kernel that has the GPU to "
+                      "itself) C=16 32x32 B=%d"
                       % ("sums folded by the last CTA" if K > 1 else "per-CTA partial sums left to the element-wise pass", B),
             "bound": "hbm",
             "achieved": alg / dt / 1e9, "peak": hbm, "unit": "GB/s", "frac": alg / dt / 1e9 / hbm, "traffic": traffic,
@@ -221,12 +227,15 @@ def dominant_kernel_roofline(torch, binding, cfg, peaks, K):
             "ncu_share_of_step": share.get("conv3x3_tc_kernel<16>") if share.get("valid") else None, "launches_timed": n,
             "tflops": flops / dt / 1e12, "tensor_frac": flops / dt / 1e12 / tflops}
     others = []
-    for form in ("plain", "stats", "partials"):
+    for form in ("plain", "stats", "stats_shared", "partials"):
         if form == step_form:
             continue
         dtc, nbytes, fl, _ = conv_case(32, 16, form=form)
         others.append({"kernel": "conv3x3_tc_kernel<16> fwd 32x32 B=%d, %s" % (B, {"plain": "without the statistics epilogue",
-                       "stats": "statistics folded by the last CTA", "partials": "partial sums left to the element-wise pass"}[form]),
+                       "stats": "statistics folded by the last CTA",
+                       "stats_shared": "statistics folded by the last CTA, launch plan of the K > 1 step (fewer CTAs, leaves "
+                                       "SMs to the other module streams)",
+                       "partials": "partial sums left to the element-wise pass"}[form]),
                        "launch_us": dtc * 1e6, "hbm_gbs": nbytes / dtc / 1e9, "hbm_frac": nbytes / dtc / 1e9 / hbm})
     for (Hh, Cc) in ((16, 32), (8, 64)):
         dtc, nbytes, fl, _ = conv_case(Hh, Cc)

@@ -248,6 +248,12 @@ ddg_status ddg_conv3x3_fwd_stats(const void *x, const void *w, const void *packe
  * training step.  For timing the kernel in the form the step launches it. */
 ddg_status ddg_conv3x3_fwd_stats_prepared(const void *x, const void *w, const void *packed, void *y, float *mean,
                                           float *invstd, float *scratch, int B, int H, int W, int C, void *stream);
+/* ddg_conv3x3_fwd_stats_prepared with the launch plan the training step uses while K > 1 module streams share the GPU
+ * (fewer CTAs with at least two tiles per pipeline, the programmatic launch attribute as on the step's convolutions):
+ * the same y bit for bit, the statistics from a different number of per-CTA partial sums.  For checking and timing the
+ * kernel in exactly the form a DDG step with several modules launches it. */
+ddg_status ddg_conv3x3_fwd_stats_shared(const void *x, const void *w, const void *packed, void *y, float *mean,
+                                        float *invstd, float *scratch, int B, int H, int W, int C, void *stream);
 ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
                                    const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
                                    const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H,

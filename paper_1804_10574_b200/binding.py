@@ -34,7 +34,7 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_load_state", "ddg_conv1x1_fwd", "ddg_conv1x1_dgrad_add", "ddg_conv1x1_wgrad_scratch_elems",
            "ddg_conv1x1_wgrad", "ddg_conv3x3_bnrelu_fwd_stats", "ddg_conv3x3_fwd_partials",
            "ddg_bn_fwd_partials", "ddg_conv3x3_dgrad_partials", "ddg_bn_bwd_partials", "ddg_conv3x3_fwd_stats_prepared",
-           "ddg_piece_times"]
+           "ddg_piece_times", "ddg_conv3x3_fwd_stats_shared"]
 
 
 class Layer(ctypes.Structure):
@@ -96,6 +96,7 @@ _lib.ddg_conv3x3_fused_scratch_elems.argtypes = [_i] * 4
 _lib.ddg_conv3x3_fused_scratch_elems.restype = _sz
 _lib.ddg_conv3x3_fwd_stats.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_fwd_stats_prepared.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
+_lib.ddg_conv3x3_fwd_stats_shared.argtypes = [_vp] * 7 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_fwd_partials.argtypes = [_vp] * 5 + [ctypes.POINTER(_i)] + [_i] * 4 + [_vp]
 _lib.ddg_bn_fwd_partials.argtypes = [_vp] * 6 + [_i, _vp, _vp, _i, _i, _i, _i, _vp]
 _lib.ddg_conv3x3_dgrad_partials.argtypes = [_vp] * 11 + [ctypes.POINTER(_i)] + [_i] * 4 + [_vp]
@@ -280,6 +281,11 @@ def conv3x3_fwd_stats(x, w, packed, y, mean, invstd, scratch, B, H, W, C, stream
 def conv3x3_fwd_stats_prepared(x, w, packed, y, mean, invstd, scratch, B, H, W, C, stream=None):
     _ok(_lib.ddg_conv3x3_fwd_stats_prepared(_ptr(x), _ptr(w), _ptr(packed), _ptr(y), _ptr(mean), _ptr(invstd),
                                             _ptr(scratch), B, H, W, C, stream))
+
+
+def conv3x3_fwd_stats_shared(x, w, packed, y, mean, invstd, scratch, B, H, W, C, stream=None):
+    _ok(_lib.ddg_conv3x3_fwd_stats_shared(_ptr(x), _ptr(w), _ptr(packed), _ptr(y), _ptr(mean), _ptr(invstd),
+                                         _ptr(scratch), B, H, W, C, stream))
 
 
 def conv3x3_fwd_partials(x, w, packed, y, part, B, H, W, C, stream=None):

@@ -136,6 +136,18 @@ ddg_status ddg_conv3x3_fwd_stats_prepared(const void *x, const void *w, const vo
     return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, (cudaStream_t)stream, bf));
 }
 
+ddg_status ddg_conv3x3_fwd_stats_shared(const void *x, const void *w, const void *packed, void *y, float *mean,
+                                        float *invstd, float *scratch, int B, int H, int W, int C, void *stream) {
+    if (!x || !w || !y || !mean || !invstd || !scratch) return DDG_ERR_INVALID_ARG;
+    if (init_once() != DDG_OK) return DDG_ERR_CUDA;
+    if (!conv_tc_supported(B, H, W, C, C, 1)) return DDG_ERR_UNSUPPORTED;
+    if (pending_error()) return DDG_ERR_CUDA;
+    BnFuse bf;
+    bf.counter = reinterpret_cast<unsigned *>(scratch); bf.part = scratch + 32; bf.o0 = mean; bf.o1 = invstd;
+    const Launch shared((cudaStream_t)stream, 2, true, nullptr);  // what the engine passes for K > 1
+    return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, shared, bf));
+}
+
 ddg_status ddg_conv3x3_fwd_partials(const void *x, const void *w, const void *packed, void *y, float *part,
                                     int *n_part_host, int B, int H, int W, int C, void *stream) {
     if (!x || !w || !y || !part || !n_part_host) return DDG_ERR_INVALID_ARG;

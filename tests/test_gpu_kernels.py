@@ -303,6 +303,35 @@ def test_conv_forward_with_batch_statistics(shape, packed):
     assert np.max(np.abs(mean.cpu().numpy() - m2)) < 1e-3 * float(np.sqrt(np.mean(y_ref ** 2))) and rel(invstd.cpu().numpy(), is2) < 1e-3
 
 
+# the shapes of the ResNet-110 batch-128 step (the plan gives their pipelines two or four tiles on fewer CTAs), small
+# batches (CTAs with a single pipeline and two tiles) and many tiles
+@pytest.mark.parametrize("shape", [(128, 32, 32, 16), (128, 16, 16, 32), (128, 8, 8, 64), (3, 32, 32, 16), (5, 16, 16, 32),
+                                   (10, 8, 8, 64), (74, 16, 16, 32), (301, 32, 32, 16), (231, 16, 16, 32), (902, 8, 8, 64)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_conv_forward_with_batch_statistics_shared_gpu_plan(shape):
+    """The launch plan of a step whose K > 1 module streams share the GPU (fewer CTAs, at least two tiles per pipeline)
+    changes neither a pixel nor, beyond the order of the additions, the statistics: y equals the single-stream plan's y
+    bit for bit, mean and invstd agree with it to fp32 rounding and with the oracle's batch norm of the stored tensor."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = shape
+    rng = np.random.default_rng(29)
+    x, _ = to_dev(rng.standard_normal((B, C, H, W)) * 1.1 - 0.2, 1)
+    w, _ = _filter(rng, C)
+    pk = torch.empty(binding.conv3x3_packed_bytes(B, H, W, C), dtype=torch.uint8, device="cuda")
+    binding.conv3x3_pack(w, pk, C)
+    y0, y1 = torch.empty_like(x), torch.full_like(x, 5.0)
+    m0, i0, m1, i1 = (torch.full((C,), 7.0, dtype=torch.float32, device="cuda") for _ in range(4))
+    scratch = torch.zeros(binding.conv3x3_fused_scratch_elems(B, H, W, C), dtype=torch.float32, device="cuda")
+    binding.conv3x3_fwd_stats(x, w, pk, y0, m0, i0, scratch, B, H, W, C)
+    for _ in range(2):     # the ticket counter is left at zero by every call
+        binding.conv3x3_fwd_stats_shared(x, w, pk, y1, m1, i1, scratch, B, H, W, C)
+    torch.cuda.synchronize()
+    assert torch.equal(y0, y1)
+    assert rel(m1.cpu().numpy(), m0.cpu().numpy()) < 2e-6 and rel(i1.cpu().numpy(), i0.cpu().numpy()) < 2e-6
+    _, m_ref, is_ref = orc.bn_forward(from_dev(y1), np.ones(C), np.zeros(C))
+    assert rel(m1.cpu().numpy(), m_ref) < 2e-5 and rel(i1.cpu().numpy(), is_ref) < 2e-5
+
+
 @pytest.mark.parametrize("shape", FUSED_SHAPES, ids=lambda s: "x".join(map(str, s)))
 @pytest.mark.parametrize("with_shortcut,with_sums", [(True, False), (False, True), (True, True)],
                          ids=["shortcut", "sums", "shortcut_sums"])
