@@ -138,6 +138,16 @@ ddg_status ddg_step(ddg_ctx *ctx, const float *x_dev, const int *y_dev, float *l
  * context's first stream, runs ddg_step and, when loss_host is non-NULL, waits and returns the loss. */
 ddg_status ddg_step_host(ddg_ctx *ctx, const float *x_host, const int *y_host, float *loss_host);
 
+/* ddg_step_host without the host waiting for the device in every iteration: the call enqueues iteration t (input
+ * copies, sweeps, updates) and the read-back of its loss, and hands out the loss of iteration t-1, which completed while
+ * the host was preparing this call (NaN at the first call).  The host therefore runs one iteration ahead of the losses it
+ * logs, and consecutive iterations overlap on the device exactly as with loss_host = NULL.  loss_prev_host: host,
+ * nullable.  x_host / y_host of iteration t must stay valid until the call for iteration t+1 has returned a loss (or
+ * ddg_sync / ddg_pipelined_loss returned).  ddg_pipelined_loss waits for the most recent iteration's loss and returns it
+ * (the one no later call will hand out).  Do not mix with loss-returning ddg_step / ddg_step_host calls in between. */
+ddg_status ddg_step_host_pipelined(ddg_ctx *ctx, const float *x_host, const int *y_host, float *loss_prev_host);
+ddg_status ddg_pipelined_loss(ddg_ctx *ctx, float *loss_host);
+
 /* The stepsize sequence {gamma_t} of Algorithm 1 is driven by the caller. */
 ddg_status ddg_set_lr(ddg_ctx *ctx, float lr);
 

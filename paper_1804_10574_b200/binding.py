@@ -34,7 +34,8 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_load_state", "ddg_conv1x1_fwd", "ddg_conv1x1_dgrad_add", "ddg_conv1x1_wgrad_scratch_elems",
            "ddg_conv1x1_wgrad", "ddg_conv3x3_bnrelu_fwd_stats", "ddg_conv3x3_fwd_partials",
            "ddg_bn_fwd_partials", "ddg_conv3x3_dgrad_partials", "ddg_bn_bwd_partials", "ddg_conv3x3_fwd_stats_prepared",
-           "ddg_piece_times", "ddg_conv3x3_fwd_stats_shared"]
+           "ddg_piece_times", "ddg_conv3x3_fwd_stats_shared",
+           "ddg_step_host_pipelined", "ddg_pipelined_loss"]
 
 
 class Layer(ctypes.Structure):
@@ -61,6 +62,8 @@ _lib.ddg_create.argtypes = [ctypes.POINTER(Layer), _i, ctypes.POINTER(_i), _i, c
 _lib.ddg_step.argtypes = [_vp, _vp, _vp, ctypes.POINTER(_f)]
 _lib.ddg_step_host.argtypes = [_vp, _vp, _vp, ctypes.POINTER(_f)]
 _lib.ddg_set_lr.argtypes = [_vp, _f]
+_lib.ddg_step_host_pipelined.argtypes = [_vp, _vp, _vp, ctypes.POINTER(_f)]
+_lib.ddg_pipelined_loss.argtypes = [_vp, ctypes.POINTER(_f)]
 _lib.ddg_piece_times.argtypes = [_vp, ctypes.POINTER(_f), ctypes.POINTER(_f)]
 _lib.ddg_param_count.argtypes = [_vp, ctypes.POINTER(_sz), ctypes.POINTER(_sz)]
 _lib.ddg_get_weights.argtypes = [_vp, _vp, _sz, _i]
@@ -193,6 +196,17 @@ class Ddg:
         loss = ctypes.c_float()
         self._check(_lib.ddg_step_host(self._h, _ptr(x_host), _ptr(y_host), ctypes.byref(loss) if want_loss else None))
         return loss.value if want_loss else None
+
+    def step_host_pipelined(self, x_host, y_host):
+        """Enqueues the iteration; returns the loss of the PREVIOUS iteration (NaN at the first call)."""
+        loss = ctypes.c_float()
+        self._check(_lib.ddg_step_host_pipelined(self._h, _ptr(x_host), _ptr(y_host), ctypes.byref(loss)))
+        return loss.value
+
+    def pipelined_loss(self):
+        loss = ctypes.c_float()
+        self._check(_lib.ddg_pipelined_loss(self._h, ctypes.byref(loss)))
+        return loss.value
 
     def set_lr(self, lr):
         self._check(_lib.ddg_set_lr(self._h, lr))

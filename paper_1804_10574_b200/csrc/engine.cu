@@ -109,6 +109,12 @@ struct ddg_ctx {
     float *dlogits = nullptr, *loss_dev = nullptr;
     float *pinned_loss = nullptr;
     cudaStream_t loss_stream = nullptr;  // carries the loss read-back, so that it waits for the forward sweep only
+    // pipelined loss read-back (ddg_step_host_pipelined): iteration t's loss and error word land in slot t mod 2 of a
+    // pinned ring, ev_loss[t mod 2] marks the copy, and the last module's next forward sweep waits for it before it
+    // overwrites the device scalar
+    float *pinned_ring = nullptr;
+    cudaEvent_t ev_loss[2] = {nullptr, nullptr};
+    long loss_pending = -1;  // iteration whose copy is the latest enqueued (-1: none)
     std::vector<cudaGraphExec_t> graphs;
     std::vector<long> graph_launches;
     bool graphs_ready = false;
@@ -704,6 +710,8 @@ ddg_status enqueue_iteration(ddg_ctx *ctx, long t, bool use_graph, long *launche
     for (int k = 0; k < K; ++k) {
         Module &m = ctx->mods[k];
         if (k > 0) CU(cudaStreamWaitEvent(m.stream, ctx->mods[k - 1].ev_fwd, 0));
+        // a pipelined read-back of the previous loss must have left the device scalar before this sweep rewrites it
+        if (k == K - 1 && ctx->loss_pending >= 0) CU(cudaStreamWaitEvent(m.stream, ctx->ev_loss[ctx->loss_pending & 1], 0));
         PieceRange range(ctx, k, 0);
         ddg_status st = run_segment(ctx, k, 0, t, use_graph, &n);
         if (st != DDG_OK) return st;
@@ -842,6 +850,8 @@ void ddg_destroy(ddg_ctx *ctx) {
     cudaFree(ctx->x_stage); cudaFree(ctx->y_stage); cudaFree(ctx->dlogits); cudaFree(ctx->loss_dev);
     cudaFree(ctx->err_word);
     if (ctx->pinned_loss) cudaFreeHost(ctx->pinned_loss);
+    if (ctx->pinned_ring) cudaFreeHost(ctx->pinned_ring);
+    for (auto e : ctx->ev_loss) if (e) cudaEventDestroy(e);
     if (ctx->loss_stream) cudaStreamDestroy(ctx->loss_stream);
     delete ctx;
 }
@@ -1084,6 +1094,8 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
     CU(cudaMalloc(&c->err_word, sizeof(int)));  // this context's own error word, clear at creation
     CU(cudaMemset(c->err_word, 0, sizeof(int)));
     CU(cudaMallocHost(&c->pinned_loss, 8));  // the loss, and the tensor-core kernels' error word read with it
+    CU(cudaMallocHost(&c->pinned_ring, 16));
+    for (auto &e : c->ev_loss) CU(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     CU(cudaStreamCreateWithFlags(&c->loss_stream, cudaStreamNonBlocking));
     // the memsets above ran on the legacy default stream, which the non-blocking module streams do not wait for
     CU(cudaDeviceSynchronize());
@@ -1093,7 +1105,8 @@ ddg_status ddg_create(const ddg_layer *layers, int n_layers, const int *split_af
     return DDG_OK;
 }
 
-static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float *loss_host, cudaMemcpyKind kind) {
+static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float *loss_host, cudaMemcpyKind kind,
+                              bool pipelined = false) {
     if (!ctx || !x || !y) return DDG_ERR_INVALID_ARG;
     if (ctx->broken) return DDG_ERR_STATE;
     const long t = ctx->t;
@@ -1111,6 +1124,27 @@ static ddg_status step_common(ddg_ctx *ctx, const float *x, const int *y, float 
     ddg_status st = enqueue_iteration(ctx, t, ctx->cfg.use_graph && steady, &ctx->launches);
     if (st != DDG_OK) { ctx->broken = true; return st; }
     ctx->t = t + 1;
+    if (pipelined) {
+        // enqueue the read-back of this iteration's loss, hand out the previous iteration's (long complete)
+        float *slot = ctx->pinned_ring + 2 * (t & 1);
+        CU(cudaStreamWaitEvent(ctx->loss_stream, ctx->mods[K - 1].ev_fwd, 0));
+        CU(cudaMemcpyAsync(slot, ctx->loss_dev, 4, cudaMemcpyDeviceToHost, ctx->loss_stream));
+        CU(cudaMemcpyAsync(slot + 1, ctx->err_word, sizeof(int), cudaMemcpyDeviceToHost, ctx->loss_stream));
+        CU(cudaEventRecord(ctx->ev_loss[t & 1], ctx->loss_stream));
+        const long prev = ctx->loss_pending;
+        ctx->loss_pending = t;
+        if (loss_host) {
+            if (prev < 0) *loss_host = nanf("");
+            else {
+                CU(cudaEventSynchronize(ctx->ev_loss[prev & 1]));
+                const float *p = ctx->pinned_ring + 2 * (prev & 1);
+                *loss_host = p[0];
+                const int flag = *reinterpret_cast<const int *>(p + 1);
+                if (flag != 0) return report_error_word(ctx, flag);
+            }
+        }
+        return DDG_OK;
+    }
     if (loss_host) {
         // The loss exists once the last module's forward sweep is done: wait for that only.  The backward sweeps and
         // updates of this iteration stay in flight and overlap the caller's next step (the decoupling DDG is about).
@@ -1133,6 +1167,25 @@ ddg_status ddg_step(ddg_ctx *ctx, const float *x_dev, const int *y_dev, float *l
 
 ddg_status ddg_step_host(ddg_ctx *ctx, const float *x_host, const int *y_host, float *loss_host) {
     return step_common(ctx, x_host, y_host, loss_host, cudaMemcpyHostToDevice);
+}
+
+ddg_status ddg_step_host_pipelined(ddg_ctx *ctx, const float *x_host, const int *y_host, float *loss_prev_host) {
+    return step_common(ctx, x_host, y_host, loss_prev_host, cudaMemcpyHostToDevice, true);
+}
+
+ddg_status ddg_pipelined_loss(ddg_ctx *ctx, float *loss_host) {
+    if (!ctx || !loss_host) return DDG_ERR_INVALID_ARG;
+    if (ctx->broken) return DDG_ERR_STATE;
+    if (ctx->loss_pending < 0) {
+        set_err(ctx, "ddg_pipelined_loss: no ddg_step_host_pipelined call has been made");
+        return DDG_ERR_INVALID_ARG;
+    }
+    CU(cudaEventSynchronize(ctx->ev_loss[ctx->loss_pending & 1]));
+    const float *p = ctx->pinned_ring + 2 * (ctx->loss_pending & 1);
+    *loss_host = p[0];
+    const int flag = *reinterpret_cast<const int *>(p + 1);
+    if (flag != 0) return report_error_word(ctx, flag);
+    return DDG_OK;
 }
 
 ddg_status ddg_set_lr(ddg_ctx *ctx, float lr) {
@@ -1303,6 +1356,7 @@ ddg_status ddg_load_state(ddg_ctx *ctx, const void *src_host, size_t bytes) {
     for (auto &q : r) { CU(cudaMemcpy(q.first, p, q.second, cudaMemcpyHostToDevice)); p += q.second; }
     CU(cudaDeviceSynchronize());  // the copies ran on the default stream; the module streams do not wait for it
     ctx->t = h.t;
+    ctx->loss_pending = -1;  // a read-back enqueued before the restore belongs to the run that was replaced
     return DDG_OK;
 }
 

@@ -329,6 +329,40 @@ def test_ring_stamps_catch_a_shifted_slot():
     d.destroy()
 
 
+@pytest.mark.parametrize("net,splits,prec", [("resnet8", [1, 2], "bf16"), ("mlp", [1], "fp32")], ids=["resnet8_K3_bf16", "mlp_K2_fp32"])
+def test_pipelined_loss_read_back_equals_the_synchronous_run(net, splits, prec):
+    """ddg_step_host_pipelined hands out, one call later, exactly the losses ddg_step_host returns (the host runs one
+    iteration ahead of the loss it logs); ddg_pipelined_loss returns the last one; the weights after the run are the
+    same bits.  Input buffers are reused two calls later, as the contract allows."""
+    from paper_1804_10574_b200 import binding, synth
+    cfg = nets.config(net)
+    B, steps = 8, 14
+    kw = dict(precision=prec, lr=0.05, momentum=0.9, weight_decay=5e-4, use_graph=True)
+    w0 = synth.init_weights(cfg["layers"], perturb_affine=0.1)
+    batches = [synth.batch(t, B, cfg["in_shape"], cfg["num_classes"]) for t in range(steps)]
+
+    a = binding.Ddg(cfg["layers"], splits, B, cfg["in_shape"], cfg["num_classes"], **kw)
+    a.set_weights(w0)
+    ref = [a.step_host(torch.from_numpy(x).pin_memory(), torch.from_numpy(y).pin_memory()) for x, y in batches]
+    wa = a.get_weights(np.empty(a.n_params, dtype=np.float32))
+    a.destroy()
+
+    b = binding.Ddg(cfg["layers"], splits, B, cfg["in_shape"], cfg["num_classes"], **kw)
+    b.set_weights(w0)
+    ring = [(torch.from_numpy(batches[0][0].copy()).pin_memory(), torch.from_numpy(batches[0][1].copy()).pin_memory()) for _ in range(2)]
+    got = []
+    for t, (x, y) in enumerate(batches):
+        xb, yb = ring[t % 2]          # the buffer of iteration t-2: its call for t-1 has returned a loss
+        xb.copy_(torch.from_numpy(x)); yb.copy_(torch.from_numpy(y))
+        got.append(b.step_host_pipelined(xb, yb))
+    last = b.pipelined_loss()
+    wb = b.get_weights(np.empty(b.n_params, dtype=np.float32))
+    b.destroy()
+    assert np.isnan(got[0])
+    assert got[1:] == ref[:-1] and last == ref[-1]
+    assert np.array_equal(wa, wb)
+
+
 @pytest.mark.parametrize("graph", [False, True], ids=["eager", "graph"])
 def test_piece_times_cover_every_module(graph):
     """time_pieces: every module's forward piece and backward + update piece of the last iteration has a positive device
