@@ -268,6 +268,12 @@ ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *pa
                                    const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
                                    const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H,
                                    int W, int C, void *stream);
+/* ddg_conv3x3_dgrad_fused under the same shared-GPU launch plan: the same dx bit for bit, the sums from a different
+ * number of per-CTA partial sums. */
+ddg_status ddg_conv3x3_dgrad_fused_shared(const void *dy, const void *w, const void *packed, void *dx,
+                                          const void *res_dout, const void *res_out, const void *bn_mask, const void *bn_x,
+                                          const float *bn_mean, const float *bn_invstd, float *dbeta, float *dgamma,
+                                          float *scratch, int B, int H, int W, int C, void *stream);
 /* The same two fused forms as a single stream launches them when it has the GPU to itself (K = 1): the convolution only
  * leaves the per-CTA partial sums of its epilogue, part [*n_part_host][2C] fp32 (device, at least
  * ddg_conv3x3_fused_scratch_elems floats; *n_part_host, host, receives the number of rows = CTAs of the launch), and

@@ -35,7 +35,7 @@ EXPORTS = ["ddg_create", "ddg_step", "ddg_step_host", "ddg_set_lr", "ddg_param_c
            "ddg_conv1x1_wgrad", "ddg_conv3x3_bnrelu_fwd_stats", "ddg_conv3x3_fwd_partials",
            "ddg_bn_fwd_partials", "ddg_conv3x3_dgrad_partials", "ddg_bn_bwd_partials", "ddg_conv3x3_fwd_stats_prepared",
            "ddg_piece_times", "ddg_conv3x3_fwd_stats_shared",
-           "ddg_step_host_pipelined", "ddg_pipelined_loss"]
+           "ddg_step_host_pipelined", "ddg_pipelined_loss", "ddg_conv3x3_dgrad_fused_shared"]
 
 
 class Layer(ctypes.Structure):
@@ -106,6 +106,7 @@ _lib.ddg_conv3x3_dgrad_partials.argtypes = [_vp] * 11 + [ctypes.POINTER(_i)] + [
 _lib.ddg_bn_bwd_partials.argtypes = [_vp] * 10 + [_i] + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_bnrelu_fwd_stats.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_dgrad_fused.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
+_lib.ddg_conv3x3_dgrad_fused_shared.argtypes = [_vp] * 13 + [_i] * 4 + [_vp]
 _lib.ddg_conv3x3_s2_dgrad_shortcut.argtypes = [_vp] * 5 + [_i] * 4 + [_vp]
 _lib.ddg_conv1x1_fwd.argtypes = [_i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]
 _lib.ddg_conv1x1_dgrad_add.argtypes = [_i, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]
@@ -340,6 +341,13 @@ def conv3x3_dgrad_fused(dy, w, packed, dx, res_dout, res_out, bn_mask, bn_x, bn_
     _ok(_lib.ddg_conv3x3_dgrad_fused(_ptr(dy), _ptr(w), _ptr(packed), _ptr(dx), _ptr(res_dout), _ptr(res_out),
                                      _ptr(bn_mask), _ptr(bn_x), _ptr(bn_mean), _ptr(bn_invstd), _ptr(dbeta), _ptr(dgamma),
                                      _ptr(scratch), B, H, W, C, stream))
+
+
+def conv3x3_dgrad_fused_shared(dy, w, packed, dx, res_dout, res_out, bn_mask, bn_x, bn_mean, bn_invstd, dbeta, dgamma,
+                               scratch, B, H, W, C, stream=None):
+    _ok(_lib.ddg_conv3x3_dgrad_fused_shared(_ptr(dy), _ptr(w), _ptr(packed), _ptr(dx), _ptr(res_dout), _ptr(res_out),
+                                            _ptr(bn_mask), _ptr(bn_x), _ptr(bn_mean), _ptr(bn_invstd), _ptr(dbeta),
+                                            _ptr(dgamma), _ptr(scratch), B, H, W, C, stream))
 
 
 def conv3x3_s2_dgrad_shortcut(dy, w, dx, res_dout, res_out, B, H, W, Cin, stream=None):

@@ -221,10 +221,32 @@ ddg_status ddg_conv3x3_bnrelu_fwd_stats(const void *x, const void *res, const vo
     return done(launch_conv_tc(0, x, w, packed, y, B, H, W, C, Shortcut{}, s, bf, xf));
 }
 
+namespace {
+ddg_status dgrad_fused(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
+                       const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
+                       const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H, int W, int C,
+                       void *stream, bool shared);
+}
 ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
                                    const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
                                    const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H,
                                    int W, int C, void *stream) {
+    return dgrad_fused(dy, w, packed, dx, res_dout, res_out, bn_mask, bn_x, bn_mean, bn_invstd, dbeta, dgamma, scratch, B, H,
+                       W, C, stream, false);
+}
+ddg_status ddg_conv3x3_dgrad_fused_shared(const void *dy, const void *w, const void *packed, void *dx,
+                                          const void *res_dout, const void *res_out, const void *bn_mask, const void *bn_x,
+                                          const float *bn_mean, const float *bn_invstd, float *dbeta, float *dgamma,
+                                          float *scratch, int B, int H, int W, int C, void *stream) {
+    return dgrad_fused(dy, w, packed, dx, res_dout, res_out, bn_mask, bn_x, bn_mean, bn_invstd, dbeta, dgamma, scratch, B, H,
+                       W, C, stream, true);
+}
+}  // extern "C"
+namespace {
+ddg_status dgrad_fused(const void *dy, const void *w, const void *packed, void *dx, const void *res_dout,
+                       const void *res_out, const void *bn_mask, const void *bn_x, const float *bn_mean,
+                       const float *bn_invstd, float *dbeta, float *dgamma, float *scratch, int B, int H, int W, int C,
+                       void *stream, bool shared) {
     if (!dy || !w || !dx || !scratch) return DDG_ERR_INVALID_ARG;
     if ((res_dout == nullptr) != (res_out == nullptr)) return DDG_ERR_INVALID_ARG;
     const bool sums = bn_mask || bn_x || bn_mean || bn_invstd || dbeta || dgamma;
@@ -241,8 +263,11 @@ ddg_status ddg_conv3x3_dgrad_fused(const void *dy, const void *w, const void *pa
         bf.counter = reinterpret_cast<unsigned *>(scratch); bf.part = scratch + 32; bf.o0 = dbeta; bf.o1 = dgamma;
         bf.mask = bn_mask; bf.x = bn_x; bf.mean = bn_mean; bf.invstd = bn_invstd;
     }
-    return done(launch_conv_tc(1, dy, w, packed, dx, B, H, W, C, sc, s, bf));
+    // shared: the launch plan and launch attribute policy the engine uses while K > 1 module streams share the GPU
+    return done(launch_conv_tc(1, dy, w, packed, dx, B, H, W, C, sc, shared ? Launch(s, 2, true, nullptr) : Launch(s), bf));
 }
+}  // namespace
+extern "C" {
 
 ddg_status ddg_conv3x3_s2_dgrad_shortcut(const void *dy, const void *w, void *dx, const void *res_dout,
                                          const void *res_out, int B, int H, int W, int Cin, void *stream) {

@@ -372,6 +372,36 @@ def test_conv_input_gradient_with_shortcut_and_batch_norm_sums(shape, with_short
         assert np.max(np.abs(dg.cpu().numpy() - dg_ref)) < 2e-5 * scale * 2, (dg.cpu().numpy(), dg_ref)
 
 
+@pytest.mark.parametrize("shape", [(128, 32, 32, 16), (128, 16, 16, 32), (128, 8, 8, 64), (5, 16, 16, 32), (10, 8, 8, 64),
+                                   (231, 16, 16, 32), (902, 8, 8, 64)], ids=lambda s: "x".join(map(str, s)))
+def test_conv_input_gradient_fused_shared_gpu_plan(shape):
+    """The input-gradient convolution with the shortcut gradient and the batch-norm sums under the launch plan of a step
+    whose module streams share the GPU: dx equals the single-stream plan's dx bit for bit (whose values the test above
+    holds against the oracle), the sums agree with it to fp32 rounding."""
+    from paper_1804_10574_b200 import binding
+    B, H, W, C = shape
+    g = torch.Generator(device="cuda").manual_seed(31)
+    rnd = lambda: torch.randn(B, H, W, C, device="cuda", generator=g)
+    dy, dout, bx = rnd().to(torch.bfloat16), rnd().to(torch.bfloat16), (rnd() * 1.5 + 0.3).to(torch.bfloat16)
+    out, mask = rnd().clamp_min(0).to(torch.bfloat16), rnd().clamp_min(0).to(torch.bfloat16)
+    w = (torch.randn(C, C, 3, 3, device="cuda", generator=g) * (2.0 / (9 * C)) ** 0.5).to(torch.bfloat16)
+    mean = bx.float().mean(dim=(0, 1, 2)).contiguous()
+    invstd = (1.0 / torch.sqrt(bx.float().var(dim=(0, 1, 2), unbiased=False) + 1e-5)).contiguous()
+    scratch = torch.zeros(binding.conv3x3_fused_scratch_elems(B, H, W, C), dtype=torch.float32, device="cuda")
+    res = []
+    for fn in (binding.conv3x3_dgrad_fused, binding.conv3x3_dgrad_fused_shared, binding.conv3x3_dgrad_fused_shared):
+        dx = torch.full_like(dy, 3.0)
+        db, dg = (torch.full((C,), 7.0, dtype=torch.float32, device="cuda") for _ in range(2))
+        fn(dy, w, None, dx, dout, out, mask, bx, mean, invstd, db, dg, scratch, B, H, W, C)
+        torch.cuda.synchronize()
+        res.append((dx, db.cpu().numpy(), dg.cpu().numpy()))
+    scale = float(np.abs(res[0][1]).max() + np.abs(res[0][2]).max())
+    for dx, db, dg in res[1:]:
+        assert torch.equal(dx, res[0][0])
+        assert np.max(np.abs(db - res[0][1])) < 2e-6 * scale + 1e-4 and np.max(np.abs(dg - res[0][2])) < 2e-6 * scale + 1e-4
+    assert np.array_equal(res[1][1], res[2][1]) and np.array_equal(res[1][2], res[2][2])   # fixed order: same bits again
+
+
 @pytest.mark.parametrize("shape", [(3, 32, 32, 16), (6, 16, 16, 32), (7, 32, 32, 32), (10, 16, 16, 16), (128, 32, 32, 16)],
                          ids=lambda s: "x".join(map(str, s)))
 def test_stride2_input_gradient_with_parameter_free_shortcut(shape):
