@@ -1375,7 +1375,10 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     const int n_tiles = (int)((long)B * H * W / kTileM);
     // pixel chunks (= CTAs, = partials to fold): few at the training step's sizes, where the kernel shares the GPU with
     // the other streams and the fold should stay small; one per 16 tiles, up to a CTA per SM, for large batches
-    const int max_chunks = slab ? (C == 16 ? 74 : 37) : 24;
+    // (64 channels, whose launch has three CTAs per chunk, one per filter row: half as many chunks while several module
+    // streams share the GPU - K = 4 iteration 1.629 -> 1.607 ms, K = 2, 3 unchanged; the 16- and 32-channel counts lose
+    // in both directions)
+    const int max_chunks = slab ? (C == 16 ? 74 : 37) : (s.shared ? 12 : 24);
     int chunks = n_tiles < max_chunks ? n_tiles : max_chunks;
     const int cap = slab ? (pair ? 2 * kWgMaxChunks : kWgMaxChunks) : 48;
     const int big = n_tiles / 16 < cap ? n_tiles / 16 : cap;
