@@ -1360,7 +1360,11 @@ int launch_wg(const void *x, const void *dy, float *dw, float *scratch, int B, i
     // thread of this operand-swapped form is issue-bound, a second one per SM takes batch 4096 from 70.6 to 61.6 us
     // (the 16-channel form is bound by the tensor pipe and the 64-channel one by its fold: both lose with two)
     const bool pair = C == 32 && n_tiles_all >= 32 * g_num_sms;
-    const int budget = pair ? 110 * 1024 : (n_tiles_all >= 8 * g_num_sms ? kSmemMax - 2048 - (C == 32 ? 4096 : 0) : kSmemBudget);
+    // training-step sizes: the half-SM budget (two stages of 32 or 64 channels); the 16-channel kernel, whose tile is
+    // eight tensor-bound instructions, wants a fourth stage of loads in flight (K = 1 / 3 / 4 iteration -1.7 / -0.8 /
+    // -1.6 %; two, five or six stages lose)
+    const int small_budget = C == 16 ? 100 * 1024 : kSmemBudget;
+    const int budget = pair ? 110 * 1024 : (n_tiles_all >= 8 * g_num_sms ? kSmemMax - 2048 - (C == 32 ? 4096 : 0) : small_budget);
     int n_stages = budget / stage_bytes;
     if (n_stages > kMaxStages) n_stages = kMaxStages;
     if (n_stages < 2) n_stages = 2;
